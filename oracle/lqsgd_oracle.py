@@ -1,0 +1,333 @@
+"""CPU oracle for one LQ-SGD compression round.  TEST INFRASTRUCTURE ONLY.
+
+A plain, slow, fp64 restatement of Algorithm 1 (iteration body, error feedback to
+error update) and of the quantiser of Eq. 4 / Eq. 5 of "Trustworthy Efficient
+Communication for Distributed Learning using LQ-SGD Algorithm".  It exists to
+check the CUDA library; the library never calls it, and it imports nothing
+from the library (numpy only).  Only tests, the smoke check and the CPU-baseline
+leg of the benchmark may execute it.
+
+Notation is the paper's Section IV: G in R^{n x m}, P in R^{n x r},
+Q in R^{m x r}, E the error buffer, M = G' = G + E, W workers.
+
+Every function states the passage it follows.  Where the paper is silent the
+reading taken is stated next to the code:
+
+* bits b = 1 sign bit + (b-1) magnitude bits, L = 2^(b-1) magnitude levels,
+  placed uniformly in the companded domain with both end points, |q|_k = k/(L-1);
+* nearest level in the companded domain, ties (exact half) away from zero;
+* one scale s per factor and layer, s = max over workers of max |x|, and the
+  division x/s is an fp32 division (the precision the library stores s and x
+  in), so that the integer decision is taken on the same number on both sides;
+* the worker average is the mean of the signed level indices (Alg. 1 applies
+  All-Reduce to the quantised factor, then dequantises once);
+* Orthonormalize = the thin-QR Q factor with positive-diagonal R, computed by
+  modified Gram-Schmidt; a column whose residual norm^2 is <= 1e-24 of its
+  original norm^2 (or that is exactly zero) becomes a zero column.
+
+Pins (tests/test_oracle_*.py): hand-worked level/threshold tables, brute-force
+nearest-level matching, closed-form inverse pair, LAPACK QR, truncated SVD,
+planted-rank recovery, error-feedback telescoping, payload closed forms.
+The value of alpha and the readings above have no printed worked example in
+the paper: against the authors' own code they are "parity unpinned".
+"""
+from __future__ import annotations
+
+import numpy as np
+
+RANK_EPS = 1e-24     # relative residual norm^2 below which a column counts as dependent
+
+
+# ----------------------------------------------------------------------------
+# Eq. 4 / Eq. 5: the compander pair
+# ----------------------------------------------------------------------------
+def compand(x, alpha):
+    """Eq. 4: q(x) = sign(x) * log(1 + alpha|x|) / log(1 + alpha)."""
+    x = np.asarray(x, dtype=np.float64)
+    return np.sign(x) * np.log1p(alpha * np.abs(x)) / np.log1p(alpha)
+
+
+def expand(q, alpha):
+    """Eq. 5: x = sign(q) * ((1 + alpha)^|q| - 1) / alpha."""
+    q = np.asarray(q, dtype=np.float64)
+    return np.sign(q) * np.expm1(np.abs(q) * np.log1p(alpha)) / alpha
+
+
+def magnitude_levels(bits):
+    """Number of magnitude levels L for a b-bit code with one sign bit."""
+    if not 2 <= bits <= 8:
+        raise ValueError("bits must be in 2..8")
+    return 1 << (bits - 1)
+
+
+def level_values(bits, alpha):
+    """x-domain magnitudes of the L levels: expand(k / (L-1)), k = 0..L-1."""
+    L = magnitude_levels(bits)
+    return expand(np.arange(L, dtype=np.float64) / (L - 1), alpha)
+
+
+# ----------------------------------------------------------------------------
+# LogQuantize / LogDequantize (Alg. 1, quantise and dequantise lines; Section IV-A)
+# ----------------------------------------------------------------------------
+def factor_scale(factors):
+    """s = max over workers and entries of |x| (fp32 values, exact)."""
+    s = np.float32(0.0)
+    for f in factors:
+        f32 = np.asarray(f, dtype=np.float32)
+        if f32.size:
+            s = max(s, np.float32(np.max(np.abs(f32))))
+    return np.float32(s)
+
+
+def log_quantize(x, s, bits, alpha, return_margin=False):
+    """b-bit code of every entry of x: (sign bit << (b-1)) | k.
+
+    k = nearest level index of compand(|x|/s) on the grid k/(L-1), half away
+    from zero.  x and s are taken as fp32 and |x|/s is an fp32 division.
+    With return_margin also returns, in level units, the distance of the
+    companded magnitude from the nearest decision threshold.
+    """
+    L = magnitude_levels(bits)
+    x32 = np.asarray(x, dtype=np.float32)
+    s32 = np.float32(s)
+    neg = x32 < 0
+    if s32 == 0:
+        v = np.zeros(x32.shape, dtype=np.float64)
+    else:
+        t = (np.abs(x32) / s32).astype(np.float32)          # fp32 division
+        v = (L - 1) * compand(t.astype(np.float64), alpha)  # in [0, L-1]
+    k = np.floor(v + 0.5)
+    k = np.clip(k, 0, L - 1).astype(np.uint8)
+    codes = (neg.astype(np.uint8) << (bits - 1)) | k
+    if return_margin:
+        return codes, np.abs(v - (np.floor(v) + 0.5))
+    return codes
+
+
+def signed_levels(codes, bits):
+    """Signed level index (-1)^sign * k of each code, as int64."""
+    codes = np.asarray(codes).astype(np.int64)
+    k = codes & ((1 << (bits - 1)) - 1)
+    neg = (codes >> (bits - 1)) & 1
+    return np.where(neg == 1, -k, k)
+
+
+def average_dequantize(codes_per_worker, s, bits, alpha):
+    """All-Reduce (mean, Eq. 1) of the signed quantised values, then Eq. 5 once.
+
+    q_bar = sum_w (+-k_w) / (W (L-1));  result = s * expand(q_bar).
+    """
+    L = magnitude_levels(bits)
+    W = len(codes_per_worker)
+    S = np.zeros(np.asarray(codes_per_worker[0]).shape, dtype=np.int64)
+    for c in codes_per_worker:
+        S += signed_levels(c, bits)
+    q_bar = S.astype(np.float64) / (W * (L - 1))
+    return np.float64(np.float32(s)) * expand(q_bar, alpha)
+
+
+def pack_codes(codes, bits):
+    """Little-endian bit stream: element i (row-major) occupies bits [i*b, (i+1)*b)."""
+    flat = np.asarray(codes, dtype=np.uint8).reshape(-1)
+    nbytes = (flat.size * bits + 7) // 8
+    out = np.zeros(nbytes, dtype=np.uint8)
+    for j in range(bits):                       # bit j of every code
+        pos = np.arange(flat.size, dtype=np.int64) * bits + j
+        bit = (flat >> j) & 1
+        np.bitwise_or.at(out, pos >> 3, (bit << (pos & 7)).astype(np.uint8))
+    return out
+
+
+def unpack_codes(stream, count, bits):
+    """Inverse of pack_codes for `count` elements."""
+    stream = np.asarray(stream, dtype=np.uint8)
+    codes = np.zeros(count, dtype=np.uint8)
+    for j in range(bits):
+        pos = np.arange(count, dtype=np.int64) * bits + j
+        bit = (stream[pos >> 3] >> (pos & 7)) & 1
+        codes |= (bit << j).astype(np.uint8)
+    return codes
+
+
+# ----------------------------------------------------------------------------
+# Orthonormalize (Alg. 1, orthonormalisation line)
+# ----------------------------------------------------------------------------
+def orthonormalize(P):
+    """Modified Gram-Schmidt, columns left to right.  Returns (P_orth, dependent_mask)."""
+    A = np.array(P, dtype=np.float64, copy=True)
+    r = A.shape[1]
+    dependent = np.zeros(r, dtype=bool)
+    for j in range(r):
+        norm0 = float(A[:, j] @ A[:, j])
+        for i in range(j):
+            A[:, j] -= (A[:, i] @ A[:, j]) * A[:, i]
+        norm1 = float(A[:, j] @ A[:, j])
+        if norm0 == 0.0 or norm1 <= RANK_EPS * norm0:
+            A[:, j] = 0.0
+            dependent[j] = True
+        else:
+            A[:, j] /= np.sqrt(norm1)
+    return A, dependent
+
+
+# ----------------------------------------------------------------------------
+# One factor exchange: scale, quantise, All-Reduce, dequantise
+# ----------------------------------------------------------------------------
+def exchange_factor(factors, bits, alpha, forced_codes=None):
+    """Quantise every worker's factor, average, dequantise (Alg. 1, the three lines
+    after each product).  bits == 32 bypasses the quantiser (plain PowerSGD mean).
+
+    forced_codes: optional list (per worker) of int16 arrays; entries >= 0 replace
+    the code computed here (used by parity tests for near-threshold elements).
+    Returns dict(scale, codes[list], margin[list], mean) with mean in fp64.
+    """
+    W = len(factors)
+    if bits == 32:
+        mean = sum(np.asarray(f, dtype=np.float64) for f in factors) / W
+        return dict(scale=np.float32(0), codes=None, margin=None, mean=mean)
+    s = factor_scale(factors)
+    codes, margins = [], []
+    for w, f in enumerate(factors):
+        c, mg = log_quantize(f, s, bits, alpha, return_margin=True)
+        if forced_codes is not None and forced_codes[w] is not None:
+            fc = np.asarray(forced_codes[w]).reshape(c.shape)
+            c = np.where(fc >= 0, fc, c).astype(np.uint8)
+        codes.append(c)
+        margins.append(mg)
+    mean = average_dequantize(codes, s, bits, alpha)
+    return dict(scale=s, codes=codes, margin=margins, mean=mean)
+
+
+# ----------------------------------------------------------------------------
+# The stages of one round for one layer (Algorithm 1, loop body)
+# ----------------------------------------------------------------------------
+def error_feedback(G, E):
+    """M = G' = G + E (Eq. 8)."""
+    return np.asarray(G, dtype=np.float64) + np.asarray(E, dtype=np.float64)
+
+
+def power_step_p(M, Q):
+    """P = M Q."""
+    return np.asarray(M, dtype=np.float64) @ np.asarray(Q, dtype=np.float64)
+
+
+def power_step_q(M, P_bar):
+    """Q = M^T P_bar, with the dequantised, averaged P."""
+    return np.asarray(M, dtype=np.float64).T @ np.asarray(P_bar, dtype=np.float64)
+
+
+def reconstruct(P_bar, Q_bar):
+    """G_hat = P Q^T (Eq. 6)."""
+    return np.asarray(P_bar, dtype=np.float64) @ np.asarray(Q_bar, dtype=np.float64).T
+
+
+def error_update(M, G_hat):
+    """E = G' - G_hat (Eq. 7)."""
+    return np.asarray(M, dtype=np.float64) - G_hat
+
+
+def effective_rank(rank, n, m):
+    return min(rank, n, m)
+
+
+def layer_round(G, E, Q, bits_p, bits_q, alpha, forced_p=None, forced_q=None):
+    """One iteration of Algorithm 1 for one n x m layer and W workers.
+
+    G, E: arrays [W, n, m];  Q: [m, r] shared by all workers (warm start).
+    Returns a dict with every intermediate:
+      M [W,n,m], P_raw [W,n,r], P [W,n,r] (orthonormal), dependent [W,r],
+      xp (exchange_factor result for P), P_bar [n,r], Qw [W,m,r], xq, Q_bar [m,r],
+      G_hat [n,m], E_new [W,n,m].
+    """
+    G = np.asarray(G)
+    W = G.shape[0]
+    M = [error_feedback(G[w], E[w]) for w in range(W)]
+    P_raw = [power_step_p(M[w], Q) for w in range(W)]
+    orth = [orthonormalize(P_raw[w]) for w in range(W)]
+    P = [o[0] for o in orth]
+    xp = exchange_factor(P, bits_p, alpha, forced_p)
+    P_bar = xp["mean"]
+    Qw = [power_step_q(M[w], P_bar) for w in range(W)]
+    xq = exchange_factor(Qw, bits_q, alpha, forced_q)
+    Q_bar = xq["mean"]
+    G_hat = reconstruct(P_bar, Q_bar)
+    E_new = [error_update(M[w], G_hat) for w in range(W)]
+    return dict(M=np.stack(M), P_raw=np.stack(P_raw), P=np.stack(P),
+                dependent=np.stack([o[1] for o in orth]), xp=xp, P_bar=P_bar,
+                Qw=np.stack(Qw), xq=xq, Q_bar=Q_bar, G_hat=G_hat, E_new=np.stack(E_new))
+
+
+def vector_mean(V):
+    """Eq. 1 for a tensor that bypasses compression: mean over workers, V is [W, len]."""
+    return np.mean(np.asarray(V, dtype=np.float64), axis=0)
+
+
+# ----------------------------------------------------------------------------
+# Communication cost (Section IV-C) and the payload the library documents
+# ----------------------------------------------------------------------------
+def factor_bits(n, m, rank, bits):
+    """r (n + m) b bits per layer and iteration."""
+    r = effective_rank(rank, n, m)
+    return r * (n + m) * bits
+
+
+def payload_bytes(layers, rank, bits_p, bits_q):
+    """Bytes one worker sends per round: for each matrix the two code streams, each
+    padded to a whole byte, plus the two fp32 scales; fp32 for every 1-D tensor."""
+    total = 0
+    for n, m in layers:
+        if n > 1 and m > 1:
+            r = effective_rank(rank, n, m)
+            total += (r * n * bits_p + 7) // 8 + (r * m * bits_q + 7) // 8 + 8
+        else:
+            total += 4 * n * m
+    return total
+
+
+def assemble_payload(layers, rank, bits_p, bits_q, scales, codes_p, codes_q, vectors):
+    """One worker's payload in the library's documented order:
+    [s_P, s_Q of every matrix][every 1-D tensor, fp32][P codes of every matrix][Q codes ...].
+    scales: list of (s_P, s_Q); codes_*: per matrix uint8 code arrays; vectors: per 1-D tensor."""
+    parts = [np.asarray([v for pair in scales for v in pair], dtype="<f4").view(np.uint8)]
+    parts += [np.asarray(v, dtype="<f4").reshape(-1).view(np.uint8) for v in vectors]
+    parts += [pack_codes(c, bits_p) for c in codes_p]
+    parts += [pack_codes(c, bits_q) for c in codes_q]
+    return np.concatenate(parts) if parts else np.zeros(0, np.uint8)
+
+
+# ----------------------------------------------------------------------------
+# Multi-layer, multi-step driver with the persistent state (E per worker, shared Q)
+# ----------------------------------------------------------------------------
+class Oracle:
+    """State machine of Algorithm 1 over a list of layers: E_0 = 0, Q_0 supplied by the
+    caller (drawn N(0,1) outside), Q_t = dequantised averaged Q of step t-1."""
+
+    def __init__(self, layers, rank, bits_p, bits_q, alpha, workers, Q0):
+        self.layers = [tuple(s) for s in layers]
+        self.rank, self.bits_p, self.bits_q = rank, bits_p, bits_q
+        self.alpha, self.W = float(alpha), workers
+        self.E, self.Q = {}, {}
+        for li, (n, m) in enumerate(self.layers):
+            if n > 1 and m > 1:
+                r = effective_rank(rank, n, m)
+                self.E[li] = np.zeros((workers, n, m), dtype=np.float64)
+                q0 = np.asarray(Q0[li], dtype=np.float64)
+                assert q0.shape == (m, r), (q0.shape, (m, r))
+                self.Q[li] = q0.copy()
+
+    def step(self, grads, forced=None):
+        """grads[w][layer] -> list over layers of layer_round dicts (or dict(mean=...) for 1-D)."""
+        out = []
+        for li, (n, m) in enumerate(self.layers):
+            Gl = np.stack([np.asarray(grads[w][li], dtype=np.float32).reshape(n, m)
+                           for w in range(self.W)])
+            if li in self.E:
+                f = (forced or {}).get(li, (None, None))
+                res = layer_round(Gl, self.E[li], self.Q[li], self.bits_p, self.bits_q,
+                                  self.alpha, f[0], f[1])
+                self.E[li] = res["E_new"]
+                self.Q[li] = res["Q_bar"]
+            else:
+                res = dict(mean=vector_mean(Gl.reshape(self.W, -1)))
+            out.append(res)
+        return out
