@@ -1,0 +1,196 @@
+/*
+ * lqsgd.h - C ABI of the LQ-SGD compression round for NVIDIA B200 (sm_100a).
+ *
+ * One call of lqsgd_step() runs the body of Algorithm 1 of "Trustworthy Efficient
+ * Communication for Distributed Learning using LQ-SGD Algorithm" for a whole set of layer
+ * gradients and W data-parallel workers whose gradients all live on one GPU:
+ *
+ *   M_w   = G_w + E_w                          error feedback        (Eq. 8)
+ *   P_w   = Orthonormalize(M_w Q)              power step            (Alg. 1)
+ *   P_bar = LogDequantize(mean_w LogQuantize(P_w, b_p, alpha))       (Eq. 4, Eq. 5, Eq. 1)
+ *   Q_w   = M_w^T P_bar                        second power step     (Alg. 1)
+ *   Q_bar = LogDequantize(mean_w LogQuantize(Q_w, b_q, alpha))
+ *   G_hat = P_bar Q_bar^T                      reconstruction        (Eq. 6)
+ *   E_w   = M_w - G_hat                        error update          (Eq. 7)
+ *   Q     = Q_bar                              warm start of the next call
+ *
+ * Notation (Section IV): a layer gradient G is n x m, row-major, n = rows (C_out) and
+ * m = cols (C_in*k*k); P is n x r, Q is m x r; r_eff = min(rank, n, m) columns are used.
+ * A tensor with rows == 1 or cols == 1 is one-dimensional: it bypasses the low-rank path
+ * and is averaged over the workers in fp32 (Eq. 1).
+ *
+ * Quantiser.  A b-bit code is one sign bit (the top bit of the code, set iff x < 0) and
+ * b-1 magnitude bits holding the level index k in 0..L-1, L = 2^(b-1).  Levels are uniform
+ * in the companded domain of Eq. 4, |q|_k = k/(L-1); k is the level nearest to
+ * q(|x|/s), an exact half rounding up.  s is one fp32 scale per factor and layer, the largest
+ * |x| over all workers; |x|/s is an IEEE fp32 division.  The worker average is the exact
+ * integer sum S of the signed level indices divided by W(L-1), to which Eq. 5 is applied once.
+ *
+ * Memory.  The library allocates no device memory: the caller passes one workspace whose size
+ * lqsgd_workspace_bytes() reports and keeps it alive, untouched, until lqsgd_destroy().  The
+ * error buffers E_w and the warm-start Q live in that workspace and persist across steps.
+ * All pointers named "dev_*" (and the entries of grads / ghat) are device pointers on the
+ * device that was current at lqsgd_create(); pointers named "host_*" are host pointers.
+ *
+ * Errors.  Every function returns LQSGD_OK (0) or a negative lqsgd_error; nothing throws,
+ * aborts or traps.  Argument errors are detected on the host before anything is launched.
+ * Numerical conditions met on the device (a dependent column, a zero scale, a non-finite
+ * value) never fault: they produce the defined result below and set a bit in the per-layer
+ * status word (lqsgd_status).
+ *
+ * Threading.  A context may be used from one host thread at a time.  lqsgd_step() is
+ * asynchronous on the given stream; steps issued on different streams must be ordered by the
+ * caller.
+ */
+#ifndef LQSGD_H_
+#define LQSGD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define LQSGD_VERSION 1
+
+typedef enum lqsgd_error {
+  LQSGD_OK = 0,
+  LQSGD_ERR_INVALID_ARG = -1,         /* null pointer, bad struct_size, rank/bits/alpha/workers out of range */
+  LQSGD_ERR_BAD_SHAPE = -2,           /* rows or cols < 1, or too large */
+  LQSGD_ERR_WORKSPACE_TOO_SMALL = -3,
+  LQSGD_ERR_MISALIGNED = -4,          /* workspace not 256-byte aligned, tensor pointer not aligned */
+  LQSGD_ERR_CUDA = -5,                /* a CUDA runtime call failed; see lqsgd_last_cuda_error() */
+  LQSGD_ERR_NO_STAGING = -6,          /* lqsgd_step_host() on a context created without LQSGD_FLAG_HOST_STAGING */
+  LQSGD_ERR_OUT_OF_RANGE = -7         /* layer / worker / state index out of range, or state not defined for that layer */
+} lqsgd_error;
+
+/* Bits of the per-layer status word. */
+#define LQSGD_STATUS_DEPENDENT_COLUMN 1u /* a column of M Q was zero or linearly dependent: it became a zero column */
+#define LQSGD_STATUS_ZERO_SCALE_P     2u /* every P entry was 0: codes and P_bar are 0 */
+#define LQSGD_STATUS_ZERO_SCALE_Q     4u /* every Q entry was 0: codes and Q_bar are 0 */
+#define LQSGD_STATUS_NONFINITE        8u /* a scale was inf or nan: the layer's outputs are undefined (no fault) */
+
+/* Config flags. */
+#define LQSGD_FLAG_HOST_STAGING 1u /* reserve device staging in the workspace so that lqsgd_step_host() works */
+
+typedef struct lqsgd_ctx lqsgd_ctx;
+
+typedef struct lqsgd_shape {
+  int32_t rows; /* n */
+  int32_t cols; /* m */
+} lqsgd_shape;
+
+/* Inputs of Algorithm 1 (rank r, bits b_p and b_q, curvature alpha) plus the worker count. */
+typedef struct lqsgd_config {
+  uint32_t struct_size; /* sizeof(lqsgd_config), for versioning */
+  int32_t rank;         /* r, 1..16 (any integer) */
+  int32_t bits_p;       /* b_p, total bits per P scalar including the sign, 2..8 */
+  int32_t bits_q;       /* b_q, likewise for Q */
+  float alpha;          /* alpha of Eq. 4 / Eq. 5, finite and > 0 */
+  int32_t workers;      /* W, 1..256 */
+  uint64_t seed;        /* seed of Q_0 ~ N(0,1) (Alg. 1 initialisation) */
+  uint32_t flags;       /* LQSGD_FLAG_* */
+} lqsgd_config;
+
+/* Where one layer's data sits inside a worker's payload (byte offsets from the payload start). */
+typedef struct lqsgd_layer_layout {
+  int32_t is_matrix;     /* 1: low-rank path, 0: one-dimensional tensor sent as fp32 */
+  int32_t rank_eff;      /* r_eff (0 for a 1-D tensor) */
+  uint64_t scale_offset; /* matrix: fp32 s_P then fp32 s_Q */
+  uint64_t p_offset;     /* matrix: P code stream, p_bytes = ceil(n * r_eff * b_p / 8) */
+  uint64_t p_bytes;
+  uint64_t q_offset;     /* matrix: Q code stream, q_bytes = ceil(m * r_eff * b_q / 8) */
+  uint64_t q_bytes;
+  uint64_t vec_offset;   /* 1-D tensor: rows*cols fp32 values */
+  uint64_t vec_bytes;
+} lqsgd_layer_layout;
+
+/* State that lqsgd_get_state / lqsgd_set_state can copy.  Shapes are dense (no padding),
+ * row-major.  "per worker" states take a worker index, the others ignore it. */
+typedef enum lqsgd_state {
+  LQSGD_STATE_E = 0,       /* fp32 n x m, per worker: error buffer (Eq. 7); settable */
+  LQSGD_STATE_Q = 1,       /* fp32 m x r_eff: warm-start Q (Q_0, then Q_bar of the last step); settable */
+  LQSGD_STATE_P_RAW = 2,   /* fp32 n x r_eff, per worker: M Q of the last step, before Orthonormalize */
+  LQSGD_STATE_P = 3,       /* fp32 n x r_eff, per worker: orthonormal P of the last step */
+  LQSGD_STATE_P_BAR = 4,   /* fp32 n x r_eff: dequantised worker average of P */
+  LQSGD_STATE_Q_W = 5,     /* fp32 m x r_eff, per worker: M^T P_bar of the last step */
+  LQSGD_STATE_CODES_P = 6, /* uint8 n x r_eff, per worker: one unpacked code per byte */
+  LQSGD_STATE_CODES_Q = 7, /* uint8 m x r_eff, per worker */
+  LQSGD_STATE_SCALES = 8   /* fp32 [2]: s_P, s_Q of the last step */
+} lqsgd_state;
+
+/* Bytes of device workspace a context for these layers needs (Algorithm 1 state E, Q, plus
+ * factors, partial sums, codes, payload and tables).  Host-only; launches nothing. */
+int lqsgd_workspace_bytes(const lqsgd_shape* host_shapes, int32_t n_layers,
+                          const lqsgd_config* host_config, size_t* host_bytes_out);
+
+/* Creates a context on the current device.  dev_workspace: caller-owned device memory,
+ * 256-byte aligned, at least lqsgd_workspace_bytes() long; the library carves it and owns its
+ * contents until lqsgd_destroy().  Initialises E_0 = 0 and Q_0 ~ N(0,1) from config->seed
+ * (Alg. 1 initialisation; the same Q_0 for every worker) and uploads the planning tables:
+ * it issues copies and a memset on the legacy default stream and synchronises it.
+ * The context itself is host memory owned by the library. */
+int lqsgd_create(const lqsgd_shape* host_shapes, int32_t n_layers, const lqsgd_config* host_config,
+                 void* dev_workspace, size_t workspace_bytes, lqsgd_ctx** ctx_out);
+
+/* One round of Algorithm 1 (error feedback to error update) for every layer.
+ * host_grads: host array of W * n_layers device pointers, worker-major
+ *   (host_grads[w * n_layers + l] = G of layer l on worker w), fp32 row-major contiguous,
+ *   read-only; a matrix whose cols is a multiple of 4 must be 16-byte aligned.
+ * host_ghat: host array of n_layers device pointers; host_ghat[l] receives G_hat of layer l
+ *   (or the worker mean of a 1-D tensor), same shape as the gradient; overwritten.
+ *   Must not alias any gradient.
+ * cuda_stream: a cudaStream_t (NULL = legacy default stream).  The call only enqueues work;
+ *   results, payload and state are valid once the stream has reached the end of that work.
+ *   The pointer arrays themselves are consumed before the call returns. */
+int lqsgd_step(lqsgd_ctx* ctx, const float* const* host_grads, float* const* host_ghat,
+               void* cuda_stream);
+
+/* Same round with HOST tensors: copies every gradient host->device into the staging area,
+ * runs lqsgd_step, copies every G_hat and all W payloads device->host, and synchronises the
+ * stream before returning.  host_grads / host_ghat are arrays of host pointers laid out as in
+ * lqsgd_step (pinned memory makes the copies asynchronous to each other, pageable works);
+ * host_payload (may be NULL) receives W * payload_bytes bytes, worker after worker.
+ * Needs LQSGD_FLAG_HOST_STAGING. */
+int lqsgd_step_host(lqsgd_ctx* ctx, const float* const* host_grads, float* const* host_ghat,
+                    void* host_payload, void* cuda_stream);
+
+/* Size of one worker's payload in bytes (Section IV-C: r(n+m)b bits per matrix, each code
+ * stream padded to a byte, + 8 bytes of scales per matrix + 4 bytes per 1-D scalar). */
+int lqsgd_payload_bytes(const lqsgd_ctx* ctx, size_t* host_bytes_out);
+
+/* Device view of what worker `worker` sends in the last enqueued step: valid until the next
+ * step.  Order: [s_P, s_Q of every matrix][every 1-D tensor, fp32][P code streams][Q code
+ * streams], each in layer order; a code stream is a little-endian bit stream in which element
+ * i of the row-major n x r_eff (or m x r_eff) factor occupies bits [i*b, (i+1)*b). */
+int lqsgd_payload(const lqsgd_ctx* ctx, int32_t worker, const void** dev_ptr_out, size_t* host_bytes_out);
+
+int lqsgd_payload_layout(const lqsgd_ctx* ctx, int32_t layer, lqsgd_layer_layout* host_out);
+
+/* Copies one piece of state to / from caller device memory (dense, row-major; see lqsgd_state),
+ * asynchronously on cuda_stream.  Setting E or Q is how a checkpoint is restored. */
+int lqsgd_get_state(const lqsgd_ctx* ctx, int32_t which, int32_t layer, int32_t worker,
+                    void* dev_dst, void* cuda_stream);
+int lqsgd_set_state(lqsgd_ctx* ctx, int32_t which, int32_t layer, int32_t worker,
+                    const void* dev_src, void* cuda_stream);
+
+/* Copies the per-layer status words of the last step into host_flags[n_layers];
+ * synchronises cuda_stream. */
+int lqsgd_status(const lqsgd_ctx* ctx, uint32_t* host_flags, void* cuda_stream);
+
+/* Kernel launches one lqsgd_step enqueues (for launch accounting). */
+int lqsgd_launches_per_step(const lqsgd_ctx* ctx, int32_t* host_out);
+
+/* Frees the host-side context.  The workspace stays the caller's. */
+void lqsgd_destroy(lqsgd_ctx* ctx);
+
+const char* lqsgd_strerror(int code);
+/* Text of the last CUDA error this library saw on the calling thread ("" if none). */
+const char* lqsgd_last_cuda_error(void);
+int lqsgd_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LQSGD_H_ */

@@ -1,0 +1,241 @@
+"""ctypes binding of liblqsgd.so (the C ABI declared in include/lqsgd.h).
+
+Argument marshalling only: every step of the LQ-SGD round runs in the library's CUDA kernels.
+PyTorch appears here as the owner of device memory (the workspace, gradients, outputs) and of
+the CUDA stream.  There is no CPU fallback: if the shared library is missing or a call fails,
+an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liblqsgd.so")
+
+# lqsgd_state
+STATE_E, STATE_Q, STATE_P_RAW, STATE_P, STATE_P_BAR, STATE_Q_W, STATE_CODES_P, STATE_CODES_Q, STATE_SCALES = range(9)
+STATUS_DEPENDENT_COLUMN, STATUS_ZERO_SCALE_P, STATUS_ZERO_SCALE_Q, STATUS_NONFINITE = 1, 2, 4, 8
+FLAG_HOST_STAGING = 1
+
+ERR_INVALID_ARG, ERR_BAD_SHAPE, ERR_WORKSPACE_TOO_SMALL, ERR_MISALIGNED = -1, -2, -3, -4
+ERR_CUDA, ERR_NO_STAGING, ERR_OUT_OF_RANGE = -5, -6, -7
+
+EXPORTED = [
+    "lqsgd_workspace_bytes", "lqsgd_create", "lqsgd_step", "lqsgd_step_host", "lqsgd_payload_bytes",
+    "lqsgd_payload", "lqsgd_payload_layout", "lqsgd_get_state", "lqsgd_set_state", "lqsgd_status",
+    "lqsgd_launches_per_step", "lqsgd_destroy", "lqsgd_strerror", "lqsgd_last_cuda_error", "lqsgd_version",
+]
+
+
+class Shape(C.Structure):
+    _fields_ = [("rows", C.c_int32), ("cols", C.c_int32)]
+
+
+class Config(C.Structure):
+    _fields_ = [("struct_size", C.c_uint32), ("rank", C.c_int32), ("bits_p", C.c_int32),
+                ("bits_q", C.c_int32), ("alpha", C.c_float), ("workers", C.c_int32),
+                ("seed", C.c_uint64), ("flags", C.c_uint32)]
+
+
+class LayerLayout(C.Structure):
+    _fields_ = [("is_matrix", C.c_int32), ("rank_eff", C.c_int32), ("scale_offset", C.c_uint64),
+                ("p_offset", C.c_uint64), ("p_bytes", C.c_uint64), ("q_offset", C.c_uint64),
+                ("q_bytes", C.c_uint64), ("vec_offset", C.c_uint64), ("vec_bytes", C.c_uint64)]
+
+
+class LqsgdError(RuntimeError):
+    def __init__(self, code: int, text: str):
+        super().__init__(f"lqsgd error {code}: {text}")
+        self.code = code
+
+
+_lib = None
+
+
+def load_library() -> C.CDLL:
+    """Loads liblqsgd.so (built in-tree by __graft_entry__.build()); raises if it is absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise FileNotFoundError(f"{LIB_PATH} not found: build the CUDA library first (no CPU fallback exists)")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, sz = C.c_void_p, C.c_int32, C.c_size_t
+    lib.lqsgd_workspace_bytes.argtypes = [C.POINTER(Shape), i32, C.POINTER(Config), C.POINTER(sz)]
+    lib.lqsgd_create.argtypes = [C.POINTER(Shape), i32, C.POINTER(Config), vp, sz, C.POINTER(vp)]
+    lib.lqsgd_step.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), vp]
+    lib.lqsgd_step_host.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), vp, vp]
+    lib.lqsgd_payload_bytes.argtypes = [vp, C.POINTER(sz)]
+    lib.lqsgd_payload.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(sz)]
+    lib.lqsgd_payload_layout.argtypes = [vp, i32, C.POINTER(LayerLayout)]
+    lib.lqsgd_get_state.argtypes = [vp, i32, i32, i32, vp, vp]
+    lib.lqsgd_set_state.argtypes = [vp, i32, i32, i32, vp, vp]
+    lib.lqsgd_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
+    lib.lqsgd_launches_per_step.argtypes = [vp, C.POINTER(i32)]
+    lib.lqsgd_destroy.argtypes = [vp]
+    lib.lqsgd_destroy.restype = None
+    lib.lqsgd_strerror.argtypes = [C.c_int]
+    lib.lqsgd_strerror.restype = C.c_char_p
+    lib.lqsgd_last_cuda_error.restype = C.c_char_p
+    lib.lqsgd_version.restype = C.c_int
+    _lib = lib
+    return lib
+
+
+def _check(rc: int) -> None:
+    if rc != 0:
+        lib = load_library()
+        text = lib.lqsgd_strerror(rc).decode()
+        if rc == ERR_CUDA:
+            text += " (" + lib.lqsgd_last_cuda_error().decode() + ")"
+        raise LqsgdError(rc, text)
+
+
+def _shapes(layers: Sequence[Tuple[int, int]]):
+    arr = (Shape * len(layers))()
+    for i, (n, m) in enumerate(layers):
+        arr[i].rows, arr[i].cols = int(n), int(m)
+    return arr
+
+
+def make_config(rank: int, bits_p: int, bits_q: int, alpha: float, workers: int, seed: int = 0,
+                flags: int = 0) -> Config:
+    return Config(C.sizeof(Config), rank, bits_p, bits_q, alpha, workers, seed, flags)
+
+
+def workspace_bytes(layers, cfg: Config) -> int:
+    out = C.c_size_t(0)
+    _check(load_library().lqsgd_workspace_bytes(_shapes(layers), len(layers), C.byref(cfg), C.byref(out)))
+    return out.value
+
+
+class LQSGD:
+    """One LQ-SGD compressor (Algorithm 1 state for a list of layers and W workers) on a CUDA device."""
+
+    def __init__(self, layers: Sequence[Tuple[int, int]], rank: int, bits_p: int, bits_q: Optional[int] = None,
+                 alpha: float = 127.0, workers: int = 1, seed: int = 0, host_staging: bool = False,
+                 device: str = "cuda:0"):
+        self.lib = load_library()
+        self.layers = [(int(n), int(m)) for n, m in layers]
+        self.rank, self.bits_p = rank, bits_p
+        self.bits_q = bits_p if bits_q is None else bits_q
+        self.alpha, self.W = float(alpha), workers
+        self.device = torch.device(device)
+        self.cfg = make_config(rank, self.bits_p, self.bits_q, alpha, workers, seed,
+                               FLAG_HOST_STAGING if host_staging else 0)
+        nbytes = workspace_bytes(self.layers, self.cfg)
+        with torch.cuda.device(self.device):
+            self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+            base = self.workspace.data_ptr()
+            self._ws_ptr = (base + 255) // 256 * 256
+            ctx = C.c_void_p()
+            _check(self.lib.lqsgd_create(_shapes(self.layers), len(self.layers), C.byref(self.cfg),
+                                         C.c_void_p(self._ws_ptr), nbytes, C.byref(ctx)))
+        self.ctx = ctx
+        self.workspace_nbytes = nbytes
+        out = C.c_size_t(0)
+        _check(self.lib.lqsgd_payload_bytes(self.ctx, C.byref(out)))
+        self.payload_nbytes = out.value
+        n = C.c_int32(0)
+        _check(self.lib.lqsgd_launches_per_step(self.ctx, C.byref(n)))
+        self.launches_per_step = n.value
+        self._keep = None
+
+    # -- lifetime
+    def close(self):
+        if getattr(self, "ctx", None):
+            self.lib.lqsgd_destroy(self.ctx)
+            self.ctx = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def r_eff(self, layer: int) -> int:
+        n, m = self.layers[layer]
+        return min(self.rank, n, m)
+
+    def is_matrix(self, layer: int) -> bool:
+        n, m = self.layers[layer]
+        return n > 1 and m > 1
+
+    # -- the round
+    def make_pointer_arrays(self, grads: Sequence[Sequence[torch.Tensor]], ghat: Sequence[torch.Tensor]):
+        """ctypes pointer arrays for step(): grads[w][l] worker-major, ghat[l]."""
+        nl = len(self.layers)
+        g = (C.c_void_p * (self.W * nl))()
+        for w in range(self.W):
+            for l in range(nl):
+                g[w * nl + l] = grads[w][l].data_ptr()
+        h = (C.c_void_p * nl)()
+        for l in range(nl):
+            h[l] = ghat[l].data_ptr()
+        return g, h
+
+    def step_ptrs(self, g_arr, h_arr, stream: Optional[torch.cuda.Stream] = None) -> None:
+        s = stream if stream is not None else torch.cuda.current_stream(self.device)
+        _check(self.lib.lqsgd_step(self.ctx, g_arr, h_arr, C.c_void_p(s.cuda_stream)))
+
+    def step(self, grads, ghat, stream: Optional[torch.cuda.Stream] = None) -> None:
+        """One round of Algorithm 1 on device tensors grads[w][l]; writes ghat[l]."""
+        g, h = self.make_pointer_arrays(grads, ghat)
+        self.step_ptrs(g, h, stream)
+
+    def step_host(self, grads, ghat, payload: Optional[torch.Tensor] = None,
+                  stream: Optional[torch.cuda.Stream] = None) -> None:
+        """Same round on HOST tensors (copies in, runs, copies G_hat and payloads out, synchronises)."""
+        g, h = self.make_pointer_arrays(grads, ghat)
+        s = stream if stream is not None else torch.cuda.current_stream(self.device)
+        pp = C.c_void_p(payload.data_ptr()) if payload is not None else C.c_void_p(0)
+        _check(self.lib.lqsgd_step_host(self.ctx, g, h, pp, C.c_void_p(s.cuda_stream)))
+
+    # -- results and state
+    def _stream_ptr(self):
+        return C.c_void_p(torch.cuda.current_stream(self.device).cuda_stream)
+
+    def payload(self, worker: int) -> torch.Tensor:
+        """Copy of worker's payload bytes (uint8 device tensor)."""
+        ptr, nb = C.c_void_p(), C.c_size_t(0)
+        _check(self.lib.lqsgd_payload(self.ctx, worker, C.byref(ptr), C.byref(nb)))
+        off = ptr.value - self.workspace.data_ptr()
+        return self.workspace[off:off + nb.value].clone()
+
+    def payload_layout(self, layer: int) -> LayerLayout:
+        out = LayerLayout()
+        _check(self.lib.lqsgd_payload_layout(self.ctx, layer, C.byref(out)))
+        return out
+
+    def _state_shape(self, which: int, layer: int):
+        if not 0 <= layer < len(self.layers) or which not in range(9):
+            return (1,), torch.float32          # the library reports the bad index
+        n, m = self.layers[layer]
+        r = self.r_eff(layer)
+        return {STATE_E: ((n, m), torch.float32), STATE_Q: ((m, r), torch.float32),
+                STATE_P_RAW: ((n, r), torch.float32), STATE_P: ((n, r), torch.float32),
+                STATE_P_BAR: ((n, r), torch.float32), STATE_Q_W: ((m, r), torch.float32),
+                STATE_CODES_P: ((n, r), torch.uint8), STATE_CODES_Q: ((m, r), torch.uint8),
+                STATE_SCALES: ((2,), torch.float32)}[which]
+
+    def get_state(self, which: int, layer: int, worker: int = 0) -> torch.Tensor:
+        shape, dt = self._state_shape(which, layer)
+        out = torch.empty(shape, dtype=dt, device=self.device)
+        _check(self.lib.lqsgd_get_state(self.ctx, which, layer, worker, C.c_void_p(out.data_ptr()), self._stream_ptr()))
+        return out
+
+    def set_state(self, which: int, layer: int, worker: int, value: torch.Tensor) -> None:
+        shape, dt = self._state_shape(which, layer)
+        v = value.to(device=self.device, dtype=dt).contiguous()
+        assert tuple(v.shape) == tuple(shape), (v.shape, shape)
+        _check(self.lib.lqsgd_set_state(self.ctx, which, layer, worker, C.c_void_p(v.data_ptr()), self._stream_ptr()))
+        torch.cuda.current_stream(self.device).synchronize()      # v may be a temporary
+
+    def status(self) -> List[int]:
+        flags = (C.c_uint32 * len(self.layers))()
+        _check(self.lib.lqsgd_status(self.ctx, flags, self._stream_ptr()))
+        return list(flags)

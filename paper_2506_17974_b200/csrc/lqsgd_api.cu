@@ -1,0 +1,623 @@
+// Host side of the LQ-SGD library: argument checking, workspace carving, the tile planner,
+// table upload and the per-step launch sequence behind the C ABI of include/lqsgd.h.
+#include "../../include/lqsgd.h"
+#include "lqsgd_dev.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+using namespace lqsgd;
+
+namespace {
+
+thread_local std::string g_cuda_error;
+
+int cuda_fail(cudaError_t e, const char* what) {
+  g_cuda_error = std::string(what) + ": " + cudaGetErrorString(e);
+  return LQSGD_ERR_CUDA;
+}
+#define CK(call)                                              \
+  do {                                                        \
+    cudaError_t e__ = (call);                                 \
+    if (e__ != cudaSuccess) return cuda_fail(e__, #call);     \
+  } while (0)
+
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Hands out 256-byte aligned pieces of the workspace; with base == nullptr it only counts.
+struct Arena {
+  char* base;
+  size_t off = 0;
+  explicit Arena(void* b) : base(static_cast<char*>(b)) {}
+  template <typename T>
+  T* take(size_t count) {
+    off = align_up(off, 256);
+    T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+    off += count * sizeof(T);
+    return p;
+  }
+};
+
+struct MatHost {
+  int n, m, r, user_index;
+};
+
+struct Plan {
+  int RP = 0, W = 0;
+  std::vector<MatHost> mats;
+  std::vector<LayerDev> layers;
+  std::vector<VectorDev> vecs;
+  std::vector<Tile> tiles1, tiles2, tiles3;
+  std::vector<FactorBlock> fbP, fbQ;
+  std::vector<ExchangeChunk> chP, chQ, chV;
+  std::vector<float> thrP, thrQ, deqP, deqQ;
+  std::vector<lqsgd_layer_layout> layout;     // by user layer index
+  size_t payload_bytes = 0, payload_stride = 0;
+  size_t elems_total = 0;                     // all layers, one worker
+  std::vector<size_t> elem_off;               // by user index, offset in a worker's staging plane
+  // device addresses (null when only counting)
+  LayerDev* d_layers = nullptr;
+  VectorDev* d_vecs = nullptr;
+  Tile *d_tiles1 = nullptr, *d_tiles2 = nullptr, *d_tiles3 = nullptr;
+  FactorBlock *d_fbP = nullptr, *d_fbQ = nullptr;
+  ExchangeChunk *d_chP = nullptr, *d_chQ = nullptr, *d_chV = nullptr;
+  float *d_thrP = nullptr, *d_thrQ = nullptr, *d_deqP = nullptr, *d_deqQ = nullptr;
+  void** d_ptrs = nullptr;                    // [grads n_mat*W | ghat n_mat | vgrads nvec*W | vghat nvec]
+  uint32_t* d_status = nullptr;
+  uint8_t* d_payload = nullptr;
+  float* d_stage_g = nullptr;                 // [W][elems_total]
+  float* d_stage_ghat = nullptr;              // [elems_total]
+  size_t state_begin = 0, state_end = 0;      // byte range to zero at create (E, factors, codes ...)
+  size_t bytes = 0;
+};
+
+int padded_rank(int r) { return r <= 1 ? 1 : r <= 2 ? 2 : r <= 4 ? 4 : r <= 8 ? 8 : 16; }
+
+int check_config(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config* c) {
+  if (!shapes || !c || n_layers < 1) return LQSGD_ERR_INVALID_ARG;
+  if (c->struct_size != sizeof(lqsgd_config)) return LQSGD_ERR_INVALID_ARG;
+  if (c->rank < 1 || c->rank > kMaxRank) return LQSGD_ERR_INVALID_ARG;
+  if (c->bits_p < 2 || c->bits_p > 8 || c->bits_q < 2 || c->bits_q > 8) return LQSGD_ERR_INVALID_ARG;
+  if (!(c->alpha > 0.f) || !std::isfinite(c->alpha)) return LQSGD_ERR_INVALID_ARG;
+  if (c->workers < 1 || c->workers > 256) return LQSGD_ERR_INVALID_ARG;
+  if (c->flags & ~LQSGD_FLAG_HOST_STAGING) return LQSGD_ERR_INVALID_ARG;
+  for (int i = 0; i < n_layers; ++i) {
+    if (shapes[i].rows < 1 || shapes[i].cols < 1) return LQSGD_ERR_BAD_SHAPE;
+    if ((int64_t)shapes[i].rows * shapes[i].cols > (int64_t)1 << 30) return LQSGD_ERR_BAD_SHAPE;
+  }
+  return LQSGD_OK;
+}
+
+// Decision thresholds and dequantisation table of the b-bit quantiser (Eq. 4 / Eq. 5):
+// boundary between levels k and k+1 at |x|/s = ((1+alpha)^((k+1/2)/(L-1)) - 1)/alpha, stored as
+// the smallest fp32 >= that value; deq[S + W(L-1)] = sign(S) ((1+alpha)^(|S|/(W(L-1))) - 1)/alpha.
+void quant_tables(int bits, double alpha, int W, std::vector<float>& thr, std::vector<float>& deq) {
+  const int L = 1 << (bits - 1);
+  const double la = std::log1p(alpha);
+  thr.resize(L - 1);
+  for (int k = 0; k < L - 1; ++k) {
+    const double T = std::expm1((k + 0.5) / (L - 1) * la) / alpha;
+    float f = (float)T;
+    if ((double)f < T) f = std::nextafterf(f, INFINITY);
+    thr[k] = f;
+  }
+  const int C = W * (L - 1);
+  deq.resize(2 * (size_t)C + 1);
+  for (int S = -C; S <= C; ++S) {
+    const double q = std::fabs((double)S) / C;
+    const double x = std::expm1(q * la) / alpha;
+    deq[S + C] = (float)(S < 0 ? -x : x);
+  }
+}
+
+// Picks the largest candidate size whose tile count reaches `want`, else the smallest.
+template <typename F>
+int pick_size(const std::vector<int>& candidates, size_t want, F count_tiles) {
+  for (int c : candidates)
+    if (count_tiles(c) >= want) return c;
+  return candidates.back();
+}
+
+// Lays out the workspace and builds every table.  base == nullptr: size only.
+void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg, void* base, int sm_count,
+               Plan& p) {
+  const int W = cfg.workers, RP = padded_rank(cfg.rank);
+  p.RP = RP;
+  p.W = W;
+  p.layout.assign(n_layers, lqsgd_layer_layout{});
+  p.elem_off.resize(n_layers);
+  for (int i = 0; i < n_layers; ++i) {
+    p.elem_off[i] = p.elems_total;
+    p.elems_total += align_up((size_t)shapes[i].rows * shapes[i].cols, 4);   // keeps 16-byte alignment
+    if (shapes[i].rows > 1 && shapes[i].cols > 1) {
+      const int r = std::min({cfg.rank, shapes[i].rows, shapes[i].cols});
+      p.mats.push_back({shapes[i].rows, shapes[i].cols, r, i});
+    } else {
+      p.vecs.push_back({shapes[i].rows * shapes[i].cols, i, 0});
+    }
+  }
+  // ---- payload layout: [scales][1-D fp32][P streams][Q streams]
+  size_t off = 0;
+  for (auto& mt : p.mats) { p.layout[mt.user_index].scale_offset = off; off += 8; }
+  for (auto& v : p.vecs) {
+    v.pay_off = off;
+    auto& lo = p.layout[v.user_index];
+    lo.vec_offset = off; lo.vec_bytes = 4 * (size_t)v.len;
+    off += lo.vec_bytes;
+  }
+  for (auto& mt : p.mats) {
+    auto& lo = p.layout[mt.user_index];
+    lo.is_matrix = 1; lo.rank_eff = mt.r;
+    lo.p_offset = off; lo.p_bytes = ((size_t)mt.n * mt.r * cfg.bits_p + 7) / 8; off += lo.p_bytes;
+  }
+  for (auto& mt : p.mats) {
+    auto& lo = p.layout[mt.user_index];
+    lo.q_offset = off; lo.q_bytes = ((size_t)mt.m * mt.r * cfg.bits_q + 7) / 8; off += lo.q_bytes;
+  }
+  p.payload_bytes = off;
+  p.payload_stride = align_up(off, 16);
+
+  // ---- tile sizes
+  const size_t slots = (size_t)sm_count * 2, want = 3 * slots;
+  auto vec_of = [](int m) { return (m % 4 == 0) ? 4 : 1; };
+  auto chunk_width = [&](int m, int cmax) {          // balanced column chunks, multiple of 32*VEC
+    const int v = vec_of(m), q = 32 * v;
+    const int lim = (v == 4) ? cmax : std::max(q, cmax / 4);
+    const int ncc = ceil_div(m, lim);
+    return (int)align_up((size_t)ceil_div(m, ncc), q);
+  };
+  const int c1 = pick_size({2048, 1024, 512}, want, [&](int c) {
+    size_t t = 0;
+    for (auto& mt : p.mats) t += (size_t)W * ceil_div(mt.n, kPass1Rows) * ceil_div(mt.m, chunk_width(mt.m, c));
+    return t;
+  });
+  const int r2max = std::max(128, 32 * RP);
+  auto colchunks = [&](int m) { return ceil_div(m, 128 * vec_of(m)); };
+  auto balanced_rows = [](int n, int rmax) { return ceil_div(n, ceil_div(n, rmax)); };
+  const int r2 = pick_size({r2max, r2max / 2, std::max(32, r2max / 4)}, want, [&](int r) {
+    size_t t = 0;
+    for (auto& mt : p.mats) t += (size_t)W * ceil_div(mt.n, balanced_rows(mt.n, r)) * colchunks(mt.m);
+    return t;
+  });
+  const int r3max = std::max(8, 64 / W);
+  const int r3 = pick_size({r3max, std::max(8, r3max / 2), 8}, want, [&](int r) {
+    size_t t = 0;
+    for (auto& mt : p.mats) t += (size_t)ceil_div(mt.n, balanced_rows(mt.n, r)) * colchunks(mt.m);
+    return t;
+  });
+
+  // ---- carve
+  Arena a(base);
+  p.d_layers = a.take<LayerDev>(p.mats.size());
+  p.d_vecs = a.take<VectorDev>(p.vecs.size());
+  p.state_begin = align_up(a.off, 256);
+  p.layers.resize(p.mats.size());
+  for (size_t li = 0; li < p.mats.size(); ++li) {
+    const MatHost& mt = p.mats[li];
+    LayerDev& L = p.layers[li];
+    std::memset(&L, 0, sizeof(L));
+    L.n = mt.n; L.m = mt.m; L.r = mt.r; L.vec = vec_of(mt.m) == 4; L.user_index = mt.user_index;
+    const int cw = chunk_width(mt.m, c1);
+    L.ncc = ceil_div(mt.m, cw);
+    const int tr2 = balanced_rows(mt.n, r2);
+    L.nrb = ceil_div(mt.n, tr2);
+    L.npb = ceil_div(mt.n, kFactorBlockRows);
+    L.nqb = ceil_div(mt.m, kFactorBlockRows);
+    const size_t nm = (size_t)mt.n * mt.m;
+    L.E = a.take<float>((size_t)W * nm);
+    L.Q = a.take<float>((size_t)mt.m * RP);
+    L.Ppart = a.take<float>((size_t)W * L.ncc * mt.n * RP);
+    L.Praw = (L.ncc == 1) ? L.Ppart : a.take<float>((size_t)W * mt.n * RP);
+    L.P = a.take<float>((size_t)W * mt.n * RP);
+    L.Pbar = a.take<float>((size_t)mt.n * RP);
+    L.Qpart = a.take<float>((size_t)W * L.nrb * mt.m * RP);
+    L.Qw = (L.nrb == 1) ? L.Qpart : a.take<float>((size_t)W * mt.m * RP);
+    L.gram_part = a.take<double>((size_t)W * L.npb * RP * RP);
+    L.rinv = a.take<double>((size_t)W * RP * RP);
+    L.maxp = a.take<float>((size_t)W * L.npb);
+    L.maxq = a.take<float>((size_t)W * L.nqb);
+    L.codesP = a.take<uint8_t>((size_t)W * mt.n * mt.r);
+    L.codesQ = a.take<uint8_t>((size_t)W * mt.m * mt.r);
+    L.scales = a.take<float>(2);
+    const auto& lo = p.layout[mt.user_index];
+    L.pay_scale_off = lo.scale_offset; L.pay_p_off = lo.p_offset; L.pay_q_off = lo.q_offset;
+
+    // tiles
+    const int li32 = (int)li;
+    for (int rb = 0; rb < ceil_div(mt.n, kPass1Rows); ++rb)
+      for (int cc = 0; cc < L.ncc; ++cc)
+        for (int w = 0; w < W; ++w) {
+          const int row0 = rb * kPass1Rows, col0 = cc * cw;
+          p.tiles1.push_back({li32, w, row0, std::min(kPass1Rows, mt.n - row0), col0, std::min(cw, mt.m - col0), cc, 0});
+        }
+    const int cw2 = 128 * vec_of(mt.m);
+    for (int w = 0; w < W; ++w)
+      for (int rb = 0; rb < L.nrb; ++rb)
+        for (int cc = 0; cc < ceil_div(mt.m, cw2); ++cc) {
+          const int row0 = rb * tr2, col0 = cc * cw2;
+          p.tiles2.push_back({li32, w, row0, std::min(tr2, mt.n - row0), col0, std::min(cw2, mt.m - col0), rb, 0});
+        }
+    const int tr3 = balanced_rows(mt.n, r3);
+    for (int rb = 0; rb < ceil_div(mt.n, tr3); ++rb)
+      for (int cc = 0; cc < ceil_div(mt.m, cw2); ++cc) {
+        const int row0 = rb * tr3, col0 = cc * cw2;
+        p.tiles3.push_back({li32, 0, row0, std::min(tr3, mt.n - row0), col0, std::min(cw2, mt.m - col0), 0, 0});
+      }
+    for (int w = 0; w < W; ++w) {
+      for (int b = 0; b < L.npb; ++b) p.fbP.push_back({li32, w, b, 0});
+      for (int b = 0; b < L.nqb; ++b) p.fbQ.push_back({li32, w, b, 0});
+    }
+    for (int c = 0; c < ceil_div(mt.n * mt.r, kExchangeChunk); ++c) p.chP.push_back({li32, c});
+    for (int c = 0; c < ceil_div(mt.m * mt.r, kExchangeChunk); ++c) p.chQ.push_back({li32, c});
+  }
+  for (size_t vi = 0; vi < p.vecs.size(); ++vi)
+    for (int c = 0; c < ceil_div(p.vecs[vi].len, 256); ++c) p.chV.push_back({(int)vi, c});
+  p.d_status = a.take<uint32_t>(p.mats.size());
+  p.d_payload = a.take<uint8_t>((size_t)W * p.payload_stride);
+  p.state_end = a.off;
+
+  quant_tables(cfg.bits_p, cfg.alpha, W, p.thrP, p.deqP);
+  quant_tables(cfg.bits_q, cfg.alpha, W, p.thrQ, p.deqQ);
+  p.d_tiles1 = a.take<Tile>(p.tiles1.size());
+  p.d_tiles2 = a.take<Tile>(p.tiles2.size());
+  p.d_tiles3 = a.take<Tile>(p.tiles3.size());
+  p.d_fbP = a.take<FactorBlock>(p.fbP.size());
+  p.d_fbQ = a.take<FactorBlock>(p.fbQ.size());
+  p.d_chP = a.take<ExchangeChunk>(p.chP.size());
+  p.d_chQ = a.take<ExchangeChunk>(p.chQ.size());
+  p.d_chV = a.take<ExchangeChunk>(p.chV.size());
+  p.d_thrP = a.take<float>(p.thrP.size());
+  p.d_thrQ = a.take<float>(p.thrQ.size());
+  p.d_deqP = a.take<float>(p.deqP.size());
+  p.d_deqQ = a.take<float>(p.deqQ.size());
+  p.d_ptrs = a.take<void*>((p.mats.size() + p.vecs.size()) * (size_t)(W + 1));
+  if (cfg.flags & LQSGD_FLAG_HOST_STAGING) {
+    p.d_stage_g = a.take<float>((size_t)W * p.elems_total);
+    p.d_stage_ghat = a.take<float>(p.elems_total);
+  }
+  p.bytes = align_up(a.off, 256);
+}
+
+// Q_0 ~ N(0,1) (Alg. 1 initialisation): counter-based, a 64-bit integer mix of
+// (seed, layer, element) feeding Box-Muller in double precision.
+uint64_t mix64(uint64_t x) {
+  x += 0x9E3779B97F4A7C15ull;
+  x = (x ^ (x >> 30)) * 0xBF58476D1CE4E5B9ull;
+  x = (x ^ (x >> 27)) * 0x94D049BB133111EBull;
+  return x ^ (x >> 31);
+}
+float normal_draw(uint64_t seed, uint64_t layer, uint64_t idx) {
+  const uint64_t k = mix64(mix64(seed ^ 0xA0761D6478BD642Full) + layer * 0xE7037ED1A0B428DBull);
+  const uint64_t a = mix64(k + 2 * idx), b = mix64(k + 2 * idx + 1);
+  const double u1 = ((double)(a >> 11) + 1.0) * (1.0 / 9007199254740992.0);   // (0, 1]
+  const double u2 = (double)(b >> 11) * (1.0 / 9007199254740992.0);           // [0, 1)
+  return (float)(std::sqrt(-2.0 * std::log(u1)) * std::cos(6.283185307179586476925 * u2));
+}
+
+}  // namespace
+
+struct lqsgd_ctx {
+  lqsgd_config cfg;
+  std::vector<lqsgd_shape> shapes;
+  Plan plan;
+  int device = 0, sm_count = 0;
+  int grid1 = 0, grid2 = 0, grid3 = 0;
+  std::vector<void*> ptrs_host;      // mirror of plan.d_ptrs
+  bool ptrs_valid = false;
+  void* workspace = nullptr;
+};
+
+extern "C" {
+
+int lqsgd_version(void) { return LQSGD_VERSION; }
+
+const char* lqsgd_last_cuda_error(void) { return g_cuda_error.c_str(); }
+
+const char* lqsgd_strerror(int code) {
+  switch (code) {
+    case LQSGD_OK: return "ok";
+    case LQSGD_ERR_INVALID_ARG: return "invalid argument";
+    case LQSGD_ERR_BAD_SHAPE: return "bad layer shape";
+    case LQSGD_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case LQSGD_ERR_MISALIGNED: return "misaligned pointer";
+    case LQSGD_ERR_CUDA: return "CUDA runtime error";
+    case LQSGD_ERR_NO_STAGING: return "context was created without host staging";
+    case LQSGD_ERR_OUT_OF_RANGE: return "index out of range";
+    default: return "unknown error";
+  }
+}
+
+int lqsgd_workspace_bytes(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config* cfg, size_t* out) {
+  if (!out) return LQSGD_ERR_INVALID_ARG;
+  const int rc = check_config(shapes, n_layers, cfg);
+  if (rc != LQSGD_OK) return rc;
+  Plan p;
+  // The size must not depend on the device: plan for the largest SM count tile sizes consider.
+  make_plan(shapes, n_layers, *cfg, nullptr, 148, p);
+  Plan p2;
+  make_plan(shapes, n_layers, *cfg, nullptr, 1, p2);
+  *out = std::max(p.bytes, p2.bytes);
+  return LQSGD_OK;
+}
+
+int lqsgd_create(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config* cfg, void* dev_workspace,
+                 size_t workspace_bytes, lqsgd_ctx** ctx_out) {
+  if (!ctx_out) return LQSGD_ERR_INVALID_ARG;
+  *ctx_out = nullptr;
+  int rc = check_config(shapes, n_layers, cfg);
+  if (rc != LQSGD_OK) return rc;
+  if (!dev_workspace) return LQSGD_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(dev_workspace) % 256) return LQSGD_ERR_MISALIGNED;
+  size_t need = 0;
+  rc = lqsgd_workspace_bytes(shapes, n_layers, cfg, &need);
+  if (rc != LQSGD_OK) return rc;
+  if (workspace_bytes < need) return LQSGD_ERR_WORKSPACE_TOO_SMALL;
+
+  lqsgd_ctx* c = new (std::nothrow) lqsgd_ctx();
+  if (!c) return LQSGD_ERR_INVALID_ARG;
+  struct Guard { lqsgd_ctx* c; ~Guard() { delete c; } } guard{c};
+  c->cfg = *cfg;
+  c->shapes.assign(shapes, shapes + n_layers);
+  c->workspace = dev_workspace;
+  CK(cudaGetDevice(&c->device));
+  CK(cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device));
+  // tile sizes for 148 or for 1 SM bound the workspace; use the device's count if it fits
+  int sm_plan = c->sm_count;
+  make_plan(shapes, n_layers, *cfg, dev_workspace, sm_plan, c->plan);
+  if (c->plan.bytes > workspace_bytes) {
+    c->plan = Plan();
+    sm_plan = 148;
+    make_plan(shapes, n_layers, *cfg, dev_workspace, sm_plan, c->plan);
+  }
+  Plan& p = c->plan;
+  if (p.bytes > workspace_bytes) return LQSGD_ERR_WORKSPACE_TOO_SMALL;
+
+  char* base = static_cast<char*>(dev_workspace);
+  CK(cudaMemset(base + p.state_begin, 0, p.state_end - p.state_begin));   // E_0 = 0, padding columns 0
+  auto up = [&](void* dst, const void* src, size_t bytes) -> cudaError_t {
+    return bytes ? cudaMemcpy(dst, src, bytes, cudaMemcpyHostToDevice) : cudaSuccess;
+  };
+  CK(up(p.d_layers, p.layers.data(), p.layers.size() * sizeof(LayerDev)));
+  CK(up(p.d_vecs, p.vecs.data(), p.vecs.size() * sizeof(VectorDev)));
+  CK(up(p.d_tiles1, p.tiles1.data(), p.tiles1.size() * sizeof(Tile)));
+  CK(up(p.d_tiles2, p.tiles2.data(), p.tiles2.size() * sizeof(Tile)));
+  CK(up(p.d_tiles3, p.tiles3.data(), p.tiles3.size() * sizeof(Tile)));
+  CK(up(p.d_fbP, p.fbP.data(), p.fbP.size() * sizeof(FactorBlock)));
+  CK(up(p.d_fbQ, p.fbQ.data(), p.fbQ.size() * sizeof(FactorBlock)));
+  CK(up(p.d_chP, p.chP.data(), p.chP.size() * sizeof(ExchangeChunk)));
+  CK(up(p.d_chQ, p.chQ.data(), p.chQ.size() * sizeof(ExchangeChunk)));
+  CK(up(p.d_chV, p.chV.data(), p.chV.size() * sizeof(ExchangeChunk)));
+  CK(up(p.d_thrP, p.thrP.data(), p.thrP.size() * sizeof(float)));
+  CK(up(p.d_thrQ, p.thrQ.data(), p.thrQ.size() * sizeof(float)));
+  CK(up(p.d_deqP, p.deqP.data(), p.deqP.size() * sizeof(float)));
+  CK(up(p.d_deqQ, p.deqQ.data(), p.deqQ.size() * sizeof(float)));
+  // Q_0
+  std::vector<float> q0;
+  for (size_t li = 0; li < p.mats.size(); ++li) {
+    const MatHost& mt = p.mats[li];
+    q0.assign((size_t)mt.m * p.RP, 0.f);
+    for (int i = 0; i < mt.m; ++i)
+      for (int j = 0; j < mt.r; ++j)
+        q0[(size_t)i * p.RP + j] = normal_draw(cfg->seed, (uint64_t)mt.user_index, (uint64_t)i * mt.r + j);
+    CK(up(p.layers[li].Q, q0.data(), q0.size() * sizeof(float)));
+  }
+  int o1 = 1, o2 = 1, o3 = 1;
+  CK(pass_occupancy(p.RP, &o1, &o2, &o3));
+  c->grid1 = (int)std::min<size_t>(p.tiles1.size(), (size_t)c->sm_count * std::max(o1, 1));
+  c->grid2 = (int)std::min<size_t>(p.tiles2.size(), (size_t)c->sm_count * std::max(o2, 1));
+  c->grid3 = (int)std::min<size_t>(p.tiles3.size(), (size_t)c->sm_count * std::max(o3, 1));
+  c->ptrs_host.assign((p.mats.size() + p.vecs.size()) * (size_t)(p.W + 1), nullptr);
+  CK(cudaDeviceSynchronize());
+  guard.c = nullptr;
+  *ctx_out = c;
+  return LQSGD_OK;
+}
+
+void lqsgd_destroy(lqsgd_ctx* ctx) { delete ctx; }
+
+int lqsgd_launches_per_step(const lqsgd_ctx* ctx, int32_t* out) {
+  if (!ctx || !out) return LQSGD_ERR_INVALID_ARG;
+  *out = (ctx->plan.mats.empty() ? 0 : 9) + (ctx->plan.chV.empty() ? 0 : 1);
+  return LQSGD_OK;
+}
+
+int lqsgd_step(lqsgd_ctx* c, const float* const* grads, float* const* ghat, void* cuda_stream) {
+  if (!c || !grads || !ghat) return LQSGD_ERR_INVALID_ARG;
+  Plan& p = c->plan;
+  const int W = p.W, nl = (int)c->shapes.size();
+  const size_t nm = p.mats.size(), nv = p.vecs.size();
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  // ---- check and gather pointers: [grads nm*W | ghat nm | vgrads nv*W | vghat nv]
+  std::vector<void*> ptrs(c->ptrs_host.size());
+  for (size_t li = 0; li < nm; ++li) {
+    const int ui = p.mats[li].user_index;
+    const uintptr_t amask = (p.mats[li].m % 4 == 0) ? 15 : 3;
+    for (int w = 0; w < W; ++w) {
+      const float* g = grads[(size_t)w * nl + ui];
+      if (!g) return LQSGD_ERR_INVALID_ARG;
+      if (reinterpret_cast<uintptr_t>(g) & amask) return LQSGD_ERR_MISALIGNED;
+      ptrs[li * W + w] = const_cast<float*>(g);
+    }
+    if (!ghat[ui]) return LQSGD_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(ghat[ui]) & amask) return LQSGD_ERR_MISALIGNED;
+    ptrs[nm * W + li] = ghat[ui];
+  }
+  const size_t vbase = nm * (W + 1);
+  for (size_t vi = 0; vi < nv; ++vi) {
+    const int ui = p.vecs[vi].user_index;
+    for (int w = 0; w < W; ++w) {
+      const float* g = grads[(size_t)w * nl + ui];
+      if (!g) return LQSGD_ERR_INVALID_ARG;
+      if (reinterpret_cast<uintptr_t>(g) & 3) return LQSGD_ERR_MISALIGNED;
+      ptrs[vbase + vi * W + w] = const_cast<float*>(g);
+    }
+    if (!ghat[ui]) return LQSGD_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(ghat[ui]) & 3) return LQSGD_ERR_MISALIGNED;
+    ptrs[vbase + nv * W + vi] = ghat[ui];
+  }
+  if (!c->ptrs_valid || ptrs != c->ptrs_host) {
+    c->ptrs_host = ptrs;
+    // pageable source: the runtime stages it before returning, so the vector may change afterwards
+    CK(cudaMemcpyAsync(p.d_ptrs, c->ptrs_host.data(), ptrs.size() * sizeof(void*), cudaMemcpyHostToDevice, st));
+    c->ptrs_valid = true;
+  }
+  Tables t;
+  t.layers = p.d_layers;
+  t.grads = reinterpret_cast<const float* const*>(p.d_ptrs);
+  t.ghat = reinterpret_cast<float* const*>(p.d_ptrs + nm * W);
+  t.payload = p.d_payload;
+  t.payload_stride = p.payload_stride;
+  t.status = p.d_status;
+  t.W = W;
+  const QuantTables qp{p.d_thrP, p.d_deqP, c->cfg.bits_p}, qq{p.d_thrQ, p.d_deqQ, c->cfg.bits_q};
+  const int RP = p.RP;
+  if (nm) {
+    CK(cudaMemsetAsync(p.d_status, 0, nm * sizeof(uint32_t), st));
+    CK(launch_pass1(RP, t, p.d_tiles1, (int)p.tiles1.size(), {st, c->grid1}));
+    CK(launch_p_reduce_gram(RP, t, p.d_fbP, (int)p.fbP.size(), {st, 0}));
+    CK(launch_p_cholesky(RP, t, (int)nm, {st, 0}));
+    CK(launch_p_apply(RP, t, p.d_fbP, (int)p.fbP.size(), {st, 0}));
+    CK(launch_exchange(RP, 0, t, qp, p.d_chP, (int)p.chP.size(), {st, 0}));
+    CK(launch_pass2(RP, t, p.d_tiles2, (int)p.tiles2.size(), {st, c->grid2}));
+    CK(launch_q_reduce(RP, t, p.d_fbQ, (int)p.fbQ.size(), {st, 0}));
+    CK(launch_exchange(RP, 1, t, qq, p.d_chQ, (int)p.chQ.size(), {st, 0}));
+    CK(launch_pass3(RP, t, p.d_tiles3, (int)p.tiles3.size(), {st, c->grid3}));
+  }
+  if (nv) {
+    CK(launch_vectors(p.d_vecs, p.d_chV, (int)p.chV.size(),
+                      reinterpret_cast<const float* const*>(p.d_ptrs + vbase),
+                      reinterpret_cast<float* const*>(p.d_ptrs + vbase + nv * W), p.d_payload,
+                      p.payload_stride, W, {st, 0}));
+  }
+  return LQSGD_OK;
+}
+
+int lqsgd_step_host(lqsgd_ctx* c, const float* const* host_grads, float* const* host_ghat,
+                    void* host_payload, void* cuda_stream) {
+  if (!c || !host_grads || !host_ghat) return LQSGD_ERR_INVALID_ARG;
+  Plan& p = c->plan;
+  if (!p.d_stage_g) return LQSGD_ERR_NO_STAGING;
+  const int W = p.W, nl = (int)c->shapes.size();
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  std::vector<const float*> dg((size_t)W * nl);
+  std::vector<float*> dh(nl);
+  for (int l = 0; l < nl; ++l) {
+    const size_t bytes = 4 * (size_t)c->shapes[l].rows * c->shapes[l].cols;
+    for (int w = 0; w < W; ++w) {
+      const float* src = host_grads[(size_t)w * nl + l];
+      if (!src) return LQSGD_ERR_INVALID_ARG;
+      float* dst = p.d_stage_g + (size_t)w * p.elems_total + p.elem_off[l];
+      CK(cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, st));
+      dg[(size_t)w * nl + l] = dst;
+    }
+    if (!host_ghat[l]) return LQSGD_ERR_INVALID_ARG;
+    dh[l] = p.d_stage_ghat + p.elem_off[l];
+  }
+  const int rc = lqsgd_step(c, dg.data(), dh.data(), cuda_stream);
+  if (rc != LQSGD_OK) return rc;
+  for (int l = 0; l < nl; ++l) {
+    const size_t bytes = 4 * (size_t)c->shapes[l].rows * c->shapes[l].cols;
+    CK(cudaMemcpyAsync(host_ghat[l], dh[l], bytes, cudaMemcpyDeviceToHost, st));
+  }
+  if (host_payload) {
+    CK(cudaMemcpy2DAsync(host_payload, p.payload_bytes, p.d_payload, p.payload_stride, p.payload_bytes, W,
+                         cudaMemcpyDeviceToHost, st));
+  }
+  CK(cudaStreamSynchronize(st));
+  return LQSGD_OK;
+}
+
+int lqsgd_payload_bytes(const lqsgd_ctx* c, size_t* out) {
+  if (!c || !out) return LQSGD_ERR_INVALID_ARG;
+  *out = c->plan.payload_bytes;
+  return LQSGD_OK;
+}
+
+int lqsgd_payload(const lqsgd_ctx* c, int32_t worker, const void** dev_ptr, size_t* bytes) {
+  if (!c || !dev_ptr || !bytes) return LQSGD_ERR_INVALID_ARG;
+  if (worker < 0 || worker >= c->plan.W) return LQSGD_ERR_OUT_OF_RANGE;
+  *dev_ptr = c->plan.d_payload + (size_t)worker * c->plan.payload_stride;
+  *bytes = c->plan.payload_bytes;
+  return LQSGD_OK;
+}
+
+int lqsgd_payload_layout(const lqsgd_ctx* c, int32_t layer, lqsgd_layer_layout* out) {
+  if (!c || !out) return LQSGD_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= (int)c->shapes.size()) return LQSGD_ERR_OUT_OF_RANGE;
+  *out = c->plan.layout[layer];
+  return LQSGD_OK;
+}
+
+// Locates a piece of state: base pointer, rows, dense row bytes, stored row pitch in bytes.
+static int locate_state(const lqsgd_ctx* c, int which, int layer, int worker, char** base, size_t* rows,
+                        size_t* row_bytes, size_t* pitch) {
+  if (layer < 0 || layer >= (int)c->shapes.size()) return LQSGD_ERR_OUT_OF_RANGE;
+  const Plan& p = c->plan;
+  int li = -1;
+  for (size_t i = 0; i < p.mats.size(); ++i)
+    if (p.mats[i].user_index == layer) li = (int)i;
+  if (li < 0) return LQSGD_ERR_OUT_OF_RANGE;          // 1-D tensors carry no state
+  const LayerDev& L = p.layers[li];
+  const size_t n = L.n, m = L.m, r = L.r, RP = p.RP, W = p.W;
+  const bool per_worker = which == LQSGD_STATE_E || which == LQSGD_STATE_P_RAW || which == LQSGD_STATE_P ||
+                          which == LQSGD_STATE_Q_W || which == LQSGD_STATE_CODES_P || which == LQSGD_STATE_CODES_Q;
+  if (per_worker && (worker < 0 || worker >= (int)W)) return LQSGD_ERR_OUT_OF_RANGE;
+  const size_t w = per_worker ? worker : 0;
+  switch (which) {
+    case LQSGD_STATE_E: *base = (char*)(L.E + w * n * m); *rows = 1; *row_bytes = *pitch = 4 * n * m; break;
+    case LQSGD_STATE_Q: *base = (char*)L.Q; *rows = m; *row_bytes = 4 * r; *pitch = 4 * RP; break;
+    case LQSGD_STATE_P_RAW: *base = (char*)(L.Praw + w * n * RP); *rows = n; *row_bytes = 4 * r; *pitch = 4 * RP; break;
+    case LQSGD_STATE_P: *base = (char*)(L.P + w * n * RP); *rows = n; *row_bytes = 4 * r; *pitch = 4 * RP; break;
+    case LQSGD_STATE_P_BAR: *base = (char*)L.Pbar; *rows = n; *row_bytes = 4 * r; *pitch = 4 * RP; break;
+    case LQSGD_STATE_Q_W: *base = (char*)(L.Qw + w * m * RP); *rows = m; *row_bytes = 4 * r; *pitch = 4 * RP; break;
+    case LQSGD_STATE_CODES_P: *base = (char*)(L.codesP + w * n * r); *rows = 1; *row_bytes = *pitch = n * r; break;
+    case LQSGD_STATE_CODES_Q: *base = (char*)(L.codesQ + w * m * r); *rows = 1; *row_bytes = *pitch = m * r; break;
+    case LQSGD_STATE_SCALES: *base = (char*)L.scales; *rows = 1; *row_bytes = *pitch = 8; break;
+    default: return LQSGD_ERR_OUT_OF_RANGE;
+  }
+  return LQSGD_OK;
+}
+
+int lqsgd_get_state(const lqsgd_ctx* c, int32_t which, int32_t layer, int32_t worker, void* dev_dst,
+                    void* cuda_stream) {
+  if (!c || !dev_dst) return LQSGD_ERR_INVALID_ARG;
+  char* base; size_t rows, rb, pitch;
+  const int rc = locate_state(c, which, layer, worker, &base, &rows, &rb, &pitch);
+  if (rc != LQSGD_OK) return rc;
+  CK(cudaMemcpy2DAsync(dev_dst, rb, base, pitch, rb, rows, cudaMemcpyDeviceToDevice,
+                       static_cast<cudaStream_t>(cuda_stream)));
+  return LQSGD_OK;
+}
+
+int lqsgd_set_state(lqsgd_ctx* c, int32_t which, int32_t layer, int32_t worker, const void* dev_src,
+                    void* cuda_stream) {
+  if (!c || !dev_src) return LQSGD_ERR_INVALID_ARG;
+  if (which != LQSGD_STATE_E && which != LQSGD_STATE_Q) return LQSGD_ERR_OUT_OF_RANGE;
+  char* base; size_t rows, rb, pitch;
+  const int rc = locate_state(c, which, layer, worker, &base, &rows, &rb, &pitch);
+  if (rc != LQSGD_OK) return rc;
+  CK(cudaMemcpy2DAsync(base, pitch, dev_src, rb, rb, rows, cudaMemcpyDeviceToDevice,
+                       static_cast<cudaStream_t>(cuda_stream)));
+  return LQSGD_OK;
+}
+
+int lqsgd_status(const lqsgd_ctx* c, uint32_t* host_flags, void* cuda_stream) {
+  if (!c || !host_flags) return LQSGD_ERR_INVALID_ARG;
+  const Plan& p = c->plan;
+  for (size_t i = 0; i < c->shapes.size(); ++i) host_flags[i] = 0;
+  std::vector<uint32_t> tmp(p.mats.size());
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (!tmp.empty()) {
+    CK(cudaMemcpyAsync(tmp.data(), p.d_status, tmp.size() * sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
+  }
+  CK(cudaStreamSynchronize(st));
+  for (size_t i = 0; i < p.mats.size(); ++i) host_flags[p.mats[i].user_index] = tmp[i];
+  return LQSGD_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,106 @@
+// Device-side tables shared by the host planner (lqsgd_api.cu) and the kernels
+// (lqsgd_kernels.cu).  Internal to the library.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace lqsgd {
+
+constexpr int kMaxRank = 16;
+constexpr int kPassThreads = 256;      // threads per CTA of the three streaming passes
+constexpr int kPass1Rows = 32;         // rows per pass-1 tile: 8 warps x 4 rows
+constexpr int kFactorBlockRows = 128;  // rows of P (or Q) per block of the small factor kernels
+constexpr int kExchangeChunk = 1024;   // factor elements per block of the exchange kernel
+
+// One matrix layer (n x m), as the kernels see it.  Factors are stored with a row stride of
+// RP floats (rank padded to 1, 2, 4, 8 or 16); columns >= r are kept zero.
+struct LayerDev {
+  int32_t n, m, r;            // r = r_eff
+  int32_t vec;                // 1: m % 4 == 0, rows are 16-byte aligned -> float4 path
+  int32_t ncc;                // column chunks of pass 1 (P partial sums)
+  int32_t nrb;                // row chunks of pass 2 (Q partial sums)
+  int32_t npb, nqb;           // factor blocks: ceil(n/128), ceil(m/128)
+  int32_t user_index;         // index in the caller's layer list
+  int32_t pad0;
+  float* E;                   // [W][n][m]   error buffer; holds M between pass 1 and pass 3
+  float* Q;                   // [m][RP]     warm start, becomes Q_bar
+  float* Ppart;               // [W][ncc][n][RP]
+  float* Praw;                // [W][n][RP]  (== Ppart when ncc == 1)
+  float* P;                   // [W][n][RP]  orthonormal
+  float* Pbar;                // [n][RP]
+  float* Qpart;               // [W][nrb][m][RP]
+  float* Qw;                  // [W][m][RP]  (== Qpart when nrb == 1)
+  double* gram_part;          // [W][npb][RP*RP]
+  double* rinv;               // [W][RP*RP]  R^-1 (upper triangular), row-major
+  float* maxp;                // [W][npb]
+  float* maxq;                // [W][nqb]
+  uint8_t* codesP;            // [W][n*r]
+  uint8_t* codesQ;            // [W][m*r]
+  float* scales;              // [2]  s_P, s_Q
+  uint64_t pay_scale_off, pay_p_off, pay_q_off;   // byte offsets inside one worker's payload
+};
+
+// One 1-D tensor.
+struct VectorDev {
+  int32_t len;
+  int32_t user_index;
+  uint64_t pay_off;           // byte offset inside one worker's payload (4-byte aligned)
+};
+
+// A rectangular piece of one layer handled by one CTA of a streaming pass.
+struct Tile {
+  int32_t layer;              // index into the LayerDev table
+  int32_t worker;             // unused by pass 3 (it loops over the workers)
+  int32_t row0, nrows;
+  int32_t col0, ncols;
+  int32_t part;               // pass 1: column-chunk index; pass 2: row-chunk index
+  int32_t pad;
+};
+
+// A block of rows of one worker's factor, handled by one CTA of a small factor kernel.
+struct FactorBlock {
+  int32_t layer, worker, blk, pad;
+};
+
+// A chunk of kExchangeChunk factor elements of one layer, all workers.
+struct ExchangeChunk {
+  int32_t layer, chunk;
+};
+
+struct Tables {
+  const LayerDev* layers;
+  const float* const* grads;  // [n_mat][W] device pointers, by LayerDev index
+  float* const* ghat;         // [n_mat]
+  uint8_t* payload;           // [W][payload_stride]
+  uint64_t payload_stride;
+  uint32_t* status;           // [n_mat]
+  int32_t W;
+};
+
+struct QuantTables {
+  const float* thr;           // [L-1] ascending decision thresholds on |x|/s
+  const float* deq;           // [2*W*(L-1)+1] expand(S / (W (L-1))), index S + W (L-1)
+  int32_t bits;
+};
+
+struct Launch {
+  cudaStream_t stream;
+  int grid;
+};
+
+cudaError_t launch_pass1(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
+cudaError_t launch_p_reduce_gram(int RP, const Tables& t, const FactorBlock* fb, int nfb, Launch l);
+cudaError_t launch_p_cholesky(int RP, const Tables& t, int n_mat, Launch l);
+cudaError_t launch_p_apply(int RP, const Tables& t, const FactorBlock* fb, int nfb, Launch l);
+cudaError_t launch_exchange(int RP, int which /*0 = P, 1 = Q*/, const Tables& t, const QuantTables& q,
+                            const ExchangeChunk* ch, int nch, Launch l);
+cudaError_t launch_pass2(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
+cudaError_t launch_q_reduce(int RP, const Tables& t, const FactorBlock* fb, int nfb, Launch l);
+cudaError_t launch_pass3(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
+cudaError_t launch_vectors(const VectorDev* vecs, const ExchangeChunk* chunks, int nchunks,
+                           const float* const* vgrads, float* const* vghat, uint8_t* payload,
+                           uint64_t payload_stride, int W, Launch l);
+// Resident CTAs per SM of each streaming pass for this RP (for persistent grid sizing).
+cudaError_t pass_occupancy(int RP, int* occ1, int* occ2, int* occ3);
+
+}  // namespace lqsgd

@@ -1,0 +1,793 @@
+// sm_100a kernels of the LQ-SGD round (Algorithm 1, loop body).
+//
+// Three streaming passes over the n x m data carry all the HBM traffic:
+//   pass 1: M = G + E (Eq. 8) written over E, partial P = M Q          (power step)
+//   pass 2: partial Q = M^T P_bar                                        (second power step)
+//   pass 3: G_hat = P_bar Q_bar^T (Eq. 6), E = M - G_hat (Eq. 7)
+// With r <= 16 the products are rank-r updates of a stream: a few FMAs per byte, on CUDA
+// cores with fp32 accumulation; the passes are bound by HBM, not by arithmetic.
+// Between the passes small kernels finish the factors: fixed-order reduction of the partial
+// sums, CholeskyQR in fp64 (Orthonormalize), scale, LogQuantize (Eq. 4 through a threshold
+// table), bit-packing, the exact integer worker sum, LogDequantize (Eq. 5 through a table).
+//
+// Every kernel is a persistent or table-driven grid: CTAs walk a tile table the host planned
+// once, so a 64 x 27 layer costs a table entry, not a launch.  Nothing here spins or waits on
+// another CTA, and every reduction has a fixed order: results are bit-reproducible.
+#include "lqsgd_dev.h"
+
+#include <math.h>
+
+namespace lqsgd {
+namespace {
+
+// ---------------------------------------------------------------------------------------
+// small helpers
+// ---------------------------------------------------------------------------------------
+template <int N>
+__device__ __forceinline__ void load_contig_ro(const float* __restrict__ p, float (&out)[N]) {
+  // N contiguous read-only floats, aligned to min(N,4)*4 bytes, through the read-only path
+  if constexpr (N % 4 == 0) {
+#pragma unroll
+    for (int i = 0; i < N / 4; ++i) {
+      float4 v = __ldg(reinterpret_cast<const float4*>(p) + i);
+      out[4 * i] = v.x; out[4 * i + 1] = v.y; out[4 * i + 2] = v.z; out[4 * i + 3] = v.w;
+    }
+  } else if constexpr (N == 2) {
+    float2 v = __ldg(reinterpret_cast<const float2*>(p));
+    out[0] = v.x; out[1] = v.y;
+  } else {
+#pragma unroll
+    for (int i = 0; i < N; ++i) out[i] = __ldg(p + i);
+  }
+}
+
+template <int N>
+__device__ __forceinline__ void store_contig(float* p, const float (&v)[N]) {
+  if constexpr (N % 4 == 0) {
+#pragma unroll
+    for (int i = 0; i < N / 4; ++i)
+      reinterpret_cast<float4*>(p)[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+  } else if constexpr (N == 2) {
+    *reinterpret_cast<float2*>(p) = make_float2(v[0], v[1]);
+  } else {
+#pragma unroll
+    for (int i = 0; i < N; ++i) p[i] = v[i];
+  }
+}
+
+// VEC consecutive floats of a streamed matrix row (VEC = 4: one 128-bit access, VEC = 1: scalar).
+template <int VEC>
+struct Pack {
+  float v[VEC];
+};
+
+template <int VEC>
+__device__ __forceinline__ Pack<VEC> ld_stream(const float* p) {   // read once: evict first
+  Pack<VEC> r;
+  if constexpr (VEC == 4) {
+    float4 t = __ldcs(reinterpret_cast<const float4*>(p));
+    r.v[0] = t.x; r.v[1] = t.y; r.v[2] = t.z; r.v[3] = t.w;
+  } else {
+    r.v[0] = __ldcs(p);
+  }
+  return r;
+}
+
+template <int VEC>
+__device__ __forceinline__ Pack<VEC> ld_l2(const float* p) {       // keep in L2, skip L1
+  Pack<VEC> r;
+  if constexpr (VEC == 4) {
+    float4 t = __ldcg(reinterpret_cast<const float4*>(p));
+    r.v[0] = t.x; r.v[1] = t.y; r.v[2] = t.z; r.v[3] = t.w;
+  } else {
+    r.v[0] = __ldcg(p);
+  }
+  return r;
+}
+
+template <int VEC>
+__device__ __forceinline__ void st_default(float* p, const Pack<VEC>& x) {
+  if constexpr (VEC == 4) *reinterpret_cast<float4*>(p) = make_float4(x.v[0], x.v[1], x.v[2], x.v[3]);
+  else *p = x.v[0];
+}
+
+template <int VEC>
+__device__ __forceinline__ void st_stream(float* p, const Pack<VEC>& x) {
+  if constexpr (VEC == 4) __stcs(reinterpret_cast<float4*>(p), make_float4(x.v[0], x.v[1], x.v[2], x.v[3]));
+  else __stcs(p, x.v[0]);
+}
+
+// Sum of v[i] over the 32 lanes for every i, in log steps that halve the live values:
+// afterwards lane l holds the totals of indices [l*N/32, (l+1)*N/32) when N >= 32, and the
+// total of index l / (32/N) when N < 32 (in v[0 .. max(N/32,1))).  Fixed order: deterministic.
+template <int N, int O>
+__device__ __forceinline__ void warp_transpose_reduce(float* v, int lane) {
+  if constexpr (O >= 1) {
+    if constexpr (N > 1) {
+      constexpr int H = N / 2;
+      const bool up = (lane & O) != 0;
+#pragma unroll
+      for (int i = 0; i < H; ++i) {
+        const float a = v[i], b = v[i + H];
+        const float send = up ? a : b;
+        const float keep = up ? b : a;
+        v[i] = keep + __shfl_xor_sync(0xffffffffu, send, O);
+      }
+      warp_transpose_reduce<H, O / 2>(v, lane);
+    } else {
+      v[0] += __shfl_xor_sync(0xffffffffu, v[0], O);
+      warp_transpose_reduce<1, O / 2>(v, lane);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// pass 1: M = G + E over E (Eq. 8), partial P = M Q (Alg. 1 power step)
+// A tile is up to 32 rows x one column chunk; each warp owns 4 rows, lanes stride the columns,
+// every lane accumulates 4 x RP partial dot products and the warp reduces them at the end.
+// ---------------------------------------------------------------------------------------
+template <int RP, int VEC>
+__device__ __forceinline__ void pass1_tile(const Tables& t, const Tile& tl) {
+  const LayerDev& L = t.layers[tl.layer];
+  const int m = L.m;
+  const float* __restrict__ G = t.grads[(size_t)tl.layer * t.W + tl.worker];
+  float* __restrict__ E = L.E + (size_t)tl.worker * L.n * m;
+  const float* __restrict__ Q = L.Q;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int r0 = tl.row0 + warp * 4;
+  const int nr = min(4, tl.row0 + tl.nrows - r0);   // rows this warp owns (may be <= 0)
+  if (nr <= 0) return;
+  const int cend = tl.col0 + tl.ncols;
+  constexpr int STEP = 32 * VEC;
+
+  float acc[4 * RP];
+#pragma unroll
+  for (int i = 0; i < 4 * RP; ++i) acc[i] = 0.f;
+
+  Pack<VEC> g[4], e[4];
+  int c = tl.col0 + lane * VEC;
+  auto fetch = [&](int col, Pack<VEC>(&gg)[4], Pack<VEC>(&ee)[4]) {
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+      if (a < nr) {
+        const size_t off = (size_t)(r0 + a) * m + col;
+        gg[a] = ld_stream<VEC>(G + off);
+        ee[a] = ld_stream<VEC>(E + off);
+      }
+    }
+  };
+  if (c < cend) fetch(c, g, e);
+  for (; c < cend; c += STEP) {
+    Pack<VEC> gn[4], en[4];
+    const int cn = c + STEP;
+    if (cn < cend) fetch(cn, gn, en);       // next column group in flight before this one is stored
+    float q[VEC * RP];
+    load_contig_ro<VEC * RP>(Q + (size_t)c * RP, q);
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+      if (a < nr) {
+        Pack<VEC> mv;
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) mv.v[k] = g[a].v[k] + e[a].v[k];
+        st_default<VEC>(E + (size_t)(r0 + a) * m + c, mv);
+#pragma unroll
+        for (int k = 0; k < VEC; ++k)
+#pragma unroll
+          for (int j = 0; j < RP; ++j) acc[a * RP + j] = fmaf(mv.v[k], q[k * RP + j], acc[a * RP + j]);
+      }
+    }
+#pragma unroll
+    for (int a = 0; a < 4; ++a) { g[a] = gn[a]; e[a] = en[a]; }
+  }
+
+  constexpr int N = 4 * RP;
+  warp_transpose_reduce<N, 16>(acc, lane);
+  float* Pp = L.Ppart + ((size_t)tl.worker * L.ncc + tl.part) * (size_t)L.n * RP;
+  if constexpr (N >= 32) {
+    constexpr int PER = N / 32;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+      const int idx = lane * PER + i;
+      const int a = idx / RP, j = idx % RP;
+      if (a < nr) Pp[(size_t)(r0 + a) * RP + j] = acc[i];
+    }
+  } else {
+    constexpr int DUP = 32 / N;
+    const int idx = lane / DUP;
+    const int a = idx / RP, j = idx % RP;
+    if ((lane % DUP) == 0 && a < nr) Pp[(size_t)(r0 + a) * RP + j] = acc[0];
+  }
+}
+
+template <int RP>
+__global__ void __launch_bounds__(kPassThreads, (RP <= 8 ? 2 : 1))
+pass1_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
+  for (int i = blockIdx.x; i < ntiles; i += gridDim.x) {
+    const Tile tl = tiles[i];
+    if (t.layers[tl.layer].vec) pass1_tile<RP, 4>(t, tl);
+    else pass1_tile<RP, 1>(t, tl);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Column-owner mapping shared by pass 2 and pass 3: a tile is nrows x up to 128*VEC columns.
+// Thread = (row group g, vector column cv); groups interleave the tile's rows.
+// ---------------------------------------------------------------------------------------
+struct ColMap {
+  int cwv, cw, ng, g, cv;
+  bool active;
+};
+
+template <int VEC>
+__device__ __forceinline__ ColMap col_map(const Tile& tl) {
+  ColMap cm;
+  cm.cwv = (tl.ncols + VEC - 1) / VEC;       // vector columns in the tile (<= 128)
+  cm.cw = (cm.cwv + 31) & ~31;                // rounded to whole warps
+  cm.ng = kPassThreads / cm.cw;               // row groups
+  cm.g = threadIdx.x / cm.cw;
+  cm.cv = threadIdx.x % cm.cw;
+  cm.active = cm.g < cm.ng && cm.cv < cm.cwv;
+  return cm;
+}
+
+// ---------------------------------------------------------------------------------------
+// pass 2: partial Q = M^T P_bar (Alg. 1, second product).  Each thread owns VEC columns and
+// accumulates VEC x RP sums over its group's rows; P_bar rows are warp-uniform loads.
+// Row groups are then summed through shared memory in group order.
+// ---------------------------------------------------------------------------------------
+template <int RP, int VEC>
+__device__ __forceinline__ void pass2_tile(const Tables& t, const Tile& tl, float* red) {
+  const LayerDev& L = t.layers[tl.layer];
+  const int m = L.m;
+  const float* __restrict__ M = L.E + (size_t)tl.worker * L.n * m;
+  const float* __restrict__ Pbar = L.Pbar;
+  const ColMap cm = col_map<VEC>(tl);
+  const int col = tl.col0 + cm.cv * VEC;
+  const int rend = tl.row0 + tl.nrows;
+
+  float acc[VEC * RP];
+#pragma unroll
+  for (int i = 0; i < VEC * RP; ++i) acc[i] = 0.f;
+
+  if (cm.active) {
+    constexpr int U = 8;
+    int i = tl.row0 + cm.g;
+    for (; i + (U - 1) * cm.ng < rend; i += U * cm.ng) {
+      Pack<VEC> mv[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) mv[u] = ld_l2<VEC>(M + (size_t)(i + u * cm.ng) * m + col);
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        float p[RP];
+        load_contig_ro<RP>(Pbar + (size_t)(i + u * cm.ng) * RP, p);
+#pragma unroll
+        for (int k = 0; k < VEC; ++k)
+#pragma unroll
+          for (int j = 0; j < RP; ++j) acc[k * RP + j] = fmaf(mv[u].v[k], p[j], acc[k * RP + j]);
+      }
+    }
+    for (; i < rend; i += cm.ng) {
+      const Pack<VEC> mv = ld_l2<VEC>(M + (size_t)i * m + col);
+      float p[RP];
+      load_contig_ro<RP>(Pbar + (size_t)i * RP, p);
+#pragma unroll
+      for (int k = 0; k < VEC; ++k)
+#pragma unroll
+        for (int j = 0; j < RP; ++j) acc[k * RP + j] = fmaf(mv.v[k], p[j], acc[k * RP + j]);
+    }
+  }
+  // fixed-order sum over the row groups: group gg hands its sums to group 0
+  for (int gg = 1; gg < cm.ng; ++gg) {
+    __syncthreads();
+    if (cm.active && cm.g == gg) {
+#pragma unroll
+      for (int k = 0; k < VEC * RP; ++k) red[k * cm.cw + cm.cv] = acc[k];
+    }
+    __syncthreads();
+    if (cm.active && cm.g == 0) {
+#pragma unroll
+      for (int k = 0; k < VEC * RP; ++k) acc[k] += red[k * cm.cw + cm.cv];
+    }
+  }
+  if (cm.active && cm.g == 0) {
+    float* dst = L.Qpart + (((size_t)tl.worker * L.nrb + tl.part) * (size_t)m + col) * RP;
+    store_contig<VEC * RP>(dst, acc);
+  }
+  __syncthreads();   // red is reused by the next tile
+}
+
+template <int RP>
+__global__ void __launch_bounds__(kPassThreads, (RP <= 8 ? 2 : 1))
+pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
+  __shared__ float red[128 * 4 * RP];
+  for (int i = blockIdx.x; i < ntiles; i += gridDim.x) {
+    const Tile tl = tiles[i];
+    if (t.layers[tl.layer].vec) pass2_tile<RP, 4>(t, tl, red);
+    else pass2_tile<RP, 1>(t, tl, red);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// pass 3: G_hat = P_bar Q_bar^T (Eq. 6) once per layer, E_w = M_w - G_hat (Eq. 7) per worker.
+// Each thread keeps its VEC rows of Q_bar in registers, forms G_hat for 4 rows at a time and
+// walks the workers with the next worker's M already in flight.
+// ---------------------------------------------------------------------------------------
+template <int RP, int VEC>
+__device__ __forceinline__ void pass3_tile(const Tables& t, const Tile& tl) {
+  const LayerDev& L = t.layers[tl.layer];
+  const int m = L.m, W = t.W;
+  const size_t plane = (size_t)L.n * m;
+  float* __restrict__ E = L.E;
+  float* __restrict__ Gh = t.ghat[tl.layer];
+  const float* __restrict__ Pbar = L.Pbar;
+  const ColMap cm = col_map<VEC>(tl);
+  if (!cm.active) return;
+  const int col = tl.col0 + cm.cv * VEC;
+  const int rend = tl.row0 + tl.nrows;
+
+  float q[VEC * RP];
+  load_contig_ro<VEC * RP>(L.Q + (size_t)col * RP, q);
+
+  constexpr int RB = 4;
+  const int rstep = RB * cm.ng;
+  auto fetch = [&](int i0, int w, Pack<VEC>(&mv)[RB]) {
+#pragma unroll
+    for (int u = 0; u < RB; ++u) {
+      const int i = i0 + u * cm.ng;
+      if (i < rend) mv[u] = ld_stream<VEC>(E + (size_t)w * plane + (size_t)i * m + col);
+    }
+  };
+  int i0 = tl.row0 + cm.g;
+  Pack<VEC> cur[RB];
+  if (i0 < rend) fetch(i0, 0, cur);
+  for (; i0 < rend; i0 += rstep) {
+    Pack<VEC> gh[RB];
+#pragma unroll
+    for (int u = 0; u < RB; ++u) {
+      const int i = i0 + u * cm.ng;
+      if (i < rend) {
+        float p[RP];
+        load_contig_ro<RP>(Pbar + (size_t)i * RP, p);
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) {
+          float s = 0.f;
+#pragma unroll
+          for (int j = 0; j < RP; ++j) s = fmaf(p[j], q[k * RP + j], s);
+          gh[u].v[k] = s;
+        }
+        st_stream<VEC>(Gh + (size_t)i * m + col, gh[u]);
+      }
+    }
+    for (int w = 0; w < W; ++w) {
+      Pack<VEC> nxt[RB];
+      if (w + 1 < W) fetch(i0, w + 1, nxt);
+      else if (i0 + rstep < rend) fetch(i0 + rstep, 0, nxt);
+#pragma unroll
+      for (int u = 0; u < RB; ++u) {
+        const int i = i0 + u * cm.ng;
+        if (i < rend) {
+          Pack<VEC> ev;
+#pragma unroll
+          for (int k = 0; k < VEC; ++k) ev.v[k] = cur[u].v[k] - gh[u].v[k];
+          st_stream<VEC>(E + (size_t)w * plane + (size_t)i * m + col, ev);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < RB; ++u) cur[u] = nxt[u];
+    }
+  }
+}
+
+template <int RP>
+__global__ void __launch_bounds__(kPassThreads, (RP <= 8 ? 2 : 1))
+pass3_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
+  for (int i = blockIdx.x; i < ntiles; i += gridDim.x) {
+    const Tile tl = tiles[i];
+    if (t.layers[tl.layer].vec) pass3_tile<RP, 4>(t, tl);
+    else pass3_tile<RP, 1>(t, tl);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Orthonormalize (Alg. 1) as CholeskyQR with the r x r part in fp64:
+//   p_reduce_gram: P_raw = sum of the column-chunk partials (fixed order); per-block Gram
+//   p_cholesky   : Gram = sum of block Grams; R^T R = Gram; R^-1
+//   p_apply      : P = P_raw R^-1 (fp64 accumulate, stored fp32); block max |P|
+// The result is the thin-QR Q factor with positive-diagonal R, the same matrix Gram-Schmidt
+// produces.  A column whose pivot is <= 1e-10 of its squared norm (or zero, or not a number)
+// becomes a zero column and the layer's status word says so.
+// ---------------------------------------------------------------------------------------
+constexpr double kPivotEps = 1e-10;
+
+template <int RP>
+__global__ void __launch_bounds__(256)
+p_reduce_gram_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
+  __shared__ float rows[kFactorBlockRows][RP];
+  const FactorBlock fb = fbs[blockIdx.x];
+  const LayerDev& L = t.layers[fb.layer];
+  const int n = L.n;
+  const int tid = threadIdx.x;
+  if (tid < kFactorBlockRows) {
+    const int row = fb.blk * kFactorBlockRows + tid;
+    float p[RP];
+#pragma unroll
+    for (int j = 0; j < RP; ++j) p[j] = 0.f;
+    if (row < n) {
+      const float* src = L.Ppart + ((size_t)fb.worker * L.ncc * n + row) * RP;
+      for (int cc = 0; cc < L.ncc; ++cc) {
+        float v[RP];
+        load_contig_ro<RP>(src + (size_t)cc * n * RP, v);
+#pragma unroll
+        for (int j = 0; j < RP; ++j) p[j] += v[j];
+      }
+      if (L.ncc > 1) store_contig<RP>(L.Praw + ((size_t)fb.worker * n + row) * RP, p);
+    }
+#pragma unroll
+    for (int j = 0; j < RP; ++j) rows[tid][j] = p[j];
+  }
+  __syncthreads();
+  if (tid < RP * RP) {
+    const int i = tid / RP, j = tid % RP;
+    double s = 0.0;
+    for (int k = 0; k < kFactorBlockRows; ++k) s = fma((double)rows[k][i], (double)rows[k][j], s);
+    L.gram_part[((size_t)fb.worker * L.npb + fb.blk) * (RP * RP) + tid] = s;
+  }
+}
+
+template <int RP>
+__global__ void __launch_bounds__(256)
+p_cholesky_kernel(Tables t) {
+  __shared__ double A[RP][RP + 1];     // Gram, overwritten by L (lower triangle)
+  __shared__ double X[RP][RP + 1];     // X[c][i] = (L^-1)[i][c]
+  __shared__ double diag0[RP];
+  __shared__ int dead[RP];
+  const int layer = blockIdx.x / t.W, worker = blockIdx.x % t.W;
+  const LayerDev& L = t.layers[layer];
+  const int r = L.r, tid = threadIdx.x;
+  if (tid < RP * RP) {
+    const double* gp = L.gram_part + (size_t)worker * L.npb * (RP * RP) + tid;
+    double s = 0.0;
+    for (int b = 0; b < L.npb; ++b) s += gp[(size_t)b * (RP * RP)];
+    A[tid / RP][tid % RP] = s;
+    X[tid / RP][tid % RP] = 0.0;
+  }
+  __syncthreads();
+  if (tid < RP) { diag0[tid] = A[tid][tid]; dead[tid] = 0; }
+  __syncthreads();
+  if (tid < 32) {
+    const int i = tid;               // lane = row of L
+    for (int j = 0; j < r; ++j) {
+      const double d = A[j][j];
+      __syncwarp();                  // every lane has read the pivot before lane j overwrites it
+      const bool ok = (d > kPivotEps * diag0[j]) && (d < INFINITY);   // false for nan too
+      double lij = 0.0;
+      if (ok) {
+        const double ljj = sqrt(d);
+        if (i == j) A[j][j] = ljj;
+        if (i > j && i < r) { lij = A[i][j] / ljj; A[i][j] = lij; }
+      } else {
+        if (i == j) { A[j][j] = 1.0; dead[j] = 1; }
+        if (i > j && i < r) A[i][j] = 0.0;
+      }
+      __syncwarp();
+      if (ok && i > j && i < r)
+        for (int k = j + 1; k <= i; ++k) A[i][k] -= lij * A[k][j];
+      __syncwarp();
+    }
+    // column c of L^-1 by forward substitution; a dead row or column stays zero
+    const int c = tid;
+    if (c < r) {
+      for (int row = c; row < r; ++row) {
+        double x = 0.0;
+        if (!dead[row]) {
+          double s = (row == c) ? 1.0 : 0.0;
+          for (int k = c; k < row; ++k) s -= A[row][k] * X[c][k];
+          x = s / A[row][row];
+        }
+        if (dead[c]) x = 0.0;
+        X[c][row] = x;
+      }
+    }
+  }
+  __syncthreads();
+  if (tid < RP * RP) {
+    const int k = tid / RP, j = tid % RP;       // R^-1[k][j] = (L^-1)[j][k], k <= j < r
+    L.rinv[(size_t)worker * (RP * RP) + tid] = (k <= j && j < r) ? X[k][j] : 0.0;
+  }
+  if (tid == 0) {
+    int any = 0;
+    for (int j = 0; j < r; ++j) any |= dead[j];
+    if (any) atomicOr(&t.status[layer], 1u);
+  }
+}
+
+__device__ __forceinline__ float block_max_128(float v, float* sm) {
+  // max over a 128-thread block; NaN compares false and is dropped (reported separately)
+#pragma unroll
+  for (int o = 16; o >= 1; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  if ((threadIdx.x & 31) == 0) sm[threadIdx.x >> 5] = v;
+  __syncthreads();
+  return fmaxf(fmaxf(sm[0], sm[1]), fmaxf(sm[2], sm[3]));
+}
+
+template <int RP>
+__global__ void __launch_bounds__(kFactorBlockRows)
+p_apply_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
+  __shared__ double Rinv[RP * RP];
+  __shared__ float smax[4];
+  const FactorBlock fb = fbs[blockIdx.x];
+  const LayerDev& L = t.layers[fb.layer];
+  const int n = L.n, tid = threadIdx.x;
+  for (int k = tid; k < RP * RP; k += kFactorBlockRows) Rinv[k] = L.rinv[(size_t)fb.worker * (RP * RP) + k];
+  __syncthreads();
+  const int row = fb.blk * kFactorBlockRows + tid;
+  float amax = 0.f;
+  if (row < n) {
+    float p[RP];
+    load_contig_ro<RP>(L.Praw + ((size_t)fb.worker * n + row) * RP, p);
+    float o[RP];
+    bool bad = false;
+#pragma unroll
+    for (int j = 0; j < RP; ++j) {
+      double s = 0.0;
+#pragma unroll
+      for (int k = 0; k <= j; ++k) s = fma((double)p[k], Rinv[k * RP + j], s);
+      o[j] = (float)s;
+      amax = fmaxf(amax, fabsf(o[j]));
+      bad |= !(fabsf(o[j]) < INFINITY);
+    }
+    store_contig<RP>(L.P + ((size_t)fb.worker * n + row) * RP, o);
+    if (bad) atomicOr(&t.status[fb.layer], 8u);
+  }
+  amax = block_max_128(amax, smax);
+  if (tid == 0) L.maxp[(size_t)fb.worker * L.npb + fb.blk] = amax;
+}
+
+// Q_w = sum of the row-chunk partials of pass 2, in chunk order; block max |Q_w|.
+template <int RP>
+__global__ void __launch_bounds__(kFactorBlockRows)
+q_reduce_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
+  __shared__ float smax[4];
+  const FactorBlock fb = fbs[blockIdx.x];
+  const LayerDev& L = t.layers[fb.layer];
+  const int m = L.m, tid = threadIdx.x;
+  const int row = fb.blk * kFactorBlockRows + tid;
+  float amax = 0.f;
+  if (row < m) {
+    float q[RP];
+#pragma unroll
+    for (int j = 0; j < RP; ++j) q[j] = 0.f;
+    const float* src = L.Qpart + ((size_t)fb.worker * L.nrb * m + row) * RP;
+    for (int rb = 0; rb < L.nrb; ++rb) {
+      float v[RP];
+      load_contig_ro<RP>(src + (size_t)rb * m * RP, v);
+#pragma unroll
+      for (int j = 0; j < RP; ++j) q[j] += v[j];
+    }
+    if (L.nrb > 1) store_contig<RP>(L.Qw + ((size_t)fb.worker * m + row) * RP, q);
+    bool bad = false;
+#pragma unroll
+    for (int j = 0; j < RP; ++j) {
+      amax = fmaxf(amax, fabsf(q[j]));
+      bad |= !(fabsf(q[j]) < INFINITY);
+    }
+    if (bad) atomicOr(&t.status[fb.layer], 8u);
+  }
+  amax = block_max_128(amax, smax);
+  if (tid == 0) L.maxq[(size_t)fb.worker * L.nqb + fb.blk] = amax;
+}
+
+// ---------------------------------------------------------------------------------------
+// Factor exchange (Alg. 1: LogQuantize, All-Reduce, LogDequantize) for one chunk of 1024
+// factor elements of one layer, all W workers:
+//   s      = max |x| over the layer's block maxima (shared scale)
+//   code_w = sign bit | k,  k = number of thresholds <= |x_w| / s        (Eq. 4, nearest level)
+//   stream = little-endian b-bit packing of code_w into worker w's payload
+//   S      = sum_w (+-k_w)   exact integer;   x_bar = s * deq[S]          (Eq. 1, Eq. 5)
+// The threshold table holds, for every level boundary, the smallest fp32 not below the exact
+// boundary, so "t >= thr" decides exactly like the real-number comparison.
+// ---------------------------------------------------------------------------------------
+template <int RP>
+__global__ void __launch_bounds__(256)
+exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __restrict__ chunks) {
+  __shared__ float thr[128];
+  __shared__ uint8_t codes[kExchangeChunk];
+  __shared__ float sred[8];
+  const ExchangeChunk ch = chunks[blockIdx.x];
+  const LayerDev& L = t.layers[ch.layer];
+  const int W = t.W, tid = threadIdx.x, b = qt.bits;
+  const int nlev = 1 << (b - 1);
+  const int rows = which ? L.m : L.n, r = L.r;
+  const int count = rows * r;
+  const int nblk = which ? L.nqb : L.npb;
+  const float* maxes = which ? L.maxq : L.maxp;
+  const float* src = which ? L.Qw : L.P;              // [W][rows][RP]
+  float* dst = which ? L.Q : L.Pbar;                  // [rows][RP]
+  uint8_t* ucodes = which ? L.codesQ : L.codesP;      // [W][count]
+  const uint64_t pay_off = which ? L.pay_q_off : L.pay_p_off;
+
+  for (int i = tid; i < nlev - 1; i += 256) thr[i] = qt.thr[i];
+  float s = 0.f;
+  for (int i = tid; i < W * nblk; i += 256) s = fmaxf(s, maxes[i]);
+#pragma unroll
+  for (int o = 16; o >= 1; o >>= 1) s = fmaxf(s, __shfl_xor_sync(0xffffffffu, s, o));
+  if ((tid & 31) == 0) sred[tid >> 5] = s;
+  __syncthreads();
+  s = sred[0];
+#pragma unroll
+  for (int i = 1; i < 8; ++i) s = fmaxf(s, sred[i]);
+  const bool s_ok = (s > 0.f) && (s < INFINITY);
+
+  const int e0 = ch.chunk * kExchangeChunk;
+  const int cnt = min(kExchangeChunk, count - e0);
+  int S[4] = {0, 0, 0, 0};
+  const size_t nbytes_total = ((size_t)count * b + 7) / 8;
+  const size_t byte0 = (size_t)ch.chunk * (kExchangeChunk / 8) * b;
+  const int nbytes = (int)min((size_t)(kExchangeChunk / 8) * b, nbytes_total - byte0);
+
+  for (int w = 0; w < W; ++w) {
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int le = tid + u * 256;
+      if (le < cnt) {
+        const int e = e0 + le;
+        const float x = src[((size_t)w * rows + e / r) * RP + (e % r)];
+        int k = 0;
+        if (s_ok) {
+          const float tt = __fdiv_rn(fabsf(x), s);
+          int lo = 0, hi = nlev - 1;                 // k = #{i : tt >= thr[i]}, thr ascending
+          while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if (tt >= thr[mid]) lo = mid + 1; else hi = mid;
+          }
+          k = lo;
+        }
+        const int neg = (x < 0.f) ? 1 : 0;
+        const uint8_t code = (uint8_t)((neg << (b - 1)) | k);
+        codes[le] = code;
+        ucodes[(size_t)w * count + e] = code;
+        S[u] += neg ? -k : k;
+      }
+    }
+    __syncthreads();
+    uint8_t* pay = t.payload + (size_t)w * t.payload_stride + pay_off + byte0;
+    for (int jb = tid; jb < nbytes; jb += 256) {
+      const int bit0 = jb * 8;
+      const int elo = bit0 / b;
+      const int ehi = min((bit0 + 7) / b, cnt - 1);
+      unsigned v = 0;
+      for (int e = elo; e <= ehi; ++e) {
+        const int sh = e * b - bit0;
+        const unsigned c = codes[e];
+        v |= (sh >= 0) ? (c << sh) : (c >> (-sh));
+      }
+      pay[jb] = (uint8_t)(v & 0xffu);
+    }
+    __syncthreads();
+  }
+
+  const int center = W * (nlev - 1);
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    const int le = tid + u * 256;
+    if (le < cnt) {
+      const int e = e0 + le;
+      const float v = s_ok ? s * qt.deq[S[u] + center] : 0.f;
+      dst[(size_t)(e / r) * RP + (e % r)] = v;
+    }
+  }
+  if (ch.chunk == 0 && tid == 0) {
+    L.scales[which] = s;
+    for (int w = 0; w < W; ++w) {
+      float* ps = reinterpret_cast<float*>(t.payload + (size_t)w * t.payload_stride + L.pay_scale_off);
+      ps[which] = s;
+    }
+    if (!(s > 0.f)) atomicOr(&t.status[ch.layer], which ? 4u : 2u);
+    if (!(s < INFINITY)) atomicOr(&t.status[ch.layer], 8u);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// 1-D tensors: mean over the workers (Eq. 1) in worker order, and the raw fp32 values into
+// each worker's payload.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+vectors_kernel(const VectorDev* __restrict__ vecs, const ExchangeChunk* __restrict__ chunks,
+               const float* const* __restrict__ vgrads, float* const* __restrict__ vghat,
+               uint8_t* payload, uint64_t payload_stride, int W) {
+  const ExchangeChunk ch = chunks[blockIdx.x];
+  const VectorDev v = vecs[ch.layer];
+  const int i = ch.chunk * 256 + threadIdx.x;
+  if (i >= v.len) return;
+  float s = 0.f;
+  for (int w = 0; w < W; ++w) {
+    const float x = vgrads[(size_t)ch.layer * W + w][i];
+    reinterpret_cast<float*>(payload + (size_t)w * payload_stride + v.pay_off)[i] = x;
+    s += x;
+  }
+  vghat[ch.layer][i] = s / (float)W;
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------
+// host launchers: dispatch on the padded rank RP in {1, 2, 4, 8, 16}
+// ---------------------------------------------------------------------------------------
+#define LQSGD_DISPATCH_RP(RPV, ...)                 \
+  switch (RPV) {                                    \
+    case 1: { constexpr int RP = 1; __VA_ARGS__; } break;   \
+    case 2: { constexpr int RP = 2; __VA_ARGS__; } break;   \
+    case 4: { constexpr int RP = 4; __VA_ARGS__; } break;   \
+    case 8: { constexpr int RP = 8; __VA_ARGS__; } break;   \
+    case 16: { constexpr int RP = 16; __VA_ARGS__; } break; \
+    default: return cudaErrorInvalidValue;          \
+  }
+
+cudaError_t launch_pass1(int rp, const Tables& t, const Tile* tiles, int ntiles, Launch l) {
+  if (ntiles == 0) return cudaSuccess;
+  LQSGD_DISPATCH_RP(rp, (pass1_kernel<RP><<<l.grid, kPassThreads, 0, l.stream>>>(t, tiles, ntiles)));
+  return cudaGetLastError();
+}
+
+cudaError_t launch_pass2(int rp, const Tables& t, const Tile* tiles, int ntiles, Launch l) {
+  if (ntiles == 0) return cudaSuccess;
+  LQSGD_DISPATCH_RP(rp, (pass2_kernel<RP><<<l.grid, kPassThreads, 0, l.stream>>>(t, tiles, ntiles)));
+  return cudaGetLastError();
+}
+
+cudaError_t launch_pass3(int rp, const Tables& t, const Tile* tiles, int ntiles, Launch l) {
+  if (ntiles == 0) return cudaSuccess;
+  LQSGD_DISPATCH_RP(rp, (pass3_kernel<RP><<<l.grid, kPassThreads, 0, l.stream>>>(t, tiles, ntiles)));
+  return cudaGetLastError();
+}
+
+cudaError_t launch_p_reduce_gram(int rp, const Tables& t, const FactorBlock* fb, int nfb, Launch l) {
+  if (nfb == 0) return cudaSuccess;
+  LQSGD_DISPATCH_RP(rp, (p_reduce_gram_kernel<RP><<<nfb, 256, 0, l.stream>>>(t, fb)));
+  return cudaGetLastError();
+}
+
+cudaError_t launch_p_cholesky(int rp, const Tables& t, int n_mat, Launch l) {
+  if (n_mat == 0) return cudaSuccess;
+  LQSGD_DISPATCH_RP(rp, (p_cholesky_kernel<RP><<<n_mat * t.W, 256, 0, l.stream>>>(t)));
+  return cudaGetLastError();
+}
+
+cudaError_t launch_p_apply(int rp, const Tables& t, const FactorBlock* fb, int nfb, Launch l) {
+  if (nfb == 0) return cudaSuccess;
+  LQSGD_DISPATCH_RP(rp, (p_apply_kernel<RP><<<nfb, kFactorBlockRows, 0, l.stream>>>(t, fb)));
+  return cudaGetLastError();
+}
+
+cudaError_t launch_q_reduce(int rp, const Tables& t, const FactorBlock* fb, int nfb, Launch l) {
+  if (nfb == 0) return cudaSuccess;
+  LQSGD_DISPATCH_RP(rp, (q_reduce_kernel<RP><<<nfb, kFactorBlockRows, 0, l.stream>>>(t, fb)));
+  return cudaGetLastError();
+}
+
+cudaError_t launch_exchange(int rp, int which, const Tables& t, const QuantTables& q,
+                            const ExchangeChunk* ch, int nch, Launch l) {
+  if (nch == 0) return cudaSuccess;
+  LQSGD_DISPATCH_RP(rp, (exchange_kernel<RP><<<nch, 256, 0, l.stream>>>(t, q, which, ch)));
+  return cudaGetLastError();
+}
+
+cudaError_t launch_vectors(const VectorDev* vecs, const ExchangeChunk* chunks, int nchunks,
+                           const float* const* vgrads, float* const* vghat, uint8_t* payload,
+                           uint64_t payload_stride, int W, Launch l) {
+  if (nchunks == 0) return cudaSuccess;
+  vectors_kernel<<<nchunks, 256, 0, l.stream>>>(vecs, chunks, vgrads, vghat, payload, payload_stride, W);
+  return cudaGetLastError();
+}
+
+cudaError_t pass_occupancy(int rp, int* occ1, int* occ2, int* occ3) {
+  cudaError_t e = cudaSuccess;
+  LQSGD_DISPATCH_RP(rp, {
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(occ1, pass1_kernel<RP>, kPassThreads, 0);
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(occ2, pass2_kernel<RP>, kPassThreads, 0);
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(occ3, pass3_kernel<RP>, kPassThreads, 0);
+  });
+  return e;
+}
+
+}  // namespace lqsgd

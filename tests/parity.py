@@ -1,0 +1,169 @@
+"""Helpers of the GPU parity tests: run one step through the C ABI and compare every stage with
+the CPU oracle on bit-identical fp32 inputs.
+
+Because the quantiser is discontinuous, comparison is stage-isolated: every oracle stage is fed
+the device's own fp32 output of the previous stage, so a stage's error is its own.  The
+free-running comparison adopts the device's code for the (rare, counted) elements whose
+companded value lies next to a decision threshold.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from oracle import lqsgd_oracle as orc
+from paper_2506_17974_b200 import binding as B
+
+TOL = 1e-4          # relative Frobenius error allowed on P, Q, G_hat, E
+MAX_FLIP_FRACTION = 1e-5
+
+
+def rel_fro(a, b):
+    a = np.asarray(a, dtype=np.float64)
+    b = np.asarray(b, dtype=np.float64)
+    nb = np.linalg.norm(b)
+    return float(np.linalg.norm(a - b) / nb) if nb > 0 else float(np.linalg.norm(a - b))
+
+
+def host(t: torch.Tensor) -> np.ndarray:
+    return t.detach().cpu().numpy()
+
+
+class StepRecord:
+    """Everything one device step produced for one matrix layer, on the host."""
+
+    def __init__(self, comp: B.LQSGD, layer: int, E_prev, Q_prev, ghat):
+        W = comp.W
+        g = lambda which, w=0: host(comp.get_state(which, layer, w))
+        self.E_prev, self.Q_prev = E_prev, Q_prev
+        self.P_raw = np.stack([g(B.STATE_P_RAW, w) for w in range(W)])
+        self.P = np.stack([g(B.STATE_P, w) for w in range(W)])
+        self.codes_p = [g(B.STATE_CODES_P, w) for w in range(W)]
+        self.P_bar = g(B.STATE_P_BAR)
+        self.Qw = np.stack([g(B.STATE_Q_W, w) for w in range(W)])
+        self.codes_q = [g(B.STATE_CODES_Q, w) for w in range(W)]
+        self.Q_bar = g(B.STATE_Q)
+        self.scales = g(B.STATE_SCALES)
+        self.E_new = np.stack([g(B.STATE_E, w) for w in range(W)])
+        self.G_hat = host(ghat)
+
+
+def snapshot_state(comp: B.LQSGD):
+    """E (per worker) and Q of every matrix layer, before a step."""
+    E, Q = {}, {}
+    for l in range(len(comp.layers)):
+        if comp.is_matrix(l):
+            E[l] = np.stack([host(comp.get_state(B.STATE_E, l, w)) for w in range(comp.W)])
+            Q[l] = host(comp.get_state(B.STATE_Q, l))
+    return E, Q
+
+
+def check_exchange(x_dev, codes_dev, scale_dev, bar_dev, bits, alpha, stats):
+    """Scale, codes and dequantised mean of one factor against the oracle, on the device's factor."""
+    s = orc.factor_scale(list(x_dev))
+    assert np.float32(scale_dev) == s, (scale_dev, s)
+    flips = 0
+    total = 0
+    for w in range(len(x_dev)):
+        c, margin = orc.log_quantize(x_dev[w], s, bits, alpha, return_margin=True)
+        bad = c != codes_dev[w]
+        if bad.any():
+            # a legitimate difference sits on a threshold (within fp32 resolution of |x|/s)
+            assert np.all(margin[bad] < 1e-4), ("codes differ away from a threshold", margin[bad].max())
+            k_o = c[bad].astype(int) & ((1 << (bits - 1)) - 1)
+            k_d = codes_dev[w][bad].astype(int) & ((1 << (bits - 1)) - 1)
+            assert np.all(np.abs(k_o - k_d) <= 1)
+        flips += int(bad.sum())
+        total += c.size
+    stats["flips"] = stats.get("flips", 0) + flips
+    stats["codes"] = stats.get("codes", 0) + total
+    mean = orc.average_dequantize(codes_dev, s, bits, alpha)       # from the device's codes
+    assert rel_fro(bar_dev, mean) <= 1e-6
+    return s
+
+
+def check_layer_stage_isolated(comp: B.LQSGD, layer: int, G, rec: StepRecord, stats):
+    """G: [W, n, m] fp32 host array of this step's gradients."""
+    W = comp.W
+    M = [orc.error_feedback(G[w], rec.E_prev[w]) for w in range(W)]
+    errs = {}
+    errs["P_raw"] = max(rel_fro(rec.P_raw[w], orc.power_step_p(M[w], rec.Q_prev)) for w in range(W))
+    orth = [orc.orthonormalize(rec.P_raw[w]) for w in range(W)]
+    errs["P"] = max(rel_fro(rec.P[w], orth[w][0]) for w in range(W))
+    check_exchange(rec.P, rec.codes_p, rec.scales[0], rec.P_bar, comp.bits_p, comp.alpha, stats)
+    errs["Qw"] = max(rel_fro(rec.Qw[w], orc.power_step_q(M[w], rec.P_bar)) for w in range(W))
+    check_exchange(rec.Qw, rec.codes_q, rec.scales[1], rec.Q_bar, comp.bits_q, comp.alpha, stats)
+    G_hat = orc.reconstruct(rec.P_bar, rec.Q_bar)
+    errs["G_hat"] = rel_fro(rec.G_hat, G_hat)
+    errs["E"] = max(rel_fro(rec.E_new[w], orc.error_update(M[w], G_hat)) for w in range(W))
+    for k, v in errs.items():
+        assert v <= TOL, (layer, k, v)
+        stats[k] = max(stats.get(k, 0.0), v)
+    return errs
+
+
+def expected_payload(comp: B.LQSGD, recs, grads_host, worker: int) -> np.ndarray:
+    """The worker's payload rebuilt by the oracle's packer from the device's codes and scales."""
+    mats = [l for l in range(len(comp.layers)) if comp.is_matrix(l)]
+    vecs = [l for l in range(len(comp.layers)) if not comp.is_matrix(l)]
+    return orc.assemble_payload(
+        comp.layers, comp.rank, comp.bits_p, comp.bits_q,
+        [(recs[l].scales[0], recs[l].scales[1]) for l in mats],
+        [recs[l].codes_p[worker] for l in mats], [recs[l].codes_q[worker] for l in mats],
+        [grads_host[worker][l] for l in vecs])
+
+
+def device_step_checked(comp: B.LQSGD, grads_dev, stats, check_payload=True):
+    """Runs one step on the device and checks every layer stage by stage.  Returns the records
+    (matrix layers) and the host copies of the gradients."""
+    E_prev, Q_prev = snapshot_state(comp)
+    ghat = [torch.empty_like(g) for g in grads_dev[0]]
+    comp.step(grads_dev, ghat)
+    torch.cuda.synchronize()
+    grads_host = [[host(g) for g in per] for per in grads_dev]
+    recs = {}
+    for l in range(len(comp.layers)):
+        if comp.is_matrix(l):
+            recs[l] = StepRecord(comp, l, E_prev[l], Q_prev[l], ghat[l])
+            G = np.stack([grads_host[w][l] for w in range(comp.W)])
+            check_layer_stage_isolated(comp, l, G, recs[l], stats)
+        else:
+            V = np.stack([grads_host[w][l].reshape(-1) for w in range(comp.W)])
+            want = orc.vector_mean(V)
+            got = host(ghat[l]).reshape(-1)
+            assert np.max(np.abs(got - want)) <= 1e-6 * max(np.max(np.abs(want)), 1e-30) + 1e-12
+    if check_payload:
+        for w in range(comp.W):
+            want = expected_payload(comp, recs, grads_host, w)
+            got = host(comp.payload(w))
+            assert got.size == comp.payload_nbytes == want.size == orc.payload_bytes(
+                comp.layers, comp.rank, comp.bits_p, comp.bits_q)
+            assert np.array_equal(got, want), f"payload bytes of worker {w} differ"
+    return recs, grads_host, ghat
+
+
+def oracle_step_forced(oracle: orc.Oracle, grads_host, recs, stats):
+    """Free-running oracle step that adopts the device's code where its own differs (counted).
+    Returns the oracle's per-layer results."""
+    forced = {}
+    for l, rec in recs.items():
+        n, m = oracle.layers[l]
+        Gl = np.stack([np.asarray(grads_host[w][l], dtype=np.float32).reshape(n, m) for w in range(oracle.W)])
+        args = (Gl, oracle.E[l], oracle.Q[l], oracle.bits_p, oracle.bits_q, oracle.alpha)
+        res = orc.layer_round(*args)
+        fp = []
+        for w in range(oracle.W):
+            diff = res["xp"]["codes"][w] != rec.codes_p[w]
+            stats["forced"] = stats.get("forced", 0) + int(diff.sum())
+            assert np.all(res["xp"]["margin"][w][diff] < 2e-2), "P code differs far from a threshold"
+            fp.append(np.where(diff, rec.codes_p[w].astype(np.int16), -1))
+        res = orc.layer_round(*args, forced_p=fp)
+        fq = []
+        for w in range(oracle.W):
+            diff = res["xq"]["codes"][w] != rec.codes_q[w]
+            stats["forced"] = stats.get("forced", 0) + int(diff.sum())
+            assert np.all(res["xq"]["margin"][w][diff] < 2e-2), "Q code differs far from a threshold"
+            fq.append(np.where(diff, rec.codes_q[w].astype(np.int16), -1))
+        forced[l] = (fp, fq)
+        stats["free_codes"] = stats.get("free_codes", 0) + sum(c.size for c in rec.codes_p + rec.codes_q)
+    return oracle.step(grads_host, forced=forced)

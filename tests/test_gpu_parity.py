@@ -1,0 +1,241 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, element by element,
+on the same seeded inputs.  Tolerances: relative Frobenius error <= 1e-4 on P, Q, G_hat and E;
+codes bit-exact except elements on a decision threshold, whose fraction (<= 1e-5) is counted;
+payload bytes exact."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import lqsgd_oracle as orc
+from paper_2506_17974_b200 import binding as B
+from paper_2506_17974_b200 import workloads as wl
+import parity as par
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def make(w: wl.Workload, **kw):
+    return B.LQSGD(w.layers, w.rank, kw.pop("bits_p", w.bits), kw.pop("bits_q", None), alpha=w.alpha,
+                   workers=w.workers, seed=w.seed, **kw)
+
+
+def new_oracle(comp: B.LQSGD):
+    Q0 = {l: par.host(comp.get_state(B.STATE_Q, l)) for l in range(len(comp.layers)) if comp.is_matrix(l)}
+    return orc.Oracle(comp.layers, comp.rank, comp.bits_p, comp.bits_q, comp.alpha, comp.W, Q0)
+
+
+def run_steps(w: wl.Workload, steps: int, free_run=True, comp=None):
+    comp = comp or make(w)
+    stats = {}
+    oracle = new_oracle(comp) if free_run else None
+    for t in range(steps):
+        grads = wl.draw_gradients(w, t, device=DEV)
+        recs, grads_host, ghat = par.device_step_checked(comp, grads, stats)
+        assert all(f == 0 for f in comp.status()), comp.status()
+        if free_run:
+            out = par.oracle_step_forced(oracle, grads_host, recs, stats)
+            for l, rec in recs.items():
+                assert par.rel_fro(rec.G_hat, out[l]["G_hat"]) <= par.TOL, (t, l)
+                assert par.rel_fro(rec.E_new, out[l]["E_new"]) <= par.TOL, (t, l)
+                assert par.rel_fro(rec.Q_bar, out[l]["Q_bar"]) <= par.TOL, (t, l)
+                assert par.rel_fro(rec.P_bar, out[l]["P_bar"]) <= par.TOL, (t, l)
+    assert stats["flips"] <= max(1, par.MAX_FLIP_FRACTION * stats["codes"]), stats
+    if free_run:
+        assert stats.get("forced", 0) <= max(2, 2e-3 * stats["free_codes"]), stats
+    print({k: (f"{v:.2e}" if isinstance(v, float) else v) for k, v in stats.items()})
+    return comp, stats
+
+
+def test_config1_single_matrix_ten_steps():
+    run_steps(wl.config1(), 10)
+
+
+def test_config2_mnist_cnn_four_workers():
+    run_steps(wl.config2(), 6)
+
+
+def test_config3_resnet18_eight_workers():
+    run_steps(wl.config3(), 2)
+
+
+@pytest.mark.parametrize("rows,cols", [(1024, 4096), (4096, 4096)])
+def test_config4_large_layers(rows, cols):
+    run_steps(wl.config4(rows, cols), 2)
+
+
+@pytest.mark.parametrize("rank,bits", [(1, 2), (2, 3), (4, 4), (8, 8), (16, 8), (16, 2)])
+def test_config5_rank_bit_points(rank, bits):
+    w = dataclasses.replace(wl.config5(rank, bits), workers=4)      # full shapes, fewer workers
+    run_steps(w, 1, free_run=False)
+
+
+def test_config5_sixteen_workers():
+    run_steps(wl.config5(2, 4), 1, free_run=False)
+
+
+@pytest.mark.parametrize("shape", [(2, 2), (3, 5), (5, 3), (17, 33), (33, 17), (40, 129), (130, 36), (64, 27), (10, 512)])
+@pytest.mark.parametrize("rank,bits,W", [(1, 2, 1), (3, 3, 2), (7, 5, 3), (16, 8, 2)])
+def test_small_and_ragged_shapes(shape, rank, bits, W):
+    w = wl.Workload("tiny", (shape, (7, 1), (1, 5)), rank=rank, bits=bits, workers=W, steps=3,
+                    dist="normal", scale="fan_in", seed=shape[0] * 1000 + shape[1])
+    comp = make(w)
+    stats = {}
+    oracle = new_oracle(comp)
+    for t in range(3):
+        grads = wl.draw_gradients(w, t, device=DEV)
+        recs, gh, _ = par.device_step_checked(comp, grads, stats)
+        out = par.oracle_step_forced(oracle, gh, recs, stats)
+        for l, rec in recs.items():
+            assert par.rel_fro(rec.G_hat, out[l]["G_hat"]) <= par.TOL
+            assert par.rel_fro(rec.E_new, out[l]["E_new"]) <= par.TOL
+
+
+def test_different_bits_for_p_and_q():
+    w = wl.Workload("bpq", ((96, 200), (48, 1)), rank=4, bits=3, workers=2, steps=2, dist="student_t3", scale="fan_in")
+    comp = make(w, bits_p=3, bits_q=6)
+    stats = {}
+    for t in range(2):
+        par.device_step_checked(comp, wl.draw_gradients(w, t, device=DEV), stats)
+    assert comp.payload_nbytes == (96 * 4 * 3 + 7) // 8 + (200 * 4 * 6 + 7) // 8 + 8 + 4 * 48
+
+
+def test_full_size_largest_layer_properties():
+    """8192 x 25088 (the largest sweep size) in the launch configuration the benchmark times:
+    products and factors against the oracle's matmuls, E and G_hat through identities and samples."""
+    w = wl.config4(8192, 25088)
+    comp = make(w)
+    g = wl.draw_gradients(w, 0, device=DEV)
+    ghat = [torch.empty_like(g[0][0])]
+    Q0 = par.host(comp.get_state(B.STATE_Q, 0)).astype(np.float64)
+    comp.step(g, ghat)
+    torch.cuda.synchronize()
+    G = par.host(g[0][0])
+    P_raw = par.host(comp.get_state(B.STATE_P_RAW, 0, 0))
+    assert par.rel_fro(P_raw, G.astype(np.float64) @ Q0) <= par.TOL          # E_0 = 0: M = G
+    P = par.host(comp.get_state(B.STATE_P, 0, 0))
+    assert par.rel_fro(P, orc.orthonormalize(P_raw)[0]) <= par.TOL
+    stats = {}
+    sc = par.host(comp.get_state(B.STATE_SCALES, 0))
+    P_bar = par.host(comp.get_state(B.STATE_P_BAR, 0))
+    par.check_exchange(P[None], [par.host(comp.get_state(B.STATE_CODES_P, 0, 0))], sc[0], P_bar, w.bits, w.alpha, stats)
+    Qw = par.host(comp.get_state(B.STATE_Q_W, 0, 0))
+    assert par.rel_fro(Qw, G.astype(np.float64).T @ P_bar.astype(np.float64)) <= par.TOL
+    Q_bar = par.host(comp.get_state(B.STATE_Q, 0))
+    par.check_exchange(Qw[None], [par.host(comp.get_state(B.STATE_CODES_Q, 0, 0))], sc[1], Q_bar, w.bits, w.alpha, stats)
+    assert stats["flips"] <= 1
+    # sampled rows of G_hat and E against the definitions (Eq. 6, Eq. 7)
+    rows = np.random.default_rng(0).choice(8192, size=64, replace=False)
+    gh_rows = ghat[0][torch.as_tensor(rows, device=DEV)].cpu().numpy()
+    E_rows = comp.get_state(B.STATE_E, 0, 0)[torch.as_tensor(rows, device=DEV)].cpu().numpy()
+    want = P_bar[rows].astype(np.float64) @ Q_bar.astype(np.float64).T
+    assert par.rel_fro(gh_rows, want) <= par.TOL
+    assert par.rel_fro(E_rows, G[rows].astype(np.float64) - want) <= par.TOL
+    # at any size: E + G_hat = G (fp32 rounding only), on the device
+    resid = (comp.get_state(B.STATE_E, 0, 0) + ghat[0] - g[0][0]).abs().max().item()
+    assert resid <= 4e-7 * g[0][0].abs().max().item()
+
+
+def test_zero_gradient_sets_status_and_zero_outputs():
+    layers = ((40, 64), (16, 1))
+    comp = B.LQSGD(layers, 3, 4, workers=2)
+    grads = [[torch.zeros(s, device=DEV) for s in layers] for _ in range(2)]
+    ghat = [torch.full(s, 7.0, device=DEV) for s in layers]
+    comp.step(grads, ghat)
+    torch.cuda.synchronize()
+    st = comp.status()
+    assert st[0] & B.STATUS_DEPENDENT_COLUMN and st[0] & B.STATUS_ZERO_SCALE_P and st[0] & B.STATUS_ZERO_SCALE_Q
+    assert st[1] == 0
+    assert all(float(g.abs().max()) == 0.0 for g in ghat)
+    assert float(comp.get_state(B.STATE_E, 0, 1).abs().max()) == 0.0
+    assert int(comp.get_state(B.STATE_CODES_P, 0, 0).max()) == 0
+    # oracle agrees: dependent columns, zero scale, zero result
+    res = orc.layer_round(np.zeros((2, 40, 64), np.float32), np.zeros((2, 40, 64)), np.ones((64, 3)), 4, 4, 127.0)
+    assert res["dependent"].all() and np.all(res["G_hat"] == 0)
+
+
+def test_dependent_column_matches_oracle():
+    """Q with two identical columns: the second column of M Q is dependent and becomes zero."""
+    layers = ((48, 80),)
+    comp = B.LQSGD(layers, 3, 4, workers=1)
+    Q = torch.randn(80, 3, generator=torch.Generator().manual_seed(3))
+    Q[:, 1] = Q[:, 0]
+    comp.set_state(B.STATE_Q, 0, 0, Q)
+    w = wl.Workload("dep", layers, rank=3, bits=4, workers=1, steps=1, dist="normal", scale="fan_in")
+    stats = {}
+    recs, _, _ = par.device_step_checked(comp, wl.draw_gradients(w, 0, device=DEV), stats)
+    assert comp.status()[0] & B.STATUS_DEPENDENT_COLUMN
+    assert np.all(recs[0].P[0][:, 1] == 0)
+
+
+def test_bit_reproducible_and_checkpoint_resume():
+    w = dataclasses.replace(wl.config2(), workers=3)
+    a, b = make(w), make(w)
+    gh = lambda: [torch.empty(s, device=DEV) for s in w.layers]
+    oa, ob = gh(), gh()
+    for t in range(4):
+        g = wl.draw_gradients(w, t, device=DEV)
+        a.step(g, oa)
+        b.step(g, ob)
+    torch.cuda.synchronize()
+    for x, y in zip(oa, ob):
+        assert torch.equal(x, y)
+    for wk in range(3):
+        assert torch.equal(a.payload(wk), b.payload(wk))
+    # resume: copy E and Q of `a` after 4 steps into a fresh context, then both take step 4
+    c = make(w)
+    for l in range(len(w.layers)):
+        if c.is_matrix(l):
+            c.set_state(B.STATE_Q, l, 0, a.get_state(B.STATE_Q, l))
+            for wk in range(3):
+                c.set_state(B.STATE_E, l, wk, a.get_state(B.STATE_E, l, wk))
+    g = wl.draw_gradients(w, 4, device=DEV)
+    oc = gh()
+    a.step(g, oa)
+    c.step(g, oc)
+    torch.cuda.synchronize()
+    for x, y in zip(oa, oc):
+        assert torch.equal(x, y)
+    assert torch.equal(a.payload(1), c.payload(1))
+    assert torch.equal(a.get_state(B.STATE_E, 2, 2), c.get_state(B.STATE_E, 2, 2))
+
+
+def test_step_host_matches_device_step():
+    w = dataclasses.replace(wl.config2(), workers=2)
+    a, b = make(w), make(w, host_staging=True)
+    g = wl.draw_gradients(w, 0, device=DEV)
+    out_a = [torch.empty(s, device=DEV) for s in w.layers]
+    a.step(g, out_a)
+    g_host = [[t.cpu().pin_memory() for t in per] for per in g]
+    out_b = [torch.empty(s).pin_memory() for s in w.layers]
+    pay = torch.empty(2 * b.payload_nbytes, dtype=torch.uint8).pin_memory()
+    b.step_host(g_host, out_b, pay)
+    torch.cuda.synchronize()
+    for x, y in zip(out_a, out_b):
+        assert torch.equal(x.cpu(), y)
+    assert torch.equal(torch.cat([a.payload(0), a.payload(1)]).cpu(), pay)
+    with pytest.raises(B.LqsgdError) as e:
+        a.step_host(g_host, out_b, pay)
+    assert e.value.code == B.ERR_NO_STAGING
+
+
+def test_argument_errors_launch_nothing():
+    layers = ((32, 64),)
+    comp = B.LQSGD(layers, 2, 4)
+    g = torch.zeros(32 * 64 + 1, device=DEV)
+    ok = g[:32 * 64].view(32, 64)
+    off = g[1:].view(32, 64)                       # 4-byte aligned only
+    out = torch.empty(32, 64, device=DEV)
+    with pytest.raises(B.LqsgdError) as e:
+        comp.step([[off]], [out])
+    assert e.value.code == B.ERR_MISALIGNED
+    with pytest.raises(B.LqsgdError) as e:
+        comp.get_state(B.STATE_E, 3, 0)
+    assert e.value.code == B.ERR_OUT_OF_RANGE
+    with pytest.raises(B.LqsgdError) as e:
+        comp.get_state(B.STATE_E, 0, 5)
+    assert e.value.code == B.ERR_OUT_OF_RANGE
+    comp.step([[ok]], [out])                       # still usable afterwards
+    torch.cuda.synchronize()
