@@ -1,0 +1,324 @@
+#!/usr/bin/env python
+"""Throughput of one LQ-SGD compression round on synthetic gradient sets.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+One "step" is one full round (Algorithm 1 body: error feedback, both power steps,
+orthonormalisation, quantise / pack / average / dequantise of P and Q, reconstruction, error
+update) over one gradient set.  The metric is GB/s of fp32 gradient processed:
+4 bytes x W workers x all gradient elements / step time.  Prints ONE JSON line on rank 0.
+
+--impl ours       the CUDA library through its C ABI (device-resident inputs for `value`,
+                  host buffers through lqsgd_step_host for `e2e`).
+--impl reference  the CPU oracle as it stands, on the host cores, on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import dataclasses
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "LQ-SGD compress+decompress GB/s of fp32 gradient"
+UNIT = "GB/s"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def get_workload(name: str):
+    from paper_2506_17974_b200 import workloads as wl
+    if name == "resnet18":
+        return wl.config3(), "resnet18_cifar W=8 r=2 b=4 (ResNet-18 gradient set, Student-t nu=3)"
+    if name == "mnist":
+        return wl.config2(), "mnist_cnn W=4 r=4 b=4"
+    if name == "single":
+        return wl.config1(), "single 256x576 W=1 r=2 b=4"
+    if name.startswith("large_"):
+        a, b = name[len("large_"):].split("x")
+        return wl.config4(int(a), int(b)), f"large layer {a}x{b} W=1 r=8 b=4, N(0, 0.01^2)"
+    raise SystemExit(f"unknown workload {name}")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def __exit__(self, *exc):
+        if self.proc:
+            self.proc.terminate()          # the exact child started above
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+            self.thread.join(timeout=2)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def phase_bytes(wl_obj):
+    """Algorithmic HBM bytes one launch of each streaming pass moves (three-pass streaming with M
+    kept in place of E): pass 1 reads G and E and writes M, pass 2 reads M, pass 3 reads M,
+    writes E per worker and G_hat once per layer."""
+    from paper_2506_17974_b200 import workloads as wl
+    W = wl_obj.workers
+    nm = wl.matrix_elements(wl_obj.layers)
+    return {"pass1": 12 * W * nm, "pass2": 4 * W * nm, "pass3": 8 * W * nm + 4 * nm}
+
+
+def time_oracle(wl_obj, budget_s: float, max_steps: int):
+    """Runs the CPU oracle on whole rounds of the workload until about budget_s has passed."""
+    import numpy as np
+    import torch
+    from oracle import lqsgd_oracle as orc
+    from paper_2506_17974_b200 import workloads as wl
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    rng = np.random.default_rng(0)
+    Q0 = {li: rng.standard_normal((m, min(wl_obj.rank, n, m)))
+          for li, (n, m) in enumerate(wl_obj.layers) if wl.is_matrix((n, m))}
+    o = orc.Oracle(wl_obj.layers, wl_obj.rank, wl_obj.bits, wl_obj.bits, wl_obj.alpha, wl_obj.workers, Q0)
+    grads = [[t.numpy() for t in per] for per in wl.draw_gradients(wl_obj, 0, device="cpu")]
+    times = []
+    t_all = time.perf_counter()
+    while len(times) < max_steps and (not times or time.perf_counter() - t_all < budget_s):
+        t0 = time.perf_counter()
+        o.step(grads)
+        times.append(time.perf_counter() - t0)
+    return times, cores
+
+
+def gradient_bytes(wl_obj):
+    return 4 * wl_obj.workers * sum(n * m for n, m in wl_obj.layers)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl_obj, desc = get_workload(args.workload)
+    times, cores = time_oracle(wl_obj, budget_s=1e9, max_steps=args.warmup + args.steps)
+    timed = times[args.warmup:] or times
+    t = sum(timed) / len(timed)
+    value = gradient_bytes(wl_obj) / t / 1e9
+    sample = f"{len(timed)} whole rounds of the workload (all layers, all W workers), numpy fp64"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": len(timed), "warmup": args.warmup, "ms_per_step": 1e3 * t, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": desc},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import __graft_entry__ as entry
+    from paper_2506_17974_b200 import binding as B
+    from paper_2506_17974_b200 import workloads as wl
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py --impl ours needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    if rank == 0:
+        entry.build()
+    if world > 1:
+        dist.barrier()
+    peak, peak_kind = load_peaks()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def bench_workload(wl_obj, steps, warmup, nsets, want_e2e, sample_clocks):
+        comp = B.LQSGD(wl_obj.layers, wl_obj.rank, wl_obj.bits, alpha=wl_obj.alpha, workers=wl_obj.workers,
+                       seed=wl_obj.seed + rank, device=dev)
+        seeded = dataclasses.replace(wl_obj, seed=wl_obj.seed + 1000 * rank)
+        sets = [wl.draw_gradients(seeded, t, device=dev) for t in range(nsets)]
+        ghat = [torch.empty_like(g) for g in sets[0][0]]
+        ptrs = [comp.make_pointer_arrays(s, ghat) for s in sets]
+        stream = torch.cuda.current_stream()
+        for t in range(warmup):
+            comp.step_ptrs(*ptrs[t % nsets], stream)
+        events = [[torch.cuda.Event(enable_timing=True) for _ in range(B.N_PHASES + 1)] for _ in range(steps)]
+        barrier()
+        sampler = ClockSampler(local) if sample_clocks else None
+        if sampler:
+            sampler.__enter__()
+            time.sleep(0.15)
+        barrier()
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        start.record(stream)
+        for t in range(steps):
+            comp.set_phase_events(events[t])
+            comp.step_ptrs(*ptrs[(warmup + t) % nsets], stream)
+        stop.record(stream)
+        barrier()
+        if sampler:
+            sampler.__exit__(None, None, None)
+        ms = start.elapsed_time(stop) / steps
+        phases = [sum(events[t][i].elapsed_time(events[t][i + 1]) for t in range(steps)) / steps
+                  for i in range(B.N_PHASES)]
+        status = comp.status()
+        assert all(s == 0 for s in status), f"device status flags set: {status}"
+        out = {"ms": ms, "phases_ms": dict(zip(B.PHASE_NAMES, phases)), "launches": comp.launches_per_step,
+               "payload": comp.payload_nbytes, "clocks": sampler.summary() if sampler else None}
+        del comp
+        if want_e2e:
+            comp = B.LQSGD(wl_obj.layers, wl_obj.rank, wl_obj.bits, alpha=wl_obj.alpha, workers=wl_obj.workers,
+                           seed=wl_obj.seed + rank, host_staging=True, device=dev)
+            hg = [[t.cpu().pin_memory() for t in per] for per in sets[0]]
+            hh = [torch.empty(t.shape).pin_memory() for t in ghat]
+            hp = torch.empty(wl_obj.workers * comp.payload_nbytes, dtype=torch.uint8).pin_memory()
+            e2e_steps = max(1, min(steps, 5))
+            comp.step_host(hg, hh, hp)
+            barrier()
+            t0 = time.perf_counter()
+            for _ in range(e2e_steps):
+                comp.step_host(hg, hh, hp)            # synchronises its stream before returning
+            torch.cuda.synchronize()
+            out["e2e_ms"] = 1e3 * (time.perf_counter() - t0) / e2e_steps
+            out["h2d"] = gradient_bytes(wl_obj)
+            out["d2h"] = 4 * sum(n * m for n, m in wl_obj.layers) + wl_obj.workers * comp.payload_nbytes
+            del comp
+        del sets, ghat
+        torch.cuda.empty_cache()
+        return out
+
+    wl_obj, desc = get_workload(args.workload)
+    gbytes = gradient_bytes(wl_obj)
+    res = bench_workload(wl_obj, args.steps, args.warmup, nsets=3, want_e2e=True, sample_clocks=True)
+
+    def allmax(x):
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    ms = allmax(res["ms"])
+    e2e_ms = allmax(res["e2e_ms"])
+    value = world * gbytes / (ms * 1e-3) / 1e9
+    pb = phase_bytes(wl_obj)
+    dom = max(("pass1", "pass2", "pass3"), key=lambda k: res["phases_ms"][k])
+    achieved = pb[dom] / (res["phases_ms"][dom] * 1e-3) / 1e9
+    round_bytes = sum(pb.values())
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": desc, "l2": "inputs larger than L2: each step streams a different "
+                   f"gradient set ({gbytes / 1e6:.0f} MB) plus the error buffers; 3 sets rotate",
+                   "rank": wl_obj.rank, "bits": wl_obj.bits, "workers": wl_obj.workers, "alpha": wl_obj.alpha,
+                   "parallelism": f"{world} independent replica(s), one per GPU, no collective"},
+        "gpu_launches": args.steps * res["launches"],
+        "clocks": res["clocks"],
+        "e2e": {"value": world * gbytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
+                "h2d_bytes_per_step": res["h2d"], "d2h_bytes_per_step": res["d2h"], "ms_per_step": e2e_ms},
+        "roofline": {"bound": "hbm", "kernel": f"{dom}_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "bytes_per_launch": pb[dom], "kernel_ms": res["phases_ms"][dom]},
+        "round": {"algorithmic_bytes": round_bytes, "achieved_gbs": round_bytes / (ms * 1e-3) / 1e9,
+                  "frac_of_peak": round_bytes / (ms * 1e-3) / 1e9 / peak, "phases_ms": res["phases_ms"]},
+        "compression_ratio": 4 * sum(n * m for n, m in wl_obj.layers) / res["payload"],
+        "payload_bytes_per_worker": res["payload"],
+    }
+    if rank == 0 and world == 1 and not args.no_sweep:
+        sweep = {}
+        for a, b in wl.CONFIG4_SIZES:
+            w4 = wl.config4(a, b)
+            r4 = bench_workload(w4, steps=10, warmup=3, nsets=2 if a * b > 5e7 else 3, want_e2e=False,
+                                sample_clocks=False)
+            rb = sum(phase_bytes(w4).values())
+            sweep[f"{a}x{b}"] = {"gbs_gradient": gradient_bytes(w4) / (r4["ms"] * 1e-3) / 1e9, "ms_per_step": r4["ms"],
+                                 "round_frac_of_peak": rb / (r4["ms"] * 1e-3) / 1e9 / peak,
+                                 "phases_ms": r4["phases_ms"]}
+        line["large_layer_sweep"] = sweep
+    if rank == 0 and world == 1:
+        times, cores = time_oracle(wl_obj, budget_s=12.0, max_steps=8)
+        t = sum(times) / len(times)
+        line["cpu_baseline"] = {"value": gbytes / t / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "sample": f"{len(times)} whole rounds of the same workload, numpy fp64, "
+                                          f"{t:.2f} s each"}
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="resnet18")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the large-layer sweep")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -179,6 +179,15 @@ int lqsgd_set_state(lqsgd_ctx* ctx, int32_t which, int32_t layer, int32_t worker
  * synchronises cuda_stream. */
 int lqsgd_status(const lqsgd_ctx* ctx, uint32_t* host_flags, void* cuda_stream);
 
+/* Profiling aid.  host_events: LQSGD_N_PHASES + 1 cudaEvent_t handles owned by the caller (or
+ * NULL to cancel).  The NEXT lqsgd_step records them on its stream at the phase boundaries and
+ * then forgets them: event i before phase i, the last one after phase LQSGD_N_PHASES - 1.
+ * Phases: 0 = pass 1 (error feedback + M Q), 1 = orthonormalise / quantise / average P,
+ * 2 = pass 2 (M^T P_bar), 3 = quantise / average Q, 4 = pass 3 (G_hat and E).  The handles are
+ * copied before the call returns. */
+#define LQSGD_N_PHASES 5
+int lqsgd_set_phase_events(lqsgd_ctx* ctx, void* const* host_events);
+
 /* Kernel launches one lqsgd_step enqueues (for launch accounting). */
 int lqsgd_launches_per_step(const lqsgd_ctx* ctx, int32_t* host_out);
 

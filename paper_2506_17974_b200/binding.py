@@ -20,6 +20,8 @@ LIB_PATH = os.path.join(_HERE, "liblqsgd.so")
 STATE_E, STATE_Q, STATE_P_RAW, STATE_P, STATE_P_BAR, STATE_Q_W, STATE_CODES_P, STATE_CODES_Q, STATE_SCALES = range(9)
 STATUS_DEPENDENT_COLUMN, STATUS_ZERO_SCALE_P, STATUS_ZERO_SCALE_Q, STATUS_NONFINITE = 1, 2, 4, 8
 FLAG_HOST_STAGING = 1
+N_PHASES = 5
+PHASE_NAMES = ("pass1", "finish_p", "pass2", "finish_q", "pass3")
 
 ERR_INVALID_ARG, ERR_BAD_SHAPE, ERR_WORKSPACE_TOO_SMALL, ERR_MISALIGNED = -1, -2, -3, -4
 ERR_CUDA, ERR_NO_STAGING, ERR_OUT_OF_RANGE = -5, -6, -7
@@ -27,7 +29,7 @@ ERR_CUDA, ERR_NO_STAGING, ERR_OUT_OF_RANGE = -5, -6, -7
 EXPORTED = [
     "lqsgd_workspace_bytes", "lqsgd_create", "lqsgd_step", "lqsgd_step_host", "lqsgd_payload_bytes",
     "lqsgd_payload", "lqsgd_payload_layout", "lqsgd_get_state", "lqsgd_set_state", "lqsgd_status",
-    "lqsgd_launches_per_step", "lqsgd_destroy", "lqsgd_strerror", "lqsgd_last_cuda_error", "lqsgd_version",
+    "lqsgd_launches_per_step", "lqsgd_set_phase_events", "lqsgd_destroy", "lqsgd_strerror", "lqsgd_last_cuda_error", "lqsgd_version",
 ]
 
 
@@ -76,6 +78,7 @@ def load_library() -> C.CDLL:
     lib.lqsgd_set_state.argtypes = [vp, i32, i32, i32, vp, vp]
     lib.lqsgd_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
     lib.lqsgd_launches_per_step.argtypes = [vp, C.POINTER(i32)]
+    lib.lqsgd_set_phase_events.argtypes = [vp, C.POINTER(vp)]
     lib.lqsgd_destroy.argtypes = [vp]
     lib.lqsgd_destroy.restype = None
     lib.lqsgd_strerror.argtypes = [C.c_int]
@@ -181,6 +184,15 @@ class LQSGD:
     def step_ptrs(self, g_arr, h_arr, stream: Optional[torch.cuda.Stream] = None) -> None:
         s = stream if stream is not None else torch.cuda.current_stream(self.device)
         _check(self.lib.lqsgd_step(self.ctx, g_arr, h_arr, C.c_void_p(s.cuda_stream)))
+
+    def set_phase_events(self, events: Optional[Sequence[torch.cuda.Event]]) -> None:
+        """Asks the next step to record N_PHASES + 1 caller-owned CUDA events at its phase boundaries."""
+        if events is None:
+            _check(self.lib.lqsgd_set_phase_events(self.ctx, None))
+            return
+        assert len(events) == N_PHASES + 1
+        arr = (C.c_void_p * len(events))(*[e.cuda_event for e in events])
+        _check(self.lib.lqsgd_set_phase_events(self.ctx, arr))
 
     def step(self, grads, ghat, stream: Optional[torch.cuda.Stream] = None) -> None:
         """One round of Algorithm 1 on device tensors grads[w][l]; writes ghat[l]."""

@@ -310,6 +310,8 @@ struct lqsgd_ctx {
   std::vector<void*> ptrs_host;      // mirror of plan.d_ptrs
   bool ptrs_valid = false;
   void* workspace = nullptr;
+  cudaEvent_t phase_events[LQSGD_N_PHASES + 1];
+  bool have_events = false;
 };
 
 extern "C" {
@@ -420,6 +422,18 @@ int lqsgd_create(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
 
 void lqsgd_destroy(lqsgd_ctx* ctx) { delete ctx; }
 
+int lqsgd_set_phase_events(lqsgd_ctx* c, void* const* host_events) {
+  if (!c) return LQSGD_ERR_INVALID_ARG;
+  c->have_events = false;
+  if (!host_events) return LQSGD_OK;
+  for (int i = 0; i <= LQSGD_N_PHASES; ++i) {
+    if (!host_events[i]) return LQSGD_ERR_INVALID_ARG;
+    c->phase_events[i] = static_cast<cudaEvent_t>(host_events[i]);
+  }
+  c->have_events = true;
+  return LQSGD_OK;
+}
+
 int lqsgd_launches_per_step(const lqsgd_ctx* ctx, int32_t* out) {
   if (!ctx || !out) return LQSGD_ERR_INVALID_ARG;
   *out = (ctx->plan.mats.empty() ? 0 : 9) + (ctx->plan.chV.empty() ? 0 : 1);
@@ -476,24 +490,36 @@ int lqsgd_step(lqsgd_ctx* c, const float* const* grads, float* const* ghat, void
   t.W = W;
   const QuantTables qp{p.d_thrP, p.d_deqP, c->cfg.bits_p}, qq{p.d_thrQ, p.d_deqQ, c->cfg.bits_q};
   const int RP = p.RP;
-  if (nm) {
-    CK(cudaMemsetAsync(p.d_status, 0, nm * sizeof(uint32_t), st));
-    CK(launch_pass1(RP, t, p.d_tiles1, (int)p.tiles1.size(), {st, c->grid1}));
-    CK(launch_p_reduce_gram(RP, t, p.d_fbP, (int)p.fbP.size(), {st, 0}));
-    CK(launch_p_cholesky(RP, t, (int)nm, {st, 0}));
-    CK(launch_p_apply(RP, t, p.d_fbP, (int)p.fbP.size(), {st, 0}));
-    CK(launch_exchange(RP, 0, t, qp, p.d_chP, (int)p.chP.size(), {st, 0}));
-    CK(launch_pass2(RP, t, p.d_tiles2, (int)p.tiles2.size(), {st, c->grid2}));
-    CK(launch_q_reduce(RP, t, p.d_fbQ, (int)p.fbQ.size(), {st, 0}));
-    CK(launch_exchange(RP, 1, t, qq, p.d_chQ, (int)p.chQ.size(), {st, 0}));
-    CK(launch_pass3(RP, t, p.d_tiles3, (int)p.tiles3.size(), {st, c->grid3}));
-  }
+  const bool ev = c->have_events;
+  c->have_events = false;
+#define PHASE_MARK(i) do { if (ev) CK(cudaEventRecord(c->phase_events[i], st)); } while (0)
   if (nv) {
     CK(launch_vectors(p.d_vecs, p.d_chV, (int)p.chV.size(),
                       reinterpret_cast<const float* const*>(p.d_ptrs + vbase),
                       reinterpret_cast<float* const*>(p.d_ptrs + vbase + nv * W), p.d_payload,
                       p.payload_stride, W, {st, 0}));
   }
+  if (nm) CK(cudaMemsetAsync(p.d_status, 0, nm * sizeof(uint32_t), st));
+  PHASE_MARK(0);
+  if (nm) CK(launch_pass1(RP, t, p.d_tiles1, (int)p.tiles1.size(), {st, c->grid1}));
+  PHASE_MARK(1);
+  if (nm) {
+    CK(launch_p_reduce_gram(RP, t, p.d_fbP, (int)p.fbP.size(), {st, 0}));
+    CK(launch_p_cholesky(RP, t, (int)nm, {st, 0}));
+    CK(launch_p_apply(RP, t, p.d_fbP, (int)p.fbP.size(), {st, 0}));
+    CK(launch_exchange(RP, 0, t, qp, p.d_chP, (int)p.chP.size(), {st, 0}));
+  }
+  PHASE_MARK(2);
+  if (nm) CK(launch_pass2(RP, t, p.d_tiles2, (int)p.tiles2.size(), {st, c->grid2}));
+  PHASE_MARK(3);
+  if (nm) {
+    CK(launch_q_reduce(RP, t, p.d_fbQ, (int)p.fbQ.size(), {st, 0}));
+    CK(launch_exchange(RP, 1, t, qq, p.d_chQ, (int)p.chQ.size(), {st, 0}));
+  }
+  PHASE_MARK(4);
+  if (nm) CK(launch_pass3(RP, t, p.d_tiles3, (int)p.tiles3.size(), {st, c->grid3}));
+  PHASE_MARK(5);
+#undef PHASE_MARK
   return LQSGD_OK;
 }
 
