@@ -191,7 +191,10 @@ class LQSGD:
             _check(self.lib.lqsgd_set_phase_events(self.ctx, None))
             return
         assert len(events) == N_PHASES + 1
-        arr = (C.c_void_p * len(events))(*[e.cuda_event for e in events])
+        for e in events:
+            if not e.cuda_event:          # torch creates the handle lazily, on the first record
+                e.record(torch.cuda.current_stream(self.device))
+        arr =(C.c_void_p * len(events))(*[e.cuda_event for e in events])
         _check(self.lib.lqsgd_set_phase_events(self.ctx, arr))
 
     def step(self, grads, ghat, stream: Optional[torch.cuda.Stream] = None) -> None:
