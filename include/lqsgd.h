@@ -62,7 +62,8 @@ typedef enum lqsgd_error {
   LQSGD_ERR_MISALIGNED = -4,          /* workspace not 256-byte aligned, tensor pointer not aligned */
   LQSGD_ERR_CUDA = -5,                /* a CUDA runtime call failed; see lqsgd_last_cuda_error() */
   LQSGD_ERR_NO_STAGING = -6,          /* lqsgd_step_host() on a context created without LQSGD_FLAG_HOST_STAGING */
-  LQSGD_ERR_OUT_OF_RANGE = -7         /* layer / worker / state index out of range, or state not defined for that layer */
+  LQSGD_ERR_OUT_OF_RANGE = -7,        /* layer / worker / state index out of range, or state not defined for that layer */
+  LQSGD_ERR_TOO_LARGE = -8            /* size beyond the fixed built-in scratch of lqsgd_orthonormalize_noalloc */
 } lqsgd_error;
 
 /* Bits of the per-layer status word. */
@@ -190,6 +191,28 @@ int lqsgd_set_phase_events(lqsgd_ctx* ctx, void* const* host_events);
 
 /* Kernel launches one lqsgd_step enqueues (for launch accounting). */
 int lqsgd_launches_per_step(const lqsgd_ctx* ctx, int32_t* host_out);
+
+/* Orthonormalises the columns of one rows x rank factor with NO workspace and NO allocation.
+ * (The paper has no counterpart: this is a packaging of the Orthonormalize step for callers that
+ * cannot obtain device memory - every byte is owned by another allocator or a start-up budget -
+ * or may not call cudaMalloc because it stalls the device, e.g. from a serving loop or from a
+ * callback inside another library.  They pass only the input and the output.)
+ * dev_p_in: fp32, dense row-major rows x rank, 4-byte aligned, read-only.  dev_p_out: same shape,
+ * overwritten with the thin-QR Q factor (positive-diagonal R; a zero or dependent column becomes
+ * zero); may be the same pointer as dev_p_in, must not overlap it otherwise.  dev_status_out:
+ * NULL, or one device uint32 that receives LQSGD_STATUS_* bits.  Asynchronous on cuda_stream.
+ * Intermediate storage (block Gram matrices, R^-1: about 1 MiB) is a fixed array inside the
+ * library image, present once on every GPU that loads the library until the process exits:
+ *  - rows > LQSGD_NOALLOC_MAX_ROWS or rank > 16 returns LQSGD_ERR_TOO_LARGE, nothing is launched;
+ *  - all calls on a device share that array (it keeps the previous call's contents; the call
+ *    clears what must start at zero): calls that can overlap on the GPU race - order them on one
+ *    stream or with events;
+ *  - the first call on each device queries the array's device address (no allocation); make
+ *    that first call before any stream capture begins.
+ * Calls no cudaMalloc / cudaFree and no allocating library routine. */
+#define LQSGD_NOALLOC_MAX_ROWS 65536
+int lqsgd_orthonormalize_noalloc(const float* dev_p_in, float* dev_p_out, int32_t rows, int32_t rank,
+                                 uint32_t* dev_status_out, void* cuda_stream);
 
 /* Frees the host-side context.  The workspace stays the caller's. */
 void lqsgd_destroy(lqsgd_ctx* ctx);

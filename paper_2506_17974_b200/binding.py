@@ -25,10 +25,13 @@ PHASE_NAMES = ("pass1", "finish_p", "pass2", "finish_q", "pass3")
 
 ERR_INVALID_ARG, ERR_BAD_SHAPE, ERR_WORKSPACE_TOO_SMALL, ERR_MISALIGNED = -1, -2, -3, -4
 ERR_CUDA, ERR_NO_STAGING, ERR_OUT_OF_RANGE = -5, -6, -7
+ERR_TOO_LARGE = -8
+NOALLOC_MAX_ROWS = 65536
 
 EXPORTED = [
     "lqsgd_workspace_bytes", "lqsgd_create", "lqsgd_step", "lqsgd_step_host", "lqsgd_payload_bytes",
     "lqsgd_payload", "lqsgd_payload_layout", "lqsgd_get_state", "lqsgd_set_state", "lqsgd_status",
+    "lqsgd_orthonormalize_noalloc",
     "lqsgd_launches_per_step", "lqsgd_set_phase_events", "lqsgd_destroy", "lqsgd_strerror", "lqsgd_last_cuda_error", "lqsgd_version",
 ]
 
@@ -78,6 +81,7 @@ def load_library() -> C.CDLL:
     lib.lqsgd_set_state.argtypes = [vp, i32, i32, i32, vp, vp]
     lib.lqsgd_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
     lib.lqsgd_launches_per_step.argtypes = [vp, C.POINTER(i32)]
+    lib.lqsgd_orthonormalize_noalloc.argtypes = [vp, vp, i32, i32, vp, vp]
     lib.lqsgd_set_phase_events.argtypes = [vp, C.POINTER(vp)]
     lib.lqsgd_destroy.argtypes = [vp]
     lib.lqsgd_destroy.restype = None
@@ -108,6 +112,21 @@ def _shapes(layers: Sequence[Tuple[int, int]]):
 def make_config(rank: int, bits_p: int, bits_q: int, alpha: float, workers: int, seed: int = 0,
                 flags: int = 0) -> Config:
     return Config(C.sizeof(Config), rank, bits_p, bits_q, alpha, workers, seed, flags)
+
+
+def orthonormalize_noalloc(p_in: torch.Tensor, p_out: torch.Tensor, status: Optional[torch.Tensor] = None,
+                           rows: Optional[int] = None, rank: Optional[int] = None) -> None:
+    """Orthonormalises the columns of the fp32 device matrix p_in (rows x rank, contiguous) into
+    p_out without any workspace: for callers that cannot allocate device memory.  The library's
+    built-in scratch is shared by all calls on a device, so keep calls ordered on one stream.
+    `status`, if given, is a one-element int32/uint32 device tensor that receives status bits.
+    rows / rank default to p_in's shape (they can be overridden to exercise the size check)."""
+    n = p_in.shape[0] if rows is None else rows
+    r = p_in.shape[1] if rank is None else rank
+    s = torch.cuda.current_stream(p_in.device)
+    _check(load_library().lqsgd_orthonormalize_noalloc(
+        C.c_void_p(p_in.data_ptr()), C.c_void_p(p_out.data_ptr()), n, r,
+        C.c_void_p(status.data_ptr() if status is not None else 0), C.c_void_p(s.cuda_stream)))
 
 
 def workspace_bytes(layers, cfg: Config) -> int:

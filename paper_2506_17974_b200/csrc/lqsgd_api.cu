@@ -330,6 +330,7 @@ const char* lqsgd_strerror(int code) {
     case LQSGD_ERR_CUDA: return "CUDA runtime error";
     case LQSGD_ERR_NO_STAGING: return "context was created without host staging";
     case LQSGD_ERR_OUT_OF_RANGE: return "index out of range";
+    case LQSGD_ERR_TOO_LARGE: return "size exceeds the built-in scratch of the no-allocation entry point";
     default: return "unknown error";
   }
 }
