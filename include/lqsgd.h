@@ -71,9 +71,11 @@ typedef enum lqsgd_error {
 #define LQSGD_STATUS_ZERO_SCALE_P     2u /* every P entry was 0: codes and P_bar are 0 */
 #define LQSGD_STATUS_ZERO_SCALE_Q     4u /* every Q entry was 0: codes and Q_bar are 0 */
 #define LQSGD_STATUS_NONFINITE        8u /* a scale was inf or nan: the layer's outputs are undefined (no fault) */
+#define LQSGD_STATUS_TIMEOUT         16u /* a bounded device-side wait ran out: the step's outputs are undefined */
 
 /* Config flags. */
 #define LQSGD_FLAG_HOST_STAGING 1u /* reserve device staging in the workspace so that lqsgd_step_host() works */
+#define LQSGD_FLAG_REGISTER_PATH 2u /* stream every layer with the register-path kernels (no bulk-copy staging) */
 
 typedef struct lqsgd_ctx lqsgd_ctx;
 

@@ -20,6 +20,8 @@ LIB_PATH = os.path.join(_HERE, "liblqsgd.so")
 STATE_E, STATE_Q, STATE_P_RAW, STATE_P, STATE_P_BAR, STATE_Q_W, STATE_CODES_P, STATE_CODES_Q, STATE_SCALES = range(9)
 STATUS_DEPENDENT_COLUMN, STATUS_ZERO_SCALE_P, STATUS_ZERO_SCALE_Q, STATUS_NONFINITE = 1, 2, 4, 8
 FLAG_HOST_STAGING = 1
+FLAG_REGISTER_PATH = 2
+STATUS_TIMEOUT = 16
 N_PHASES = 5
 PHASE_NAMES = ("pass1", "finish_p", "pass2", "finish_q", "pass3")
 
@@ -140,7 +142,7 @@ class LQSGD:
 
     def __init__(self, layers: Sequence[Tuple[int, int]], rank: int, bits_p: int, bits_q: Optional[int] = None,
                  alpha: float = 127.0, workers: int = 1, seed: int = 0, host_staging: bool = False,
-                 device: str = "cuda:0"):
+                 device: str = "cuda:0", register_path: bool = False):
         self.lib = load_library()
         self.layers = [(int(n), int(m)) for n, m in layers]
         self.rank, self.bits_p = rank, bits_p
@@ -148,7 +150,8 @@ class LQSGD:
         self.alpha, self.W = float(alpha), workers
         self.device = torch.device(device)
         self.cfg = make_config(rank, self.bits_p, self.bits_q, alpha, workers, seed,
-                               FLAG_HOST_STAGING if host_staging else 0)
+                               (FLAG_HOST_STAGING if host_staging else 0)
+                               | (FLAG_REGISTER_PATH if register_path else 0))
         nbytes = workspace_bytes(self.layers, self.cfg)
         with torch.cuda.device(self.device):
             self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)

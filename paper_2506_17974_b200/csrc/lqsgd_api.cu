@@ -52,7 +52,8 @@ struct Plan {
   std::vector<MatHost> mats;
   std::vector<LayerDev> layers;
   std::vector<VectorDev> vecs;
-  std::vector<Tile> tiles1, tiles2, tiles3;
+  std::vector<Tile> tiles1, tiles2, tiles3;      // register-path passes
+  std::vector<Tile> stiles1, stiles2, stiles3;   // bulk-copy staged passes
   std::vector<FactorBlock> fbP, fbQ;
   std::vector<ExchangeChunk> chP, chQ, chV;
   std::vector<float> thrP, thrQ, deqP, deqQ;
@@ -64,6 +65,7 @@ struct Plan {
   LayerDev* d_layers = nullptr;
   VectorDev* d_vecs = nullptr;
   Tile *d_tiles1 = nullptr, *d_tiles2 = nullptr, *d_tiles3 = nullptr;
+  Tile *d_stiles1 = nullptr, *d_stiles2 = nullptr, *d_stiles3 = nullptr;
   FactorBlock *d_fbP = nullptr, *d_fbQ = nullptr;
   ExchangeChunk *d_chP = nullptr, *d_chQ = nullptr, *d_chV = nullptr;
   float *d_thrP = nullptr, *d_thrQ = nullptr, *d_deqP = nullptr, *d_deqQ = nullptr;
@@ -85,7 +87,7 @@ int check_config(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
   if (c->bits_p < 2 || c->bits_p > 8 || c->bits_q < 2 || c->bits_q > 8) return LQSGD_ERR_INVALID_ARG;
   if (!(c->alpha > 0.f) || !std::isfinite(c->alpha)) return LQSGD_ERR_INVALID_ARG;
   if (c->workers < 1 || c->workers > 256) return LQSGD_ERR_INVALID_ARG;
-  if (c->flags & ~LQSGD_FLAG_HOST_STAGING) return LQSGD_ERR_INVALID_ARG;
+  if (c->flags & ~(LQSGD_FLAG_HOST_STAGING | LQSGD_FLAG_REGISTER_PATH)) return LQSGD_ERR_INVALID_ARG;
   for (int i = 0; i < n_layers; ++i) {
     if (shapes[i].rows < 1 || shapes[i].cols < 1) return LQSGD_ERR_BAD_SHAPE;
     if ((int64_t)shapes[i].rows * shapes[i].cols > (int64_t)1 << 30) return LQSGD_ERR_BAD_SHAPE;
@@ -190,6 +192,36 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
     for (auto& mt : p.mats) t += (size_t)ceil_div(mt.n, balanced_rows(mt.n, r)) * colchunks(mt.m);
     return t;
   });
+  // Bulk-copy staged passes: layers with 16-byte aligned rows, RP <= 8.  Column chunks are
+  // balanced in units of 128 columns (at most 512 per tile); row chunks are multiples of 16.
+  auto staged = [&](const MatHost& mt) {
+    return !(cfg.flags & LQSGD_FLAG_REGISTER_PATH) && RP <= kStreamMaxRP && mt.m % 4 == 0;
+  };
+  auto staged_cols = [](int m) {                       // list of (col0, ncols)
+    std::vector<std::pair<int, int>> out;
+    const int units = ceil_div(m, 128), ncc = ceil_div(units, kStreamTileCols / 128);
+    int u0 = 0;
+    for (int c = 0; c < ncc; ++c) {
+      const int nu = units / ncc + (c < units % ncc ? 1 : 0);
+      out.push_back({u0 * 128, std::min(nu * 128, m - u0 * 128)});
+      u0 += nu;
+    }
+    return out;
+  };
+  auto rows16 = [&](int n, int rmax) {                  // balanced row chunk, multiple of 16
+    return (int)align_up((size_t)balanced_rows(n, rmax), kStreamStageRows);
+  };
+  const size_t want_s = 4 * (size_t)sm_count;
+  auto count_staged = [&](int rmax, bool per_worker) {
+    size_t t = 0;
+    for (auto& mt : p.mats)
+      if (staged(mt)) t += (size_t)(per_worker ? W : 1) * ceil_div(mt.n, rows16(mt.n, rmax)) * staged_cols(mt.m).size();
+    return t;
+  };
+  const int s1 = pick_size({64, 32, 16}, want_s, [&](int r) { return count_staged(r, true); });
+  const int s2 = pick_size({r2max, r2max / 2, std::max(32, r2max / 4)}, want_s, [&](int r) { return count_staged(r, true); });
+  const int s3max = std::max(16, (int)align_up((size_t)std::max(1, 64 / W), 16));
+  const int s3 = pick_size({s3max, 16}, want_s, [&](int r) { return count_staged(r, false); });
 
   // ---- carve
   Arena a(base);
@@ -202,19 +234,23 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
     LayerDev& L = p.layers[li];
     std::memset(&L, 0, sizeof(L));
     L.n = mt.n; L.m = mt.m; L.r = mt.r; L.vec = vec_of(mt.m) == 4; L.user_index = mt.user_index;
+    const bool st = staged(mt);
+    const auto scols = staged_cols(mt.m);
     const int cw = chunk_width(mt.m, c1);
-    L.ncc = ceil_div(mt.m, cw);
-    const int tr2 = balanced_rows(mt.n, r2);
+    const int tr2 = st ? rows16(mt.n, s2) : balanced_rows(mt.n, r2);
+    L.ncc = st ? (int)scols.size() : ceil_div(mt.m, cw);
     L.nrb = ceil_div(mt.n, tr2);
     L.npb = ceil_div(mt.n, kFactorBlockRows);
     L.nqb = ceil_div(mt.m, kFactorBlockRows);
     const size_t nm = (size_t)mt.n * mt.m;
     L.E = a.take<float>((size_t)W * nm);
     L.Q = a.take<float>((size_t)mt.m * RP);
+    L.mt = (int)align_up((size_t)mt.m, 4);
+    L.Qt = a.take<float>((size_t)RP * L.mt);
     L.Ppart = a.take<float>((size_t)W * L.ncc * mt.n * RP);
     L.Praw = (L.ncc == 1) ? L.Ppart : a.take<float>((size_t)W * mt.n * RP);
     L.P = a.take<float>((size_t)W * mt.n * RP);
-    L.Pbar = a.take<float>((size_t)mt.n * RP);
+    L.Pbar = a.take<float>(align_up((size_t)mt.n, kStreamStageRows) * RP);   // whole 16-row blocks for bulk copies
     L.Qpart = a.take<float>((size_t)W * L.nrb * mt.m * RP);
     L.Qw = (L.nrb == 1) ? L.Qpart : a.take<float>((size_t)W * mt.m * RP);
     L.gram_part = a.take<double>((size_t)W * L.npb * RP * RP);
@@ -229,21 +265,35 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
 
     // tiles
     const int li32 = (int)li;
-    for (int rb = 0; rb < ceil_div(mt.n, kPass1Rows); ++rb)
+    if (st) {
+      const int tr1 = rows16(mt.n, s1), tr3 = rows16(mt.n, s3);
+      for (int rb = 0; rb < ceil_div(mt.n, tr1); ++rb)
+        for (int cc = 0; cc < (int)scols.size(); ++cc)
+          for (int w = 0; w < W; ++w)
+            p.stiles1.push_back({li32, w, rb * tr1, std::min(tr1, mt.n - rb * tr1), scols[cc].first, scols[cc].second, cc, 0});
+      for (int w = 0; w < W; ++w)
+        for (int rb = 0; rb < L.nrb; ++rb)
+          for (int cc = 0; cc < (int)scols.size(); ++cc)
+            p.stiles2.push_back({li32, w, rb * tr2, std::min(tr2, mt.n - rb * tr2), scols[cc].first, scols[cc].second, rb, 0});
+      for (int rb = 0; rb < ceil_div(mt.n, tr3); ++rb)
+        for (int cc = 0; cc < (int)scols.size(); ++cc)
+          p.stiles3.push_back({li32, 0, rb * tr3, std::min(tr3, mt.n - rb * tr3), scols[cc].first, scols[cc].second, 0, 0});
+    }
+    for (int rb = 0; !st && rb < ceil_div(mt.n, kPass1Rows); ++rb)
       for (int cc = 0; cc < L.ncc; ++cc)
         for (int w = 0; w < W; ++w) {
           const int row0 = rb * kPass1Rows, col0 = cc * cw;
           p.tiles1.push_back({li32, w, row0, std::min(kPass1Rows, mt.n - row0), col0, std::min(cw, mt.m - col0), cc, 0});
         }
     const int cw2 = 128 * vec_of(mt.m);
-    for (int w = 0; w < W; ++w)
+    for (int w = 0; !st && w < W; ++w)
       for (int rb = 0; rb < L.nrb; ++rb)
         for (int cc = 0; cc < ceil_div(mt.m, cw2); ++cc) {
           const int row0 = rb * tr2, col0 = cc * cw2;
           p.tiles2.push_back({li32, w, row0, std::min(tr2, mt.n - row0), col0, std::min(cw2, mt.m - col0), rb, 0});
         }
     const int tr3 = balanced_rows(mt.n, r3);
-    for (int rb = 0; rb < ceil_div(mt.n, tr3); ++rb)
+    for (int rb = 0; !st && rb < ceil_div(mt.n, tr3); ++rb)
       for (int cc = 0; cc < ceil_div(mt.m, cw2); ++cc) {
         const int row0 = rb * tr3, col0 = cc * cw2;
         p.tiles3.push_back({li32, 0, row0, std::min(tr3, mt.n - row0), col0, std::min(cw2, mt.m - col0), 0, 0});
@@ -266,6 +316,9 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   p.d_tiles1 = a.take<Tile>(p.tiles1.size());
   p.d_tiles2 = a.take<Tile>(p.tiles2.size());
   p.d_tiles3 = a.take<Tile>(p.tiles3.size());
+  p.d_stiles1 = a.take<Tile>(p.stiles1.size());
+  p.d_stiles2 = a.take<Tile>(p.stiles2.size());
+  p.d_stiles3 = a.take<Tile>(p.stiles3.size());
   p.d_fbP = a.take<FactorBlock>(p.fbP.size());
   p.d_fbQ = a.take<FactorBlock>(p.fbQ.size());
   p.d_chP = a.take<ExchangeChunk>(p.chP.size());
@@ -390,6 +443,9 @@ int lqsgd_create(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
   CK(up(p.d_tiles1, p.tiles1.data(), p.tiles1.size() * sizeof(Tile)));
   CK(up(p.d_tiles2, p.tiles2.data(), p.tiles2.size() * sizeof(Tile)));
   CK(up(p.d_tiles3, p.tiles3.data(), p.tiles3.size() * sizeof(Tile)));
+  CK(up(p.d_stiles1, p.stiles1.data(), p.stiles1.size() * sizeof(Tile)));
+  CK(up(p.d_stiles2, p.stiles2.data(), p.stiles2.size() * sizeof(Tile)));
+  CK(up(p.d_stiles3, p.stiles3.data(), p.stiles3.size() * sizeof(Tile)));
   CK(up(p.d_fbP, p.fbP.data(), p.fbP.size() * sizeof(FactorBlock)));
   CK(up(p.d_fbQ, p.fbQ.data(), p.fbQ.size() * sizeof(FactorBlock)));
   CK(up(p.d_chP, p.chP.data(), p.chP.size() * sizeof(ExchangeChunk)));
@@ -408,6 +464,7 @@ int lqsgd_create(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
       for (int j = 0; j < mt.r; ++j)
         q0[(size_t)i * p.RP + j] = normal_draw(cfg->seed, (uint64_t)mt.user_index, (uint64_t)i * mt.r + j);
     CK(up(p.layers[li].Q, q0.data(), q0.size() * sizeof(float)));
+    CK(launch_q_transpose(p.layers[li].Q, p.layers[li].Qt, mt.m, p.RP, p.layers[li].mt, nullptr));
   }
   int o1 = 1, o2 = 1, o3 = 1;
   CK(pass_occupancy(p.RP, &o1, &o2, &o3));
@@ -437,7 +494,8 @@ int lqsgd_set_phase_events(lqsgd_ctx* c, void* const* host_events) {
 
 int lqsgd_launches_per_step(const lqsgd_ctx* ctx, int32_t* out) {
   if (!ctx || !out) return LQSGD_ERR_INVALID_ARG;
-  *out = (ctx->plan.mats.empty() ? 0 : 9) + (ctx->plan.chV.empty() ? 0 : 1);
+  const Plan& p = ctx->plan;
+  *out = (p.mats.empty() ? 0 : 6) + (p.tiles1.empty() ? 0 : 3) + (p.stiles1.empty() ? 0 : 3) + (p.chV.empty() ? 0 : 1);
   return LQSGD_OK;
 }
 
@@ -502,7 +560,10 @@ int lqsgd_step(lqsgd_ctx* c, const float* const* grads, float* const* ghat, void
   }
   if (nm) CK(cudaMemsetAsync(p.d_status, 0, nm * sizeof(uint32_t), st));
   PHASE_MARK(0);
-  if (nm) CK(launch_pass1(RP, t, p.d_tiles1, (int)p.tiles1.size(), {st, c->grid1}));
+  if (nm) {
+    CK(launch_pass1(RP, t, p.d_tiles1, (int)p.tiles1.size(), {st, c->grid1}));
+    CK(launch_stream_pass1(RP, t, p.d_stiles1, (int)p.stiles1.size(), {st, (int)std::min<size_t>(p.stiles1.size(), c->sm_count)}));
+  }
   PHASE_MARK(1);
   if (nm) {
     CK(launch_p_reduce_gram(RP, t, p.d_fbP, (int)p.fbP.size(), {st, 0}));
@@ -511,14 +572,20 @@ int lqsgd_step(lqsgd_ctx* c, const float* const* grads, float* const* ghat, void
     CK(launch_exchange(RP, 0, t, qp, p.d_chP, (int)p.chP.size(), {st, 0}));
   }
   PHASE_MARK(2);
-  if (nm) CK(launch_pass2(RP, t, p.d_tiles2, (int)p.tiles2.size(), {st, c->grid2}));
+  if (nm) {
+    CK(launch_pass2(RP, t, p.d_tiles2, (int)p.tiles2.size(), {st, c->grid2}));
+    CK(launch_stream_pass2(RP, t, p.d_stiles2, (int)p.stiles2.size(), {st, (int)std::min<size_t>(p.stiles2.size(), c->sm_count)}));
+  }
   PHASE_MARK(3);
   if (nm) {
     CK(launch_q_reduce(RP, t, p.d_fbQ, (int)p.fbQ.size(), {st, 0}));
     CK(launch_exchange(RP, 1, t, qq, p.d_chQ, (int)p.chQ.size(), {st, 0}));
   }
   PHASE_MARK(4);
-  if (nm) CK(launch_pass3(RP, t, p.d_tiles3, (int)p.tiles3.size(), {st, c->grid3}));
+  if (nm) {
+    CK(launch_pass3(RP, t, p.d_tiles3, (int)p.tiles3.size(), {st, c->grid3}));
+    CK(launch_stream_pass3(RP, t, p.d_stiles3, (int)p.stiles3.size(), {st, (int)std::min<size_t>(p.stiles3.size(), c->sm_count)}));
+  }
   PHASE_MARK(5);
 #undef PHASE_MARK
   return LQSGD_OK;
@@ -630,6 +697,11 @@ int lqsgd_set_state(lqsgd_ctx* c, int32_t which, int32_t layer, int32_t worker, 
   if (rc != LQSGD_OK) return rc;
   CK(cudaMemcpy2DAsync(base, pitch, dev_src, rb, rb, rows, cudaMemcpyDeviceToDevice,
                        static_cast<cudaStream_t>(cuda_stream)));
+  if (which == LQSGD_STATE_Q) {
+    for (const LayerDev& L : c->plan.layers)
+      if (L.user_index == layer)
+        CK(launch_q_transpose(L.Q, L.Qt, L.m, c->plan.RP, L.mt, static_cast<cudaStream_t>(cuda_stream)));
+  }
   return LQSGD_OK;
 }
 

@@ -10,7 +10,7 @@ constexpr int kMaxRank = 16;
 constexpr int kPassThreads = 256;      // threads per CTA of the three streaming passes
 constexpr int kPass1Rows = 32;         // rows per pass-1 tile: 8 warps x 4 rows
 constexpr int kFactorBlockRows = 128;  // rows of P (or Q) per block of the small factor kernels
-constexpr int kExchangeChunk = 1024;   // factor elements per block of the exchange kernel
+constexpr int kExchangeChunk = 256;    // factor elements per block of the exchange kernel
 
 // One matrix layer (n x m), as the kernels see it.  Factors are stored with a row stride of
 // RP floats (rank padded to 1, 2, 4, 8 or 16); columns >= r are kept zero.
@@ -21,9 +21,10 @@ struct LayerDev {
   int32_t nrb;                // row chunks of pass 2 (Q partial sums)
   int32_t npb, nqb;           // factor blocks: ceil(n/128), ceil(m/128)
   int32_t user_index;         // index in the caller's layer list
-  int32_t pad0;
+  int32_t mt;                 // row stride of Qt: m rounded up to a multiple of 4
   float* E;                   // [W][n][m]   error buffer; holds M between pass 1 and pass 3
   float* Q;                   // [m][RP]     warm start, becomes Q_bar
+  float* Qt;                  // [RP][mt]    transposed copy of Q read by pass 1 and pass 3
   float* Ppart;               // [W][ncc][n][RP]
   float* Praw;                // [W][n][RP]  (== Ppart when ncc == 1)
   float* P;                   // [W][n][RP]  orthonormal
@@ -94,12 +95,22 @@ cudaError_t launch_p_cholesky(int RP, const Tables& t, int n_mat, Launch l);
 cudaError_t launch_p_apply(int RP, const Tables& t, const FactorBlock* fb, int nfb, Launch l);
 cudaError_t launch_exchange(int RP, int which /*0 = P, 1 = Q*/, const Tables& t, const QuantTables& q,
                             const ExchangeChunk* ch, int nch, Launch l);
+cudaError_t launch_q_transpose(const float* Q, float* Qt, int m, int RP, int mt, cudaStream_t stream);
 cudaError_t launch_pass2(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
 cudaError_t launch_q_reduce(int RP, const Tables& t, const FactorBlock* fb, int nfb, Launch l);
 cudaError_t launch_pass3(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
 cudaError_t launch_vectors(const VectorDev* vecs, const ExchangeChunk* chunks, int nchunks,
                            const float* const* vgrads, float* const* vghat, uint8_t* payload,
                            uint64_t payload_stride, int W, Launch l);
+// Bulk-copy staged passes (lqsgd_stream.cu): layers with m % 4 == 0 and RP <= 8.  Tiles are at
+// most kStreamTileCols columns wide; pass 2 / pass 3 tiles start on a multiple of
+// kStreamStageRows rows.  One CTA per SM.
+constexpr int kStreamTileCols = 512;
+constexpr int kStreamStageRows = 16;
+constexpr int kStreamMaxRP = 8;
+cudaError_t launch_stream_pass1(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
+cudaError_t launch_stream_pass2(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
+cudaError_t launch_stream_pass3(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
 // Resident CTAs per SM of each streaming pass for this RP (for persistent grid sizing).
 cudaError_t pass_occupancy(int RP, int* occ1, int* occ2, int* occ3);
 

@@ -86,6 +86,30 @@ __device__ __forceinline__ Pack<VEC> ld_l2(const float* p) {       // keep in L2
 }
 
 template <int VEC>
+__device__ __forceinline__ Pack<VEC> ld_ro(const float* __restrict__ p) {   // read-only data, cached in L1
+  Pack<VEC> r;
+  if constexpr (VEC == 4) {
+    float4 t = __ldg(reinterpret_cast<const float4*>(p));
+    r.v[0] = t.x; r.v[1] = t.y; r.v[2] = t.z; r.v[3] = t.w;
+  } else {
+    r.v[0] = __ldg(p);
+  }
+  return r;
+}
+
+// q[k * RP + j] = Q[col + k][j] for k < VEC, read from the transposed copy Qt[j][col + k] so
+// that the lanes of a warp (consecutive columns) read consecutive addresses.
+template <int RP, int VEC>
+__device__ __forceinline__ void load_q_slice(const float* __restrict__ Qt, int mt, int col, float (&q)[VEC * RP]) {
+#pragma unroll
+  for (int j = 0; j < RP; ++j) {
+    const Pack<VEC> v = ld_ro<VEC>(Qt + (size_t)j * mt + col);
+#pragma unroll
+    for (int k = 0; k < VEC; ++k) q[k * RP + j] = v.v[k];
+  }
+}
+
+template <int VEC>
 __device__ __forceinline__ void st_default(float* p, const Pack<VEC>& x) {
   if constexpr (VEC == 4) *reinterpret_cast<float4*>(p) = make_float4(x.v[0], x.v[1], x.v[2], x.v[3]);
   else *p = x.v[0];
@@ -132,7 +156,7 @@ __device__ __forceinline__ void pass1_tile(const Tables& t, const Tile& tl) {
   const int m = L.m;
   const float* __restrict__ G = t.grads[(size_t)tl.layer * t.W + tl.worker];
   float* __restrict__ E = L.E + (size_t)tl.worker * L.n * m;
-  const float* __restrict__ Q = L.Q;
+  const float* __restrict__ Qt = L.Qt;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r0 = tl.row0 + warp * 4;
   const int nr = min(4, tl.row0 + tl.nrows - r0);   // rows this warp owns (may be <= 0)
@@ -162,7 +186,7 @@ __device__ __forceinline__ void pass1_tile(const Tables& t, const Tile& tl) {
     const int cn = c + STEP;
     if (cn < cend) fetch(cn, gn, en);       // next column group in flight before this one is stored
     float q[VEC * RP];
-    load_contig_ro<VEC * RP>(Q + (size_t)c * RP, q);
+    load_q_slice<RP, VEC>(Qt, L.mt, c, q);
 #pragma unroll
     for (int a = 0; a < 4; ++a) {
       if (a < nr) {
@@ -250,7 +274,7 @@ __device__ __forceinline__ void pass2_tile(const Tables& t, const Tile& tl, floa
   for (int i = 0; i < VEC * RP; ++i) acc[i] = 0.f;
 
   if (cm.active) {
-    constexpr int U = 8;
+    constexpr int U = (RP <= 8) ? 16 : 8;
     int i = tl.row0 + cm.g;
     for (; i + (U - 1) * cm.ng < rend; i += U * cm.ng) {
       Pack<VEC> mv[U];
@@ -326,7 +350,7 @@ __device__ __forceinline__ void pass3_tile(const Tables& t, const Tile& tl) {
   const int rend = tl.row0 + tl.nrows;
 
   float q[VEC * RP];
-  load_contig_ro<VEC * RP>(L.Q + (size_t)col * RP, q);
+  load_q_slice<RP, VEC>(L.Qt, L.mt, col, q);
 
   constexpr int RB = 4;
   const int rstep = RB * cm.ng;
@@ -578,7 +602,7 @@ q_reduce_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
 }
 
 // ---------------------------------------------------------------------------------------
-// Factor exchange (Alg. 1: LogQuantize, All-Reduce, LogDequantize) for one chunk of 1024
+// Factor exchange (Alg. 1: LogQuantize, All-Reduce, LogDequantize) for one chunk of 256
 // factor elements of one layer, all W workers:
 //   s      = max |x| over the layer's block maxima (shared scale)
 //   code_w = sign bit | k,  k = number of thresholds <= |x_w| / s        (Eq. 4, nearest level)
@@ -590,8 +614,10 @@ q_reduce_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
 template <int RP>
 __global__ void __launch_bounds__(256)
 exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __restrict__ chunks) {
+  constexpr int CH = kExchangeChunk;   // 256 factor elements per block, one per thread
+  constexpr int WB = 8;                // workers handled per round
   __shared__ float thr[128];
-  __shared__ uint8_t codes[kExchangeChunk];
+  __shared__ uint8_t codes[WB][CH];
   __shared__ float sred[8];
   const ExchangeChunk ch = chunks[blockIdx.x];
   const LayerDev& L = t.layers[ch.layer];
@@ -600,15 +626,15 @@ exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __rest
   const int rows = which ? L.m : L.n, r = L.r;
   const int count = rows * r;
   const int nblk = which ? L.nqb : L.npb;
-  const float* maxes = which ? L.maxq : L.maxp;
-  const float* src = which ? L.Qw : L.P;              // [W][rows][RP]
-  float* dst = which ? L.Q : L.Pbar;                  // [rows][RP]
-  uint8_t* ucodes = which ? L.codesQ : L.codesP;      // [W][count]
+  const float* __restrict__ maxes = which ? L.maxq : L.maxp;
+  const float* __restrict__ src = which ? L.Qw : L.P;   // [W][rows][RP]
+  float* dst = which ? L.Q : L.Pbar;                    // [rows][RP]
+  uint8_t* ucodes = which ? L.codesQ : L.codesP;        // [W][count]
   const uint64_t pay_off = which ? L.pay_q_off : L.pay_p_off;
 
   for (int i = tid; i < nlev - 1; i += 256) thr[i] = qt.thr[i];
   float s = 0.f;
-  for (int i = tid; i < W * nblk; i += 256) s = fmaxf(s, maxes[i]);
+  for (int i = tid; i < W * nblk; i += 256) s = fmaxf(s, __ldg(maxes + i));
 #pragma unroll
   for (int o = 16; o >= 1; o >>= 1) s = fmaxf(s, __shfl_xor_sync(0xffffffffu, s, o));
   if ((tid & 31) == 0) sred[tid >> 5] = s;
@@ -618,23 +644,28 @@ exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __rest
   for (int i = 1; i < 8; ++i) s = fmaxf(s, sred[i]);
   const bool s_ok = (s > 0.f) && (s < INFINITY);
 
-  const int e0 = ch.chunk * kExchangeChunk;
-  const int cnt = min(kExchangeChunk, count - e0);
-  int S[4] = {0, 0, 0, 0};
+  const int e0 = ch.chunk * CH;
+  const int cnt = min(CH, count - e0);
+  const bool valid = tid < cnt;
+  const int e = e0 + tid;
+  const int row = valid ? e / r : 0, col = valid ? e % r : 0;
   const size_t nbytes_total = ((size_t)count * b + 7) / 8;
-  const size_t byte0 = (size_t)ch.chunk * (kExchangeChunk / 8) * b;
-  const int nbytes = (int)min((size_t)(kExchangeChunk / 8) * b, nbytes_total - byte0);
+  const size_t byte0 = (size_t)ch.chunk * (CH / 8) * b;
+  const int nbytes = (int)min((size_t)(CH / 8) * b, nbytes_total - byte0);
+  int S = 0;
 
-  for (int w = 0; w < W; ++w) {
+  for (int w0 = 0; w0 < W; w0 += WB) {
+    const int wn = min(WB, W - w0);
+    float x[WB];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int le = tid + u * 256;
-      if (le < cnt) {
-        const int e = e0 + le;
-        const float x = src[((size_t)w * rows + e / r) * RP + (e % r)];
+    for (int u = 0; u < WB; ++u)
+      x[u] = (valid && u < wn) ? __ldg(src + ((size_t)(w0 + u) * rows + row) * RP + col) : 0.f;
+#pragma unroll
+    for (int u = 0; u < WB; ++u) {
+      if (u < wn) {
         int k = 0;
-        if (s_ok) {
-          const float tt = __fdiv_rn(fabsf(x), s);
+        if (s_ok && valid) {
+          const float tt = __fdiv_rn(fabsf(x[u]), s);
           int lo = 0, hi = nlev - 1;                 // k = #{i : tt >= thr[i]}, thr ascending
           while (lo < hi) {
             const int mid = (lo + hi) >> 1;
@@ -642,39 +673,34 @@ exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __rest
           }
           k = lo;
         }
-        const int neg = (x < 0.f) ? 1 : 0;
+        const int neg = (valid && x[u] < 0.f) ? 1 : 0;
         const uint8_t code = (uint8_t)((neg << (b - 1)) | k);
-        codes[le] = code;
-        ucodes[(size_t)w * count + e] = code;
-        S[u] += neg ? -k : k;
+        codes[u][tid] = code;                        // 0 beyond the factor's end: pads the last byte
+        if (valid) ucodes[(size_t)(w0 + u) * count + e] = code;
+        S += neg ? -k : k;
       }
     }
     __syncthreads();
-    uint8_t* pay = t.payload + (size_t)w * t.payload_stride + pay_off + byte0;
-    for (int jb = tid; jb < nbytes; jb += 256) {
+    for (int idx = tid; idx < wn * nbytes; idx += 256) {
+      const int u = idx / nbytes, jb = idx - u * nbytes;
       const int bit0 = jb * 8;
       const int elo = bit0 / b;
-      const int ehi = min((bit0 + 7) / b, cnt - 1);
+      const int ehi = min((bit0 + 7) / b, CH - 1);
       unsigned v = 0;
-      for (int e = elo; e <= ehi; ++e) {
-        const int sh = e * b - bit0;
-        const unsigned c = codes[e];
+      for (int q = elo; q <= ehi; ++q) {
+        const int sh = q * b - bit0;
+        const unsigned c = codes[u][q];
         v |= (sh >= 0) ? (c << sh) : (c >> (-sh));
       }
-      pay[jb] = (uint8_t)(v & 0xffu);
+      t.payload[(size_t)(w0 + u) * t.payload_stride + pay_off + byte0 + jb] = (uint8_t)(v & 0xffu);
     }
     __syncthreads();
   }
 
-  const int center = W * (nlev - 1);
-#pragma unroll
-  for (int u = 0; u < 4; ++u) {
-    const int le = tid + u * 256;
-    if (le < cnt) {
-      const int e = e0 + le;
-      const float v = s_ok ? s * qt.deq[S[u] + center] : 0.f;
-      dst[(size_t)(e / r) * RP + (e % r)] = v;
-    }
+  if (valid) {
+    const float v = s_ok ? s * __ldg(qt.deq + S + W * (nlev - 1)) : 0.f;
+    dst[(size_t)row * RP + col] = v;
+    if (which) L.Qt[(size_t)col * L.mt + row] = v;
   }
   if (ch.chunk == 0 && tid == 0) {
     L.scales[which] = s;
@@ -685,6 +711,14 @@ exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __rest
     if (!(s > 0.f)) atomicOr(&t.status[ch.layer], which ? 4u : 2u);
     if (!(s < INFINITY)) atomicOr(&t.status[ch.layer], 8u);
   }
+}
+
+// Qt[j][i] = Q[i][j]: refreshes the transposed copy after Q was set from outside.
+__global__ void __launch_bounds__(256)
+q_transpose_kernel(const float* __restrict__ Q, float* __restrict__ Qt, int m, int RP, int mt) {
+  const int i = blockIdx.x * 256 + threadIdx.x;
+  if (i >= m) return;
+  for (int j = 0; j < RP; ++j) Qt[(size_t)j * mt + i] = Q[(size_t)i * RP + j];
 }
 
 // ---------------------------------------------------------------------------------------
@@ -726,6 +760,11 @@ vectors_kernel(const VectorDev* __restrict__ vecs, const ExchangeChunk* __restri
 cudaError_t launch_pass1(int rp, const Tables& t, const Tile* tiles, int ntiles, Launch l) {
   if (ntiles == 0) return cudaSuccess;
   LQSGD_DISPATCH_RP(rp, (pass1_kernel<RP><<<l.grid, kPassThreads, 0, l.stream>>>(t, tiles, ntiles)));
+  return cudaGetLastError();
+}
+
+cudaError_t launch_q_transpose(const float* Q, float* Qt, int m, int RP, int mt, cudaStream_t stream) {
+  q_transpose_kernel<<<(m + 255) / 256, 256, 0, stream>>>(Q, Qt, m, RP, mt);
   return cudaGetLastError();
 }
 

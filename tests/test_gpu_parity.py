@@ -76,6 +76,34 @@ def test_config5_sixteen_workers():
     run_steps(wl.config5(2, 4), 1, free_run=False)
 
 
+@pytest.mark.parametrize("name", ["mnist", "resnet", "large", "rank8_workers3"])
+def test_register_path_kernels(name):
+    """The same rounds with every layer on the register-path passes (no bulk-copy staging)."""
+    w = {"mnist": wl.config2(), "resnet": dataclasses.replace(wl.config3(), workers=3),
+         "large": wl.config4(1024, 4096),
+         "rank8_workers3": dataclasses.replace(wl.config5(8, 4), workers=3)}[name]
+    run_steps(w, 2, free_run=False, comp=make(w, register_path=True))
+
+
+def test_staged_and_register_paths_agree():
+    """Both kernel families implement the same arithmetic up to summation order: M Q agrees within
+    rounding, and where the codes coincide so does everything downstream."""
+    w = dataclasses.replace(wl.config2(), workers=2)
+    a, b = make(w), make(w, register_path=True)
+    g = wl.draw_gradients(w, 0, device=DEV)
+    oa = [torch.empty(s, device=DEV) for s in w.layers]
+    ob = [torch.empty(s, device=DEV) for s in w.layers]
+    a.step(g, oa)
+    b.step(g, ob)
+    torch.cuda.synchronize()
+    for l in range(4):
+        assert par.rel_fro(par.host(a.get_state(B.STATE_P_RAW, l, 1)), par.host(b.get_state(B.STATE_P_RAW, l, 1))) <= 1e-5
+        same = all(torch.equal(a.get_state(s, l, k), b.get_state(s, l, k))
+                   for s in (B.STATE_CODES_P, B.STATE_CODES_Q) for k in range(2))
+        if same:
+            assert par.rel_fro(par.host(oa[l]), par.host(ob[l])) <= 1e-5
+
+
 @pytest.mark.parametrize("shape", [(2, 2), (3, 5), (5, 3), (17, 33), (33, 17), (40, 129), (130, 36), (64, 27), (10, 512)])
 @pytest.mark.parametrize("rank,bits,W", [(1, 2, 1), (3, 3, 2), (7, 5, 3), (16, 8, 2)])
 def test_small_and_ragged_shapes(shape, rank, bits, W):
