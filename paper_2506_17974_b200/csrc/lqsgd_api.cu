@@ -53,7 +53,7 @@ struct Plan {
   std::vector<LayerDev> layers;
   std::vector<VectorDev> vecs;
   std::vector<Tile> tiles1, tiles2, tiles3;      // register-path passes
-  std::vector<Tile> stiles1, stiles2, stiles3;   // bulk-copy staged passes
+  std::vector<Tile> stiles1, stiles3;            // bulk-copy staged passes 1 and 3
   std::vector<FactorBlock> fbP, fbQ;
   std::vector<ExchangeChunk> chP, chQ, chV;
   std::vector<float> thrP, thrQ, deqP, deqQ;
@@ -65,7 +65,7 @@ struct Plan {
   LayerDev* d_layers = nullptr;
   VectorDev* d_vecs = nullptr;
   Tile *d_tiles1 = nullptr, *d_tiles2 = nullptr, *d_tiles3 = nullptr;
-  Tile *d_stiles1 = nullptr, *d_stiles2 = nullptr, *d_stiles3 = nullptr;
+  Tile *d_stiles1 = nullptr, *d_stiles3 = nullptr;
   FactorBlock *d_fbP = nullptr, *d_fbQ = nullptr;
   ExchangeChunk *d_chP = nullptr, *d_chQ = nullptr, *d_chV = nullptr;
   float *d_thrP = nullptr, *d_thrQ = nullptr, *d_deqP = nullptr, *d_deqQ = nullptr;
@@ -192,14 +192,18 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
     for (auto& mt : p.mats) t += (size_t)ceil_div(mt.n, balanced_rows(mt.n, r)) * colchunks(mt.m);
     return t;
   });
-  // Bulk-copy staged passes: layers with 16-byte aligned rows, RP <= 8.  Column chunks are
-  // balanced in units of 128 columns (at most 512 per tile); row chunks are multiples of 16.
+  // Bulk-copy staged passes: layers with 16-byte aligned rows, RP <= 8.  A layer no wider than
+  // stream_max_cols(RP) is one column chunk (its rows are then contiguous: one copy per stage);
+  // wider layers get chunks balanced in units of 128 columns.  Row chunks hold a target number
+  // of elements and are multiples of the rows one stage takes.
   auto staged = [&](const MatHost& mt) {
     return !(cfg.flags & LQSGD_FLAG_REGISTER_PATH) && RP <= kStreamMaxRP && mt.m % 4 == 0;
   };
-  auto staged_cols = [](int m) {                       // list of (col0, ncols)
+  auto staged_cols = [&](int m) {                      // list of (col0, ncols)
     std::vector<std::pair<int, int>> out;
-    const int units = ceil_div(m, 128), ncc = ceil_div(units, kStreamTileCols / 128);
+    const int maxc = stream_max_cols(RP);
+    if (m <= maxc) { out.push_back({0, m}); return out; }
+    const int units = ceil_div(m, 128), ncc = ceil_div(units, maxc / 128);
     int u0 = 0;
     for (int c = 0; c < ncc; ++c) {
       const int nu = units / ncc + (c < units % ncc ? 1 : 0);
@@ -208,20 +212,35 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
     }
     return out;
   };
-  auto rows16 = [&](int n, int rmax) {                  // balanced row chunk, multiple of 16
-    return (int)align_up((size_t)balanced_rows(n, rmax), kStreamStageRows);
+  auto stage_rows = [&](int m) {                        // most rows a stage of this layer takes
+    int r = 1;
+    for (auto& c : staged_cols(m)) r = std::max(r, stream_geo(c.second, RP).R);
+    return r;
+  };
+  auto widest = [&](int m) {
+    int w = 0;
+    for (auto& c : staged_cols(m)) w = std::max(w, c.second);
+    return w;
+  };
+  // rows per tile: about `elems` elements, at least rmin rows, balanced over n, multiple of R
+  auto tile_rows = [&](int n, int m, size_t elems, int rmin) {
+    const int R = stage_rows(m);
+    int r = (int)std::max<size_t>(elems / (size_t)widest(m), (size_t)std::max(rmin, R));
+    r = std::min(r, n);
+    r = ceil_div(n, ceil_div(n, r));
+    return (int)align_up((size_t)r, R);
   };
   const size_t want_s = 4 * (size_t)sm_count;
-  auto count_staged = [&](int rmax, bool per_worker) {
+  auto count_staged = [&](size_t elems, int rmin, bool per_worker) {
     size_t t = 0;
     for (auto& mt : p.mats)
-      if (staged(mt)) t += (size_t)(per_worker ? W : 1) * ceil_div(mt.n, rows16(mt.n, rmax)) * staged_cols(mt.m).size();
+      if (staged(mt))
+        t += (size_t)(per_worker ? W : 1) * ceil_div(mt.n, tile_rows(mt.n, mt.m, elems, rmin)) * staged_cols(mt.m).size();
     return t;
   };
-  const int s1 = pick_size({64, 32, 16}, want_s, [&](int r) { return count_staged(r, true); });
-  const int s2 = pick_size({r2max, r2max / 2, std::max(32, r2max / 4)}, want_s, [&](int r) { return count_staged(r, true); });
-  const int s3max = std::max(16, (int)align_up((size_t)std::max(1, 64 / W), 16));
-  const int s3 = pick_size({s3max, 16}, want_s, [&](int r) { return count_staged(r, false); });
+  const size_t s1 = (size_t)pick_size({65536, 32768, 16384}, want_s, [&](int e) { return count_staged(e, 1, true); });
+  const size_t s3 = (size_t)pick_size({65536, 32768, 16384}, want_s,
+                                      [&](int e) { return count_staged(std::max(1, e / W), 1, false); }) / W;
 
   // ---- carve
   Arena a(base);
@@ -237,7 +256,7 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
     const bool st = staged(mt);
     const auto scols = staged_cols(mt.m);
     const int cw = chunk_width(mt.m, c1);
-    const int tr2 = st ? rows16(mt.n, s2) : balanced_rows(mt.n, r2);
+    const int tr2 = balanced_rows(mt.n, r2);   // pass 2 runs on the register path for every layer
     L.ncc = st ? (int)scols.size() : ceil_div(mt.m, cw);
     L.nrb = ceil_div(mt.n, tr2);
     L.npb = ceil_div(mt.n, kFactorBlockRows);
@@ -250,7 +269,7 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
     L.Ppart = a.take<float>((size_t)W * L.ncc * mt.n * RP);
     L.Praw = (L.ncc == 1) ? L.Ppart : a.take<float>((size_t)W * mt.n * RP);
     L.P = a.take<float>((size_t)W * mt.n * RP);
-    L.Pbar = a.take<float>(align_up((size_t)mt.n, kStreamStageRows) * RP);   // whole 16-row blocks for bulk copies
+    L.Pbar = a.take<float>((size_t)mt.n * RP);
     L.Qpart = a.take<float>((size_t)W * L.nrb * mt.m * RP);
     L.Qw = (L.nrb == 1) ? L.Qpart : a.take<float>((size_t)W * mt.m * RP);
     L.gram_part = a.take<double>((size_t)W * L.npb * RP * RP);
@@ -266,15 +285,11 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
     // tiles
     const int li32 = (int)li;
     if (st) {
-      const int tr1 = rows16(mt.n, s1), tr3 = rows16(mt.n, s3);
+      const int tr1 = tile_rows(mt.n, mt.m, s1, 1), tr3 = tile_rows(mt.n, mt.m, std::max<size_t>(s3, 1), 1);
       for (int rb = 0; rb < ceil_div(mt.n, tr1); ++rb)
         for (int cc = 0; cc < (int)scols.size(); ++cc)
           for (int w = 0; w < W; ++w)
             p.stiles1.push_back({li32, w, rb * tr1, std::min(tr1, mt.n - rb * tr1), scols[cc].first, scols[cc].second, cc, 0});
-      for (int w = 0; w < W; ++w)
-        for (int rb = 0; rb < L.nrb; ++rb)
-          for (int cc = 0; cc < (int)scols.size(); ++cc)
-            p.stiles2.push_back({li32, w, rb * tr2, std::min(tr2, mt.n - rb * tr2), scols[cc].first, scols[cc].second, rb, 0});
       for (int rb = 0; rb < ceil_div(mt.n, tr3); ++rb)
         for (int cc = 0; cc < (int)scols.size(); ++cc)
           p.stiles3.push_back({li32, 0, rb * tr3, std::min(tr3, mt.n - rb * tr3), scols[cc].first, scols[cc].second, 0, 0});
@@ -286,7 +301,7 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
           p.tiles1.push_back({li32, w, row0, std::min(kPass1Rows, mt.n - row0), col0, std::min(cw, mt.m - col0), cc, 0});
         }
     const int cw2 = 128 * vec_of(mt.m);
-    for (int w = 0; !st && w < W; ++w)
+    for (int w = 0; w < W; ++w)
       for (int rb = 0; rb < L.nrb; ++rb)
         for (int cc = 0; cc < ceil_div(mt.m, cw2); ++cc) {
           const int row0 = rb * tr2, col0 = cc * cw2;
@@ -317,7 +332,6 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   p.d_tiles2 = a.take<Tile>(p.tiles2.size());
   p.d_tiles3 = a.take<Tile>(p.tiles3.size());
   p.d_stiles1 = a.take<Tile>(p.stiles1.size());
-  p.d_stiles2 = a.take<Tile>(p.stiles2.size());
   p.d_stiles3 = a.take<Tile>(p.stiles3.size());
   p.d_fbP = a.take<FactorBlock>(p.fbP.size());
   p.d_fbQ = a.take<FactorBlock>(p.fbQ.size());
@@ -444,7 +458,6 @@ int lqsgd_create(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
   CK(up(p.d_tiles2, p.tiles2.data(), p.tiles2.size() * sizeof(Tile)));
   CK(up(p.d_tiles3, p.tiles3.data(), p.tiles3.size() * sizeof(Tile)));
   CK(up(p.d_stiles1, p.stiles1.data(), p.stiles1.size() * sizeof(Tile)));
-  CK(up(p.d_stiles2, p.stiles2.data(), p.stiles2.size() * sizeof(Tile)));
   CK(up(p.d_stiles3, p.stiles3.data(), p.stiles3.size() * sizeof(Tile)));
   CK(up(p.d_fbP, p.fbP.data(), p.fbP.size() * sizeof(FactorBlock)));
   CK(up(p.d_fbQ, p.fbQ.data(), p.fbQ.size() * sizeof(FactorBlock)));
@@ -469,7 +482,7 @@ int lqsgd_create(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
   int o1 = 1, o2 = 1, o3 = 1;
   CK(pass_occupancy(p.RP, &o1, &o2, &o3));
   c->grid1 = (int)std::min<size_t>(p.tiles1.size(), (size_t)c->sm_count * std::max(o1, 1));
-  c->grid2 = (int)std::min<size_t>(p.tiles2.size(), (size_t)c->sm_count * std::max(o2, 1));
+  c->grid2 = (int)p.tiles2.size();   // one CTA per tile: the hardware scheduler balances them
   c->grid3 = (int)std::min<size_t>(p.tiles3.size(), (size_t)c->sm_count * std::max(o3, 1));
   c->ptrs_host.assign((p.mats.size() + p.vecs.size()) * (size_t)(p.W + 1), nullptr);
   CK(cudaDeviceSynchronize());
@@ -495,7 +508,7 @@ int lqsgd_set_phase_events(lqsgd_ctx* c, void* const* host_events) {
 int lqsgd_launches_per_step(const lqsgd_ctx* ctx, int32_t* out) {
   if (!ctx || !out) return LQSGD_ERR_INVALID_ARG;
   const Plan& p = ctx->plan;
-  *out = (p.mats.empty() ? 0 : 6) + (p.tiles1.empty() ? 0 : 3) + (p.stiles1.empty() ? 0 : 3) + (p.chV.empty() ? 0 : 1);
+  *out = (p.mats.empty() ? 0 : 7) + (p.tiles1.empty() ? 0 : 2) + (p.stiles1.empty() ? 0 : 2) + (p.chV.empty() ? 0 : 1);
   return LQSGD_OK;
 }
 
@@ -574,7 +587,6 @@ int lqsgd_step(lqsgd_ctx* c, const float* const* grads, float* const* ghat, void
   PHASE_MARK(2);
   if (nm) {
     CK(launch_pass2(RP, t, p.d_tiles2, (int)p.tiles2.size(), {st, c->grid2}));
-    CK(launch_stream_pass2(RP, t, p.d_stiles2, (int)p.stiles2.size(), {st, (int)std::min<size_t>(p.stiles2.size(), c->sm_count)}));
   }
   PHASE_MARK(3);
   if (nm) {

@@ -102,14 +102,43 @@ cudaError_t launch_pass3(int RP, const Tables& t, const Tile* tiles, int ntiles,
 cudaError_t launch_vectors(const VectorDev* vecs, const ExchangeChunk* chunks, int nchunks,
                            const float* const* vgrads, float* const* vghat, uint8_t* payload,
                            uint64_t payload_stride, int W, Launch l);
-// Bulk-copy staged passes (lqsgd_stream.cu): layers with m % 4 == 0 and RP <= 8.  Tiles are at
-// most kStreamTileCols columns wide; pass 2 / pass 3 tiles start on a multiple of
-// kStreamStageRows rows.  One CTA per SM.
-constexpr int kStreamTileCols = 512;
-constexpr int kStreamStageRows = 16;
+// Bulk-copy staged passes (lqsgd_stream.cu): layers with m % 4 == 0 and RP <= 8.  One CTA per SM,
+// 512 consumer threads.  The copy engine limits the number of bulk copies in flight, not their
+// bytes, so tiles are wide (few, large row segments per stage) and a tile that spans whole rows
+// is fetched with ONE copy per stage (consecutive rows are contiguous).
 constexpr int kStreamMaxRP = 8;
+constexpr int kStreamConsumers = 512;
+constexpr int kStreamSlabFloats = 9216;   // one stage of one array: 36 KB = 16 x 576 = 8 x 1152 = 2 x 4608 floats
+
+// Widest tile (columns) the staged passes take at this padded rank: a thread keeps the Q rows
+// of all the column quads it owns in registers (quads per thread x 4 x RP <= 32 floats).
+__host__ __device__ inline int stream_max_cols(int RP) { return RP >= 8 ? 2048 : (RP == 4 ? 4096 : 6144); }
+
+// How the 512 consumers cover one stage of a tile `ncols` wide.
+struct StreamGeo {
+  int quads;   // float4 columns per row
+  int qpt;     // quads per thread (1..3); > 1 only when one row needs more than 512 threads
+  int tpr;     // threads per row (multiple of 32, <= 512)
+  int ng;      // row groups working side by side (512 / tpr)
+  int rpg;     // rows per group per stage (<= stream_rows_per_thread(RP))
+  int R;       // rows per stage
+};
+__host__ __device__ inline int stream_rows_per_thread(int RP) { return RP >= 8 ? 4 : 8; }
+__host__ __device__ inline StreamGeo stream_geo(int ncols, int RP) {
+  StreamGeo g;
+  g.quads = ncols >> 2;
+  g.qpt = (g.quads + kStreamConsumers - 1) / kStreamConsumers;
+  g.tpr = g.quads >= kStreamConsumers ? kStreamConsumers : ((g.quads + 31) & ~31);
+  g.ng = kStreamConsumers / g.tpr;
+  int R = kStreamSlabFloats / ncols;
+  const int cap = g.ng * stream_rows_per_thread(RP);
+  if (R > cap) R = cap;
+  if (R < 1) R = 1;
+  g.R = R;
+  g.rpg = (R + g.ng - 1) / g.ng;
+  return g;
+}
 cudaError_t launch_stream_pass1(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
-cudaError_t launch_stream_pass2(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
 cudaError_t launch_stream_pass3(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
 // Resident CTAs per SM of each streaming pass for this RP (for persistent grid sizing).
 cudaError_t pass_occupancy(int RP, int* occ1, int* occ2, int* occ3);

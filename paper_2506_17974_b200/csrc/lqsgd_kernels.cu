@@ -274,7 +274,7 @@ __device__ __forceinline__ void pass2_tile(const Tables& t, const Tile& tl, floa
   for (int i = 0; i < VEC * RP; ++i) acc[i] = 0.f;
 
   if (cm.active) {
-    constexpr int U = (RP <= 8) ? 16 : 8;
+    constexpr int U = 8;
     int i = tl.row0 + cm.g;
     for (; i + (U - 1) * cm.ng < rend; i += U * cm.ng) {
       Pack<VEC> mv[U];
@@ -321,7 +321,7 @@ __device__ __forceinline__ void pass2_tile(const Tables& t, const Tile& tl, floa
 }
 
 template <int RP>
-__global__ void __launch_bounds__(kPassThreads, (RP <= 8 ? 2 : 1))
+__global__ void __launch_bounds__(kPassThreads, (RP <= 2 ? 4 : (RP <= 8 ? 3 : 1)))
 pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
   __shared__ float red[128 * 4 * RP];
   for (int i = blockIdx.x; i < ntiles; i += gridDim.x) {
