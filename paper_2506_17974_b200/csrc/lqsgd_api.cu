@@ -322,6 +322,9 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   }
   for (size_t vi = 0; vi < p.vecs.size(); ++vi)
     for (int c = 0; c < ceil_div(p.vecs[vi].len, 256); ++c) p.chV.push_back({(int)vi, c});
+  // Pass 2 walks the data in the reverse of pass 1's order and pass 3 again in pass 1's order:
+  // each pass starts on what the previous one touched last, which is still in L2.
+  std::reverse(p.tiles2.begin(), p.tiles2.end());
   p.d_status = a.take<uint32_t>(p.mats.size());
   p.d_payload = a.take<uint8_t>((size_t)W * p.payload_stride);
   p.state_end = a.off;

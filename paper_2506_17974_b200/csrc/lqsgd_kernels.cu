@@ -85,6 +85,19 @@ __device__ __forceinline__ Pack<VEC> ld_l2(const float* p) {       // keep in L2
   return r;
 }
 
+// Streamed load that asks L2 to keep the line (the next pass starts on the data this pass reads last).
+template <int VEC>
+__device__ __forceinline__ Pack<VEC> ld_keep(const float* p, uint64_t pol) {
+  Pack<VEC> r;
+  if constexpr (VEC == 4) {
+    asm("ld.global.cg.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
+                 : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3]) : "l"(p), "l"(pol));
+  } else {
+    asm("ld.global.cg.L2::cache_hint.f32 %0, [%1], %2;" : "=f"(r.v[0]) : "l"(p), "l"(pol));
+  }
+  return r;
+}
+
 template <int VEC>
 __device__ __forceinline__ Pack<VEC> ld_ro(const float* __restrict__ p) {   // read-only data, cached in L1
   Pack<VEC> r;
@@ -260,7 +273,7 @@ __device__ __forceinline__ ColMap col_map(const Tile& tl) {
 // Row groups are then summed through shared memory in group order.
 // ---------------------------------------------------------------------------------------
 template <int RP, int VEC>
-__device__ __forceinline__ void pass2_tile(const Tables& t, const Tile& tl, float* red) {
+__device__ __forceinline__ void pass2_tile(const Tables& t, const Tile& tl, float* red, uint64_t pol) {
   const LayerDev& L = t.layers[tl.layer];
   const int m = L.m;
   const float* __restrict__ M = L.E + (size_t)tl.worker * L.n * m;
@@ -279,7 +292,7 @@ __device__ __forceinline__ void pass2_tile(const Tables& t, const Tile& tl, floa
     for (; i + (U - 1) * cm.ng < rend; i += U * cm.ng) {
       Pack<VEC> mv[U];
 #pragma unroll
-      for (int u = 0; u < U; ++u) mv[u] = ld_l2<VEC>(M + (size_t)(i + u * cm.ng) * m + col);
+      for (int u = 0; u < U; ++u) mv[u] = ld_keep<VEC>(M + (size_t)(i + u * cm.ng) * m + col, pol);
 #pragma unroll
       for (int u = 0; u < U; ++u) {
         float p[RP];
@@ -291,7 +304,7 @@ __device__ __forceinline__ void pass2_tile(const Tables& t, const Tile& tl, floa
       }
     }
     for (; i < rend; i += cm.ng) {
-      const Pack<VEC> mv = ld_l2<VEC>(M + (size_t)i * m + col);
+      const Pack<VEC> mv = ld_keep<VEC>(M + (size_t)i * m + col, pol);
       float p[RP];
       load_contig_ro<RP>(Pbar + (size_t)i * RP, p);
 #pragma unroll
@@ -324,10 +337,12 @@ template <int RP>
 __global__ void __launch_bounds__(kPassThreads, (RP <= 2 ? 4 : (RP <= 8 ? 3 : 1)))
 pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
   __shared__ float red[128 * 4 * RP];
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
   for (int i = blockIdx.x; i < ntiles; i += gridDim.x) {
     const Tile tl = tiles[i];
-    if (t.layers[tl.layer].vec) pass2_tile<RP, 4>(t, tl, red);
-    else pass2_tile<RP, 1>(t, tl, red);
+    if (t.layers[tl.layer].vec) pass2_tile<RP, 4>(t, tl, red, pol);
+    else pass2_tile<RP, 1>(t, tl, red, pol);
   }
 }
 

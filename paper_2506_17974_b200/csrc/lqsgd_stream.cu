@@ -118,6 +118,7 @@ stream_pass1_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   if (warp == kConsumerWarps) {                 // ---- loader
+    const uint64_t pol_first = policy_evict_first();
     bool ok = true;
     int last_layer = 0;
     uint32_t it = 0;
@@ -134,14 +135,15 @@ stream_pass1_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
         if (!ok) break;
         if (lane == 0) mbar_arrive_expect_tx(ring.full + s, 2u * rows * c.ncols * 4u);
         __syncwarp();
-        load_slab(sG + s * kSlab, G, c, sr, rows, ring.full + s, lane);
-        load_slab(sE + s * kSlab, E, c, sr, rows, ring.full + s, lane);
+        load_slab(sG + s * kSlab, G, c, sr, rows, ring.full + s, lane, pol_first);
+        load_slab(sE + s * kSlab, E, c, sr, rows, ring.full + s, lane, pol_first);
       }
     }
     if (!ok && lane == 0) { report_timeout(t, last_layer); loader_drain<NST>(ring, it); }
     return;
   }
   if (warp == kConsumerWarps + 1) {             // ---- storer: M slabs back over E
+    const uint64_t pol_last = policy_evict_last();
     bool ok = true;
     uint32_t it = 0;
     for (int ti = blockIdx.x; ti < ntiles && ok; ti += gridDim.x) {
@@ -152,7 +154,7 @@ stream_pass1_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
         const int rows = min(c.geo.R, c.nrows - sr);
         ok = warp_wait(ring.consumed + s, (it / NST) & 1, ring.abort_flag, lane);
         if (!ok) break;
-        store_slab(E, sE + s * kSlab, c, sr, rows, lane);
+        store_slab(E, sE + s * kSlab, c, sr, rows, lane, pol_last);     // pass 2 starts on the M written last
         bulk_commit();
         bulk_wait_read0();
         __syncwarp();
@@ -291,6 +293,7 @@ stream_pass3_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
   const int W = t.W;
 
   if (warp == kConsumerWarps) {                 // ---- loader
+    const uint64_t pol_first = policy_evict_first();
     bool ok = true;
     int last_layer = 0;
     uint32_t it = 0;
@@ -308,7 +311,7 @@ stream_pass3_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
           if (!ok) break;
           if (lane == 0) mbar_arrive_expect_tx(ring.full + s, (uint32_t)rows * c.ncols * 4u);
           __syncwarp();
-          load_slab(sM + s * kSlab, M0 + (size_t)w * plane, c, sr, rows, ring.full + s, lane);
+          load_slab(sM + s * kSlab, M0 + (size_t)w * plane, c, sr, rows, ring.full + s, lane, pol_first);
         }
       }
     }
@@ -316,6 +319,7 @@ stream_pass3_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
     return;
   }
   if (warp == kConsumerWarps + 1) {             // ---- storer: E slabs
+    const uint64_t pol_first = policy_evict_first();
     bool ok = true;
     uint32_t it = 0;
     for (int ti = blockIdx.x; ti < ntiles && ok; ti += gridDim.x) {
@@ -328,7 +332,7 @@ stream_pass3_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
           const int s = it % NST;
           ok = warp_wait(ring.consumed + s, (it / NST) & 1, ring.abort_flag, lane);
           if (!ok) break;
-          store_slab(E0 + (size_t)w * plane, sM + s * kSlab, c, sr, rows, lane);
+          store_slab(E0 + (size_t)w * plane, sM + s * kSlab, c, sr, rows, lane, pol_first);
           bulk_commit();
           bulk_wait_read0();
           __syncwarp();

@@ -71,6 +71,26 @@ __device__ __forceinline__ void bulk_store(void* gdst, const void* smem_src, uin
   asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
                ::"l"(gdst), "r"(smem_u32(smem_src)), "r"(bytes) : "memory");
 }
+// L2 eviction policies for the streams: data that will not be read again in this round goes
+// out first; data the next pass starts on (it walks the previous pass's order backwards) stays.
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void bulk_load_hint(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar, uint64_t pol) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+               ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(smem_u32(bar)), "l"(pol) : "memory");
+}
+__device__ __forceinline__ void bulk_store_hint(void* gdst, const void* smem_src, uint32_t bytes, uint64_t pol) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;"
+               ::"l"(gdst), "r"(smem_u32(smem_src)), "r"(bytes), "l"(pol) : "memory");
+}
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
@@ -157,20 +177,21 @@ __device__ __forceinline__ TileCtx tile_ctx(const Tables& t, const Tile& tl) {
 // Loads `rows` row segments of the tile (starting at tile row sr) into a slab: one copy if the
 // rows are contiguous, else one per row (lanes take rows).  Returns nothing; all on `bar`.
 __device__ __forceinline__ void load_slab(float* slab, const float* src_tile, const TileCtx& c, int sr, int rows,
-                                          uint64_t* bar, int lane) {
+                                          uint64_t* bar, int lane, uint64_t pol) {
   if (c.contig) {
-    if (lane == 0) bulk_load(slab, src_tile + (size_t)sr * c.m, (uint32_t)rows * c.ncols * 4u, bar);
+    if (lane == 0) bulk_load_hint(slab, src_tile + (size_t)sr * c.m, (uint32_t)rows * c.ncols * 4u, bar, pol);
   } else {
     for (int row = lane; row < rows; row += 32)
-      bulk_load(slab + row * c.ncols, src_tile + (size_t)(sr + row) * c.m, (uint32_t)c.ncols * 4u, bar);
+      bulk_load_hint(slab + row * c.ncols, src_tile + (size_t)(sr + row) * c.m, (uint32_t)c.ncols * 4u, bar, pol);
   }
 }
-__device__ __forceinline__ void store_slab(float* dst_tile, const float* slab, const TileCtx& c, int sr, int rows, int lane) {
+__device__ __forceinline__ void store_slab(float* dst_tile, const float* slab, const TileCtx& c, int sr, int rows, int lane,
+                                           uint64_t pol) {
   if (c.contig) {
-    if (lane == 0) bulk_store(dst_tile + (size_t)sr * c.m, slab, (uint32_t)rows * c.ncols * 4u);
+    if (lane == 0) bulk_store_hint(dst_tile + (size_t)sr * c.m, slab, (uint32_t)rows * c.ncols * 4u, pol);
   } else {
     for (int row = lane; row < rows; row += 32)
-      bulk_store(dst_tile + (size_t)(sr + row) * c.m, slab + row * c.ncols, (uint32_t)c.ncols * 4u);
+      bulk_store_hint(dst_tile + (size_t)(sr + row) * c.m, slab + row * c.ncols, (uint32_t)c.ncols * 4u, pol);
   }
 }
 
