@@ -239,6 +239,7 @@ __device__ __forceinline__ void pass1_tile(const Tables& t, const Tile& tl) {
 template <int RP>
 __global__ void __launch_bounds__(kPassThreads, (RP <= 8 ? 2 : 1))
 pass1_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
+  pdl_wait();
   for (int i = blockIdx.x; i < ntiles; i += gridDim.x) {
     const Tile tl = tiles[i];
     if (t.layers[tl.layer].vec) pass1_tile<RP, 4>(t, tl);
@@ -336,6 +337,7 @@ __device__ __forceinline__ void pass2_tile(const Tables& t, const Tile& tl, floa
 template <int RP>
 __global__ void __launch_bounds__(kPassThreads, (RP <= 2 ? 4 : (RP <= 8 ? 3 : 1)))
 pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
+  pdl_wait();
   __shared__ float red[128 * 4 * RP];
   uint64_t pol;
   asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
@@ -420,6 +422,7 @@ __device__ __forceinline__ void pass3_tile(const Tables& t, const Tile& tl) {
 template <int RP>
 __global__ void __launch_bounds__(kPassThreads, (RP <= 8 ? 2 : 1))
 pass3_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
+  pdl_wait();
   for (int i = blockIdx.x; i < ntiles; i += gridDim.x) {
     const Tile tl = tiles[i];
     if (t.layers[tl.layer].vec) pass3_tile<RP, 4>(t, tl);
@@ -441,6 +444,7 @@ constexpr double kPivotEps = 1e-10;
 template <int RP>
 __global__ void __launch_bounds__(256)
 p_reduce_gram_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
+  pdl_wait();
   __shared__ float rows[kFactorBlockRows][RP];
   const FactorBlock fb = fbs[blockIdx.x];
   const LayerDev& L = t.layers[fb.layer];
@@ -476,6 +480,7 @@ p_reduce_gram_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
 template <int RP>
 __global__ void __launch_bounds__(256)
 p_cholesky_kernel(Tables t) {
+  pdl_wait();
   __shared__ double A[RP][RP + 1];     // Gram, overwritten by L (lower triangle)
   __shared__ double X[RP][RP + 1];     // X[c][i] = (L^-1)[i][c]
   __shared__ double diag0[RP];
@@ -552,6 +557,7 @@ __device__ __forceinline__ float block_max_128(float v, float* sm) {
 template <int RP>
 __global__ void __launch_bounds__(kFactorBlockRows)
 p_apply_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
+  pdl_wait();
   __shared__ double Rinv[RP * RP];
   __shared__ float smax[4];
   const FactorBlock fb = fbs[blockIdx.x];
@@ -586,6 +592,7 @@ p_apply_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
 template <int RP>
 __global__ void __launch_bounds__(kFactorBlockRows)
 q_reduce_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
+  pdl_wait();
   __shared__ float smax[4];
   const FactorBlock fb = fbs[blockIdx.x];
   const LayerDev& L = t.layers[fb.layer];
@@ -629,6 +636,7 @@ q_reduce_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
 template <int RP>
 __global__ void __launch_bounds__(256)
 exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __restrict__ chunks) {
+  pdl_wait();
   constexpr int CH = kExchangeChunk;   // 256 factor elements per block, one per thread
   constexpr int WB = 8;                // workers handled per round
   __shared__ float thr[128];
@@ -731,6 +739,7 @@ exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __rest
 // Qt[j][i] = Q[i][j]: refreshes the transposed copy after Q was set from outside.
 __global__ void __launch_bounds__(256)
 q_transpose_kernel(const float* __restrict__ Q, float* __restrict__ Qt, int m, int RP, int mt) {
+  pdl_wait();
   const int i = blockIdx.x * 256 + threadIdx.x;
   if (i >= m) return;
   for (int j = 0; j < RP; ++j) Qt[(size_t)j * mt + i] = Q[(size_t)i * RP + j];
@@ -744,6 +753,7 @@ __global__ void __launch_bounds__(256)
 vectors_kernel(const VectorDev* __restrict__ vecs, const ExchangeChunk* __restrict__ chunks,
                const float* const* __restrict__ vgrads, float* const* __restrict__ vghat,
                uint8_t* payload, uint64_t payload_stride, int W) {
+  pdl_wait();
   const ExchangeChunk ch = chunks[blockIdx.x];
   const VectorDev v = vecs[ch.layer];
   const int i = ch.chunk * 256 + threadIdx.x;
@@ -774,55 +784,55 @@ vectors_kernel(const VectorDev* __restrict__ vecs, const ExchangeChunk* __restri
 
 cudaError_t launch_pass1(int rp, const Tables& t, const Tile* tiles, int ntiles, Launch l) {
   if (ntiles == 0) return cudaSuccess;
-  LQSGD_DISPATCH_RP(rp, (pass1_kernel<RP><<<l.grid, kPassThreads, 0, l.stream>>>(t, tiles, ntiles)));
+  LQSGD_DISPATCH_RP(rp, (launch_pdl(pass1_kernel<RP>, l.grid, kPassThreads, 0, l.stream, t, tiles, ntiles)));
   return cudaGetLastError();
 }
 
 cudaError_t launch_q_transpose(const float* Q, float* Qt, int m, int RP, int mt, cudaStream_t stream) {
-  q_transpose_kernel<<<(m + 255) / 256, 256, 0, stream>>>(Q, Qt, m, RP, mt);
+  launch_pdl(q_transpose_kernel, (m + 255) / 256, 256, 0, stream, Q, Qt, m, RP, mt);
   return cudaGetLastError();
 }
 
 cudaError_t launch_pass2(int rp, const Tables& t, const Tile* tiles, int ntiles, Launch l) {
   if (ntiles == 0) return cudaSuccess;
-  LQSGD_DISPATCH_RP(rp, (pass2_kernel<RP><<<l.grid, kPassThreads, 0, l.stream>>>(t, tiles, ntiles)));
+  LQSGD_DISPATCH_RP(rp, (launch_pdl(pass2_kernel<RP>, l.grid, kPassThreads, 0, l.stream, t, tiles, ntiles)));
   return cudaGetLastError();
 }
 
 cudaError_t launch_pass3(int rp, const Tables& t, const Tile* tiles, int ntiles, Launch l) {
   if (ntiles == 0) return cudaSuccess;
-  LQSGD_DISPATCH_RP(rp, (pass3_kernel<RP><<<l.grid, kPassThreads, 0, l.stream>>>(t, tiles, ntiles)));
+  LQSGD_DISPATCH_RP(rp, (launch_pdl(pass3_kernel<RP>, l.grid, kPassThreads, 0, l.stream, t, tiles, ntiles)));
   return cudaGetLastError();
 }
 
 cudaError_t launch_p_reduce_gram(int rp, const Tables& t, const FactorBlock* fb, int nfb, Launch l) {
   if (nfb == 0) return cudaSuccess;
-  LQSGD_DISPATCH_RP(rp, (p_reduce_gram_kernel<RP><<<nfb, 256, 0, l.stream>>>(t, fb)));
+  LQSGD_DISPATCH_RP(rp, (launch_pdl(p_reduce_gram_kernel<RP>, nfb, 256, 0, l.stream, t, fb)));
   return cudaGetLastError();
 }
 
 cudaError_t launch_p_cholesky(int rp, const Tables& t, int n_mat, Launch l) {
   if (n_mat == 0) return cudaSuccess;
-  LQSGD_DISPATCH_RP(rp, (p_cholesky_kernel<RP><<<n_mat * t.W, 256, 0, l.stream>>>(t)));
+  LQSGD_DISPATCH_RP(rp, (launch_pdl(p_cholesky_kernel<RP>, n_mat * t.W, 256, 0, l.stream, t)));
   return cudaGetLastError();
 }
 
 cudaError_t launch_p_apply(int rp, const Tables& t, const FactorBlock* fb, int nfb, Launch l) {
   if (nfb == 0) return cudaSuccess;
-  LQSGD_DISPATCH_RP(rp, (p_apply_kernel<RP><<<nfb, kFactorBlockRows, 0, l.stream>>>(t, fb)));
+  LQSGD_DISPATCH_RP(rp, (launch_pdl(p_apply_kernel<RP>, nfb, kFactorBlockRows, 0, l.stream, t, fb)));
   return cudaGetLastError();
 }
 
 cudaError_t launch_q_reduce(int rp, const Tables& t, const FactorBlock* fb, int nfb, Launch l) {
   if (nfb == 0) return cudaSuccess;
-  LQSGD_DISPATCH_RP(rp, (q_reduce_kernel<RP><<<nfb, kFactorBlockRows, 0, l.stream>>>(t, fb)));
+  LQSGD_DISPATCH_RP(rp, (launch_pdl(q_reduce_kernel<RP>, nfb, kFactorBlockRows, 0, l.stream, t, fb)));
   return cudaGetLastError();
 }
 
 cudaError_t launch_exchange(int rp, int which, const Tables& t, const QuantTables& q,
                             const ExchangeChunk* ch, int nch, Launch l) {
   if (nch == 0) return cudaSuccess;
-  LQSGD_DISPATCH_RP(rp, (exchange_kernel<RP><<<nch, 256, 0, l.stream>>>(t, q, which, ch)));
+  LQSGD_DISPATCH_RP(rp, (launch_pdl(exchange_kernel<RP>, nch, 256, 0, l.stream, t, q, which, ch)));
   return cudaGetLastError();
 }
 
@@ -830,7 +840,7 @@ cudaError_t launch_vectors(const VectorDev* vecs, const ExchangeChunk* chunks, i
                            const float* const* vgrads, float* const* vghat, uint8_t* payload,
                            uint64_t payload_stride, int W, Launch l) {
   if (nchunks == 0) return cudaSuccess;
-  vectors_kernel<<<nchunks, 256, 0, l.stream>>>(vecs, chunks, vgrads, vghat, payload, payload_stride, W);
+  launch_pdl(vectors_kernel, nchunks, 256, 0, l.stream, vecs, chunks, vgrads, vghat, payload, payload_stride, W);
   return cudaGetLastError();
 }
 

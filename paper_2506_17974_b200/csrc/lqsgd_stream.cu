@@ -107,6 +107,7 @@ __device__ __forceinline__ bool pass1_consume(const Tables& t, const TileCtx& c,
 template <int RP, int NST>
 __global__ void __launch_bounds__(kThreads, 1)
 stream_pass1_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
+  pdl_wait();
   extern __shared__ __align__(128) unsigned char smem_raw[];
   float* sG = reinterpret_cast<float*>(smem_raw);
   float* sE = sG + NST * kSlab;
@@ -283,6 +284,7 @@ __device__ __forceinline__ bool pass3_consume(const Tables& t, const TileCtx& c,
 template <int RP, int NST>
 __global__ void __launch_bounds__(kThreads, 1)
 stream_pass3_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
+  pdl_wait();
   extern __shared__ __align__(128) unsigned char smem_raw[];
   float* sM = reinterpret_cast<float*>(smem_raw);
   uint64_t* bars = reinterpret_cast<uint64_t*>(sM + NST * kSlab);
@@ -363,7 +365,7 @@ template <typename K>
 cudaError_t launch_staged(K kernel, size_t smem, const Tables& t, const Tile* tiles, int ntiles, Launch l) {
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  kernel<<<l.grid, kThreads, smem, l.stream>>>(t, tiles, ntiles);
+  launch_pdl(kernel, l.grid, kThreads, smem, l.stream, t, tiles, ntiles);
   return cudaGetLastError();
 }
 
