@@ -273,7 +273,6 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
     L.Qpart = a.take<float>((size_t)W * L.nrb * mt.m * RP);
     L.Qw = (L.nrb == 1) ? L.Qpart : a.take<float>((size_t)W * mt.m * RP);
     L.gram_part = a.take<double>((size_t)W * L.npb * RP * RP);
-    L.rinv = a.take<double>((size_t)W * RP * RP);
     L.maxp = a.take<float>((size_t)W * L.npb);
     L.maxq = a.take<float>((size_t)W * L.nqb);
     L.codesP = a.take<uint8_t>((size_t)W * mt.n * mt.r);
@@ -511,7 +510,7 @@ int lqsgd_set_phase_events(lqsgd_ctx* c, void* const* host_events) {
 int lqsgd_launches_per_step(const lqsgd_ctx* ctx, int32_t* out) {
   if (!ctx || !out) return LQSGD_ERR_INVALID_ARG;
   const Plan& p = ctx->plan;
-  *out = (p.mats.empty() ? 0 : 7) + (p.tiles1.empty() ? 0 : 2) + (p.stiles1.empty() ? 0 : 2) + (p.chV.empty() ? 0 : 1);
+  *out = (p.mats.empty() ? 0 : 6) + (p.tiles1.empty() ? 0 : 2) + (p.stiles1.empty() ? 0 : 2) + (p.chV.empty() ? 0 : 1);
   return LQSGD_OK;
 }
 
@@ -583,7 +582,6 @@ int lqsgd_step(lqsgd_ctx* c, const float* const* grads, float* const* ghat, void
   PHASE_MARK(1);
   if (nm) {
     CK(launch_p_reduce_gram(RP, t, p.d_fbP, (int)p.fbP.size(), {st, 0}));
-    CK(launch_p_cholesky(RP, t, (int)nm, {st, 0}));
     CK(launch_p_apply(RP, t, p.d_fbP, (int)p.fbP.size(), {st, 0}));
     CK(launch_exchange(RP, 0, t, qp, p.d_chP, (int)p.chP.size(), {st, 0}));
   }

@@ -32,7 +32,6 @@ struct LayerDev {
   float* Qpart;               // [W][nrb][m][RP]
   float* Qw;                  // [W][m][RP]  (== Qpart when nrb == 1)
   double* gram_part;          // [W][npb][RP*RP]
-  double* rinv;               // [W][RP*RP]  R^-1 (upper triangular), row-major
   float* maxp;                // [W][npb]
   float* maxq;                // [W][nqb]
   uint8_t* codesP;            // [W][n*r]
@@ -115,7 +114,6 @@ struct Launch {
 
 cudaError_t launch_pass1(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
 cudaError_t launch_p_reduce_gram(int RP, const Tables& t, const FactorBlock* fb, int nfb, Launch l);
-cudaError_t launch_p_cholesky(int RP, const Tables& t, int n_mat, Launch l);
 cudaError_t launch_p_apply(int RP, const Tables& t, const FactorBlock* fb, int nfb, Launch l);
 cudaError_t launch_exchange(int RP, int which /*0 = P, 1 = Q*/, const Tables& t, const QuantTables& q,
                             const ExchangeChunk* ch, int nch, Launch l);

@@ -433,8 +433,8 @@ pass3_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
 // ---------------------------------------------------------------------------------------
 // Orthonormalize (Alg. 1) as CholeskyQR with the r x r part in fp64:
 //   p_reduce_gram: P_raw = sum of the column-chunk partials (fixed order); per-block Gram
-//   p_cholesky   : Gram = sum of block Grams; R^T R = Gram; R^-1
-//   p_apply      : P = P_raw R^-1 (fp64 accumulate, stored fp32); block max |P|
+//   p_apply      : Gram = sum of block Grams; R^T R = Gram; R^-1 (redone by every CTA);
+//                  P = P_raw R^-1 (fp64 accumulate, stored fp32); block max |P|
 // The result is the thin-QR Q factor with positive-diagonal R, the same matrix Gram-Schmidt
 // produces.  A column whose pivot is <= 1e-10 of its squared norm (or zero, or not a number)
 // becomes a zero column and the layer's status word says so.
@@ -477,23 +477,23 @@ p_reduce_gram_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
   }
 }
 
+// Gram = sum of the block Grams (block order), Cholesky R^T R = Gram, R^-1 into Rinv (shared,
+// RP*RP doubles, row-major, upper triangular).  Run by a whole CTA; every CTA that applies R^-1
+// to a block of rows redoes this small factorisation itself, which costs less than a kernel
+// boundary.  Returns true if a column was dropped as dependent.
 template <int RP>
-__global__ void __launch_bounds__(256)
-p_cholesky_kernel(Tables t) {
-  pdl_wait();
+__device__ __forceinline__ bool cholesky_rinv(const LayerDev& L, int worker, double* Rinv) {
   __shared__ double A[RP][RP + 1];     // Gram, overwritten by L (lower triangle)
   __shared__ double X[RP][RP + 1];     // X[c][i] = (L^-1)[i][c]
   __shared__ double diag0[RP];
   __shared__ int dead[RP];
-  const int layer = blockIdx.x / t.W, worker = blockIdx.x % t.W;
-  const LayerDev& L = t.layers[layer];
-  const int r = L.r, tid = threadIdx.x;
-  if (tid < RP * RP) {
-    const double* gp = L.gram_part + (size_t)worker * L.npb * (RP * RP) + tid;
+  const int r = L.r, tid = threadIdx.x, nt = blockDim.x;
+  for (int e = tid; e < RP * RP; e += nt) {
+    const double* gp = L.gram_part + (size_t)worker * L.npb * (RP * RP) + e;
     double s = 0.0;
     for (int b = 0; b < L.npb; ++b) s += gp[(size_t)b * (RP * RP)];
-    A[tid / RP][tid % RP] = s;
-    X[tid / RP][tid % RP] = 0.0;
+    A[e / RP][e % RP] = s;
+    X[e / RP][e % RP] = 0.0;
   }
   __syncthreads();
   if (tid < RP) { diag0[tid] = A[tid][tid]; dead[tid] = 0; }
@@ -534,15 +534,14 @@ p_cholesky_kernel(Tables t) {
     }
   }
   __syncthreads();
-  if (tid < RP * RP) {
-    const int k = tid / RP, j = tid % RP;       // R^-1[k][j] = (L^-1)[j][k], k <= j < r
-    L.rinv[(size_t)worker * (RP * RP) + tid] = (k <= j && j < r) ? X[k][j] : 0.0;
+  for (int e = tid; e < RP * RP; e += nt) {
+    const int k = e / RP, j = e % RP;           // R^-1[k][j] = (L^-1)[j][k], k <= j < r
+    Rinv[e] = (k <= j && j < r) ? X[k][j] : 0.0;
   }
-  if (tid == 0) {
-    int any = 0;
-    for (int j = 0; j < r; ++j) any |= dead[j];
-    if (any) atomicOr(&t.status[layer], 1u);
-  }
+  int any = 0;
+  for (int j = 0; j < r; ++j) any |= dead[j];
+  __syncthreads();
+  return any != 0;
 }
 
 __device__ __forceinline__ float block_max_128(float v, float* sm) {
@@ -563,8 +562,8 @@ p_apply_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
   const FactorBlock fb = fbs[blockIdx.x];
   const LayerDev& L = t.layers[fb.layer];
   const int n = L.n, tid = threadIdx.x;
-  for (int k = tid; k < RP * RP; k += kFactorBlockRows) Rinv[k] = L.rinv[(size_t)fb.worker * (RP * RP) + k];
-  __syncthreads();
+  const bool dropped = cholesky_rinv<RP>(L, fb.worker, Rinv);
+  if (dropped && fb.blk == 0 && tid == 0) atomicOr(&t.status[fb.layer], 1u);
   const int row = fb.blk * kFactorBlockRows + tid;
   float amax = 0.f;
   if (row < n) {
@@ -808,12 +807,6 @@ cudaError_t launch_pass3(int rp, const Tables& t, const Tile* tiles, int ntiles,
 cudaError_t launch_p_reduce_gram(int rp, const Tables& t, const FactorBlock* fb, int nfb, Launch l) {
   if (nfb == 0) return cudaSuccess;
   LQSGD_DISPATCH_RP(rp, (launch_pdl(p_reduce_gram_kernel<RP>, nfb, 256, 0, l.stream, t, fb)));
-  return cudaGetLastError();
-}
-
-cudaError_t launch_p_cholesky(int rp, const Tables& t, int n_mat, Launch l) {
-  if (n_mat == 0) return cudaSuccess;
-  LQSGD_DISPATCH_RP(rp, (launch_pdl(p_cholesky_kernel<RP>, n_mat * t.W, 256, 0, l.stream, t)));
   return cudaGetLastError();
 }
 
