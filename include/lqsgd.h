@@ -88,7 +88,8 @@ typedef struct lqsgd_shape {
 typedef struct lqsgd_config {
   uint32_t struct_size; /* sizeof(lqsgd_config), for versioning */
   int32_t rank;         /* r, 1..16 (any integer) */
-  int32_t bits_p;       /* b_p, total bits per P scalar including the sign, 2..8 */
+  int32_t bits_p;       /* b_p, total bits per P scalar including the sign, 2..8; 32 = no quantiser: the
+                           factor is sent as fp32 and averaged directly (the PowerSGD exchange of Section III-B) */
   int32_t bits_q;       /* b_q, likewise for Q */
   float alpha;          /* alpha of Eq. 4 / Eq. 5, finite and > 0 */
   int32_t workers;      /* W, 1..256 */
@@ -118,7 +119,7 @@ typedef enum lqsgd_state {
   LQSGD_STATE_P = 3,       /* fp32 n x r_eff, per worker: orthonormal P of the last step */
   LQSGD_STATE_P_BAR = 4,   /* fp32 n x r_eff: dequantised worker average of P */
   LQSGD_STATE_Q_W = 5,     /* fp32 m x r_eff, per worker: M^T P_bar of the last step */
-  LQSGD_STATE_CODES_P = 6, /* uint8 n x r_eff, per worker: one unpacked code per byte */
+  LQSGD_STATE_CODES_P = 6, /* uint8 n x r_eff, per worker: one unpacked code per byte (not with bits 32) */
   LQSGD_STATE_CODES_Q = 7, /* uint8 m x r_eff, per worker */
   LQSGD_STATE_SCALES = 8   /* fp32 [2]: s_P, s_Q of the last step */
 } lqsgd_state;

@@ -84,7 +84,8 @@ int check_config(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
   if (!shapes || !c || n_layers < 1) return LQSGD_ERR_INVALID_ARG;
   if (c->struct_size != sizeof(lqsgd_config)) return LQSGD_ERR_INVALID_ARG;
   if (c->rank < 1 || c->rank > kMaxRank) return LQSGD_ERR_INVALID_ARG;
-  if (c->bits_p < 2 || c->bits_p > 8 || c->bits_q < 2 || c->bits_q > 8) return LQSGD_ERR_INVALID_ARG;
+  auto bits_ok = [](int b) { return (b >= 2 && b <= 8) || b == 32; };
+  if (!bits_ok(c->bits_p) || !bits_ok(c->bits_q)) return LQSGD_ERR_INVALID_ARG;
   if (!(c->alpha > 0.f) || !std::isfinite(c->alpha)) return LQSGD_ERR_INVALID_ARG;
   if (c->workers < 1 || c->workers > 256) return LQSGD_ERR_INVALID_ARG;
   if (c->flags & ~(LQSGD_FLAG_HOST_STAGING | LQSGD_FLAG_REGISTER_PATH)) return LQSGD_ERR_INVALID_ARG;
@@ -99,6 +100,7 @@ int check_config(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
 // boundary between levels k and k+1 at |x|/s = ((1+alpha)^((k+1/2)/(L-1)) - 1)/alpha, stored as
 // the smallest fp32 >= that value; deq[S + W(L-1)] = sign(S) ((1+alpha)^(|S|/(W(L-1))) - 1)/alpha.
 void quant_tables(int bits, double alpha, int W, std::vector<float>& thr, std::vector<float>& deq) {
+  if (bits == 32) { thr.assign(1, 0.f); deq.assign(1, 0.f); return; }   // quantiser bypassed: no tables
   const int L = 1 << (bits - 1);
   const double la = std::log1p(alpha);
   thr.resize(L - 1);
@@ -155,7 +157,7 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   for (auto& mt : p.mats) {
     auto& lo = p.layout[mt.user_index];
     lo.is_matrix = 1; lo.rank_eff = mt.r;
-    lo.p_offset = off; lo.p_bytes = ((size_t)mt.n * mt.r * cfg.bits_p + 7) / 8; off += lo.p_bytes;
+    lo.p_offset = off; lo.p_bytes = ((size_t)mt.n * mt.r * cfg.bits_p + 7) / 8; off += lo.p_bytes;   // bits 32: the fp32 factor
   }
   for (auto& mt : p.mats) {
     auto& lo = p.layout[mt.user_index];
@@ -682,8 +684,8 @@ static int locate_state(const lqsgd_ctx* c, int which, int layer, int worker, ch
     case LQSGD_STATE_P: *base = (char*)(L.P + w * n * RP); *rows = n; *row_bytes = 4 * r; *pitch = 4 * RP; break;
     case LQSGD_STATE_P_BAR: *base = (char*)L.Pbar; *rows = n; *row_bytes = 4 * r; *pitch = 4 * RP; break;
     case LQSGD_STATE_Q_W: *base = (char*)(L.Qw + w * m * RP); *rows = m; *row_bytes = 4 * r; *pitch = 4 * RP; break;
-    case LQSGD_STATE_CODES_P: *base = (char*)(L.codesP + w * n * r); *rows = 1; *row_bytes = *pitch = n * r; break;
-    case LQSGD_STATE_CODES_Q: *base = (char*)(L.codesQ + w * m * r); *rows = 1; *row_bytes = *pitch = m * r; break;
+    case LQSGD_STATE_CODES_P: if (c->cfg.bits_p == 32) return LQSGD_ERR_OUT_OF_RANGE; *base = (char*)(L.codesP + w * n * r); *rows = 1; *row_bytes = *pitch = n * r; break;
+    case LQSGD_STATE_CODES_Q: if (c->cfg.bits_q == 32) return LQSGD_ERR_OUT_OF_RANGE; *base = (char*)(L.codesQ + w * m * r); *rows = 1; *row_bytes = *pitch = m * r; break;
     case LQSGD_STATE_SCALES: *base = (char*)L.scales; *rows = 1; *row_bytes = *pitch = 8; break;
     default: return LQSGD_ERR_OUT_OF_RANGE;
   }

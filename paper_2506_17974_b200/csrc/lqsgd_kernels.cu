@@ -644,7 +644,7 @@ exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __rest
   const ExchangeChunk ch = chunks[blockIdx.x];
   const LayerDev& L = t.layers[ch.layer];
   const int W = t.W, tid = threadIdx.x, b = qt.bits;
-  const int nlev = 1 << (b - 1);
+  const int nlev = (b == 32) ? 2 : 1 << (b - 1);
   const int rows = which ? L.m : L.n, r = L.r;
   const int count = rows * r;
   const int nblk = which ? L.nqb : L.npb;
@@ -665,6 +665,35 @@ exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __rest
 #pragma unroll
   for (int i = 1; i < 8; ++i) s = fmaxf(s, sred[i]);
   const bool s_ok = (s > 0.f) && (s < INFINITY);
+
+  if (b == 32) {
+    // Quantiser bypassed (plain PowerSGD exchange): the factor travels as fp32 and the workers'
+    // factors are averaged directly (Eq. 1), in worker order.
+    const int e = ch.chunk * CH + tid;
+    if (e < count) {
+      const int row = e / r, col = e - row * r;
+      float sum = 0.f;
+      for (int w = 0; w < W; ++w) {
+        const float x = __ldg(src + ((size_t)w * rows + row) * RP + col);
+        sum += x;
+        uint8_t* pay = t.payload + (size_t)w * t.payload_stride + pay_off + (size_t)e * 4;
+        const unsigned bits32 = __float_as_uint(x);               // the stream may start on any byte
+        pay[0] = bits32 & 0xff; pay[1] = (bits32 >> 8) & 0xff; pay[2] = (bits32 >> 16) & 0xff; pay[3] = bits32 >> 24;
+      }
+      const float v = sum / (float)W;
+      dst[(size_t)row * RP + col] = v;
+      if (which) L.Qt[(size_t)col * L.mt + row] = v;
+    }
+    if (ch.chunk == 0 && tid == 0) {
+      L.scales[which] = s;
+      for (int w = 0; w < W; ++w) {
+        float* ps = reinterpret_cast<float*>(t.payload + (size_t)w * t.payload_stride + L.pay_scale_off);
+        ps[which] = s;
+      }
+      if (!(s < INFINITY)) atomicOr(&t.status[ch.layer], 8u);
+    }
+    return;
+  }
 
   const int e0 = ch.chunk * CH;
   const int cnt = min(CH, count - e0);

@@ -267,3 +267,53 @@ def test_argument_errors_launch_nothing():
     assert e.value.code == B.ERR_OUT_OF_RANGE
     comp.step([[ok]], [out])                       # still usable afterwards
     torch.cuda.synchronize()
+
+
+def test_quantiser_bypass_is_plain_powersgd():
+    """bits = 32: factors travel as fp32 and are averaged directly (Section III-B, Eq. 1)."""
+    w = wl.Workload("bypass", ((96, 200), (130, 36), (20, 1)), rank=4, bits=32, workers=3, steps=3,
+                    dist="student_t3", scale="fan_in", seed=9)
+    comp = make(w)
+    oracle = new_oracle(comp)
+    assert comp.payload_nbytes == orc.payload_bytes(w.layers, 4, 32, 32) == 4 * 4 * (96 + 200 + 130 + 36) + 16 + 80
+    for t in range(3):
+        g = wl.draw_gradients(w, t, device=DEV)
+        E_prev, _ = par.snapshot_state(comp)
+        ghat = [torch.empty_like(x) for x in g[0]]
+        comp.step(g, ghat)
+        torch.cuda.synchronize()
+        gh = [[par.host(x) for x in per] for per in g]
+        out = oracle.step(gh)
+        for l in (0, 1):
+            n, m = w.layers[l]
+            P = np.stack([par.host(comp.get_state(B.STATE_P, l, k)) for k in range(3)])
+            Qw = np.stack([par.host(comp.get_state(B.STATE_Q_W, l, k)) for k in range(3)])
+            P_bar, Q_bar = par.host(comp.get_state(B.STATE_P_BAR, l)), par.host(comp.get_state(B.STATE_Q, l))
+            assert par.rel_fro(P_bar, P.astype(np.float64).mean(0)) <= 1e-6
+            assert par.rel_fro(Q_bar, Qw.astype(np.float64).mean(0)) <= 1e-6
+            for k in range(3):
+                M = orc.error_feedback(gh[k][l], E_prev[l][k])
+                assert par.rel_fro(Qw[k], orc.power_step_q(M, P_bar)) <= par.TOL
+            for name, dev_val in (("P_bar", P_bar), ("Q_bar", Q_bar), ("G_hat", par.host(ghat[l]))):
+                assert par.rel_fro(dev_val, out[l][name]) <= par.TOL, (t, l, name)
+            lo = comp.payload_layout(l)
+            for k in range(3):
+                pay = par.host(comp.payload(k))
+                assert pay[lo.p_offset:lo.p_offset + lo.p_bytes].tobytes() == P[k].astype("<f4").tobytes()
+                assert pay[lo.q_offset:lo.q_offset + lo.q_bytes].tobytes() == Qw[k].astype("<f4").tobytes()
+        with pytest.raises(B.LqsgdError):
+            comp.get_state(B.STATE_CODES_P, 0, 0)
+
+
+def test_planted_rank_r_gradient_is_recovered_on_the_device():
+    """G = A B^T of rank r, E = 0, no quantiser: one round returns G itself (Eq. 3)."""
+    gen = torch.Generator().manual_seed(2)
+    A = torch.randint(-4, 5, (160, 3), generator=gen).float()
+    Bm = torch.randint(-4, 5, (264, 3), generator=gen).float()
+    G = (A @ Bm.T).to(DEV)
+    comp = B.LQSGD(((160, 264),), 3, 32)
+    out = torch.empty_like(G)
+    comp.step([[G]], [out])
+    torch.cuda.synchronize()
+    assert par.rel_fro(par.host(out), par.host(G)) <= 1e-5
+    assert float(comp.get_state(B.STATE_E, 0, 0).abs().max()) <= 1e-4 * float(G.abs().max())
