@@ -151,6 +151,16 @@ int lqsgd_create(const lqsgd_shape* host_shapes, int32_t n_layers, const lqsgd_c
 int lqsgd_step(lqsgd_ctx* ctx, const float* const* host_grads, float* const* host_ghat,
                void* cuda_stream);
 
+/* lqsgd_step followed, inside the reconstruction pass, by the model update that ends an
+ * iteration of Algorithm 1:  w <- w - lr * G_hat  for every layer (for a 1-D tensor G_hat is the
+ * worker mean).  host_weights: host array of n_layers device pointers, fp32, shaped and aligned
+ * like the gradients, updated in place; an entry may be NULL (that layer is not updated).
+ * host_ghat may be NULL, or hold NULL entries: G_hat of those layers is then not written at all,
+ * which saves its 4/W bytes per worker-element of traffic; every layer needs at least one of the two.
+ * Everything else as lqsgd_step. */
+int lqsgd_step_update(lqsgd_ctx* ctx, const float* const* host_grads, float* const* host_ghat,
+                      float* const* host_weights, float lr, void* cuda_stream);
+
 /* Same round with HOST tensors: copies every gradient host->device into the staging area,
  * runs lqsgd_step, copies every G_hat and all W payloads device->host, and synchronises the
  * stream before returning.  host_grads / host_ghat are arrays of host pointers laid out as in

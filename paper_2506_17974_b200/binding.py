@@ -31,7 +31,7 @@ ERR_TOO_LARGE = -8
 NOALLOC_MAX_ROWS = 65536
 
 EXPORTED = [
-    "lqsgd_workspace_bytes", "lqsgd_create", "lqsgd_step", "lqsgd_step_host", "lqsgd_payload_bytes",
+    "lqsgd_workspace_bytes", "lqsgd_create", "lqsgd_step", "lqsgd_step_update", "lqsgd_step_host", "lqsgd_payload_bytes",
     "lqsgd_payload", "lqsgd_payload_layout", "lqsgd_get_state", "lqsgd_set_state", "lqsgd_status",
     "lqsgd_orthonormalize_noalloc",
     "lqsgd_launches_per_step", "lqsgd_set_phase_events", "lqsgd_destroy", "lqsgd_strerror", "lqsgd_last_cuda_error", "lqsgd_version",
@@ -75,6 +75,7 @@ def load_library() -> C.CDLL:
     lib.lqsgd_workspace_bytes.argtypes = [C.POINTER(Shape), i32, C.POINTER(Config), C.POINTER(sz)]
     lib.lqsgd_create.argtypes = [C.POINTER(Shape), i32, C.POINTER(Config), vp, sz, C.POINTER(vp)]
     lib.lqsgd_step.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), vp]
+    lib.lqsgd_step_update.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.c_float, vp]
     lib.lqsgd_step_host.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), vp, vp]
     lib.lqsgd_payload_bytes.argtypes = [vp, C.POINTER(sz)]
     lib.lqsgd_payload.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(sz)]
@@ -223,6 +224,22 @@ class LQSGD:
         """One round of Algorithm 1 on device tensors grads[w][l]; writes ghat[l]."""
         g, h = self.make_pointer_arrays(grads, ghat)
         self.step_ptrs(g, h, stream)
+
+    def step_update(self, grads, ghat, weights, lr: float, stream: Optional[torch.cuda.Stream] = None) -> None:
+        """One round plus the model update w <- w - lr * G_hat (Algorithm 1, last line) fused into the
+        reconstruction pass.  weights[l] (device tensors, or None entries) are updated in place;
+        ghat may be None or hold None entries: G_hat of those layers is not materialised."""
+        nl = len(self.layers)
+        g = (C.c_void_p * (self.W * nl))()
+        for w in range(self.W):
+            for l in range(nl):
+                g[w * nl + l] = grads[w][l].data_ptr()
+        h = None
+        if ghat is not None:
+            h = (C.c_void_p * nl)(*[(t.data_ptr() if t is not None else None) for t in ghat])
+        wt = (C.c_void_p * nl)(*[(t.data_ptr() if t is not None else None) for t in weights])
+        s = stream if stream is not None else torch.cuda.current_stream(self.device)
+        _check(self.lib.lqsgd_step_update(self.ctx, g, h, wt, C.c_float(lr), C.c_void_p(s.cuda_stream)))
 
     def step_host(self, grads, ghat, payload: Optional[torch.Tensor] = None,
                   stream: Optional[torch.cuda.Stream] = None) -> None:

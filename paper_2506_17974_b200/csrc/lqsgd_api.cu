@@ -69,7 +69,7 @@ struct Plan {
   FactorBlock *d_fbP = nullptr, *d_fbQ = nullptr;
   ExchangeChunk *d_chP = nullptr, *d_chQ = nullptr, *d_chV = nullptr;
   float *d_thrP = nullptr, *d_thrQ = nullptr, *d_deqP = nullptr, *d_deqQ = nullptr;
-  void** d_ptrs = nullptr;                    // [grads n_mat*W | ghat n_mat | vgrads nvec*W | vghat nvec]
+  void** d_ptrs = nullptr;                    // see step_impl for the layout
   uint32_t* d_status = nullptr;
   uint8_t* d_payload = nullptr;
   float* d_stage_g = nullptr;                 // [W][elems_total]
@@ -346,7 +346,7 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   p.d_thrQ = a.take<float>(p.thrQ.size());
   p.d_deqP = a.take<float>(p.deqP.size());
   p.d_deqQ = a.take<float>(p.deqQ.size());
-  p.d_ptrs = a.take<void*>((p.mats.size() + p.vecs.size()) * (size_t)(W + 1));
+  p.d_ptrs = a.take<void*>((p.mats.size() + p.vecs.size()) * (size_t)(W + 2));
   if (cfg.flags & LQSGD_FLAG_HOST_STAGING) {
     p.d_stage_g = a.take<float>((size_t)W * p.elems_total);
     p.d_stage_ghat = a.take<float>(p.elems_total);
@@ -488,7 +488,7 @@ int lqsgd_create(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
   c->grid1 = (int)std::min<size_t>(p.tiles1.size(), (size_t)c->sm_count * std::max(o1, 1));
   c->grid2 = (int)p.tiles2.size();   // one CTA per tile: the hardware scheduler balances them
   c->grid3 = (int)std::min<size_t>(p.tiles3.size(), (size_t)c->sm_count * std::max(o3, 1));
-  c->ptrs_host.assign((p.mats.size() + p.vecs.size()) * (size_t)(p.W + 1), nullptr);
+  c->ptrs_host.assign((p.mats.size() + p.vecs.size()) * (size_t)(p.W + 2), nullptr);
   CK(cudaDeviceSynchronize());
   guard.c = nullptr;
   *ctx_out = c;
@@ -516,14 +516,22 @@ int lqsgd_launches_per_step(const lqsgd_ctx* ctx, int32_t* out) {
   return LQSGD_OK;
 }
 
-int lqsgd_step(lqsgd_ctx* c, const float* const* grads, float* const* ghat, void* cuda_stream) {
-  if (!c || !grads || !ghat) return LQSGD_ERR_INVALID_ARG;
+// The round, with the optional model update.  ghat == nullptr (only with weights): G_hat is not
+// written.  Pointer table: [grads nm*W | ghat nm | weights nm | vgrads nv*W | vghat nv | vweights nv].
+static int step_impl(lqsgd_ctx* c, const float* const* grads, float* const* ghat, float* const* weights, float lr,
+                     void* cuda_stream) {
+  if (!c || !grads || (!ghat && !weights)) return LQSGD_ERR_INVALID_ARG;
   Plan& p = c->plan;
   const int W = p.W, nl = (int)c->shapes.size();
   const size_t nm = p.mats.size(), nv = p.vecs.size();
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  // ---- check and gather pointers: [grads nm*W | ghat nm | vgrads nv*W | vghat nv]
   std::vector<void*> ptrs(c->ptrs_host.size());
+  auto out_ptr = [&](float* const* arr, int ui, uintptr_t amask, void** slot) -> int {
+    float* q = arr ? arr[ui] : nullptr;
+    if (reinterpret_cast<uintptr_t>(q) & amask) return LQSGD_ERR_MISALIGNED;
+    *slot = q;
+    return LQSGD_OK;
+  };
   for (size_t li = 0; li < nm; ++li) {
     const int ui = p.mats[li].user_index;
     const uintptr_t amask = (p.mats[li].m % 4 == 0) ? 15 : 3;
@@ -533,11 +541,12 @@ int lqsgd_step(lqsgd_ctx* c, const float* const* grads, float* const* ghat, void
       if (reinterpret_cast<uintptr_t>(g) & amask) return LQSGD_ERR_MISALIGNED;
       ptrs[li * W + w] = const_cast<float*>(g);
     }
-    if (!ghat[ui]) return LQSGD_ERR_INVALID_ARG;
-    if (reinterpret_cast<uintptr_t>(ghat[ui]) & amask) return LQSGD_ERR_MISALIGNED;
-    ptrs[nm * W + li] = ghat[ui];
+    int rc = out_ptr(ghat, ui, amask, &ptrs[nm * W + li]);
+    if (rc == LQSGD_OK) rc = out_ptr(weights, ui, amask, &ptrs[nm * (W + 1) + li]);
+    if (rc != LQSGD_OK) return rc;
+    if (!ptrs[nm * W + li] && !ptrs[nm * (W + 1) + li]) return LQSGD_ERR_INVALID_ARG;   // nowhere to put the result
   }
-  const size_t vbase = nm * (W + 1);
+  const size_t vbase = nm * (W + 2);
   for (size_t vi = 0; vi < nv; ++vi) {
     const int ui = p.vecs[vi].user_index;
     for (int w = 0; w < W; ++w) {
@@ -546,9 +555,10 @@ int lqsgd_step(lqsgd_ctx* c, const float* const* grads, float* const* ghat, void
       if (reinterpret_cast<uintptr_t>(g) & 3) return LQSGD_ERR_MISALIGNED;
       ptrs[vbase + vi * W + w] = const_cast<float*>(g);
     }
-    if (!ghat[ui]) return LQSGD_ERR_INVALID_ARG;
-    if (reinterpret_cast<uintptr_t>(ghat[ui]) & 3) return LQSGD_ERR_MISALIGNED;
-    ptrs[vbase + nv * W + vi] = ghat[ui];
+    int rc = out_ptr(ghat, ui, 3, &ptrs[vbase + nv * W + vi]);
+    if (rc == LQSGD_OK) rc = out_ptr(weights, ui, 3, &ptrs[vbase + nv * (W + 1) + vi]);
+    if (rc != LQSGD_OK) return rc;
+    if (!ptrs[vbase + nv * W + vi] && !ptrs[vbase + nv * (W + 1) + vi]) return LQSGD_ERR_INVALID_ARG;
   }
   if (!c->ptrs_valid || ptrs != c->ptrs_host) {
     c->ptrs_host = ptrs;
@@ -560,6 +570,8 @@ int lqsgd_step(lqsgd_ctx* c, const float* const* grads, float* const* ghat, void
   t.layers = p.d_layers;
   t.grads = reinterpret_cast<const float* const*>(p.d_ptrs);
   t.ghat = reinterpret_cast<float* const*>(p.d_ptrs + nm * W);
+  t.weights = weights ? reinterpret_cast<float* const*>(p.d_ptrs + nm * (W + 1)) : nullptr;
+  t.lr = lr;
   t.payload = p.d_payload;
   t.payload_stride = p.payload_stride;
   t.status = p.d_status;
@@ -572,8 +584,9 @@ int lqsgd_step(lqsgd_ctx* c, const float* const* grads, float* const* ghat, void
   if (nv) {
     CK(launch_vectors(p.d_vecs, p.d_chV, (int)p.chV.size(),
                       reinterpret_cast<const float* const*>(p.d_ptrs + vbase),
-                      reinterpret_cast<float* const*>(p.d_ptrs + vbase + nv * W), p.d_payload,
-                      p.payload_stride, W, {st, 0}));
+                      reinterpret_cast<float* const*>(p.d_ptrs + vbase + nv * W),
+                      weights ? reinterpret_cast<float* const*>(p.d_ptrs + vbase + nv * (W + 1)) : nullptr, lr,
+                      p.d_payload, p.payload_stride, W, {st, 0}));
   }
   if (nm) CK(cudaMemsetAsync(p.d_status, 0, nm * sizeof(uint32_t), st));
   PHASE_MARK(0);
@@ -604,6 +617,17 @@ int lqsgd_step(lqsgd_ctx* c, const float* const* grads, float* const* ghat, void
   PHASE_MARK(5);
 #undef PHASE_MARK
   return LQSGD_OK;
+}
+
+int lqsgd_step(lqsgd_ctx* c, const float* const* grads, float* const* ghat, void* cuda_stream) {
+  if (!ghat) return LQSGD_ERR_INVALID_ARG;
+  return step_impl(c, grads, ghat, nullptr, 0.f, cuda_stream);
+}
+
+int lqsgd_step_update(lqsgd_ctx* c, const float* const* grads, float* const* ghat, float* const* weights, float lr,
+                      void* cuda_stream) {
+  if (!weights) return LQSGD_ERR_INVALID_ARG;
+  return step_impl(c, grads, ghat, weights, lr, cuda_stream);
 }
 
 int lqsgd_step_host(lqsgd_ctx* c, const float* const* host_grads, float* const* host_ghat,

@@ -70,7 +70,9 @@ struct ExchangeChunk {
 struct Tables {
   const LayerDev* layers;
   const float* const* grads;  // [n_mat][W] device pointers, by LayerDev index
-  float* const* ghat;         // [n_mat]
+  float* const* ghat;         // [n_mat]; an entry may be null: G_hat of that layer is not written
+  float* const* weights;      // [n_mat] or null; non-null entry: w <- w - lr * G_hat in pass 3 (Alg. 1 model update)
+  float lr;
   uint8_t* payload;           // [W][payload_stride]
   uint64_t payload_stride;
   uint32_t* status;           // [n_mat]
@@ -122,8 +124,8 @@ cudaError_t launch_pass2(int RP, const Tables& t, const Tile* tiles, int ntiles,
 cudaError_t launch_q_reduce(int RP, const Tables& t, const FactorBlock* fb, int nfb, Launch l);
 cudaError_t launch_pass3(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
 cudaError_t launch_vectors(const VectorDev* vecs, const ExchangeChunk* chunks, int nchunks,
-                           const float* const* vgrads, float* const* vghat, uint8_t* payload,
-                           uint64_t payload_stride, int W, Launch l);
+                           const float* const* vgrads, float* const* vghat, float* const* vweights, float lr,
+                           uint8_t* payload, uint64_t payload_stride, int W, Launch l);
 // Bulk-copy staged passes (lqsgd_stream.cu): layers with m % 4 == 0 and RP <= 8.  One CTA per SM,
 // 512 consumer threads.  The copy engine limits the number of bulk copies in flight, not their
 // bytes, so tiles are wide (few, large row segments per stage) and a tile that spans whole rows

@@ -359,7 +359,9 @@ __device__ __forceinline__ void pass3_tile(const Tables& t, const Tile& tl) {
   const int m = L.m, W = t.W;
   const size_t plane = (size_t)L.n * m;
   float* __restrict__ E = L.E;
-  float* __restrict__ Gh = t.ghat[tl.layer];
+  float* __restrict__ Gh = t.ghat[tl.layer];                                  // may be null
+  float* __restrict__ Wt = t.weights ? t.weights[tl.layer] : nullptr;         // may be null
+  const float lr = t.lr;
   const float* __restrict__ Pbar = L.Pbar;
   const ColMap cm = col_map<VEC>(tl);
   if (!cm.active) return;
@@ -396,7 +398,13 @@ __device__ __forceinline__ void pass3_tile(const Tables& t, const Tile& tl) {
           for (int j = 0; j < RP; ++j) s = fmaf(p[j], q[k * RP + j], s);
           gh[u].v[k] = s;
         }
-        st_stream<VEC>(Gh + (size_t)i * m + col, gh[u]);
+        if (Gh) st_stream<VEC>(Gh + (size_t)i * m + col, gh[u]);
+        if (Wt) {                                  // model update of Alg. 1: w <- w - lr * G_hat
+          Pack<VEC> wv = ld_stream<VEC>(Wt + (size_t)i * m + col);
+#pragma unroll
+          for (int k = 0; k < VEC; ++k) wv.v[k] = fmaf(-lr, gh[u].v[k], wv.v[k]);
+          st_stream<VEC>(Wt + (size_t)i * m + col, wv);
+        }
       }
     }
     for (int w = 0; w < W; ++w) {
@@ -780,7 +788,7 @@ q_transpose_kernel(const float* __restrict__ Q, float* __restrict__ Qt, int m, i
 __global__ void __launch_bounds__(256)
 vectors_kernel(const VectorDev* __restrict__ vecs, const ExchangeChunk* __restrict__ chunks,
                const float* const* __restrict__ vgrads, float* const* __restrict__ vghat,
-               uint8_t* payload, uint64_t payload_stride, int W) {
+               float* const* __restrict__ vweights, float lr, uint8_t* payload, uint64_t payload_stride, int W) {
   pdl_wait();
   const ExchangeChunk ch = chunks[blockIdx.x];
   const VectorDev v = vecs[ch.layer];
@@ -792,7 +800,9 @@ vectors_kernel(const VectorDev* __restrict__ vecs, const ExchangeChunk* __restri
     reinterpret_cast<float*>(payload + (size_t)w * payload_stride + v.pay_off)[i] = x;
     s += x;
   }
-  vghat[ch.layer][i] = s / (float)W;
+  const float mean = s / (float)W;
+  if (vghat[ch.layer]) vghat[ch.layer][i] = mean;
+  if (vweights && vweights[ch.layer]) vweights[ch.layer][i] = fmaf(-lr, mean, vweights[ch.layer][i]);
 }
 
 }  // namespace
@@ -859,10 +869,10 @@ cudaError_t launch_exchange(int rp, int which, const Tables& t, const QuantTable
 }
 
 cudaError_t launch_vectors(const VectorDev* vecs, const ExchangeChunk* chunks, int nchunks,
-                           const float* const* vgrads, float* const* vghat, uint8_t* payload,
-                           uint64_t payload_stride, int W, Launch l) {
+                           const float* const* vgrads, float* const* vghat, float* const* vweights, float lr,
+                           uint8_t* payload, uint64_t payload_stride, int W, Launch l) {
   if (nchunks == 0) return cudaSuccess;
-  launch_pdl(vectors_kernel, nchunks, 256, 0, l.stream, vecs, chunks, vgrads, vghat, payload, payload_stride, W);
+  launch_pdl(vectors_kernel, nchunks, 256, 0, l.stream, vecs, chunks, vgrads, vghat, vweights, lr, payload, payload_stride, W);
   return cudaGetLastError();
 }
 

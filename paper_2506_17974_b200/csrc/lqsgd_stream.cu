@@ -219,7 +219,11 @@ __device__ __forceinline__ bool pass3_consume(const Tables& t, const TileCtx& c,
   const int row_f4 = c.ncols >> 2, m = c.m, W = t.W;
   float q[QPT * 4 * RP];
   load_q<RP, QPT>(L.Qt, L.mt, c.col0, geo, o, q);
-  float* Gh = t.ghat[c.layer] + (size_t)c.row0 * m + c.col0;
+  float* Gh0 = t.ghat[c.layer];                                            // may be null
+  float* Wt0 = t.weights ? t.weights[c.layer] : nullptr;                   // may be null
+  float* Gh = Gh0 ? Gh0 + (size_t)c.row0 * m + c.col0 : nullptr;
+  float* Wt = Wt0 ? Wt0 + (size_t)c.row0 * m + c.col0 : nullptr;
+  const float step = t.lr;
   for (int sr = 0; sr < c.nrows; sr += geo.R) {
     const int rows = min(geo.R, c.nrows - sr);
     float4 gh[RPT * QPT];
@@ -242,8 +246,17 @@ __device__ __forceinline__ bool pass3_consume(const Tables& t, const TileCtx& c,
           }
           gh[u * QPT + k] = make_float4(a0, a1, a2, a3);
           const int quad = o.cq + k * kConsumers;
-          if (o.in_group && lr < rows && quad < geo.quads)
-            __stcs(reinterpret_cast<float4*>(Gh + (size_t)(sr + lr) * m) + quad, gh[u * QPT + k]);
+          if (o.in_group && lr < rows && quad < geo.quads) {
+            const float4 g4 = gh[u * QPT + k];
+            if (Gh) __stcs(reinterpret_cast<float4*>(Gh + (size_t)(sr + lr) * m) + quad, g4);
+            if (Wt) {                              // model update of Alg. 1: w <- w - lr * G_hat
+              float4* wp = reinterpret_cast<float4*>(Wt + (size_t)(sr + lr) * m) + quad;
+              float4 wv = __ldcs(wp);
+              wv.x = fmaf(-step, g4.x, wv.x); wv.y = fmaf(-step, g4.y, wv.y);
+              wv.z = fmaf(-step, g4.z, wv.z); wv.w = fmaf(-step, g4.w, wv.w);
+              __stcs(wp, wv);
+            }
+          }
         }
       }
     }

@@ -317,3 +317,31 @@ def test_planted_rank_r_gradient_is_recovered_on_the_device():
     torch.cuda.synchronize()
     assert par.rel_fro(par.host(out), par.host(G)) <= 1e-5
     assert float(comp.get_state(B.STATE_E, 0, 0).abs().max()) <= 1e-4 * float(G.abs().max())
+
+
+def test_fused_model_update_matches_separate_update():
+    """Algorithm 1's last line, w <- w - lr * G_hat, fused into pass 3: same weights as updating
+    from the G_hat a plain step returns (and as the oracle's G_hat), with and without G_hat output."""
+    w = dataclasses.replace(wl.config2(), workers=2)          # includes a 32 x 25 layer and 1-D tensors
+    a, b, c = make(w), make(w), make(w)
+    lr = 0.125
+    gen = torch.Generator(DEV).manual_seed(1)
+    w0 = [torch.randn(s, device=DEV, generator=gen) for s in w.layers]
+    wb = [x.clone() for x in w0]
+    wc = [x.clone() for x in w0]
+    for t in range(2):
+        g = wl.draw_gradients(w, t, device=DEV)
+        gh_a = [torch.empty(s, device=DEV) for s in w.layers]
+        gh_b = [torch.empty(s, device=DEV) for s in w.layers]
+        a.step(g, gh_a)
+        b.step_update(g, gh_b, wb, lr)
+        c.step_update(g, None, wc, lr)
+        torch.cuda.synchronize()
+        for l in range(len(w.layers)):
+            assert torch.equal(gh_a[l], gh_b[l])
+            w0[l] = torch.addcmul(w0[l], gh_a[l], torch.tensor(-lr, device=DEV))   # fp32 reference update
+            assert torch.allclose(wb[l], w0[l], rtol=0, atol=1e-6 * float(w0[l].abs().max()))
+            assert torch.equal(wb[l], wc[l])
+    assert torch.equal(a.get_state(B.STATE_E, 2, 1), c.get_state(B.STATE_E, 2, 1))
+    with pytest.raises(B.LqsgdError):                          # a layer with neither output nor weights
+        c.step_update(wl.draw_gradients(w, 0, device=DEV), None, [None] * len(w.layers), lr)
