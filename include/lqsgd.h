@@ -95,6 +95,8 @@ typedef struct lqsgd_config {
   int32_t workers;      /* W, 1..256 */
   uint64_t seed;        /* seed of Q_0 ~ N(0,1) (Alg. 1 initialisation) */
   uint32_t flags;       /* LQSGD_FLAG_* */
+  int32_t world_workers; /* 0, or the number of workers of ALL processes taking part in the averages when the
+                            workers are spread over several GPUs (a multiple of `workers`); see lqsgd_round_begin */
 } lqsgd_config;
 
 /* Where one layer's data sits inside a worker's payload (byte offsets from the payload start). */
@@ -160,6 +162,41 @@ int lqsgd_step(lqsgd_ctx* ctx, const float* const* host_grads, float* const* hos
  * Everything else as lqsgd_step. */
 int lqsgd_step_update(lqsgd_ctx* ctx, const float* const* host_grads, float* const* host_ghat,
                       float* const* host_weights, float lr, void* cuda_stream);
+
+/* ---- Workers on several GPUs: the round in pieces, with the exchanges left to the caller. ----
+ * Algorithm 1 sends the quantised factors "across workers via All-Reduce" twice per iteration.
+ * With the workers of one process on one GPU that exchange is a sum inside lqsgd_step.  When
+ * other processes hold more workers (config.world_workers = total over all ranks, each rank
+ * simulating `workers` of them), a rank runs the round as
+ *
+ *   lqsgd_round_begin(grads, ghat, weights, lr)   pass 1, Orthonormalize, local scales of P
+ *   all-reduce MAX over ranks of  view(LQSGD_XCHG_SCALES_P)     (one fp32 per matrix)
+ *   lqsgd_round_pack(0)                            quantise + pack this rank's P with those scales
+ *   all-gather of                 view(LQSGD_XCHG_STREAMS_P)    (workers x P-stream bytes, contiguous)
+ *   lqsgd_round_reduce(0, gathered, n_ranks)       exact integer sum over ALL workers' codes,
+ *                                                  Eq. 5, pass 2, local scales of Q
+ *   all-reduce MAX of view(LQSGD_XCHG_SCALES_Q);  lqsgd_round_pack(1);  all-gather of
+ *   view(LQSGD_XCHG_STREAMS_Q);  lqsgd_round_reduce(1, gathered, n_ranks)
+ *   lqsgd_round_end()                              pass 3 (G_hat, E, optional model update)
+ *
+ * The collectives run on the same stream between the calls (NCCL, or any other transport: the
+ * library only reads and writes the buffers).  `gathered` is n_ranks x the bytes of the STREAMS
+ * view, rank after rank, in caller memory.  The wire carries exactly the b-bit streams
+ * (r(n+m)b bits per worker, Section IV-C) plus one scale per factor and layer.  Results are
+ * identical, bit for bit, to one process simulating all world_workers workers.  G_hat of a
+ * 1-D tensor comes out as this rank's share of the mean (local sum / world_workers): sum it
+ * over the ranks.  Calls out of order return LQSGD_ERR_INVALID_ARG; the bits = 32 bypass is not
+ * available across ranks.  ghat / weights as in lqsgd_step_update (weights may be NULL). */
+#define LQSGD_XCHG_SCALES_P 0
+#define LQSGD_XCHG_SCALES_Q 1
+#define LQSGD_XCHG_STREAMS_P 2
+#define LQSGD_XCHG_STREAMS_Q 3
+int lqsgd_round_begin(lqsgd_ctx* ctx, const float* const* host_grads, float* const* host_ghat,
+                      float* const* host_weights, float lr, void* cuda_stream);
+int lqsgd_round_pack(lqsgd_ctx* ctx, int32_t which, void* cuda_stream);
+int lqsgd_round_reduce(lqsgd_ctx* ctx, int32_t which, const void* dev_gathered, int32_t n_ranks, void* cuda_stream);
+int lqsgd_round_end(lqsgd_ctx* ctx, void* cuda_stream);
+int lqsgd_exchange_view(const lqsgd_ctx* ctx, int32_t which, void** dev_ptr_out, size_t* host_bytes_out);
 
 /* Same round with HOST tensors: copies every gradient host->device into the staging area,
  * runs lqsgd_step, copies every G_hat and all W payloads device->host, and synchronises the

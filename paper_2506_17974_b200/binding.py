@@ -23,6 +23,7 @@ FLAG_HOST_STAGING = 1
 FLAG_REGISTER_PATH = 2
 STATUS_TIMEOUT = 16
 N_PHASES = 5
+XCHG_SCALES_P, XCHG_SCALES_Q, XCHG_STREAMS_P, XCHG_STREAMS_Q = range(4)
 PHASE_NAMES = ("pass1", "finish_p", "pass2", "finish_q", "pass3")
 
 ERR_INVALID_ARG, ERR_BAD_SHAPE, ERR_WORKSPACE_TOO_SMALL, ERR_MISALIGNED = -1, -2, -3, -4
@@ -34,6 +35,7 @@ EXPORTED = [
     "lqsgd_workspace_bytes", "lqsgd_create", "lqsgd_step", "lqsgd_step_update", "lqsgd_step_host", "lqsgd_payload_bytes",
     "lqsgd_payload", "lqsgd_payload_layout", "lqsgd_get_state", "lqsgd_set_state", "lqsgd_status",
     "lqsgd_orthonormalize_noalloc",
+    "lqsgd_round_begin", "lqsgd_round_pack", "lqsgd_round_reduce", "lqsgd_round_end", "lqsgd_exchange_view",
     "lqsgd_launches_per_step", "lqsgd_set_phase_events", "lqsgd_destroy", "lqsgd_strerror", "lqsgd_last_cuda_error", "lqsgd_version",
 ]
 
@@ -45,7 +47,7 @@ class Shape(C.Structure):
 class Config(C.Structure):
     _fields_ = [("struct_size", C.c_uint32), ("rank", C.c_int32), ("bits_p", C.c_int32),
                 ("bits_q", C.c_int32), ("alpha", C.c_float), ("workers", C.c_int32),
-                ("seed", C.c_uint64), ("flags", C.c_uint32)]
+                ("seed", C.c_uint64), ("flags", C.c_uint32), ("world_workers", C.c_int32)]
 
 
 class LayerLayout(C.Structure):
@@ -77,6 +79,11 @@ def load_library() -> C.CDLL:
     lib.lqsgd_step.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), vp]
     lib.lqsgd_step_update.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.c_float, vp]
     lib.lqsgd_step_host.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), vp, vp]
+    lib.lqsgd_round_begin.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.c_float, vp]
+    lib.lqsgd_round_pack.argtypes = [vp, i32, vp]
+    lib.lqsgd_round_reduce.argtypes = [vp, i32, vp, i32, vp]
+    lib.lqsgd_round_end.argtypes = [vp, vp]
+    lib.lqsgd_exchange_view.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(sz)]
     lib.lqsgd_payload_bytes.argtypes = [vp, C.POINTER(sz)]
     lib.lqsgd_payload.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(sz)]
     lib.lqsgd_payload_layout.argtypes = [vp, i32, C.POINTER(LayerLayout)]
@@ -113,8 +120,8 @@ def _shapes(layers: Sequence[Tuple[int, int]]):
 
 
 def make_config(rank: int, bits_p: int, bits_q: int, alpha: float, workers: int, seed: int = 0,
-                flags: int = 0) -> Config:
-    return Config(C.sizeof(Config), rank, bits_p, bits_q, alpha, workers, seed, flags)
+                flags: int = 0, world_workers: int = 0) -> Config:
+    return Config(C.sizeof(Config), rank, bits_p, bits_q, alpha, workers, seed, flags, world_workers)
 
 
 def orthonormalize_noalloc(p_in: torch.Tensor, p_out: torch.Tensor, status: Optional[torch.Tensor] = None,
@@ -143,7 +150,7 @@ class LQSGD:
 
     def __init__(self, layers: Sequence[Tuple[int, int]], rank: int, bits_p: int, bits_q: Optional[int] = None,
                  alpha: float = 127.0, workers: int = 1, seed: int = 0, host_staging: bool = False,
-                 device: str = "cuda:0", register_path: bool = False):
+                 device: str = "cuda:0", register_path: bool = False, world_workers: int = 0):
         self.lib = load_library()
         self.layers = [(int(n), int(m)) for n, m in layers]
         self.rank, self.bits_p = rank, bits_p
@@ -152,7 +159,7 @@ class LQSGD:
         self.device = torch.device(device)
         self.cfg = make_config(rank, self.bits_p, self.bits_q, alpha, workers, seed,
                                (FLAG_HOST_STAGING if host_staging else 0)
-                               | (FLAG_REGISTER_PATH if register_path else 0))
+                               | (FLAG_REGISTER_PATH if register_path else 0), world_workers)
         nbytes = workspace_bytes(self.layers, self.cfg)
         with torch.cuda.device(self.device):
             self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
@@ -240,6 +247,34 @@ class LQSGD:
         wt = (C.c_void_p * nl)(*[(t.data_ptr() if t is not None else None) for t in weights])
         s = stream if stream is not None else torch.cuda.current_stream(self.device)
         _check(self.lib.lqsgd_step_update(self.ctx, g, h, wt, C.c_float(lr), C.c_void_p(s.cuda_stream)))
+
+    # -- the round in pieces (workers on several GPUs; see paper_2506_17974_b200/distributed.py)
+    def round_begin(self, grads, ghat, weights=None, lr: float = 0.0) -> None:
+        nl = len(self.layers)
+        g = (C.c_void_p * (self.W * nl))()
+        for w in range(self.W):
+            for l in range(nl):
+                g[w * nl + l] = grads[w][l].data_ptr()
+        h = (C.c_void_p * nl)(*[(t.data_ptr() if t is not None else None) for t in ghat]) if ghat is not None else None
+        wt = (C.c_void_p * nl)(*[(t.data_ptr() if t is not None else None) for t in weights]) if weights is not None else None
+        _check(self.lib.lqsgd_round_begin(self.ctx, g, h, wt, C.c_float(lr), self._stream_ptr()))
+
+    def round_pack(self, which: int) -> None:
+        _check(self.lib.lqsgd_round_pack(self.ctx, which, self._stream_ptr()))
+
+    def round_reduce(self, which: int, gathered: torch.Tensor, n_ranks: int) -> None:
+        _check(self.lib.lqsgd_round_reduce(self.ctx, which, C.c_void_p(gathered.data_ptr()), n_ranks, self._stream_ptr()))
+
+    def round_end(self) -> None:
+        _check(self.lib.lqsgd_round_end(self.ctx, self._stream_ptr()))
+
+    def exchange_view(self, which: int) -> torch.Tensor:
+        """The exchange buffer `which` (XCHG_*) as a tensor aliasing the workspace: fp32 scales or uint8 streams."""
+        ptr, nb = C.c_void_p(), C.c_size_t(0)
+        _check(self.lib.lqsgd_exchange_view(self.ctx, which, C.byref(ptr), C.byref(nb)))
+        off = ptr.value - self.workspace.data_ptr()
+        raw = self.workspace[off:off + nb.value]
+        return raw.view(torch.float32) if which in (XCHG_SCALES_P, XCHG_SCALES_Q) else raw
 
     def step_host(self, grads, ghat, payload: Optional[torch.Tensor] = None,
                   stream: Optional[torch.cuda.Stream] = None) -> None:

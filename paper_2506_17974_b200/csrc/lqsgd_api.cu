@@ -48,7 +48,7 @@ struct MatHost {
 };
 
 struct Plan {
-  int RP = 0, W = 0;
+  int RP = 0, W = 0, W_total = 0;             // W_total: workers of all ranks (== W on one GPU)
   std::vector<MatHost> mats;
   std::vector<LayerDev> layers;
   std::vector<VectorDev> vecs;
@@ -72,6 +72,9 @@ struct Plan {
   void** d_ptrs = nullptr;                    // see step_impl for the layout
   uint32_t* d_status = nullptr;
   uint8_t* d_payload = nullptr;
+  float* d_xscales = nullptr;                 // [2][n_mat] scales the ranks agree on (split exchange)
+  uint8_t* d_xsend[2] = {nullptr, nullptr};   // [W][region_bytes]: local P / Q streams, contiguous, for the all-gather
+  uint64_t region_off[2] = {0, 0}, region_bytes[2] = {0, 0};
   float* d_stage_g = nullptr;                 // [W][elems_total]
   float* d_stage_ghat = nullptr;              // [elems_total]
   size_t state_begin = 0, state_end = 0;      // byte range to zero at create (E, factors, codes ...)
@@ -88,6 +91,10 @@ int check_config(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
   if (!bits_ok(c->bits_p) || !bits_ok(c->bits_q)) return LQSGD_ERR_INVALID_ARG;
   if (!(c->alpha > 0.f) || !std::isfinite(c->alpha)) return LQSGD_ERR_INVALID_ARG;
   if (c->workers < 1 || c->workers > 256) return LQSGD_ERR_INVALID_ARG;
+  if (c->world_workers != 0) {     // workers of all ranks: a multiple of the local ones; no bypass mode across ranks
+    if (c->world_workers < c->workers || c->world_workers > 4096 || c->world_workers % c->workers) return LQSGD_ERR_INVALID_ARG;
+    if (c->world_workers > c->workers && (c->bits_p == 32 || c->bits_q == 32)) return LQSGD_ERR_INVALID_ARG;
+  }
   if (c->flags & ~(LQSGD_FLAG_HOST_STAGING | LQSGD_FLAG_REGISTER_PATH)) return LQSGD_ERR_INVALID_ARG;
   for (int i = 0; i < n_layers; ++i) {
     if (shapes[i].rows < 1 || shapes[i].cols < 1) return LQSGD_ERR_BAD_SHAPE;
@@ -133,6 +140,7 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   const int W = cfg.workers, RP = padded_rank(cfg.rank);
   p.RP = RP;
   p.W = W;
+  p.W_total = cfg.world_workers > 0 ? cfg.world_workers : W;
   p.layout.assign(n_layers, lqsgd_layer_layout{});
   p.elem_off.resize(n_layers);
   for (int i = 0; i < n_layers; ++i) {
@@ -164,6 +172,12 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
     lo.q_offset = off; lo.q_bytes = ((size_t)mt.m * mt.r * cfg.bits_q + 7) / 8; off += lo.q_bytes;
   }
   p.payload_bytes = off;
+  if (!p.mats.empty()) {
+    const auto& first = p.layout[p.mats.front().user_index];
+    const auto& last = p.layout[p.mats.back().user_index];
+    p.region_off[0] = first.p_offset; p.region_bytes[0] = last.p_offset + last.p_bytes - first.p_offset;
+    p.region_off[1] = first.q_offset; p.region_bytes[1] = last.q_offset + last.q_bytes - first.q_offset;
+  }
   p.payload_stride = align_up(off, 16);
 
   // ---- tile sizes
@@ -328,10 +342,13 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   std::reverse(p.tiles2.begin(), p.tiles2.end());
   p.d_status = a.take<uint32_t>(p.mats.size());
   p.d_payload = a.take<uint8_t>((size_t)W * p.payload_stride);
+  p.d_xscales = a.take<float>(2 * p.mats.size());
+  p.d_xsend[0] = a.take<uint8_t>((size_t)W * p.region_bytes[0]);
+  p.d_xsend[1] = a.take<uint8_t>((size_t)W * p.region_bytes[1]);
   p.state_end = a.off;
 
-  quant_tables(cfg.bits_p, cfg.alpha, W, p.thrP, p.deqP);
-  quant_tables(cfg.bits_q, cfg.alpha, W, p.thrQ, p.deqQ);
+  quant_tables(cfg.bits_p, cfg.alpha, p.W_total, p.thrP, p.deqP);
+  quant_tables(cfg.bits_q, cfg.alpha, p.W_total, p.thrQ, p.deqQ);
   p.d_tiles1 = a.take<Tile>(p.tiles1.size());
   p.d_tiles2 = a.take<Tile>(p.tiles2.size());
   p.d_tiles3 = a.take<Tile>(p.tiles3.size());
@@ -383,6 +400,9 @@ struct lqsgd_ctx {
   void* workspace = nullptr;
   cudaEvent_t phase_events[LQSGD_N_PHASES + 1];
   bool have_events = false;
+  Tables tables{};                   // filled by prepare_step
+  bool has_weights = false;
+  int round_stage = 0;               // progress of a split round (lqsgd_round_*)
 };
 
 extern "C" {
@@ -516,10 +536,10 @@ int lqsgd_launches_per_step(const lqsgd_ctx* ctx, int32_t* out) {
   return LQSGD_OK;
 }
 
-// The round, with the optional model update.  ghat == nullptr (only with weights): G_hat is not
+// Checks and uploads the step's pointers and fills the kernels' table.  ghat == nullptr (only with weights): G_hat is not
 // written.  Pointer table: [grads nm*W | ghat nm | weights nm | vgrads nv*W | vghat nv | vweights nv].
-static int step_impl(lqsgd_ctx* c, const float* const* grads, float* const* ghat, float* const* weights, float lr,
-                     void* cuda_stream) {
+static int prepare_step(lqsgd_ctx* c, const float* const* grads, float* const* ghat, float* const* weights, float lr,
+                        void* cuda_stream) {
   if (!c || !grads || (!ghat && !weights)) return LQSGD_ERR_INVALID_ARG;
   Plan& p = c->plan;
   const int W = p.W, nl = (int)c->shapes.size();
@@ -566,7 +586,7 @@ static int step_impl(lqsgd_ctx* c, const float* const* grads, float* const* ghat
     CK(cudaMemcpyAsync(p.d_ptrs, c->ptrs_host.data(), ptrs.size() * sizeof(void*), cudaMemcpyHostToDevice, st));
     c->ptrs_valid = true;
   }
-  Tables t;
+  Tables& t = c->tables;
   t.layers = p.d_layers;
   t.grads = reinterpret_cast<const float* const*>(p.d_ptrs);
   t.ghat = reinterpret_cast<float* const*>(p.d_ptrs + nm * W);
@@ -576,46 +596,100 @@ static int step_impl(lqsgd_ctx* c, const float* const* grads, float* const* ghat
   t.payload_stride = p.payload_stride;
   t.status = p.d_status;
   t.W = W;
+  c->has_weights = weights != nullptr;
+  return LQSGD_OK;
+}
+
+// The launch sequence, cut into the segments between which a multi-GPU run exchanges data.
+//   0: 1-D tensors, pass 1, Orthonormalize (+ local scales of P when split)
+//   1: exchange of P - fused (quantise, pack, sum, dequantise) or, when split, quantise + pack only
+//   2: (split: sum over all ranks' streams + dequantise P) pass 2, Q_w (+ local scales of Q when split)
+//   3: exchange of Q, as segment 1
+//   4: (split: sum + dequantise Q)     5: pass 3
+static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, int n_streams, cudaStream_t st) {
+  Plan& p = c->plan;
+  const Tables& t = c->tables;
+  const int W = p.W, RP = p.RP;
+  const size_t nm = p.mats.size(), nv = p.vecs.size();
+  const size_t vbase = nm * (W + 2);
   const QuantTables qp{p.d_thrP, p.d_deqP, c->cfg.bits_p}, qq{p.d_thrQ, p.d_deqQ, c->cfg.bits_q};
-  const int RP = p.RP;
-  const bool ev = c->have_events;
-  c->have_events = false;
+  SplitExchange sx{};
+  sx.pack_only = split ? 1 : 0;
+  sx.n_mat = (int)nm;
+  sx.scales = p.d_xscales;
+  sx.send[0] = p.d_xsend[0]; sx.send[1] = p.d_xsend[1];
+  sx.region_bytes[0] = p.region_bytes[0]; sx.region_bytes[1] = p.region_bytes[1];
+  sx.region_off[0] = p.region_off[0]; sx.region_off[1] = p.region_off[1];
+  const bool ev = c->have_events && !split;
 #define PHASE_MARK(i) do { if (ev) CK(cudaEventRecord(c->phase_events[i], st)); } while (0)
-  if (nv) {
-    CK(launch_vectors(p.d_vecs, p.d_chV, (int)p.chV.size(),
-                      reinterpret_cast<const float* const*>(p.d_ptrs + vbase),
-                      reinterpret_cast<float* const*>(p.d_ptrs + vbase + nv * W),
-                      weights ? reinterpret_cast<float* const*>(p.d_ptrs + vbase + nv * (W + 1)) : nullptr, lr,
-                      p.d_payload, p.payload_stride, W, {st, 0}));
+  switch (seg) {
+    case 0:
+      if (nv) {
+        CK(launch_vectors(p.d_vecs, p.d_chV, (int)p.chV.size(),
+                          reinterpret_cast<const float* const*>(p.d_ptrs + vbase),
+                          reinterpret_cast<float* const*>(p.d_ptrs + vbase + nv * W),
+                          c->has_weights ? reinterpret_cast<float* const*>(p.d_ptrs + vbase + nv * (W + 1)) : nullptr,
+                          t.lr, p.d_payload, p.payload_stride, W, p.W_total, {st, 0}));
+      }
+      if (nm) CK(cudaMemsetAsync(p.d_status, 0, nm * sizeof(uint32_t), st));
+      PHASE_MARK(0);
+      if (nm) {
+        CK(launch_pass1(RP, t, p.d_tiles1, (int)p.tiles1.size(), {st, c->grid1}));
+        CK(launch_stream_pass1(RP, t, p.d_stiles1, (int)p.stiles1.size(), {st, (int)std::min<size_t>(p.stiles1.size(), c->sm_count)}));
+      }
+      PHASE_MARK(1);
+      if (nm) {
+        CK(launch_p_reduce_gram(RP, t, p.d_fbP, (int)p.fbP.size(), {st, 0}));
+        CK(launch_p_apply(RP, t, p.d_fbP, (int)p.fbP.size(), {st, 0}));
+        if (split) CK(launch_scale_reduce(t, 0, p.d_xscales, (int)nm, {st, 0}));
+      }
+      break;
+    case 1:
+      if (nm) CK(launch_exchange(RP, 0, t, qp, p.d_chP, (int)p.chP.size(), sx, {st, 0}));
+      PHASE_MARK(2);
+      break;
+    case 2:
+      if (nm) {
+        if (split) CK(launch_sum_dequant(RP, 0, t, qp, p.d_chP, (int)p.chP.size(), sx, static_cast<const uint8_t*>(gathered), n_streams, {st, 0}));
+        CK(launch_pass2(RP, t, p.d_tiles2, (int)p.tiles2.size(), {st, c->grid2}));
+      }
+      PHASE_MARK(3);
+      if (nm) {
+        CK(launch_q_reduce(RP, t, p.d_fbQ, (int)p.fbQ.size(), {st, 0}));
+        if (split) CK(launch_scale_reduce(t, 1, p.d_xscales, (int)nm, {st, 0}));
+      }
+      break;
+    case 3:
+      if (nm) CK(launch_exchange(RP, 1, t, qq, p.d_chQ, (int)p.chQ.size(), sx, {st, 0}));
+      PHASE_MARK(4);
+      break;
+    case 4:
+      if (nm && split) CK(launch_sum_dequant(RP, 1, t, qq, p.d_chQ, (int)p.chQ.size(), sx, static_cast<const uint8_t*>(gathered), n_streams, {st, 0}));
+      break;
+    case 5:
+      if (nm) {
+        CK(launch_pass3(RP, t, p.d_tiles3, (int)p.tiles3.size(), {st, c->grid3}));
+        CK(launch_stream_pass3(RP, t, p.d_stiles3, (int)p.stiles3.size(), {st, (int)std::min<size_t>(p.stiles3.size(), c->sm_count)}));
+      }
+      PHASE_MARK(5);
+      break;
+    default: return LQSGD_ERR_INVALID_ARG;
   }
-  if (nm) CK(cudaMemsetAsync(p.d_status, 0, nm * sizeof(uint32_t), st));
-  PHASE_MARK(0);
-  if (nm) {
-    CK(launch_pass1(RP, t, p.d_tiles1, (int)p.tiles1.size(), {st, c->grid1}));
-    CK(launch_stream_pass1(RP, t, p.d_stiles1, (int)p.stiles1.size(), {st, (int)std::min<size_t>(p.stiles1.size(), c->sm_count)}));
-  }
-  PHASE_MARK(1);
-  if (nm) {
-    CK(launch_p_reduce_gram(RP, t, p.d_fbP, (int)p.fbP.size(), {st, 0}));
-    CK(launch_p_apply(RP, t, p.d_fbP, (int)p.fbP.size(), {st, 0}));
-    CK(launch_exchange(RP, 0, t, qp, p.d_chP, (int)p.chP.size(), {st, 0}));
-  }
-  PHASE_MARK(2);
-  if (nm) {
-    CK(launch_pass2(RP, t, p.d_tiles2, (int)p.tiles2.size(), {st, c->grid2}));
-  }
-  PHASE_MARK(3);
-  if (nm) {
-    CK(launch_q_reduce(RP, t, p.d_fbQ, (int)p.fbQ.size(), {st, 0}));
-    CK(launch_exchange(RP, 1, t, qq, p.d_chQ, (int)p.chQ.size(), {st, 0}));
-  }
-  PHASE_MARK(4);
-  if (nm) {
-    CK(launch_pass3(RP, t, p.d_tiles3, (int)p.tiles3.size(), {st, c->grid3}));
-    CK(launch_stream_pass3(RP, t, p.d_stiles3, (int)p.stiles3.size(), {st, (int)std::min<size_t>(p.stiles3.size(), c->sm_count)}));
-  }
-  PHASE_MARK(5);
 #undef PHASE_MARK
+  return LQSGD_OK;
+}
+
+static int step_impl(lqsgd_ctx* c, const float* const* grads, float* const* ghat, float* const* weights, float lr,
+                     void* cuda_stream) {
+  int rc = prepare_step(c, grads, ghat, weights, lr, cuda_stream);
+  if (rc != LQSGD_OK) return rc;
+  if (c->plan.W_total != c->plan.W) return LQSGD_ERR_INVALID_ARG;   // workers elsewhere: use the lqsgd_round_* calls
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  for (int seg = 0; seg <= 5; ++seg) {
+    rc = run_segment(c, seg, false, nullptr, 0, st);
+    if (rc != LQSGD_OK) return rc;
+  }
+  c->have_events = false;
   return LQSGD_OK;
 }
 
@@ -628,6 +702,55 @@ int lqsgd_step_update(lqsgd_ctx* c, const float* const* grads, float* const* gha
                       void* cuda_stream) {
   if (!weights) return LQSGD_ERR_INVALID_ARG;
   return step_impl(c, grads, ghat, weights, lr, cuda_stream);
+}
+
+// ---- the same round in pieces, for workers spread over several GPUs (see include/lqsgd.h)
+int lqsgd_round_begin(lqsgd_ctx* c, const float* const* grads, float* const* ghat, float* const* weights, float lr,
+                      void* cuda_stream) {
+  const int rc = prepare_step(c, grads, ghat, weights, lr, cuda_stream);
+  if (rc != LQSGD_OK) return rc;
+  if (c->cfg.bits_p == 32 || c->cfg.bits_q == 32) return LQSGD_ERR_INVALID_ARG;
+  c->round_stage = 0;
+  const int rs = run_segment(c, 0, true, nullptr, 0, static_cast<cudaStream_t>(cuda_stream));
+  if (rs == LQSGD_OK) c->round_stage = 1;
+  return rs;
+}
+
+int lqsgd_round_pack(lqsgd_ctx* c, int32_t which, void* cuda_stream) {
+  if (!c || (which != 0 && which != 1)) return LQSGD_ERR_INVALID_ARG;
+  if (c->round_stage != (which ? 3 : 1)) return LQSGD_ERR_INVALID_ARG;       // out of order
+  const int rs = run_segment(c, which ? 3 : 1, true, nullptr, 0, static_cast<cudaStream_t>(cuda_stream));
+  if (rs == LQSGD_OK) c->round_stage += 1;
+  return rs;
+}
+
+int lqsgd_round_reduce(lqsgd_ctx* c, int32_t which, const void* dev_gathered, int32_t n_ranks, void* cuda_stream) {
+  if (!c || !dev_gathered || (which != 0 && which != 1)) return LQSGD_ERR_INVALID_ARG;
+  if (c->round_stage != (which ? 4 : 2)) return LQSGD_ERR_INVALID_ARG;       // out of order
+  if (n_ranks < 1 || n_ranks * c->plan.W != c->plan.W_total) return LQSGD_ERR_INVALID_ARG;
+  const int rs = run_segment(c, which ? 4 : 2, true, dev_gathered, c->plan.W_total, static_cast<cudaStream_t>(cuda_stream));
+  if (rs == LQSGD_OK) c->round_stage += 1;
+  return rs;
+}
+
+int lqsgd_round_end(lqsgd_ctx* c, void* cuda_stream) {
+  if (!c || c->round_stage != 5) return LQSGD_ERR_INVALID_ARG;
+  const int rs = run_segment(c, 5, true, nullptr, 0, static_cast<cudaStream_t>(cuda_stream));
+  c->round_stage = 0;
+  return rs;
+}
+
+int lqsgd_exchange_view(const lqsgd_ctx* c, int32_t which, void** dev_ptr, size_t* bytes) {
+  if (!c || !dev_ptr || !bytes) return LQSGD_ERR_INVALID_ARG;
+  const Plan& p = c->plan;
+  switch (which) {
+    case LQSGD_XCHG_SCALES_P: *dev_ptr = p.d_xscales; *bytes = 4 * p.mats.size(); break;
+    case LQSGD_XCHG_SCALES_Q: *dev_ptr = p.d_xscales + p.mats.size(); *bytes = 4 * p.mats.size(); break;
+    case LQSGD_XCHG_STREAMS_P: *dev_ptr = p.d_xsend[0]; *bytes = (size_t)p.W * p.region_bytes[0]; break;
+    case LQSGD_XCHG_STREAMS_Q: *dev_ptr = p.d_xsend[1]; *bytes = (size_t)p.W * p.region_bytes[1]; break;
+    default: return LQSGD_ERR_OUT_OF_RANGE;
+  }
+  return LQSGD_OK;
 }
 
 int lqsgd_step_host(lqsgd_ctx* c, const float* const* host_grads, float* const* host_ghat,

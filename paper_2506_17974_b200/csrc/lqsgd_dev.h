@@ -117,15 +117,29 @@ struct Launch {
 cudaError_t launch_pass1(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
 cudaError_t launch_p_reduce_gram(int RP, const Tables& t, const FactorBlock* fb, int nfb, Launch l);
 cudaError_t launch_p_apply(int RP, const Tables& t, const FactorBlock* fb, int nfb, Launch l);
+// Split exchange (workers on several GPUs).  pack_only: quantise and pack with the scales in
+// `scales` ([2][n_mat], agreed between the ranks) and also write the streams into `send`
+// ([which][W][region_bytes], contiguous, ready for an all-gather); no sum, no dequantisation.
+struct SplitExchange {
+  int32_t pack_only;
+  int32_t n_mat;
+  const float* scales;
+  uint8_t* send[2];
+  uint64_t region_bytes[2];   // bytes of all layers' P (or Q) streams of one worker
+  uint64_t region_off[2];     // offset of that region inside a payload
+};
 cudaError_t launch_exchange(int RP, int which /*0 = P, 1 = Q*/, const Tables& t, const QuantTables& q,
-                            const ExchangeChunk* ch, int nch, Launch l);
+                            const ExchangeChunk* ch, int nch, const SplitExchange& sx, Launch l);
+cudaError_t launch_scale_reduce(const Tables& t, int which, float* scales, int n_mat, Launch l);
+cudaError_t launch_sum_dequant(int RP, int which, const Tables& t, const QuantTables& q, const ExchangeChunk* ch,
+                               int nch, const SplitExchange& sx, const uint8_t* gathered, int n_streams, Launch l);
 cudaError_t launch_q_transpose(const float* Q, float* Qt, int m, int RP, int mt, cudaStream_t stream);
 cudaError_t launch_pass2(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
 cudaError_t launch_q_reduce(int RP, const Tables& t, const FactorBlock* fb, int nfb, Launch l);
 cudaError_t launch_pass3(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
 cudaError_t launch_vectors(const VectorDev* vecs, const ExchangeChunk* chunks, int nchunks,
                            const float* const* vgrads, float* const* vghat, float* const* vweights, float lr,
-                           uint8_t* payload, uint64_t payload_stride, int W, Launch l);
+                           uint8_t* payload, uint64_t payload_stride, int W, int W_total, Launch l);
 // Bulk-copy staged passes (lqsgd_stream.cu): layers with m % 4 == 0 and RP <= 8.  One CTA per SM,
 // 512 consumer threads.  The copy engine limits the number of bulk copies in flight, not their
 // bytes, so tiles are wide (few, large row segments per stage) and a tile that spans whole rows

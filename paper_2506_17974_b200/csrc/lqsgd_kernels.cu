@@ -642,7 +642,7 @@ q_reduce_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
 // ---------------------------------------------------------------------------------------
 template <int RP>
 __global__ void __launch_bounds__(256)
-exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __restrict__ chunks) {
+exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __restrict__ chunks, SplitExchange sx) {
   pdl_wait();
   constexpr int CH = kExchangeChunk;   // 256 factor elements per block, one per thread
   constexpr int WB = 8;                // workers handled per round
@@ -672,6 +672,7 @@ exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __rest
   s = sred[0];
 #pragma unroll
   for (int i = 1; i < 8; ++i) s = fmaxf(s, sred[i]);
+  if (sx.pack_only) s = sx.scales[which * sx.n_mat + ch.layer];   // scale agreed between the ranks
   const bool s_ok = (s > 0.f) && (s < INFINITY);
 
   if (b == 32) {
@@ -752,11 +753,14 @@ exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __rest
         v |= (sh >= 0) ? (c << sh) : (c >> (-sh));
       }
       t.payload[(size_t)(w0 + u) * t.payload_stride + pay_off + byte0 + jb] = (uint8_t)(v & 0xffu);
+      if (sx.pack_only)      // the same stream, contiguous over the local workers, for the all-gather
+        sx.send[which][(size_t)(w0 + u) * sx.region_bytes[which] + (pay_off - sx.region_off[which]) + byte0 + jb] =
+            (uint8_t)(v & 0xffu);
     }
     __syncthreads();
   }
 
-  if (valid) {
+  if (valid && !sx.pack_only) {
     const float v = s_ok ? s * __ldg(qt.deq + S + W * (nlev - 1)) : 0.f;
     dst[(size_t)row * RP + col] = v;
     if (which) L.Qt[(size_t)col * L.mt + row] = v;
@@ -782,13 +786,86 @@ q_transpose_kernel(const float* __restrict__ Q, float* __restrict__ Qt, int m, i
 }
 
 // ---------------------------------------------------------------------------------------
+// Split exchange, for workers spread over several GPUs (the All-Reduce of Alg. 1 as a real
+// exchange): every rank reduces its block maxima to one local scale per layer
+// (scale_reduce_kernel), the ranks agree on the maximum, each packs its workers' codes with that
+// scale (exchange_kernel in pack-only mode), the packed streams are all-gathered, and
+// sum_dequant_kernel adds the signed levels of ALL workers (exact integers) and applies Eq. 5.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+scale_reduce_kernel(Tables t, int which, float* scales, int n_mat) {
+  pdl_wait();
+  __shared__ float sred[8];
+  const int layer = blockIdx.x, tid = threadIdx.x;
+  const LayerDev& L = t.layers[layer];
+  const int nblk = which ? L.nqb : L.npb;
+  const float* __restrict__ maxes = which ? L.maxq : L.maxp;
+  float s = 0.f;
+  for (int i = tid; i < t.W * nblk; i += 256) s = fmaxf(s, maxes[i]);
+#pragma unroll
+  for (int o = 16; o >= 1; o >>= 1) s = fmaxf(s, __shfl_xor_sync(0xffffffffu, s, o));
+  if ((tid & 31) == 0) sred[tid >> 5] = s;
+  __syncthreads();
+  if (tid == 0) {
+    for (int i = 1; i < 8; ++i) s = fmaxf(s, sred[i]);
+    scales[which * n_mat + layer] = fmaxf(s, sred[0]);
+  }
+}
+
+template <int RP>
+__global__ void __launch_bounds__(256)
+sum_dequant_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __restrict__ chunks, SplitExchange sx,
+                   const uint8_t* __restrict__ gathered, int n_streams) {
+  pdl_wait();
+  const ExchangeChunk ch = chunks[blockIdx.x];
+  const LayerDev& L = t.layers[ch.layer];
+  const int tid = threadIdx.x, b = qt.bits;
+  const int nlev = 1 << (b - 1);
+  const int rows = which ? L.m : L.n, r = L.r;
+  const int count = rows * r;
+  const int e = ch.chunk * kExchangeChunk + tid;
+  const float s = sx.scales[which * sx.n_mat + ch.layer];
+  const bool s_ok = (s > 0.f) && (s < INFINITY);
+  if (e < count) {
+    const uint64_t off = (which ? L.pay_q_off : L.pay_p_off) - sx.region_off[which];   // this layer's stream
+    const size_t nbytes = ((size_t)count * b + 7) / 8;
+    const size_t bit = (size_t)e * b, byte = bit >> 3;
+    const int sh = (int)(bit & 7);
+    int S = 0;
+    for (int w = 0; w < n_streams; ++w) {
+      const uint8_t* st = gathered + (size_t)w * sx.region_bytes[which] + off;
+      unsigned v = st[byte];
+      if (sh + b > 8 && byte + 1 < nbytes) v |= (unsigned)st[byte + 1] << 8;
+      const unsigned code = (v >> sh) & ((1u << b) - 1u);
+      const int k = (int)(code & (unsigned)(nlev - 1));
+      S += (code >> (b - 1)) ? -k : k;
+    }
+    const float v = s_ok ? s * __ldg(qt.deq + S + n_streams * (nlev - 1)) : 0.f;
+    const int row = e / r, col = e - row * r;
+    float* dst = which ? L.Q : L.Pbar;
+    dst[(size_t)row * RP + col] = v;
+    if (which) L.Qt[(size_t)col * L.mt + row] = v;
+  }
+  if (ch.chunk == 0 && tid == 0) {
+    L.scales[which] = s;
+    for (int w = 0; w < t.W; ++w) {
+      float* ps = reinterpret_cast<float*>(t.payload + (size_t)w * t.payload_stride + L.pay_scale_off);
+      ps[which] = s;
+    }
+    if (!(s > 0.f)) atomicOr(&t.status[ch.layer], which ? 4u : 2u);
+    if (!(s < INFINITY)) atomicOr(&t.status[ch.layer], 8u);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
 // 1-D tensors: mean over the workers (Eq. 1) in worker order, and the raw fp32 values into
 // each worker's payload.
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 vectors_kernel(const VectorDev* __restrict__ vecs, const ExchangeChunk* __restrict__ chunks,
                const float* const* __restrict__ vgrads, float* const* __restrict__ vghat,
-               float* const* __restrict__ vweights, float lr, uint8_t* payload, uint64_t payload_stride, int W) {
+               float* const* __restrict__ vweights, float lr, uint8_t* payload, uint64_t payload_stride, int W,
+               int W_total) {
   pdl_wait();
   const ExchangeChunk ch = chunks[blockIdx.x];
   const VectorDev v = vecs[ch.layer];
@@ -800,7 +877,7 @@ vectors_kernel(const VectorDev* __restrict__ vecs, const ExchangeChunk* __restri
     reinterpret_cast<float*>(payload + (size_t)w * payload_stride + v.pay_off)[i] = x;
     s += x;
   }
-  const float mean = s / (float)W;
+  const float mean = s / (float)W_total;     // with workers on other GPUs too: this rank's share of the mean
   if (vghat[ch.layer]) vghat[ch.layer][i] = mean;
   if (vweights && vweights[ch.layer]) vweights[ch.layer][i] = fmaf(-lr, mean, vweights[ch.layer][i]);
 }
@@ -862,17 +939,31 @@ cudaError_t launch_q_reduce(int rp, const Tables& t, const FactorBlock* fb, int 
 }
 
 cudaError_t launch_exchange(int rp, int which, const Tables& t, const QuantTables& q,
-                            const ExchangeChunk* ch, int nch, Launch l) {
+                            const ExchangeChunk* ch, int nch, const SplitExchange& sx, Launch l) {
   if (nch == 0) return cudaSuccess;
-  LQSGD_DISPATCH_RP(rp, (launch_pdl(exchange_kernel<RP>, nch, 256, 0, l.stream, t, q, which, ch)));
+  LQSGD_DISPATCH_RP(rp, (launch_pdl(exchange_kernel<RP>, nch, 256, 0, l.stream, t, q, which, ch, sx)));
+  return cudaGetLastError();
+}
+
+cudaError_t launch_scale_reduce(const Tables& t, int which, float* scales, int n_mat, Launch l) {
+  if (n_mat == 0) return cudaSuccess;
+  launch_pdl(scale_reduce_kernel, n_mat, 256, 0, l.stream, t, which, scales, n_mat);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_sum_dequant(int rp, int which, const Tables& t, const QuantTables& q, const ExchangeChunk* ch,
+                               int nch, const SplitExchange& sx, const uint8_t* gathered, int n_streams, Launch l) {
+  if (nch == 0) return cudaSuccess;
+  LQSGD_DISPATCH_RP(rp, (launch_pdl(sum_dequant_kernel<RP>, nch, 256, 0, l.stream, t, q, which, ch, sx, gathered,
+                                    n_streams)));
   return cudaGetLastError();
 }
 
 cudaError_t launch_vectors(const VectorDev* vecs, const ExchangeChunk* chunks, int nchunks,
                            const float* const* vgrads, float* const* vghat, float* const* vweights, float lr,
-                           uint8_t* payload, uint64_t payload_stride, int W, Launch l) {
+                           uint8_t* payload, uint64_t payload_stride, int W, int W_total, Launch l) {
   if (nchunks == 0) return cudaSuccess;
-  launch_pdl(vectors_kernel, nchunks, 256, 0, l.stream, vecs, chunks, vgrads, vghat, vweights, lr, payload, payload_stride, W);
+  launch_pdl(vectors_kernel, nchunks, 256, 0, l.stream, vecs, chunks, vgrads, vghat, vweights, lr, payload, payload_stride, W, W_total);
   return cudaGetLastError();
 }
 
