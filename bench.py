@@ -315,6 +315,69 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_exchange(args):
+    """Opt-in (--exchange): the workers of all ranks take part in ONE average, with the real
+    exchange of Algorithm 1 between the GPUs (two MAX all-reduces of the scales and two
+    all-gathers of the packed codes per step, NCCL).  Every rank simulates the workload's W
+    workers, so the average is over W x n_gpus workers (weak scaling)."""
+    import torch
+    import torch.distributed as dist
+    import __graft_entry__ as entry
+    from paper_2506_17974_b200 import binding as B
+    from paper_2506_17974_b200 import distributed as D
+    from paper_2506_17974_b200 import workloads as wl
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    os.environ.setdefault("MASTER_PORT", "29511")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    dist.init_process_group("nccl", rank=rank, world_size=world, device_id=torch.device(dev))
+    if rank == 0:
+        entry.build()
+    dist.barrier()
+    peak, peak_kind = load_peaks()
+    wl_obj, desc = get_workload(args.workload)
+    comp = B.LQSGD(wl_obj.layers, wl_obj.rank, wl_obj.bits, alpha=wl_obj.alpha, workers=wl_obj.workers,
+                   seed=wl_obj.seed, device=dev, world_workers=wl_obj.workers * world)
+    seeded = dataclasses.replace(wl_obj, seed=wl_obj.seed + 1000 * rank)
+    sets = [wl.draw_gradients(seeded, t, device=dev) for t in range(3)]
+    ghat = [torch.empty_like(g) for g in sets[0][0]]
+    for t in range(args.warmup):
+        D.distributed_round(comp, sets[t % 3], ghat)
+    dist.barrier()
+    torch.cuda.synchronize()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for t in range(args.steps):
+        D.distributed_round(comp, sets[(args.warmup + t) % 3], ghat)
+    stop.record()
+    dist.barrier()
+    torch.cuda.synchronize()
+    tms = torch.tensor([start.elapsed_time(stop) / args.steps], dtype=torch.float64, device=dev)
+    dist.all_reduce(tms, op=dist.ReduceOp.MAX)
+    ms = float(tms.item())
+    gbytes = gradient_bytes(wl_obj)
+    rb = sum(phase_bytes(wl_obj).values())
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": world * gbytes / (ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": desc, "l2": "inputs larger than L2; 3 gradient sets rotate",
+                       "parallelism": f"{wl_obj.workers} workers per GPU x {world} GPUs in one average: 2 MAX "
+                                      "all-reduces of scales + 2 all-gathers of packed codes per step (NCCL)"},
+            "gpu_launches": args.steps * (comp.launches_per_step + 4),
+            "roofline": {"bound": "hbm", "kernel": "whole round per GPU", "achieved": rb / (ms * 1e-3) / 1e9, "peak": peak,
+                         "unit": "GB/s", "frac": rb / (ms * 1e-3) / 1e9 / peak, "peak_kind": f"of {peak_kind}", "traffic": None},
+            "exchange_bytes_per_rank_per_step": int(comp.exchange_view(B.XCHG_STREAMS_P).numel()
+                                                    + comp.exchange_view(B.XCHG_STREAMS_Q).numel()),
+        }))
+    dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -325,9 +388,13 @@ def main():
     ap.add_argument("--no-sweep", action="store_true", help="skip the large-layer sweep")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer (end-to-end) measurement")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle")
+    ap.add_argument("--exchange", action="store_true",
+                    help="workers of all GPUs in one average, with the real NCCL exchange (default: independent replicas)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.exchange:
+        run_exchange(args)
     else:
         run_ours(args)
 

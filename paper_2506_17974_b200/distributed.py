@@ -28,13 +28,23 @@ def distributed_round(comp, grads, ghat: Sequence[torch.Tensor], group: Optional
     # the fused model update only sees this rank's share of a 1-D tensor's mean: update those here
     fused = None if weights is None else [wt if comp.is_matrix(l) else None for l, wt in enumerate(weights)]
     comp.round_begin(grads, ghat, fused, lr)
+    cache = getattr(comp, "_xchg_cache", None)          # views of fixed buffers and the gather targets
+    if cache is None or cache.get("world") != world:
+        cache = {"world": world}
+        try:
+            comp._xchg_cache = cache
+        except AttributeError:
+            pass
     for which, scales_id, streams_id in ((0, XCHG_SCALES_P, XCHG_STREAMS_P), (1, XCHG_SCALES_Q, XCHG_STREAMS_Q)):
         scales = comp.exchange_view(scales_id)
         if scales.numel():
             dist.all_reduce(scales, op=dist.ReduceOp.MAX, group=group)       # one shared scale per factor and layer
         comp.round_pack(which)
         send = comp.exchange_view(streams_id)
-        gathered = torch.empty(world * send.numel(), dtype=send.dtype, device=send.device)
+        gathered = cache.get(("gathered", which))
+        if gathered is None or gathered.numel() != world * send.numel() or gathered.device != send.device:
+            gathered = torch.empty(world * send.numel(), dtype=send.dtype, device=send.device)
+            cache[("gathered", which)] = gathered
         if send.numel():
             dist.all_gather_into_tensor(gathered, send, group=group)          # the packed codes of every worker
         comp.round_reduce(which, gathered, world)
