@@ -16,6 +16,7 @@ from __future__ import annotations
 
 import argparse
 import dataclasses
+import hashlib
 import json
 import os
 import subprocess
@@ -39,6 +40,31 @@ def load_peaks():
     return 6650.0, "fallback"
 
 
+def csrc_digest() -> str:
+    """SHA-256 over the kernel sources: ties a stored ncu figure to the code it was taken from."""
+    h = hashlib.sha256()
+    d = os.path.join(ROOT, "paper_2506_17974_b200", "csrc")
+    for name in sorted(os.listdir(d)):
+        if name.endswith((".cu", ".cuh", ".h")):
+            h.update(name.encode())
+            with open(os.path.join(d, name), "rb") as f:
+                h.update(f.read())
+    return h.hexdigest()
+
+
+def recorded_traffic(workload: str, phase: str):
+    """DRAM bytes (read + write) per launch of that phase's kernel from the ncu capture summarised under
+    profiles/, or None when there is no capture of this workload or the kernels changed since."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if not os.path.exists(path):
+        return None
+    with open(path) as f:
+        rec = json.load(f)
+    if rec.get("csrc_sha256") != csrc_digest():
+        return None
+    return rec.get("workloads", {}).get(workload, {}).get(phase)
+
+
 def get_workload(name: str):
     from paper_2506_17974_b200 import workloads as wl
     if name == "resnet18":
@@ -50,6 +76,9 @@ def get_workload(name: str):
     if name.startswith("large_"):
         a, b = name[len("large_"):].split("x")
         return wl.config4(int(a), int(b)), f"large layer {a}x{b} W=1 r=8 b=4, N(0, 0.01^2)"
+    if name.startswith("config5_r"):
+        r, b = name[len("config5_r"):].split("_b")
+        return wl.config5(int(r), int(b)), f"resnet18_cifar100 W=16 r={r} b={b} (ResNet-18 gradient set, Student-t nu=3)"
     raise SystemExit(f"unknown workload {name}")
 
 
@@ -189,7 +218,7 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    def bench_workload(wl_obj, steps, warmup, nsets, want_e2e, sample_clocks):
+    def bench_workload(wl_obj, steps, warmup, nsets, want_e2e, sample_clocks, want_graph=False):
         comp = B.LQSGD(wl_obj.layers, wl_obj.rank, wl_obj.bits, alpha=wl_obj.alpha, workers=wl_obj.workers,
                        seed=wl_obj.seed + rank, device=dev)
         seeded = dataclasses.replace(wl_obj, seed=wl_obj.seed + 1000 * rank)
@@ -224,13 +253,38 @@ def run_ours(args):
         barrier()
         if sampler:
             sampler.__exit__(None, None, None)
+        # the same step replayed from a CUDA graph (kernels only): what launch overhead is left in `ms`
+        graph_ms = None
+        if want_graph:
+            comp.set_phase_events(None)
+            comp.step_ptrs(*ptrs[0], stream)               # the captured call must repeat these pointers
+            side = torch.cuda.Stream(device=dev)
+            side.wait_stream(stream)
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side, capture_error_mode="thread_local"):
+                comp.step_ptrs(*ptrs[0], torch.cuda.current_stream())
+            stream.wait_stream(side)
+            for _ in range(3):
+                graph.replay()
+            barrier()
+            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            g0.record(stream)
+            for _ in range(steps):
+                graph.replay()
+            g1.record(stream)
+            barrier()
+            graph_ms = g0.elapsed_time(g1) / steps
+            del graph
         ms = start.elapsed_time(stop) / steps
         phases = [sum(events[t][i].elapsed_time(events[t][i + 1]) for t in range(psteps)) / psteps
                   for i in range(B.N_PHASES)]
         status = comp.status()
-        assert all(s == 0 for s in status), f"device status flags set: {status}"
+        # a dependent column or a zero scale is a property of the data (it happens with 2-bit codes);
+        # a non-finite value or an expired wait would make the timing meaningless
+        assert all(s & (B.STATUS_NONFINITE | B.STATUS_TIMEOUT) == 0 for s in status), f"device status flags: {status}"
         out = {"ms": ms, "phases_ms": dict(zip(B.PHASE_NAMES, phases)), "launches": comp.launches_per_step,
-               "payload": comp.payload_nbytes, "clocks": sampler.summary() if sampler else None}
+               "payload": comp.payload_nbytes, "clocks": sampler.summary() if sampler else None, "graph_ms": graph_ms,
+               "flagged_layers": sum(1 for x in status if x)}
         del comp
         if want_e2e:
             comp = B.LQSGD(wl_obj.layers, wl_obj.rank, wl_obj.bits, alpha=wl_obj.alpha, workers=wl_obj.workers,
@@ -253,9 +307,33 @@ def run_ours(args):
         torch.cuda.empty_cache()
         return out
 
+    def residual_rel(wl_obj, steps):
+        """||M - G_hat||_F / ||M||_F (Eq. 7: the new error buffer against what was compressed), over all 2-D
+        layers and workers, at step `steps` of a fresh context."""
+        comp = B.LQSGD(wl_obj.layers, wl_obj.rank, wl_obj.bits, alpha=wl_obj.alpha, workers=wl_obj.workers,
+                       seed=wl_obj.seed, device=dev)
+        mats = [l for l in range(len(wl_obj.layers)) if comp.is_matrix(l)]
+        num = den = 0.0
+        for t in range(steps):
+            g = wl.draw_gradients(wl_obj, t, device=dev)
+            last = t == steps - 1
+            if last:
+                for l in mats:
+                    for w in range(wl_obj.workers):
+                        den += float((g[w][l].double() + comp.get_state(B.STATE_E, l, w).double()).pow(2).sum())
+            ghat = [torch.empty_like(x) for x in g[0]]
+            comp.step(g, ghat)
+            if last:
+                for l in mats:
+                    for w in range(wl_obj.workers):
+                        num += float(comp.get_state(B.STATE_E, l, w).double().pow(2).sum())
+        torch.cuda.synchronize()
+        return (num / den) ** 0.5
+
     wl_obj, desc = get_workload(args.workload)
     gbytes = gradient_bytes(wl_obj)
-    res = bench_workload(wl_obj, args.steps, args.warmup, nsets=3, want_e2e=not args.no_e2e, sample_clocks=True)
+    res = bench_workload(wl_obj, args.steps, args.warmup, nsets=3, want_e2e=not args.no_e2e, sample_clocks=True,
+                         want_graph=not args.no_graph)
 
     def allmax(x):
         if world == 1:
@@ -285,10 +363,12 @@ def run_ours(args):
                 "h2d_bytes_per_step": res.get("h2d"), "d2h_bytes_per_step": res.get("d2h"), "ms_per_step": e2e_ms}
         if "e2e_ms" in res else None,
         "roofline": {"bound": "hbm", "kernel": f"{dom}_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": recorded_traffic(args.workload, dom),
                      "bytes_per_launch": pb[dom], "kernel_ms": res["phases_ms"][dom]},
         "round": {"algorithmic_bytes": round_bytes, "achieved_gbs": round_bytes / (ms * 1e-3) / 1e9,
                   "frac_of_peak": round_bytes / (ms * 1e-3) / 1e9 / peak, "phases_ms": res["phases_ms"]},
+        "cuda_graph": {"ms_per_step": res["graph_ms"], "what": "one captured step replayed on one gradient set "
+                       "(larger than L2); the timed `value` above uses plain launches"} if res.get("graph_ms") else None,
         "compression_ratio": 4 * sum(n * m for n, m in wl_obj.layers) / res["payload"],
         "payload_bytes_per_worker": res["payload"],
     }
@@ -303,6 +383,22 @@ def run_ours(args):
                                  "round_frac_of_peak": rb / (r4["ms"] * 1e-3) / 1e9 / peak,
                                  "phases_ms": r4["phases_ms"]}
         line["large_layer_sweep"] = sweep
+    if rank == 0 and world == 1 and args.config5_sweep:
+        # rank x bits grid on the 16-worker ResNet-18 (100 classes) set: throughput, compression ratio and
+        # what the round loses, ||M - G_hat||_F / ||M||_F over all layers and workers at the last step
+        grid = {}
+        for r5 in (1, 2, 4, 8, 16):
+            for b5 in (2, 3, 4, 8):
+                w5 = wl.config5(r5, b5)
+                r = bench_workload(w5, steps=min(args.steps, 100), warmup=3, nsets=2, want_e2e=False, sample_clocks=False)
+                rb = sum(phase_bytes(w5).values())
+                grid[f"r{r5}_b{b5}"] = {
+                    "gbs_gradient": gradient_bytes(w5) / (r["ms"] * 1e-3) / 1e9, "ms_per_step": r["ms"],
+                    "round_frac_of_peak": rb / (r["ms"] * 1e-3) / 1e9 / peak, "phases_ms": r["phases_ms"],
+                    "compression_ratio": 4 * sum(n * m for n, m in w5.layers) / r["payload"],
+                    "payload_bytes_per_worker": r["payload"], "residual_rel": residual_rel(w5, 10),
+                    "layers_with_dependent_column_or_zero_scale": r["flagged_layers"]}
+        line["config5_sweep"] = grid
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         times, cores = time_oracle(wl_obj, budget_s=12.0, max_steps=8)
         t = sum(times) / len(times)
@@ -387,10 +483,18 @@ def main():
     ap.add_argument("--workload", default="resnet18")
     ap.add_argument("--no-sweep", action="store_true", help="skip the large-layer sweep")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer (end-to-end) measurement")
+    ap.add_argument("--source-digest", action="store_true",
+                    help="print the digest of the kernel sources that profiles/dram_traffic.json is keyed on, and exit")
+    ap.add_argument("--config5-sweep", action="store_true",
+                    help="also time the rank x bits grid on the 16-worker ResNet-18 set (a few minutes)")
+    ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay measurement")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle")
     ap.add_argument("--exchange", action="store_true",
                     help="workers of all GPUs in one average, with the real NCCL exchange (default: independent replicas)")
     args = ap.parse_args()
+    if args.source_digest:
+        print(csrc_digest())
+        return
     if args.impl == "reference":
         run_reference(args)
     elif args.exchange:

@@ -63,7 +63,8 @@ typedef enum lqsgd_error {
   LQSGD_ERR_CUDA = -5,                /* a CUDA runtime call failed; see lqsgd_last_cuda_error() */
   LQSGD_ERR_NO_STAGING = -6,          /* lqsgd_step_host() on a context created without LQSGD_FLAG_HOST_STAGING */
   LQSGD_ERR_OUT_OF_RANGE = -7,        /* layer / worker / state index out of range, or state not defined for that layer */
-  LQSGD_ERR_TOO_LARGE = -8            /* size beyond the fixed built-in scratch of lqsgd_orthonormalize_noalloc */
+  LQSGD_ERR_TOO_LARGE = -8,           /* size beyond the fixed built-in scratch of lqsgd_orthonormalize_noalloc */
+  LQSGD_ERR_CAPTURE = -9              /* stream is capturing and the tensor pointers differ from the previous call's */
 } lqsgd_error;
 
 /* Bits of the per-layer status word. */
@@ -149,7 +150,12 @@ int lqsgd_create(const lqsgd_shape* host_shapes, int32_t n_layers, const lqsgd_c
  *   Must not alias any gradient.
  * cuda_stream: a cudaStream_t (NULL = legacy default stream).  The call only enqueues work;
  *   results, payload and state are valid once the stream has reached the end of that work.
- *   The pointer arrays themselves are consumed before the call returns. */
+ *   The pointer arrays themselves are consumed before the call returns.
+ * CUDA graphs: the call may be made on a capturing stream when its tensor pointers equal those
+ *   of the previous call on this context (the captured work is then kernels only; the graph
+ *   reads and writes those same tensors at every replay).  With different pointers a capturing
+ *   stream gets LQSGD_ERR_CAPTURE and nothing is enqueued: the upload of the pointer table
+ *   cannot be part of a graph. */
 int lqsgd_step(lqsgd_ctx* ctx, const float* const* host_grads, float* const* host_ghat,
                void* cuda_stream);
 

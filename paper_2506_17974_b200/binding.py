@@ -29,6 +29,7 @@ PHASE_NAMES = ("pass1", "finish_p", "pass2", "finish_q", "pass3")
 ERR_INVALID_ARG, ERR_BAD_SHAPE, ERR_WORKSPACE_TOO_SMALL, ERR_MISALIGNED = -1, -2, -3, -4
 ERR_CUDA, ERR_NO_STAGING, ERR_OUT_OF_RANGE = -5, -6, -7
 ERR_TOO_LARGE = -8
+ERR_CAPTURE = -9
 NOALLOC_MAX_ROWS = 65536
 
 EXPORTED = [

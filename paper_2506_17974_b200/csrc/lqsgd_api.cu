@@ -422,6 +422,7 @@ const char* lqsgd_strerror(int code) {
     case LQSGD_ERR_NO_STAGING: return "context was created without host staging";
     case LQSGD_ERR_OUT_OF_RANGE: return "index out of range";
     case LQSGD_ERR_TOO_LARGE: return "size exceeds the built-in scratch of the no-allocation entry point";
+    case LQSGD_ERR_CAPTURE: return "stream is capturing and the tensor pointers changed since the previous call";
     default: return "unknown error";
   }
 }
@@ -581,6 +582,9 @@ static int prepare_step(lqsgd_ctx* c, const float* const* grads, float* const* g
     if (!ptrs[vbase + nv * W + vi] && !ptrs[vbase + nv * (W + 1) + vi]) return LQSGD_ERR_INVALID_ARG;
   }
   if (!c->ptrs_valid || ptrs != c->ptrs_host) {
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    CK(cudaStreamIsCapturing(st, &cap));
+    if (cap != cudaStreamCaptureStatusNone) return LQSGD_ERR_CAPTURE;   // a copy from this host vector cannot be replayed
     c->ptrs_host = ptrs;
     // pageable source: the runtime stages it before returning, so the vector may change afterwards
     CK(cudaMemcpyAsync(p.d_ptrs, c->ptrs_host.data(), ptrs.size() * sizeof(void*), cudaMemcpyHostToDevice, st));

@@ -230,6 +230,48 @@ def test_bit_reproducible_and_checkpoint_resume():
     assert torch.equal(a.get_state(B.STATE_E, 2, 2), c.get_state(B.STATE_E, 2, 2))
 
 
+def test_step_replays_from_a_cuda_graph():
+    """A step captured into a CUDA graph (kernels only, dependent launches included) replays to
+    the same bits as eager steps; a capture with unseen tensor pointers is refused."""
+    w = dataclasses.replace(wl.config2(), workers=2)
+    a, b = make(w), make(w)
+    g0 = wl.draw_gradients(w, 0, device=DEV)
+    bufs = [[torch.empty_like(x) for x in per] for per in g0]
+    other = [[torch.empty_like(x) for x in per] for per in g0]
+    oa = [torch.empty(s, device=DEV) for s in w.layers]
+    ob = [torch.empty(s, device=DEV) for s in w.layers]
+
+    def fill(t):
+        g = wl.draw_gradients(w, t, device=DEV)
+        for per, src in zip(bufs, g):
+            for dst, x in zip(per, src):
+                dst.copy_(x)
+        return g
+
+    ga, ha = a.make_pointer_arrays(bufs, oa)
+    go, _ = a.make_pointer_arrays(other, oa)
+    g = fill(0)
+    a.step_ptrs(ga, ha)                              # eager: uploads the pointer table
+    b.step(g, ob)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, capture_error_mode="thread_local"):
+        with pytest.raises(B.LqsgdError) as e:
+            a.step_ptrs(go, ha, torch.cuda.current_stream())
+        assert e.value.code == B.ERR_CAPTURE
+        a.step_ptrs(ga, ha, torch.cuda.current_stream())
+    for t in range(1, 4):
+        g = fill(t)
+        graph.replay()
+        b.step(g, ob)
+        torch.cuda.synchronize()
+        for x, y in zip(oa, ob):
+            assert torch.equal(x, y)
+        assert torch.equal(a.payload(1), b.payload(1))
+    assert all(s == 0 for s in a.status())
+    assert torch.equal(a.get_state(B.STATE_E, 2, 1), b.get_state(B.STATE_E, 2, 1))
+
+
 def test_step_host_matches_device_step():
     w = dataclasses.replace(wl.config2(), workers=2)
     a, b = make(w), make(w, host_staging=True)
