@@ -331,6 +331,9 @@ def run_ours(args):
         return (num / den) ** 0.5
 
     wl_obj, desc = get_workload(args.workload)
+    if args.workers:
+        wl_obj = dataclasses.replace(wl_obj, workers=args.workers)
+        desc += f" [workers overridden: W={args.workers}]"
     gbytes = gradient_bytes(wl_obj)
     res = bench_workload(wl_obj, args.steps, args.warmup, nsets=3, want_e2e=not args.no_e2e, sample_clocks=True,
                          want_graph=not args.no_graph)
@@ -487,6 +490,8 @@ def main():
                     help="print the digest of the kernel sources that profiles/dram_traffic.json is keyed on, and exit")
     ap.add_argument("--config5-sweep", action="store_true",
                     help="also time the rank x bits grid on the 16-worker ResNet-18 set (a few minutes)")
+    ap.add_argument("--workers", type=int, default=0,
+                    help="override the workload's worker count (smaller cases for profiler captures)")
     ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay measurement")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle")
     ap.add_argument("--exchange", action="store_true",

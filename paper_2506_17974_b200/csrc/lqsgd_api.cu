@@ -54,6 +54,8 @@ struct Plan {
   std::vector<VectorDev> vecs;
   std::vector<Tile> tiles1, tiles2, tiles3;      // register-path passes
   std::vector<Tile> stiles1, stiles3;            // bulk-copy staged passes 1 and 3
+  std::vector<Tile> tctiles2;                    // tensor-core pass 2
+  std::vector<uint8_t> tcmaps;                   // tensor maps of the tensor-core passes (filled at create)
   std::vector<FactorBlock> fbP, fbQ;
   std::vector<ExchangeChunk> chP, chQ, chV;
   std::vector<float> thrP, thrQ, deqP, deqQ;
@@ -66,6 +68,8 @@ struct Plan {
   VectorDev* d_vecs = nullptr;
   Tile *d_tiles1 = nullptr, *d_tiles2 = nullptr, *d_tiles3 = nullptr;
   Tile *d_stiles1 = nullptr, *d_stiles3 = nullptr;
+  Tile* d_tctiles2 = nullptr;
+  uint8_t* d_tcmaps = nullptr;
   FactorBlock *d_fbP = nullptr, *d_fbQ = nullptr;
   ExchangeChunk *d_chP = nullptr, *d_chQ = nullptr, *d_chV = nullptr;
   float *d_thrP = nullptr, *d_thrQ = nullptr, *d_deqP = nullptr, *d_deqQ = nullptr;
@@ -215,6 +219,10 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   auto staged = [&](const MatHost& mt) {
     return !(cfg.flags & LQSGD_FLAG_REGISTER_PATH) && RP <= kStreamMaxRP && mt.m % 4 == 0;
   };
+  // Tensor-core passes: padded rank 16, rows 16-byte aligned.
+  auto on_tc = [&](const MatHost& mt) {
+    return !(cfg.flags & LQSGD_FLAG_REGISTER_PATH) && RP >= 16 && mt.m % 4 == 0;
+  };
   auto staged_cols = [&](int m) {                      // list of (col0, ncols)
     std::vector<std::pair<int, int>> out;
     const int maxc = stream_max_cols(RP);
@@ -269,10 +277,11 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
     LayerDev& L = p.layers[li];
     std::memset(&L, 0, sizeof(L));
     L.n = mt.n; L.m = mt.m; L.r = mt.r; L.vec = vec_of(mt.m) == 4; L.user_index = mt.user_index;
-    const bool st = staged(mt);
+    const bool st = staged(mt), tc = on_tc(mt);
     const auto scols = staged_cols(mt.m);
     const int cw = chunk_width(mt.m, c1);
-    const int tr2 = balanced_rows(mt.n, r2);   // pass 2 runs on the register path for every layer
+    // pass 2: register path, or tensor cores (row chunks in multiples of the 64 rows of an operand slot)
+    const int tr2 = tc ? (int)align_up((size_t)balanced_rows(mt.n, kTcRowChunk), 64) : balanced_rows(mt.n, r2);
     L.ncc = st ? (int)scols.size() : ceil_div(mt.m, cw);
     L.nrb = ceil_div(mt.n, tr2);
     L.npb = ceil_div(mt.n, kFactorBlockRows);
@@ -281,7 +290,10 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
     L.E = a.take<float>((size_t)W * nm);
     L.Q = a.take<float>((size_t)mt.m * RP);
     L.mt = (int)align_up((size_t)mt.m, 4);
-    L.Qt = a.take<float>((size_t)RP * L.mt);
+    L.tc = tc ? 1 : 0;
+    L.nt = (int)align_up((size_t)mt.n, 4);
+    L.Qt = a.take<float>((size_t)(tc ? 2 : 1) * RP * L.mt);
+    L.Pbt = tc ? a.take<float>((size_t)3 * RP * L.nt) : nullptr;
     L.Ppart = a.take<float>((size_t)W * L.ncc * mt.n * RP);
     L.Praw = (L.ncc == 1) ? L.Ppart : a.take<float>((size_t)W * mt.n * RP);
     L.P = a.take<float>((size_t)W * mt.n * RP);
@@ -320,7 +332,14 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
       for (int rb = 0; rb < L.nrb; ++rb)
         for (int cc = 0; cc < ceil_div(mt.m, cw2); ++cc) {
           const int row0 = rb * tr2, col0 = cc * cw2;
+          if (tc) continue;
           p.tiles2.push_back({li32, w, row0, std::min(tr2, mt.n - row0), col0, std::min(cw2, mt.m - col0), rb, 0});
+        }
+    for (int w = 0; tc && w < W; ++w)
+      for (int rb = 0; rb < L.nrb; ++rb)
+        for (int cc = 0; cc < ceil_div(mt.m, 128); ++cc) {
+          const int row0 = rb * tr2, col0 = cc * 128;
+          p.tctiles2.push_back({li32, w, row0, std::min(tr2, mt.n - row0), col0, std::min(128, mt.m - col0), rb, 0});
         }
     const int tr3 = balanced_rows(mt.n, r3);
     for (int rb = 0; !st && rb < ceil_div(mt.n, tr3); ++rb)
@@ -340,6 +359,9 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   // Pass 2 walks the data in the reverse of pass 1's order and pass 3 again in pass 1's order:
   // each pass starts on what the previous one touched last, which is still in L2.
   std::reverse(p.tiles2.begin(), p.tiles2.end());
+  // The tensor-core kernels deal their tiles round-robin to one CTA per SM: largest first, so the
+  // CTAs finish together.
+  std::stable_sort(p.tctiles2.begin(), p.tctiles2.end(), [](const Tile& x, const Tile& y) { return x.nrows > y.nrows; });
   p.d_status = a.take<uint32_t>(p.mats.size());
   p.d_payload = a.take<uint8_t>((size_t)W * p.payload_stride);
   p.d_xscales = a.take<float>(2 * p.mats.size());
@@ -354,6 +376,8 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   p.d_tiles3 = a.take<Tile>(p.tiles3.size());
   p.d_stiles1 = a.take<Tile>(p.stiles1.size());
   p.d_stiles3 = a.take<Tile>(p.stiles3.size());
+  p.d_tctiles2 = a.take<Tile>(p.tctiles2.size());
+  p.d_tcmaps = a.take<uint8_t>(p.mats.size() * kTcMapsPerLayer * kTcMapBytes);
   p.d_fbP = a.take<FactorBlock>(p.fbP.size());
   p.d_fbQ = a.take<FactorBlock>(p.fbQ.size());
   p.d_chP = a.take<ExchangeChunk>(p.chP.size());
@@ -484,6 +508,11 @@ int lqsgd_create(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
   CK(up(p.d_tiles3, p.tiles3.data(), p.tiles3.size() * sizeof(Tile)));
   CK(up(p.d_stiles1, p.stiles1.data(), p.stiles1.size() * sizeof(Tile)));
   CK(up(p.d_stiles3, p.stiles3.data(), p.stiles3.size() * sizeof(Tile)));
+  CK(up(p.d_tctiles2, p.tctiles2.data(), p.tctiles2.size() * sizeof(Tile)));
+  p.tcmaps.resize(p.mats.size() * kTcMapsPerLayer * kTcMapBytes + 1);
+  rc = tc_encode_maps(p.layers.data(), (int)p.layers.size(), p.W, p.RP, p.tcmaps.data());
+  if (rc != LQSGD_OK) { g_cuda_error = "cuTensorMapEncodeTiled failed or is not available"; return rc; }
+  CK(up(p.d_tcmaps, p.tcmaps.data(), p.mats.size() * kTcMapsPerLayer * kTcMapBytes));
   CK(up(p.d_fbP, p.fbP.data(), p.fbP.size() * sizeof(FactorBlock)));
   CK(up(p.d_fbQ, p.fbQ.data(), p.fbQ.size() * sizeof(FactorBlock)));
   CK(up(p.d_chP, p.chP.data(), p.chP.size() * sizeof(ExchangeChunk)));
@@ -502,7 +531,7 @@ int lqsgd_create(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
       for (int j = 0; j < mt.r; ++j)
         q0[(size_t)i * p.RP + j] = normal_draw(cfg->seed, (uint64_t)mt.user_index, (uint64_t)i * mt.r + j);
     CK(up(p.layers[li].Q, q0.data(), q0.size() * sizeof(float)));
-    CK(launch_q_transpose(p.layers[li].Q, p.layers[li].Qt, mt.m, p.RP, p.layers[li].mt, nullptr));
+    CK(launch_q_transpose(p.layers[li].Q, p.layers[li].Qt, mt.m, p.RP, p.layers[li].mt, p.layers[li].tc, nullptr));
   }
   int o1 = 1, o2 = 1, o3 = 1;
   CK(pass_occupancy(p.RP, &o1, &o2, &o3));
@@ -533,7 +562,9 @@ int lqsgd_set_phase_events(lqsgd_ctx* c, void* const* host_events) {
 int lqsgd_launches_per_step(const lqsgd_ctx* ctx, int32_t* out) {
   if (!ctx || !out) return LQSGD_ERR_INVALID_ARG;
   const Plan& p = ctx->plan;
-  *out = (p.mats.empty() ? 0 : 6) + (p.tiles1.empty() ? 0 : 2) + (p.stiles1.empty() ? 0 : 2) + (p.chV.empty() ? 0 : 1);
+  // Orthonormalize (2), exchange of P, Q_w reduction, exchange of Q; then one launch per non-empty tile list
+  *out = (p.mats.empty() ? 0 : 5) + (p.tiles1.empty() ? 0 : 2) + (p.stiles1.empty() ? 0 : 2) + (p.tiles2.empty() ? 0 : 1) +
+         (p.tctiles2.empty() ? 0 : 1) + (p.chV.empty() ? 0 : 1);
   return LQSGD_OK;
 }
 
@@ -656,6 +687,8 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
       if (nm) {
         if (split) CK(launch_sum_dequant(RP, 0, t, qp, p.d_chP, (int)p.chP.size(), sx, static_cast<const uint8_t*>(gathered), n_streams, {st, 0}));
         CK(launch_pass2(RP, t, p.d_tiles2, (int)p.tiles2.size(), {st, c->grid2}));
+        CK(launch_tc_pass2(RP, t, p.d_tctiles2, (int)p.tctiles2.size(), p.d_tcmaps,
+                           {st, (int)std::min<size_t>(p.tctiles2.size(), c->sm_count)}));
       }
       PHASE_MARK(3);
       if (nm) {
@@ -866,7 +899,7 @@ int lqsgd_set_state(lqsgd_ctx* c, int32_t which, int32_t layer, int32_t worker, 
   if (which == LQSGD_STATE_Q) {
     for (const LayerDev& L : c->plan.layers)
       if (L.user_index == layer)
-        CK(launch_q_transpose(L.Q, L.Qt, L.m, c->plan.RP, L.mt, static_cast<cudaStream_t>(cuda_stream)));
+        CK(launch_q_transpose(L.Q, L.Qt, L.m, c->plan.RP, L.mt, L.tc, static_cast<cudaStream_t>(cuda_stream)));
   }
   return LQSGD_OK;
 }

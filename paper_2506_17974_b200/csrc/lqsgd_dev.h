@@ -22,9 +22,13 @@ struct LayerDev {
   int32_t npb, nqb;           // factor blocks: ceil(n/128), ceil(m/128)
   int32_t user_index;         // index in the caller's layer list
   int32_t mt;                 // row stride of Qt: m rounded up to a multiple of 4
+  int32_t tc;                 // 1: the tensor-core passes take this layer (padded rank >= 16, m % 4 == 0)
+  int32_t nt;                 // row stride of Pbt: n rounded up to a multiple of 4
   float* E;                   // [W][n][m]   error buffer; holds M between pass 1 and pass 3
   float* Q;                   // [m][RP]     warm start, becomes Q_bar
-  float* Qt;                  // [RP][mt]    transposed copy of Q read by pass 1 and pass 3
+  float* Qt;                  // [RP][mt]    transposed copy of Q read by pass 1 and pass 3;
+                              // tc layers: [2 RP][mt], rows RP.. hold the tf32 remainders of rows 0..
+  float* Pbt;                 // tc layers: [3 RP][nt] words: P_bar transposed, as three stacked bf16 terms (pass 2 operand)
   float* Ppart;               // [W][ncc][n][RP]
   float* Praw;                // [W][n][RP]  (== Ppart when ncc == 1)
   float* P;                   // [W][n][RP]  orthonormal
@@ -133,7 +137,7 @@ cudaError_t launch_exchange(int RP, int which /*0 = P, 1 = Q*/, const Tables& t,
 cudaError_t launch_scale_reduce(const Tables& t, int which, float* scales, int n_mat, Launch l);
 cudaError_t launch_sum_dequant(int RP, int which, const Tables& t, const QuantTables& q, const ExchangeChunk* ch,
                                int nch, const SplitExchange& sx, const uint8_t* gathered, int n_streams, Launch l);
-cudaError_t launch_q_transpose(const float* Q, float* Qt, int m, int RP, int mt, cudaStream_t stream);
+cudaError_t launch_q_transpose(const float* Q, float* Qt, int m, int RP, int mt, int tc, cudaStream_t stream);
 cudaError_t launch_pass2(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
 cudaError_t launch_q_reduce(int RP, const Tables& t, const FactorBlock* fb, int nfb, Launch l);
 cudaError_t launch_pass3(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
@@ -176,6 +180,15 @@ __host__ __device__ inline StreamGeo stream_geo(int ncols, int RP) {
   g.rpg = (R + g.ng - 1) / g.ng;
   return g;
 }
+// Tensor-core passes (lqsgd_tc.cu): layers with m % 4 == 0 at padded rank >= 16.  The products run
+// on tcgen05 with every fp32 operand fed as a sum of narrow terms, fp32 accumulation in tensor
+// memory.  `maps` is the layer-major array of tensor maps (kTcMapsPerLayer per layer) that
+// tc_encode_maps() filled.
+constexpr int kTcMapsPerLayer = 2;   // 0: M as [W][n][m], box 128 x 32 x 1;  1: Pbt, box 32 x 3RP, 128-byte swizzle
+constexpr int kTcMapBytes = 128;
+constexpr int kTcRowChunk = 4096;    // most rows of a layer one pass-2 tile sums over (multiple of 64)
+int tc_encode_maps(const LayerDev* host_layers, int n_layers, int W, int RP, void* host_maps_out);   // 0 or LQSGD_ERR_CUDA
+cudaError_t launch_tc_pass2(int RP, const Tables& t, const Tile* tiles, int ntiles, const void* maps, Launch l);
 cudaError_t launch_stream_pass1(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
 cudaError_t launch_stream_pass3(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
 // Resident CTAs per SM of each streaming pass for this RP (for persistent grid sizing).

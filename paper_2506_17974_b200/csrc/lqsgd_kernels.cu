@@ -15,6 +15,8 @@
 // another CTA, and every reduction has a fixed order: results are bit-reproducible.
 #include "lqsgd_dev.h"
 
+#include <cuda_bf16.h>
+
 #include <math.h>
 
 namespace lqsgd {
@@ -630,6 +632,35 @@ q_reduce_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
   if (tid == 0) L.maxq[(size_t)fb.worker * L.nqb + fb.blk] = amax;
 }
 
+// One element of an averaged factor (P_bar or Q_bar) goes to its row-major home and to the
+// copies the passes read: the transposed Q of passes 1 and 3 and, for layers on the tensor-core
+// passes, the operands in the narrow terms those passes multiply (see lqsgd_tc.cu).
+__device__ __forceinline__ float tf32_remainder(float x) {
+  return x - __uint_as_float(__float_as_uint(x) & 0xffffe000u);
+}
+template <int RP>
+__device__ __forceinline__ void store_factor(const LayerDev& L, int which, int row, int col, float v) {
+  if (which) {
+    L.Q[(size_t)row * RP + col] = v;
+    L.Qt[(size_t)col * L.mt + row] = v;
+    if (L.tc) L.Qt[(size_t)(RP + col) * L.mt + row] = tf32_remainder(v);
+  } else {
+    L.Pbar[(size_t)row * RP + col] = v;
+    if (L.tc) {
+      // three bf16 terms v = b1 + b2 + b3 (24 bits), each stored twice in one word: the two K slots
+      // that face the bf16 pair of an element of M in the tensor-core pass 2
+      float rest = v;
+#pragma unroll
+      for (int term = 0; term < 3; ++term) {
+        const __nv_bfloat16 b = __float2bfloat16_rn(rest);
+        rest -= __bfloat162float(b);
+        const uint32_t h = __bfloat16_as_ushort(b);
+        reinterpret_cast<uint32_t*>(L.Pbt)[(size_t)(term * RP + col) * L.nt + row] = h | (h << 16);
+      }
+    }
+  }
+}
+
 // ---------------------------------------------------------------------------------------
 // Factor exchange (Alg. 1: LogQuantize, All-Reduce, LogDequantize) for one chunk of 256
 // factor elements of one layer, all W workers:
@@ -690,8 +721,7 @@ exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __rest
         pay[0] = bits32 & 0xff; pay[1] = (bits32 >> 8) & 0xff; pay[2] = (bits32 >> 16) & 0xff; pay[3] = bits32 >> 24;
       }
       const float v = sum / (float)W;
-      dst[(size_t)row * RP + col] = v;
-      if (which) L.Qt[(size_t)col * L.mt + row] = v;
+      store_factor<RP>(L, which, row, col, v);
     }
     if (ch.chunk == 0 && tid == 0) {
       L.scales[which] = s;
@@ -762,8 +792,7 @@ exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __rest
 
   if (valid && !sx.pack_only) {
     const float v = s_ok ? s * __ldg(qt.deq + S + W * (nlev - 1)) : 0.f;
-    dst[(size_t)row * RP + col] = v;
-    if (which) L.Qt[(size_t)col * L.mt + row] = v;
+    store_factor<RP>(L, which, row, col, v);
   }
   if (ch.chunk == 0 && tid == 0) {
     L.scales[which] = s;
@@ -778,11 +807,15 @@ exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __rest
 
 // Qt[j][i] = Q[i][j]: refreshes the transposed copy after Q was set from outside.
 __global__ void __launch_bounds__(256)
-q_transpose_kernel(const float* __restrict__ Q, float* __restrict__ Qt, int m, int RP, int mt) {
+q_transpose_kernel(const float* __restrict__ Q, float* __restrict__ Qt, int m, int RP, int mt, int tc) {
   pdl_wait();
   const int i = blockIdx.x * 256 + threadIdx.x;
   if (i >= m) return;
-  for (int j = 0; j < RP; ++j) Qt[(size_t)j * mt + i] = Q[(size_t)i * RP + j];
+  for (int j = 0; j < RP; ++j) {
+    const float v = Q[(size_t)i * RP + j];
+    Qt[(size_t)j * mt + i] = v;
+    if (tc) Qt[(size_t)(RP + j) * mt + i] = tf32_remainder(v);
+  }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -843,8 +876,7 @@ sum_dequant_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __r
     const float v = s_ok ? s * __ldg(qt.deq + S + n_streams * (nlev - 1)) : 0.f;
     const int row = e / r, col = e - row * r;
     float* dst = which ? L.Q : L.Pbar;
-    dst[(size_t)row * RP + col] = v;
-    if (which) L.Qt[(size_t)col * L.mt + row] = v;
+    store_factor<RP>(L, which, row, col, v);
   }
   if (ch.chunk == 0 && tid == 0) {
     L.scales[which] = s;
@@ -903,8 +935,8 @@ cudaError_t launch_pass1(int rp, const Tables& t, const Tile* tiles, int ntiles,
   return cudaGetLastError();
 }
 
-cudaError_t launch_q_transpose(const float* Q, float* Qt, int m, int RP, int mt, cudaStream_t stream) {
-  launch_pdl(q_transpose_kernel, (m + 255) / 256, 256, 0, stream, Q, Qt, m, RP, mt);
+cudaError_t launch_q_transpose(const float* Q, float* Qt, int m, int RP, int mt, int tc, cudaStream_t stream) {
+  launch_pdl(q_transpose_kernel, (m + 255) / 256, 256, 0, stream, Q, Qt, m, RP, mt, tc);
   return cudaGetLastError();
 }
 

@@ -72,8 +72,10 @@ def test_config5_rank_bit_points(rank, bits):
     run_steps(w, 1, free_run=False)
 
 
-def test_config5_sixteen_workers():
-    run_steps(wl.config5(2, 4), 1, free_run=False)
+@pytest.mark.parametrize("rank", [2, 16])
+def test_config5_sixteen_workers(rank):
+    """rank 16 puts the aligned layers on the tensor-core pass 2 with all 16 workers' tiles in one launch."""
+    run_steps(wl.config5(rank, 4), 1, free_run=False)
 
 
 @pytest.mark.parametrize("name", ["mnist", "resnet", "large", "rank8_workers3"])
