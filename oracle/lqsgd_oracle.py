@@ -128,6 +128,20 @@ def average_dequantize(codes_per_worker, s, bits, alpha):
     return np.float64(np.float32(s)) * expand(q_bar, alpha)
 
 
+def dequantize_average(codes_per_worker, s, bits, alpha):
+    """The other reading of the exchange (a parameter server that decodes what it receives,
+    Section V set-up): Eq. 5 applied to every worker's quantised value, then the mean of Eq. 1
+    over the dequantised values.  Not Algorithm 1's order (which averages first); offered as
+    a variant.  result = (1/W) sum_w s * expand(+-k_w / (L-1))."""
+    L = magnitude_levels(bits)
+    W = len(codes_per_worker)
+    total = np.zeros(np.asarray(codes_per_worker[0]).shape, dtype=np.float64)
+    for c in codes_per_worker:                      # worker order
+        q = signed_levels(c, bits).astype(np.float64) / (L - 1)
+        total += np.float64(np.float32(s)) * expand(q, alpha)
+    return total / W
+
+
 def pack_codes(codes, bits):
     """Little-endian bit stream: element i (row-major) occupies bits [i*b, (i+1)*b)."""
     flat = np.asarray(codes, dtype=np.uint8).reshape(-1)
@@ -175,14 +189,17 @@ def orthonormalize(P):
 # ----------------------------------------------------------------------------
 # One factor exchange: scale, quantise, All-Reduce, dequantise
 # ----------------------------------------------------------------------------
-def exchange_factor(factors, bits, alpha, forced_codes=None):
+def exchange_factor(factors, bits, alpha, forced_codes=None, average="codes"):
     """Quantise every worker's factor, average, dequantise (Alg. 1, the three lines
     after each product).  bits == 32 bypasses the quantiser (plain PowerSGD mean).
 
     forced_codes: optional list (per worker) of int16 arrays; entries >= 0 replace
     the code computed here (used by parity tests for near-threshold elements).
+    average: "codes" (Algorithm 1: mean of the quantised values, then Eq. 5) or "values"
+    (Eq. 5 per worker, then the mean).
     Returns dict(scale, codes[list], margin[list], mean) with mean in fp64.
     """
+    assert average in ("codes", "values")
     W = len(factors)
     if bits == 32:
         mean = sum(np.asarray(f, dtype=np.float64) for f in factors) / W
@@ -196,7 +213,7 @@ def exchange_factor(factors, bits, alpha, forced_codes=None):
             c = np.where(fc >= 0, fc, c).astype(np.uint8)
         codes.append(c)
         margins.append(mg)
-    mean = average_dequantize(codes, s, bits, alpha)
+    mean = (average_dequantize if average == "codes" else dequantize_average)(codes, s, bits, alpha)
     return dict(scale=s, codes=codes, margin=margins, mean=mean)
 
 
@@ -232,7 +249,7 @@ def effective_rank(rank, n, m):
     return min(rank, n, m)
 
 
-def layer_round(G, E, Q, bits_p, bits_q, alpha, forced_p=None, forced_q=None):
+def layer_round(G, E, Q, bits_p, bits_q, alpha, forced_p=None, forced_q=None, average="codes"):
     """One iteration of Algorithm 1 for one n x m layer and W workers.
 
     G, E: arrays [W, n, m];  Q: [m, r] shared by all workers (warm start).
@@ -247,10 +264,10 @@ def layer_round(G, E, Q, bits_p, bits_q, alpha, forced_p=None, forced_q=None):
     P_raw = [power_step_p(M[w], Q) for w in range(W)]
     orth = [orthonormalize(P_raw[w]) for w in range(W)]
     P = [o[0] for o in orth]
-    xp = exchange_factor(P, bits_p, alpha, forced_p)
+    xp = exchange_factor(P, bits_p, alpha, forced_p, average)
     P_bar = xp["mean"]
     Qw = [power_step_q(M[w], P_bar) for w in range(W)]
-    xq = exchange_factor(Qw, bits_q, alpha, forced_q)
+    xq = exchange_factor(Qw, bits_q, alpha, forced_q, average)
     Q_bar = xq["mean"]
     G_hat = reconstruct(P_bar, Q_bar)
     E_new = [error_update(M[w], G_hat) for w in range(W)]
@@ -304,8 +321,9 @@ class Oracle:
     """State machine of Algorithm 1 over a list of layers: E_0 = 0, Q_0 supplied by the
     caller (drawn N(0,1) outside), Q_t = dequantised averaged Q of step t-1."""
 
-    def __init__(self, layers, rank, bits_p, bits_q, alpha, workers, Q0):
+    def __init__(self, layers, rank, bits_p, bits_q, alpha, workers, Q0, average="codes"):
         self.layers = [tuple(s) for s in layers]
+        self.average = average
         self.rank, self.bits_p, self.bits_q = rank, bits_p, bits_q
         self.alpha, self.W = float(alpha), workers
         self.E, self.Q = {}, {}
@@ -326,7 +344,7 @@ class Oracle:
             if li in self.E:
                 f = (forced or {}).get(li, (None, None))
                 res = layer_round(Gl, self.E[li], self.Q[li], self.bits_p, self.bits_q,
-                                  self.alpha, f[0], f[1])
+                                  self.alpha, f[0], f[1], self.average)
                 self.E[li] = res["E_new"]
                 self.Q[li] = res["Q_bar"]
             else:

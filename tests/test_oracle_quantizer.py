@@ -148,6 +148,41 @@ def test_worker_average_is_exact_integer_mean():
     assert v[0] == 0.0
 
 
+def test_value_domain_average_variant():
+    """Eq. 5 per worker, then the mean (the parameter-server reading): hand cases with
+    b = 4, alpha = 127 (levels (2^k - 1)/127), the one-worker case, and the convexity relation
+    to Algorithm 1's order."""
+    # k = +3 and k = -1, s = 2:  (7/127 - 1/127) / 2 * 2 = 6/127
+    v = orc.dequantize_average([np.array([3], np.uint8), np.array([8 | 1], np.uint8)], np.float32(2.0), 4, 127.0)
+    assert v[0] == pytest.approx(6.0 / 127.0, rel=1e-13)
+    # k = +7 and k = 0: half of full scale, where the code-domain mean gives (128^(1/2) - 1)/127
+    v = orc.dequantize_average([np.array([7], np.uint8), np.array([0], np.uint8)], np.float32(1), 4, 127.0)
+    c = orc.average_dequantize([np.array([7], np.uint8), np.array([0], np.uint8)], np.float32(1), 4, 127.0)
+    assert v[0] == pytest.approx(0.5, rel=1e-13)
+    assert c[0] == pytest.approx((np.sqrt(128.0) - 1) / 127.0, rel=1e-13)
+    rng = np.random.default_rng(5)
+    bits, alpha, W = 5, 50.0, 6
+    xs = [rng.standard_normal(400).astype(np.float32) for _ in range(W)]
+    s = orc.factor_scale(xs)
+    codes = [orc.log_quantize(x, s, bits, alpha) for x in xs]
+    # one worker: both orders are the plain dequantisation
+    assert np.array_equal(orc.dequantize_average(codes[:1], s, bits, alpha), orc.average_dequantize(codes[:1], s, bits, alpha))
+    # it is the mean of the per-worker dequantised values, whatever the order of the workers
+    per = np.stack([orc.average_dequantize([c], s, bits, alpha) for c in codes])
+    assert np.allclose(orc.dequantize_average(codes, s, bits, alpha), per.mean(axis=0), rtol=1e-14, atol=0)
+    assert np.allclose(orc.dequantize_average(codes[::-1], s, bits, alpha), per.mean(axis=0), rtol=1e-14, atol=0)
+    # expand() is convex on [0, 1] and odd: where all workers agree in sign, averaging after
+    # dequantisation is at least as large in magnitude as dequantising the average
+    sg = np.stack([orc.signed_levels(c, bits) for c in codes])
+    same_sign = (sg >= 0).all(axis=0) | (sg <= 0).all(axis=0)
+    a = np.abs(orc.dequantize_average(codes, s, bits, alpha))[same_sign]
+    b = np.abs(orc.average_dequantize(codes, s, bits, alpha))[same_sign]
+    assert same_sign.sum() > 5 and np.all(a >= b * (1 - 1e-14))
+    # exchange_factor routes to it
+    x = orc.exchange_factor(xs, bits, alpha, average="values")
+    assert np.array_equal(x["mean"], orc.dequantize_average(codes, s, bits, alpha))
+
+
 @pytest.mark.parametrize("bits", [2, 3, 4, 5, 8])
 def test_pack_layout_and_size(bits):
     rng = np.random.default_rng(bits)
