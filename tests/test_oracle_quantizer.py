@@ -169,8 +169,8 @@ def test_value_domain_average_variant():
     assert np.array_equal(orc.dequantize_average(codes[:1], s, bits, alpha), orc.average_dequantize(codes[:1], s, bits, alpha))
     # it is the mean of the per-worker dequantised values, whatever the order of the workers
     per = np.stack([orc.average_dequantize([c], s, bits, alpha) for c in codes])
-    assert np.allclose(orc.dequantize_average(codes, s, bits, alpha), per.mean(axis=0), rtol=1e-14, atol=0)
-    assert np.allclose(orc.dequantize_average(codes[::-1], s, bits, alpha), per.mean(axis=0), rtol=1e-14, atol=0)
+    assert np.allclose(orc.dequantize_average(codes, s, bits, alpha), per.mean(axis=0), rtol=1e-13, atol=1e-13 * float(s))
+    assert np.allclose(orc.dequantize_average(codes[::-1], s, bits, alpha), per.mean(axis=0), rtol=1e-13, atol=1e-13 * float(s))
     # expand() is convex on [0, 1] and odd: where all workers agree in sign, averaging after
     # dequantisation is at least as large in magnitude as dequantising the average
     sg = np.stack([orc.signed_levels(c, bits) for c in codes])
