@@ -77,6 +77,10 @@ typedef enum lqsgd_error {
 /* Config flags. */
 #define LQSGD_FLAG_HOST_STAGING 1u /* reserve device staging in the workspace so that lqsgd_step_host() works */
 #define LQSGD_FLAG_REGISTER_PATH 2u /* stream every layer with the register-path kernels (no bulk-copy staging) */
+#define LQSGD_FLAG_AVERAGE_VALUES 4u /* variant of the exchange: Eq. 5 on every worker's quantised factor, then the mean
+                                        of Eq. 1 over the dequantised values (a parameter server that decodes what it
+                                        receives, Section V).  Default, as Algorithm 1 writes it: mean of the quantised
+                                        values, then Eq. 5 once.  Codes, scales and payload are the same in both. */
 
 typedef struct lqsgd_ctx lqsgd_ctx;
 

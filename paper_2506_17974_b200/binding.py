@@ -21,6 +21,7 @@ STATE_E, STATE_Q, STATE_P_RAW, STATE_P, STATE_P_BAR, STATE_Q_W, STATE_CODES_P, S
 STATUS_DEPENDENT_COLUMN, STATUS_ZERO_SCALE_P, STATUS_ZERO_SCALE_Q, STATUS_NONFINITE = 1, 2, 4, 8
 FLAG_HOST_STAGING = 1
 FLAG_REGISTER_PATH = 2
+FLAG_AVERAGE_VALUES = 4
 STATUS_TIMEOUT = 16
 N_PHASES = 5
 XCHG_SCALES_P, XCHG_SCALES_Q, XCHG_STREAMS_P, XCHG_STREAMS_Q = range(4)
@@ -151,16 +152,21 @@ class LQSGD:
 
     def __init__(self, layers: Sequence[Tuple[int, int]], rank: int, bits_p: int, bits_q: Optional[int] = None,
                  alpha: float = 127.0, workers: int = 1, seed: int = 0, host_staging: bool = False,
-                 device: str = "cuda:0", register_path: bool = False, world_workers: int = 0):
+                 device: str = "cuda:0", register_path: bool = False, world_workers: int = 0,
+                 average: str = "codes"):
         self.lib = load_library()
         self.layers = [(int(n), int(m)) for n, m in layers]
         self.rank, self.bits_p = rank, bits_p
         self.bits_q = bits_p if bits_q is None else bits_q
         self.alpha, self.W = float(alpha), workers
+        if average not in ("codes", "values"):
+            raise ValueError("average must be 'codes' (Algorithm 1) or 'values'")
+        self.average = average
         self.device = torch.device(device)
         self.cfg = make_config(rank, self.bits_p, self.bits_q, alpha, workers, seed,
                                (FLAG_HOST_STAGING if host_staging else 0)
-                               | (FLAG_REGISTER_PATH if register_path else 0), world_workers)
+                               | (FLAG_REGISTER_PATH if register_path else 0)
+                               | (FLAG_AVERAGE_VALUES if average == "values" else 0), world_workers)
         nbytes = workspace_bytes(self.layers, self.cfg)
         with torch.cuda.device(self.device):
             self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)

@@ -99,7 +99,7 @@ int check_config(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
     if (c->world_workers < c->workers || c->world_workers > 4096 || c->world_workers % c->workers) return LQSGD_ERR_INVALID_ARG;
     if (c->world_workers > c->workers && (c->bits_p == 32 || c->bits_q == 32)) return LQSGD_ERR_INVALID_ARG;
   }
-  if (c->flags & ~(LQSGD_FLAG_HOST_STAGING | LQSGD_FLAG_REGISTER_PATH)) return LQSGD_ERR_INVALID_ARG;
+  if (c->flags & ~(LQSGD_FLAG_HOST_STAGING | LQSGD_FLAG_REGISTER_PATH | LQSGD_FLAG_AVERAGE_VALUES)) return LQSGD_ERR_INVALID_ARG;
   for (int i = 0; i < n_layers; ++i) {
     if (shapes[i].rows < 1 || shapes[i].cols < 1) return LQSGD_ERR_BAD_SHAPE;
     if ((int64_t)shapes[i].rows * shapes[i].cols > (int64_t)1 << 30) return LQSGD_ERR_BAD_SHAPE;
@@ -369,8 +369,10 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   p.d_xsend[1] = a.take<uint8_t>((size_t)W * p.region_bytes[1]);
   p.state_end = a.off;
 
-  quant_tables(cfg.bits_p, cfg.alpha, p.W_total, p.thrP, p.deqP);
-  quant_tables(cfg.bits_q, cfg.alpha, p.W_total, p.thrQ, p.deqQ);
+  // value-domain average: the table of one worker's dequantised levels serves every worker
+  const int table_w = (cfg.flags & LQSGD_FLAG_AVERAGE_VALUES) ? 1 : p.W_total;
+  quant_tables(cfg.bits_p, cfg.alpha, table_w, p.thrP, p.deqP);
+  quant_tables(cfg.bits_q, cfg.alpha, table_w, p.thrQ, p.deqQ);
   p.d_tiles1 = a.take<Tile>(p.tiles1.size());
   p.d_tiles2 = a.take<Tile>(p.tiles2.size());
   p.d_tiles3 = a.take<Tile>(p.tiles3.size());
@@ -647,7 +649,8 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
   const int W = p.W, RP = p.RP;
   const size_t nm = p.mats.size(), nv = p.vecs.size();
   const size_t vbase = nm * (W + 2);
-  const QuantTables qp{p.d_thrP, p.d_deqP, c->cfg.bits_p}, qq{p.d_thrQ, p.d_deqQ, c->cfg.bits_q};
+  const int avg_values = (c->cfg.flags & LQSGD_FLAG_AVERAGE_VALUES) ? 1 : 0;
+  const QuantTables qp{p.d_thrP, p.d_deqP, c->cfg.bits_p, avg_values}, qq{p.d_thrQ, p.d_deqQ, c->cfg.bits_q, avg_values};
   SplitExchange sx{};
   sx.pack_only = split ? 1 : 0;
   sx.n_mat = (int)nm;

@@ -85,8 +85,10 @@ struct Tables {
 
 struct QuantTables {
   const float* thr;           // [L-1] ascending decision thresholds on |x|/s
-  const float* deq;           // [2*W*(L-1)+1] expand(S / (W (L-1))), index S + W (L-1)
+  const float* deq;           // [2*W*(L-1)+1] expand(S / (W (L-1))), index S + W (L-1); with avg_values the
+                              // table is the one of a single worker: [2*(L-1)+1], index (+-k) + (L-1)
   int32_t bits;
+  int32_t avg_values;         // 1: dequantise every worker's code, then average (variant); 0: Algorithm 1's order
 };
 
 // Programmatic dependent launch: every kernel of the round is launched so that its launch may

@@ -743,6 +743,7 @@ exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __rest
   const size_t byte0 = (size_t)ch.chunk * (CH / 8) * b;
   const int nbytes = (int)min((size_t)(CH / 8) * b, nbytes_total - byte0);
   int S = 0;
+  float Sv = 0.f;          // value-domain variant: sum of the workers' dequantised levels, in worker order
 
   for (int w0 = 0; w0 < W; w0 += WB) {
     const int wn = min(WB, W - w0);
@@ -768,6 +769,7 @@ exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __rest
         codes[u][tid] = code;                        // 0 beyond the factor's end: pads the last byte
         if (valid) ucodes[(size_t)(w0 + u) * count + e] = code;
         S += neg ? -k : k;
+        if (qt.avg_values) Sv += __ldg(qt.deq + (neg ? -k : k) + (nlev - 1));
       }
     }
     __syncthreads();
@@ -791,7 +793,8 @@ exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __rest
   }
 
   if (valid && !sx.pack_only) {
-    const float v = s_ok ? s * __ldg(qt.deq + S + W * (nlev - 1)) : 0.f;
+    float v = 0.f;
+    if (s_ok) v = qt.avg_values ? s * (Sv / (float)W) : s * __ldg(qt.deq + S + W * (nlev - 1));
     store_factor<RP>(L, which, row, col, v);
   }
   if (ch.chunk == 0 && tid == 0) {
@@ -865,15 +868,19 @@ sum_dequant_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __r
     const size_t bit = (size_t)e * b, byte = bit >> 3;
     const int sh = (int)(bit & 7);
     int S = 0;
+    float Sv = 0.f;
     for (int w = 0; w < n_streams; ++w) {
       const uint8_t* st = gathered + (size_t)w * sx.region_bytes[which] + off;
       unsigned v = st[byte];
       if (sh + b > 8 && byte + 1 < nbytes) v |= (unsigned)st[byte + 1] << 8;
       const unsigned code = (v >> sh) & ((1u << b) - 1u);
       const int k = (int)(code & (unsigned)(nlev - 1));
-      S += (code >> (b - 1)) ? -k : k;
+      const int sk = (code >> (b - 1)) ? -k : k;
+      S += sk;
+      if (qt.avg_values) Sv += __ldg(qt.deq + sk + (nlev - 1));
     }
-    const float v = s_ok ? s * __ldg(qt.deq + S + n_streams * (nlev - 1)) : 0.f;
+    float v = 0.f;
+    if (s_ok) v = qt.avg_values ? s * (Sv / (float)n_streams) : s * __ldg(qt.deq + S + n_streams * (nlev - 1));
     const int row = e / r, col = e - row * r;
     float* dst = which ? L.Q : L.Pbar;
     store_factor<RP>(L, which, row, col, v);

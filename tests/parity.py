@@ -58,7 +58,7 @@ def snapshot_state(comp: B.LQSGD):
     return E, Q
 
 
-def check_exchange(x_dev, codes_dev, scale_dev, bar_dev, bits, alpha, stats):
+def check_exchange(x_dev, codes_dev, scale_dev, bar_dev, bits, alpha, stats, average="codes"):
     """Scale, codes and dequantised mean of one factor against the oracle, on the device's factor."""
     s = orc.factor_scale(list(x_dev))
     assert np.float32(scale_dev) == s, (scale_dev, s)
@@ -77,7 +77,8 @@ def check_exchange(x_dev, codes_dev, scale_dev, bar_dev, bits, alpha, stats):
         total += c.size
     stats["flips"] = stats.get("flips", 0) + flips
     stats["codes"] = stats.get("codes", 0) + total
-    mean = orc.average_dequantize(codes_dev, s, bits, alpha)       # from the device's codes
+    avg = orc.average_dequantize if average == "codes" else orc.dequantize_average
+    mean = avg(codes_dev, s, bits, alpha)                          # from the device's codes
     assert rel_fro(bar_dev, mean) <= 1e-6
     return s
 
@@ -90,9 +91,9 @@ def check_layer_stage_isolated(comp: B.LQSGD, layer: int, G, rec: StepRecord, st
     errs["P_raw"] = max(rel_fro(rec.P_raw[w], orc.power_step_p(M[w], rec.Q_prev)) for w in range(W))
     orth = [orc.orthonormalize(rec.P_raw[w]) for w in range(W)]
     errs["P"] = max(rel_fro(rec.P[w], orth[w][0]) for w in range(W))
-    check_exchange(rec.P, rec.codes_p, rec.scales[0], rec.P_bar, comp.bits_p, comp.alpha, stats)
+    check_exchange(rec.P, rec.codes_p, rec.scales[0], rec.P_bar, comp.bits_p, comp.alpha, stats, comp.average)
     errs["Qw"] = max(rel_fro(rec.Qw[w], orc.power_step_q(M[w], rec.P_bar)) for w in range(W))
-    check_exchange(rec.Qw, rec.codes_q, rec.scales[1], rec.Q_bar, comp.bits_q, comp.alpha, stats)
+    check_exchange(rec.Qw, rec.codes_q, rec.scales[1], rec.Q_bar, comp.bits_q, comp.alpha, stats, comp.average)
     G_hat = orc.reconstruct(rec.P_bar, rec.Q_bar)
     errs["G_hat"] = rel_fro(rec.G_hat, G_hat)
     errs["E"] = max(rel_fro(rec.E_new[w], orc.error_update(M[w], G_hat)) for w in range(W))
@@ -150,14 +151,14 @@ def oracle_step_forced(oracle: orc.Oracle, grads_host, recs, stats):
         n, m = oracle.layers[l]
         Gl = np.stack([np.asarray(grads_host[w][l], dtype=np.float32).reshape(n, m) for w in range(oracle.W)])
         args = (Gl, oracle.E[l], oracle.Q[l], oracle.bits_p, oracle.bits_q, oracle.alpha)
-        res = orc.layer_round(*args)
+        res = orc.layer_round(*args, average=oracle.average)
         fp = []
         for w in range(oracle.W):
             diff = res["xp"]["codes"][w] != rec.codes_p[w]
             stats["forced"] = stats.get("forced", 0) + int(diff.sum())
             assert np.all(res["xp"]["margin"][w][diff] < 2e-2), "P code differs far from a threshold"
             fp.append(np.where(diff, rec.codes_p[w].astype(np.int16), -1))
-        res = orc.layer_round(*args, forced_p=fp)
+        res = orc.layer_round(*args, forced_p=fp, average=oracle.average)
         fq = []
         for w in range(oracle.W):
             diff = res["xq"]["codes"][w] != rec.codes_q[w]

@@ -21,13 +21,13 @@ DEV = "cuda:0"
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("bits", [4, 3])
-def test_two_emulated_ranks_equal_one_process_bitwise(bits):
+@pytest.mark.parametrize("bits,average", [(4, "codes"), (3, "codes"), (4, "values")])
+def test_two_emulated_ranks_equal_one_process_bitwise(bits, average):
     from paper_2506_17974_b200 import binding as B
     w = wl.Workload("dist", ((96, 200), (64, 27), (130, 36), (20, 1), (512, 1152)), rank=4, bits=bits, workers=4,
                     steps=3, dist="student_t3", scale="fan_in", seed=5)
-    ref = B.LQSGD(w.layers, w.rank, bits, workers=4, seed=5)
-    ranks = [B.LQSGD(w.layers, w.rank, bits, workers=2, seed=5, world_workers=4) for _ in range(2)]
+    ref = B.LQSGD(w.layers, w.rank, bits, workers=4, seed=5, average=average)
+    ranks = [B.LQSGD(w.layers, w.rank, bits, workers=2, seed=5, world_workers=4, average=average) for _ in range(2)]
     nl = len(w.layers)
     for t in range(3):
         g = wl.draw_gradients(w, t, device=DEV)

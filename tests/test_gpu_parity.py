@@ -24,7 +24,7 @@ def make(w: wl.Workload, **kw):
 
 def new_oracle(comp: B.LQSGD):
     Q0 = {l: par.host(comp.get_state(B.STATE_Q, l)) for l in range(len(comp.layers)) if comp.is_matrix(l)}
-    return orc.Oracle(comp.layers, comp.rank, comp.bits_p, comp.bits_q, comp.alpha, comp.W, Q0)
+    return orc.Oracle(comp.layers, comp.rank, comp.bits_p, comp.bits_q, comp.alpha, comp.W, Q0, average=comp.average)
 
 
 def run_steps(w: wl.Workload, steps: int, free_run=True, comp=None):
@@ -121,6 +121,27 @@ def test_small_and_ragged_shapes(shape, rank, bits, W):
         for l, rec in recs.items():
             assert par.rel_fro(rec.G_hat, out[l]["G_hat"]) <= par.TOL
             assert par.rel_fro(rec.E_new, out[l]["E_new"]) <= par.TOL
+
+
+@pytest.mark.parametrize("W,bits", [(3, 4), (5, 3), (2, 8)])
+def test_value_domain_average_variant(W, bits):
+    """LQSGD_FLAG_AVERAGE_VALUES: every worker's code dequantised (Eq. 5), then averaged (Eq. 1).
+    Same codes and payload as Algorithm 1's order, another P_bar / Q_bar; checked stage by stage and
+    over free-running steps against the oracle in the same mode."""
+    w = wl.Workload("avgv", ((96, 200), (130, 36), (64, 27), (20, 1)), rank=4, bits=bits, workers=W, steps=3,
+                    dist="student_t3", scale="fan_in", seed=31)
+    a = make(w, average="values")
+    run_steps(w, 3, comp=a)
+    # against the default mode: identical codes on the first exchange of P, different averages when W > 1
+    b, c = make(w, average="values"), make(w)
+    g = wl.draw_gradients(w, 0, device=DEV)
+    ob = [torch.empty(s, device=DEV) for s in w.layers]
+    oc = [torch.empty(s, device=DEV) for s in w.layers]
+    b.step(g, ob)
+    c.step(g, oc)
+    torch.cuda.synchronize()
+    assert torch.equal(b.get_state(B.STATE_CODES_P, 0, W - 1), c.get_state(B.STATE_CODES_P, 0, W - 1))
+    assert not torch.equal(b.get_state(B.STATE_P_BAR, 0), c.get_state(B.STATE_P_BAR, 0))
 
 
 def test_different_bits_for_p_and_q():
