@@ -55,6 +55,9 @@ struct Plan {
   std::vector<Tile> tiles1, tiles2, tiles3;      // register-path passes
   std::vector<Tile> stiles1, stiles3;            // bulk-copy staged passes 1 and 3
   std::vector<Tile> tctiles2;                    // tensor-core pass 2
+  std::vector<Tile> tctiles1;                    // tensor-core pass 1, grouped by CTA
+  std::vector<int> tcbegin1;                     // [tc_grid + 1]
+  int tc_grid = 0;
   std::vector<uint8_t> tcmaps;                   // tensor maps of the tensor-core passes (filled at create)
   std::vector<FactorBlock> fbP, fbQ;
   std::vector<ExchangeChunk> chP, chQ, chV;
@@ -69,6 +72,8 @@ struct Plan {
   Tile *d_tiles1 = nullptr, *d_tiles2 = nullptr, *d_tiles3 = nullptr;
   Tile *d_stiles1 = nullptr, *d_stiles3 = nullptr;
   Tile* d_tctiles2 = nullptr;
+  Tile* d_tctiles1 = nullptr;
+  int* d_tcbegin1 = nullptr;
   uint8_t* d_tcmaps = nullptr;
   FactorBlock *d_fbP = nullptr, *d_fbQ = nullptr;
   ExchangeChunk *d_chP = nullptr, *d_chQ = nullptr, *d_chV = nullptr;
@@ -282,7 +287,9 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
     const int cw = chunk_width(mt.m, c1);
     // pass 2: register path, or tensor cores (row chunks in multiples of the 64 rows of an operand slot)
     const int tr2 = tc ? (int)align_up((size_t)balanced_rows(mt.n, kTcRowChunk), 64) : balanced_rows(mt.n, r2);
-    L.ncc = st ? (int)scols.size() : ceil_div(mt.m, cw);
+    // tensor-core pass 1: column chunks balanced in units of 32 columns, at most kTcPass1Cols wide
+    const int tc_units = ceil_div(mt.m, 32), tc_ncc = ceil_div(tc_units * 32, kTcPass1Cols);
+    L.ncc = tc ? tc_ncc : (st ? (int)scols.size() : ceil_div(mt.m, cw));
     L.nrb = ceil_div(mt.n, tr2);
     L.npb = ceil_div(mt.n, kFactorBlockRows);
     L.nqb = ceil_div(mt.m, kFactorBlockRows);
@@ -321,7 +328,18 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
         for (int cc = 0; cc < (int)scols.size(); ++cc)
           p.stiles3.push_back({li32, 0, rb * tr3, std::min(tr3, mt.n - rb * tr3), scols[cc].first, scols[cc].second, 0, 0});
     }
-    for (int rb = 0; !st && rb < ceil_div(mt.n, kPass1Rows); ++rb)
+    if (tc) {
+      int u0 = 0;
+      for (int cc = 0; cc < tc_ncc; ++cc) {
+        const int nu = tc_units / tc_ncc + (cc < tc_units % tc_ncc ? 1 : 0);
+        const int col0 = u0 * 32, ncols = std::min(nu * 32, mt.m - col0);
+        for (int rb = 0; rb < ceil_div(mt.n, kTcRowsPerTile); ++rb)
+          for (int w = 0; w < W; ++w)
+            p.tctiles1.push_back({li32, w, rb * kTcRowsPerTile, std::min(kTcRowsPerTile, mt.n - rb * kTcRowsPerTile), col0, ncols, cc, 0});
+        u0 += nu;
+      }
+    }
+    for (int rb = 0; !st && !tc && rb < ceil_div(mt.n, kPass1Rows); ++rb)
       for (int cc = 0; cc < L.ncc; ++cc)
         for (int w = 0; w < W; ++w) {
           const int row0 = rb * kPass1Rows, col0 = cc * cw;
@@ -362,6 +380,26 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   // The tensor-core kernels deal their tiles round-robin to one CTA per SM: largest first, so the
   // CTAs finish together.
   std::stable_sort(p.tctiles2.begin(), p.tctiles2.end(), [](const Tile& x, const Tile& y) { return x.nrows > y.nrows; });
+  // Pass 1: longest tile first to the CTA with the least work so far (a tile costs its column count:
+  // every stage is 128 rows deep whatever the tile's row count), then grouped by CTA.
+  p.tc_grid = sm_count;
+  {
+    std::vector<Tile> sorted = p.tctiles1;
+    std::stable_sort(sorted.begin(), sorted.end(), [](const Tile& x, const Tile& y) { return x.ncols > y.ncols; });
+    std::vector<std::vector<Tile>> per(p.tc_grid);
+    std::vector<long> load(p.tc_grid, 0);
+    for (const Tile& tl : sorted) {
+      const int b = (int)(std::min_element(load.begin(), load.end()) - load.begin());
+      per[b].push_back(tl);
+      load[b] += ceil_div(tl.ncols, 32);
+    }
+    p.tctiles1.clear();
+    p.tcbegin1.assign(p.tc_grid + 1, 0);
+    for (int b = 0; b < p.tc_grid; ++b) {
+      p.tctiles1.insert(p.tctiles1.end(), per[b].begin(), per[b].end());
+      p.tcbegin1[b + 1] = (int)p.tctiles1.size();
+    }
+  }
   p.d_status = a.take<uint32_t>(p.mats.size());
   p.d_payload = a.take<uint8_t>((size_t)W * p.payload_stride);
   p.d_xscales = a.take<float>(2 * p.mats.size());
@@ -379,6 +417,8 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   p.d_stiles1 = a.take<Tile>(p.stiles1.size());
   p.d_stiles3 = a.take<Tile>(p.stiles3.size());
   p.d_tctiles2 = a.take<Tile>(p.tctiles2.size());
+  p.d_tctiles1 = a.take<Tile>(p.tctiles1.size());
+  p.d_tcbegin1 = a.take<int>(p.tcbegin1.size());
   p.d_tcmaps = a.take<uint8_t>(p.mats.size() * kTcMapsPerLayer * kTcMapBytes);
   p.d_fbP = a.take<FactorBlock>(p.fbP.size());
   p.d_fbQ = a.take<FactorBlock>(p.fbQ.size());
@@ -511,6 +551,8 @@ int lqsgd_create(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
   CK(up(p.d_stiles1, p.stiles1.data(), p.stiles1.size() * sizeof(Tile)));
   CK(up(p.d_stiles3, p.stiles3.data(), p.stiles3.size() * sizeof(Tile)));
   CK(up(p.d_tctiles2, p.tctiles2.data(), p.tctiles2.size() * sizeof(Tile)));
+  CK(up(p.d_tctiles1, p.tctiles1.data(), p.tctiles1.size() * sizeof(Tile)));
+  CK(up(p.d_tcbegin1, p.tcbegin1.data(), p.tcbegin1.size() * sizeof(int)));
   p.tcmaps.resize(p.mats.size() * kTcMapsPerLayer * kTcMapBytes + 1);
   rc = tc_encode_maps(p.layers.data(), (int)p.layers.size(), p.W, p.RP, p.tcmaps.data());
   if (rc != LQSGD_OK) { g_cuda_error = "cuTensorMapEncodeTiled failed or is not available"; return rc; }
@@ -566,7 +608,7 @@ int lqsgd_launches_per_step(const lqsgd_ctx* ctx, int32_t* out) {
   const Plan& p = ctx->plan;
   // Orthonormalize (2), exchange of P, Q_w reduction, exchange of Q; then one launch per non-empty tile list
   *out = (p.mats.empty() ? 0 : 5) + (p.tiles1.empty() ? 0 : 2) + (p.stiles1.empty() ? 0 : 2) + (p.tiles2.empty() ? 0 : 1) +
-         (p.tctiles2.empty() ? 0 : 1) + (p.chV.empty() ? 0 : 1);
+         (p.tctiles2.empty() ? 0 : 1) + (p.tctiles1.empty() ? 0 : 1) + (p.chV.empty() ? 0 : 1);
   return LQSGD_OK;
 }
 
@@ -674,6 +716,7 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
       if (nm) {
         CK(launch_pass1(RP, t, p.d_tiles1, (int)p.tiles1.size(), {st, c->grid1}));
         CK(launch_stream_pass1(RP, t, p.d_stiles1, (int)p.stiles1.size(), {st, (int)std::min<size_t>(p.stiles1.size(), c->sm_count)}));
+        CK(launch_tc_pass1(RP, t, p.d_tctiles1, (int)p.tctiles1.size(), p.d_tcbegin1, p.d_tcmaps, {st, p.tc_grid}));
       }
       PHASE_MARK(1);
       if (nm) {

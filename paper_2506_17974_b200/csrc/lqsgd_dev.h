@@ -186,11 +186,17 @@ __host__ __device__ inline StreamGeo stream_geo(int ncols, int RP) {
 // on tcgen05 with every fp32 operand fed as a sum of narrow terms, fp32 accumulation in tensor
 // memory.  `maps` is the layer-major array of tensor maps (kTcMapsPerLayer per layer) that
 // tc_encode_maps() filled.
-constexpr int kTcMapsPerLayer = 2;   // 0: M as [W][n][m], box 128 x 32 x 1;  1: Pbt, box 32 x 3RP, 128-byte swizzle
+constexpr int kTcMapsPerLayer = 4;   // 0: M as [W][n][m], box 128 x 32 x 1;  1: Pbt, box 32 x 3RP, 128-byte swizzle;
+                                     // 2: E / M as [W][n][m], box 32 x 128 x 1, swizzled;  3: Qt, box 32 x 2RP, swizzled
+constexpr int kTcRowsPerTile = 128;  // rows of a pass-1 tile: the M extent of one MMA
+constexpr int kTcPass1Cols = 576;    // most columns of a pass-1 tile (multiple of 32): small enough to balance the SMs
 constexpr int kTcMapBytes = 128;
 constexpr int kTcRowChunk = 4096;    // most rows of a layer one pass-2 tile sums over (multiple of 64)
 int tc_encode_maps(const LayerDev* host_layers, int n_layers, int W, int RP, void* host_maps_out);   // 0 or LQSGD_ERR_CUDA
 cudaError_t launch_tc_pass2(int RP, const Tables& t, const Tile* tiles, int ntiles, const void* maps, Launch l);
+// tiles are grouped by CTA: CTA b takes tiles [cta_begin[b], cta_begin[b + 1]); l.grid CTAs
+cudaError_t launch_tc_pass1(int RP, const Tables& t, const Tile* tiles, int ntiles, const int* cta_begin, const void* maps,
+                            Launch l);
 cudaError_t launch_stream_pass1(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
 cudaError_t launch_stream_pass3(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
 // Resident CTAs per SM of each streaming pass for this RP (for persistent grid sizing).

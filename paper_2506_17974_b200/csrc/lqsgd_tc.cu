@@ -331,6 +331,316 @@ tc_pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, const uint
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)S::kTmemCols) : "memory");
 }
 
+// ---------------------------------------------------------------------------------------
+// Pass 1 on the tensor core (P_w = M_w Q with M = G + E, Alg. 1; M is written over E).
+//
+// A tile is 128 rows of one worker's layer over a chunk of columns; the rows are the M extent
+// of the MMA (TMEM lane = row), the columns the K extent, 32 per stage.  The HBM traffic per
+// element is three times that of pass 2 (read G, read E, write M), so the tensor core has
+// slack and the product keeps fp32 accuracy: tf32 operands, m = hi + lo with hi the truncation
+// the hardware applies to the fp32 container and lo = m - hi, and per k-step
+//   D[:, 0:2RP) += A_hi [Q_hi ; Q_lo]^T ,   D[:, 0:RP) += A_lo Q_hi^T
+// (Q^T and its tf32 remainders are kept as 2 RP rows in global memory).  The epilogue adds the
+// two halves of D.
+//
+// Stage of the ring: the 128 x 32 piece of E by TMA (128-byte swizzle: a thread reading its own
+// row touches every bank once per quarter warp) and the same piece of G by cp.async from the
+// caller's tensor (16-byte granules placed at the swizzled positions; rows and columns past the
+// layer are zero-filled).  A consumer thread adds its row of the two pieces, puts m back into the
+// E piece (a storer thread sends it to global memory with a TMA tensor store) and writes hi and
+// lo to TMEM.
+// ---------------------------------------------------------------------------------------
+constexpr int kT1Stages = 5;          // ring of (G, E) pieces, 2 x 16 KB each
+constexpr int kT1AB = 4;              // ring of A (TMEM, hi + lo: 64 columns) and B (shared memory) buffers
+constexpr uint32_t kT1PieceBytes = 128 * 128;   // 128 rows x 32 fp32
+
+__device__ __forceinline__ void tc_mma_tf32_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n}"
+               ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Instruction descriptor: tf32 x tf32 -> fp32, both operands K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t tc_idesc_tf32(int n) {
+  return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tma_store_3d(const void* tmap, int x, int y, int z, const void* smem_src) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3}], [%4];"
+               ::"l"(tmap), "r"(x), "r"(y), "r"(z), "r"(smem_u32(smem_src)) : "memory");
+}
+// 16 bytes global -> shared, asynchronous; src_bytes = 0 writes zeros and reads nothing
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(src_bytes) : "memory");
+}
+// the executing thread's cp.async copies issued so far arrive on `bar` when they have landed
+__device__ __forceinline__ void cp_async_arrive(uint64_t* bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+template <int RP>
+struct Pass1Cfg {
+  static constexpr int kDStride = 2 * RP <= 64 ? 64 : (2 * RP <= 128 ? 128 : 256);
+  static constexpr int kACol0 = 2 * kDStride;
+  static constexpr int kTmemCols = 512;
+  static constexpr uint32_t kBBytes = 2 * RP * 128;                      // Q_hi rows, then Q_lo rows, 32 columns
+  static constexpr uint32_t kBOff = kT1Stages * 2 * kT1PieceBytes;
+  static constexpr uint32_t kBarOff = kBOff + kT1AB * kBBytes;
+  static constexpr int kBars = 3 * kT1Stages + 2 * kT1AB + 2 + 2 + 1;
+  static constexpr uint32_t kTotal = kBarOff + kBars * 8 + 16 + 1024;
+  static_assert(kACol0 + kT1AB * 64 <= 512, "tensor memory");
+  static_assert(kBBytes % 1024 == 0, "B stages stay 1024-byte aligned");
+};
+
+template <int RP>
+__global__ void __launch_bounds__(kTcThreads, 1)
+tc_pass1_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict__ cta_begin, const uint8_t* __restrict__ maps) {
+  pdl_wait();
+  using S = Pass1Cfg<RP>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* bring = base + S::kBOff;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(base + S::kBarOff);
+  uint64_t* ge_full = bars;                      // [kT1Stages] G (32 cp.async arrivals) and E (TMA) landed
+  uint64_t* m_ready = ge_full + kT1Stages;       // [kT1Stages] consumers have put m into the E piece
+  uint64_t* ge_empty = m_ready + kT1Stages;      // [kT1Stages] the store of m has read the piece: refill
+  uint64_t* ab_full = ge_empty + kT1Stages;      // [kT1AB] A written to TMEM (4 warps) and B landed
+  uint64_t* ab_empty = ab_full + kT1AB;          // [kT1AB] the MMAs that read buffer i have completed
+  uint64_t* d_full = ab_empty + kT1AB;           // [2]
+  uint64_t* d_empty = d_full + 2;                // [2]
+  uint64_t* fin = d_empty + 2;                   // [1]
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(fin + 1);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(fin + 1) + 1;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int t_begin = cta_begin[blockIdx.x], t_end = cta_begin[blockIdx.x + 1];
+  if (tid == 0) {
+    for (int s = 0; s < kT1Stages; ++s) { mbar_init(ge_full + s, 33); mbar_init(m_ready + s, 4); mbar_init(ge_empty + s, 1); }
+    for (int s = 0; s < kT1AB; ++s) { mbar_init(ab_full + s, 5); mbar_init(ab_empty + s, 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(d_full + s, 1); mbar_init(d_empty + s, 4); }
+    mbar_init(fin, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_async_smem();
+  }
+  if (warp == 2) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)S::kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  auto g_piece = [&](int s) { return base + (size_t)s * 2 * kT1PieceBytes; };
+  auto e_piece = [&](int s) { return base + (size_t)s * 2 * kT1PieceBytes + kT1PieceBytes; };
+
+  if (warp == 0) {
+    // ---- loader: E by TMA (lane 0), G by cp.async (all lanes)
+    uint32_t kc = 0;
+    bool ok = true;
+    for (int ti = t_begin; ti < t_end && ok; ++ti) {
+      const Tile tl = tiles[ti];
+      const LayerDev& L = t.layers[tl.layer];
+      const uint8_t* map = maps + ((size_t)tl.layer * kTcMapsPerLayer + 2) * kTcMapBytes;
+      const float* G = t.grads[(size_t)tl.layer * t.W + tl.worker];
+      const int n = L.n, m = L.m;
+      const int nk = (tl.ncols + kTcK - 1) / kTcK;
+      for (int k = 0; k < nk; ++k, ++kc) {
+        const int s = kc % kT1Stages;
+        if (!warp_wait(ge_empty + s, ((kc / kT1Stages) & 1) ^ 1, abort_flag, lane)) { ok = false; break; }
+        const int c0 = tl.col0 + k * kTcK;
+        if (lane == 0) {
+          mbar_arrive_expect_tx(ge_full + s, kT1PieceBytes);
+          tma_load_3d(e_piece(s), map, c0, tl.row0, tl.worker, ge_full + s);
+        }
+        // lane = (row within a group of 4, 16-byte granule): per iteration 4 rows further down
+        const int r0 = lane >> 3, c16 = lane & 7, gc = c0 + c16 * 4;
+        const int rows_in = (gc < m) ? n - (tl.row0 + r0) : 0;          // row 4 it + r0 is inside iff 4 it < rows_in
+        const float* src = G + (size_t)(tl.row0 + r0) * m + gc;
+        const uint32_t dst = smem_u32(g_piece(s)) + r0 * 128;
+        const uint32_t sw_even = (uint32_t)(c16 ^ r0) << 4, sw_odd = (uint32_t)(c16 ^ (r0 + 4)) << 4;
+#pragma unroll
+        for (int it = 0; it < 32; ++it) {
+          const bool in = 4 * it < rows_in;
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;"
+                       ::"r"(dst + it * 512 + ((it & 1) ? sw_odd : sw_even)), "l"(in ? src : G), "r"(in ? 16u : 0u) : "memory");
+          src += 4 * (size_t)m;
+        }
+        cp_async_arrive(ge_full + s);
+      }
+    }
+    if (!ok && lane == 0)
+      for (uint32_t it = kc > (uint32_t)kT1Stages ? kc - kT1Stages : 0; it < kc; ++it)
+        drain(ge_full + it % kT1Stages, (it / kT1Stages) & 1);
+    asm volatile("cp.async.wait_all;" ::: "memory");
+  } else if (warp == 1) {
+    // ---- B loader: columns [c0, c0 + 32) of Q^T and of its remainders
+    uint32_t kc = 0;
+    bool ok = true;
+    for (int ti = t_begin; ti < t_end && ok; ++ti) {
+      const Tile tl = tiles[ti];
+      const uint8_t* map = maps + ((size_t)tl.layer * kTcMapsPerLayer + 3) * kTcMapBytes;
+      const int nk = (tl.ncols + kTcK - 1) / kTcK;
+      for (int k = 0; k < nk; ++k, ++kc) {
+        const int s = kc % kT1AB;
+        if (!warp_wait(ab_empty + s, ((kc / kT1AB) & 1) ^ 1, abort_flag, lane)) { ok = false; break; }
+        if (lane == 0) {
+          mbar_arrive_expect_tx(ab_full + s, S::kBBytes);
+          tma_load_2d(bring + (size_t)s * S::kBBytes, map, tl.col0 + k * kTcK, 0, ab_full + s);
+        }
+      }
+    }
+    if (!ok && lane == 0)
+      for (uint32_t it = kc > (uint32_t)kT1AB ? kc - kT1AB : 0; it < kc; ++it) drain(ab_full + it % kT1AB, (it / kT1AB) & 1);
+  } else if (warp == 2) {
+    // ---- MMA issue: one thread
+    if (lane == 0) {
+      uint32_t kc = 0, tseq = 0;
+      bool ok = true;
+      const uint32_t idesc2 = tc_idesc_tf32(2 * RP), idesc1 = tc_idesc_tf32(RP);
+      const uint64_t bdesc0 = tc_desc_sw128(smem_u32(bring));
+      for (int ti = t_begin; ti < t_end && ok; ++ti, ++tseq) {
+        const int nk = (tiles[ti].ncols + kTcK - 1) / kTcK;
+        const uint32_t db = tseq & 1;
+        const uint32_t dcol = tmem + db * S::kDStride;
+        if (!thread_wait(d_empty + db, ((tseq >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+        for (int k = 0; k < nk; ++k, ++kc) {
+          const int s = kc % kT1AB;
+          if (!thread_wait(ab_full + s, (kc / kT1AB) & 1, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t bd0 = bdesc0 + (uint64_t)((s * S::kBBytes) >> 4);
+          const uint32_t acol = tmem + S::kACol0 + s * 64;
+#pragma unroll
+          for (int ks = 0; ks < kTcK / 8; ++ks) {
+            tc_mma_tf32_ts(dcol, acol + ks * 8, bd0 + (uint64_t)((ks * 32) >> 4), idesc2, (k > 0 || ks > 0) ? 1u : 0u);
+            tc_mma_tf32_ts(dcol, acol + 32 + ks * 8, bd0 + (uint64_t)((ks * 32) >> 4), idesc1, 1u);
+          }
+          tc_commit(ab_empty + s);
+          if (k == nk - 1) tc_commit(d_full + db);
+        }
+      }
+      tc_commit(fin);
+      drain(fin, 0);
+    }
+    __syncwarp();
+  } else if (warp == 3) {
+    // ---- storer: m pieces back to global memory (over E)
+    uint32_t kc = 0;
+    bool ok = true;
+    for (int ti = t_begin; ti < t_end && ok; ++ti) {
+      const Tile tl = tiles[ti];
+      const uint8_t* map = maps + ((size_t)tl.layer * kTcMapsPerLayer + 2) * kTcMapBytes;
+      const int nk = (tl.ncols + kTcK - 1) / kTcK;
+      for (int k = 0; k < nk; ++k, ++kc) {
+        const int s = kc % kT1Stages;
+        if (!warp_wait(m_ready + s, (kc / kT1Stages) & 1, abort_flag, lane)) { ok = false; break; }
+        if (lane == 0) {
+          tma_store_3d(map, tl.col0 + k * kTcK, tl.row0, tl.worker, e_piece(s));
+          bulk_commit();
+          // one store stays in flight: the stage of the store before this one is free once that one has been read
+          if (kc > 0) {
+            asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+            mbar_arrive(ge_empty + (kc - 1) % kT1Stages);
+          }
+        }
+        __syncwarp();
+      }
+    }
+    if (lane == 0) {
+      bulk_wait_read0();
+      if (ok && kc > 0) mbar_arrive(ge_empty + (kc - 1) % kT1Stages);
+      bulk_wait_all0();
+    }
+  } else if (warp < 8) {
+    // ---- epilogue: P_part[row][j] = D[row][j] + D[row][RP + j]
+    uint32_t tseq = 0;
+    const int q = warp & 3;
+    for (int ti = t_begin; ti < t_end; ++ti, ++tseq) {
+      const Tile tl = tiles[ti];
+      const LayerDev& L = t.layers[tl.layer];
+      const uint32_t db = tseq & 1;
+      if (!warp_wait(d_full + db, (tseq >> 1) & 1, abort_flag, lane)) break;
+      tc_fence_after();
+      const uint32_t taddr = tmem + ((uint32_t)(32 * q) << 16) + db * S::kDStride;
+      const int row = tl.row0 + 32 * q + lane;
+      float* dst = L.Ppart + (((size_t)tl.worker * L.ncc + tl.part) * L.n + (size_t)min(row, L.n - 1)) * RP;
+#pragma unroll
+      for (int j0 = 0; j0 < RP; j0 += 16) {
+        uint32_t a[16], b[16];
+        tc_ld16(taddr + j0, a);
+        tc_ld16(taddr + RP + j0, b);
+        tc_wait_ld();
+        if (row < L.n) {
+#pragma unroll
+          for (int j = 0; j < 16; j += 4)
+            *reinterpret_cast<float4*>(dst + j0 + j) =
+                make_float4(__uint_as_float(a[j]) + __uint_as_float(b[j]), __uint_as_float(a[j + 1]) + __uint_as_float(b[j + 1]),
+                            __uint_as_float(a[j + 2]) + __uint_as_float(b[j + 2]), __uint_as_float(a[j + 3]) + __uint_as_float(b[j + 3]));
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(d_empty + db);
+    }
+  } else {
+    // ---- consumers: lane = row; m = g + e -> E piece (for the store) and hi / lo -> tensor memory
+    const int g = (warp - 8) >> 2, q = warp & 3;
+    uint32_t kc = 0;
+    bool ok = true;
+    const uint32_t lane_base = tmem + ((uint32_t)(32 * q) << 16) + S::kACol0;
+    const int row = 32 * q + lane;
+    for (int ti = t_begin; ti < t_end && ok; ++ti) {
+      const int nk = (tiles[ti].ncols + kTcK - 1) / kTcK;
+      for (int k = 0; k < nk; ++k, ++kc) {
+        if ((int)(kc % kTcGroups) != g) continue;
+        const int s = kc % kT1Stages, ab = kc % kT1AB;
+        if (!warp_wait(ge_full + s, (kc / kT1Stages) & 1, abort_flag, lane)) { ok = false; break; }
+        const uint8_t* gp = g_piece(s) + row * 128;
+        uint8_t* ep = e_piece(s) + row * 128;
+        uint32_t v[32];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          const int off = (c ^ (row & 7)) << 4;
+          const float4 g4 = *reinterpret_cast<const float4*>(gp + off);
+          float4 e4 = *reinterpret_cast<const float4*>(ep + off);
+          e4.x += g4.x; e4.y += g4.y; e4.z += g4.z; e4.w += g4.w;
+          *reinterpret_cast<float4*>(ep + off) = e4;
+          v[4 * c] = __float_as_uint(e4.x); v[4 * c + 1] = __float_as_uint(e4.y);
+          v[4 * c + 2] = __float_as_uint(e4.z); v[4 * c + 3] = __float_as_uint(e4.w);
+        }
+        fence_async_smem();                       // the TMA store reads what was just written
+        __syncwarp();
+        if (lane == 0) mbar_arrive(m_ready + s);
+        if (!warp_wait(ab_empty + ab, ((kc / kT1AB) & 1) ^ 1, abort_flag, lane)) { ok = false; break; }
+        tc_fence_after();
+        tc_st32(lane_base + ab * 64, v);
+#pragma unroll
+        for (int kk = 0; kk < 32; ++kk) {
+          const float x = __uint_as_float(v[kk]);
+          v[kk] = __float_as_uint(x - __uint_as_float(v[kk] & 0xffffe000u));
+        }
+        tc_st32(lane_base + ab * 64 + 32, v);
+        tc_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(ab_full + ab);
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (tid == 0 && *abort_flag && t_end > t_begin) report_timeout(t, tiles[t_begin].layer);
+  if (warp == 2)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)S::kTmemCols) : "memory");
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -373,8 +683,37 @@ int tc_encode_maps(const LayerDev* layers, int n_layers, int W, int RP, void* ou
                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return LQSGD_ERR_CUDA;
     }
+    {   // E / M as [W][n][m]: pieces of 128 rows x 32 columns, 128-byte swizzle (pass 1: load E, store M)
+      const cuuint64_t dim[3] = {(cuuint64_t)L.m, (cuuint64_t)L.n, (cuuint64_t)W};
+      const cuuint64_t stride[2] = {(cuuint64_t)L.m * 4, (cuuint64_t)L.n * L.m * 4};
+      const cuuint32_t box[3] = {kTcK, 128, 1}, es[3] = {1, 1, 1};
+      if (encode(&maps[i * kTcMapsPerLayer + 2], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, L.E, dim, stride, box, es,
+                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return LQSGD_ERR_CUDA;
+    }
+    {   // Q^T and its tf32 remainders, [2 RP][mt]: 32 columns of Q for all 2 RP operand rows (pass 1)
+      const cuuint64_t dim[2] = {(cuuint64_t)L.mt, (cuuint64_t)(2 * RP)};
+      const cuuint64_t stride[1] = {(cuuint64_t)L.mt * 4};
+      const cuuint32_t box[2] = {kTcK, (cuuint32_t)(2 * RP)}, es[2] = {1, 1};
+      if (encode(&maps[i * kTcMapsPerLayer + 3], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, L.Qt, dim, stride, box, es,
+                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return LQSGD_ERR_CUDA;
+    }
   }
   return LQSGD_OK;
+}
+
+cudaError_t launch_tc_pass1(int RP, const Tables& t, const Tile* tiles, int ntiles, const int* cta_begin, const void* maps,
+                            Launch l) {
+  if (ntiles == 0) return cudaSuccess;
+  if (RP != 16) return cudaErrorInvalidValue;
+  using S = Pass1Cfg<16>;
+  cudaError_t e = cudaFuncSetAttribute(tc_pass1_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)S::kTotal);
+  if (e != cudaSuccess) return e;
+  return launch_pdl(tc_pass1_kernel<16>, dim3(l.grid), dim3(kTcThreads), S::kTotal, l.stream, t, tiles, cta_begin,
+                    static_cast<const uint8_t*>(maps));
 }
 
 cudaError_t launch_tc_pass2(int RP, const Tables& t, const Tile* tiles, int ntiles, const void* maps, Launch l) {
