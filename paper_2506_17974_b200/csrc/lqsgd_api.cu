@@ -57,6 +57,8 @@ struct Plan {
   std::vector<Tile> tctiles2;                    // tensor-core pass 2
   std::vector<Tile> tctiles1;                    // tensor-core pass 1, grouped by CTA
   std::vector<int> tcbegin1;                     // [tc_grid + 1]
+  std::vector<Tile> tctiles3;                    // tensor-core pass 3 (all workers per tile), grouped by CTA
+  std::vector<int> tcbegin3;
   int tc_grid = 0;
   std::vector<uint8_t> tcmaps;                   // tensor maps of the tensor-core passes (filled at create)
   std::vector<FactorBlock> fbP, fbQ;
@@ -74,6 +76,8 @@ struct Plan {
   Tile* d_tctiles2 = nullptr;
   Tile* d_tctiles1 = nullptr;
   int* d_tcbegin1 = nullptr;
+  Tile* d_tctiles3 = nullptr;
+  int* d_tcbegin3 = nullptr;
   uint8_t* d_tcmaps = nullptr;
   FactorBlock *d_fbP = nullptr, *d_fbQ = nullptr;
   ExchangeChunk *d_chP = nullptr, *d_chQ = nullptr, *d_chV = nullptr;
@@ -301,6 +305,9 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
     L.nt = (int)align_up((size_t)mt.n, 4);
     L.Qt = a.take<float>((size_t)(tc ? 2 : 1) * RP * L.mt);
     L.Pbt = tc ? a.take<float>((size_t)3 * RP * L.nt) : nullptr;
+    L.kcat = (int)align_up((size_t)3 * RP, 32);
+    L.Pcat = tc ? a.take<float>((size_t)mt.n * L.kcat) : nullptr;
+    L.Qcat = tc ? a.take<float>((size_t)mt.m * L.kcat) : nullptr;
     L.Ppart = a.take<float>((size_t)W * L.ncc * mt.n * RP);
     L.Praw = (L.ncc == 1) ? L.Ppart : a.take<float>((size_t)W * mt.n * RP);
     L.P = a.take<float>((size_t)W * mt.n * RP);
@@ -339,6 +346,10 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
         u0 += nu;
       }
     }
+    for (int rb = 0; tc && rb < ceil_div(mt.n, kTcRowsPerTile); ++rb)
+      for (int cb = 0; cb < ceil_div(mt.m, 128); ++cb)
+        p.tctiles3.push_back({li32, 0, rb * kTcRowsPerTile, std::min(kTcRowsPerTile, mt.n - rb * kTcRowsPerTile), cb * 128,
+                              std::min(128, mt.m - cb * 128), 0, 0});
     for (int rb = 0; !st && !tc && rb < ceil_div(mt.n, kPass1Rows); ++rb)
       for (int cc = 0; cc < L.ncc; ++cc)
         for (int w = 0; w < W; ++w) {
@@ -360,7 +371,7 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
           p.tctiles2.push_back({li32, w, row0, std::min(tr2, mt.n - row0), col0, std::min(128, mt.m - col0), rb, 0});
         }
     const int tr3 = balanced_rows(mt.n, r3);
-    for (int rb = 0; !st && rb < ceil_div(mt.n, tr3); ++rb)
+    for (int rb = 0; !st && !tc && rb < ceil_div(mt.n, tr3); ++rb)
       for (int cc = 0; cc < ceil_div(mt.m, cw2); ++cc) {
         const int row0 = rb * tr3, col0 = cc * cw2;
         p.tiles3.push_back({li32, 0, row0, std::min(tr3, mt.n - row0), col0, std::min(cw2, mt.m - col0), 0, 0});
@@ -383,8 +394,8 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   // Pass 1: longest tile first to the CTA with the least work so far (a tile costs its column count:
   // every stage is 128 rows deep whatever the tile's row count), then grouped by CTA.
   p.tc_grid = sm_count;
-  {
-    std::vector<Tile> sorted = p.tctiles1;
+  auto deal = [&](std::vector<Tile>& tiles, std::vector<int>& begin) {
+    std::vector<Tile> sorted = tiles;
     std::stable_sort(sorted.begin(), sorted.end(), [](const Tile& x, const Tile& y) { return x.ncols > y.ncols; });
     std::vector<std::vector<Tile>> per(p.tc_grid);
     std::vector<long> load(p.tc_grid, 0);
@@ -393,13 +404,15 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
       per[b].push_back(tl);
       load[b] += ceil_div(tl.ncols, 32);
     }
-    p.tctiles1.clear();
-    p.tcbegin1.assign(p.tc_grid + 1, 0);
+    tiles.clear();
+    begin.assign(p.tc_grid + 1, 0);
     for (int b = 0; b < p.tc_grid; ++b) {
-      p.tctiles1.insert(p.tctiles1.end(), per[b].begin(), per[b].end());
-      p.tcbegin1[b + 1] = (int)p.tctiles1.size();
+      tiles.insert(tiles.end(), per[b].begin(), per[b].end());
+      begin[b + 1] = (int)tiles.size();
     }
-  }
+  };
+  deal(p.tctiles1, p.tcbegin1);
+  deal(p.tctiles3, p.tcbegin3);     // same cost model: pieces of 32 columns (times W for every tile alike)
   p.d_status = a.take<uint32_t>(p.mats.size());
   p.d_payload = a.take<uint8_t>((size_t)W * p.payload_stride);
   p.d_xscales = a.take<float>(2 * p.mats.size());
@@ -419,6 +432,8 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   p.d_tctiles2 = a.take<Tile>(p.tctiles2.size());
   p.d_tctiles1 = a.take<Tile>(p.tctiles1.size());
   p.d_tcbegin1 = a.take<int>(p.tcbegin1.size());
+  p.d_tctiles3 = a.take<Tile>(p.tctiles3.size());
+  p.d_tcbegin3 = a.take<int>(p.tcbegin3.size());
   p.d_tcmaps = a.take<uint8_t>(p.mats.size() * kTcMapsPerLayer * kTcMapBytes);
   p.d_fbP = a.take<FactorBlock>(p.fbP.size());
   p.d_fbQ = a.take<FactorBlock>(p.fbQ.size());
@@ -553,6 +568,8 @@ int lqsgd_create(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
   CK(up(p.d_tctiles2, p.tctiles2.data(), p.tctiles2.size() * sizeof(Tile)));
   CK(up(p.d_tctiles1, p.tctiles1.data(), p.tctiles1.size() * sizeof(Tile)));
   CK(up(p.d_tcbegin1, p.tcbegin1.data(), p.tcbegin1.size() * sizeof(int)));
+  CK(up(p.d_tctiles3, p.tctiles3.data(), p.tctiles3.size() * sizeof(Tile)));
+  CK(up(p.d_tcbegin3, p.tcbegin3.data(), p.tcbegin3.size() * sizeof(int)));
   p.tcmaps.resize(p.mats.size() * kTcMapsPerLayer * kTcMapBytes + 1);
   rc = tc_encode_maps(p.layers.data(), (int)p.layers.size(), p.W, p.RP, p.tcmaps.data());
   if (rc != LQSGD_OK) { g_cuda_error = "cuTensorMapEncodeTiled failed or is not available"; return rc; }
@@ -575,7 +592,8 @@ int lqsgd_create(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
       for (int j = 0; j < mt.r; ++j)
         q0[(size_t)i * p.RP + j] = normal_draw(cfg->seed, (uint64_t)mt.user_index, (uint64_t)i * mt.r + j);
     CK(up(p.layers[li].Q, q0.data(), q0.size() * sizeof(float)));
-    CK(launch_q_transpose(p.layers[li].Q, p.layers[li].Qt, mt.m, p.RP, p.layers[li].mt, p.layers[li].tc, nullptr));
+    CK(launch_q_transpose(p.layers[li].Q, p.layers[li].Qt, p.layers[li].Qcat, mt.m, p.RP, p.layers[li].mt, p.layers[li].kcat,
+                          p.layers[li].tc, nullptr));
   }
   int o1 = 1, o2 = 1, o3 = 1;
   CK(pass_occupancy(p.RP, &o1, &o2, &o3));
@@ -608,7 +626,7 @@ int lqsgd_launches_per_step(const lqsgd_ctx* ctx, int32_t* out) {
   const Plan& p = ctx->plan;
   // Orthonormalize (2), exchange of P, Q_w reduction, exchange of Q; then one launch per non-empty tile list
   *out = (p.mats.empty() ? 0 : 5) + (p.tiles1.empty() ? 0 : 2) + (p.stiles1.empty() ? 0 : 2) + (p.tiles2.empty() ? 0 : 1) +
-         (p.tctiles2.empty() ? 0 : 1) + (p.tctiles1.empty() ? 0 : 1) + (p.chV.empty() ? 0 : 1);
+         (p.tctiles2.empty() ? 0 : 1) + (p.tctiles1.empty() ? 0 : 1) + (p.tctiles3.empty() ? 0 : 1) + (p.chV.empty() ? 0 : 1);
   return LQSGD_OK;
 }
 
@@ -753,6 +771,7 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
       if (nm) {
         CK(launch_pass3(RP, t, p.d_tiles3, (int)p.tiles3.size(), {st, c->grid3}));
         CK(launch_stream_pass3(RP, t, p.d_stiles3, (int)p.stiles3.size(), {st, (int)std::min<size_t>(p.stiles3.size(), c->sm_count)}));
+        CK(launch_tc_pass3(RP, t, p.d_tctiles3, (int)p.tctiles3.size(), p.d_tcbegin3, p.d_tcmaps, {st, p.tc_grid}));
       }
       PHASE_MARK(5);
       break;
@@ -945,7 +964,7 @@ int lqsgd_set_state(lqsgd_ctx* c, int32_t which, int32_t layer, int32_t worker, 
   if (which == LQSGD_STATE_Q) {
     for (const LayerDev& L : c->plan.layers)
       if (L.user_index == layer)
-        CK(launch_q_transpose(L.Q, L.Qt, L.m, c->plan.RP, L.mt, L.tc, static_cast<cudaStream_t>(cuda_stream)));
+        CK(launch_q_transpose(L.Q, L.Qt, L.Qcat, L.m, c->plan.RP, L.mt, L.kcat, L.tc, static_cast<cudaStream_t>(cuda_stream)));
   }
   return LQSGD_OK;
 }

@@ -24,11 +24,14 @@ struct LayerDev {
   int32_t mt;                 // row stride of Qt: m rounded up to a multiple of 4
   int32_t tc;                 // 1: the tensor-core passes take this layer (padded rank >= 16, m % 4 == 0)
   int32_t nt;                 // row stride of Pbt: n rounded up to a multiple of 4
+  int32_t kcat;               // row stride of Pcat / Qcat: 3 RP rounded up to a multiple of 32
   float* E;                   // [W][n][m]   error buffer; holds M between pass 1 and pass 3
   float* Q;                   // [m][RP]     warm start, becomes Q_bar
   float* Qt;                  // [RP][mt]    transposed copy of Q read by pass 1 and pass 3;
                               // tc layers: [2 RP][mt], rows RP.. hold the tf32 remainders of rows 0..
   float* Pbt;                 // tc layers: [3 RP][nt] words: P_bar transposed, as three stacked bf16 terms (pass 2 operand)
+  float* Pcat;                // tc layers: [n][kcat]  P_bar | P_bar | tf32 remainder of P_bar | 0   (pass 3 operand)
+  float* Qcat;                // tc layers: [m][kcat]  Q_bar | tf32 remainder of Q_bar | Q_bar | 0
   float* Ppart;               // [W][ncc][n][RP]
   float* Praw;                // [W][n][RP]  (== Ppart when ncc == 1)
   float* P;                   // [W][n][RP]  orthonormal
@@ -139,7 +142,8 @@ cudaError_t launch_exchange(int RP, int which /*0 = P, 1 = Q*/, const Tables& t,
 cudaError_t launch_scale_reduce(const Tables& t, int which, float* scales, int n_mat, Launch l);
 cudaError_t launch_sum_dequant(int RP, int which, const Tables& t, const QuantTables& q, const ExchangeChunk* ch,
                                int nch, const SplitExchange& sx, const uint8_t* gathered, int n_streams, Launch l);
-cudaError_t launch_q_transpose(const float* Q, float* Qt, int m, int RP, int mt, int tc, cudaStream_t stream);
+cudaError_t launch_q_transpose(const float* Q, float* Qt, float* Qcat, int m, int RP, int mt, int kcat, int tc,
+                               cudaStream_t stream);
 cudaError_t launch_pass2(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
 cudaError_t launch_q_reduce(int RP, const Tables& t, const FactorBlock* fb, int nfb, Launch l);
 cudaError_t launch_pass3(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
@@ -186,8 +190,9 @@ __host__ __device__ inline StreamGeo stream_geo(int ncols, int RP) {
 // on tcgen05 with every fp32 operand fed as a sum of narrow terms, fp32 accumulation in tensor
 // memory.  `maps` is the layer-major array of tensor maps (kTcMapsPerLayer per layer) that
 // tc_encode_maps() filled.
-constexpr int kTcMapsPerLayer = 4;   // 0: M as [W][n][m], box 128 x 32 x 1;  1: Pbt, box 32 x 3RP, 128-byte swizzle;
+constexpr int kTcMapsPerLayer = 6;   // 0: M as [W][n][m], box 128 x 32 x 1;  1: Pbt, box 32 x 3RP, 128-byte swizzle;
                                      // 2: E / M as [W][n][m], box 32 x 128 x 1, swizzled;  3: Qt, box 32 x 2RP, swizzled
+                                     // 4: Pcat, 5: Qcat, box 32 x 128, swizzled
 constexpr int kTcRowsPerTile = 128;  // rows of a pass-1 tile: the M extent of one MMA
 constexpr int kTcPass1Cols = 576;    // most columns of a pass-1 tile (multiple of 32): small enough to balance the SMs
 constexpr int kTcMapBytes = 128;
@@ -196,6 +201,8 @@ int tc_encode_maps(const LayerDev* host_layers, int n_layers, int W, int RP, voi
 cudaError_t launch_tc_pass2(int RP, const Tables& t, const Tile* tiles, int ntiles, const void* maps, Launch l);
 // tiles are grouped by CTA: CTA b takes tiles [cta_begin[b], cta_begin[b + 1]); l.grid CTAs
 cudaError_t launch_tc_pass1(int RP, const Tables& t, const Tile* tiles, int ntiles, const int* cta_begin, const void* maps,
+                            Launch l);
+cudaError_t launch_tc_pass3(int RP, const Tables& t, const Tile* tiles, int ntiles, const int* cta_begin, const void* maps,
                             Launch l);
 cudaError_t launch_stream_pass1(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
 cudaError_t launch_stream_pass3(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);

@@ -643,10 +643,17 @@ __device__ __forceinline__ void store_factor(const LayerDev& L, int which, int r
   if (which) {
     L.Q[(size_t)row * RP + col] = v;
     L.Qt[(size_t)col * L.mt + row] = v;
-    if (L.tc) L.Qt[(size_t)(RP + col) * L.mt + row] = tf32_remainder(v);
+    if (L.tc) {
+      const float lo = tf32_remainder(v);
+      L.Qt[(size_t)(RP + col) * L.mt + row] = lo;
+      float* qc = L.Qcat + (size_t)row * L.kcat + col;
+      qc[0] = v; qc[RP] = lo; qc[2 * RP] = v;
+    }
   } else {
     L.Pbar[(size_t)row * RP + col] = v;
     if (L.tc) {
+      float* pc = L.Pcat + (size_t)row * L.kcat + col;
+      pc[0] = v; pc[RP] = v; pc[2 * RP] = tf32_remainder(v);
       // three bf16 terms v = b1 + b2 + b3 (24 bits), each stored twice in one word: the two K slots
       // that face the bf16 pair of an element of M in the tensor-core pass 2
       float rest = v;
@@ -810,14 +817,20 @@ exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __rest
 
 // Qt[j][i] = Q[i][j]: refreshes the transposed copy after Q was set from outside.
 __global__ void __launch_bounds__(256)
-q_transpose_kernel(const float* __restrict__ Q, float* __restrict__ Qt, int m, int RP, int mt, int tc) {
+q_transpose_kernel(const float* __restrict__ Q, float* __restrict__ Qt, float* __restrict__ Qcat, int m, int RP, int mt,
+                   int kcat, int tc) {
   pdl_wait();
   const int i = blockIdx.x * 256 + threadIdx.x;
   if (i >= m) return;
   for (int j = 0; j < RP; ++j) {
     const float v = Q[(size_t)i * RP + j];
     Qt[(size_t)j * mt + i] = v;
-    if (tc) Qt[(size_t)(RP + j) * mt + i] = tf32_remainder(v);
+    if (tc) {
+      const float lo = tf32_remainder(v);
+      Qt[(size_t)(RP + j) * mt + i] = lo;
+      float* qc = Qcat + (size_t)i * kcat + j;
+      qc[0] = v; qc[RP] = lo; qc[2 * RP] = v;
+    }
   }
 }
 
@@ -942,8 +955,9 @@ cudaError_t launch_pass1(int rp, const Tables& t, const Tile* tiles, int ntiles,
   return cudaGetLastError();
 }
 
-cudaError_t launch_q_transpose(const float* Q, float* Qt, int m, int RP, int mt, int tc, cudaStream_t stream) {
-  launch_pdl(q_transpose_kernel, (m + 255) / 256, 256, 0, stream, Q, Qt, m, RP, mt, tc);
+cudaError_t launch_q_transpose(const float* Q, float* Qt, float* Qcat, int m, int RP, int mt, int kcat, int tc,
+                               cudaStream_t stream) {
+  launch_pdl(q_transpose_kernel, (m + 255) / 256, 256, 0, stream, Q, Qt, Qcat, m, RP, mt, kcat, tc);
   return cudaGetLastError();
 }
 

@@ -641,6 +641,250 @@ tc_pass1_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)S::kTmemCols) : "memory");
 }
 
+// ---------------------------------------------------------------------------------------
+// Pass 3 on the tensor core (G_hat = P_bar Q_bar^T, E_w = M_w - G_hat, Alg. 1; optional model
+// update).  A tile is 128 rows x 128 columns of one layer, for all workers.  Once per tile the
+// accumulator D = G_hat tile is formed from the factors: both operands come from shared memory,
+// K-major, as rows of kCat = 3 RP (padded to a multiple of 32) tf32 values
+//   P side: [P_bar | P_bar | P_bar_lo | 0]      Q side: [Q_bar | Q_bar_lo | Q_bar | 0]
+// (lo = the remainder after the truncation to tf32 the hardware applies), so that one K loop
+// yields hi*hi + hi*lo + lo*hi.  Then, for every worker, the 128 x 128 piece of M streams through
+// a ring in four 128 x 32 pieces (TMA, 128-byte swizzle); a consumer thread (lane = row) reads its
+// row of G_hat from tensor memory, subtracts, puts E back into the piece (a storer thread sends
+// it to global memory with a TMA tensor store); the warpgroup that meets worker 0 also writes
+// G_hat and applies the model update.
+// ---------------------------------------------------------------------------------------
+constexpr int kT3Stages = 8;          // ring of M pieces, 16 KB each
+constexpr int kT3Groups = 4;          // consumer warpgroups (warps 4..19)
+
+__device__ __forceinline__ void tc_mma_tf32_ss(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}"
+               ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+template <int RP>
+struct Pass3Cfg {
+  static constexpr int kCat = (3 * RP + 31) / 32 * 32;                   // K extent of the factor product
+  static constexpr int kSub = kCat / 32;                                 // 128-byte sub-tiles per operand
+  static constexpr uint32_t kOpBytes = kSub * kT1PieceBytes;             // one operand: kSub pieces of 128 rows x 32
+  static constexpr uint32_t kOpOff = kT3Stages * kT1PieceBytes;
+  static constexpr uint32_t kBarOff = kOpOff + 2 * kOpBytes;
+  static constexpr int kBars = 3 * kT3Stages + 2 + 2 + 2 + 1;
+  static constexpr uint32_t kTotal = kBarOff + kBars * 8 + 16 + 1024;
+  static constexpr int kTmemCols = 256;                                  // two accumulators of 128 columns
+};
+
+template <int RP>
+__global__ void __launch_bounds__(kTcThreads, 1)
+tc_pass3_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict__ cta_begin, const uint8_t* __restrict__ maps) {
+  pdl_wait();
+  using S = Pass3Cfg<RP>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* opa = base + S::kOpOff;               // P side
+  uint8_t* opb = opa + S::kOpBytes;              // Q side
+  uint64_t* bars = reinterpret_cast<uint64_t*>(base + S::kBarOff);
+  uint64_t* m_full = bars;                       // [kT3Stages] piece of M landed
+  uint64_t* e_ready = m_full + kT3Stages;        // [kT3Stages] consumers have put E into the piece
+  uint64_t* m_empty = e_ready + kT3Stages;       // [kT3Stages] the store of E has read the piece
+  uint64_t* op_full = m_empty + kT3Stages;       // [1] operands of the tile landed   (+1 spare)
+  uint64_t* op_empty = op_full + 2;              // [1] the tile's MMAs have completed (+1 spare)
+  uint64_t* d_full = op_empty + 2;               // [2]
+  uint64_t* d_empty = d_full + 2;                // [2] all 16 consumer warps are past the tile
+  uint64_t* fin = d_empty + 2;
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(fin + 1);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(fin + 1) + 1;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int t_begin = cta_begin[blockIdx.x], t_end = cta_begin[blockIdx.x + 1];
+  const int W = t.W;
+  if (tid == 0) {
+    for (int s = 0; s < kT3Stages; ++s) { mbar_init(m_full + s, 1); mbar_init(e_ready + s, 4); mbar_init(m_empty + s, 1); }
+    mbar_init(op_full, 1); mbar_init(op_empty, 1);
+    for (int s = 0; s < 2; ++s) { mbar_init(d_full + s, 1); mbar_init(d_empty + s, 4 * kT3Groups); }
+    mbar_init(fin, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_async_smem();
+  }
+  if (warp == 2) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)S::kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  auto piece = [&](int s) { return base + (size_t)s * kT1PieceBytes; };
+  auto pieces_of = [](const Tile& tl) { return (tl.ncols + kTcK - 1) / kTcK; };
+
+  if (warp == 0) {
+    // ---- M loader
+    uint32_t kc = 0;
+    bool ok = true;
+    for (int ti = t_begin; ti < t_end && ok; ++ti) {
+      const Tile tl = tiles[ti];
+      const uint8_t* map = maps + ((size_t)tl.layer * kTcMapsPerLayer + 2) * kTcMapBytes;
+      const int np = pieces_of(tl);
+      for (int w = 0; w < W && ok; ++w)
+        for (int pc = 0; pc < np; ++pc, ++kc) {
+          const int s = kc % kT3Stages;
+          if (!warp_wait(m_empty + s, ((kc / kT3Stages) & 1) ^ 1, abort_flag, lane)) { ok = false; break; }
+          if (lane == 0) {
+            mbar_arrive_expect_tx(m_full + s, kT1PieceBytes);
+            tma_load_3d(piece(s), map, tl.col0 + pc * kTcK, tl.row0, w, m_full + s);
+          }
+        }
+    }
+    if (!ok && lane == 0)
+      for (uint32_t it = kc > (uint32_t)kT3Stages ? kc - kT3Stages : 0; it < kc; ++it)
+        drain(m_full + it % kT3Stages, (it / kT3Stages) & 1);
+  } else if (warp == 1) {
+    // ---- operand loader: the tile's rows of the stacked P_bar terms and its columns' rows of the Q_bar terms
+    uint32_t tseq = 0;
+    bool ok = true;
+    for (int ti = t_begin; ti < t_end && ok; ++ti, ++tseq) {
+      const Tile tl = tiles[ti];
+      const uint8_t* mapp = maps + ((size_t)tl.layer * kTcMapsPerLayer + 4) * kTcMapBytes;
+      const uint8_t* mapq = maps + ((size_t)tl.layer * kTcMapsPerLayer + 5) * kTcMapBytes;
+      if (!warp_wait(op_empty, (tseq & 1) ^ 1, abort_flag, lane)) { ok = false; break; }
+      if (lane == 0) {
+        mbar_arrive_expect_tx(op_full, 2 * S::kOpBytes);
+#pragma unroll
+        for (int kt = 0; kt < S::kSub; ++kt) {
+          tma_load_2d(opa + (size_t)kt * kT1PieceBytes, mapp, kt * 32, tl.row0, op_full);
+          tma_load_2d(opb + (size_t)kt * kT1PieceBytes, mapq, kt * 32, tl.col0, op_full);
+        }
+      }
+    }
+    if (!ok && lane == 0 && tseq > 0) drain(op_full, (tseq - 1) & 1);
+  } else if (warp == 2) {
+    // ---- MMA issue: one thread, once per tile
+    if (lane == 0) {
+      uint32_t tseq = 0;
+      bool ok = true;
+      const uint32_t idesc = tc_idesc_tf32(128);
+      const uint64_t adesc0 = tc_desc_sw128(smem_u32(opa)), bdesc0 = tc_desc_sw128(smem_u32(opb));
+      for (int ti = t_begin; ti < t_end && ok; ++ti, ++tseq) {
+        const uint32_t db = tseq & 1;
+        if (!thread_wait(d_empty + db, ((tseq >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+        if (!thread_wait(op_full, tseq & 1, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+#pragma unroll
+        for (int kt = 0; kt < S::kSub; ++kt)
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks) {
+            const uint64_t off = (uint64_t)((kt * kT1PieceBytes + ks * 32) >> 4);
+            tc_mma_tf32_ss(tmem + db * 128, adesc0 + off, bdesc0 + off, idesc, (kt > 0 || ks > 0) ? 1u : 0u);
+          }
+        tc_commit(op_empty);
+        tc_commit(d_full + db);
+      }
+      tc_commit(fin);
+      drain(fin, 0);
+    }
+    __syncwarp();
+  } else if (warp == 3) {
+    // ---- storer: E pieces back to global memory
+    uint32_t kc = 0;
+    bool ok = true;
+    for (int ti = t_begin; ti < t_end && ok; ++ti) {
+      const Tile tl = tiles[ti];
+      const uint8_t* map = maps + ((size_t)tl.layer * kTcMapsPerLayer + 2) * kTcMapBytes;
+      const int np = pieces_of(tl);
+      for (int w = 0; w < W && ok; ++w)
+        for (int pc = 0; pc < np; ++pc, ++kc) {
+          const int s = kc % kT3Stages;
+          if (!warp_wait(e_ready + s, (kc / kT3Stages) & 1, abort_flag, lane)) { ok = false; break; }
+          if (lane == 0) {
+            tma_store_3d(map, tl.col0 + pc * kTcK, tl.row0, w, piece(s));
+            bulk_commit();
+            if (kc > 0) {
+              asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+              mbar_arrive(m_empty + (kc - 1) % kT3Stages);
+            }
+          }
+          __syncwarp();
+        }
+    }
+    if (lane == 0) {
+      bulk_wait_read0();
+      if (ok && kc > 0) mbar_arrive(m_empty + (kc - 1) % kT3Stages);
+      bulk_wait_all0();
+    }
+  } else {
+    // ---- consumers (warps 4..19): lane = row
+    const int g = (warp - 4) >> 2, q = warp & 3;
+    uint32_t kc = 0, tseq = 0;
+    bool ok = true;
+    const int row_in_tile = 32 * q + lane;
+    for (int ti = t_begin; ti < t_end && ok; ++ti, ++tseq) {
+      const Tile tl = tiles[ti];
+      const LayerDev& L = t.layers[tl.layer];
+      const int np = pieces_of(tl);
+      const uint32_t db = tseq & 1;
+      const uint32_t taddr = tmem + ((uint32_t)(32 * q) << 16) + db * 128;
+      const int row = tl.row0 + row_in_tile;
+      float* Gh = t.ghat[tl.layer];
+      float* Wt = t.weights ? t.weights[tl.layer] : nullptr;
+      // every warp waits for the tile's accumulator, also one that meets none of its pieces: its
+      // arrival on d_empty below must not run ahead of the tile
+      if (!warp_wait(d_full + db, (tseq >> 1) & 1, abort_flag, lane)) { ok = false; break; }
+      tc_fence_after();
+      for (int w = 0; w < W && ok; ++w)
+        for (int pc = 0; pc < np; ++pc, ++kc) {
+          if ((int)(kc % kT3Groups) != g) continue;
+          const int s = kc % kT3Stages;
+          uint32_t gh[32];
+          tc_ld32(taddr + pc * 32, gh);
+          if (!warp_wait(m_full + s, (kc / kT3Stages) & 1, abort_flag, lane)) { ok = false; break; }
+          tc_wait_ld();
+          uint8_t* mp = piece(s) + row_in_tile * 128;
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            const int off = (c ^ (row_in_tile & 7)) << 4;
+            float4 m4 = *reinterpret_cast<const float4*>(mp + off);
+            m4.x -= __uint_as_float(gh[4 * c]); m4.y -= __uint_as_float(gh[4 * c + 1]);
+            m4.z -= __uint_as_float(gh[4 * c + 2]); m4.w -= __uint_as_float(gh[4 * c + 3]);
+            *reinterpret_cast<float4*>(mp + off) = m4;
+          }
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(e_ready + s);
+          if (w == 0 && row < L.n) {
+            // G_hat itself (and the model update w <- w - lr * G_hat): the thread's 32 consecutive columns
+            const int c0 = tl.col0 + pc * kTcK;
+            const size_t o = (size_t)row * L.m + c0;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+              if (c0 + 4 * c < L.m) {
+                const float4 g4 = make_float4(__uint_as_float(gh[4 * c]), __uint_as_float(gh[4 * c + 1]),
+                                              __uint_as_float(gh[4 * c + 2]), __uint_as_float(gh[4 * c + 3]));
+                if (Gh) __stcs(reinterpret_cast<float4*>(Gh + o) + c, g4);
+                if (Wt) {
+                  float4* wp = reinterpret_cast<float4*>(Wt + o) + c;
+                  float4 wv = __ldcs(wp);
+                  wv.x = fmaf(-t.lr, g4.x, wv.x); wv.y = fmaf(-t.lr, g4.y, wv.y);
+                  wv.z = fmaf(-t.lr, g4.z, wv.z); wv.w = fmaf(-t.lr, g4.w, wv.w);
+                  __stcs(wp, wv);
+                }
+              }
+            }
+          }
+        }
+      // past the tile: this warp no longer reads its accumulator
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(d_empty + db);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (tid == 0 && *abort_flag && t_end > t_begin) report_timeout(t, tiles[t_begin].layer);
+  if (warp == 2)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)S::kTmemCols) : "memory");
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -692,6 +936,18 @@ int tc_encode_maps(const LayerDev* layers, int n_layers, int W, int RP, void* ou
                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return LQSGD_ERR_CUDA;
     }
+    {   // stacked terms of P_bar, [n][kcat], and of Q_bar, [m][kcat]: 128 rows x 32 values (pass 3 operands)
+      const cuuint32_t box[2] = {kTcK, 128}, es[2] = {1, 1};
+      const cuuint64_t dimp[2] = {(cuuint64_t)L.kcat, (cuuint64_t)L.n}, dimq[2] = {(cuuint64_t)L.kcat, (cuuint64_t)L.m};
+      const cuuint64_t stride[1] = {(cuuint64_t)L.kcat * 4};
+      if (encode(&maps[i * kTcMapsPerLayer + 4], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, L.Pcat, dimp, stride, box, es,
+                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS ||
+          encode(&maps[i * kTcMapsPerLayer + 5], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, L.Qcat, dimq, stride, box, es,
+                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return LQSGD_ERR_CUDA;
+    }
     {   // Q^T and its tf32 remainders, [2 RP][mt]: 32 columns of Q for all 2 RP operand rows (pass 1)
       const cuuint64_t dim[2] = {(cuuint64_t)L.mt, (cuuint64_t)(2 * RP)};
       const cuuint64_t stride[1] = {(cuuint64_t)L.mt * 4};
@@ -703,6 +959,17 @@ int tc_encode_maps(const LayerDev* layers, int n_layers, int W, int RP, void* ou
     }
   }
   return LQSGD_OK;
+}
+
+cudaError_t launch_tc_pass3(int RP, const Tables& t, const Tile* tiles, int ntiles, const int* cta_begin, const void* maps,
+                            Launch l) {
+  if (ntiles == 0) return cudaSuccess;
+  if (RP != 16) return cudaErrorInvalidValue;
+  using S = Pass3Cfg<16>;
+  cudaError_t e = cudaFuncSetAttribute(tc_pass3_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)S::kTotal);
+  if (e != cudaSuccess) return e;
+  return launch_pdl(tc_pass3_kernel<16>, dim3(l.grid), dim3(kTcThreads), S::kTotal, l.stream, t, tiles, cta_begin,
+                    static_cast<const uint8_t*>(maps));
 }
 
 cudaError_t launch_tc_pass1(int RP, const Tables& t, const Tile* tiles, int ntiles, const int* cta_begin, const void* maps,
