@@ -384,10 +384,12 @@ def test_planted_rank_r_gradient_is_recovered_on_the_device():
     assert float(comp.get_state(B.STATE_E, 0, 0).abs().max()) <= 1e-4 * float(G.abs().max())
 
 
-def test_fused_model_update_matches_separate_update():
+@pytest.mark.parametrize("rank", [4, 16])
+def test_fused_model_update_matches_separate_update(rank):
     """Algorithm 1's last line, w <- w - lr * G_hat, fused into pass 3: same weights as updating
-    from the G_hat a plain step returns (and as the oracle's G_hat), with and without G_hat output."""
-    w = dataclasses.replace(wl.config2(), workers=2)          # includes a 32 x 25 layer and 1-D tensors
+    from the G_hat a plain step returns (and as the oracle's G_hat), with and without G_hat output.
+    Rank 16 runs it in the tensor-core pass 3."""
+    w = dataclasses.replace(wl.config2(), workers=2, rank=rank)   # includes a 32 x 25 layer and 1-D tensors
     a, b, c = make(w), make(w), make(w)
     lr = 0.125
     gen = torch.Generator(DEV).manual_seed(1)
