@@ -94,7 +94,7 @@ struct Plan {
   size_t bytes = 0;
 };
 
-int padded_rank(int r) { return r <= 1 ? 1 : r <= 2 ? 2 : r <= 4 ? 4 : r <= 8 ? 8 : 16; }
+int padded_rank(int r) { return r <= 1 ? 1 : r <= 2 ? 2 : r <= 4 ? 4 : r <= 8 ? 8 : r <= 16 ? 16 : 32; }
 
 int check_config(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config* c) {
   if (!shapes || !c || n_layers < 1) return LQSGD_ERR_INVALID_ARG;
@@ -195,7 +195,8 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
 
   // ---- tile sizes
   const size_t slots = (size_t)sm_count * 2, want = 3 * slots;
-  auto vec_of = [](int m) { return (m % 4 == 0) ? 4 : 1; };
+  // above padded rank 16 the register kernels run scalar only (they keep what the tensor-core passes cannot take)
+  auto vec_of = [&](int m) { return (RP <= 16 && m % 4 == 0) ? 4 : 1; };
   auto chunk_width = [&](int m, int cmax) {          // balanced column chunks, multiple of 32*VEC
     const int v = vec_of(m), q = 32 * v;
     const int lim = (v == 4) ? cmax : std::max(q, cmax / 4);

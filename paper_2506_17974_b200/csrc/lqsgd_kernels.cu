@@ -244,7 +244,8 @@ pass1_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
   pdl_wait();
   for (int i = blockIdx.x; i < ntiles; i += gridDim.x) {
     const Tile tl = tiles[i];
-    if (t.layers[tl.layer].vec) pass1_tile<RP, 4>(t, tl);
+    if constexpr (RP > 16) pass1_tile<RP, 1>(t, tl);   // above rank 16 these kernels only take what the tensor-core passes cannot
+    else if (t.layers[tl.layer].vec) pass1_tile<RP, 4>(t, tl);
     else pass1_tile<RP, 1>(t, tl);
   }
 }
@@ -340,12 +341,13 @@ template <int RP>
 __global__ void __launch_bounds__(kPassThreads, (RP <= 2 ? 4 : (RP <= 8 ? 3 : 1)))
 pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
   pdl_wait();
-  __shared__ float red[128 * 4 * RP];
+  __shared__ float red[128 * (RP > 16 ? 1 : 4) * RP];
   uint64_t pol;
   asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
   for (int i = blockIdx.x; i < ntiles; i += gridDim.x) {
     const Tile tl = tiles[i];
-    if (t.layers[tl.layer].vec) pass2_tile<RP, 4>(t, tl, red, pol);
+    if constexpr (RP > 16) pass2_tile<RP, 1>(t, tl, red, pol);
+    else if (t.layers[tl.layer].vec) pass2_tile<RP, 4>(t, tl, red, pol);
     else pass2_tile<RP, 1>(t, tl, red, pol);
   }
 }
@@ -435,7 +437,8 @@ pass3_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
   pdl_wait();
   for (int i = blockIdx.x; i < ntiles; i += gridDim.x) {
     const Tile tl = tiles[i];
-    if (t.layers[tl.layer].vec) pass3_tile<RP, 4>(t, tl);
+    if constexpr (RP > 16) pass3_tile<RP, 1>(t, tl);
+    else if (t.layers[tl.layer].vec) pass3_tile<RP, 4>(t, tl);
     else pass3_tile<RP, 1>(t, tl);
   }
 }
@@ -479,11 +482,11 @@ p_reduce_gram_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
     for (int j = 0; j < RP; ++j) rows[tid][j] = p[j];
   }
   __syncthreads();
-  if (tid < RP * RP) {
-    const int i = tid / RP, j = tid % RP;
+  for (int e = tid; e < RP * RP; e += 256) {
+    const int i = e / RP, j = e % RP;
     double s = 0.0;
     for (int k = 0; k < kFactorBlockRows; ++k) s = fma((double)rows[k][i], (double)rows[k][j], s);
-    L.gram_part[((size_t)fb.worker * L.npb + fb.blk) * (RP * RP) + tid] = s;
+    L.gram_part[((size_t)fb.worker * L.npb + fb.blk) * (RP * RP) + e] = s;
   }
 }
 
@@ -946,6 +949,7 @@ vectors_kernel(const VectorDev* __restrict__ vecs, const ExchangeChunk* __restri
     case 4: { constexpr int RP = 4; __VA_ARGS__; } break;   \
     case 8: { constexpr int RP = 8; __VA_ARGS__; } break;   \
     case 16: { constexpr int RP = 16; __VA_ARGS__; } break; \
+    case 32: { constexpr int RP = 32; __VA_ARGS__; } break; \
     default: return cudaErrorInvalidValue;          \
   }
 

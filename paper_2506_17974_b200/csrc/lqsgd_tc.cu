@@ -41,7 +41,6 @@ namespace {
 constexpr int kTcThreads = 640;       // 20 warps: M loader, B loader, MMA, spare, 4 epilogue, 12 consumers
 constexpr int kTcK = 32;              // rows of M per stage
 constexpr int kTcCols = 128;          // columns of M per tile: the M extent of one MMA
-constexpr int kTcMStages = 8;         // ring of M pieces (16 KB each)
 constexpr int kTcPair = 2;            // stages per operand slot: the MMA thread waits, issues and commits once per
                                       // slot (a lone thread runs a few cycles per instruction: its bookkeeping counts)
 constexpr int kTcAB = 4;              // ring of operand slots: A in TMEM, B in shared memory; deep enough to hide the
@@ -129,9 +128,10 @@ struct Pass2Cfg {
   static constexpr int kTmemCols = (kACol0 + kTcAB * kTcSlotK) <= 256 ? 256 : 512;
   static constexpr uint32_t kBBytes = kN * 128;                          // one B stage: 3 RP rows of 64 bf16
   static constexpr uint32_t kBStride = (kBBytes + 1023) / 1024 * 1024;   // stages stay 1024-byte aligned
-  static constexpr uint32_t kBOff = kTcMStages * kTcMBytes;
+  static constexpr int kMStages = RP <= 16 ? 8 : 6;                      // ring of M pieces (16 KB each): what fits beside B
+  static constexpr uint32_t kBOff = kMStages * kTcMBytes;
   static constexpr uint32_t kBarOff = kBOff + kTcAB * kTcPair * kBStride;
-  static constexpr int kBars = 2 * kTcMStages + 2 * kTcAB + 2 + 2 + 1;
+  static constexpr int kBars = 2 * kMStages + 2 * kTcAB + 2 + 2 + 1;
   static constexpr uint32_t kTotal = kBarOff + kBars * 8 + 16 + 1024;    // + abort flag, TMEM slot, alignment slack
   static_assert(kACol0 + kTcAB * kTcSlotK <= 512, "tensor memory");
   static_assert(kN % 16 == 0 && kN <= 256, "N of one MMA");
@@ -147,9 +147,9 @@ tc_pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, const uint
   float* mring = reinterpret_cast<float*>(base);
   uint8_t* bring = base + S::kBOff;
   uint64_t* bars = reinterpret_cast<uint64_t*>(base + S::kBarOff);
-  uint64_t* m_full = bars;                       // [kTcMStages] TMA landed
-  uint64_t* m_empty = m_full + kTcMStages;       // [kTcMStages] consumer warps have the piece in registers
-  uint64_t* ab_full = m_empty + kTcMStages;      // [kTcAB] slot ready: A written to TMEM (4 warps per stage) and B landed
+  uint64_t* m_full = bars;                       // [S::kMStages] TMA landed
+  uint64_t* m_empty = m_full + S::kMStages;       // [S::kMStages] consumer warps have the piece in registers
+  uint64_t* ab_full = m_empty + S::kMStages;      // [kTcAB] slot ready: A written to TMEM (4 warps per stage) and B landed
   uint64_t* ab_empty = ab_full + kTcAB;          // [kTcAB] the MMAs that read buffer i have completed
   uint64_t* d_full = ab_empty + kTcAB;           // [2] accumulator complete
   uint64_t* d_empty = d_full + 2;                // [2] accumulator drained
@@ -159,7 +159,7 @@ tc_pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, const uint
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
-    for (int s = 0; s < kTcMStages; ++s) { mbar_init(m_full + s, 1); mbar_init(m_empty + s, 4); }
+    for (int s = 0; s < S::kMStages; ++s) { mbar_init(m_full + s, 1); mbar_init(m_empty + s, 4); }
     for (int s = 0; s < kTcAB; ++s) { mbar_init(ab_full + s, 4 * kTcPair + 1); mbar_init(ab_empty + s, 1); }
     for (int s = 0; s < 2; ++s) { mbar_init(d_full + s, 1); mbar_init(d_empty + s, 4); }
     mbar_init(fin, 1);
@@ -185,8 +185,8 @@ tc_pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, const uint
       const uint8_t* map = maps + (size_t)tl.layer * kTcMapsPerLayer * kTcMapBytes;
       const int nk = tile_stages(tl.nrows);
       for (int k = 0; k < nk; ++k, ++kc) {
-        const int s = kc % kTcMStages;
-        if (!warp_wait(m_empty + s, ((kc / kTcMStages) & 1) ^ 1, abort_flag, lane)) { ok = false; break; }
+        const int s = kc % S::kMStages;
+        if (!warp_wait(m_empty + s, ((kc / S::kMStages) & 1) ^ 1, abort_flag, lane)) { ok = false; break; }
         if (lane == 0) {
           mbar_arrive_expect_tx(m_full + s, kTcMBytes);
           tma_load_3d(mring + (size_t)s * (kTcMBytes / 4), map, tl.col0, tl.row0 + k * kTcK, tl.worker, m_full + s);
@@ -194,8 +194,8 @@ tc_pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, const uint
       }
     }
     if (!ok && lane == 0)
-      for (uint32_t it = kc > (uint32_t)kTcMStages ? kc - kTcMStages : 0; it < kc; ++it)
-        drain(m_full + it % kTcMStages, (it / kTcMStages) & 1);
+      for (uint32_t it = kc > (uint32_t)S::kMStages ? kc - S::kMStages : 0; it < kc; ++it)
+        drain(m_full + it % S::kMStages, (it / S::kMStages) & 1);
   } else if (warp == 1) {
     // ---- B loader: rows [row0 + 32 k, +32) of the stacked P_bar terms
     uint32_t kc = 0;
@@ -298,9 +298,9 @@ tc_pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, const uint
       const int nk = tile_stages(tiles[ti].nrows);
       for (int k = 0; k < nk; ++k, ++kc) {
         if ((int)(kc % kTcGroups) != g) continue;
-        const int s = kc % kTcMStages;
+        const int s = kc % S::kMStages;
         const uint32_t slot = kc / kTcPair, ab = slot % kTcAB;
-        if (!warp_wait(m_full + s, (kc / kTcMStages) & 1, abort_flag, lane)) { ok = false; break; }
+        if (!warp_wait(m_full + s, (kc / S::kMStages) & 1, abort_flag, lane)) { ok = false; break; }
         const float* src = mring + (size_t)s * (kTcMBytes / 4) + 32 * q + lane;
         uint32_t v[32];
 #pragma unroll
@@ -964,33 +964,39 @@ int tc_encode_maps(const LayerDev* layers, int n_layers, int W, int RP, void* ou
 cudaError_t launch_tc_pass3(int RP, const Tables& t, const Tile* tiles, int ntiles, const int* cta_begin, const void* maps,
                             Launch l) {
   if (ntiles == 0) return cudaSuccess;
-  if (RP != 16) return cudaErrorInvalidValue;
-  using S = Pass3Cfg<16>;
-  cudaError_t e = cudaFuncSetAttribute(tc_pass3_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)S::kTotal);
-  if (e != cudaSuccess) return e;
-  return launch_pdl(tc_pass3_kernel<16>, dim3(l.grid), dim3(kTcThreads), S::kTotal, l.stream, t, tiles, cta_begin,
-                    static_cast<const uint8_t*>(maps));
+  auto go = [&](auto kernel, size_t smem) -> cudaError_t {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    return launch_pdl(kernel, dim3(l.grid), dim3(kTcThreads), smem, l.stream, t, tiles, cta_begin, static_cast<const uint8_t*>(maps));
+  };
+  if (RP == 16) return go(tc_pass3_kernel<16>, Pass3Cfg<16>::kTotal);
+  if (RP == 32) return go(tc_pass3_kernel<32>, Pass3Cfg<32>::kTotal);
+  return cudaErrorInvalidValue;
 }
 
 cudaError_t launch_tc_pass1(int RP, const Tables& t, const Tile* tiles, int ntiles, const int* cta_begin, const void* maps,
                             Launch l) {
   if (ntiles == 0) return cudaSuccess;
-  if (RP != 16) return cudaErrorInvalidValue;
-  using S = Pass1Cfg<16>;
-  cudaError_t e = cudaFuncSetAttribute(tc_pass1_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)S::kTotal);
-  if (e != cudaSuccess) return e;
-  return launch_pdl(tc_pass1_kernel<16>, dim3(l.grid), dim3(kTcThreads), S::kTotal, l.stream, t, tiles, cta_begin,
-                    static_cast<const uint8_t*>(maps));
+  auto go = [&](auto kernel, size_t smem) -> cudaError_t {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    return launch_pdl(kernel, dim3(l.grid), dim3(kTcThreads), smem, l.stream, t, tiles, cta_begin, static_cast<const uint8_t*>(maps));
+  };
+  if (RP == 16) return go(tc_pass1_kernel<16>, Pass1Cfg<16>::kTotal);
+  if (RP == 32) return go(tc_pass1_kernel<32>, Pass1Cfg<32>::kTotal);
+  return cudaErrorInvalidValue;
 }
 
 cudaError_t launch_tc_pass2(int RP, const Tables& t, const Tile* tiles, int ntiles, const void* maps, Launch l) {
   if (ntiles == 0) return cudaSuccess;
-  if (RP != 16) return cudaErrorInvalidValue;
-  using S = Pass2Cfg<16>;
-  cudaError_t e = cudaFuncSetAttribute(tc_pass2_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)S::kTotal);
-  if (e != cudaSuccess) return e;
-  return launch_pdl(tc_pass2_kernel<16>, dim3(l.grid), dim3(kTcThreads), S::kTotal, l.stream, t, tiles, ntiles,
-                    static_cast<const uint8_t*>(maps));
+  auto go = [&](auto kernel, size_t smem) -> cudaError_t {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    return launch_pdl(kernel, dim3(l.grid), dim3(kTcThreads), smem, l.stream, t, tiles, ntiles, static_cast<const uint8_t*>(maps));
+  };
+  if (RP == 16) return go(tc_pass2_kernel<16>, Pass2Cfg<16>::kTotal);
+  if (RP == 32) return go(tc_pass2_kernel<32>, Pass2Cfg<32>::kTotal);
+  return cudaErrorInvalidValue;
 }
 
 }  // namespace lqsgd

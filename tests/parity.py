@@ -143,6 +143,18 @@ def device_step_checked(comp: B.LQSGD, grads_dev, stats, check_payload=True):
     return recs, grads_host, ghat
 
 
+def codes_differ(a, b, bits):
+    """Element-wise: do two codes stand for different quantised values?  Magnitude 0 is the same
+    value under either sign bit (a factor entry within rounding of zero may come out as +0 or -0
+    on the two sides); with bits = 32 there are no codes."""
+    if bits == 32:
+        return np.zeros(np.shape(a), dtype=bool)
+    kmask = (1 << (bits - 1)) - 1
+    a = np.asarray(a).astype(np.int32)
+    b = np.asarray(b).astype(np.int32)
+    return (a != b) & (((a & kmask) != 0) | ((b & kmask) != 0))
+
+
 def oracle_step_forced(oracle: orc.Oracle, grads_host, recs, stats):
     """Free-running oracle step that adopts the device's code where its own differs (counted).
     Returns the oracle's per-layer results."""
@@ -154,14 +166,14 @@ def oracle_step_forced(oracle: orc.Oracle, grads_host, recs, stats):
         res = orc.layer_round(*args, average=oracle.average)
         fp = []
         for w in range(oracle.W):
-            diff = res["xp"]["codes"][w] != rec.codes_p[w]
+            diff = codes_differ(res["xp"]["codes"][w], rec.codes_p[w], oracle.bits_p)
             stats["forced"] = stats.get("forced", 0) + int(diff.sum())
             assert np.all(res["xp"]["margin"][w][diff] < 2e-2), "P code differs far from a threshold"
             fp.append(np.where(diff, rec.codes_p[w].astype(np.int16), -1))
         res = orc.layer_round(*args, forced_p=fp, average=oracle.average)
         fq = []
         for w in range(oracle.W):
-            diff = res["xq"]["codes"][w] != rec.codes_q[w]
+            diff = codes_differ(res["xq"]["codes"][w], rec.codes_q[w], oracle.bits_q)
             stats["forced"] = stats.get("forced", 0) + int(diff.sum())
             assert np.all(res["xq"]["margin"][w][diff] < 2e-2), "Q code differs far from a threshold"
             fq.append(np.where(diff, rec.codes_q[w].astype(np.int16), -1))

@@ -144,6 +144,21 @@ def test_value_domain_average_variant(W, bits):
     assert not torch.equal(b.get_state(B.STATE_P_BAR, 0), c.get_state(B.STATE_P_BAR, 0))
 
 
+@pytest.mark.parametrize("rank,W", [(30, 3), (32, 2), (20, 1)])
+def test_ranks_above_sixteen(rank, W):
+    """Ranks 17..32 (the paper's figures go to 30 and beyond): padded rank 32, products of the
+    aligned layers on the tensor cores, the 64 x 27 and 33 x 17 layers on the scalar register
+    kernels; stage by stage and free-running against the oracle."""
+    w = wl.Workload("r32", ((128, 576), (512, 1152), (64, 27), (100, 512), (33, 17), (40, 129), (130, 36), (24, 1)),
+                    rank=rank, bits=6, workers=W, steps=2, dist="student_t3", scale="fan_in", seed=rank)
+    run_steps(w, 2)
+
+
+def test_rank_thirty_on_the_resnet_set():
+    w = dataclasses.replace(wl.config5(30, 8), workers=2)
+    run_steps(w, 1, free_run=False)
+
+
 def test_different_bits_for_p_and_q():
     w = wl.Workload("bpq", ((96, 200), (48, 1)), rank=4, bits=3, workers=2, steps=2, dist="student_t3", scale="fan_in")
     comp = make(w, bits_p=3, bits_q=6)
