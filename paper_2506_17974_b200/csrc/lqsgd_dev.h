@@ -194,7 +194,7 @@ constexpr int kTcMapsPerLayer = 6;   // 0: M as [W][n][m], box 128 x 32 x 1;  1:
                                      // 2: E / M as [W][n][m], box 32 x 128 x 1, swizzled;  3: Qt, box 32 x 2RP, swizzled
                                      // 4: Pcat, 5: Qcat, box 32 x 128, swizzled
 constexpr int kTcRowsPerTile = 128;  // rows of a pass-1 tile: the M extent of one MMA
-constexpr int kTcPass1Cols = 576;    // most columns of a pass-1 tile (multiple of 32): small enough to balance the SMs
+constexpr int kTcPass1Cols = 1152;   // most columns of a pass-1 tile (multiple of 32): small enough to balance the SMs
 constexpr int kTcMapBytes = 128;
 constexpr int kTcRowChunk = 4096;    // most rows of a layer one pass-2 tile sums over (multiple of 64)
 int tc_encode_maps(const LayerDev* host_layers, int n_layers, int W, int RP, void* host_maps_out);   // 0 or LQSGD_ERR_CUDA

@@ -458,7 +458,7 @@ template <int RP>
 __global__ void __launch_bounds__(256)
 p_reduce_gram_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
   pdl_wait();
-  __shared__ float rows[kFactorBlockRows][RP];
+  __shared__ double rows[kFactorBlockRows][RP];     // the block's rows, converted once
   const FactorBlock fb = fbs[blockIdx.x];
   const LayerDev& L = t.layers[fb.layer];
   const int n = L.n;
@@ -479,77 +479,65 @@ p_reduce_gram_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
       if (L.ncc > 1) store_contig<RP>(L.Praw + ((size_t)fb.worker * n + row) * RP, p);
     }
 #pragma unroll
-    for (int j = 0; j < RP; ++j) rows[tid][j] = p[j];
+    for (int j = 0; j < RP; ++j) rows[tid][j] = (double)p[j];
   }
   __syncthreads();
   for (int e = tid; e < RP * RP; e += 256) {
     const int i = e / RP, j = e % RP;
+    if (j < i) continue;                                 // the Gram matrix is symmetric: upper triangle, mirrored
     double s = 0.0;
-    for (int k = 0; k < kFactorBlockRows; ++k) s = fma((double)rows[k][i], (double)rows[k][j], s);
-    L.gram_part[((size_t)fb.worker * L.npb + fb.blk) * (RP * RP) + e] = s;
+    for (int k = 0; k < kFactorBlockRows; ++k) s = fma(rows[k][i], rows[k][j], s);
+    double* gp = L.gram_part + ((size_t)fb.worker * L.npb + fb.blk) * (RP * RP);
+    gp[i * RP + j] = s;
+    gp[j * RP + i] = s;
   }
 }
 
-// Gram = sum of the block Grams (block order), Cholesky R^T R = Gram, R^-1 into Rinv (shared,
-// RP*RP doubles, row-major, upper triangular).  Run by a whole CTA; every CTA that applies R^-1
-// to a block of rows redoes this small factorisation itself, which costs less than a kernel
-// boundary.  Returns true if a column was dropped as dependent.
+// Gram = sum of the block Grams (block order), Cholesky  Gram = L L^T  (R = L^T), by a whole CTA;
+// every CTA that orthonormalises a block of rows redoes this small factorisation itself, which
+// costs less than a kernel boundary.  Lf (shared, RP*RP doubles, row-major) receives L, invd the
+// reciprocals of its diagonal, dead[j] = 1 for a column dropped as dependent (its row and column
+// of L are then those of the identity).  Returns true if any column was dropped.
 template <int RP>
-__device__ __forceinline__ bool cholesky_rinv(const LayerDev& L, int worker, double* Rinv) {
+__device__ __forceinline__ bool cholesky_lower(const LayerDev& L, int worker, double* Lf, double* invd, int* dead) {
   __shared__ double A[RP][RP + 1];     // Gram, overwritten by L (lower triangle)
-  __shared__ double X[RP][RP + 1];     // X[c][i] = (L^-1)[i][c]
   __shared__ double diag0[RP];
-  __shared__ int dead[RP];
   const int r = L.r, tid = threadIdx.x, nt = blockDim.x;
   for (int e = tid; e < RP * RP; e += nt) {
     const double* gp = L.gram_part + (size_t)worker * L.npb * (RP * RP) + e;
     double s = 0.0;
     for (int b = 0; b < L.npb; ++b) s += gp[(size_t)b * (RP * RP)];
     A[e / RP][e % RP] = s;
-    X[e / RP][e % RP] = 0.0;
   }
   __syncthreads();
-  if (tid < RP) { diag0[tid] = A[tid][tid]; dead[tid] = 0; }
+  if (tid < RP) { diag0[tid] = A[tid][tid]; dead[tid] = 0; invd[tid] = 1.0; }
   __syncthreads();
-  if (tid < 32) {
-    const int i = tid;               // lane = row of L
-    for (int j = 0; j < r; ++j) {
-      const double d = A[j][j];
-      __syncwarp();                  // every lane has read the pivot before lane j overwrites it
-      const bool ok = (d > kPivotEps * diag0[j]) && (d < INFINITY);   // false for nan too
-      double lij = 0.0;
-      if (ok) {
-        const double ljj = sqrt(d);
-        if (i == j) A[j][j] = ljj;
-        if (i > j && i < r) { lij = A[i][j] / ljj; A[i][j] = lij; }
-      } else {
-        if (i == j) { A[j][j] = 1.0; dead[j] = 1; }
-        if (i > j && i < r) A[i][j] = 0.0;
-      }
-      __syncwarp();
-      if (ok && i > j && i < r)
-        for (int k = j + 1; k <= i; ++k) A[i][k] -= lij * A[k][j];
-      __syncwarp();
+  // right-looking Cholesky, the whole CTA on every step: pivot, column j, then the rank-1 update of
+  // the trailing lower triangle with its entries dealt to the threads (every entry sees the
+  // updates in the order of j, so the result does not depend on the thread count)
+  for (int j = 0; j < r; ++j) {
+    const double d = A[j][j];
+    const bool ok = (d > kPivotEps * diag0[j]) && (d < INFINITY);   // false for nan too
+    const double ljj = ok ? sqrt(d) : 1.0;
+    const double inv = 1.0 / ljj;
+    __syncthreads();                   // everybody has read the pivot
+    for (int i = j + tid; i < r; i += nt) {
+      if (i == j) { A[j][j] = ljj; invd[j] = inv; if (!ok) dead[j] = 1; }
+      else A[i][j] = ok ? A[i][j] * inv : 0.0;
     }
-    // column c of L^-1 by forward substitution; a dead row or column stays zero
-    const int c = tid;
-    if (c < r) {
-      for (int row = c; row < r; ++row) {
-        double x = 0.0;
-        if (!dead[row]) {
-          double s = (row == c) ? 1.0 : 0.0;
-          for (int k = c; k < row; ++k) s -= A[row][k] * X[c][k];
-          x = s / A[row][row];
-        }
-        if (dead[c]) x = 0.0;
-        X[c][row] = x;
+    __syncthreads();
+    if (ok) {
+      const int w = r - j - 1;         // trailing block: rows and columns j+1 .. r-1
+      for (int e = tid; e < w * w; e += nt) {
+        const int i = j + 1 + e / w, k = j + 1 + e % w;
+        if (k <= i) A[i][k] -= A[i][j] * A[k][j];
       }
     }
+    __syncthreads();
   }
-  __syncthreads();
   for (int e = tid; e < RP * RP; e += nt) {
-    const int k = e / RP, j = e % RP;           // R^-1[k][j] = (L^-1)[j][k], k <= j < r
-    Rinv[e] = (k <= j && j < r) ? X[k][j] : 0.0;
+    const int i = e / RP, k = e % RP;
+    Lf[e] = (k <= i && i < r) ? A[i][k] : 0.0;
   }
   int any = 0;
   for (int j = 0; j < r; ++j) any |= dead[j];
@@ -570,26 +558,32 @@ template <int RP>
 __global__ void __launch_bounds__(kFactorBlockRows)
 p_apply_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
   pdl_wait();
-  __shared__ double Rinv[RP * RP];
+  __shared__ double Lf[RP * RP];
+  __shared__ double invd[RP];
+  __shared__ int dead[RP];
   __shared__ float smax[4];
   const FactorBlock fb = fbs[blockIdx.x];
   const LayerDev& L = t.layers[fb.layer];
   const int n = L.n, tid = threadIdx.x;
-  const bool dropped = cholesky_rinv<RP>(L, fb.worker, Rinv);
+  const bool dropped = cholesky_lower<RP>(L, fb.worker, Lf, invd, dead);
   if (dropped && fb.blk == 0 && tid == 0) atomicOr(&t.status[fb.layer], 1u);
   const int row = fb.blk * kFactorBlockRows + tid;
   float amax = 0.f;
   if (row < n) {
+    // the row of P solves  o R = p  with R = L^T upper triangular: forward substitution in fp64,
+    //   o[j] = (p[j] - sum_{k<j} o[k] L[j][k]) / L[j][j];   a dropped column gives 0
     float p[RP];
     load_contig_ro<RP>(L.Praw + ((size_t)fb.worker * n + row) * RP, p);
+    double od[RP];
     float o[RP];
     bool bad = false;
 #pragma unroll
     for (int j = 0; j < RP; ++j) {
-      double s = 0.0;
+      double s = (double)p[j];
 #pragma unroll
-      for (int k = 0; k <= j; ++k) s = fma((double)p[k], Rinv[k * RP + j], s);
-      o[j] = (float)s;
+      for (int k = 0; k < j; ++k) s = fma(-od[k], Lf[j * RP + k], s);
+      od[j] = (j < L.r && !dead[j]) ? s * invd[j] : 0.0;
+      o[j] = (float)od[j];
       amax = fmaxf(amax, fabsf(o[j]));
       bad |= !(fabsf(o[j]) < INFINITY);
     }
