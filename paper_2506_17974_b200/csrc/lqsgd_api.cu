@@ -318,8 +318,6 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
     L.gram_part = a.take<double>((size_t)W * L.npb * RP * RP);
     L.maxp = a.take<float>((size_t)W * L.npb);
     L.maxq = a.take<float>((size_t)W * L.nqb);
-    L.codesP = a.take<uint8_t>((size_t)W * mt.n * mt.r);
-    L.codesQ = a.take<uint8_t>((size_t)W * mt.m * mt.r);
     L.scales = a.take<float>(2);
     const auto& lo = p.layout[mt.user_index];
     L.pay_scale_off = lo.scale_offset; L.pay_p_off = lo.p_offset; L.pay_q_off = lo.q_offset;
@@ -934,8 +932,9 @@ static int locate_state(const lqsgd_ctx* c, int which, int layer, int worker, ch
     case LQSGD_STATE_P: *base = (char*)(L.P + w * n * RP); *rows = n; *row_bytes = 4 * r; *pitch = 4 * RP; break;
     case LQSGD_STATE_P_BAR: *base = (char*)L.Pbar; *rows = n; *row_bytes = 4 * r; *pitch = 4 * RP; break;
     case LQSGD_STATE_Q_W: *base = (char*)(L.Qw + w * m * RP); *rows = m; *row_bytes = 4 * r; *pitch = 4 * RP; break;
-    case LQSGD_STATE_CODES_P: if (c->cfg.bits_p == 32) return LQSGD_ERR_OUT_OF_RANGE; *base = (char*)(L.codesP + w * n * r); *rows = 1; *row_bytes = *pitch = n * r; break;
-    case LQSGD_STATE_CODES_Q: if (c->cfg.bits_q == 32) return LQSGD_ERR_OUT_OF_RANGE; *base = (char*)(L.codesQ + w * m * r); *rows = 1; *row_bytes = *pitch = m * r; break;
+    // codes are not kept unpacked: base = the worker's packed stream, rows = number of codes (see lqsgd_get_state)
+    case LQSGD_STATE_CODES_P: if (c->cfg.bits_p == 32) return LQSGD_ERR_OUT_OF_RANGE; *base = (char*)(p.d_payload + w * p.payload_stride + L.pay_p_off); *rows = n * r; *row_bytes = *pitch = 1; break;
+    case LQSGD_STATE_CODES_Q: if (c->cfg.bits_q == 32) return LQSGD_ERR_OUT_OF_RANGE; *base = (char*)(p.d_payload + w * p.payload_stride + L.pay_q_off); *rows = m * r; *row_bytes = *pitch = 1; break;
     case LQSGD_STATE_SCALES: *base = (char*)L.scales; *rows = 1; *row_bytes = *pitch = 8; break;
     default: return LQSGD_ERR_OUT_OF_RANGE;
   }
@@ -948,6 +947,12 @@ int lqsgd_get_state(const lqsgd_ctx* c, int32_t which, int32_t layer, int32_t wo
   char* base; size_t rows, rb, pitch;
   const int rc = locate_state(c, which, layer, worker, &base, &rows, &rb, &pitch);
   if (rc != LQSGD_OK) return rc;
+  if (which == LQSGD_STATE_CODES_P || which == LQSGD_STATE_CODES_Q) {   // unpacked on demand from the payload
+    CK(launch_unpack_codes(reinterpret_cast<const uint8_t*>(base), (int)rows,
+                           which == LQSGD_STATE_CODES_P ? c->cfg.bits_p : c->cfg.bits_q, static_cast<uint8_t*>(dev_dst),
+                           static_cast<cudaStream_t>(cuda_stream)));
+    return LQSGD_OK;
+  }
   CK(cudaMemcpy2DAsync(dev_dst, rb, base, pitch, rb, rows, cudaMemcpyDeviceToDevice,
                        static_cast<cudaStream_t>(cuda_stream)));
   return LQSGD_OK;

@@ -41,8 +41,6 @@ struct LayerDev {
   double* gram_part;          // [W][npb][RP*RP]
   float* maxp;                // [W][npb]
   float* maxq;                // [W][nqb]
-  uint8_t* codesP;            // [W][n*r]
-  uint8_t* codesQ;            // [W][m*r]
   float* scales;              // [2]  s_P, s_Q
   uint64_t pay_scale_off, pay_p_off, pay_q_off;   // byte offsets inside one worker's payload
 };
@@ -139,6 +137,7 @@ struct SplitExchange {
 };
 cudaError_t launch_exchange(int RP, int which /*0 = P, 1 = Q*/, const Tables& t, const QuantTables& q,
                             const ExchangeChunk* ch, int nch, const SplitExchange& sx, Launch l);
+cudaError_t launch_unpack_codes(const uint8_t* stream, int count, int bits, uint8_t* out, cudaStream_t st);
 cudaError_t launch_scale_reduce(const Tables& t, int which, float* scales, int n_mat, Launch l);
 cudaError_t launch_sum_dequant(int RP, int which, const Tables& t, const QuantTables& q, const ExchangeChunk* ch,
                                int nch, const SplitExchange& sx, const uint8_t* gathered, int n_streams, Launch l);

@@ -675,29 +675,29 @@ __device__ __forceinline__ void store_factor(const LayerDev& L, int which, int r
 // The threshold table holds, for every level boundary, the smallest fp32 not below the exact
 // boundary, so "t >= thr" decides exactly like the real-number comparison.
 // ---------------------------------------------------------------------------------------
-template <int RP>
+// B = bits per code (2..8), or 32: quantiser bypassed.  One block = 256 factor elements.
+template <int RP, int B>
 __global__ void __launch_bounds__(256)
 exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __restrict__ chunks, SplitExchange sx) {
   pdl_wait();
   constexpr int CH = kExchangeChunk;   // 256 factor elements per block, one per thread
   constexpr int WB = 8;                // workers handled per round
+  constexpr int NLEV = (B == 32) ? 2 : 1 << (B - 1);
   __shared__ float thr[128];
-  __shared__ uint8_t codes[WB][CH];
+  __shared__ __align__(4) uint8_t codes[WB][CH + 4];
   __shared__ float sred[8];
   const ExchangeChunk ch = chunks[blockIdx.x];
   const LayerDev& L = t.layers[ch.layer];
-  const int W = t.W, tid = threadIdx.x, b = qt.bits;
-  const int nlev = (b == 32) ? 2 : 1 << (b - 1);
+  const int W = t.W, tid = threadIdx.x;
   const int rows = which ? L.m : L.n, r = L.r;
   const int count = rows * r;
   const int nblk = which ? L.nqb : L.npb;
   const float* __restrict__ maxes = which ? L.maxq : L.maxp;
   const float* __restrict__ src = which ? L.Qw : L.P;   // [W][rows][RP]
-  float* dst = which ? L.Q : L.Pbar;                    // [rows][RP]
-  uint8_t* ucodes = which ? L.codesQ : L.codesP;        // [W][count]
   const uint64_t pay_off = which ? L.pay_q_off : L.pay_p_off;
 
-  for (int i = tid; i < nlev - 1; i += 256) thr[i] = qt.thr[i];
+  for (int i = tid; i < NLEV - 1; i += 256) thr[i] = qt.thr[i];
+  if (tid < WB) *reinterpret_cast<uint32_t*>(&codes[tid][CH]) = 0u;     // what a word task reads past the chunk
   float s = 0.f;
   for (int i = tid; i < W * nblk; i += 256) s = fmaxf(s, __ldg(maxes + i));
 #pragma unroll
@@ -710,7 +710,7 @@ exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __rest
   if (sx.pack_only) s = sx.scales[which * sx.n_mat + ch.layer];   // scale agreed between the ranks
   const bool s_ok = (s > 0.f) && (s < INFINITY);
 
-  if (b == 32) {
+  if constexpr (B == 32) {
     // Quantiser bypassed (plain PowerSGD exchange): the factor travels as fp32 and the workers'
     // factors are averaged directly (Eq. 1), in worker order.
     const int e = ch.chunk * CH + tid;
@@ -724,8 +724,7 @@ exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __rest
         const unsigned bits32 = __float_as_uint(x);               // the stream may start on any byte
         pay[0] = bits32 & 0xff; pay[1] = (bits32 >> 8) & 0xff; pay[2] = (bits32 >> 16) & 0xff; pay[3] = bits32 >> 24;
       }
-      const float v = sum / (float)W;
-      store_factor<RP>(L, which, row, col, v);
+      store_factor<RP>(L, which, row, col, sum / (float)W);
     }
     if (ch.chunk == 0 && tid == 0) {
       L.scales[which] = s;
@@ -736,80 +735,106 @@ exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __rest
       if (!(s < INFINITY)) atomicOr(&t.status[ch.layer], 8u);
     }
     return;
-  }
+  } else {
+    constexpr int NW = CH * B / 32;      // 32-bit words of one worker's stream in this chunk
+    const int e0 = ch.chunk * CH;
+    const int cnt = min(CH, count - e0);
+    const bool valid = tid < cnt;
+    const int e = e0 + tid;
+    const int row = valid ? e / r : 0, col = valid ? e % r : 0;
+    const size_t nbytes_total = ((size_t)count * B + 7) / 8;
+    const size_t byte0 = (size_t)ch.chunk * (CH / 8) * B;
+    const int nbytes = (int)min((size_t)(CH / 8) * B, nbytes_total - byte0);
+    int S = 0;
+    float Sv = 0.f;          // value-domain variant: sum of the workers' dequantised levels, in worker order
 
-  const int e0 = ch.chunk * CH;
-  const int cnt = min(CH, count - e0);
-  const bool valid = tid < cnt;
-  const int e = e0 + tid;
-  const int row = valid ? e / r : 0, col = valid ? e % r : 0;
-  const size_t nbytes_total = ((size_t)count * b + 7) / 8;
-  const size_t byte0 = (size_t)ch.chunk * (CH / 8) * b;
-  const int nbytes = (int)min((size_t)(CH / 8) * b, nbytes_total - byte0);
-  int S = 0;
-  float Sv = 0.f;          // value-domain variant: sum of the workers' dequantised levels, in worker order
-
-  for (int w0 = 0; w0 < W; w0 += WB) {
-    const int wn = min(WB, W - w0);
-    float x[WB];
+    for (int w0 = 0; w0 < W; w0 += WB) {
+      const int wn = min(WB, W - w0);
+      float x[WB];
 #pragma unroll
-    for (int u = 0; u < WB; ++u)
-      x[u] = (valid && u < wn) ? __ldg(src + ((size_t)(w0 + u) * rows + row) * RP + col) : 0.f;
+      for (int u = 0; u < WB; ++u)
+        x[u] = (valid && u < wn) ? __ldg(src + ((size_t)(w0 + u) * rows + row) * RP + col) : 0.f;
 #pragma unroll
-    for (int u = 0; u < WB; ++u) {
-      if (u < wn) {
-        int k = 0;
-        if (s_ok && valid) {
-          const float tt = __fdiv_rn(fabsf(x[u]), s);
-          int lo = 0, hi = nlev - 1;                 // k = #{i : tt >= thr[i]}, thr ascending
-          while (lo < hi) {
-            const int mid = (lo + hi) >> 1;
-            if (tt >= thr[mid]) lo = mid + 1; else hi = mid;
+      for (int u = 0; u < WB; ++u) {
+        if (u < wn) {
+          int k = 0;
+          if (s_ok && valid) {
+            const float tt = __fdiv_rn(fabsf(x[u]), s);
+            // k = #{i : tt >= thr[i]}, thr ascending, NLEV - 1 = 2^(B-1) - 1 entries: B - 1 halving steps
+#pragma unroll
+            for (int step = NLEV / 2; step >= 1; step >>= 1)
+              if (tt >= thr[k + step - 1]) k += step;
           }
-          k = lo;
+          const int neg = (valid && x[u] < 0.f) ? 1 : 0;
+          codes[u][tid] = (uint8_t)((neg << (B - 1)) | k);   // 0 beyond the factor's end: pads the last byte
+          const int sk = neg ? -k : k;
+          S += sk;
+          if (qt.avg_values) Sv += __ldg(qt.deq + sk + (NLEV - 1));
         }
-        const int neg = (valid && x[u] < 0.f) ? 1 : 0;
-        const uint8_t code = (uint8_t)((neg << (b - 1)) | k);
-        codes[u][tid] = code;                        // 0 beyond the factor's end: pads the last byte
-        if (valid) ucodes[(size_t)(w0 + u) * count + e] = code;
-        S += neg ? -k : k;
-        if (qt.avg_values) Sv += __ldg(qt.deq + (neg ? -k : k) + (nlev - 1));
       }
-    }
-    __syncthreads();
-    for (int idx = tid; idx < wn * nbytes; idx += 256) {
-      const int u = idx / nbytes, jb = idx - u * nbytes;
-      const int bit0 = jb * 8;
-      const int elo = bit0 / b;
-      const int ehi = min((bit0 + 7) / b, CH - 1);
-      unsigned v = 0;
-      for (int q = elo; q <= ehi; ++q) {
-        const int sh = q * b - bit0;
-        const unsigned c = codes[u][q];
-        v |= (sh >= 0) ? (c << sh) : (c >> (-sh));
+      __syncthreads();
+      // little-endian bit stream: word j of the chunk holds bits [32 j, 32 j + 32) = the codes of
+      // elements 32 j / B .. (32 j + 31) / B
+      for (int task = tid; task < wn * NW; task += 256) {
+        const int u = task / NW, j = task - u * NW;
+        const int bit0 = 32 * j;
+        const int q0 = bit0 / B;
+        uint32_t word = 0;
+#pragma unroll
+        for (int i = 0; i < 32 / B + 2; ++i) {
+          const int q = q0 + i;
+          const int sh = q * B - bit0;
+          if (sh < 32) {
+            const uint32_t c = codes[u][min(q, CH + 3)];
+            word |= (sh >= 0) ? (c << sh) : (c >> (-sh));
+          }
+        }
+        const int nb = min(4, nbytes - 4 * j);       // bytes of this word inside the stream
+        uint8_t* pay = t.payload + (size_t)(w0 + u) * t.payload_stride + pay_off + byte0 + 4 * j;
+        uint8_t* snd = sx.pack_only
+            ? sx.send[which] + (size_t)(w0 + u) * sx.region_bytes[which] + (pay_off - sx.region_off[which]) + byte0 + 4 * j
+            : nullptr;
+        if (nb == 4 && (reinterpret_cast<uintptr_t>(pay) & 3) == 0) *reinterpret_cast<uint32_t*>(pay) = word;
+        else
+          for (int i = 0; i < nb; ++i) pay[i] = (uint8_t)(word >> (8 * i));
+        if (snd) {           // the same stream, contiguous over the local workers, for the all-gather
+          if (nb == 4 && (reinterpret_cast<uintptr_t>(snd) & 3) == 0) *reinterpret_cast<uint32_t*>(snd) = word;
+          else
+            for (int i = 0; i < nb; ++i) snd[i] = (uint8_t)(word >> (8 * i));
+        }
       }
-      t.payload[(size_t)(w0 + u) * t.payload_stride + pay_off + byte0 + jb] = (uint8_t)(v & 0xffu);
-      if (sx.pack_only)      // the same stream, contiguous over the local workers, for the all-gather
-        sx.send[which][(size_t)(w0 + u) * sx.region_bytes[which] + (pay_off - sx.region_off[which]) + byte0 + jb] =
-            (uint8_t)(v & 0xffu);
+      __syncthreads();
     }
-    __syncthreads();
-  }
 
-  if (valid && !sx.pack_only) {
-    float v = 0.f;
-    if (s_ok) v = qt.avg_values ? s * (Sv / (float)W) : s * __ldg(qt.deq + S + W * (nlev - 1));
-    store_factor<RP>(L, which, row, col, v);
-  }
-  if (ch.chunk == 0 && tid == 0) {
-    L.scales[which] = s;
-    for (int w = 0; w < W; ++w) {
-      float* ps = reinterpret_cast<float*>(t.payload + (size_t)w * t.payload_stride + L.pay_scale_off);
-      ps[which] = s;
+    if (valid && !sx.pack_only) {
+      float v = 0.f;
+      if (s_ok) v = qt.avg_values ? s * (Sv / (float)W) : s * __ldg(qt.deq + S + W * (NLEV - 1));
+      store_factor<RP>(L, which, row, col, v);
     }
-    if (!(s > 0.f)) atomicOr(&t.status[ch.layer], which ? 4u : 2u);
-    if (!(s < INFINITY)) atomicOr(&t.status[ch.layer], 8u);
+    if (ch.chunk == 0 && tid == 0) {
+      L.scales[which] = s;
+      for (int w = 0; w < W; ++w) {
+        float* ps = reinterpret_cast<float*>(t.payload + (size_t)w * t.payload_stride + L.pay_scale_off);
+        ps[which] = s;
+      }
+      if (!(s > 0.f)) atomicOr(&t.status[ch.layer], which ? 4u : 2u);
+      if (!(s < INFINITY)) atomicOr(&t.status[ch.layer], 8u);
+    }
   }
+}
+
+// One worker's unpacked codes (one per byte) from its packed stream: what lqsgd_get_state returns
+// for LQSGD_STATE_CODES_*.
+__global__ void __launch_bounds__(256)
+unpack_codes_kernel(const uint8_t* __restrict__ stream, int count, int b, uint8_t* __restrict__ out) {
+  const int e = blockIdx.x * 256 + threadIdx.x;
+  if (e >= count) return;
+  const size_t nbytes = ((size_t)count * b + 7) / 8;
+  const size_t bit = (size_t)e * b, byte = bit >> 3;
+  const int sh = (int)(bit & 7);
+  unsigned v = stream[byte];
+  if (sh + b > 8 && byte + 1 < nbytes) v |= (unsigned)stream[byte + 1] << 8;
+  out[e] = (uint8_t)((v >> sh) & ((1u << b) - 1u));
 }
 
 // Qt[j][i] = Q[i][j]: refreshes the transposed copy after Q was set from outside.
@@ -992,7 +1017,21 @@ cudaError_t launch_q_reduce(int rp, const Tables& t, const FactorBlock* fb, int 
 cudaError_t launch_exchange(int rp, int which, const Tables& t, const QuantTables& q,
                             const ExchangeChunk* ch, int nch, const SplitExchange& sx, Launch l) {
   if (nch == 0) return cudaSuccess;
-  LQSGD_DISPATCH_RP(rp, (launch_pdl(exchange_kernel<RP>, nch, 256, 0, l.stream, t, q, which, ch, sx)));
+#define LQSGD_EXCHANGE_BITS(BV) case BV: launch_pdl(exchange_kernel<RP, BV>, nch, 256, 0, l.stream, t, q, which, ch, sx); break;
+  LQSGD_DISPATCH_RP(rp, {
+    switch (q.bits) {
+      LQSGD_EXCHANGE_BITS(2) LQSGD_EXCHANGE_BITS(3) LQSGD_EXCHANGE_BITS(4) LQSGD_EXCHANGE_BITS(5)
+      LQSGD_EXCHANGE_BITS(6) LQSGD_EXCHANGE_BITS(7) LQSGD_EXCHANGE_BITS(8) LQSGD_EXCHANGE_BITS(32)
+      default: return cudaErrorInvalidValue;
+    }
+  });
+#undef LQSGD_EXCHANGE_BITS
+  return cudaGetLastError();
+}
+
+cudaError_t launch_unpack_codes(const uint8_t* stream, int count, int bits, uint8_t* out, cudaStream_t st) {
+  if (count == 0) return cudaSuccess;
+  unpack_codes_kernel<<<(count + 255) / 256, 256, 0, st>>>(stream, count, bits, out);
   return cudaGetLastError();
 }
 
