@@ -669,7 +669,7 @@ struct Pass3Cfg {
   static constexpr uint32_t kOpBytes = kSub * kT1PieceBytes;             // one operand: kSub pieces of 128 rows x 32
   static constexpr uint32_t kOpOff = kT3Stages * kT1PieceBytes;
   static constexpr uint32_t kBarOff = kOpOff + 2 * kOpBytes;
-  static constexpr int kBars = 3 * kT3Stages + 2 + 2 + 2 + 1;
+  static constexpr int kBars = 3 * kT3Stages + 2 + 2 + 2 + 2 + 1;      // m_full, e_ready, m_empty; op_full, op_empty, d_full, d_empty (2 each); fin
   static constexpr uint32_t kTotal = kBarOff + kBars * 8 + 16 + 1024;
   static constexpr int kTmemCols = 256;                                  // two accumulators of 128 columns
 };
