@@ -290,25 +290,35 @@ def factor_bits(n, m, rank, bits):
     return r * (n + m) * bits
 
 
-def payload_bytes(layers, rank, bits_p, bits_q):
+def payload_bytes(layers, rank, bits_p, bits_q, quantize_vectors=False):
     """Bytes one worker sends per round: for each matrix the two code streams, each
-    padded to a whole byte, plus the two fp32 scales; fp32 for every 1-D tensor."""
+    padded to a whole byte, plus the two fp32 scales; fp32 for every 1-D tensor, or, with
+    quantize_vectors (the variant that log-quantises them too, b_p bits), one fp32 scale and
+    a code stream padded to a whole byte."""
     total = 0
     for n, m in layers:
         if n > 1 and m > 1:
             r = effective_rank(rank, n, m)
             total += (r * n * bits_p + 7) // 8 + (r * m * bits_q + 7) // 8 + 8
+        elif quantize_vectors and bits_p != 32:
+            total += 4 + (n * m * bits_p + 7) // 8
         else:
             total += 4 * n * m
     return total
 
 
-def assemble_payload(layers, rank, bits_p, bits_q, scales, codes_p, codes_q, vectors):
+def assemble_payload(layers, rank, bits_p, bits_q, scales, codes_p, codes_q, vectors, vector_scales=None):
     """One worker's payload in the library's documented order:
     [s_P, s_Q of every matrix][every 1-D tensor, fp32][P codes of every matrix][Q codes ...].
-    scales: list of (s_P, s_Q); codes_*: per matrix uint8 code arrays; vectors: per 1-D tensor."""
+    scales: list of (s_P, s_Q); codes_*: per matrix uint8 code arrays; vectors: per 1-D tensor.
+    With vector_scales (the variant that quantises the 1-D tensors): `vectors` holds their uint8
+    codes, and the order is [matrix scales][one scale per 1-D tensor][their code streams][P][Q]."""
     parts = [np.asarray([v for pair in scales for v in pair], dtype="<f4").view(np.uint8)]
-    parts += [np.asarray(v, dtype="<f4").reshape(-1).view(np.uint8) for v in vectors]
+    if vector_scales is not None:
+        parts += [np.asarray(list(vector_scales), dtype="<f4").view(np.uint8)]
+        parts += [pack_codes(c, bits_p) for c in vectors]
+    else:
+        parts += [np.asarray(v, dtype="<f4").reshape(-1).view(np.uint8) for v in vectors]
     parts += [pack_codes(c, bits_p) for c in codes_p]
     parts += [pack_codes(c, bits_q) for c in codes_q]
     return np.concatenate(parts) if parts else np.zeros(0, np.uint8)
@@ -321,9 +331,10 @@ class Oracle:
     """State machine of Algorithm 1 over a list of layers: E_0 = 0, Q_0 supplied by the
     caller (drawn N(0,1) outside), Q_t = dequantised averaged Q of step t-1."""
 
-    def __init__(self, layers, rank, bits_p, bits_q, alpha, workers, Q0, average="codes"):
+    def __init__(self, layers, rank, bits_p, bits_q, alpha, workers, Q0, average="codes", quantize_vectors=False):
         self.layers = [tuple(s) for s in layers]
         self.average = average
+        self.quantize_vectors = bool(quantize_vectors) and bits_p != 32
         self.rank, self.bits_p, self.bits_q = rank, bits_p, bits_q
         self.alpha, self.W = float(alpha), workers
         self.E, self.Q = {}, {}
@@ -347,6 +358,11 @@ class Oracle:
                                   self.alpha, f[0], f[1], self.average)
                 self.E[li] = res["E_new"]
                 self.Q[li] = res["Q_bar"]
+            elif self.quantize_vectors:
+                # variant: a 1-D tensor goes through the same exchange as a factor (one scale, b_p bits)
+                x = exchange_factor([Gl[w].reshape(-1, 1) for w in range(self.W)], self.bits_p, self.alpha,
+                                    average=self.average)
+                res = dict(mean=x["mean"].reshape(-1), scale=x["scale"], codes=[c.reshape(-1) for c in x["codes"]])
             else:
                 res = dict(mean=vector_mean(Gl.reshape(self.W, -1)))
             out.append(res)

@@ -206,3 +206,29 @@ def test_resnet18_shape_list_reproduces_published_epoch_sizes():
     assert round(full) == 3339 and round(r1) == 14                       # Table II
     full, r1 = sizes(wl.resnet18_layers(10, in_channels=1), 93)
     assert round(full) == 3964 and round(r1) == 16                       # Table III
+
+
+def test_quantised_vectors_variant():
+    """1-D tensors through the factor exchange: payload closed form, one-worker round trip of the
+    levels, and agreement with exchange_factor on the reshaped tensor."""
+    layers = ((6, 5), (1, 9), (7, 1))
+    assert orc.payload_bytes(layers, 2, 4, 4, quantize_vectors=True) == (2 * 6 * 4 + 7) // 8 + (2 * 5 * 4 + 7) // 8 + 8 \
+        + (4 + (9 * 4 + 7) // 8) + (4 + (7 * 4 + 7) // 8)
+    assert orc.payload_bytes(layers, 2, 32, 32, quantize_vectors=True) == orc.payload_bytes(layers, 2, 32, 32)
+    rng = np.random.default_rng(3)
+    Q0 = {0: rng.standard_normal((5, 2))}
+    o = orc.Oracle(layers, 2, 4, 4, 127.0, 1, Q0, quantize_vectors=True)
+    lev = orc.level_values(4, 127.0)
+    v = np.float32(2.0) * np.array([lev[7], -lev[3], lev[0], lev[5], -lev[7], lev[1], lev[2], -lev[6], lev[4]], np.float32)
+    g = [[rng.standard_normal((6, 5)).astype(np.float32), v.reshape(1, 9), rng.standard_normal((7, 1)).astype(np.float32)]]
+    out = o.step(g)
+    assert out[1]["scale"] == np.float32(2.0)
+    assert np.allclose(out[1]["mean"], v.astype(np.float64), rtol=1e-6, atol=0)       # every level round-trips
+    assert list(out[1]["codes"][0] & 7) == [7, 3, 0, 5, 7, 1, 2, 6, 4]
+    x = orc.exchange_factor([g[0][2].reshape(-1, 1)], 4, 127.0)
+    assert np.array_equal(out[2]["mean"], x["mean"].reshape(-1))
+    pay = orc.assemble_payload(layers, 2, 4, 4, [(out[0]["xp"]["scale"], out[0]["xq"]["scale"])],
+                               [out[0]["xp"]["codes"][0]], [out[0]["xq"]["codes"][0]],
+                               [out[1]["codes"][0], out[2]["codes"][0]], vector_scales=[out[1]["scale"], out[2]["scale"]])
+    assert pay.size == orc.payload_bytes(layers, 2, 4, 4, quantize_vectors=True)
+    assert np.array_equal(pay[8:16].view("<f4"), np.array([out[1]["scale"], out[2]["scale"]], dtype="<f4"))
