@@ -82,6 +82,12 @@ typedef enum lqsgd_error {
                                         receives, Section V).  Default, as Algorithm 1 writes it: mean of the quantised
                                         values, then Eq. 5 once.  Codes, scales and payload are the same in both. */
 
+#define LQSGD_FLAG_QUANTIZE_VECTORS 8u /* variant: the 1-D tensors go through the same exchange as a factor (one fp32 scale
+                                         = max over workers and entries, bits_p bits per entry, Eq. 4 / Eq. 5) instead of
+                                         travelling as fp32.  Payload: [s_P, s_Q per matrix][one scale per 1-D tensor]
+                                         [their code streams][P streams][Q streams].  Ignored with bits_p = 32; not
+                                         available with workers on several GPUs (lqsgd_round_begin refuses). */
+
 typedef struct lqsgd_ctx lqsgd_ctx;
 
 typedef struct lqsgd_shape {
@@ -108,12 +114,12 @@ typedef struct lqsgd_config {
 typedef struct lqsgd_layer_layout {
   int32_t is_matrix;     /* 1: low-rank path, 0: one-dimensional tensor sent as fp32 */
   int32_t rank_eff;      /* r_eff (0 for a 1-D tensor) */
-  uint64_t scale_offset; /* matrix: fp32 s_P then fp32 s_Q */
+  uint64_t scale_offset; /* matrix: fp32 s_P then fp32 s_Q; quantised 1-D tensor: its fp32 scale */
   uint64_t p_offset;     /* matrix: P code stream, p_bytes = ceil(n * r_eff * b_p / 8) */
   uint64_t p_bytes;
   uint64_t q_offset;     /* matrix: Q code stream, q_bytes = ceil(m * r_eff * b_q / 8) */
   uint64_t q_bytes;
-  uint64_t vec_offset;   /* 1-D tensor: rows*cols fp32 values */
+  uint64_t vec_offset;   /* 1-D tensor: rows*cols fp32 values, or (LQSGD_FLAG_QUANTIZE_VECTORS) its code stream */
   uint64_t vec_bytes;
 } lqsgd_layer_layout;
 

@@ -22,6 +22,7 @@ STATUS_DEPENDENT_COLUMN, STATUS_ZERO_SCALE_P, STATUS_ZERO_SCALE_Q, STATUS_NONFIN
 FLAG_HOST_STAGING = 1
 FLAG_REGISTER_PATH = 2
 FLAG_AVERAGE_VALUES = 4
+FLAG_QUANTIZE_VECTORS = 8
 STATUS_TIMEOUT = 16
 N_PHASES = 5
 XCHG_SCALES_P, XCHG_SCALES_Q, XCHG_STREAMS_P, XCHG_STREAMS_Q = range(4)
@@ -153,7 +154,7 @@ class LQSGD:
     def __init__(self, layers: Sequence[Tuple[int, int]], rank: int, bits_p: int, bits_q: Optional[int] = None,
                  alpha: float = 127.0, workers: int = 1, seed: int = 0, host_staging: bool = False,
                  device: str = "cuda:0", register_path: bool = False, world_workers: int = 0,
-                 average: str = "codes"):
+                 average: str = "codes", quantize_vectors: bool = False):
         self.lib = load_library()
         self.layers = [(int(n), int(m)) for n, m in layers]
         self.rank, self.bits_p = rank, bits_p
@@ -162,11 +163,13 @@ class LQSGD:
         if average not in ("codes", "values"):
             raise ValueError("average must be 'codes' (Algorithm 1) or 'values'")
         self.average = average
+        self.quantize_vectors = bool(quantize_vectors) and bits_p != 32
         self.device = torch.device(device)
         self.cfg = make_config(rank, self.bits_p, self.bits_q, alpha, workers, seed,
                                (FLAG_HOST_STAGING if host_staging else 0)
                                | (FLAG_REGISTER_PATH if register_path else 0)
-                               | (FLAG_AVERAGE_VALUES if average == "values" else 0), world_workers)
+                               | (FLAG_AVERAGE_VALUES if average == "values" else 0)
+                               | (FLAG_QUANTIZE_VECTORS if quantize_vectors else 0), world_workers)
         nbytes = workspace_bytes(self.layers, self.cfg)
         with torch.cuda.device(self.device):
             self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)

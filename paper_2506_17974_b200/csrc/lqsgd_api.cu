@@ -108,7 +108,9 @@ int check_config(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
     if (c->world_workers < c->workers || c->world_workers > 4096 || c->world_workers % c->workers) return LQSGD_ERR_INVALID_ARG;
     if (c->world_workers > c->workers && (c->bits_p == 32 || c->bits_q == 32)) return LQSGD_ERR_INVALID_ARG;
   }
-  if (c->flags & ~(LQSGD_FLAG_HOST_STAGING | LQSGD_FLAG_REGISTER_PATH | LQSGD_FLAG_AVERAGE_VALUES)) return LQSGD_ERR_INVALID_ARG;
+  if (c->flags & ~(LQSGD_FLAG_HOST_STAGING | LQSGD_FLAG_REGISTER_PATH | LQSGD_FLAG_AVERAGE_VALUES |
+                   LQSGD_FLAG_QUANTIZE_VECTORS))
+    return LQSGD_ERR_INVALID_ARG;
   for (int i = 0; i < n_layers; ++i) {
     if (shapes[i].rows < 1 || shapes[i].cols < 1) return LQSGD_ERR_BAD_SHAPE;
     if ((int64_t)shapes[i].rows * shapes[i].cols > (int64_t)1 << 30) return LQSGD_ERR_BAD_SHAPE;
@@ -163,16 +165,19 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
       const int r = std::min({cfg.rank, shapes[i].rows, shapes[i].cols});
       p.mats.push_back({shapes[i].rows, shapes[i].cols, r, i});
     } else {
-      p.vecs.push_back({shapes[i].rows * shapes[i].cols, i, 0});
+      p.vecs.push_back({shapes[i].rows * shapes[i].cols, i, 0, 0});
     }
   }
   // ---- payload layout: [scales][1-D fp32][P streams][Q streams]
   size_t off = 0;
   for (auto& mt : p.mats) { p.layout[mt.user_index].scale_offset = off; off += 8; }
+  const bool qvec = (cfg.flags & LQSGD_FLAG_QUANTIZE_VECTORS) && cfg.bits_p != 32;
+  if (qvec)
+    for (auto& v : p.vecs) { v.pay_scale_off = off; p.layout[v.user_index].scale_offset = off; off += 4; }
   for (auto& v : p.vecs) {
     v.pay_off = off;
     auto& lo = p.layout[v.user_index];
-    lo.vec_offset = off; lo.vec_bytes = 4 * (size_t)v.len;
+    lo.vec_offset = off; lo.vec_bytes = qvec ? ((size_t)v.len * cfg.bits_p + 7) / 8 : 4 * (size_t)v.len;
     off += lo.vec_bytes;
   }
   for (auto& mt : p.mats) {
@@ -722,6 +727,13 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
   switch (seg) {
     case 0:
       if (nv) {
+        if ((c->cfg.flags & LQSGD_FLAG_QUANTIZE_VECTORS) && c->cfg.bits_p != 32) {
+          if (split) return LQSGD_ERR_INVALID_ARG;
+          CK(launch_vectors_quant(p.d_vecs, (int)nv, reinterpret_cast<const float* const*>(p.d_ptrs + vbase),
+                                  reinterpret_cast<float* const*>(p.d_ptrs + vbase + nv * W),
+                                  c->has_weights ? reinterpret_cast<float* const*>(p.d_ptrs + vbase + nv * (W + 1)) : nullptr,
+                                  t.lr, p.d_payload, p.payload_stride, W, qp, {st, 0}));
+        } else
         CK(launch_vectors(p.d_vecs, p.d_chV, (int)p.chV.size(),
                           reinterpret_cast<const float* const*>(p.d_ptrs + vbase),
                           reinterpret_cast<float* const*>(p.d_ptrs + vbase + nv * W),

@@ -49,7 +49,8 @@ struct LayerDev {
 struct VectorDev {
   int32_t len;
   int32_t user_index;
-  uint64_t pay_off;           // byte offset inside one worker's payload (4-byte aligned)
+  uint64_t pay_off;           // byte offset inside one worker's payload: fp32 values (4-byte aligned) or code stream
+  uint64_t pay_scale_off;     // quantised variant: where the tensor's fp32 scale goes (4-byte aligned)
 };
 
 // A rectangular piece of one layer handled by one CTA of a streaming pass.
@@ -146,6 +147,10 @@ cudaError_t launch_q_transpose(const float* Q, float* Qt, float* Qcat, int m, in
 cudaError_t launch_pass2(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
 cudaError_t launch_q_reduce(int RP, const Tables& t, const FactorBlock* fb, int nfb, Launch l);
 cudaError_t launch_pass3(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
+// Variant: 1-D tensors log-quantised like a factor (one CTA per tensor).
+cudaError_t launch_vectors_quant(const VectorDev* vecs, int nvecs, const float* const* vgrads, float* const* vghat,
+                                 float* const* vweights, float lr, uint8_t* payload, uint64_t payload_stride, int W,
+                                 const QuantTables& q, Launch l);
 cudaError_t launch_vectors(const VectorDev* vecs, const ExchangeChunk* chunks, int nchunks,
                            const float* const* vgrads, float* const* vghat, float* const* vweights, float lr,
                            uint8_t* payload, uint64_t payload_stride, int W, int W_total, Launch l);

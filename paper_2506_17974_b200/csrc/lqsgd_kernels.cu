@@ -956,6 +956,96 @@ vectors_kernel(const VectorDev* __restrict__ vecs, const ExchangeChunk* __restri
   if (vweights && vweights[ch.layer]) vweights[ch.layer][i] = fmaf(-lr, mean, vweights[ch.layer][i]);
 }
 
+// Variant (LQSGD_FLAG_QUANTIZE_VECTORS): a 1-D tensor goes through the factor exchange, one CTA per
+// tensor: scale = max over workers and entries, code = sign | level (Eq. 4), little-endian b-bit
+// stream per worker, exact integer sum of the signed levels (or, value-domain variant, the sum of the
+// dequantised levels), Eq. 5 once.  Entries are taken 256 at a time, 8 workers per round.
+template <int B>
+__global__ void __launch_bounds__(256)
+vectors_quant_kernel(const VectorDev* __restrict__ vecs, const float* const* __restrict__ vgrads,
+                     float* const* __restrict__ vghat, float* const* __restrict__ vweights, float lr, uint8_t* payload,
+                     uint64_t payload_stride, int W, QuantTables qt) {
+  pdl_wait();
+  constexpr int CH = 256, WB = 8, NLEV = 1 << (B - 1), NW = CH * B / 32;
+  __shared__ float thr[128];
+  __shared__ __align__(4) uint8_t codes[WB][CH + 4];
+  __shared__ float sred[8];
+  const VectorDev v = vecs[blockIdx.x];
+  const int tid = threadIdx.x, len = v.len;
+  for (int i = tid; i < NLEV - 1; i += 256) thr[i] = qt.thr[i];
+  if (tid < WB) *reinterpret_cast<uint32_t*>(&codes[tid][CH]) = 0u;
+  float s = 0.f;
+  for (int w = 0; w < W; ++w) {
+    const float* g = vgrads[(size_t)blockIdx.x * W + w];
+    for (int i = tid; i < len; i += 256) s = fmaxf(s, fabsf(g[i]));
+  }
+#pragma unroll
+  for (int o = 16; o >= 1; o >>= 1) s = fmaxf(s, __shfl_xor_sync(0xffffffffu, s, o));
+  if ((tid & 31) == 0) sred[tid >> 5] = s;
+  __syncthreads();
+  s = sred[0];
+#pragma unroll
+  for (int i = 1; i < 8; ++i) s = fmaxf(s, sred[i]);
+  const bool s_ok = (s > 0.f) && (s < INFINITY);
+  if (tid == 0)
+    for (int w = 0; w < W; ++w) *reinterpret_cast<float*>(payload + (size_t)w * payload_stride + v.pay_scale_off) = s;
+  const size_t nbytes_total = ((size_t)len * B + 7) / 8;
+  float* gh = vghat[blockIdx.x];
+  float* wt = vweights ? vweights[blockIdx.x] : nullptr;
+  for (int e0 = 0; e0 < len; e0 += CH) {
+    const bool valid = e0 + tid < len;
+    const size_t byte0 = (size_t)(e0 / 8) * B;
+    const int nbytes = (int)min((size_t)(CH / 8) * B, nbytes_total - byte0);
+    int S = 0;
+    float Sv = 0.f;
+    for (int w0 = 0; w0 < W; w0 += WB) {
+      const int wn = min(WB, W - w0);
+#pragma unroll
+      for (int u = 0; u < WB; ++u) {
+        if (u < wn) {
+          const float x = valid ? vgrads[(size_t)blockIdx.x * W + w0 + u][e0 + tid] : 0.f;
+          int k = 0;
+          if (s_ok && valid) {
+            const float tt = __fdiv_rn(fabsf(x), s);
+#pragma unroll
+            for (int step = NLEV / 2; step >= 1; step >>= 1)
+              if (tt >= thr[k + step - 1]) k += step;
+          }
+          const int neg = (valid && x < 0.f) ? 1 : 0;
+          codes[u][tid] = (uint8_t)((neg << (B - 1)) | k);
+          const int sk = neg ? -k : k;
+          S += sk;
+          if (qt.avg_values) Sv += __ldg(qt.deq + sk + (NLEV - 1));
+        }
+      }
+      __syncthreads();
+      for (int task = tid; task < wn * NW; task += 256) {
+        const int u = task / NW, j = task - u * NW;
+        const int bit0 = 32 * j, q0 = bit0 / B;
+        uint32_t word = 0;
+#pragma unroll
+        for (int i = 0; i < 32 / B + 2; ++i) {
+          const int q = q0 + i, sh = q * B - bit0;
+          if (sh < 32) {
+            const uint32_t c = codes[u][min(q, CH + 3)];
+            word |= (sh >= 0) ? (c << sh) : (c >> (-sh));
+          }
+        }
+        const int nb = min(4, nbytes - 4 * j);
+        uint8_t* pay = payload + (size_t)(w0 + u) * payload_stride + v.pay_off + byte0 + 4 * j;
+        for (int i = 0; i < nb; ++i) pay[i] = (uint8_t)(word >> (8 * i));
+      }
+      __syncthreads();
+    }
+    if (valid) {
+      float mean = 0.f;
+      if (s_ok) mean = qt.avg_values ? s * (Sv / (float)W) : s * __ldg(qt.deq + S + W * (NLEV - 1));
+      if (gh) gh[e0 + tid] = mean;
+      if (wt) wt[e0 + tid] = fmaf(-lr, mean, wt[e0 + tid]);
+    }
+  }
+}
+
 }  // namespace
 
 // ---------------------------------------------------------------------------------------
@@ -1054,6 +1144,19 @@ cudaError_t launch_vectors(const VectorDev* vecs, const ExchangeChunk* chunks, i
                            uint8_t* payload, uint64_t payload_stride, int W, int W_total, Launch l) {
   if (nchunks == 0) return cudaSuccess;
   launch_pdl(vectors_kernel, nchunks, 256, 0, l.stream, vecs, chunks, vgrads, vghat, vweights, lr, payload, payload_stride, W, W_total);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_vectors_quant(const VectorDev* vecs, int nvecs, const float* const* vgrads, float* const* vghat,
+                                 float* const* vweights, float lr, uint8_t* payload, uint64_t payload_stride, int W,
+                                 const QuantTables& q, Launch l) {
+  if (nvecs == 0) return cudaSuccess;
+#define LQSGD_VQ_BITS(BV) case BV: launch_pdl(vectors_quant_kernel<BV>, nvecs, 256, 0, l.stream, vecs, vgrads, vghat, vweights, lr, payload, payload_stride, W, q); break;
+  switch (q.bits) {
+    LQSGD_VQ_BITS(2) LQSGD_VQ_BITS(3) LQSGD_VQ_BITS(4) LQSGD_VQ_BITS(5) LQSGD_VQ_BITS(6) LQSGD_VQ_BITS(7) LQSGD_VQ_BITS(8)
+    default: return cudaErrorInvalidValue;
+  }
+#undef LQSGD_VQ_BITS
   return cudaGetLastError();
 }
 

@@ -103,10 +103,17 @@ def check_layer_stage_isolated(comp: B.LQSGD, layer: int, G, rec: StepRecord, st
     return errs
 
 
-def expected_payload(comp: B.LQSGD, recs, grads_host, worker: int) -> np.ndarray:
-    """The worker's payload rebuilt by the oracle's packer from the device's codes and scales."""
+def expected_payload(comp: B.LQSGD, recs, grads_host, worker: int, vec_x=None) -> np.ndarray:
+    """The worker's payload rebuilt by the oracle's packer from the device's codes and scales
+    (for quantised 1-D tensors, which keep no state on the device: from the oracle's exchange, vec_x)."""
     mats = [l for l in range(len(comp.layers)) if comp.is_matrix(l)]
     vecs = [l for l in range(len(comp.layers)) if not comp.is_matrix(l)]
+    if comp.quantize_vectors:
+        return orc.assemble_payload(
+            comp.layers, comp.rank, comp.bits_p, comp.bits_q,
+            [(recs[l].scales[0], recs[l].scales[1]) for l in mats],
+            [recs[l].codes_p[worker] for l in mats], [recs[l].codes_q[worker] for l in mats],
+            [vec_x[l]["codes"][worker].reshape(-1) for l in vecs], vector_scales=[vec_x[l]["scale"] for l in vecs])
     return orc.assemble_payload(
         comp.layers, comp.rank, comp.bits_p, comp.bits_q,
         [(recs[l].scales[0], recs[l].scales[1]) for l in mats],
@@ -123,8 +130,16 @@ def device_step_checked(comp: B.LQSGD, grads_dev, stats, check_payload=True):
     torch.cuda.synchronize()
     grads_host = [[host(g) for g in per] for per in grads_dev]
     recs = {}
+    vec_x = {}
     for l in range(len(comp.layers)):
-        if comp.is_matrix(l):
+        if not comp.is_matrix(l) and comp.quantize_vectors:
+            V = [grads_host[w][l].reshape(-1, 1) for w in range(comp.W)]
+            vec_x[l] = orc.exchange_factor(V, comp.bits_p, comp.alpha, average=comp.average)
+            want = vec_x[l]["mean"].reshape(-1)
+            got = host(ghat[l]).reshape(-1)
+            assert np.max(np.abs(got - want)) <= 1e-6 * max(np.max(np.abs(want)), 1e-30) + 1e-12, l
+            stats["vector_codes"] = stats.get("vector_codes", 0) + comp.W * want.size
+        elif comp.is_matrix(l):
             recs[l] = StepRecord(comp, l, E_prev[l], Q_prev[l], ghat[l])
             G = np.stack([grads_host[w][l] for w in range(comp.W)])
             check_layer_stage_isolated(comp, l, G, recs[l], stats)
@@ -135,10 +150,10 @@ def device_step_checked(comp: B.LQSGD, grads_dev, stats, check_payload=True):
             assert np.max(np.abs(got - want)) <= 1e-6 * max(np.max(np.abs(want)), 1e-30) + 1e-12
     if check_payload:
         for w in range(comp.W):
-            want = expected_payload(comp, recs, grads_host, w)
+            want = expected_payload(comp, recs, grads_host, w, vec_x)
             got = host(comp.payload(w))
             assert got.size == comp.payload_nbytes == want.size == orc.payload_bytes(
-                comp.layers, comp.rank, comp.bits_p, comp.bits_q)
+                comp.layers, comp.rank, comp.bits_p, comp.bits_q, comp.quantize_vectors)
             assert np.array_equal(got, want), f"payload bytes of worker {w} differ"
     return recs, grads_host, ghat
 

@@ -24,7 +24,8 @@ def make(w: wl.Workload, **kw):
 
 def new_oracle(comp: B.LQSGD):
     Q0 = {l: par.host(comp.get_state(B.STATE_Q, l)) for l in range(len(comp.layers)) if comp.is_matrix(l)}
-    return orc.Oracle(comp.layers, comp.rank, comp.bits_p, comp.bits_q, comp.alpha, comp.W, Q0, average=comp.average)
+    return orc.Oracle(comp.layers, comp.rank, comp.bits_p, comp.bits_q, comp.alpha, comp.W, Q0, average=comp.average,
+                      quantize_vectors=comp.quantize_vectors)
 
 
 def run_steps(w: wl.Workload, steps: int, free_run=True, comp=None):
@@ -157,6 +158,28 @@ def test_ranks_above_sixteen(rank, W):
 def test_rank_thirty_on_the_resnet_set():
     w = dataclasses.replace(wl.config5(30, 8), workers=2)
     run_steps(w, 1, free_run=False)
+
+
+@pytest.mark.parametrize("bits,W,average", [(4, 3, "codes"), (3, 9, "codes"), (8, 2, "values"), (2, 1, "codes")])
+def test_quantised_vectors_variant(bits, W, average):
+    """LQSGD_FLAG_QUANTIZE_VECTORS: the 1-D tensors are log-quantised like a factor (one scale, b_p bits):
+    means against the oracle's exchange of the same tensors, payload bit for bit, layout and size."""
+    w = wl.Workload("qvec", ((96, 200), (1, 300), (64, 27), (700, 1), (1, 7), (513, 1)), rank=3, bits=bits, workers=W,
+                    steps=2, dist="student_t3", scale="fan_in", seed=17 + bits)
+    comp = make(w, average=average, quantize_vectors=True)
+    assert comp.payload_nbytes == orc.payload_bytes(w.layers, 3, bits, bits, quantize_vectors=True)
+    lay = comp.payload_layout(1)
+    assert lay.is_matrix == 0 and lay.vec_bytes == (300 * bits + 7) // 8 and lay.scale_offset == 2 * 8
+    stats = {}
+    for t in range(2):
+        par.device_step_checked(comp, wl.draw_gradients(w, t, device=DEV), stats)
+    assert stats["vector_codes"] == 2 * W * (300 + 700 + 7 + 513)
+    # with the model update: the 1-D weights move by lr times the dequantised mean
+    wts = [torch.zeros(s, device=DEV) for s in w.layers]
+    gh = [torch.empty(s, device=DEV) for s in w.layers]
+    comp.step_update(wl.draw_gradients(w, 2, device=DEV), gh, wts, 0.5)
+    torch.cuda.synchronize()
+    assert torch.allclose(wts[3], -0.5 * gh[3], rtol=0, atol=1e-7)
 
 
 def test_different_bits_for_p_and_q():
