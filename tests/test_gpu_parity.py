@@ -227,9 +227,10 @@ def test_full_size_largest_layer_properties():
     assert resid <= 4e-7 * g[0][0].abs().max().item()
 
 
-def test_zero_gradient_sets_status_and_zero_outputs():
+@pytest.mark.parametrize("rank", [3, 16])
+def test_zero_gradient_sets_status_and_zero_outputs(rank):
     layers = ((40, 64), (16, 1))
-    comp = B.LQSGD(layers, 3, 4, workers=2)
+    comp = B.LQSGD(layers, rank, 4, workers=2)
     grads = [[torch.zeros(s, device=DEV) for s in layers] for _ in range(2)]
     ghat = [torch.full(s, 7.0, device=DEV) for s in layers]
     comp.step(grads, ghat)
@@ -241,26 +242,54 @@ def test_zero_gradient_sets_status_and_zero_outputs():
     assert float(comp.get_state(B.STATE_E, 0, 1).abs().max()) == 0.0
     assert int(comp.get_state(B.STATE_CODES_P, 0, 0).max()) == 0
     # oracle agrees: dependent columns, zero scale, zero result
-    res = orc.layer_round(np.zeros((2, 40, 64), np.float32), np.zeros((2, 40, 64)), np.ones((64, 3)), 4, 4, 127.0)
+    res = orc.layer_round(np.zeros((2, 40, 64), np.float32), np.zeros((2, 40, 64)), np.ones((64, rank)), 4, 4, 127.0)
     assert res["dependent"].all() and np.all(res["G_hat"] == 0)
 
 
-def test_dependent_column_matches_oracle():
-    """Q with two identical columns: the second column of M Q is dependent and becomes zero."""
+@pytest.mark.parametrize("rank", [3, 12, 24])
+def test_dependent_column_matches_oracle(rank):
+    """Q with two identical columns: the second column of M Q is dependent and becomes zero
+    (ranks 12 and 24 run the products on the tensor cores)."""
     layers = ((48, 80),)
-    comp = B.LQSGD(layers, 3, 4, workers=1)
-    Q = torch.randn(80, 3, generator=torch.Generator().manual_seed(3))
+    comp = B.LQSGD(layers, rank, 4, workers=1)
+    Q = torch.randn(80, rank, generator=torch.Generator().manual_seed(3))
     Q[:, 1] = Q[:, 0]
     comp.set_state(B.STATE_Q, 0, 0, Q)
-    w = wl.Workload("dep", layers, rank=3, bits=4, workers=1, steps=1, dist="normal", scale="fan_in")
+    w = wl.Workload("dep", layers, rank=rank, bits=4, workers=1, steps=1, dist="normal", scale="fan_in")
     stats = {}
     recs, _, _ = par.device_step_checked(comp, wl.draw_gradients(w, 0, device=DEV), stats)
     assert comp.status()[0] & B.STATUS_DEPENDENT_COLUMN
     assert np.all(recs[0].P[0][:, 1] == 0)
 
 
-def test_bit_reproducible_and_checkpoint_resume():
-    w = dataclasses.replace(wl.config2(), workers=3)
+@pytest.mark.parametrize("rank", [16, 2])
+def test_non_finite_gradient_is_flagged_without_a_fault(rank):
+    """An inf or nan in one worker's gradient: undefined numbers for that layer, LQSGD_STATUS_NONFINITE,
+    the other layers untouched, the context usable afterwards."""
+    layers = ((64, 128), (40, 96))
+    w = wl.Workload("nonfinite", layers, rank=rank, bits=4, workers=2, steps=2, dist="normal", scale="fan_in", seed=4)
+    a, b = make(w), make(w)
+    g = wl.draw_gradients(w, 0, device=DEV)
+    bad = [[x.clone() for x in per] for per in g]
+    bad[1][0][5, 7] = float("inf")
+    bad[0][0][9, 3] = float("nan")
+    oa = [torch.empty(s, device=DEV) for s in layers]
+    ob = [torch.empty(s, device=DEV) for s in layers]
+    a.step(bad, oa)
+    b.step(g, ob)
+    torch.cuda.synchronize()
+    st = a.status()
+    assert st[0] & B.STATUS_NONFINITE and st[1] == 0 and not (st[0] & B.STATUS_TIMEOUT)
+    assert torch.equal(oa[1], ob[1])                       # the clean layer is what it is without the bad one
+    a.set_state(B.STATE_E, 0, 0, torch.zeros(layers[0], device=DEV))
+    a.set_state(B.STATE_E, 0, 1, torch.zeros(layers[0], device=DEV))
+    a.set_state(B.STATE_Q, 0, 0, b.get_state(B.STATE_Q, 0))
+    assert b.status() == [0, 0]
+
+
+@pytest.mark.parametrize("rank", [4, 16])
+def test_bit_reproducible_and_checkpoint_resume(rank):
+    w = dataclasses.replace(wl.config2(), workers=3, rank=rank)
     a, b = make(w), make(w)
     gh = lambda: [torch.empty(s, device=DEV) for s in w.layers]
     oa, ob = gh(), gh()
