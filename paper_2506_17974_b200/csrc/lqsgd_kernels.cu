@@ -518,8 +518,10 @@ __device__ __forceinline__ bool cholesky_lower(const LayerDev& L, int worker, do
   for (int j = 0; j < r; ++j) {
     const double d = A[j][j];
     const bool ok = (d > kPivotEps * diag0[j]) && (d < INFINITY);   // false for nan too
-    const double ljj = ok ? sqrt(d) : 1.0;
-    const double inv = 1.0 / ljj;
+    // 1 / sqrt(d) by the hardware seed plus refinement (the library sqrt and division are long
+    // software sequences, and this loop is a chain of r of them); l_jj = d / sqrt(d)
+    const double inv = ok ? rsqrt(d) : 1.0;
+    const double ljj = ok ? d * inv : 1.0;
     __syncthreads();                   // everybody has read the pivot
     for (int i = j + tid; i < r; i += nt) {
       if (i == j) { A[j][j] = ljj; invd[j] = inv; if (!ok) dead[j] = 1; }
