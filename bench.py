@@ -40,29 +40,31 @@ def load_peaks():
     return 6650.0, "fallback"
 
 
-def csrc_digest() -> str:
-    """SHA-256 over the kernel sources: ties a stored ncu figure to the code it was taken from."""
+def csrc_digest(files=None) -> str:
+    """SHA-256 over kernel sources (all of csrc, or the named files): ties a stored ncu figure to the
+    code it was taken from."""
     h = hashlib.sha256()
     d = os.path.join(ROOT, "paper_2506_17974_b200", "csrc")
-    for name in sorted(os.listdir(d)):
-        if name.endswith((".cu", ".cuh", ".h")):
-            h.update(name.encode())
-            with open(os.path.join(d, name), "rb") as f:
-                h.update(f.read())
+    names = sorted(files) if files else sorted(n for n in os.listdir(d) if n.endswith((".cu", ".cuh", ".h")))
+    for name in names:
+        h.update(name.encode())
+        with open(os.path.join(d, name), "rb") as f:
+            h.update(f.read())
     return h.hexdigest()
 
 
 def recorded_traffic(workload: str, phase: str):
     """DRAM bytes (read + write) per launch of that phase's kernel from the ncu capture summarised under
-    profiles/, or None when there is no capture of this workload or the kernels changed since."""
+    profiles/, or None when there is no capture of this workload or the kernel's sources changed since."""
     path = os.path.join(ROOT, "profiles", "dram_traffic.json")
     if not os.path.exists(path):
         return None
     with open(path) as f:
         rec = json.load(f)
-    if rec.get("csrc_sha256") != csrc_digest():
-        return None
-    return rec.get("workloads", {}).get(workload, {}).get(phase)
+    for e in rec.get("entries", []):
+        if e.get("workload") == workload and e.get("phase") == phase:
+            return e["dram_bytes"] if e.get("sha256") == csrc_digest(e.get("sources")) else None
+    return None
 
 
 def kernel_name(phase: str, rank: int) -> str:
@@ -508,7 +510,9 @@ def main():
                     help="workers of all GPUs in one average, with the real NCCL exchange (default: independent replicas)")
     args = ap.parse_args()
     if args.source_digest:
-        print(csrc_digest())
+        for group in (["lqsgd_stream.cu", "lqsgd_stream_common.cuh", "lqsgd_dev.h"], ["lqsgd_kernels.cu", "lqsgd_dev.h"],
+                      ["lqsgd_tc.cu", "lqsgd_stream_common.cuh", "lqsgd_dev.h"]):
+            print(" ".join(group), csrc_digest(group))
         return
     if args.impl == "reference":
         run_reference(args)
