@@ -249,8 +249,12 @@ def effective_rank(rank, n, m):
     return min(rank, n, m)
 
 
-def layer_round(G, E, Q, bits_p, bits_q, alpha, forced_p=None, forced_q=None, average="codes"):
+def layer_round(G, E, Q, bits_p, bits_q, alpha, forced_p=None, forced_q=None, average="codes", power_iters=1):
     """One iteration of Algorithm 1 for one n x m layer and W workers.
+
+    power_iters > 1 (an option, Algorithm 1 does one): the power step with its two exchanges is
+    repeated on the same M, each time from the Q_bar just obtained; the last P_bar, Q_bar form
+    G_hat.  forced_* apply to the last repetition; the returned intermediates are the last ones.
 
     G, E: arrays [W, n, m];  Q: [m, r] shared by all workers (warm start).
     Returns a dict with every intermediate:
@@ -261,14 +265,17 @@ def layer_round(G, E, Q, bits_p, bits_q, alpha, forced_p=None, forced_q=None, av
     G = np.asarray(G)
     W = G.shape[0]
     M = [error_feedback(G[w], E[w]) for w in range(W)]
-    P_raw = [power_step_p(M[w], Q) for w in range(W)]
-    orth = [orthonormalize(P_raw[w]) for w in range(W)]
-    P = [o[0] for o in orth]
-    xp = exchange_factor(P, bits_p, alpha, forced_p, average)
-    P_bar = xp["mean"]
-    Qw = [power_step_q(M[w], P_bar) for w in range(W)]
-    xq = exchange_factor(Qw, bits_q, alpha, forced_q, average)
-    Q_bar = xq["mean"]
+    for it in range(power_iters):
+        last = it == power_iters - 1
+        P_raw = [power_step_p(M[w], Q) for w in range(W)]
+        orth = [orthonormalize(P_raw[w]) for w in range(W)]
+        P = [o[0] for o in orth]
+        xp = exchange_factor(P, bits_p, alpha, forced_p if last else None, average)
+        P_bar = xp["mean"]
+        Qw = [power_step_q(M[w], P_bar) for w in range(W)]
+        xq = exchange_factor(Qw, bits_q, alpha, forced_q if last else None, average)
+        Q_bar = xq["mean"]
+        Q = Q_bar
     G_hat = reconstruct(P_bar, Q_bar)
     E_new = [error_update(M[w], G_hat) for w in range(W)]
     return dict(M=np.stack(M), P_raw=np.stack(P_raw), P=np.stack(P),
@@ -331,8 +338,10 @@ class Oracle:
     """State machine of Algorithm 1 over a list of layers: E_0 = 0, Q_0 supplied by the
     caller (drawn N(0,1) outside), Q_t = dequantised averaged Q of step t-1."""
 
-    def __init__(self, layers, rank, bits_p, bits_q, alpha, workers, Q0, average="codes", quantize_vectors=False):
+    def __init__(self, layers, rank, bits_p, bits_q, alpha, workers, Q0, average="codes", quantize_vectors=False,
+                 power_iters=1):
         self.layers = [tuple(s) for s in layers]
+        self.power_iters = int(power_iters)
         self.average = average
         self.quantize_vectors = bool(quantize_vectors) and bits_p != 32
         self.rank, self.bits_p, self.bits_q = rank, bits_p, bits_q
@@ -355,7 +364,7 @@ class Oracle:
             if li in self.E:
                 f = (forced or {}).get(li, (None, None))
                 res = layer_round(Gl, self.E[li], self.Q[li], self.bits_p, self.bits_q,
-                                  self.alpha, f[0], f[1], self.average)
+                                  self.alpha, f[0], f[1], self.average, self.power_iters)
                 self.E[li] = res["E_new"]
                 self.Q[li] = res["Q_bar"]
             elif self.quantize_vectors:

@@ -232,3 +232,33 @@ def test_quantised_vectors_variant():
                                [out[1]["codes"][0], out[2]["codes"][0]], vector_scales=[out[1]["scale"], out[2]["scale"]])
     assert pay.size == orc.payload_bytes(layers, 2, 4, 4, quantize_vectors=True)
     assert np.array_equal(pay[8:16].view("<f4"), np.array([out[1]["scale"], out[2]["scale"]], dtype="<f4"))
+
+
+def test_several_power_iterations_option():
+    """power_iters = T repeats the power step on the same M: with the quantiser bypassed and one
+    worker it is T steps of subspace iteration written out by hand (library QR), it leaves a
+    rank-r matrix fixed, and more iterations bring P_bar Q_bar^T closer to the truncated SVD."""
+    rng = np.random.default_rng(8)
+    n, m, r = 30, 22, 3
+    G = rng.standard_normal((1, n, m)).astype(np.float32)
+    E = np.zeros((1, n, m))
+    Q0 = rng.standard_normal((m, r))
+    res = orc.layer_round(G, E, Q0, 32, 32, 127.0, power_iters=3)
+    M, Q = G[0].astype(np.float64), Q0
+    for _ in range(3):
+        P, R = np.linalg.qr(M @ Q)
+        P = P * np.sign(np.diag(R))
+        Q = M.T @ P
+    assert np.allclose(res["P_bar"], P, atol=1e-10) and np.allclose(res["Q_bar"], Q, atol=1e-10)
+    assert np.allclose(res["G_hat"], P @ Q.T, atol=1e-10)
+    U, sv, Vt = np.linalg.svd(M)
+    best = (U[:, :r] * sv[:r]) @ Vt[:r]
+    err = [np.linalg.norm(orc.layer_round(G, E, Q0, 32, 32, 127.0, power_iters=T)["G_hat"] - best) for T in (1, 4, 16)]
+    assert err[0] > err[1] > err[2]
+    A, Bm = rng.integers(-3, 4, (n, r)).astype(np.float32), rng.integers(-3, 4, (m, r)).astype(np.float32)
+    low = (A @ Bm.T)[None]
+    for T in (1, 2, 5):
+        assert np.allclose(orc.layer_round(low, E, Q0, 32, 32, 127.0, power_iters=T)["G_hat"], low[0], atol=1e-9)
+    # one iteration is Algorithm 1 as it stands
+    one = orc.layer_round(G, E, Q0, 4, 4, 127.0)
+    assert np.array_equal(one["G_hat"], orc.layer_round(G, E, Q0, 4, 4, 127.0, power_iters=1)["G_hat"])
