@@ -108,6 +108,10 @@ typedef struct lqsgd_config {
   uint32_t flags;       /* LQSGD_FLAG_* */
   int32_t world_workers; /* 0, or the number of workers of ALL processes taking part in the averages when the
                             workers are spread over several GPUs (a multiple of `workers`); see lqsgd_round_begin */
+  int32_t power_iters;   /* 0 or 1: Algorithm 1 (one power step per round).  2..8 (an option): the power step with its
+                            two exchanges is repeated on the same M = G + E, each time from the Q_bar just obtained; the
+                            payload holds the streams of the last repetition (each repetition sends as much).  Needs a
+                            zero buffer of the largest matrix in the workspace; not with workers on several GPUs. */
 } lqsgd_config;
 
 /* Where one layer's data sits inside a worker's payload (byte offsets from the payload start). */

@@ -50,7 +50,7 @@ class Shape(C.Structure):
 class Config(C.Structure):
     _fields_ = [("struct_size", C.c_uint32), ("rank", C.c_int32), ("bits_p", C.c_int32),
                 ("bits_q", C.c_int32), ("alpha", C.c_float), ("workers", C.c_int32),
-                ("seed", C.c_uint64), ("flags", C.c_uint32), ("world_workers", C.c_int32)]
+                ("seed", C.c_uint64), ("flags", C.c_uint32), ("world_workers", C.c_int32), ("power_iters", C.c_int32)]
 
 
 class LayerLayout(C.Structure):
@@ -123,8 +123,8 @@ def _shapes(layers: Sequence[Tuple[int, int]]):
 
 
 def make_config(rank: int, bits_p: int, bits_q: int, alpha: float, workers: int, seed: int = 0,
-                flags: int = 0, world_workers: int = 0) -> Config:
-    return Config(C.sizeof(Config), rank, bits_p, bits_q, alpha, workers, seed, flags, world_workers)
+                flags: int = 0, world_workers: int = 0, power_iters: int = 0) -> Config:
+    return Config(C.sizeof(Config), rank, bits_p, bits_q, alpha, workers, seed, flags, world_workers, power_iters)
 
 
 def orthonormalize_noalloc(p_in: torch.Tensor, p_out: torch.Tensor, status: Optional[torch.Tensor] = None,
@@ -154,7 +154,7 @@ class LQSGD:
     def __init__(self, layers: Sequence[Tuple[int, int]], rank: int, bits_p: int, bits_q: Optional[int] = None,
                  alpha: float = 127.0, workers: int = 1, seed: int = 0, host_staging: bool = False,
                  device: str = "cuda:0", register_path: bool = False, world_workers: int = 0,
-                 average: str = "codes", quantize_vectors: bool = False):
+                 average: str = "codes", quantize_vectors: bool = False, power_iters: int = 1):
         self.lib = load_library()
         self.layers = [(int(n), int(m)) for n, m in layers]
         self.rank, self.bits_p = rank, bits_p
@@ -164,12 +164,13 @@ class LQSGD:
             raise ValueError("average must be 'codes' (Algorithm 1) or 'values'")
         self.average = average
         self.quantize_vectors = bool(quantize_vectors) and bits_p != 32
+        self.power_iters = max(1, int(power_iters))
         self.device = torch.device(device)
         self.cfg = make_config(rank, self.bits_p, self.bits_q, alpha, workers, seed,
                                (FLAG_HOST_STAGING if host_staging else 0)
                                | (FLAG_REGISTER_PATH if register_path else 0)
                                | (FLAG_AVERAGE_VALUES if average == "values" else 0)
-                               | (FLAG_QUANTIZE_VECTORS if quantize_vectors else 0), world_workers)
+                               | (FLAG_QUANTIZE_VECTORS if quantize_vectors else 0), world_workers, power_iters)
         nbytes = workspace_bytes(self.layers, self.cfg)
         with torch.cuda.device(self.device):
             self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)

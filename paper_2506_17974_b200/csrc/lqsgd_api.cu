@@ -88,6 +88,9 @@ struct Plan {
   float* d_xscales = nullptr;                 // [2][n_mat] scales the ranks agree on (split exchange)
   uint8_t* d_xsend[2] = {nullptr, nullptr};   // [W][region_bytes]: local P / Q streams, contiguous, for the all-gather
   uint64_t region_off[2] = {0, 0}, region_bytes[2] = {0, 0};
+  size_t zero_elems = 0;
+  float* d_zero = nullptr;                    // power_iters > 1: zeros, as large as the largest matrix
+  void** d_zero_ptrs = nullptr;               // [n_mat * W] pointers to d_zero: the "gradient" of a repeated power step
   float* d_stage_g = nullptr;                 // [W][elems_total]
   float* d_stage_ghat = nullptr;              // [elems_total]
   size_t state_begin = 0, state_end = 0;      // byte range to zero at create (E, factors, codes ...)
@@ -104,6 +107,8 @@ int check_config(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
   if (!bits_ok(c->bits_p) || !bits_ok(c->bits_q)) return LQSGD_ERR_INVALID_ARG;
   if (!(c->alpha > 0.f) || !std::isfinite(c->alpha)) return LQSGD_ERR_INVALID_ARG;
   if (c->workers < 1 || c->workers > 256) return LQSGD_ERR_INVALID_ARG;
+  if (c->power_iters < 0 || c->power_iters > 8) return LQSGD_ERR_INVALID_ARG;
+  if (c->power_iters > 1 && c->world_workers > c->workers) return LQSGD_ERR_INVALID_ARG;
   if (c->world_workers != 0) {     // workers of all ranks: a multiple of the local ones; no bypass mode across ranks
     if (c->world_workers < c->workers || c->world_workers > 4096 || c->world_workers % c->workers) return LQSGD_ERR_INVALID_ARG;
     if (c->world_workers > c->workers && (c->bits_p == 32 || c->bits_q == 32)) return LQSGD_ERR_INVALID_ARG;
@@ -449,6 +454,13 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   p.d_deqP = a.take<float>(p.deqP.size());
   p.d_deqQ = a.take<float>(p.deqQ.size());
   p.d_ptrs = a.take<void*>((p.mats.size() + p.vecs.size()) * (size_t)(W + 2));
+  if (cfg.power_iters > 1) {
+    size_t big = 0;
+    for (auto& mt : p.mats) big = std::max(big, (size_t)mt.n * mt.m);
+    p.zero_elems = big;
+    p.d_zero_ptrs = a.take<void*>(p.mats.size() * (size_t)W);
+    p.d_zero = a.take<float>(big);
+  }
   if (cfg.flags & LQSGD_FLAG_HOST_STAGING) {
     p.d_stage_g = a.take<float>((size_t)W * p.elems_total);
     p.d_stage_ghat = a.take<float>(p.elems_total);
@@ -587,6 +599,11 @@ int lqsgd_create(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
   CK(up(p.d_thrQ, p.thrQ.data(), p.thrQ.size() * sizeof(float)));
   CK(up(p.d_deqP, p.deqP.data(), p.deqP.size() * sizeof(float)));
   CK(up(p.d_deqQ, p.deqQ.data(), p.deqQ.size() * sizeof(float)));
+  if (p.d_zero) {
+    CK(cudaMemset(p.d_zero, 0, p.zero_elems * sizeof(float)));
+    std::vector<void*> zp(p.mats.size() * (size_t)p.W, p.d_zero);
+    CK(up(p.d_zero_ptrs, zp.data(), zp.size() * sizeof(void*)));
+  }
   // Q_0
   std::vector<float> q0;
   for (size_t li = 0; li < p.mats.size(); ++li) {
@@ -629,8 +646,11 @@ int lqsgd_launches_per_step(const lqsgd_ctx* ctx, int32_t* out) {
   if (!ctx || !out) return LQSGD_ERR_INVALID_ARG;
   const Plan& p = ctx->plan;
   // Orthonormalize (2), exchange of P, Q_w reduction, exchange of Q; then one launch per non-empty tile list
-  *out = (p.mats.empty() ? 0 : 5) + (p.tiles1.empty() ? 0 : 2) + (p.stiles1.empty() ? 0 : 2) + (p.tiles2.empty() ? 0 : 1) +
-         (p.tctiles2.empty() ? 0 : 1) + (p.tctiles1.empty() ? 0 : 1) + (p.tctiles3.empty() ? 0 : 1) + (p.chV.empty() ? 0 : 1);
+  const int pass1 = (p.tiles1.empty() ? 0 : 1) + (p.stiles1.empty() ? 0 : 1) + (p.tctiles1.empty() ? 0 : 1);
+  const int pass2 = (p.tiles2.empty() ? 0 : 1) + (p.tctiles2.empty() ? 0 : 1);
+  const int pass3 = (p.tiles3.empty() ? 0 : 1) + (p.stiles3.empty() ? 0 : 1) + (p.tctiles3.empty() ? 0 : 1);
+  const int iters = std::max(1, ctx->cfg.power_iters);
+  *out = iters * ((p.mats.empty() ? 0 : 5) + pass1 + pass2) + pass3 + (p.chV.empty() ? 0 : 1);
   return LQSGD_OK;
 }
 
@@ -707,9 +727,12 @@ static int prepare_step(lqsgd_ctx* c, const float* const* grads, float* const* g
 //   2: (split: sum over all ranks' streams + dequantise P) pass 2, Q_w (+ local scales of Q when split)
 //   3: exchange of Q, as segment 1
 //   4: (split: sum + dequantise Q)     5: pass 3
-static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, int n_streams, cudaStream_t st) {
+static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, int n_streams, cudaStream_t st,
+                       bool repeat = false) {
   Plan& p = c->plan;
-  const Tables& t = c->tables;
+  // a repeated power step (power_iters > 1) runs pass 1 on M itself: its "gradient" is the zero buffer
+  Tables t = c->tables;
+  if (repeat) t.grads = reinterpret_cast<const float* const*>(p.d_zero_ptrs);
   const int W = p.W, RP = p.RP;
   const size_t nm = p.mats.size(), nv = p.vecs.size();
   const size_t vbase = nm * (W + 2);
@@ -726,7 +749,7 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
 #define PHASE_MARK(i) do { if (ev) CK(cudaEventRecord(c->phase_events[i], st)); } while (0)
   switch (seg) {
     case 0:
-      if (nv) {
+      if (nv && !repeat) {
         if ((c->cfg.flags & LQSGD_FLAG_QUANTIZE_VECTORS) && c->cfg.bits_p != 32) {
           if (split) return LQSGD_ERR_INVALID_ARG;
           CK(launch_vectors_quant(p.d_vecs, (int)nv, reinterpret_cast<const float* const*>(p.d_ptrs + vbase),
@@ -740,8 +763,8 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
                           c->has_weights ? reinterpret_cast<float* const*>(p.d_ptrs + vbase + nv * (W + 1)) : nullptr,
                           t.lr, p.d_payload, p.payload_stride, W, p.W_total, {st, 0}));
       }
-      if (nm) CK(cudaMemsetAsync(p.d_status, 0, nm * sizeof(uint32_t), st));
-      PHASE_MARK(0);
+      if (nm && !repeat) CK(cudaMemsetAsync(p.d_status, 0, nm * sizeof(uint32_t), st));
+      if (!repeat) PHASE_MARK(0);
       if (nm) {
         CK(launch_pass1(RP, t, p.d_tiles1, (int)p.tiles1.size(), {st, c->grid1}));
         CK(launch_stream_pass1(RP, t, p.d_stiles1, (int)p.stiles1.size(), {st, (int)std::min<size_t>(p.stiles1.size(), c->sm_count)}));
@@ -798,10 +821,14 @@ static int step_impl(lqsgd_ctx* c, const float* const* grads, float* const* ghat
   if (rc != LQSGD_OK) return rc;
   if (c->plan.W_total != c->plan.W) return LQSGD_ERR_INVALID_ARG;   // workers elsewhere: use the lqsgd_round_* calls
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  for (int seg = 0; seg <= 5; ++seg) {
-    rc = run_segment(c, seg, false, nullptr, 0, st);
-    if (rc != LQSGD_OK) return rc;
-  }
+  const int iters = std::max(1, c->cfg.power_iters);
+  for (int it = 0; it < iters; ++it)
+    for (int seg = 0; seg <= 4; ++seg) {
+      rc = run_segment(c, seg, false, nullptr, 0, st, it > 0);
+      if (rc != LQSGD_OK) return rc;
+    }
+  rc = run_segment(c, 5, false, nullptr, 0, st);
+  if (rc != LQSGD_OK) return rc;
   c->have_events = false;
   return LQSGD_OK;
 }
@@ -822,7 +849,7 @@ int lqsgd_round_begin(lqsgd_ctx* c, const float* const* grads, float* const* gha
                       void* cuda_stream) {
   const int rc = prepare_step(c, grads, ghat, weights, lr, cuda_stream);
   if (rc != LQSGD_OK) return rc;
-  if (c->cfg.bits_p == 32 || c->cfg.bits_q == 32) return LQSGD_ERR_INVALID_ARG;
+  if (c->cfg.bits_p == 32 || c->cfg.bits_q == 32 || c->cfg.power_iters > 1) return LQSGD_ERR_INVALID_ARG;
   c->round_stage = 0;
   const int rs = run_segment(c, 0, true, nullptr, 0, static_cast<cudaStream_t>(cuda_stream));
   if (rs == LQSGD_OK) c->round_stage = 1;

@@ -30,7 +30,7 @@ def test_library_exports_every_declared_symbol(lib):
 
 
 def test_config_struct_matches_header_layout():
-    assert C.sizeof(B.Config) == 40 and C.sizeof(B.Shape) == 8 and C.sizeof(B.LayerLayout) == 64
+    assert C.sizeof(B.Config) == 48 and C.sizeof(B.Shape) == 8 and C.sizeof(B.LayerLayout) == 64
 
 
 def test_workspace_bytes_covers_the_persistent_state(lib):
@@ -49,7 +49,8 @@ def test_workspace_bytes_covers_the_persistent_state(lib):
     (dict(bits_p=1), B.ERR_INVALID_ARG), (dict(bits_q=9), B.ERR_INVALID_ARG),
     (dict(alpha=0.0), B.ERR_INVALID_ARG), (dict(alpha=float("nan")), B.ERR_INVALID_ARG),
     (dict(workers=0), B.ERR_INVALID_ARG), (dict(workers=257), B.ERR_INVALID_ARG),
-    (dict(flags=64), B.ERR_INVALID_ARG),
+    (dict(flags=64), B.ERR_INVALID_ARG), (dict(power_iters=9), B.ERR_INVALID_ARG), (dict(power_iters=-1), B.ERR_INVALID_ARG),
+    (dict(power_iters=2, world_workers=2), B.ERR_INVALID_ARG),
 ])
 def test_bad_config_is_rejected_on_the_host(lib, kw, code):
     base = dict(rank=2, bits_p=4, bits_q=4, alpha=127.0, workers=1, seed=0, flags=0)

@@ -182,6 +182,43 @@ def test_quantised_vectors_variant(bits, W, average):
     assert torch.allclose(wts[3], -0.5 * gh[3], rtol=0, atol=1e-7)
 
 
+@pytest.mark.parametrize("rank,T", [(3, 2), (3, 4), (16, 3)])
+def test_several_power_iterations(rank, T):
+    """power_iters = T: the power step and its exchanges repeated on the same M.  With the quantiser
+    bypassed the device follows the oracle's T-fold round to rounding; with it, the error-feedback
+    identity still holds and the result differs from one iteration's."""
+    w = wl.Workload("iters", ((96, 200), (130, 36), (64, 27), (20, 1)), rank=rank, bits=32, workers=2, steps=2,
+                    dist="student_t3", scale="fan_in", seed=21)
+    comp = make(w, power_iters=T)
+    Q0 = {l: par.host(comp.get_state(B.STATE_Q, l)) for l in range(3)}
+    oracle = orc.Oracle(w.layers, rank, 32, 32, w.alpha, 2, Q0, power_iters=T)
+    for t in range(2):
+        g = wl.draw_gradients(w, t, device=DEV)
+        ghat = [torch.empty_like(x) for x in g[0]]
+        comp.step(g, ghat)
+        torch.cuda.synchronize()
+        assert comp.status() == [0, 0, 0, 0]
+        out = oracle.step([[par.host(x) for x in per] for per in g])
+        for l in range(3):
+            assert par.rel_fro(par.host(ghat[l]), out[l]["G_hat"]) <= par.TOL, (t, l)
+            assert par.rel_fro(par.host(comp.get_state(B.STATE_Q, l)), out[l]["Q_bar"]) <= par.TOL, (t, l)
+            assert par.rel_fro(par.host(comp.get_state(B.STATE_E, l, 1)), out[l]["E_new"][1]) <= par.TOL, (t, l)
+    # quantised: E_new + G_hat = G + E_prev (Eq. 7, Eq. 8), and more iterations change the result
+    wq = dataclasses.replace(w, bits=6)
+    a, b = make(wq, power_iters=T), make(wq)
+    g = wl.draw_gradients(wq, 0, device=DEV)
+    oa = [torch.empty_like(x) for x in g[0]]
+    ob = [torch.empty_like(x) for x in g[0]]
+    a.step(g, oa)
+    b.step(g, ob)
+    torch.cuda.synchronize()
+    for l in range(3):
+        lhs = a.get_state(B.STATE_E, l, 0) + oa[l]
+        assert torch.allclose(lhs, g[0][l], rtol=0, atol=1e-6 * float(g[0][l].abs().max()))
+        assert not torch.equal(oa[l], ob[l])
+    assert a.launches_per_step > b.launches_per_step
+
+
 def test_different_bits_for_p_and_q():
     w = wl.Workload("bpq", ((96, 200), (48, 1)), rank=4, bits=3, workers=2, steps=2, dist="student_t3", scale="fan_in")
     comp = make(w, bits_p=3, bits_q=6)
