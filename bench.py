@@ -289,13 +289,16 @@ def run_ours(args):
         ms = start.elapsed_time(stop) / steps
         phases = [sum(events[t][i].elapsed_time(events[t][i + 1]) for t in range(psteps)) / psteps
                   for i in range(B.N_PHASES)]
+        per_step = sorted(events[t][0].elapsed_time(events[t][B.N_PHASES]) for t in range(psteps))
         status = comp.status()
         # a dependent column or a zero scale is a property of the data (it happens with 2-bit codes);
         # a non-finite value or an expired wait would make the timing meaningless
         assert all(s & (B.STATUS_NONFINITE | B.STATUS_TIMEOUT) == 0 for s in status), f"device status flags: {status}"
         out = {"ms": ms, "phases_ms": dict(zip(B.PHASE_NAMES, phases)), "launches": comp.launches_per_step,
                "payload": comp.payload_nbytes, "clocks": sampler.summary() if sampler else None, "graph_ms": graph_ms,
-               "flagged_layers": sum(1 for x in status if x)}
+               "flagged_layers": sum(1 for x in status if x),
+               "profiled_step_ms": {"min": per_step[0], "median": per_step[len(per_step) // 2], "max": per_step[-1],
+                                    "steps": psteps}}
         del comp
         if want_e2e:
             comp = B.LQSGD(wl_obj.layers, wl_obj.rank, wl_obj.bits, alpha=wl_obj.alpha, workers=wl_obj.workers,
@@ -380,7 +383,8 @@ def run_ours(args):
                      "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": recorded_traffic(args.workload, dom),
                      "bytes_per_launch": pb[dom], "kernel_ms": res["phases_ms"][dom]},
         "round": {"algorithmic_bytes": round_bytes, "achieved_gbs": round_bytes / (ms * 1e-3) / 1e9,
-                  "frac_of_peak": round_bytes / (ms * 1e-3) / 1e9 / peak, "phases_ms": res["phases_ms"]},
+                  "frac_of_peak": round_bytes / (ms * 1e-3) / 1e9 / peak, "phases_ms": res["phases_ms"],
+                  "profiled_step_ms": res["profiled_step_ms"]},
         "cuda_graph": {"ms_per_step": res["graph_ms"], "what": "one captured step replayed on one gradient set "
                        "(larger than L2); the timed `value` above uses plain launches"} if res.get("graph_ms") else None,
         "compression_ratio": 4 * sum(n * m for n, m in wl_obj.layers) / res["payload"],
