@@ -4,8 +4,10 @@
 //   pass 1: M = G + E (Eq. 8) written over E, partial P = M Q          (power step)
 //   pass 2: partial Q = M^T P_bar                                        (second power step)
 //   pass 3: G_hat = P_bar Q_bar^T (Eq. 6), E = M - G_hat (Eq. 7)
-// With r <= 16 the products are rank-r updates of a stream: a few FMAs per byte, on CUDA
-// cores with fp32 accumulation; the passes are bound by HBM, not by arithmetic.
+// The products are rank-r updates of a stream.  The kernels of this file do them on CUDA cores
+// with fp32 accumulation: a few FMAs per byte up to r = 8 (layers with 16-byte aligned rows then
+// run on the bulk-copy staged versions in lqsgd_stream.cu); above that the tensor-core passes of
+// lqsgd_tc.cu take the aligned layers and these kernels keep the rest.
 // Between the passes small kernels finish the factors: fixed-order reduction of the partial
 // sums, CholeskyQR in fp64 (Orthonormalize), scale, LogQuantize (Eq. 4 through a threshold
 // table), bit-packing, the exact integer worker sum, LogDequantize (Eq. 5 through a table).
@@ -919,7 +921,6 @@ sum_dequant_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __r
     float v = 0.f;
     if (s_ok) v = qt.avg_values ? s * (Sv / (float)n_streams) : s * __ldg(qt.deq + S + n_streams * (nlev - 1));
     const int row = e / r, col = e - row * r;
-    float* dst = which ? L.Q : L.Pbar;
     store_factor<RP>(L, which, row, col, v);
   }
   if (ch.chunk == 0 && tid == 0) {
@@ -1051,7 +1052,7 @@ vectors_quant_kernel(const VectorDev* __restrict__ vecs, const float* const* __r
 }  // namespace
 
 // ---------------------------------------------------------------------------------------
-// host launchers: dispatch on the padded rank RP in {1, 2, 4, 8, 16}
+// host launchers: dispatch on the padded rank RP in {1, 2, 4, 8, 16, 32}
 // ---------------------------------------------------------------------------------------
 #define LQSGD_DISPATCH_RP(RPV, ...)                 \
   switch (RPV) {                                    \

@@ -372,7 +372,7 @@ size_t smem_pass1(int RP, int NST) {
   const int nred = (RP >= 8 ? 4 : 8) * RP;
   return (size_t)NST * 2 * kSlab * 4 + 2 * kConsumerWarps * nred * 4 + (3 * NST + 2) * 8;
 }
-size_t smem_pass3(int RP, int NST) { return (size_t)NST * kSlab * 4 + (3 * NST + 2) * 8; }
+size_t smem_pass3(int /*RP*/, int NST) { return (size_t)NST * kSlab * 4 + (3 * NST + 2) * 8; }
 
 template <typename K>
 cudaError_t launch_staged(K kernel, size_t smem, const Tables& t, const Tile* tiles, int ntiles, Launch l) {
