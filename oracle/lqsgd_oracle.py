@@ -71,8 +71,17 @@ def level_values(bits, alpha):
 # ----------------------------------------------------------------------------
 # LogQuantize / LogDequantize (Alg. 1, quantise and dequantise lines; Section IV-A)
 # ----------------------------------------------------------------------------
-def factor_scale(factors):
-    """s = max over workers and entries of |x| (fp32 values, exact)."""
+def factor_scale(factors, per_column=False):
+    """s = max over workers and entries of |x| (fp32 values, exact).  per_column (a variant):
+    one scale per column of the factor, s_j = max over workers and rows of |x[:, j]|."""
+    if per_column:
+        cols = np.asarray(factors[0]).shape[1]
+        s = np.zeros(cols, dtype=np.float32)
+        for f in factors:
+            f32 = np.asarray(f, dtype=np.float32)
+            if f32.size:
+                s = np.maximum(s, np.max(np.abs(f32), axis=0))
+        return s.astype(np.float32)
     s = np.float32(0.0)
     for f in factors:
         f32 = np.asarray(f, dtype=np.float32)
@@ -91,12 +100,14 @@ def log_quantize(x, s, bits, alpha, return_margin=False):
     """
     L = magnitude_levels(bits)
     x32 = np.asarray(x, dtype=np.float32)
-    s32 = np.float32(s)
+    s32 = np.asarray(s, dtype=np.float32)                   # a scalar, or one scale per column
     neg = x32 < 0
-    if s32 == 0:
+    if s32.ndim == 0 and s32 == 0:
         v = np.zeros(x32.shape, dtype=np.float64)
     else:
-        t = (np.abs(x32) / s32).astype(np.float32)          # fp32 division
+        with np.errstate(divide="ignore", invalid="ignore"):
+            t = (np.abs(x32) / s32).astype(np.float32)      # fp32 division
+        t = np.where(np.broadcast_to(s32 == 0, x32.shape), np.float32(0), t)   # a zero scale: all codes 0
         v = (L - 1) * compand(t.astype(np.float64), alpha)  # in [0, L-1]
     k = np.floor(v + 0.5)
     k = np.clip(k, 0, L - 1).astype(np.uint8)
@@ -125,7 +136,7 @@ def average_dequantize(codes_per_worker, s, bits, alpha):
     for c in codes_per_worker:
         S += signed_levels(c, bits)
     q_bar = S.astype(np.float64) / (W * (L - 1))
-    return np.float64(np.float32(s)) * expand(q_bar, alpha)
+    return np.asarray(s, dtype=np.float32).astype(np.float64) * expand(q_bar, alpha)
 
 
 def dequantize_average(codes_per_worker, s, bits, alpha):
@@ -138,7 +149,7 @@ def dequantize_average(codes_per_worker, s, bits, alpha):
     total = np.zeros(np.asarray(codes_per_worker[0]).shape, dtype=np.float64)
     for c in codes_per_worker:                      # worker order
         q = signed_levels(c, bits).astype(np.float64) / (L - 1)
-        total += np.float64(np.float32(s)) * expand(q, alpha)
+        total += np.asarray(s, dtype=np.float32).astype(np.float64) * expand(q, alpha)
     return total / W
 
 
@@ -189,7 +200,7 @@ def orthonormalize(P):
 # ----------------------------------------------------------------------------
 # One factor exchange: scale, quantise, All-Reduce, dequantise
 # ----------------------------------------------------------------------------
-def exchange_factor(factors, bits, alpha, forced_codes=None, average="codes"):
+def exchange_factor(factors, bits, alpha, forced_codes=None, average="codes", column_scales=False):
     """Quantise every worker's factor, average, dequantise (Alg. 1, the three lines
     after each product).  bits == 32 bypasses the quantiser (plain PowerSGD mean).
 
@@ -204,7 +215,7 @@ def exchange_factor(factors, bits, alpha, forced_codes=None, average="codes"):
     if bits == 32:
         mean = sum(np.asarray(f, dtype=np.float64) for f in factors) / W
         return dict(scale=np.float32(0), codes=None, margin=None, mean=mean)
-    s = factor_scale(factors)
+    s = factor_scale(factors, per_column=column_scales)
     codes, margins = [], []
     for w, f in enumerate(factors):
         c, mg = log_quantize(f, s, bits, alpha, return_margin=True)
@@ -249,7 +260,8 @@ def effective_rank(rank, n, m):
     return min(rank, n, m)
 
 
-def layer_round(G, E, Q, bits_p, bits_q, alpha, forced_p=None, forced_q=None, average="codes", power_iters=1):
+def layer_round(G, E, Q, bits_p, bits_q, alpha, forced_p=None, forced_q=None, average="codes", power_iters=1,
+                column_scales=False):
     """One iteration of Algorithm 1 for one n x m layer and W workers.
 
     power_iters > 1 (an option, Algorithm 1 does one): the power step with its two exchanges is
@@ -270,10 +282,10 @@ def layer_round(G, E, Q, bits_p, bits_q, alpha, forced_p=None, forced_q=None, av
         P_raw = [power_step_p(M[w], Q) for w in range(W)]
         orth = [orthonormalize(P_raw[w]) for w in range(W)]
         P = [o[0] for o in orth]
-        xp = exchange_factor(P, bits_p, alpha, forced_p if last else None, average)
+        xp = exchange_factor(P, bits_p, alpha, forced_p if last else None, average, column_scales)
         P_bar = xp["mean"]
         Qw = [power_step_q(M[w], P_bar) for w in range(W)]
-        xq = exchange_factor(Qw, bits_q, alpha, forced_q if last else None, average)
+        xq = exchange_factor(Qw, bits_q, alpha, forced_q if last else None, average, column_scales)
         Q_bar = xq["mean"]
         Q = Q_bar
     G_hat = reconstruct(P_bar, Q_bar)
@@ -297,7 +309,7 @@ def factor_bits(n, m, rank, bits):
     return r * (n + m) * bits
 
 
-def payload_bytes(layers, rank, bits_p, bits_q, quantize_vectors=False):
+def payload_bytes(layers, rank, bits_p, bits_q, quantize_vectors=False, column_scales=False):
     """Bytes one worker sends per round: for each matrix the two code streams, each
     padded to a whole byte, plus the two fp32 scales; fp32 for every 1-D tensor, or, with
     quantize_vectors (the variant that log-quantises them too, b_p bits), one fp32 scale and
@@ -306,7 +318,7 @@ def payload_bytes(layers, rank, bits_p, bits_q, quantize_vectors=False):
     for n, m in layers:
         if n > 1 and m > 1:
             r = effective_rank(rank, n, m)
-            total += (r * n * bits_p + 7) // 8 + (r * m * bits_q + 7) // 8 + 8
+            total += (r * n * bits_p + 7) // 8 + (r * m * bits_q + 7) // 8 + (8 * r if column_scales else 8)
         elif quantize_vectors and bits_p != 32:
             total += 4 + (n * m * bits_p + 7) // 8
         else:
@@ -320,7 +332,9 @@ def assemble_payload(layers, rank, bits_p, bits_q, scales, codes_p, codes_q, vec
     scales: list of (s_P, s_Q); codes_*: per matrix uint8 code arrays; vectors: per 1-D tensor.
     With vector_scales (the variant that quantises the 1-D tensors): `vectors` holds their uint8
     codes, and the order is [matrix scales][one scale per 1-D tensor][their code streams][P][Q]."""
-    parts = [np.asarray([v for pair in scales for v in pair], dtype="<f4").view(np.uint8)]
+    # a matrix's scales: s_P then s_Q, each one value or (column-scale variant) r values
+    parts = [np.concatenate([np.atleast_1d(np.asarray(v, dtype="<f4")) for pair in scales for v in pair]).view(np.uint8)
+             if scales else np.zeros(0, np.uint8)]
     if vector_scales is not None:
         parts += [np.asarray(list(vector_scales), dtype="<f4").view(np.uint8)]
         parts += [pack_codes(c, bits_p) for c in vectors]
@@ -339,8 +353,9 @@ class Oracle:
     caller (drawn N(0,1) outside), Q_t = dequantised averaged Q of step t-1."""
 
     def __init__(self, layers, rank, bits_p, bits_q, alpha, workers, Q0, average="codes", quantize_vectors=False,
-                 power_iters=1):
+                 power_iters=1, column_scales=False):
         self.layers = [tuple(s) for s in layers]
+        self.column_scales = bool(column_scales)
         self.power_iters = int(power_iters)
         self.average = average
         self.quantize_vectors = bool(quantize_vectors) and bits_p != 32
@@ -364,7 +379,7 @@ class Oracle:
             if li in self.E:
                 f = (forced or {}).get(li, (None, None))
                 res = layer_round(Gl, self.E[li], self.Q[li], self.bits_p, self.bits_q,
-                                  self.alpha, f[0], f[1], self.average, self.power_iters)
+                                  self.alpha, f[0], f[1], self.average, self.power_iters, self.column_scales)
                 self.E[li] = res["E_new"]
                 self.Q[li] = res["Q_bar"]
             elif self.quantize_vectors:

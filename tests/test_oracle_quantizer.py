@@ -183,6 +183,31 @@ def test_value_domain_average_variant():
     assert np.array_equal(x["mean"], orc.dequantize_average(codes, s, bits, alpha))
 
 
+def test_column_scales_variant():
+    """One scale per column: every column is quantised exactly as if it were a factor of its own
+    with the scalar rule; a zero column gets scale 0 and codes 0; the levels of each column
+    round-trip with that column's scale."""
+    rng = np.random.default_rng(12)
+    bits, alpha, W = 4, 127.0, 3
+    fs = [(rng.standard_normal((40, 5)) * np.array([1.0, 10.0, 0.01, 0.0, 3.0])).astype(np.float32) for _ in range(W)]
+    s = orc.factor_scale(fs, per_column=True)
+    assert s.shape == (5,) and s.dtype == np.float32 and s[3] == 0
+    assert np.array_equal(s, np.array([orc.factor_scale([f[:, j:j + 1] for f in fs]) for j in range(5)], np.float32))
+    x = orc.exchange_factor(fs, bits, alpha, column_scales=True)
+    for j in range(5):
+        xj = orc.exchange_factor([f[:, j:j + 1] for f in fs], bits, alpha)
+        for w in range(W):
+            assert np.array_equal(x["codes"][w][:, j], xj["codes"][w][:, 0])
+        assert np.array_equal(x["mean"][:, j], xj["mean"][:, 0])
+    assert np.all(x["mean"][:, 3] == 0) and all(np.all(c[:, 3] == 0) for c in x["codes"])
+    lev = orc.level_values(4, 127.0)
+    one = np.stack([np.float32(2.0) * lev, np.float32(0.5) * lev[::-1]], axis=1).astype(np.float32)
+    y = orc.exchange_factor([one], 4, 127.0, column_scales=True)
+    assert np.array_equal(y["scale"], np.array([2.0, 0.5], np.float32))
+    assert np.allclose(y["mean"], one.astype(np.float64), rtol=1e-6, atol=0)
+    assert orc.payload_bytes(((6, 5), (1, 9)), 2, 4, 4, column_scales=True) == 6 + 5 + 16 + 36
+
+
 @pytest.mark.parametrize("bits", [2, 3, 4, 5, 8])
 def test_pack_layout_and_size(bits):
     rng = np.random.default_rng(bits)
