@@ -87,6 +87,13 @@ typedef enum lqsgd_error {
                                          travelling as fp32.  Payload: [s_P, s_Q per matrix][one scale per 1-D tensor]
                                          [their code streams][P streams][Q streams].  Ignored with bits_p = 32; not
                                          available with workers on several GPUs (lqsgd_round_begin refuses). */
+#define LQSGD_FLAG_COLUMN_SCALES 16u /* variant: one scale per COLUMN of a factor, s_j = max over workers and rows of
+                                        |x[:, j]|, instead of one per factor; column j is normalised by s_j in Eq. 4 and
+                                        rescaled by s_j after Eq. 5.  A matrix then sends 2 r_eff scales: in the payload
+                                        s_P[0..r_eff) is followed by s_Q[0..r_eff) (8 r_eff bytes at scale_offset), and
+                                        LQSGD_STATE_SCALES is fp32 [2][r_eff].  The zero-scale status bits are set when
+                                        any column's scale is 0 (that column's codes and averages are 0).  Not available
+                                        with workers on several GPUs (lqsgd_round_begin refuses). */
 
 typedef struct lqsgd_ctx lqsgd_ctx;
 
@@ -118,7 +125,8 @@ typedef struct lqsgd_config {
 typedef struct lqsgd_layer_layout {
   int32_t is_matrix;     /* 1: low-rank path, 0: one-dimensional tensor sent as fp32 */
   int32_t rank_eff;      /* r_eff (0 for a 1-D tensor) */
-  uint64_t scale_offset; /* matrix: fp32 s_P then fp32 s_Q; quantised 1-D tensor: its fp32 scale */
+  uint64_t scale_offset; /* matrix: fp32 s_P then fp32 s_Q (LQSGD_FLAG_COLUMN_SCALES: r_eff values each);
+                            quantised 1-D tensor: its fp32 scale */
   uint64_t p_offset;     /* matrix: P code stream, p_bytes = ceil(n * r_eff * b_p / 8) */
   uint64_t p_bytes;
   uint64_t q_offset;     /* matrix: Q code stream, q_bytes = ceil(m * r_eff * b_q / 8) */
@@ -138,7 +146,7 @@ typedef enum lqsgd_state {
   LQSGD_STATE_Q_W = 5,     /* fp32 m x r_eff, per worker: M^T P_bar of the last step */
   LQSGD_STATE_CODES_P = 6, /* uint8 n x r_eff, per worker: one unpacked code per byte (not with bits 32) */
   LQSGD_STATE_CODES_Q = 7, /* uint8 m x r_eff, per worker */
-  LQSGD_STATE_SCALES = 8   /* fp32 [2]: s_P, s_Q of the last step */
+  LQSGD_STATE_SCALES = 8   /* fp32 [2]: s_P, s_Q of the last step (LQSGD_FLAG_COLUMN_SCALES: fp32 [2][r_eff]) */
 } lqsgd_state;
 
 /* Bytes of device workspace a context for these layers needs (Algorithm 1 state E, Q, plus
@@ -228,7 +236,8 @@ int lqsgd_step_host(lqsgd_ctx* ctx, const float* const* host_grads, float* const
                     void* host_payload, void* cuda_stream);
 
 /* Size of one worker's payload in bytes (Section IV-C: r(n+m)b bits per matrix, each code
- * stream padded to a byte, + 8 bytes of scales per matrix + 4 bytes per 1-D scalar). */
+ * stream padded to a byte, + 8 bytes of scales per matrix (8 r_eff with LQSGD_FLAG_COLUMN_SCALES)
+ * + 4 bytes per 1-D scalar). */
 int lqsgd_payload_bytes(const lqsgd_ctx* ctx, size_t* host_bytes_out);
 
 /* Device view of what worker `worker` sends in the last enqueued step: valid until the next

@@ -23,6 +23,7 @@ FLAG_HOST_STAGING = 1
 FLAG_REGISTER_PATH = 2
 FLAG_AVERAGE_VALUES = 4
 FLAG_QUANTIZE_VECTORS = 8
+FLAG_COLUMN_SCALES = 16
 STATUS_TIMEOUT = 16
 N_PHASES = 5
 XCHG_SCALES_P, XCHG_SCALES_Q, XCHG_STREAMS_P, XCHG_STREAMS_Q = range(4)
@@ -154,7 +155,8 @@ class LQSGD:
     def __init__(self, layers: Sequence[Tuple[int, int]], rank: int, bits_p: int, bits_q: Optional[int] = None,
                  alpha: float = 127.0, workers: int = 1, seed: int = 0, host_staging: bool = False,
                  device: str = "cuda:0", register_path: bool = False, world_workers: int = 0,
-                 average: str = "codes", quantize_vectors: bool = False, power_iters: int = 1):
+                 average: str = "codes", quantize_vectors: bool = False, power_iters: int = 1,
+                 column_scales: bool = False):
         self.lib = load_library()
         self.layers = [(int(n), int(m)) for n, m in layers]
         self.rank, self.bits_p = rank, bits_p
@@ -165,12 +167,14 @@ class LQSGD:
         self.average = average
         self.quantize_vectors = bool(quantize_vectors) and bits_p != 32
         self.power_iters = max(1, int(power_iters))
+        self.column_scales = bool(column_scales)
         self.device = torch.device(device)
         self.cfg = make_config(rank, self.bits_p, self.bits_q, alpha, workers, seed,
                                (FLAG_HOST_STAGING if host_staging else 0)
                                | (FLAG_REGISTER_PATH if register_path else 0)
                                | (FLAG_AVERAGE_VALUES if average == "values" else 0)
-                               | (FLAG_QUANTIZE_VECTORS if quantize_vectors else 0), world_workers, power_iters)
+                               | (FLAG_QUANTIZE_VECTORS if quantize_vectors else 0)
+                               | (FLAG_COLUMN_SCALES if column_scales else 0), world_workers, power_iters)
         nbytes = workspace_bytes(self.layers, self.cfg)
         with torch.cuda.device(self.device):
             self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
@@ -320,7 +324,7 @@ class LQSGD:
                 STATE_P_RAW: ((n, r), torch.float32), STATE_P: ((n, r), torch.float32),
                 STATE_P_BAR: ((n, r), torch.float32), STATE_Q_W: ((m, r), torch.float32),
                 STATE_CODES_P: ((n, r), torch.uint8), STATE_CODES_Q: ((m, r), torch.uint8),
-                STATE_SCALES: ((2,), torch.float32)}[which]
+                STATE_SCALES: (((2, r) if self.column_scales else (2,)), torch.float32)}[which]
 
     def get_state(self, which: int, layer: int, worker: int = 0) -> torch.Tensor:
         shape, dt = self._state_shape(which, layer)

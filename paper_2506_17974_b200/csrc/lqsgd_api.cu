@@ -114,7 +114,7 @@ int check_config(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
     if (c->world_workers > c->workers && (c->bits_p == 32 || c->bits_q == 32)) return LQSGD_ERR_INVALID_ARG;
   }
   if (c->flags & ~(LQSGD_FLAG_HOST_STAGING | LQSGD_FLAG_REGISTER_PATH | LQSGD_FLAG_AVERAGE_VALUES |
-                   LQSGD_FLAG_QUANTIZE_VECTORS))
+                   LQSGD_FLAG_QUANTIZE_VECTORS | LQSGD_FLAG_COLUMN_SCALES))
     return LQSGD_ERR_INVALID_ARG;
   for (int i = 0; i < n_layers; ++i) {
     if (shapes[i].rows < 1 || shapes[i].cols < 1) return LQSGD_ERR_BAD_SHAPE;
@@ -175,7 +175,8 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   }
   // ---- payload layout: [scales][1-D fp32][P streams][Q streams]
   size_t off = 0;
-  for (auto& mt : p.mats) { p.layout[mt.user_index].scale_offset = off; off += 8; }
+  const bool colscales = (cfg.flags & LQSGD_FLAG_COLUMN_SCALES) != 0;   // s_P[r] then s_Q[r] instead of s_P, s_Q
+  for (auto& mt : p.mats) { p.layout[mt.user_index].scale_offset = off; off += colscales ? 8 * (size_t)mt.r : 8; }
   const bool qvec = (cfg.flags & LQSGD_FLAG_QUANTIZE_VECTORS) && cfg.bits_p != 32;
   if (qvec)
     for (auto& v : p.vecs) { v.pay_scale_off = off; p.layout[v.user_index].scale_offset = off; off += 4; }
@@ -326,9 +327,9 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
     L.Qpart = a.take<float>((size_t)W * L.nrb * mt.m * RP);
     L.Qw = (L.nrb == 1) ? L.Qpart : a.take<float>((size_t)W * mt.m * RP);
     L.gram_part = a.take<double>((size_t)W * L.npb * RP * RP);
-    L.maxp = a.take<float>((size_t)W * L.npb);
-    L.maxq = a.take<float>((size_t)W * L.nqb);
-    L.scales = a.take<float>(2);
+    L.maxp = a.take<float>((size_t)W * L.npb * (colscales ? RP : 1));
+    L.maxq = a.take<float>((size_t)W * L.nqb * (colscales ? RP : 1));
+    L.scales = a.take<float>(2 * (size_t)RP);
     const auto& lo = p.layout[mt.user_index];
     L.pay_scale_off = lo.scale_offset; L.pay_p_off = lo.p_offset; L.pay_q_off = lo.q_offset;
 
@@ -717,6 +718,7 @@ static int prepare_step(lqsgd_ctx* c, const float* const* grads, float* const* g
   t.payload_stride = p.payload_stride;
   t.status = p.d_status;
   t.W = W;
+  t.col_scales = (c->cfg.flags & LQSGD_FLAG_COLUMN_SCALES) ? 1 : 0;
   c->has_weights = weights != nullptr;
   return LQSGD_OK;
 }
@@ -850,6 +852,7 @@ int lqsgd_round_begin(lqsgd_ctx* c, const float* const* grads, float* const* gha
   const int rc = prepare_step(c, grads, ghat, weights, lr, cuda_stream);
   if (rc != LQSGD_OK) return rc;
   if (c->cfg.bits_p == 32 || c->cfg.bits_q == 32 || c->cfg.power_iters > 1) return LQSGD_ERR_INVALID_ARG;
+  if (c->cfg.flags & LQSGD_FLAG_COLUMN_SCALES) return LQSGD_ERR_INVALID_ARG;   // the ranks agree on one scale per factor
   c->round_stage = 0;
   const int rs = run_segment(c, 0, true, nullptr, 0, static_cast<cudaStream_t>(cuda_stream));
   if (rs == LQSGD_OK) c->round_stage = 1;
@@ -974,7 +977,11 @@ static int locate_state(const lqsgd_ctx* c, int which, int layer, int worker, ch
     // codes are not kept unpacked: base = the worker's packed stream, rows = number of codes (see lqsgd_get_state)
     case LQSGD_STATE_CODES_P: if (c->cfg.bits_p == 32) return LQSGD_ERR_OUT_OF_RANGE; *base = (char*)(p.d_payload + w * p.payload_stride + L.pay_p_off); *rows = n * r; *row_bytes = *pitch = 1; break;
     case LQSGD_STATE_CODES_Q: if (c->cfg.bits_q == 32) return LQSGD_ERR_OUT_OF_RANGE; *base = (char*)(p.d_payload + w * p.payload_stride + L.pay_q_off); *rows = m * r; *row_bytes = *pitch = 1; break;
-    case LQSGD_STATE_SCALES: *base = (char*)L.scales; *rows = 1; *row_bytes = *pitch = 8; break;
+    case LQSGD_STATE_SCALES:
+      *base = (char*)L.scales;
+      if (c->cfg.flags & LQSGD_FLAG_COLUMN_SCALES) { *rows = 2; *row_bytes = 4 * r; *pitch = 4 * RP; }
+      else { *rows = 1; *row_bytes = *pitch = 8; }
+      break;
     default: return LQSGD_ERR_OUT_OF_RANGE;
   }
   return LQSGD_OK;

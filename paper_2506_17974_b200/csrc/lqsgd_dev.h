@@ -39,9 +39,9 @@ struct LayerDev {
   float* Qpart;               // [W][nrb][m][RP]
   float* Qw;                  // [W][m][RP]  (== Qpart when nrb == 1)
   double* gram_part;          // [W][npb][RP*RP]
-  float* maxp;                // [W][npb]
-  float* maxq;                // [W][nqb]
-  float* scales;              // [2]  s_P, s_Q
+  float* maxp;                // [W][npb] block maxima of |P|; with column scales [W][npb][RP], one per column
+  float* maxq;                // [W][nqb] (or [W][nqb][RP])
+  float* scales;              // [2 RP]: s_P at [0], s_Q at [1]; with column scales s_P[j] at [j], s_Q[j] at [RP + j]
   uint64_t pay_scale_off, pay_p_off, pay_q_off;   // byte offsets inside one worker's payload
 };
 
@@ -83,6 +83,7 @@ struct Tables {
   uint64_t payload_stride;
   uint32_t* status;           // [n_mat]
   int32_t W;
+  int32_t col_scales;         // 1: one quantiser scale per factor column (variant), 0: one per factor
 };
 
 struct QuantTables {

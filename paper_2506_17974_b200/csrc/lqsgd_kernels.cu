@@ -472,7 +472,20 @@ p_reduce_gram_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
     for (int j = 0; j < RP; ++j) p[j] = 0.f;
     if (row < n) {
       const float* src = L.Ppart + ((size_t)fb.worker * L.ncc * n + row) * RP;
-      for (int cc = 0; cc < L.ncc; ++cc) {
+      // the partials' loads go out together (4 at a time); the additions keep the chunk order
+      int cc = 0;
+      if constexpr (RP <= 8) {
+        for (; cc + 4 <= L.ncc; cc += 4) {
+          float v[4][RP];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) load_contig_ro<RP>(src + (size_t)(cc + u) * n * RP, v[u]);
+#pragma unroll
+          for (int u = 0; u < 4; ++u)
+#pragma unroll
+            for (int j = 0; j < RP; ++j) p[j] += v[u][j];
+        }
+      }
+      for (; cc < L.ncc; ++cc) {
         float v[RP];
         load_contig_ro<RP>(src + (size_t)cc * n * RP, v);
 #pragma unroll
@@ -508,7 +521,15 @@ __device__ __forceinline__ bool cholesky_lower(const LayerDev& L, int worker, do
   for (int e = tid; e < RP * RP; e += nt) {
     const double* gp = L.gram_part + (size_t)worker * L.npb * (RP * RP) + e;
     double s = 0.0;
-    for (int b = 0; b < L.npb; ++b) s += gp[(size_t)b * (RP * RP)];
+    int b = 0;
+    for (; b + 8 <= L.npb; b += 8) {        // eight loads in flight, additions in block order
+      double x[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) x[u] = gp[(size_t)(b + u) * (RP * RP)];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) s += x[u];
+    }
+    for (; b < L.npb; ++b) s += gp[(size_t)b * (RP * RP)];
     A[e / RP][e % RP] = s;
   }
   __syncthreads();
@@ -566,6 +587,7 @@ p_apply_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
   __shared__ double invd[RP];
   __shared__ int dead[RP];
   __shared__ float smax[4];
+  __shared__ float scol[4][RP];
   const FactorBlock fb = fbs[blockIdx.x];
   const LayerDev& L = t.layers[fb.layer];
   const int n = L.n, tid = threadIdx.x;
@@ -573,13 +595,15 @@ p_apply_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
   if (dropped && fb.blk == 0 && tid == 0) atomicOr(&t.status[fb.layer], 1u);
   const int row = fb.blk * kFactorBlockRows + tid;
   float amax = 0.f;
+  float o[RP];
+#pragma unroll
+  for (int j = 0; j < RP; ++j) o[j] = 0.f;
   if (row < n) {
     // the row of P solves  o R = p  with R = L^T upper triangular: forward substitution in fp64,
     //   o[j] = (p[j] - sum_{k<j} o[k] L[j][k]) / L[j][j];   a dropped column gives 0
     float p[RP];
     load_contig_ro<RP>(L.Praw + ((size_t)fb.worker * n + row) * RP, p);
     double od[RP];
-    float o[RP];
     bool bad = false;
 #pragma unroll
     for (int j = 0; j < RP; ++j) {
@@ -594,43 +618,106 @@ p_apply_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
     store_contig<RP>(L.P + ((size_t)fb.worker * n + row) * RP, o);
     if (bad) atomicOr(&t.status[fb.layer], 8u);
   }
+  if (t.col_scales) {            // variant: one maximum per column
+#pragma unroll
+    for (int j = 0; j < RP; ++j) {
+      float v = fabsf(o[j]);
+#pragma unroll
+      for (int off = 16; off >= 1; off >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, off));
+      if ((tid & 31) == 0) scol[tid >> 5][j] = v;
+    }
+    __syncthreads();
+    if (tid < RP)
+      L.maxp[((size_t)fb.worker * L.npb + fb.blk) * RP + tid] =
+          fmaxf(fmaxf(scol[0][tid], scol[1][tid]), fmaxf(scol[2][tid], scol[3][tid]));
+    return;
+  }
   amax = block_max_128(amax, smax);
   if (tid == 0) L.maxp[(size_t)fb.worker * L.npb + fb.blk] = amax;
 }
 
-// Q_w = sum of the row-chunk partials of pass 2, in chunk order; block max |Q_w|.
+// Q_w = sum of the row-chunk partials of pass 2, in chunk order; block max |Q_w|.  A thread owns
+// V = min(RP, 4) consecutive columns of a row (one 128-bit load per partial when RP >= 4) and the
+// loads of several partials are in flight together: the chain of nrb dependent additions, not a
+// chain of nrb memory latencies, is what a row costs.
+constexpr int kQReduceThreads = 256;
 template <int RP>
-__global__ void __launch_bounds__(kFactorBlockRows)
+__global__ void __launch_bounds__(kQReduceThreads)
 q_reduce_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
   pdl_wait();
-  __shared__ float smax[4];
+  constexpr int V = RP < 4 ? RP : 4;        // floats per thread item
+  constexpr int TPR = RP / V;               // items per row: 1, 2, 4 or 8 (divides 256 and 32)
+  __shared__ float smax[kQReduceThreads / 32][TPR * V];
   const FactorBlock fb = fbs[blockIdx.x];
   const LayerDev& L = t.layers[fb.layer];
-  const int m = L.m, tid = threadIdx.x;
-  const int row = fb.blk * kFactorBlockRows + tid;
-  float amax = 0.f;
-  if (row < m) {
-    float q[RP];
+  const int m = L.m, tid = threadIdx.x, nrb = L.nrb;
+  const size_t plane = (size_t)m * RP;      // floats of one partial
+  float cmax[V];
 #pragma unroll
-    for (int j = 0; j < RP; ++j) q[j] = 0.f;
-    const float* src = L.Qpart + ((size_t)fb.worker * L.nrb * m + row) * RP;
-    for (int rb = 0; rb < L.nrb; ++rb) {
-      float v[RP];
-      load_contig_ro<RP>(src + (size_t)rb * m * RP, v);
+  for (int v = 0; v < V; ++v) cmax[v] = 0.f;
+  bool bad = false;
+  for (int item = tid; item < kFactorBlockRows * TPR; item += kQReduceThreads) {
+    const int row = fb.blk * kFactorBlockRows + item / TPR;
+    if (row >= m) break;
+    const size_t off = (size_t)row * RP + (size_t)(item % TPR) * V;
+    const float* src = L.Qpart + (size_t)fb.worker * nrb * plane + off;
+    float q[V];
 #pragma unroll
-      for (int j = 0; j < RP; ++j) q[j] += v[j];
+    for (int v = 0; v < V; ++v) q[v] = 0.f;
+    int rb = 0;
+    for (; rb + 8 <= nrb; rb += 8) {
+      float x[8][V];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) load_contig_ro<V>(src + (size_t)(rb + u) * plane, x[u]);
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+#pragma unroll
+        for (int v = 0; v < V; ++v) q[v] += x[u][v];
     }
-    if (L.nrb > 1) store_contig<RP>(L.Qw + ((size_t)fb.worker * m + row) * RP, q);
-    bool bad = false;
+    for (; rb < nrb; ++rb) {
+      float x[V];
+      load_contig_ro<V>(src + (size_t)rb * plane, x);
 #pragma unroll
-    for (int j = 0; j < RP; ++j) {
-      amax = fmaxf(amax, fabsf(q[j]));
-      bad |= !(fabsf(q[j]) < INFINITY);
+      for (int v = 0; v < V; ++v) q[v] += x[v];
     }
-    if (bad) atomicOr(&t.status[fb.layer], 8u);
+    if (nrb > 1) store_contig<V>(L.Qw + (size_t)fb.worker * plane + off, q);
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+      cmax[v] = fmaxf(cmax[v], fabsf(q[v]));
+      bad |= !(fabsf(q[v]) < INFINITY);
+    }
   }
-  amax = block_max_128(amax, smax);
-  if (tid == 0) L.maxq[(size_t)fb.worker * L.nqb + fb.blk] = amax;
+  if (bad) atomicOr(&t.status[fb.layer], 8u);
+  // maxima: the columns a thread owns are fixed (256 and 32 are multiples of TPR): columns (tid % TPR) V + v
+  const int warp = tid >> 5, lane = tid & 31;
+  if (t.col_scales) {
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+#pragma unroll
+      for (int o = 16; o >= TPR; o >>= 1) cmax[v] = fmaxf(cmax[v], __shfl_xor_sync(0xffffffffu, cmax[v], o));
+      if (lane < TPR) smax[warp][lane * V + v] = cmax[v];
+    }
+    __syncthreads();
+    if (tid < RP) {
+      float a = smax[0][tid];
+#pragma unroll
+      for (int w = 1; w < kQReduceThreads / 32; ++w) a = fmaxf(a, smax[w][tid]);
+      L.maxq[((size_t)fb.worker * L.nqb + fb.blk) * RP + tid] = a;
+    }
+    return;
+  }
+  float amax = cmax[0];
+#pragma unroll
+  for (int v = 1; v < V; ++v) amax = fmaxf(amax, cmax[v]);
+#pragma unroll
+  for (int o = 16; o >= 1; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+  if (lane == 0) smax[warp][0] = amax;
+  __syncthreads();
+  if (tid == 0) {
+#pragma unroll
+    for (int w = 1; w < kQReduceThreads / 32; ++w) amax = fmaxf(amax, smax[w][0]);
+    L.maxq[(size_t)fb.worker * L.nqb + fb.blk] = amax;
+  }
 }
 
 // One element of an averaged factor (P_bar or Q_bar) goes to its row-major home and to the
@@ -690,6 +777,8 @@ exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __rest
   __shared__ float thr[128];
   __shared__ __align__(4) uint8_t codes[WB][CH + 4];
   __shared__ float sred[8];
+  __shared__ float scol8[8][RP];
+  __shared__ float scol[RP];
   const ExchangeChunk ch = chunks[blockIdx.x];
   const LayerDev& L = t.layers[ch.layer];
   const int W = t.W, tid = threadIdx.x;
@@ -703,16 +792,43 @@ exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __rest
   for (int i = tid; i < NLEV - 1; i += 256) thr[i] = qt.thr[i];
   if (tid < WB) *reinterpret_cast<uint32_t*>(&codes[tid][CH]) = 0u;     // what a word task reads past the chunk
   float s = 0.f;
-  for (int i = tid; i < W * nblk; i += 256) s = fmaxf(s, __ldg(maxes + i));
+  const bool cs = t.col_scales != 0;
+  if (cs) {
+    // variant: one scale per column.  Block maxima are [W][nblk][RP]; thread tid only meets column tid % RP.
+    for (int i = tid; i < W * nblk * RP; i += 256) s = fmaxf(s, __ldg(maxes + i));
 #pragma unroll
-  for (int o = 16; o >= 1; o >>= 1) s = fmaxf(s, __shfl_xor_sync(0xffffffffu, s, o));
-  if ((tid & 31) == 0) sred[tid >> 5] = s;
-  __syncthreads();
-  s = sred[0];
+    for (int o = 16; o >= RP; o >>= 1) s = fmaxf(s, __shfl_xor_sync(0xffffffffu, s, o));
+    if ((tid & 31) < RP) scol8[tid >> 5][tid & 31] = s;
+    __syncthreads();
+    if (tid < RP) {
+      float a = scol8[0][tid];
 #pragma unroll
-  for (int i = 1; i < 8; ++i) s = fmaxf(s, sred[i]);
-  if (sx.pack_only) s = sx.scales[which * sx.n_mat + ch.layer];   // scale agreed between the ranks
-  const bool s_ok = (s > 0.f) && (s < INFINITY);
+      for (int i = 1; i < 8; ++i) a = fmaxf(a, scol8[i][tid]);
+      scol[tid] = a;
+    }
+    __syncthreads();
+  } else {
+    for (int i = tid; i < W * nblk; i += 256) s = fmaxf(s, __ldg(maxes + i));
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) s = fmaxf(s, __shfl_xor_sync(0xffffffffu, s, o));
+    if ((tid & 31) == 0) sred[tid >> 5] = s;
+    __syncthreads();
+    s = sred[0];
+#pragma unroll
+    for (int i = 1; i < 8; ++i) s = fmaxf(s, sred[i]);
+    if (sx.pack_only) s = sx.scales[which * sx.n_mat + ch.layer];   // scale agreed between the ranks
+  }
+  // scales, status: once per layer
+  if (ch.chunk == 0 && (cs ? tid < r : tid == 0)) {
+    const float sj = cs ? scol[tid] : s;
+    L.scales[cs ? which * RP + tid : which] = sj;
+    for (int w = 0; w < W; ++w) {
+      float* ps = reinterpret_cast<float*>(t.payload + (size_t)w * t.payload_stride + L.pay_scale_off);
+      ps[cs ? which * r + tid : which] = sj;
+    }
+    if (B != 32 && !(sj > 0.f)) atomicOr(&t.status[ch.layer], which ? 4u : 2u);
+    if (!(sj < INFINITY)) atomicOr(&t.status[ch.layer], 8u);
+  }
 
   if constexpr (B == 32) {
     // Quantiser bypassed (plain PowerSGD exchange): the factor travels as fp32 and the workers'
@@ -730,14 +846,6 @@ exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __rest
       }
       store_factor<RP>(L, which, row, col, sum / (float)W);
     }
-    if (ch.chunk == 0 && tid == 0) {
-      L.scales[which] = s;
-      for (int w = 0; w < W; ++w) {
-        float* ps = reinterpret_cast<float*>(t.payload + (size_t)w * t.payload_stride + L.pay_scale_off);
-        ps[which] = s;
-      }
-      if (!(s < INFINITY)) atomicOr(&t.status[ch.layer], 8u);
-    }
     return;
   } else {
     constexpr int NW = CH * B / 32;      // 32-bit words of one worker's stream in this chunk
@@ -746,6 +854,8 @@ exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __rest
     const bool valid = tid < cnt;
     const int e = e0 + tid;
     const int row = valid ? e / r : 0, col = valid ? e % r : 0;
+    if (cs) s = scol[col];
+    const bool s_ok = (s > 0.f) && (s < INFINITY);
     const size_t nbytes_total = ((size_t)count * B + 7) / 8;
     const size_t byte0 = (size_t)ch.chunk * (CH / 8) * B;
     const int nbytes = (int)min((size_t)(CH / 8) * B, nbytes_total - byte0);
@@ -814,15 +924,6 @@ exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __rest
       float v = 0.f;
       if (s_ok) v = qt.avg_values ? s * (Sv / (float)W) : s * __ldg(qt.deq + S + W * (NLEV - 1));
       store_factor<RP>(L, which, row, col, v);
-    }
-    if (ch.chunk == 0 && tid == 0) {
-      L.scales[which] = s;
-      for (int w = 0; w < W; ++w) {
-        float* ps = reinterpret_cast<float*>(t.payload + (size_t)w * t.payload_stride + L.pay_scale_off);
-        ps[which] = s;
-      }
-      if (!(s > 0.f)) atomicOr(&t.status[ch.layer], which ? 4u : 2u);
-      if (!(s < INFINITY)) atomicOr(&t.status[ch.layer], 8u);
     }
   }
 }
@@ -1103,7 +1204,7 @@ cudaError_t launch_p_apply(int rp, const Tables& t, const FactorBlock* fb, int n
 
 cudaError_t launch_q_reduce(int rp, const Tables& t, const FactorBlock* fb, int nfb, Launch l) {
   if (nfb == 0) return cudaSuccess;
-  LQSGD_DISPATCH_RP(rp, (launch_pdl(q_reduce_kernel<RP>, nfb, kFactorBlockRows, 0, l.stream, t, fb)));
+  LQSGD_DISPATCH_RP(rp, (launch_pdl(q_reduce_kernel<RP>, nfb, kQReduceThreads, 0, l.stream, t, fb)));
   return cudaGetLastError();
 }
 

@@ -58,10 +58,10 @@ def snapshot_state(comp: B.LQSGD):
     return E, Q
 
 
-def check_exchange(x_dev, codes_dev, scale_dev, bar_dev, bits, alpha, stats, average="codes"):
-    """Scale, codes and dequantised mean of one factor against the oracle, on the device's factor."""
-    s = orc.factor_scale(list(x_dev))
-    assert np.float32(scale_dev) == s, (scale_dev, s)
+def check_exchange(x_dev, codes_dev, scale_dev, bar_dev, bits, alpha, stats, average="codes", column_scales=False):
+    """Scale(s), codes and dequantised mean of one factor against the oracle, on the device's factor."""
+    s = orc.factor_scale(list(x_dev), per_column=column_scales)
+    assert np.array_equal(np.asarray(scale_dev, dtype=np.float32), s), (scale_dev, s)
     flips = 0
     total = 0
     for w in range(len(x_dev)):
@@ -91,9 +91,10 @@ def check_layer_stage_isolated(comp: B.LQSGD, layer: int, G, rec: StepRecord, st
     errs["P_raw"] = max(rel_fro(rec.P_raw[w], orc.power_step_p(M[w], rec.Q_prev)) for w in range(W))
     orth = [orc.orthonormalize(rec.P_raw[w]) for w in range(W)]
     errs["P"] = max(rel_fro(rec.P[w], orth[w][0]) for w in range(W))
-    check_exchange(rec.P, rec.codes_p, rec.scales[0], rec.P_bar, comp.bits_p, comp.alpha, stats, comp.average)
+    cs = comp.column_scales
+    check_exchange(rec.P, rec.codes_p, rec.scales[0], rec.P_bar, comp.bits_p, comp.alpha, stats, comp.average, cs)
     errs["Qw"] = max(rel_fro(rec.Qw[w], orc.power_step_q(M[w], rec.P_bar)) for w in range(W))
-    check_exchange(rec.Qw, rec.codes_q, rec.scales[1], rec.Q_bar, comp.bits_q, comp.alpha, stats, comp.average)
+    check_exchange(rec.Qw, rec.codes_q, rec.scales[1], rec.Q_bar, comp.bits_q, comp.alpha, stats, comp.average, cs)
     G_hat = orc.reconstruct(rec.P_bar, rec.Q_bar)
     errs["G_hat"] = rel_fro(rec.G_hat, G_hat)
     errs["E"] = max(rel_fro(rec.E_new[w], orc.error_update(M[w], G_hat)) for w in range(W))
@@ -153,7 +154,7 @@ def device_step_checked(comp: B.LQSGD, grads_dev, stats, check_payload=True):
             want = expected_payload(comp, recs, grads_host, w, vec_x)
             got = host(comp.payload(w))
             assert got.size == comp.payload_nbytes == want.size == orc.payload_bytes(
-                comp.layers, comp.rank, comp.bits_p, comp.bits_q, comp.quantize_vectors)
+                comp.layers, comp.rank, comp.bits_p, comp.bits_q, comp.quantize_vectors, comp.column_scales)
             assert np.array_equal(got, want), f"payload bytes of worker {w} differ"
     return recs, grads_host, ghat
 
@@ -178,14 +179,15 @@ def oracle_step_forced(oracle: orc.Oracle, grads_host, recs, stats):
         n, m = oracle.layers[l]
         Gl = np.stack([np.asarray(grads_host[w][l], dtype=np.float32).reshape(n, m) for w in range(oracle.W)])
         args = (Gl, oracle.E[l], oracle.Q[l], oracle.bits_p, oracle.bits_q, oracle.alpha)
-        res = orc.layer_round(*args, average=oracle.average)
+        kw = dict(average=oracle.average, column_scales=oracle.column_scales)
+        res = orc.layer_round(*args, **kw)
         fp = []
         for w in range(oracle.W):
             diff = codes_differ(res["xp"]["codes"][w], rec.codes_p[w], oracle.bits_p)
             stats["forced"] = stats.get("forced", 0) + int(diff.sum())
             assert np.all(res["xp"]["margin"][w][diff] < 2e-2), "P code differs far from a threshold"
             fp.append(np.where(diff, rec.codes_p[w].astype(np.int16), -1))
-        res = orc.layer_round(*args, forced_p=fp, average=oracle.average)
+        res = orc.layer_round(*args, forced_p=fp, **kw)
         fq = []
         for w in range(oracle.W):
             diff = codes_differ(res["xq"]["codes"][w], rec.codes_q[w], oracle.bits_q)

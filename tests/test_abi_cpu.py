@@ -49,7 +49,7 @@ def test_workspace_bytes_covers_the_persistent_state(lib):
     (dict(bits_p=1), B.ERR_INVALID_ARG), (dict(bits_q=9), B.ERR_INVALID_ARG),
     (dict(alpha=0.0), B.ERR_INVALID_ARG), (dict(alpha=float("nan")), B.ERR_INVALID_ARG),
     (dict(workers=0), B.ERR_INVALID_ARG), (dict(workers=257), B.ERR_INVALID_ARG),
-    (dict(flags=64), B.ERR_INVALID_ARG), (dict(power_iters=9), B.ERR_INVALID_ARG), (dict(power_iters=-1), B.ERR_INVALID_ARG),
+    (dict(flags=64), B.ERR_INVALID_ARG), (dict(flags=32), B.ERR_INVALID_ARG), (dict(power_iters=9), B.ERR_INVALID_ARG), (dict(power_iters=-1), B.ERR_INVALID_ARG),
     (dict(power_iters=2, world_workers=2), B.ERR_INVALID_ARG),
 ])
 def test_bad_config_is_rejected_on_the_host(lib, kw, code):
@@ -59,6 +59,13 @@ def test_bad_config_is_rejected_on_the_host(lib, kw, code):
     with pytest.raises(B.LqsgdError) as e:
         B.workspace_bytes([(8, 8)], cfg)
     assert e.value.code == code
+
+
+def test_column_scales_flag_changes_only_the_scale_bytes(lib):
+    layers = [(96, 200), (20, 1), (3, 5)]
+    plain = B.workspace_bytes(layers, B.make_config(4, 4, 4, 127.0, 2))
+    cols = B.workspace_bytes(layers, B.make_config(4, 4, 4, 127.0, 2, flags=B.FLAG_COLUMN_SCALES))
+    assert plain <= cols <= plain + (1 << 16)
 
 
 def test_bad_shapes_struct_size_and_null_pointers(lib):

@@ -25,7 +25,7 @@ def make(w: wl.Workload, **kw):
 def new_oracle(comp: B.LQSGD):
     Q0 = {l: par.host(comp.get_state(B.STATE_Q, l)) for l in range(len(comp.layers)) if comp.is_matrix(l)}
     return orc.Oracle(comp.layers, comp.rank, comp.bits_p, comp.bits_q, comp.alpha, comp.W, Q0, average=comp.average,
-                      quantize_vectors=comp.quantize_vectors)
+                      quantize_vectors=comp.quantize_vectors, column_scales=comp.column_scales)
 
 
 def run_steps(w: wl.Workload, steps: int, free_run=True, comp=None):
@@ -180,6 +180,63 @@ def test_quantised_vectors_variant(bits, W, average):
     comp.step_update(wl.draw_gradients(w, 2, device=DEV), gh, wts, 0.5)
     torch.cuda.synchronize()
     assert torch.allclose(wts[3], -0.5 * gh[3], rtol=0, atol=1e-7)
+
+
+@pytest.mark.parametrize("rank,bits,W,average", [(3, 4, 3, "codes"), (8, 3, 2, "values"), (1, 2, 1, "codes"),
+                                                  (16, 6, 2, "codes"), (30, 8, 9, "codes")])
+def test_column_scales_variant(rank, bits, W, average):
+    """LQSGD_FLAG_COLUMN_SCALES: one scale per factor column.  Scales, codes, averages, payload (2 r_eff
+    scales per matrix) and the free-running trajectory against the oracle in the same mode; the columns'
+    scales differ from one another and from the single-scale mode's."""
+    w = wl.Workload("cols", ((96, 200), (130, 36), (64, 27), (20, 1), (300, 512), (33, 17)), rank=rank, bits=bits,
+                    workers=W, steps=3, dist="student_t3", scale="fan_in", seed=41 + rank)
+    comp = make(w, average=average, column_scales=True)
+    assert comp.payload_nbytes == orc.payload_bytes(w.layers, rank, bits, bits, column_scales=True)
+    run_steps(w, 3, comp=comp)
+    sc = par.host(comp.get_state(B.STATE_SCALES, 4))
+    r = min(rank, 300)
+    assert sc.shape == (2, r)
+    one = make(w, average=average)
+    g = wl.draw_gradients(w, 0, device=DEV)
+    one.step(g, [torch.empty(s, device=DEV) for s in w.layers])
+    torch.cuda.synchronize()
+    s1 = par.host(one.get_state(B.STATE_SCALES, 4))
+    fresh = make(w, average=average, column_scales=True)
+    fresh.step(g, [torch.empty(s, device=DEV) for s in w.layers])
+    torch.cuda.synchronize()
+    sc0 = par.host(fresh.get_state(B.STATE_SCALES, 4))
+    assert np.float32(sc0[0].max()) == np.float32(s1[0])           # the factor's scale is the largest column scale
+    if r > 1:
+        assert len(set(sc0[0].tolist())) > 1
+    # workers on several GPUs agree on one scale per factor: the split round refuses the variant
+    with pytest.raises(B.LqsgdError) as ei:
+        fresh.round_begin(g, [torch.empty(s, device=DEV) for s in w.layers])
+    assert ei.value.code == B.ERR_INVALID_ARG
+
+
+def test_column_scales_zero_column_sets_the_status_bit():
+    """A dependent column of M Q becomes a zero column of P: its scale is 0, its codes and averages are 0,
+    and the zero-scale bit is set next to the dependent-column bit; the other columns are unaffected."""
+    w = wl.Workload("colz", ((64, 48),), rank=3, bits=4, workers=1, steps=1, dist="normal", scale="fan_in", seed=5)
+    comp = make(w, column_scales=True)
+    q = par.host(comp.get_state(B.STATE_Q, 0)).copy()
+    q[:, 2] = 2.0 * q[:, 0]                                         # third column of M Q depends on the first
+    comp.set_state(B.STATE_Q, 0, 0, torch.from_numpy(q))
+    g = wl.draw_gradients(w, 0, device=DEV)
+    gh = [torch.empty(s, device=DEV) for s in w.layers]
+    comp.step(g, gh)
+    torch.cuda.synchronize()
+    st = comp.status()[0]
+    assert st & B.STATUS_DEPENDENT_COLUMN and st & B.STATUS_ZERO_SCALE_P and not st & B.STATUS_NONFINITE
+    sc = par.host(comp.get_state(B.STATE_SCALES, 0))
+    assert sc[0, 2] == 0 and sc[0, 0] > 0 and sc[0, 1] > 0
+    assert not par.host(comp.get_state(B.STATE_P_BAR, 0))[:, 2].any()
+    assert not par.host(comp.get_state(B.STATE_CODES_P, 0, 0))[:, 2].any()
+    # and stage by stage against the oracle (which drops the same column and gives it scale 0)
+    comp2 = make(w, column_scales=True)
+    comp2.set_state(B.STATE_Q, 0, 0, torch.from_numpy(q))
+    recs, _, _ = par.device_step_checked(comp2, g, {})
+    assert np.all(recs[0].P[0][:, 2] == 0) and recs[0].scales[0][2] == 0
 
 
 @pytest.mark.parametrize("rank,T", [(3, 2), (3, 4), (16, 3)])
