@@ -7,6 +7,7 @@
 #include <cmath>
 #include <cstring>
 #include <new>
+#include <queue>
 #include <string>
 #include <vector>
 
@@ -154,6 +155,28 @@ int pick_size(const std::vector<int>& candidates, size_t want, F count_tiles) {
   return candidates.back();
 }
 
+// Finishing time of a list of tile costs handed, in order, to `slots` CTA slots as they become free
+// (what the hardware does with a one-CTA-per-tile grid).
+double makespan_dynamic(const std::vector<double>& cost, size_t slots) {
+  std::priority_queue<double, std::vector<double>, std::greater<double>> free_at;
+  for (size_t i = 0; i < std::min(slots, cost.size()); ++i) free_at.push(0.0);
+  double end = 0.0;
+  for (double c : cost) {
+    const double t = free_at.top() + c;
+    free_at.pop();
+    free_at.push(t);
+    end = std::max(end, t);
+  }
+  return end;
+}
+// Finishing time when CTA b of `ctas` takes tiles b, b + ctas, ... (the persistent staged kernels).
+double makespan_strided(const std::vector<double>& cost, size_t ctas) {
+  ctas = std::max<size_t>(1, std::min(ctas, cost.size()));
+  std::vector<double> load(ctas, 0.0);
+  for (size_t i = 0; i < cost.size(); ++i) load[i % ctas] += cost[i];
+  return cost.empty() ? 0.0 : *std::max_element(load.begin(), load.end());
+}
+
 // Lays out the workspace and builds every table.  base == nullptr: size only.
 void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg, void* base, int sm_count,
                Plan& p) {
@@ -216,17 +239,34 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   };
   const int c1 = pick_size({2048, 1024, 512}, want, [&](int c) {
     size_t t = 0;
-    for (auto& mt : p.mats) t += (size_t)W * ceil_div(mt.n, kPass1Rows) * ceil_div(mt.m, chunk_width(mt.m, c));
+    for (auto& mt : p.mats) t += (size_t)p.W_total * ceil_div(mt.n, kPass1Rows) * ceil_div(mt.m, chunk_width(mt.m, c));
     return t;
   });
   const int r2max = std::max(128, 32 * RP);
   auto colchunks = [&](int m) { return ceil_div(m, 128 * vec_of(m)); };
   auto balanced_rows = [](int n, int rmax) { return ceil_div(n, ceil_div(n, rmax)); };
-  const int r2 = pick_size({r2max, r2max / 2, std::max(32, r2max / 4)}, want, [&](int r) {
-    size_t t = 0;
-    for (auto& mt : p.mats) t += (size_t)W * ceil_div(mt.n, balanced_rows(mt.n, r)) * colchunks(mt.m);
-    return t;
-  });
+  // Pass 2 (register kernel, one CTA per tile): rows per tile by a model of the schedule.  A tile costs
+  // its rows plus a fixed part (start-up, the sum over the row groups) plus its partial sums' way to
+  // memory and back (RP floats per column twice, against one float per column and row); the tiles run
+  // in launch order on as many CTAs as fit the GPU at once.  Fewer, larger tiles save partial sums;
+  // the model stops where the last wave would run half empty.  The chunking of a sum decides its
+  // rounding, so the sizes that set it (here and c1 above) count the workers of ALL ranks: a rank that
+  // holds some of the workers then rounds like one process that holds them all.
+  const size_t slots2 = (size_t)sm_count * (RP <= 2 ? 4 : (RP <= 8 ? 3 : 1));
+  int r2 = r2max;
+  {
+    double best = -1.0;
+    for (int r = r2max; r >= 16; r -= 16) {
+      std::vector<double> cost;
+      for (auto& mt : p.mats) {
+        if (!(cfg.flags & LQSGD_FLAG_REGISTER_PATH) && RP >= 16 && mt.m % 4 == 0) continue;   // tensor-core pass 2
+        const int tr = balanced_rows(mt.n, r), nrb = ceil_div(mt.n, tr);
+        for (size_t i = 0; i < (size_t)p.W_total * nrb * colchunks(mt.m); ++i) cost.push_back(tr + 2.0 * RP + 16.0);
+      }
+      const double t = makespan_dynamic(cost, slots2);
+      if (best < 0.0 || t < best * 0.97) { best = t; r2 = r; }     // a smaller size must earn 3 %
+    }
+  }
   const int r3max = std::max(8, 64 / W);
   const int r3 = pick_size({r3max, std::max(8, r3max / 2), 8}, want, [&](int r) {
     size_t t = 0;
@@ -275,17 +315,43 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
     r = ceil_div(n, ceil_div(n, r));
     return (int)align_up((size_t)r, R);
   };
-  const size_t want_s = 4 * (size_t)sm_count;
-  auto count_staged = [&](size_t elems, int rmin, bool per_worker) {
-    size_t t = 0;
-    for (auto& mt : p.mats)
-      if (staged(mt))
-        t += (size_t)(per_worker ? W : 1) * ceil_div(mt.n, tile_rows(mt.n, mt.m, elems, rmin)) * staged_cols(mt.m).size();
-    return t;
+  // Tile sizes of the staged passes, again by a model of the schedule: CTA b of one per SM takes tiles
+  // b, b + SMs, ... in table order.  A tile costs its bytes (in full 36 KB stages; pass 3: every
+  // worker's, plus G_hat once), a little per stage (barriers) and a fixed start (its rows of Q).
+  // Small tiles balance the SMs, large ones save starts.  The two constants were fitted to measured
+  // pass times over tile sizes on the ResNet-18 set and on single matrices of 16 to 200 M elements;
+  // pass 1 then ran fastest at the model's minimum, pass 3 at the smallest size within 1 % of it.
+  constexpr double kStageCost = 0.05, kTileCost = 0.1;
+  auto staged_makespan = [&](size_t elems, bool pass3) {
+    std::vector<double> cost;
+    for (auto& mt : p.mats) {
+      if (!staged(mt)) continue;
+      const auto scols = staged_cols(mt.m);
+      const int tr = tile_rows(mt.n, mt.m, elems, 1);
+      for (int rb = 0; rb < ceil_div(mt.n, tr); ++rb)
+        for (auto& c : scols) {
+          const int nrows = std::min(tr, mt.n - rb * tr);
+          const double full = (double)nrows * c.second / kStreamSlabFloats;
+          const double nst = ceil_div(nrows, stream_geo(c.second, RP).R);
+          if (pass3) cost.push_back(W * (full + kStageCost * nst) + 0.5 * full + kTileCost);
+          else for (int w = 0; w < W; ++w) cost.push_back(full + kStageCost * nst + kTileCost);
+        }
+    }
+    return makespan_strided(cost, (size_t)sm_count);
   };
-  const size_t s1 = (size_t)pick_size({65536, 32768, 16384}, want_s, [&](int e) { return count_staged(e, 1, true); });
-  const size_t s3 = (size_t)pick_size({65536, 32768, 16384}, want_s,
-                                      [&](int e) { return count_staged(std::max(1, e / W), 1, false); }) / W;
+  auto pick_staged = [&](bool pass3) {
+    size_t best_e = 0;
+    double best = -1.0;
+    for (int i = 2; i <= 32; ++i) {
+      const int k = pass3 ? i : 34 - i;            // pass 3 from the smallest size up, pass 1 from the largest down
+      const size_t e = pass3 ? std::max<size_t>(1, (size_t)4096 * k / W) : (size_t)4096 * k;
+      const double t = staged_makespan(e, pass3);
+      if (best < 0.0 || t < best * (pass3 ? 0.99 : 0.995)) { best = t; best_e = e; }
+    }
+    return best_e;
+  };
+  const size_t s1 = pick_staged(false);
+  const size_t s3 = pick_staged(true);
 
   // ---- carve
   Arena a(base);
