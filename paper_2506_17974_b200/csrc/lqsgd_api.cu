@@ -280,6 +280,11 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   auto staged = [&](const MatHost& mt) {
     return !(cfg.flags & LQSGD_FLAG_REGISTER_PATH) && RP <= kStreamMaxRP && mt.m % 4 == 0;
   };
+  // A small layer with unaligned rows rides in the staged kernels as plain tiles (no launch of its own).
+  auto plain = [&](const MatHost& mt) {
+    return !(cfg.flags & LQSGD_FLAG_REGISTER_PATH) && RP <= kStreamMaxRP && mt.m % 4 != 0 &&
+           (size_t)mt.n * mt.m <= (size_t)kStreamPlainElems;
+  };
   // Tensor-core passes: padded rank 16, rows 16-byte aligned.
   auto on_tc = [&](const MatHost& mt) {
     return !(cfg.flags & LQSGD_FLAG_REGISTER_PATH) && RP >= 16 && mt.m % 4 == 0;
@@ -364,14 +369,14 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
     LayerDev& L = p.layers[li];
     std::memset(&L, 0, sizeof(L));
     L.n = mt.n; L.m = mt.m; L.r = mt.r; L.vec = vec_of(mt.m) == 4; L.user_index = mt.user_index;
-    const bool st = staged(mt), tc = on_tc(mt);
+    const bool st = staged(mt), tc = on_tc(mt), pl = plain(mt);
     const auto scols = staged_cols(mt.m);
     const int cw = chunk_width(mt.m, c1);
     // pass 2: register path, or tensor cores (row chunks in multiples of the 64 rows of an operand slot)
     const int tr2 = tc ? (int)align_up((size_t)balanced_rows(mt.n, kTcRowChunk), 64) : balanced_rows(mt.n, r2);
     // tensor-core pass 1: column chunks balanced in units of 32 columns, at most kTcPass1Cols wide
     const int tc_units = ceil_div(mt.m, 32), tc_ncc = ceil_div(tc_units * 32, kTcPass1Cols);
-    L.ncc = tc ? tc_ncc : (st ? (int)scols.size() : ceil_div(mt.m, cw));
+    L.ncc = tc ? tc_ncc : (st ? (int)scols.size() : (pl ? 1 : ceil_div(mt.m, cw)));
     L.nrb = ceil_div(mt.n, tr2);
     L.npb = ceil_div(mt.n, kFactorBlockRows);
     L.nqb = ceil_div(mt.m, kFactorBlockRows);
@@ -411,6 +416,13 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
         for (int cc = 0; cc < (int)scols.size(); ++cc)
           p.stiles3.push_back({li32, 0, rb * tr3, std::min(tr3, mt.n - rb * tr3), scols[cc].first, scols[cc].second, 0, 0});
     }
+    if (pl) {
+      for (int rb = 0; rb < ceil_div(mt.n, kStreamPlainRows); ++rb) {
+        const int row0 = rb * kStreamPlainRows, nrows = std::min(kStreamPlainRows, mt.n - row0);
+        for (int w = 0; w < W; ++w) p.stiles1.push_back({li32, w, row0, nrows, 0, mt.m, 0, 1});
+        p.stiles3.push_back({li32, 0, row0, nrows, 0, mt.m, 0, 1});
+      }
+    }
     if (tc) {
       int u0 = 0;
       for (int cc = 0; cc < tc_ncc; ++cc) {
@@ -426,7 +438,7 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
       for (int cb = 0; cb < ceil_div(mt.m, 128); ++cb)
         p.tctiles3.push_back({li32, 0, rb * kTcRowsPerTile, std::min(kTcRowsPerTile, mt.n - rb * kTcRowsPerTile), cb * 128,
                               std::min(128, mt.m - cb * 128), 0, 0});
-    for (int rb = 0; !st && !tc && rb < ceil_div(mt.n, kPass1Rows); ++rb)
+    for (int rb = 0; !st && !tc && !pl && rb < ceil_div(mt.n, kPass1Rows); ++rb)
       for (int cc = 0; cc < L.ncc; ++cc)
         for (int w = 0; w < W; ++w) {
           const int row0 = rb * kPass1Rows, col0 = cc * cw;
@@ -447,7 +459,7 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
           p.tctiles2.push_back({li32, w, row0, std::min(tr2, mt.n - row0), col0, std::min(128, mt.m - col0), rb, 0});
         }
     const int tr3 = balanced_rows(mt.n, r3);
-    for (int rb = 0; !st && !tc && rb < ceil_div(mt.n, tr3); ++rb)
+    for (int rb = 0; !st && !tc && !pl && rb < ceil_div(mt.n, tr3); ++rb)
       for (int cc = 0; cc < ceil_div(mt.m, cw2); ++cc) {
         const int row0 = rb * tr3, col0 = cc * cw2;
         p.tiles3.push_back({li32, 0, row0, std::min(tr3, mt.n - row0), col0, std::min(cw2, mt.m - col0), 0, 0});
@@ -568,6 +580,13 @@ struct lqsgd_ctx {
   bool has_weights = false;
   int round_stage = 0;               // progress of a split round (lqsgd_round_*)
 };
+
+// The fp32 1-D tensors need no kernel of their own when the fused exchange of P runs anyway: their blocks (same
+// shape) are appended to that launch.  Not in a split round (its exchange only packs), not in the quantised variant.
+static bool vectors_ride(const lqsgd_ctx* c) {
+  const bool quantised = (c->cfg.flags & LQSGD_FLAG_QUANTIZE_VECTORS) && c->cfg.bits_p != 32;
+  return !c->plan.mats.empty() && !c->plan.chV.empty() && !quantised && c->plan.W_total == c->plan.W;
+}
 
 extern "C" {
 
@@ -717,7 +736,7 @@ int lqsgd_launches_per_step(const lqsgd_ctx* ctx, int32_t* out) {
   const int pass2 = (p.tiles2.empty() ? 0 : 1) + (p.tctiles2.empty() ? 0 : 1);
   const int pass3 = (p.tiles3.empty() ? 0 : 1) + (p.stiles3.empty() ? 0 : 1) + (p.tctiles3.empty() ? 0 : 1);
   const int iters = std::max(1, ctx->cfg.power_iters);
-  *out = iters * ((p.mats.empty() ? 0 : 5) + pass1 + pass2) + pass3 + (p.chV.empty() ? 0 : 1);
+  *out = iters * ((p.mats.empty() ? 0 : 5) + pass1 + pass2) + pass3 + ((p.chV.empty() || vectors_ride(ctx)) ? 0 : 1);
   return LQSGD_OK;
 }
 
@@ -813,6 +832,13 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
   sx.send[0] = p.d_xsend[0]; sx.send[1] = p.d_xsend[1];
   sx.region_bytes[0] = p.region_bytes[0]; sx.region_bytes[1] = p.region_bytes[1];
   sx.region_off[0] = p.region_off[0]; sx.region_off[1] = p.region_off[1];
+  VectorJob vj{};
+  vj.vecs = p.d_vecs; vj.chunks = p.d_chV; vj.nchunks = (int)p.chV.size(); vj.W_total = p.W_total;
+  vj.vgrads = reinterpret_cast<const float* const*>(p.d_ptrs + vbase);
+  vj.vghat = reinterpret_cast<float* const*>(p.d_ptrs + vbase + nv * W);
+  vj.vweights = c->has_weights ? reinterpret_cast<float* const*>(p.d_ptrs + vbase + nv * (W + 1)) : nullptr;
+  vj.lr = t.lr;
+  const bool ride = vectors_ride(c);     // the 1-D tensors travel as extra blocks of the exchange of P
   const bool ev = c->have_events && !split;
 #define PHASE_MARK(i) do { if (ev) CK(cudaEventRecord(c->phase_events[i], st)); } while (0)
   switch (seg) {
@@ -824,12 +850,9 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
                                   reinterpret_cast<float* const*>(p.d_ptrs + vbase + nv * W),
                                   c->has_weights ? reinterpret_cast<float* const*>(p.d_ptrs + vbase + nv * (W + 1)) : nullptr,
                                   t.lr, p.d_payload, p.payload_stride, W, qp, {st, 0}));
-        } else
-        CK(launch_vectors(p.d_vecs, p.d_chV, (int)p.chV.size(),
-                          reinterpret_cast<const float* const*>(p.d_ptrs + vbase),
-                          reinterpret_cast<float* const*>(p.d_ptrs + vbase + nv * W),
-                          c->has_weights ? reinterpret_cast<float* const*>(p.d_ptrs + vbase + nv * (W + 1)) : nullptr,
-                          t.lr, p.d_payload, p.payload_stride, W, p.W_total, {st, 0}));
+        } else if (!ride) {
+          CK(launch_vectors(vj, p.d_payload, p.payload_stride, W, {st, 0}));
+        }
       }
       if (nm && !repeat) CK(cudaMemsetAsync(p.d_status, 0, nm * sizeof(uint32_t), st));
       if (!repeat) PHASE_MARK(0);
@@ -846,7 +869,7 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
       }
       break;
     case 1:
-      if (nm) CK(launch_exchange(RP, 0, t, qp, p.d_chP, (int)p.chP.size(), sx, {st, 0}));
+      if (nm) CK(launch_exchange(RP, 0, t, qp, p.d_chP, (int)p.chP.size(), sx, (ride && !repeat) ? &vj : nullptr, {st, 0}));
       PHASE_MARK(2);
       break;
     case 2:
@@ -863,7 +886,7 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
       }
       break;
     case 3:
-      if (nm) CK(launch_exchange(RP, 1, t, qq, p.d_chQ, (int)p.chQ.size(), sx, {st, 0}));
+      if (nm) CK(launch_exchange(RP, 1, t, qq, p.d_chQ, (int)p.chQ.size(), sx, nullptr, {st, 0}));
       PHASE_MARK(4);
       break;
     case 4:

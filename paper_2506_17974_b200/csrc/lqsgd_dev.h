@@ -60,7 +60,8 @@ struct Tile {
   int32_t row0, nrows;
   int32_t col0, ncols;
   int32_t part;               // pass 1: column-chunk index; pass 2: row-chunk index
-  int32_t pad;
+  int32_t pad;                // staged passes: 1 = plain tile (whole rows of a small layer with unaligned rows,
+                              // taken by the consumers with ordinary loads), else 0
 };
 
 // A block of rows of one worker's factor, handled by one CTA of a small factor kernel.
@@ -137,8 +138,20 @@ struct SplitExchange {
   uint64_t region_bytes[2];   // bytes of all layers' P (or Q) streams of one worker
   uint64_t region_off[2];     // offset of that region inside a payload
 };
+// The round's 1-D tensors (fp32 mean over the workers): tables, the step's pointers, what the model update needs.
+struct VectorJob {
+  const VectorDev* vecs;
+  const ExchangeChunk* chunks;   // (tensor, block of 256 entries)
+  int32_t nchunks;
+  int32_t W_total;               // workers of all ranks (the divisor of the mean)
+  const float* const* vgrads;    // [n_vec][W]
+  float* const* vghat;           // [n_vec], entries may be null
+  float* const* vweights;        // [n_vec] or null
+  float lr;
+};
+// ride: the 1-D tensors' blocks appended to this launch (or null)
 cudaError_t launch_exchange(int RP, int which /*0 = P, 1 = Q*/, const Tables& t, const QuantTables& q,
-                            const ExchangeChunk* ch, int nch, const SplitExchange& sx, Launch l);
+                            const ExchangeChunk* ch, int nch, const SplitExchange& sx, const VectorJob* ride, Launch l);
 cudaError_t launch_unpack_codes(const uint8_t* stream, int count, int bits, uint8_t* out, cudaStream_t st);
 cudaError_t launch_scale_reduce(const Tables& t, int which, float* scales, int n_mat, Launch l);
 cudaError_t launch_sum_dequant(int RP, int which, const Tables& t, const QuantTables& q, const ExchangeChunk* ch,
@@ -152,15 +165,15 @@ cudaError_t launch_pass3(int RP, const Tables& t, const Tile* tiles, int ntiles,
 cudaError_t launch_vectors_quant(const VectorDev* vecs, int nvecs, const float* const* vgrads, float* const* vghat,
                                  float* const* vweights, float lr, uint8_t* payload, uint64_t payload_stride, int W,
                                  const QuantTables& q, Launch l);
-cudaError_t launch_vectors(const VectorDev* vecs, const ExchangeChunk* chunks, int nchunks,
-                           const float* const* vgrads, float* const* vghat, float* const* vweights, float lr,
-                           uint8_t* payload, uint64_t payload_stride, int W, int W_total, Launch l);
+cudaError_t launch_vectors(const VectorJob& vj, uint8_t* payload, uint64_t payload_stride, int W, Launch l);
 // Bulk-copy staged passes (lqsgd_stream.cu): layers with m % 4 == 0 and RP <= 8.  One CTA per SM,
 // 512 consumer threads.  The copy engine limits the number of bulk copies in flight, not their
 // bytes, so tiles are wide (few, large row segments per stage) and a tile that spans whole rows
 // is fetched with ONE copy per stage (consecutive rows are contiguous).
 constexpr int kStreamMaxRP = 8;
 constexpr int kStreamConsumers = 512;
+constexpr int kStreamPlainElems = 65536;  // largest layer (elements per worker) with unaligned rows the staged kernels take as plain tiles
+constexpr int kStreamPlainRows = 16;      // rows of a plain tile: one per consumer warp
 constexpr int kStreamSlabFloats = 9216;   // one stage of one array: 36 KB = 16 x 576 = 8 x 1152 = 2 x 4608 floats
 
 // Widest tile (columns) the staged passes take at this padded rank: a thread keeps the Q rows

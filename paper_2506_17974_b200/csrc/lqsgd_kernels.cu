@@ -757,6 +757,33 @@ __device__ __forceinline__ void store_factor(const LayerDev& L, int which, int r
 }
 
 // ---------------------------------------------------------------------------------------
+// 1-D tensors: mean over the workers (Eq. 1) in worker order, and the raw fp32 values into
+// each worker's payload.  One block = 256 entries of one tensor.  Runs as a kernel of its own or
+// as extra blocks of the exchange of P (same block shape), which saves a launch per round.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ void vectors_block(const VectorJob& vj, int blk, uint8_t* payload, uint64_t payload_stride,
+                                              int W) {
+  const ExchangeChunk ch = vj.chunks[blk];
+  const VectorDev v = vj.vecs[ch.layer];
+  const int i = ch.chunk * 256 + threadIdx.x;
+  if (i >= v.len) return;
+  float s = 0.f;
+  for (int w = 0; w < W; ++w) {
+    const float x = vj.vgrads[(size_t)ch.layer * W + w][i];
+    reinterpret_cast<float*>(payload + (size_t)w * payload_stride + v.pay_off)[i] = x;
+    s += x;
+  }
+  const float mean = s / (float)vj.W_total;     // with workers on other GPUs too: this rank's share of the mean
+  if (vj.vghat[ch.layer]) vj.vghat[ch.layer][i] = mean;
+  if (vj.vweights && vj.vweights[ch.layer]) vj.vweights[ch.layer][i] = fmaf(-vj.lr, mean, vj.vweights[ch.layer][i]);
+}
+__global__ void __launch_bounds__(256)
+vectors_kernel(VectorJob vj, uint8_t* payload, uint64_t payload_stride, int W) {
+  pdl_wait();
+  vectors_block(vj, blockIdx.x, payload, payload_stride, W);
+}
+
+// ---------------------------------------------------------------------------------------
 // Factor exchange (Alg. 1: LogQuantize, All-Reduce, LogDequantize) for one chunk of 256
 // factor elements of one layer, all W workers:
 //   s      = max |x| over the layer's block maxima (shared scale)
@@ -769,8 +796,13 @@ __device__ __forceinline__ void store_factor(const LayerDev& L, int which, int r
 // B = bits per code (2..8), or 32: quantiser bypassed.  One block = 256 factor elements.
 template <int RP, int B>
 __global__ void __launch_bounds__(256)
-exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __restrict__ chunks, SplitExchange sx) {
+exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __restrict__ chunks, int nchunks,
+                SplitExchange sx, VectorJob vj) {
   pdl_wait();
+  if ((int)blockIdx.x >= nchunks) {      // blocks past the factor chunks: the round's 1-D tensors
+    vectors_block(vj, (int)blockIdx.x - nchunks, t.payload, t.payload_stride, t.W);
+    return;
+  }
   constexpr int CH = kExchangeChunk;   // 256 factor elements per block, one per thread
   constexpr int WB = 8;                // workers handled per round
   constexpr int NLEV = (B == 32) ? 2 : 1 << (B - 1);
@@ -1035,31 +1067,6 @@ sum_dequant_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __r
   }
 }
 
-// ---------------------------------------------------------------------------------------
-// 1-D tensors: mean over the workers (Eq. 1) in worker order, and the raw fp32 values into
-// each worker's payload.
-// ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256)
-vectors_kernel(const VectorDev* __restrict__ vecs, const ExchangeChunk* __restrict__ chunks,
-               const float* const* __restrict__ vgrads, float* const* __restrict__ vghat,
-               float* const* __restrict__ vweights, float lr, uint8_t* payload, uint64_t payload_stride, int W,
-               int W_total) {
-  pdl_wait();
-  const ExchangeChunk ch = chunks[blockIdx.x];
-  const VectorDev v = vecs[ch.layer];
-  const int i = ch.chunk * 256 + threadIdx.x;
-  if (i >= v.len) return;
-  float s = 0.f;
-  for (int w = 0; w < W; ++w) {
-    const float x = vgrads[(size_t)ch.layer * W + w][i];
-    reinterpret_cast<float*>(payload + (size_t)w * payload_stride + v.pay_off)[i] = x;
-    s += x;
-  }
-  const float mean = s / (float)W_total;     // with workers on other GPUs too: this rank's share of the mean
-  if (vghat[ch.layer]) vghat[ch.layer][i] = mean;
-  if (vweights && vweights[ch.layer]) vweights[ch.layer][i] = fmaf(-lr, mean, vweights[ch.layer][i]);
-}
-
 // Variant (LQSGD_FLAG_QUANTIZE_VECTORS): a 1-D tensor goes through the factor exchange, one CTA per
 // tensor: scale = max over workers and entries, code = sign | level (Eq. 4), little-endian b-bit
 // stream per worker, exact integer sum of the signed levels (or, value-domain variant, the sum of the
@@ -1209,9 +1216,11 @@ cudaError_t launch_q_reduce(int rp, const Tables& t, const FactorBlock* fb, int 
 }
 
 cudaError_t launch_exchange(int rp, int which, const Tables& t, const QuantTables& q,
-                            const ExchangeChunk* ch, int nch, const SplitExchange& sx, Launch l) {
+                            const ExchangeChunk* ch, int nch, const SplitExchange& sx, const VectorJob* ride, Launch l) {
   if (nch == 0) return cudaSuccess;
-#define LQSGD_EXCHANGE_BITS(BV) case BV: launch_pdl(exchange_kernel<RP, BV>, nch, 256, 0, l.stream, t, q, which, ch, sx); break;
+  const VectorJob vj = ride ? *ride : VectorJob{};
+  const int grid = nch + vj.nchunks;
+#define LQSGD_EXCHANGE_BITS(BV) case BV: launch_pdl(exchange_kernel<RP, BV>, grid, 256, 0, l.stream, t, q, which, ch, nch, sx, vj); break;
   LQSGD_DISPATCH_RP(rp, {
     switch (q.bits) {
       LQSGD_EXCHANGE_BITS(2) LQSGD_EXCHANGE_BITS(3) LQSGD_EXCHANGE_BITS(4) LQSGD_EXCHANGE_BITS(5)
@@ -1243,11 +1252,9 @@ cudaError_t launch_sum_dequant(int rp, int which, const Tables& t, const QuantTa
   return cudaGetLastError();
 }
 
-cudaError_t launch_vectors(const VectorDev* vecs, const ExchangeChunk* chunks, int nchunks,
-                           const float* const* vgrads, float* const* vghat, float* const* vweights, float lr,
-                           uint8_t* payload, uint64_t payload_stride, int W, int W_total, Launch l) {
-  if (nchunks == 0) return cudaSuccess;
-  launch_pdl(vectors_kernel, nchunks, 256, 0, l.stream, vecs, chunks, vgrads, vghat, vweights, lr, payload, payload_stride, W, W_total);
+cudaError_t launch_vectors(const VectorJob& vj, uint8_t* payload, uint64_t payload_stride, int W, Launch l) {
+  if (vj.nchunks == 0) return cudaSuccess;
+  launch_pdl(vectors_kernel, vj.nchunks, 256, 0, l.stream, vj, payload, payload_stride, W);
   return cudaGetLastError();
 }
 

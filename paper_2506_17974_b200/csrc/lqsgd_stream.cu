@@ -24,6 +24,74 @@ struct ConsumerState {
 };
 
 // ---------------------------------------------------------------------------------------
+// Plain tiles.  A small layer whose rows are not 16-byte aligned (m % 4 != 0: the 64 x 27 first
+// convolution) cannot come through the bulk-copy ring.  Rather than pay a kernel launch per pass
+// for a few KB, the consumers of the staged kernels take such a layer with ordinary loads while
+// the loader already fills the ring for the next tile: a tile is a few whole rows, one warp per
+// row, lanes across the columns.  Loader and storer skip these tiles.
+// ---------------------------------------------------------------------------------------
+template <int RP>
+__device__ __forceinline__ void pass1_plain_tile(const Tables& t, const Tile& tl) {
+  const LayerDev& L = t.layers[tl.layer];
+  const int m = L.m, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const float* __restrict__ G = t.grads[(size_t)tl.layer * t.W + tl.worker];
+  float* E = L.E + (size_t)tl.worker * L.n * m;
+  const float* __restrict__ Qt = L.Qt;
+  float* Pp = L.Ppart + (size_t)tl.worker * L.ncc * (size_t)L.n * RP;      // one column chunk: the whole row
+  for (int row = tl.row0 + warp; row < tl.row0 + tl.nrows; row += kConsumerWarps) {
+    float acc[RP];
+#pragma unroll
+    for (int j = 0; j < RP; ++j) acc[j] = 0.f;
+    for (int c = lane; c < m; c += 32) {
+      const size_t off = (size_t)row * m + c;
+      const float mv = __ldcs(G + off) + E[off];                             // M = G + E (Eq. 8)
+      E[off] = mv;
+#pragma unroll
+      for (int j = 0; j < RP; ++j) acc[j] = fmaf(mv, __ldg(Qt + (size_t)j * L.mt + c), acc[j]);
+    }
+#pragma unroll
+    for (int j = 0; j < RP; ++j) {
+#pragma unroll
+      for (int o = 16; o >= 1; o >>= 1) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], o);
+      if (lane == 0) Pp[(size_t)row * RP + j] = acc[j];
+    }
+  }
+}
+
+template <int RP>
+__device__ __forceinline__ void pass3_plain_tile(const Tables& t, const Tile& tl) {
+  const LayerDev& L = t.layers[tl.layer];
+  const int m = L.m, W = t.W, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const float* __restrict__ Qt = L.Qt;
+  const size_t plane = (size_t)L.n * m;
+  float* Gh = t.ghat[tl.layer];                                              // may be null
+  float* Wt = t.weights ? t.weights[tl.layer] : nullptr;                     // may be null
+  for (int row = tl.row0 + warp; row < tl.row0 + tl.nrows; row += kConsumerWarps) {
+    float p[RP];
+#pragma unroll
+    for (int j = 0; j < RP; ++j) p[j] = __ldg(L.Pbar + (size_t)row * RP + j);
+    for (int c = lane; c < m; c += 32) {
+      const size_t off = (size_t)row * m + c;
+      float gh = 0.f;                                                        // G_hat = P_bar Q_bar^T (Eq. 6)
+#pragma unroll
+      for (int j = 0; j < RP; ++j) gh = fmaf(p[j], __ldg(Qt + (size_t)j * L.mt + c), gh);
+      if (Gh) __stcs(Gh + off, gh);
+      if (Wt) Wt[off] = fmaf(-t.lr, gh, Wt[off]);                            // model update of Alg. 1
+      float* e = L.E + off;
+      int w = 0;
+      for (; w + 4 <= W; w += 4) {                                           // E_w = M_w - G_hat (Eq. 7)
+        float mv[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) mv[u] = e[(size_t)(w + u) * plane];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) e[(size_t)(w + u) * plane] = mv[u] - gh;
+      }
+      for (; w < W; ++w) e[(size_t)w * plane] -= gh;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
 // pass 1: M = G + E (Eq. 8) over E, partial P = M Q (Alg. 1) per column chunk.
 // ---------------------------------------------------------------------------------------
 template <int RP, int NST, int QPT, int RPT>
@@ -124,6 +192,7 @@ stream_pass1_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
     int last_layer = 0;
     uint32_t it = 0;
     for (int ti = blockIdx.x; ti < ntiles && ok; ti += gridDim.x) {
+      if (tiles[ti].pad) continue;              // plain tile: the consumers fetch it themselves
       const TileCtx c = tile_ctx<RP>(t, tiles[ti]);
       last_layer = c.layer;
       const float* G = t.grads[(size_t)c.layer * t.W + c.worker] + (size_t)c.row0 * c.m + c.col0;
@@ -148,6 +217,7 @@ stream_pass1_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
     bool ok = true;
     uint32_t it = 0;
     for (int ti = blockIdx.x; ti < ntiles && ok; ti += gridDim.x) {
+      if (tiles[ti].pad) continue;
       const TileCtx c = tile_ctx<RP>(t, tiles[ti]);
       float* E = t.layers[c.layer].E + ((size_t)c.worker * c.n + c.row0) * c.m + c.col0;
       for (int sr = 0; sr < c.nrows; sr += c.geo.R, ++it) {
@@ -167,6 +237,7 @@ stream_pass1_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
   }
   ConsumerState st{0, 0};
   for (int ti = blockIdx.x; ti < ntiles; ti += gridDim.x) {
+    if (tiles[ti].pad) { pass1_plain_tile<RP>(t, tiles[ti]); continue; }
     const TileCtx c = tile_ctx<RP>(t, tiles[ti]);
     bool ok;
     if (c.geo.qpt == 1) ok = pass1_consume<RP, NST, 1, Shape<RP>::RPT_NARROW>(t, c, ring, sG, sE, red, flags + 1, st);
@@ -313,6 +384,7 @@ stream_pass3_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
     int last_layer = 0;
     uint32_t it = 0;
     for (int ti = blockIdx.x; ti < ntiles && ok; ti += gridDim.x) {
+      if (tiles[ti].pad) continue;
       const TileCtx c = tile_ctx<RP>(t, tiles[ti]);
       last_layer = c.layer;
       const size_t plane = (size_t)c.n * c.m;
@@ -338,6 +410,7 @@ stream_pass3_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
     bool ok = true;
     uint32_t it = 0;
     for (int ti = blockIdx.x; ti < ntiles && ok; ti += gridDim.x) {
+      if (tiles[ti].pad) continue;
       const TileCtx c = tile_ctx<RP>(t, tiles[ti]);
       const size_t plane = (size_t)c.n * c.m;
       float* E0 = t.layers[c.layer].E + (size_t)c.row0 * c.m + c.col0;
@@ -360,6 +433,7 @@ stream_pass3_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
   }
   uint32_t it = 0;
   for (int ti = blockIdx.x; ti < ntiles; ti += gridDim.x) {
+    if (tiles[ti].pad) { pass3_plain_tile<RP>(t, tiles[ti]); continue; }
     const TileCtx c = tile_ctx<RP>(t, tiles[ti]);
     bool ok;
     if (c.geo.qpt == 1) ok = pass3_consume<RP, NST, 1, Shape<RP>::RPT_NARROW>(t, c, ring, sM, it);
