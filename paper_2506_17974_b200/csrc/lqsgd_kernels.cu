@@ -59,6 +59,24 @@ __device__ __forceinline__ void store_contig(float* p, const float (&v)[N]) {
   }
 }
 
+// Packed fp32 arithmetic of sm_100: one instruction, two fused multiply-adds on a register pair,
+// d.lo = a.lo * b.lo + c.lo and d.hi likewise, each half rounded exactly like fmaf.  Pass 2 at
+// rank 8 issues 8 multiply-adds per 4 bytes it streams and is bound by instruction issue, not by
+// HBM, unless they go out in pairs.
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+
 // VEC consecutive floats of a streamed matrix row (VEC = 4: one 128-bit access, VEC = 1: scalar).
 template <int VEC>
 struct Pack {
@@ -279,7 +297,7 @@ __device__ __forceinline__ ColMap col_map(const Tile& tl) {
 // Row groups are then summed through shared memory in group order.
 // ---------------------------------------------------------------------------------------
 template <int RP, int VEC>
-__device__ __forceinline__ void pass2_tile(const Tables& t, const Tile& tl, float* red, uint64_t pol) {
+__device__ __forceinline__ void pass2_tile(const Tables& t, const Tile& tl, float* red, float* pb, uint64_t pol) {
   const LayerDev& L = t.layers[tl.layer];
   const int m = L.m;
   const float* __restrict__ M = L.E + (size_t)tl.worker * L.n * m;
@@ -292,9 +310,62 @@ __device__ __forceinline__ void pass2_tile(const Tables& t, const Tile& tl, floa
 #pragma unroll
   for (int i = 0; i < VEC * RP; ++i) acc[i] = 0.f;
 
+  constexpr bool kPaired = RP >= 2 && RP <= 8 && VEC == 4;
+  if constexpr (kPaired) {
+    // the tile's rows of P_bar wait in shared memory: every thread needs every row, and reading them
+    // there leaves the L1 path to the stream of M (158 instead of 191 us on 8192 x 25088 at rank 8)
+    constexpr int VW = RP < 4 ? RP : 4;
+    for (int e = threadIdx.x; e < tl.nrows * (RP / VW); e += kPassThreads) {
+      float v[VW];
+      load_contig_ro<VW>(Pbar + (size_t)tl.row0 * RP + (size_t)e * VW, v);
+      store_contig<VW>(pb + (size_t)e * VW, v);
+    }
+    __syncthreads();
+  }
   if (cm.active) {
     constexpr int U = 8;
     int i = tl.row0 + cm.g;
+    if constexpr (kPaired) {
+      // the sums of columns j, j + 1 of P_bar travel as a pair: half the multiply-add instructions
+      constexpr int H = RP / 2;
+      uint64_t acc2[VEC * H];
+#pragma unroll
+      for (int k = 0; k < VEC * H; ++k) acc2[k] = 0ull;                      // (+0, +0)
+      auto row_update = [&](const Pack<VEC>& mv, int row) {
+        float p[RP];
+        if constexpr (RP >= 4) {
+#pragma unroll
+          for (int q4 = 0; q4 < RP / 4; ++q4) {
+            const float4 v = reinterpret_cast<const float4*>(pb + (size_t)(row - tl.row0) * RP)[q4];
+            p[4 * q4] = v.x; p[4 * q4 + 1] = v.y; p[4 * q4 + 2] = v.z; p[4 * q4 + 3] = v.w;
+          }
+        } else {
+          const float2 v = *reinterpret_cast<const float2*>(pb + (size_t)(row - tl.row0) * RP);
+          p[0] = v.x; p[1] = v.y;
+        }
+        uint64_t p2[H];
+#pragma unroll
+        for (int jj = 0; jj < H; ++jj) p2[jj] = pack2(p[2 * jj], p[2 * jj + 1]);
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) {
+          const uint64_t mk = pack2(mv.v[k], mv.v[k]);
+#pragma unroll
+          for (int jj = 0; jj < H; ++jj) acc2[k * H + jj] = fma2(mk, p2[jj], acc2[k * H + jj]);
+        }
+      };
+      for (; i + (U - 1) * cm.ng < rend; i += U * cm.ng) {
+        Pack<VEC> mv[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) mv[u] = ld_keep<VEC>(M + (size_t)(i + u * cm.ng) * m + col, pol);
+#pragma unroll
+        for (int u = 0; u < U; ++u) row_update(mv[u], i + u * cm.ng);
+      }
+      for (; i < rend; i += cm.ng) row_update(ld_keep<VEC>(M + (size_t)i * m + col, pol), i);
+#pragma unroll
+      for (int k = 0; k < VEC; ++k)
+#pragma unroll
+        for (int jj = 0; jj < H; ++jj) unpack2(acc2[k * H + jj], acc[k * RP + 2 * jj], acc[k * RP + 2 * jj + 1]);
+    } else {
     for (; i + (U - 1) * cm.ng < rend; i += U * cm.ng) {
       Pack<VEC> mv[U];
 #pragma unroll
@@ -317,6 +388,7 @@ __device__ __forceinline__ void pass2_tile(const Tables& t, const Tile& tl, floa
       for (int k = 0; k < VEC; ++k)
 #pragma unroll
         for (int j = 0; j < RP; ++j) acc[k * RP + j] = fmaf(mv.v[k], p[j], acc[k * RP + j]);
+    }
     }
   }
   // fixed-order sum over the row groups: group gg hands its sums to group 0
@@ -344,13 +416,14 @@ __global__ void __launch_bounds__(kPassThreads, (RP <= 2 ? 4 : (RP <= 8 ? 3 : 1)
 pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
   pdl_wait();
   __shared__ float red[128 * (RP > 16 ? 1 : 4) * RP];
+  __shared__ __align__(16) float pb[(RP >= 2 && RP <= 8) ? (RP <= 4 ? 128 : 32 * RP) * RP : 4];   // a tile's rows of P_bar: up to max(128, 32 RP)
   uint64_t pol;
   asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
   for (int i = blockIdx.x; i < ntiles; i += gridDim.x) {
     const Tile tl = tiles[i];
-    if constexpr (RP > 16) pass2_tile<RP, 1>(t, tl, red, pol);
-    else if (t.layers[tl.layer].vec) pass2_tile<RP, 4>(t, tl, red, pol);
-    else pass2_tile<RP, 1>(t, tl, red, pol);
+    if constexpr (RP > 16) pass2_tile<RP, 1>(t, tl, red, pb, pol);
+    else if (t.layers[tl.layer].vec) pass2_tile<RP, 4>(t, tl, red, pb, pol);
+    else pass2_tile<RP, 1>(t, tl, red, pb, pol);
   }
 }
 
