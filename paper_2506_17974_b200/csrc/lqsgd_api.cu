@@ -248,8 +248,10 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   // Pass 2 (register kernel, one CTA per tile): rows per tile by a model of the schedule.  A tile costs
   // its rows plus a fixed part (start-up, the sum over the row groups) plus its partial sums' way to
   // memory and back (RP floats per column twice, against one float per column and row); the tiles run
-  // in launch order on as many CTAs as fit the GPU at once.  Fewer, larger tiles save partial sums;
-  // the model stops where the last wave would run half empty.  The chunking of a sum decides its
+  // in launch order on 0.6 of the CTAs that fit the GPU at once (the pass is bound by bandwidth: beyond
+  // that many, more CTAs side by side do not finish sooner), and the longest chain of partial sums that
+  // the reduction after the pass adds up costs 0.7 of a row each.  Fewer, larger tiles save partial
+  // sums; the model stops where waves would run too empty.  (Fitted to rounds timed over tile sizes.)  The chunking of a sum decides its
   // rounding, so the sizes that set it (here and c1 above) count the workers of ALL ranks: a rank that
   // holds some of the workers then rounds like one process that holds them all.
   const size_t slots2 = (size_t)sm_count * (RP <= 2 ? 4 : (RP <= 8 ? 3 : 1));
@@ -258,12 +260,14 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
     double best = -1.0;
     for (int r = r2max; r >= 16; r -= 16) {
       std::vector<double> cost;
+      int chain = 0;
       for (auto& mt : p.mats) {
         if (!(cfg.flags & LQSGD_FLAG_REGISTER_PATH) && RP >= 16 && mt.m % 4 == 0) continue;   // tensor-core pass 2
         const int tr = balanced_rows(mt.n, r), nrb = ceil_div(mt.n, tr);
+        chain = std::max(chain, nrb);
         for (size_t i = 0; i < (size_t)p.W_total * nrb * colchunks(mt.m); ++i) cost.push_back(tr + 2.0 * RP + 16.0);
       }
-      const double t = makespan_dynamic(cost, slots2);
+      const double t = makespan_dynamic(cost, std::max<size_t>(1, slots2 * 6 / 10)) + 0.7 * chain;
       if (best < 0.0 || t < best * 0.97) { best = t; r2 = r; }     // a smaller size must earn 3 %
     }
   }
