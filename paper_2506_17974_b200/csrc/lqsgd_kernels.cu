@@ -545,15 +545,15 @@ p_reduce_gram_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
     for (int j = 0; j < RP; ++j) p[j] = 0.f;
     if (row < n) {
       const float* src = L.Ppart + ((size_t)fb.worker * L.ncc * n + row) * RP;
-      // the partials' loads go out together (4 at a time); the additions keep the chunk order
+      // the partials' loads go out together (8 at a time); the additions keep the chunk order
       int cc = 0;
       if constexpr (RP <= 8) {
-        for (; cc + 4 <= L.ncc; cc += 4) {
-          float v[4][RP];
+        for (; cc + 8 <= L.ncc; cc += 8) {
+          float v[8][RP];
 #pragma unroll
-          for (int u = 0; u < 4; ++u) load_contig_ro<RP>(src + (size_t)(cc + u) * n * RP, v[u]);
+          for (int u = 0; u < 8; ++u) load_contig_ro<RP>(src + (size_t)(cc + u) * n * RP, v[u]);
 #pragma unroll
-          for (int u = 0; u < 4; ++u)
+          for (int u = 0; u < 8; ++u)
 #pragma unroll
             for (int j = 0; j < RP; ++j) p[j] += v[u][j];
         }
@@ -591,19 +591,49 @@ __device__ __forceinline__ bool cholesky_lower(const LayerDev& L, int worker, do
   __shared__ double A[RP][RP + 1];     // Gram, overwritten by L (lower triangle)
   __shared__ double diag0[RP];
   const int r = L.r, tid = threadIdx.x, nt = blockDim.x;
-  for (int e = tid; e < RP * RP; e += nt) {
-    const double* gp = L.gram_part + (size_t)worker * L.npb * (RP * RP) + e;
-    double s = 0.0;
-    int b = 0;
-    for (; b + 8 <= L.npb; b += 8) {        // eight loads in flight, additions in block order
-      double x[8];
+  // Gram = sum of the block Grams.  With more threads than entries the blocks are dealt to SEG
+  // segments (segment g takes blocks g, g + SEG, ...), eight loads in flight each; the segments'
+  // sums are then added in segment order: a fixed order, and a chain SEG times shorter.
+  constexpr int SEG = (RP * RP <= 64) ? 128 / (RP * RP) : 1;      // the factor kernels run 128 threads
+  if constexpr (SEG > 1) {
+    __shared__ double segsum[SEG][RP * RP];
+    if (tid < SEG * RP * RP) {
+      const int e = tid % (RP * RP), g = tid / (RP * RP);
+      const double* gp = L.gram_part + (size_t)worker * L.npb * (RP * RP) + e;
+      double s = 0.0;
+      int b = g;
+      for (; b + 7 * SEG < L.npb; b += 8 * SEG) {
+        double x[8];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) x[u] = gp[(size_t)(b + u) * (RP * RP)];
+        for (int u = 0; u < 8; ++u) x[u] = gp[(size_t)(b + u * SEG) * (RP * RP)];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) s += x[u];
+        for (int u = 0; u < 8; ++u) s += x[u];
+      }
+      for (; b < L.npb; b += SEG) s += gp[(size_t)b * (RP * RP)];
+      segsum[g][e] = s;
     }
-    for (; b < L.npb; ++b) s += gp[(size_t)b * (RP * RP)];
-    A[e / RP][e % RP] = s;
+    __syncthreads();
+    if (tid < RP * RP) {
+      double s = segsum[0][tid];
+#pragma unroll
+      for (int g = 1; g < SEG; ++g) s += segsum[g][tid];
+      A[tid / RP][tid % RP] = s;
+    }
+  } else {
+    for (int e = tid; e < RP * RP; e += nt) {
+      const double* gp = L.gram_part + (size_t)worker * L.npb * (RP * RP) + e;
+      double s = 0.0;
+      int b = 0;
+      for (; b + 8 <= L.npb; b += 8) {        // eight loads in flight, additions in block order
+        double x[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) x[u] = gp[(size_t)(b + u) * (RP * RP)];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) s += x[u];
+      }
+      for (; b < L.npb; ++b) s += gp[(size_t)b * (RP * RP)];
+      A[e / RP][e % RP] = s;
+    }
   }
   __syncthreads();
   if (tid < RP) { diag0[tid] = A[tid][tid]; dead[tid] = 0; invd[tid] = 1.0; }
@@ -713,13 +743,14 @@ p_apply_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
 // V = min(RP, 4) consecutive columns of a row (one 128-bit load per partial when RP >= 4) and the
 // loads of several partials are in flight together: the chain of nrb dependent additions, not a
 // chain of nrb memory latencies, is what a row costs.
-constexpr int kQReduceThreads = 256;
+template <int RP> struct QReduceThreads { static constexpr int value = RP >= 8 ? 256 : 128; };   // one item per thread up to rank 8
 template <int RP>
-__global__ void __launch_bounds__(kQReduceThreads)
+__global__ void __launch_bounds__(QReduceThreads<RP>::value)
 q_reduce_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
   pdl_wait();
+  constexpr int kQReduceThreads = QReduceThreads<RP>::value;
   constexpr int V = RP < 4 ? RP : 4;        // floats per thread item
-  constexpr int TPR = RP / V;               // items per row: 1, 2, 4 or 8 (divides 256 and 32)
+  constexpr int TPR = RP / V;               // items per row: 1, 2, 4 or 8 (divides the block size and 32)
   __shared__ float smax[kQReduceThreads / 32][TPR * V];
   const FactorBlock fb = fbs[blockIdx.x];
   const LayerDev& L = t.layers[fb.layer];
@@ -1284,7 +1315,7 @@ cudaError_t launch_p_apply(int rp, const Tables& t, const FactorBlock* fb, int n
 
 cudaError_t launch_q_reduce(int rp, const Tables& t, const FactorBlock* fb, int nfb, Launch l) {
   if (nfb == 0) return cudaSuccess;
-  LQSGD_DISPATCH_RP(rp, (launch_pdl(q_reduce_kernel<RP>, nfb, kQReduceThreads, 0, l.stream, t, fb)));
+  LQSGD_DISPATCH_RP(rp, (launch_pdl(q_reduce_kernel<RP>, nfb, QReduceThreads<RP>::value, 0, l.stream, t, fb)));
   return cudaGetLastError();
 }
 
