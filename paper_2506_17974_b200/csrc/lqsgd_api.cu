@@ -62,7 +62,8 @@ struct Plan {
   std::vector<int> tcbegin3;
   int tc_grid = 0;
   std::vector<uint8_t> tcmaps;                   // tensor maps of the tensor-core passes (filled at create)
-  std::vector<FactorBlock> fbP, fbQ;
+  std::vector<FactorBlock> fbP, fbQ;             // 128-row blocks of P (layers orthonormalised in two launches) and of Q
+  std::vector<FactorBlock> fbS;                  // (layer, worker) of the layers orthonormalised by one CTA
   std::vector<ExchangeChunk> chP, chQ, chV;
   std::vector<float> thrP, thrQ, deqP, deqQ;
   std::vector<lqsgd_layer_layout> layout;     // by user layer index
@@ -80,7 +81,7 @@ struct Plan {
   Tile* d_tctiles3 = nullptr;
   int* d_tcbegin3 = nullptr;
   uint8_t* d_tcmaps = nullptr;
-  FactorBlock *d_fbP = nullptr, *d_fbQ = nullptr;
+  FactorBlock *d_fbP = nullptr, *d_fbQ = nullptr, *d_fbS = nullptr;
   ExchangeChunk *d_chP = nullptr, *d_chQ = nullptr, *d_chV = nullptr;
   float *d_thrP = nullptr, *d_thrQ = nullptr, *d_deqP = nullptr, *d_deqQ = nullptr;
   void** d_ptrs = nullptr;                    // see step_impl for the layout
@@ -468,8 +469,10 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
         const int row0 = rb * tr3, col0 = cc * cw2;
         p.tiles3.push_back({li32, 0, row0, std::min(tr3, mt.n - row0), col0, std::min(cw2, mt.m - col0), 0, 0});
       }
+    const bool one_cta = RP <= 8 && mt.n <= kOrthSmallMaxRows;
     for (int w = 0; w < W; ++w) {
-      for (int b = 0; b < L.npb; ++b) p.fbP.push_back({li32, w, b, 0});
+      if (one_cta) p.fbS.push_back({li32, w, 0, 0});
+      for (int b = 0; !one_cta && b < L.npb; ++b) p.fbP.push_back({li32, w, b, 0});
       for (int b = 0; b < L.nqb; ++b) p.fbQ.push_back({li32, w, b, 0});
     }
     for (int c = 0; c < ceil_div(mt.n * mt.r, kExchangeChunk); ++c) p.chP.push_back({li32, c});
@@ -529,6 +532,7 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   p.d_tcmaps = a.take<uint8_t>(p.mats.size() * kTcMapsPerLayer * kTcMapBytes);
   p.d_fbP = a.take<FactorBlock>(p.fbP.size());
   p.d_fbQ = a.take<FactorBlock>(p.fbQ.size());
+  p.d_fbS = a.take<FactorBlock>(p.fbS.size());
   p.d_chP = a.take<ExchangeChunk>(p.chP.size());
   p.d_chQ = a.take<ExchangeChunk>(p.chQ.size());
   p.d_chV = a.take<ExchangeChunk>(p.chV.size());
@@ -682,6 +686,7 @@ int lqsgd_create(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
   CK(up(p.d_tcmaps, p.tcmaps.data(), p.mats.size() * kTcMapsPerLayer * kTcMapBytes));
   CK(up(p.d_fbP, p.fbP.data(), p.fbP.size() * sizeof(FactorBlock)));
   CK(up(p.d_fbQ, p.fbQ.data(), p.fbQ.size() * sizeof(FactorBlock)));
+  CK(up(p.d_fbS, p.fbS.data(), p.fbS.size() * sizeof(FactorBlock)));
   CK(up(p.d_chP, p.chP.data(), p.chP.size() * sizeof(ExchangeChunk)));
   CK(up(p.d_chQ, p.chQ.data(), p.chQ.size() * sizeof(ExchangeChunk)));
   CK(up(p.d_chV, p.chV.data(), p.chV.size() * sizeof(ExchangeChunk)));
@@ -735,12 +740,13 @@ int lqsgd_set_phase_events(lqsgd_ctx* c, void* const* host_events) {
 int lqsgd_launches_per_step(const lqsgd_ctx* ctx, int32_t* out) {
   if (!ctx || !out) return LQSGD_ERR_INVALID_ARG;
   const Plan& p = ctx->plan;
-  // Orthonormalize (2), exchange of P, Q_w reduction, exchange of Q; then one launch per non-empty tile list
+  // Orthonormalize, exchange of P, Q_w reduction, exchange of Q; then one launch per non-empty tile list
   const int pass1 = (p.tiles1.empty() ? 0 : 1) + (p.stiles1.empty() ? 0 : 1) + (p.tctiles1.empty() ? 0 : 1);
   const int pass2 = (p.tiles2.empty() ? 0 : 1) + (p.tctiles2.empty() ? 0 : 1);
   const int pass3 = (p.tiles3.empty() ? 0 : 1) + (p.stiles3.empty() ? 0 : 1) + (p.tctiles3.empty() ? 0 : 1);
   const int iters = std::max(1, ctx->cfg.power_iters);
-  *out = iters * ((p.mats.empty() ? 0 : 5) + pass1 + pass2) + pass3 + ((p.chV.empty() || vectors_ride(ctx)) ? 0 : 1);
+  const int orth = (p.fbS.empty() ? 0 : 1) + (p.fbP.empty() ? 0 : 2);     // one CTA per small layer / Gram + apply
+  *out = iters * ((p.mats.empty() ? 0 : orth + 3) + pass1 + pass2) + pass3 + ((p.chV.empty() || vectors_ride(ctx)) ? 0 : 1);
   return LQSGD_OK;
 }
 
@@ -867,6 +873,7 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
       }
       PHASE_MARK(1);
       if (nm) {
+        CK(launch_p_orth_small(RP, t, p.d_fbS, (int)p.fbS.size(), {st, 0}));
         CK(launch_p_reduce_gram(RP, t, p.d_fbP, (int)p.fbP.size(), {st, 0}));
         CK(launch_p_apply(RP, t, p.d_fbP, (int)p.fbP.size(), {st, 0}));
         if (split) CK(launch_scale_reduce(t, 0, p.d_xscales, (int)nm, {st, 0}));

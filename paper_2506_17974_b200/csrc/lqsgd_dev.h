@@ -127,6 +127,9 @@ struct Launch {
 cudaError_t launch_pass1(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
 cudaError_t launch_p_reduce_gram(int RP, const Tables& t, const FactorBlock* fb, int nfb, Launch l);
 cudaError_t launch_p_apply(int RP, const Tables& t, const FactorBlock* fb, int nfb, Launch l);
+// Orthonormalize in one launch for layers of at most kOrthSmallMaxRows rows at RP <= 8: one CTA per (layer, worker)
+constexpr int kOrthSmallMaxRows = 512;
+cudaError_t launch_p_orth_small(int RP, const Tables& t, const FactorBlock* fb, int nfb, Launch l);
 // Split exchange (workers on several GPUs).  pack_only: quantise and pack with the scales in
 // `scales` ([2][n_mat], agreed between the ranks) and also write the streams into `send`
 // ([which][W][region_bytes], contiguous, ready for an all-gather); no sum, no dequantisation.

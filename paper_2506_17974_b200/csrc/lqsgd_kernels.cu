@@ -587,10 +587,12 @@ p_reduce_gram_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
 // reciprocals of its diagonal, dead[j] = 1 for a column dropped as dependent (its row and column
 // of L are then those of the identity).  Returns true if any column was dropped.
 template <int RP>
+__device__ __forceinline__ bool cholesky_factor(double (*A)[RP + 1], int r, double* Lf, double* invd, int* dead);
+
+template <int RP>
 __device__ __forceinline__ bool cholesky_lower(const LayerDev& L, int worker, double* Lf, double* invd, int* dead) {
   __shared__ double A[RP][RP + 1];     // Gram, overwritten by L (lower triangle)
-  __shared__ double diag0[RP];
-  const int r = L.r, tid = threadIdx.x, nt = blockDim.x;
+  const int tid = threadIdx.x, nt = blockDim.x;
   // Gram = sum of the block Grams.  With more threads than entries the blocks are dealt to SEG
   // segments (segment g takes blocks g, g + SEG, ...), eight loads in flight each; the segments'
   // sums are then added in segment order: a fixed order, and a chain SEG times shorter.
@@ -636,6 +638,14 @@ __device__ __forceinline__ bool cholesky_lower(const LayerDev& L, int worker, do
     }
   }
   __syncthreads();
+  return cholesky_factor<RP>(A, L.r, Lf, invd, dead);
+}
+
+// Cholesky of the Gram matrix in A (shared, complete and visible to the CTA on entry).
+template <int RP>
+__device__ __forceinline__ bool cholesky_factor(double (*A)[RP + 1], int r, double* Lf, double* invd, int* dead) {
+  __shared__ double diag0[RP];
+  const int tid = threadIdx.x, nt = blockDim.x;
   if (tid < RP) { diag0[tid] = A[tid][tid]; dead[tid] = 0; invd[tid] = 1.0; }
   __syncthreads();
   // right-looking Cholesky, the whole CTA on every step: pivot, column j, then the rank-1 update of
@@ -737,6 +747,101 @@ p_apply_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
   }
   amax = block_max_128(amax, smax);
   if (tid == 0) L.maxp[(size_t)fb.worker * L.npb + fb.blk] = amax;
+}
+
+// Orthonormalize for a layer of at most 512 rows (every layer of the ResNet-18 set), one CTA per
+// (layer, worker), one thread per row: the sum of pass 1's column-chunk partials, the Gram matrix in
+// fp64 (every entry summed over eight 64-row segments, the segments then added in order), its
+// Cholesky factor, the rows of P by substitution and the block maxima: what p_reduce_gram and
+// p_apply do in two launches for taller layers.
+constexpr int kOrthSmallRows = 512;
+template <int RP>
+__global__ void __launch_bounds__(kOrthSmallRows)
+p_orth_small_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
+  pdl_wait();
+  constexpr int NE = RP * RP, NSEG = 8, SEGROWS = kOrthSmallRows / NSEG;
+  __shared__ double rows[kOrthSmallRows][RP];
+  __shared__ double seg[NSEG][NE];
+  __shared__ double A[RP][RP + 1];
+  __shared__ double Lf[NE];
+  __shared__ double invd[RP];
+  __shared__ int dead[RP];
+  __shared__ float wmax[kOrthSmallRows / 32][RP];
+  const FactorBlock fb = fbs[blockIdx.x];
+  const LayerDev& L = t.layers[fb.layer];
+  const int n = L.n, tid = threadIdx.x, row = tid;
+  float p[RP];
+#pragma unroll
+  for (int j = 0; j < RP; ++j) p[j] = 0.f;
+  if (row < n) {
+    const float* src = L.Ppart + ((size_t)fb.worker * L.ncc * n + row) * RP;
+    for (int cc = 0; cc < L.ncc; ++cc) {
+      float v[RP];
+      load_contig_ro<RP>(src + (size_t)cc * n * RP, v);
+#pragma unroll
+      for (int j = 0; j < RP; ++j) p[j] += v[j];
+    }
+    if (L.ncc > 1) store_contig<RP>(L.Praw + ((size_t)fb.worker * n + row) * RP, p);
+  }
+#pragma unroll
+  for (int j = 0; j < RP; ++j) rows[tid][j] = (double)p[j];
+  __syncthreads();
+  for (int idx = tid; idx < NSEG * NE; idx += kOrthSmallRows) {
+    const int e = idx % NE, g = idx / NE, i = e / RP, j = e % RP;
+    if (j < i) continue;                                   // upper triangle; mirrored below
+    double s = 0.0;
+    for (int k = g * SEGROWS; k < (g + 1) * SEGROWS; ++k) s = fma(rows[k][i], rows[k][j], s);
+    seg[g][e] = s;
+  }
+  __syncthreads();
+  if (tid < NE) {
+    const int i = tid / RP, j = tid % RP;
+    if (j >= i) {
+      double s = seg[0][tid];
+#pragma unroll
+      for (int g = 1; g < NSEG; ++g) s += seg[g][tid];
+      A[i][j] = s;
+      A[j][i] = s;
+    }
+  }
+  __syncthreads();
+  const bool dropped = cholesky_factor<RP>(A, L.r, Lf, invd, dead);
+  if (dropped && tid == 0) atomicOr(&t.status[fb.layer], 1u);
+  float o[RP];
+#pragma unroll
+  for (int j = 0; j < RP; ++j) o[j] = 0.f;
+  if (row < n) {
+    double od[RP];
+    bool bad = false;
+#pragma unroll
+    for (int j = 0; j < RP; ++j) {
+      double s = (double)p[j];
+#pragma unroll
+      for (int k = 0; k < j; ++k) s = fma(-od[k], Lf[j * RP + k], s);
+      od[j] = (j < L.r && !dead[j]) ? s * invd[j] : 0.0;
+      o[j] = (float)od[j];
+      bad |= !(fabsf(o[j]) < INFINITY);
+    }
+    store_contig<RP>(L.P + ((size_t)fb.worker * n + row) * RP, o);
+    if (bad) atomicOr(&t.status[fb.layer], 8u);
+  }
+  // maxima per block of 128 rows (4 warps), as the exchange reads them; one per column in the column-scale variant
+#pragma unroll
+  for (int j = 0; j < RP; ++j) {
+    float v = fabsf(o[j]);
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, off));
+    if ((tid & 31) == 0) wmax[tid >> 5][j] = v;
+  }
+  __syncthreads();
+  const int ncs = t.col_scales ? RP : 1;
+  if (tid < L.npb * ncs) {
+    const int blk = tid / ncs, j0 = tid % ncs;
+    float a = 0.f;
+    for (int w4 = 4 * blk; w4 < 4 * blk + 4; ++w4)
+      for (int j = (t.col_scales ? j0 : 0); j < (t.col_scales ? j0 + 1 : RP); ++j) a = fmaxf(a, wmax[w4][j]);
+    L.maxp[((size_t)fb.worker * L.npb + blk) * ncs + j0] = a;
+  }
 }
 
 // Q_w = sum of the row-chunk partials of pass 2, in chunk order; block max |Q_w|.  A thread owns
@@ -1310,6 +1415,18 @@ cudaError_t launch_p_reduce_gram(int rp, const Tables& t, const FactorBlock* fb,
 cudaError_t launch_p_apply(int rp, const Tables& t, const FactorBlock* fb, int nfb, Launch l) {
   if (nfb == 0) return cudaSuccess;
   LQSGD_DISPATCH_RP(rp, (launch_pdl(p_apply_kernel<RP>, nfb, kFactorBlockRows, 0, l.stream, t, fb)));
+  return cudaGetLastError();
+}
+
+cudaError_t launch_p_orth_small(int rp, const Tables& t, const FactorBlock* fb, int nfb, Launch l) {
+  if (nfb == 0) return cudaSuccess;
+  switch (rp) {
+    case 1: launch_pdl(p_orth_small_kernel<1>, nfb, kOrthSmallRows, 0, l.stream, t, fb); break;
+    case 2: launch_pdl(p_orth_small_kernel<2>, nfb, kOrthSmallRows, 0, l.stream, t, fb); break;
+    case 4: launch_pdl(p_orth_small_kernel<4>, nfb, kOrthSmallRows, 0, l.stream, t, fb); break;
+    case 8: launch_pdl(p_orth_small_kernel<8>, nfb, kOrthSmallRows, 0, l.stream, t, fb); break;
+    default: return cudaErrorInvalidValue;
+  }
   return cudaGetLastError();
 }
 
