@@ -276,6 +276,24 @@ def test_several_power_iterations(rank, T):
     assert a.launches_per_step > b.launches_per_step
 
 
+@pytest.mark.parametrize("rank", [3, 8])
+def test_unaligned_layers_as_plain_tiles_and_on_the_register_path(rank):
+    """Layers whose rows are not 16-byte aligned: up to 65,536 elements they ride in the staged passes as
+    plain tiles (250 x 250, 64 x 27), larger ones (300 x 251) take the register-path kernels.  Both against
+    the oracle stage by stage and free-running, and the launch count says which path each set takes."""
+    small = ((250, 250), (64, 27), (128, 64), (9, 1))
+    w = wl.Workload("plain", small + ((300, 251),), rank=rank, bits=5, workers=3, steps=2, dist="student_t3",
+                    scale="fan_in", seed=77)
+    comp = make(w)
+    run_steps(w, 2, comp=comp)
+    # staged pass 1 + register pass 1, Orthonormalize in one launch (no layer above 512 rows), exchange of P
+    # (with the 1-D tensor's block), pass 2, Q_w reduction, exchange of Q, staged pass 3 + register pass 3
+    assert comp.launches_per_step == 9
+    only_small = make(dataclasses.replace(w, layers=small))
+    assert only_small.launches_per_step == 7
+    run_steps(dataclasses.replace(w, layers=small), 1, comp=only_small)
+
+
 def test_different_bits_for_p_and_q():
     w = wl.Workload("bpq", ((96, 200), (48, 1)), rank=4, bits=3, workers=2, steps=2, dist="student_t3", scale="fan_in")
     comp = make(w, bits_p=3, bits_q=6)
