@@ -648,31 +648,35 @@ __device__ __forceinline__ bool cholesky_factor(double (*A)[RP + 1], int r, doub
   const int tid = threadIdx.x, nt = blockDim.x;
   if (tid < RP) { diag0[tid] = A[tid][tid]; dead[tid] = 0; invd[tid] = 1.0; }
   __syncthreads();
-  // right-looking Cholesky, the whole CTA on every step: pivot, column j, then the rank-1 update of
-  // the trailing lower triangle with its entries dealt to the threads (every entry sees the
-  // updates in the order of j, so the result does not depend on the thread count)
-  for (int j = 0; j < r; ++j) {
-    const double d = A[j][j];
-    const bool ok = (d > kPivotEps * diag0[j]) && (d < INFINITY);   // false for nan too
-    // 1 / sqrt(d) by the hardware seed plus refinement (the library sqrt and division are long
-    // software sequences, and this loop is a chain of r of them); l_jj = d / sqrt(d)
-    const double inv = ok ? rsqrt(d) : 1.0;
-    const double ljj = ok ? d * inv : 1.0;
-    __syncthreads();                   // everybody has read the pivot
-    for (int i = j + tid; i < r; i += nt) {
-      if (i == j) { A[j][j] = ljj; invd[j] = inv; if (!ok) dead[j] = 1; }
-      else A[i][j] = ok ? A[i][j] * inv : 0.0;
-    }
-    __syncthreads();
-    if (ok) {
-      const int w = r - j - 1;         // trailing block: rows and columns j+1 .. r-1
-      for (int e = tid; e < w * w; e += nt) {
-        const int i = j + 1 + e / w, k = j + 1 + e % w;
-        if (k <= i) A[i][k] -= A[i][j] * A[k][j];
+  // right-looking Cholesky by ONE warp (warp-level barriers only; the other warps wait once, below):
+  // pivot, column j, then the rank-1 update of the trailing lower triangle with its entries dealt to
+  // the lanes (every entry sees the updates in the order of j, so the result does not depend on how
+  // the entries are dealt)
+  if (tid < 32) {
+    for (int j = 0; j < r; ++j) {
+      const double d = A[j][j];
+      const bool ok = (d > kPivotEps * diag0[j]) && (d < INFINITY);   // false for nan too
+      // 1 / sqrt(d) by the hardware seed plus refinement (the library sqrt and division are long
+      // software sequences, and this loop is a chain of r of them); l_jj = d / sqrt(d)
+      const double inv = ok ? rsqrt(d) : 1.0;
+      const double ljj = ok ? d * inv : 1.0;
+      __syncwarp();                      // every lane has read the pivot
+      for (int i = j + tid; i < r; i += 32) {
+        if (i == j) { A[j][j] = ljj; invd[j] = inv; if (!ok) dead[j] = 1; }
+        else A[i][j] = ok ? A[i][j] * inv : 0.0;
       }
+      __syncwarp();
+      if (ok) {
+        const int w = r - j - 1;         // trailing block: rows and columns j+1 .. r-1
+        for (int e = tid; e < w * w; e += 32) {
+          const int i = j + 1 + e / w, k = j + 1 + e % w;
+          if (k <= i) A[i][k] -= A[i][j] * A[k][j];
+        }
+      }
+      __syncwarp();
     }
-    __syncthreads();
   }
+  __syncthreads();
   for (int e = tid; e < RP * RP; e += nt) {
     const int i = e / RP, k = e % RP;
     Lf[e] = (k <= i && i < r) ? A[i][k] : 0.0;
