@@ -760,7 +760,7 @@ p_apply_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
 // p_apply do in two launches for taller layers.
 constexpr int kOrthSmallRows = 512;
 template <int RP>
-__global__ void __launch_bounds__(kOrthSmallRows)
+__global__ void __launch_bounds__(kOrthSmallRows, 3)   // three CTAs per SM: 444 at once, one wave for 21 layers x 16 workers
 p_orth_small_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
   pdl_wait();
   constexpr int NE = RP * RP, NSEG = 8, SEGROWS = kOrthSmallRows / NSEG;
