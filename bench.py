@@ -187,7 +187,9 @@ def run_reference(args):
     if rank != 0:
         return
     wl_obj, desc = get_workload(args.workload)
-    times, cores = time_oracle(wl_obj, budget_s=1e9, max_steps=args.warmup + args.steps)
+    # whole rounds until warm-up + steps are done or 150 s have passed, whichever comes first (the line
+    # says how many rounds were timed): the run ends within a few minutes on any host
+    times, cores = time_oracle(wl_obj, budget_s=150.0, max_steps=args.warmup + args.steps)
     timed = times[args.warmup:] or times
     t = sum(timed) / len(timed)
     value = gradient_bytes(wl_obj) / t / 1e9
