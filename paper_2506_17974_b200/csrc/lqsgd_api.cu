@@ -814,6 +814,7 @@ static int prepare_step(lqsgd_ctx* c, const float* const* grads, float* const* g
   t.status = p.d_status;
   t.W = W;
   t.col_scales = (c->cfg.flags & LQSGD_FLAG_COLUMN_SCALES) ? 1 : 0;
+  t.clear_status = 0;
   c->has_weights = weights != nullptr;
   return LQSGD_OK;
 }
@@ -864,12 +865,18 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
           CK(launch_vectors(vj, p.d_payload, p.payload_stride, W, {st, 0}));
         }
       }
-      if (nm && !repeat) CK(cudaMemsetAsync(p.d_status, 0, nm * sizeof(uint32_t), st));
       if (!repeat) PHASE_MARK(0);
       if (nm) {
-        CK(launch_pass1(RP, t, p.d_tiles1, (int)p.tiles1.size(), {st, c->grid1}));
-        CK(launch_stream_pass1(RP, t, p.d_stiles1, (int)p.stiles1.size(), {st, (int)std::min<size_t>(p.stiles1.size(), c->sm_count)}));
-        CK(launch_tc_pass1(RP, t, p.d_tctiles1, (int)p.tctiles1.size(), p.d_tcbegin1, p.d_tcmaps, {st, p.tc_grid}));
+        // the first pass-1 launch of the round zeroes the status words (see clear_status_words)
+        Tables first = t, rest = t;
+        first.clear_status = repeat ? 0 : (int)nm;
+        rest.clear_status = 0;
+        const bool reg1 = !p.tiles1.empty(), st1 = !p.stiles1.empty();
+        CK(launch_pass1(RP, reg1 ? first : rest, p.d_tiles1, (int)p.tiles1.size(), {st, c->grid1}));
+        CK(launch_stream_pass1(RP, (!reg1 && st1) ? first : rest, p.d_stiles1, (int)p.stiles1.size(),
+                               {st, (int)std::min<size_t>(p.stiles1.size(), c->sm_count)}));
+        CK(launch_tc_pass1(RP, (!reg1 && !st1) ? first : rest, p.d_tctiles1, (int)p.tctiles1.size(), p.d_tcbegin1, p.d_tcmaps,
+                           {st, p.tc_grid}));
       }
       PHASE_MARK(1);
       if (nm) {

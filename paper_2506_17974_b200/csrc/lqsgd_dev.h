@@ -85,6 +85,7 @@ struct Tables {
   uint32_t* status;           // [n_mat]
   int32_t W;
   int32_t col_scales;         // 1: one quantiser scale per factor column (variant), 0: one per factor
+  int32_t clear_status;       // > 0 only in the round's first pass-1 launch: that many status words are zeroed by CTA 0
 };
 
 struct QuantTables {
@@ -102,6 +103,15 @@ __device__ __forceinline__ void pdl_wait() {
 #if defined(__CUDA_ARCH__)
   asm volatile("griddepcontrol.wait;" ::: "memory");
 #endif
+}
+// The status words of a round start at zero.  The first pass-1 kernel of the round clears them itself (CTA 0, right
+// after its wait on the previous kernel), which saves a memset node between two rounds and lets this kernel's launch
+// overlap the previous round's tail.  Nothing can set a bit before the clear: the only bits a pass-1 kernel sets are
+// time-outs, and a wait gives up after 2^18 polls (milliseconds), while CTA 0 of a grid that fits the GPU at once
+// runs its first instructions in the kernel's first microseconds; every other bit comes from later kernels.
+__device__ __forceinline__ void clear_status_words(const Tables& t) {
+  if (t.clear_status > 0 && blockIdx.x == 0)
+    for (int i = threadIdx.x; i < t.clear_status; i += blockDim.x) t.status[i] = 0u;
 }
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,

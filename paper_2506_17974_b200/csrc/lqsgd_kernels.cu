@@ -262,6 +262,7 @@ template <int RP>
 __global__ void __launch_bounds__(kPassThreads, (RP <= 8 ? 2 : 1))
 pass1_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
   pdl_wait();
+  clear_status_words(t);
   for (int i = blockIdx.x; i < ntiles; i += gridDim.x) {
     const Tile tl = tiles[i];
     if constexpr (RP > 16) pass1_tile<RP, 1>(t, tl);   // above rank 16 these kernels only take what the tensor-core passes cannot

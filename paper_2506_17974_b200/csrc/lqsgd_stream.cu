@@ -176,6 +176,7 @@ template <int RP, int NST>
 __global__ void __launch_bounds__(kThreads, 1)
 stream_pass1_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
   pdl_wait();
+  clear_status_words(t);
   extern __shared__ __align__(128) unsigned char smem_raw[];
   float* sG = reinterpret_cast<float*>(smem_raw);
   float* sE = sG + NST * kSlab;

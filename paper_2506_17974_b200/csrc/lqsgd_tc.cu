@@ -399,6 +399,7 @@ template <int RP>
 __global__ void __launch_bounds__(kTcThreads, 1)
 tc_pass1_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict__ cta_begin, const uint8_t* __restrict__ maps) {
   pdl_wait();
+  clear_status_words(t);
   using S = Pass1Cfg<RP>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
