@@ -173,11 +173,15 @@ int lqsgd_create(const lqsgd_shape* host_shapes, int32_t n_layers, const lqsgd_c
  * cuda_stream: a cudaStream_t (NULL = legacy default stream).  The call only enqueues work;
  *   results, payload and state are valid once the stream has reached the end of that work.
  *   The pointer arrays themselves are consumed before the call returns.
+ * Pointer tables: the context keeps device copies of the tables of the last 16 distinct pointer
+ *   sets it was called with; a call with one of them enqueues kernels only (no copy between two
+ *   rounds), any other set costs one small host-to-device copy on the stream.
  * CUDA graphs: the call may be made on a capturing stream when its tensor pointers equal those
- *   of the previous call on this context (the captured work is then kernels only; the graph
- *   reads and writes those same tensors at every replay).  With different pointers a capturing
- *   stream gets LQSGD_ERR_CAPTURE and nothing is enqueued: the upload of the pointer table
- *   cannot be part of a graph. */
+ *   of an earlier call on this context whose table is still kept (the captured work is then
+ *   kernels only; the graph reads and writes those same tensors at every replay, and its table
+ *   is kept for the life of the context).  With other pointers a capturing stream gets
+ *   LQSGD_ERR_CAPTURE and nothing is enqueued: the upload of the pointer table cannot be part of
+ *   a graph.  (Also returned once 16 tables belong to captured graphs and a 17th set arrives.) */
 int lqsgd_step(lqsgd_ctx* ctx, const float* const* host_grads, float* const* host_ghat,
                void* cuda_stream);
 

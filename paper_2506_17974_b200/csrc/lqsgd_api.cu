@@ -44,6 +44,11 @@ struct Arena {
   }
 };
 
+// Device copies of the tensor-pointer tables of the last kPtrSets distinct pointer sets a context was stepped with: a
+// trainer that rotates a few gradient buffers (or always passes the same ones) uploads each table once, and a round
+// is then kernels only, with no copy node between two rounds.
+constexpr int kPtrSets = 16;
+
 struct MatHost {
   int n, m, r, user_index;
 };
@@ -84,7 +89,7 @@ struct Plan {
   FactorBlock *d_fbP = nullptr, *d_fbQ = nullptr, *d_fbS = nullptr;
   ExchangeChunk *d_chP = nullptr, *d_chQ = nullptr, *d_chV = nullptr;
   float *d_thrP = nullptr, *d_thrQ = nullptr, *d_deqP = nullptr, *d_deqQ = nullptr;
-  void** d_ptrs = nullptr;                    // see step_impl for the layout
+  void** d_ptrs = nullptr;                    // kPtrSets pointer tables, see prepare_step for the layout of one
   uint32_t* d_status = nullptr;
   uint8_t* d_payload = nullptr;
   float* d_xscales = nullptr;                 // [2][n_mat] scales the ranks agree on (split exchange)
@@ -540,7 +545,7 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   p.d_thrQ = a.take<float>(p.thrQ.size());
   p.d_deqP = a.take<float>(p.deqP.size());
   p.d_deqQ = a.take<float>(p.deqQ.size());
-  p.d_ptrs = a.take<void*>((p.mats.size() + p.vecs.size()) * (size_t)(W + 2));
+  p.d_ptrs = a.take<void*>(kPtrSets * (p.mats.size() + p.vecs.size()) * (size_t)(W + 2));
   if (cfg.power_iters > 1) {
     size_t big = 0;
     for (auto& mt : p.mats) big = std::max(big, (size_t)mt.n * mt.m);
@@ -579,8 +584,12 @@ struct lqsgd_ctx {
   Plan plan;
   int device = 0, sm_count = 0;
   int grid1 = 0, grid2 = 0, grid3 = 0;
-  std::vector<void*> ptrs_host;      // mirror of plan.d_ptrs
-  bool ptrs_valid = false;
+  std::vector<std::vector<void*>> ptr_sets;   // host mirrors of the device pointer tables (empty: slot unused)
+  std::vector<uint64_t> ptr_used;             // last use of each slot (step counter), for eviction
+  std::vector<char> ptr_pinned;               // slot was used by a capturing stream: a graph may replay it, never evicted
+  uint64_t step_counter = 0;
+  size_t ptr_count = 0;                       // pointers per table
+  void** ptrs_cur = nullptr;                  // the device table of the current step
   void* workspace = nullptr;
   cudaEvent_t phase_events[LQSGD_N_PHASES + 1];
   bool have_events = false;
@@ -716,7 +725,10 @@ int lqsgd_create(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
   c->grid1 = (int)std::min<size_t>(p.tiles1.size(), (size_t)c->sm_count * std::max(o1, 1));
   c->grid2 = (int)p.tiles2.size();   // one CTA per tile: the hardware scheduler balances them
   c->grid3 = (int)std::min<size_t>(p.tiles3.size(), (size_t)c->sm_count * std::max(o3, 1));
-  c->ptrs_host.assign((p.mats.size() + p.vecs.size()) * (size_t)(p.W + 2), nullptr);
+  c->ptr_count = (p.mats.size() + p.vecs.size()) * (size_t)(p.W + 2);
+  c->ptr_sets.assign(kPtrSets, std::vector<void*>());
+  c->ptr_used.assign(kPtrSets, 0);
+  c->ptr_pinned.assign(kPtrSets, 0);
   CK(cudaDeviceSynchronize());
   guard.c = nullptr;
   *ctx_out = c;
@@ -759,7 +771,7 @@ static int prepare_step(lqsgd_ctx* c, const float* const* grads, float* const* g
   const int W = p.W, nl = (int)c->shapes.size();
   const size_t nm = p.mats.size(), nv = p.vecs.size();
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  std::vector<void*> ptrs(c->ptrs_host.size());
+  std::vector<void*> ptrs(c->ptr_count);
   auto out_ptr = [&](float* const* arr, int ui, uintptr_t amask, void** slot) -> int {
     float* q = arr ? arr[ui] : nullptr;
     if (reinterpret_cast<uintptr_t>(q) & amask) return LQSGD_ERR_MISALIGNED;
@@ -794,20 +806,33 @@ static int prepare_step(lqsgd_ctx* c, const float* const* grads, float* const* g
     if (rc != LQSGD_OK) return rc;
     if (!ptrs[vbase + nv * W + vi] && !ptrs[vbase + nv * (W + 1) + vi]) return LQSGD_ERR_INVALID_ARG;
   }
-  if (!c->ptrs_valid || ptrs != c->ptrs_host) {
-    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
-    CK(cudaStreamIsCapturing(st, &cap));
+  // a table already on the device?  else upload it over the slot used longest ago
+  int slot = -1;
+  for (int k = 0; k < kPtrSets && slot < 0; ++k)
+    if (c->ptr_sets[k] == ptrs) slot = k;
+  ++c->step_counter;
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  CK(cudaStreamIsCapturing(st, &cap));
+  if (slot < 0) {
     if (cap != cudaStreamCaptureStatusNone) return LQSGD_ERR_CAPTURE;   // a copy from this host vector cannot be replayed
-    c->ptrs_host = ptrs;
-    // pageable source: the runtime stages it before returning, so the vector may change afterwards
-    CK(cudaMemcpyAsync(p.d_ptrs, c->ptrs_host.data(), ptrs.size() * sizeof(void*), cudaMemcpyHostToDevice, st));
-    c->ptrs_valid = true;
+    for (int k = 0; k < kPtrSets; ++k)
+      if (!c->ptr_pinned[k] && (slot < 0 || c->ptr_used[k] < c->ptr_used[slot])) slot = k;
+    if (slot < 0) return LQSGD_ERR_CAPTURE;                             // every table belongs to a captured graph
+    c->ptr_sets[slot] = ptrs;
+    // stream-ordered after the kernels that may still read the slot; pageable source: the runtime stages it before
+    // returning, so the vector may change afterwards
+    CK(cudaMemcpyAsync(p.d_ptrs + (size_t)slot * c->ptr_count, c->ptr_sets[slot].data(), ptrs.size() * sizeof(void*),
+                       cudaMemcpyHostToDevice, st));
   }
+  c->ptr_used[slot] = c->step_counter;
+  if (cap != cudaStreamCaptureStatusNone) c->ptr_pinned[slot] = 1;
+  void** dp = p.d_ptrs + (size_t)slot * c->ptr_count;
+  c->ptrs_cur = dp;
   Tables& t = c->tables;
   t.layers = p.d_layers;
-  t.grads = reinterpret_cast<const float* const*>(p.d_ptrs);
-  t.ghat = reinterpret_cast<float* const*>(p.d_ptrs + nm * W);
-  t.weights = weights ? reinterpret_cast<float* const*>(p.d_ptrs + nm * (W + 1)) : nullptr;
+  t.grads = reinterpret_cast<const float* const*>(dp);
+  t.ghat = reinterpret_cast<float* const*>(dp + nm * W);
+  t.weights = weights ? reinterpret_cast<float* const*>(dp + nm * (W + 1)) : nullptr;
   t.lr = lr;
   t.payload = p.d_payload;
   t.payload_stride = p.payload_stride;
@@ -845,9 +870,9 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
   sx.region_off[0] = p.region_off[0]; sx.region_off[1] = p.region_off[1];
   VectorJob vj{};
   vj.vecs = p.d_vecs; vj.chunks = p.d_chV; vj.nchunks = (int)p.chV.size(); vj.W_total = p.W_total;
-  vj.vgrads = reinterpret_cast<const float* const*>(p.d_ptrs + vbase);
-  vj.vghat = reinterpret_cast<float* const*>(p.d_ptrs + vbase + nv * W);
-  vj.vweights = c->has_weights ? reinterpret_cast<float* const*>(p.d_ptrs + vbase + nv * (W + 1)) : nullptr;
+  vj.vgrads = reinterpret_cast<const float* const*>(c->ptrs_cur + vbase);
+  vj.vghat = reinterpret_cast<float* const*>(c->ptrs_cur + vbase + nv * W);
+  vj.vweights = c->has_weights ? reinterpret_cast<float* const*>(c->ptrs_cur + vbase + nv * (W + 1)) : nullptr;
   vj.lr = t.lr;
   const bool ride = vectors_ride(c);     // the 1-D tensors travel as extra blocks of the exchange of P
   const bool ev = c->have_events && !split;
@@ -857,9 +882,9 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
       if (nv && !repeat) {
         if ((c->cfg.flags & LQSGD_FLAG_QUANTIZE_VECTORS) && c->cfg.bits_p != 32) {
           if (split) return LQSGD_ERR_INVALID_ARG;
-          CK(launch_vectors_quant(p.d_vecs, (int)nv, reinterpret_cast<const float* const*>(p.d_ptrs + vbase),
-                                  reinterpret_cast<float* const*>(p.d_ptrs + vbase + nv * W),
-                                  c->has_weights ? reinterpret_cast<float* const*>(p.d_ptrs + vbase + nv * (W + 1)) : nullptr,
+          CK(launch_vectors_quant(p.d_vecs, (int)nv, reinterpret_cast<const float* const*>(c->ptrs_cur + vbase),
+                                  reinterpret_cast<float* const*>(c->ptrs_cur + vbase + nv * W),
+                                  c->has_weights ? reinterpret_cast<float* const*>(c->ptrs_cur + vbase + nv * (W + 1)) : nullptr,
                                   t.lr, p.d_payload, p.payload_stride, W, qp, {st, 0}));
         } else if (!ride) {
           CK(launch_vectors(vj, p.d_payload, p.payload_stride, W, {st, 0}));

@@ -472,6 +472,20 @@ def test_step_replays_from_a_cuda_graph():
         assert torch.equal(a.payload(1), b.payload(1))
     assert all(s == 0 for s in a.status())
     assert torch.equal(a.get_state(B.STATE_E, 2, 1), b.get_state(B.STATE_E, 2, 1))
+    # eager steps with more distinct pointer sets than the context keeps tables for: the graph's table stays
+    keep = []
+    for t in range(4, 4 + 18):
+        g = wl.draw_gradients(w, t, device=DEV)
+        keep.append(g)                                   # distinct live buffers: distinct pointers
+        a.step(g, oa)
+        b.step(g, ob)
+    g = fill(30)
+    graph.replay()
+    b.step(g, ob)
+    torch.cuda.synchronize()
+    for x, y in zip(oa, ob):
+        assert torch.equal(x, y)
+    assert torch.equal(a.get_state(B.STATE_E, 2, 1), b.get_state(B.STATE_E, 2, 1))
 
 
 def test_step_host_matches_device_step():
