@@ -29,7 +29,8 @@ reading taken is stated next to the code:
 
 Pins (tests/test_oracle_*.py): hand-worked level/threshold tables, brute-force
 nearest-level matching, closed-form inverse pair, LAPACK QR, truncated SVD,
-planted-rank recovery, error-feedback telescoping, payload closed forms.
+planted-rank recovery, error-feedback telescoping, payload closed forms, and the payload
+layout against a byte string written out by hand (tests/golden/payload_layout.txt).
 The value of alpha and the readings above have no printed worked example in
 the paper: against the authors' own code they are "parity unpinned".
 """

@@ -186,6 +186,71 @@ def test_payload_closed_forms(golden_dir):
     assert orc.factor_bits(10, 512, 16, 4) == 10 * (10 + 512) * 4          # r_eff = min(r, n, m)
 
 
+def _payload_layout_case(golden_dir):
+    want = {}
+    for line in open(f"{golden_dir}/payload_layout.txt"):
+        if line.strip() and not line.startswith("#"):
+            name, *hexes = line.split()
+            want[name] = np.frombuffer(bytes.fromhex("".join(hexes)), dtype=np.uint8)
+    layers = ((2, 3), (3, 2), (2, 1))
+    scales = [(np.float32(1.0), np.float32(2.0)), (np.float32(0.5), np.float32(4.0))]
+    codes_p = [np.array([[5], [3]], np.uint8), np.array([[7], [0], [6]], np.uint8)]
+    codes_q = [np.array([[1], [2], [4]], np.uint8), np.array([[6], [1]], np.uint8)]
+    return want, layers, scales, codes_p, codes_q
+
+
+def check_payload_layout(golden_dir):
+    want, layers, scales, codes_p, codes_q = _payload_layout_case(golden_dir)
+    got = orc.assemble_payload(layers, 1, 3, 3, scales, codes_p, codes_q, [np.array([1.5, -2.0], np.float32)])
+    assert got.dtype == np.uint8 and got.tobytes() == want["default"].tobytes(), got.tobytes().hex()
+    assert got.size == orc.payload_bytes(layers, 1, 3, 3) == 30
+    got = orc.assemble_payload(layers, 1, 3, 3, scales, codes_p, codes_q, [np.array([4, 7], np.uint8)],
+                               vector_scales=[np.float32(3.0)])
+    assert got.tobytes() == want["quantized_vectors"].tobytes(), got.tobytes().hex()
+    assert got.size == orc.payload_bytes(layers, 1, 3, 3, quantize_vectors=True) == 27
+
+
+def test_payload_layout_byte_for_byte(golden_dir):
+    """assemble_payload against a byte string written out by hand from the documented order
+    (scales, 1-D tensors, P streams, Q streams; Section IV-C bit streams), both layouts."""
+    check_payload_layout(golden_dir)
+
+
+@pytest.mark.parametrize("mistake", ["p_q_swapped", "scales_last", "per_layer_interleaved", "big_endian_codes"])
+def test_payload_layout_pin_catches_a_wrong_order(mistake, golden_dir, monkeypatch):
+    """Plausible layout mistakes planted in the oracle must fail the byte-for-byte pin."""
+    good = orc.assemble_payload
+    pack = orc.pack_codes
+
+    def bad(layers, rank, bits_p, bits_q, scales, codes_p, codes_q, vectors, vector_scales=None):
+        if mistake == "p_q_swapped":
+            return good(layers, rank, bits_q, bits_p, scales, codes_q, codes_p, vectors, vector_scales)
+        if mistake == "scales_last":
+            out = good(layers, rank, bits_p, bits_q, scales, codes_p, codes_q, vectors, vector_scales)
+            k = 8 * len(scales)
+            return np.concatenate([out[k:], out[:k]])
+        if mistake == "per_layer_interleaved":
+            head = good(layers, rank, bits_p, bits_q, scales, [], [], vectors, vector_scales)
+            return np.concatenate([head] + [x for cp, cq in zip(codes_p, codes_q)
+                                            for x in (pack(cp, bits_p), pack(cq, bits_q))])
+        return good(layers, rank, bits_p, bits_q, scales, codes_p, codes_q, vectors, vector_scales)
+
+    def msb_first(codes, bits):                       # element 0 in the HIGHEST bits of the first byte
+        flat = np.asarray(codes, np.uint8).reshape(-1)
+        out = np.zeros((flat.size * bits + 7) // 8, np.uint8)
+        for i, c in enumerate(flat):
+            for j in range(bits):
+                pos = i * bits + j
+                out[pos >> 3] |= ((int(c) >> (bits - 1 - j)) & 1) << (7 - (pos & 7))
+        return out
+
+    if mistake == "big_endian_codes":
+        monkeypatch.setattr(orc, "pack_codes", msb_first)
+    monkeypatch.setattr(orc, "assemble_payload", bad)
+    with pytest.raises(AssertionError):
+        check_payload_layout(golden_dir)
+
+
 def test_resnet18_shape_list_reproduces_published_epoch_sizes():
     """Tables I-III: MB sent per epoch by uncompressed SGD and by rank-1 PowerSGD.  With 5
     workers and batch 128, CIFAR has 50000/640 = 78 iterations per epoch and MNIST 60000/640 = 93."""
