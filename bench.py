@@ -98,8 +98,10 @@ class ClockSampler:
     FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, index: int):
-        self.index, self.rows, self.proc = index, [], None
+    def __init__(self, gpu_id: str):
+        # gpu_id: what nvidia-smi --id takes - the device's UUID ("GPU-..."), so that the samples are this
+        # process's GPU whatever CUDA_VISIBLE_DEVICES maps ordinal 0 to (an index only as a last resort)
+        self.index, self.rows, self.proc = gpu_id, [], None
 
     def __enter__(self):
         try:
@@ -138,9 +140,19 @@ class ClockSampler:
                 if v.lower().startswith("active"):
                     reasons.add(n)
         if not sm:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "gpu": self.index}
         sm.sort()
-        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm),
+                "gpu": self.index}
+
+
+def gpu_smi_id(torch, local: int) -> str:
+    """The UUID nvidia-smi knows this CUDA device by (read-only query)."""
+    try:
+        u = str(torch.cuda.get_device_properties(local).uuid)
+        return u if u.startswith("GPU-") else "GPU-" + u
+    except Exception:
+        return str(local)
 
 
 def phase_bytes(wl_obj):
@@ -182,6 +194,14 @@ def gradient_bytes(wl_obj):
     return 4 * wl_obj.workers * sum(n * m for n, m in wl_obj.layers)
 
 
+def config_dict(wl_obj, desc):
+    """What both arms print as `config`: the workload, and nothing that depends on the arm."""
+    return {"workload": desc, "rank": wl_obj.rank, "bits": wl_obj.bits, "workers": wl_obj.workers,
+            "alpha": wl_obj.alpha,
+            "l2": f"inputs larger than L2: each step streams a gradient set of {gradient_bytes(wl_obj) / 1e6:.0f} MB "
+                  "plus the error buffers; the CUDA arm rotates gradient sets between steps"}
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -198,7 +218,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": len(timed), "warmup": args.warmup, "ms_per_step": 1e3 * t, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": desc},
+        "config": config_dict(wl_obj, desc),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
@@ -216,6 +236,8 @@ def run_ours(args):
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py --impl ours needs a CUDA device: there is no CPU fallback")
+    if local >= torch.cuda.device_count():
+        raise SystemExit(f"rank {rank} has no GPU: {torch.cuda.device_count()} visible, {world} ranks asked for")
     torch.cuda.set_device(local)
     dev = f"cuda:{local}"
     if world > 1:
@@ -231,7 +253,21 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    def bench_workload(wl_obj, steps, warmup, nsets, want_e2e, sample_clocks, want_graph=False):
+    def allmax(x):
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def allmax_list(xs):
+        if world == 1:
+            return list(xs)
+        t = torch.tensor(list(xs), dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return [float(v) for v in t.tolist()]
+
+    def bench_workload(wl_obj, steps, warmup, nsets, want_e2e, sample_clocks, want_graph=False, min_ms=0.0):
         comp = B.LQSGD(wl_obj.layers, wl_obj.rank, wl_obj.bits, alpha=wl_obj.alpha, workers=wl_obj.workers,
                        seed=wl_obj.seed + rank, device=dev)
         seeded = dataclasses.replace(wl_obj, seed=wl_obj.seed + 1000 * rank)
@@ -247,22 +283,33 @@ def run_ours(args):
             for e in evs:
                 e.record(stream)
         barrier()
-        sampler = ClockSampler(local) if sample_clocks else None
+        sampler = ClockSampler(gpu_smi_id(torch, local)) if sample_clocks else None
         if sampler:
             sampler.__enter__()
             time.sleep(0.15)
         barrier()
-        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        start.record(stream)
-        for t in range(steps):             # the timed region: nothing but the steps
-            comp.step_ptrs(*ptrs[(warmup + t) % nsets], stream)
-        stop.record(stream)
-        barrier()
+        # The timed region: blocks of exactly `steps` steps, each bracketed by a barrier + synchronize and timed with
+        # CUDA events on the launching stream; the block is repeated until min_ms of device time has passed
+        # (every rank runs the same number of blocks: the count comes from the slowest rank's first block), so that
+        # the region is long enough for the clock samples whatever `steps` the caller passed.
+        blocks = []
+        repeats, pos = 1, warmup
+        while len(blocks) < repeats:
+            start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            start.record(stream)
+            for t in range(steps):         # nothing but the steps
+                comp.step_ptrs(*ptrs[(pos + t) % nsets], stream)
+            stop.record(stream)
+            barrier()
+            pos += steps
+            blocks.append(start.elapsed_time(stop) / steps)
+            if len(blocks) == 1 and min_ms > 0:
+                repeats = int(min(1000, max(1, -(-min_ms // max(allmax(blocks[0]) * steps, 1e-6)))))
         # per-kernel times: the same steps again, with CUDA events recorded at the phase boundaries
         # on the launching stream (the records cost a little, so they stay out of the timed region)
         for t in range(psteps):
             comp.set_phase_events(events[t])
-            comp.step_ptrs(*ptrs[(warmup + steps + t) % nsets], stream)
+            comp.step_ptrs(*ptrs[(pos + t) % nsets], stream)
         barrier()
         if sampler:
             sampler.__exit__(None, None, None)
@@ -288,7 +335,8 @@ def run_ours(args):
             barrier()
             graph_ms = g0.elapsed_time(g1) / steps
             del graph
-        ms = start.elapsed_time(stop) / steps
+        blocks = sorted(allmax_list(blocks))      # per block: the slowest rank; then the median block
+        ms = blocks[len(blocks) // 2]
         phases = [sum(events[t][i].elapsed_time(events[t][i + 1]) for t in range(psteps)) / psteps
                   for i in range(B.N_PHASES)]
         per_step = sorted(events[t][0].elapsed_time(events[t][B.N_PHASES]) for t in range(psteps))
@@ -296,7 +344,8 @@ def run_ours(args):
         # a dependent column or a zero scale is a property of the data (it happens with 2-bit codes);
         # a non-finite value or an expired wait would make the timing meaningless
         assert all(s & (B.STATUS_NONFINITE | B.STATUS_TIMEOUT) == 0 for s in status), f"device status flags: {status}"
-        out = {"ms": ms, "phases_ms": dict(zip(B.PHASE_NAMES, phases)), "launches": comp.launches_per_step,
+        out = {"ms": ms, "repeats": len(blocks), "block_ms_min_max": [blocks[0], blocks[-1]],
+               "phases_ms": dict(zip(B.PHASE_NAMES, phases)), "launches": comp.launches_per_step,
                "payload": comp.payload_nbytes, "clocks": sampler.summary() if sampler else None, "graph_ms": graph_ms,
                "flagged_layers": sum(1 for x in status if x),
                "profiled_step_ms": {"min": per_step[0], "median": per_step[len(per_step) // 2], "max": per_step[-1],
@@ -305,8 +354,22 @@ def run_ours(args):
         if want_e2e:
             comp = B.LQSGD(wl_obj.layers, wl_obj.rank, wl_obj.bits, alpha=wl_obj.alpha, workers=wl_obj.workers,
                            seed=wl_obj.seed + rank, host_staging=True, device=dev)
-            hg = [[t.cpu().pin_memory() for t in per] for per in sets[0]]
-            hh = [torch.empty(t.shape).pin_memory() for t in ghat]
+            # host side as a trainer keeps it: one pinned flat buffer per worker (and one for G_hat), every tensor on
+            # a 16-byte boundary; lqsgd_step_host then moves each buffer in a few large copies
+            offs, total = [], 0
+            for t in ghat:
+                offs.append(total)
+                total += (t.numel() + 3) // 4 * 4
+
+            def flat_views(src):
+                buf = torch.empty(total, dtype=torch.float32).pin_memory()
+                views = [buf[o:o + t.numel()].view(t.shape) for o, t in zip(offs, ghat)]
+                if src is not None:
+                    for v, x in zip(views, src):
+                        v.copy_(x)
+                return views
+            hg = [flat_views(per) for per in sets[0]]
+            hh = flat_views(None)
             hp = torch.empty(wl_obj.workers * comp.payload_nbytes, dtype=torch.uint8).pin_memory()
             e2e_steps = max(1, min(steps, 5))
             comp.step_host(hg, hh, hp)
@@ -346,64 +409,115 @@ def run_ours(args):
         torch.cuda.synchronize()
         return (num / den) ** 0.5
 
+    def oracle_reconstruction_error(wl_obj):
+        """Part of the CPU-baseline leg (the one place this arm runs the oracle): one round of the workload on the
+        device and, on the same inputs and the same Q_0, one round of the oracle running free on the host;
+        returns ||G_hat - G_hat_oracle||_F / ||G_hat_oracle||_F over all matrices, the share of codes that
+        differ (a code next to a decision threshold moves its entry by a whole level) and the oracle's time."""
+        import numpy as np
+        from oracle import lqsgd_oracle as orc
+        comp = B.LQSGD(wl_obj.layers, wl_obj.rank, wl_obj.bits, alpha=wl_obj.alpha, workers=wl_obj.workers,
+                       seed=wl_obj.seed, device=dev)
+        mats = [l for l in range(len(wl_obj.layers)) if comp.is_matrix(l)]
+        Q0 = {l: comp.get_state(B.STATE_Q, l).cpu().numpy() for l in mats}
+        g = wl.draw_gradients(wl_obj, 0, device=dev)
+        ghat = [torch.empty_like(x) for x in g[0]]
+        comp.step(g, ghat)
+        torch.cuda.synchronize()
+        o = orc.Oracle(wl_obj.layers, wl_obj.rank, wl_obj.bits, wl_obj.bits, wl_obj.alpha, wl_obj.workers, Q0)
+        t0 = time.perf_counter()
+        out = o.step([[x.cpu().numpy() for x in per] for per in g])
+        secs = time.perf_counter() - t0
+        num = den = 0.0
+        differ = total = 0
+        for l in mats:
+            d = ghat[l].cpu().numpy().astype(np.float64) - out[l]["G_hat"]
+            num += float((d * d).sum())
+            den += float((out[l]["G_hat"] ** 2).sum())
+            for w in range(wl_obj.workers):
+                for which, key in ((B.STATE_CODES_P, "xp"), (B.STATE_CODES_Q, "xq")):
+                    c = comp.get_state(which, l, w).cpu().numpy()
+                    differ += int((c != out[l][key]["codes"][w]).sum())
+                    total += c.size
+        del comp
+        return {"ghat_vs_oracle_rel": (num / den) ** 0.5 if den > 0 else 0.0, "codes_differing": differ,
+                "codes": total, "oracle_s": secs}
+
     wl_obj, desc = get_workload(args.workload)
     if args.workers:
         wl_obj = dataclasses.replace(wl_obj, workers=args.workers)
         desc += f" [workers overridden: W={args.workers}]"
     gbytes = gradient_bytes(wl_obj)
     res = bench_workload(wl_obj, args.steps, args.warmup, nsets=3, want_e2e=not args.no_e2e, sample_clocks=True,
-                         want_graph=not args.no_graph)
+                         want_graph=not args.no_graph, min_ms=args.min_ms)
 
-    def allmax(x):
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
-
-    ms = allmax(res["ms"])
+    ms = res["ms"]
     e2e_ms = allmax(res.get("e2e_ms", float("nan")))
     value = world * gbytes / (ms * 1e-3) / 1e9
     pb = phase_bytes(wl_obj)
     dom = max(("pass1", "pass2", "pass3"), key=lambda k: res["phases_ms"][k])
     achieved = pb[dom] / (res["phases_ms"][dom] * 1e-3) / 1e9
     round_bytes = sum(pb.values())
+    traffic = recorded_traffic(args.workload, dom)
+    cfg = config_dict(wl_obj, desc)
+    cfg["parallelism"] = f"{world} independent replica(s), one per GPU, no collective"
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": desc, "l2": "inputs larger than L2: each step streams a different "
-                   f"gradient set ({gbytes / 1e6:.0f} MB) plus the error buffers; 3 sets rotate",
-                   "rank": wl_obj.rank, "bits": wl_obj.bits, "workers": wl_obj.workers, "alpha": wl_obj.alpha,
-                   "parallelism": f"{world} independent replica(s), one per GPU, no collective"},
-        "gpu_launches": args.steps * res["launches"],
+        "config": cfg,
+        "repeats": res["repeats"],
+        "timed_region": {"what": f"{res['repeats']} block(s) of {args.steps} steps, each bracketed by barrier + synchronize; "
+                                 "ms_per_step is the median over blocks of the per-block mean (max over ranks)",
+                         "block_ms_min": res["block_ms_min_max"][0], "block_ms_max": res["block_ms_min_max"][1]},
+        "gpu_launches": res["repeats"] * args.steps * res["launches"],
         "clocks": res["clocks"],
         "e2e": {"value": world * gbytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
                 "h2d_bytes_per_step": res.get("h2d"), "d2h_bytes_per_step": res.get("d2h"), "ms_per_step": e2e_ms}
         if "e2e_ms" in res else None,
+        # frac: algorithmic bytes of the pass / its CUDA-event time / peak.  traffic: DRAM bytes per launch of that
+        # kernel from the ncu capture summarised under profiles/ (a stored figure, not measured by this run; null when
+        # the kernel's sources changed since).  frac_min_bytes counts min(stored traffic, algorithmic bytes): bytes that
+        # an earlier pass left in L2 are not credited.
         "roofline": {"bound": "hbm", "kernel": kernel_name(dom, wl_obj.rank), "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": recorded_traffic(args.workload, dom),
+                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": traffic,
+                     "traffic_source": "stored: profiles/dram_traffic.json (ncu capture of this workload)" if traffic else None,
+                     "frac_min_bytes": (min(traffic, pb[dom]) / (res["phases_ms"][dom] * 1e-3) / 1e9 / peak) if traffic else None,
                      "bytes_per_launch": pb[dom], "kernel_ms": res["phases_ms"][dom]},
         "round": {"algorithmic_bytes": round_bytes, "achieved_gbs": round_bytes / (ms * 1e-3) / 1e9,
-                  "frac_of_peak": round_bytes / (ms * 1e-3) / 1e9 / peak, "phases_ms": res["phases_ms"],
-                  "profiled_step_ms": res["profiled_step_ms"]},
+                  "frac_of_peak": round_bytes / (ms * 1e-3) / 1e9 / peak, "frac_of_nominal_8tbs": round_bytes / (ms * 1e-3) / 8e12,
+                  "phases_ms": res["phases_ms"], "profiled_step_ms": res["profiled_step_ms"]},
         "cuda_graph": {"ms_per_step": res["graph_ms"], "what": "one captured step replayed on one gradient set "
                        "(larger than L2); the timed `value` above uses plain launches"} if res.get("graph_ms") else None,
         "compression_ratio": 4 * sum(n * m for n, m in wl_obj.layers) / res["payload"],
         "payload_bytes_per_worker": res["payload"],
     }
+
+    def compact(w, r):
+        rb = sum(phase_bytes(w).values())
+        return {"gbs_gradient": gradient_bytes(w) / (r["ms"] * 1e-3) / 1e9, "ms_per_step": r["ms"],
+                "round_frac_of_peak": rb / (r["ms"] * 1e-3) / 1e9 / peak, "round_frac_of_nominal_8tbs": rb / (r["ms"] * 1e-3) / 8e12,
+                "launches_per_step": r["launches"], "phases_ms": r["phases_ms"]}
+
     if rank == 0 and world == 1 and not args.no_sweep:
         sweep = {}
         for a, b in wl.CONFIG4_SIZES:
             w4 = wl.config4(a, b)
             # enough gradient sets that a rotation streams more than twice the L2 (126 MB) before a set returns
             nsets4 = max(2, min(16, -(-int(2.5e8) // gradient_bytes(w4))))
-            r4 = bench_workload(w4, steps=max(10, 2 * nsets4), warmup=3, nsets=nsets4, want_e2e=False, sample_clocks=False)
-            rb = sum(phase_bytes(w4).values())
-            sweep[f"{a}x{b}"] = {"gbs_gradient": gradient_bytes(w4) / (r4["ms"] * 1e-3) / 1e9, "ms_per_step": r4["ms"],
-                                 "round_frac_of_peak": rb / (r4["ms"] * 1e-3) / 1e9 / peak,
-                                 "phases_ms": r4["phases_ms"], "gradient_sets_rotated": nsets4}
+            r4 = bench_workload(w4, steps=max(20, 2 * nsets4), warmup=3, nsets=nsets4, want_e2e=False, sample_clocks=False,
+                                min_ms=50.0)
+            sweep[f"{a}x{b}"] = dict(compact(w4, r4), gradient_sets_rotated=nsets4)
         line["large_layer_sweep"] = sweep
+        # the other configurations, briefly (each a few tens of ms of device time)
+        others = {}
+        for name in ("single", "mnist", "config5_r1_b4", "config5_r8_b4", "config5_r16_b4"):
+            wo, _ = get_workload(name)
+            nso = max(2, min(16, -(-int(2.5e8) // gradient_bytes(wo))))
+            ro = bench_workload(wo, steps=20, warmup=3, nsets=nso, want_e2e=False, sample_clocks=False, min_ms=30.0)
+            others[name] = dict(compact(wo, ro), gradient_sets_rotated=nso,
+                                compression_ratio=4 * sum(n * m for n, m in wo.layers) / ro["payload"])
+        line["other_configs"] = others
     if rank == 0 and world == 1 and args.config5_sweep:
         # rank x bits grid on the 16-worker ResNet-18 (100 classes) set: throughput, compression ratio and
         # what the round loses, ||M - G_hat||_F / ||M||_F over all layers and workers at the last step
@@ -412,20 +526,25 @@ def run_ours(args):
             for b5 in (2, 3, 4, 8):
                 w5 = wl.config5(r5, b5)
                 r = bench_workload(w5, steps=min(args.steps, 100), warmup=3, nsets=2, want_e2e=False, sample_clocks=False)
-                rb = sum(phase_bytes(w5).values())
-                grid[f"r{r5}_b{b5}"] = {
-                    "gbs_gradient": gradient_bytes(w5) / (r["ms"] * 1e-3) / 1e9, "ms_per_step": r["ms"],
-                    "round_frac_of_peak": rb / (r["ms"] * 1e-3) / 1e9 / peak, "phases_ms": r["phases_ms"],
-                    "compression_ratio": 4 * sum(n * m for n, m in w5.layers) / r["payload"],
-                    "payload_bytes_per_worker": r["payload"], "residual_rel": residual_rel(w5, 10),
-                    "layers_with_dependent_column_or_zero_scale": r["flagged_layers"]}
+                grid[f"r{r5}_b{b5}"] = dict(
+                    compact(w5, r), compression_ratio=4 * sum(n * m for n, m in w5.layers) / r["payload"],
+                    payload_bytes_per_worker=r["payload"], residual_rel=residual_rel(w5, 10),
+                    layers_with_dependent_column_or_zero_scale=r["flagged_layers"])
         line["config5_sweep"] = grid
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        # The CPU-baseline leg: the oracle as it stands, on the host cores, on a bounded sample.
         times, cores = time_oracle(wl_obj, budget_s=12.0, max_steps=8)
         t = sum(times) / len(times)
         line["cpu_baseline"] = {"value": gbytes / t / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
                                 "sample": f"{len(times)} whole rounds of the same workload, numpy fp64, "
                                           f"{t:.2f} s each"}
+        # and, with the oracle's output at hand, the reconstruction error against it on points of the rank / bit grid
+        # (one round each: what the rank / bit sweep asks to be reported next to the throughput)
+        if not args.no_sweep:
+            err = {}
+            for r5, b5 in ((1, 4), (8, 4), (16, 4)):
+                err[f"config5_r{r5}_b{b5}"] = oracle_reconstruction_error(wl.config5(r5, b5))
+            line["cpu_baseline"]["reconstruction_error_vs_oracle"] = err
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
@@ -512,6 +631,8 @@ def main():
                     help="override the workload's worker count (smaller cases for profiler captures)")
     ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay measurement")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle")
+    ap.add_argument("--min-ms", type=float, default=500.0,
+                    help="repeat the block of --steps steps until this much device time has been timed (0: one block)")
     ap.add_argument("--exchange", action="store_true",
                     help="workers of all GPUs in one average, with the real NCCL exchange (default: independent replicas)")
     args = ap.parse_args()
@@ -520,6 +641,15 @@ def main():
                       ["lqsgd_tc.cu", "lqsgd_stream_common.cuh", "lqsgd_dev.h"]):
             print(" ".join(group), csrc_digest(group))
         return
+    if args.impl == "ours" and args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # plain `python bench.py --gpus N`: become N ranks, one per GPU, under torchrun on this node
+        import socket
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+        os.execv(sys.executable, [sys.executable, "-m", "torch.distributed.run", "--nnodes=1",
+                                  f"--nproc-per-node={args.gpus}", "--master-addr", "127.0.0.1", "--master-port", str(port),
+                                  os.path.abspath(__file__)] + sys.argv[1:])
     if args.impl == "reference":
         run_reference(args)
     elif args.exchange:

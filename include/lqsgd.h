@@ -185,6 +185,13 @@ int lqsgd_create(const lqsgd_shape* host_shapes, int32_t n_layers, const lqsgd_c
 int lqsgd_step(lqsgd_ctx* ctx, const float* const* host_grads, float* const* host_ghat,
                void* cuda_stream);
 
+/* Declares that every CUDA graph captured from this context's steps has been destroyed (or will never be
+ * replayed again): the pointer tables those captures pinned may be reused from now on.  Without this call a
+ * trainer that re-captures its step with new tensors would, after 16 captured pointer sets, get
+ * LQSGD_ERR_CAPTURE for every new set.  Replaying an old graph after this call reads whatever table has
+ * taken its slot since: do not.  Host-only. */
+int lqsgd_release_graph_tables(lqsgd_ctx* ctx);
+
 /* lqsgd_step followed, inside the reconstruction pass, by the model update that ends an
  * iteration of Algorithm 1:  w <- w - lr * G_hat  for every layer (for a 1-D tensor G_hat is the
  * worker mean).  host_weights: host array of n_layers device pointers, fp32, shaped and aligned
@@ -196,7 +203,7 @@ int lqsgd_step_update(lqsgd_ctx* ctx, const float* const* host_grads, float* con
                       float* const* host_weights, float lr, void* cuda_stream);
 
 /* ---- Workers on several GPUs: the round in pieces, with the exchanges left to the caller. ----
- * Algorithm 1 sends the quantised factors "across workers via All-Reduce" twice per iteration.
+ * Algorithm 1 has two All-Reduce steps per iteration, one for each quantised factor (Section IV-A).
  * With the workers of one process on one GPU that exchange is a sum inside lqsgd_step.  When
  * other processes hold more workers (config.world_workers = total over all ranks, each rank
  * simulating `workers` of them), a rank runs the round as
@@ -235,6 +242,9 @@ int lqsgd_exchange_view(const lqsgd_ctx* ctx, int32_t which, void** dev_ptr_out,
  * stream before returning.  host_grads / host_ghat are arrays of host pointers laid out as in
  * lqsgd_step (pinned memory makes the copies asynchronous to each other, pageable works);
  * host_payload (may be NULL) receives W * payload_bytes bytes, worker after worker.
+ * The staging area holds a worker's tensors in layer order, each starting on a 16-byte boundary; host tensors
+ * that follow one another in memory the same way (one flat gradient buffer per worker, tensors 16-byte aligned)
+ * are copied in one piece instead of one copy per tensor, and likewise the G_hat outputs.
  * Needs LQSGD_FLAG_HOST_STAGING. */
 int lqsgd_step_host(lqsgd_ctx* ctx, const float* const* host_grads, float* const* host_ghat,
                     void* host_payload, void* cuda_stream);
@@ -271,6 +281,19 @@ int lqsgd_status(const lqsgd_ctx* ctx, uint32_t* host_flags, void* cuda_stream);
  * copied before the call returns. */
 #define LQSGD_N_PHASES 5
 int lqsgd_set_phase_events(lqsgd_ctx* ctx, void* const* host_events);
+
+/* TEST SUPPORT - exercises the path a bounded device-side wait takes when it runs out, without any fault.
+ * The streaming passes wait on shared-memory barriers for their asynchronous copies; every such wait gives up
+ * after a fixed number of timed polls, the CTA's roles then leave their loops, copies in flight are waited for,
+ * tensor memory is released, the layer's status word gets LQSGD_STATUS_TIMEOUT and the kernel returns.  This
+ * call arms the NEXT step only: in pass `pass` (1, 2 or 3; pass 2 only where it runs on the tensor cores) the
+ * loader of CTA 0 leaves out the copies of its stage number `stage` (counted from 0 over the CTA's tiles), and
+ * every bounded wait of that step gives up after `wait_limit` polls (16 .. 2^18, about a microsecond each)
+ * instead of the built-in 2^18.  All addresses stay valid and nothing spins without a limit; the step's outputs
+ * (E of the affected layer included) are undefined, as after any time-out: restore E and Q with
+ * lqsgd_set_state, or use a fresh context, before relying on results again.  If the armed pass has no such
+ * stage the step runs normally.  Host-only; never needed in production. */
+int lqsgd_test_expire_wait(lqsgd_ctx* ctx, int32_t pass, int32_t stage, uint32_t wait_limit);
 
 /* Kernel launches one lqsgd_step enqueues (for launch accounting). */
 int lqsgd_launches_per_step(const lqsgd_ctx* ctx, int32_t* host_out);

@@ -40,7 +40,7 @@ EXPORTED = [
     "lqsgd_payload", "lqsgd_payload_layout", "lqsgd_get_state", "lqsgd_set_state", "lqsgd_status",
     "lqsgd_orthonormalize_noalloc",
     "lqsgd_round_begin", "lqsgd_round_pack", "lqsgd_round_reduce", "lqsgd_round_end", "lqsgd_exchange_view",
-    "lqsgd_launches_per_step", "lqsgd_set_phase_events", "lqsgd_destroy", "lqsgd_strerror", "lqsgd_last_cuda_error", "lqsgd_version",
+    "lqsgd_launches_per_step", "lqsgd_set_phase_events", "lqsgd_release_graph_tables", "lqsgd_test_expire_wait", "lqsgd_destroy", "lqsgd_strerror", "lqsgd_last_cuda_error", "lqsgd_version",
 ]
 
 
@@ -97,6 +97,8 @@ def load_library() -> C.CDLL:
     lib.lqsgd_launches_per_step.argtypes = [vp, C.POINTER(i32)]
     lib.lqsgd_orthonormalize_noalloc.argtypes = [vp, vp, i32, i32, vp, vp]
     lib.lqsgd_set_phase_events.argtypes = [vp, C.POINTER(vp)]
+    lib.lqsgd_release_graph_tables.argtypes = [vp]
+    lib.lqsgd_test_expire_wait.argtypes = [vp, i32, i32, C.c_uint32]
     lib.lqsgd_destroy.argtypes = [vp]
     lib.lqsgd_destroy.restype = None
     lib.lqsgd_strerror.argtypes = [C.c_int]
@@ -229,6 +231,15 @@ class LQSGD:
     def step_ptrs(self, g_arr, h_arr, stream: Optional[torch.cuda.Stream] = None) -> None:
         s = stream if stream is not None else torch.cuda.current_stream(self.device)
         _check(self.lib.lqsgd_step(self.ctx, g_arr, h_arr, C.c_void_p(s.cuda_stream)))
+
+    def release_graph_tables(self) -> None:
+        """Every graph captured from this context's steps is gone: its pointer tables may be reused."""
+        _check(self.lib.lqsgd_release_graph_tables(self.ctx))
+
+    def test_expire_wait(self, pass_: int, stage: int, wait_limit: int = 256) -> None:
+        """Test support: the next step's pass `pass_` leaves out one stage of copies on CTA 0 and every bounded
+        wait gives up after wait_limit polls, so that LQSGD_STATUS_TIMEOUT is raised without any fault."""
+        _check(self.lib.lqsgd_test_expire_wait(self.ctx, pass_, stage, wait_limit))
 
     def set_phase_events(self, events: Optional[Sequence[torch.cuda.Event]]) -> None:
         """Asks the next step to record N_PHASES + 1 caller-owned CUDA events at its phase boundaries."""

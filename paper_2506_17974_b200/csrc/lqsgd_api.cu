@@ -27,6 +27,13 @@ int cuda_fail(cudaError_t e, const char* what) {
     if (e__ != cudaSuccess) return cuda_fail(e__, #call);     \
   } while (0)
 
+}  // namespace
+namespace lqsgd {
+// for the library's other translation units: records the text lqsgd_last_cuda_error() returns
+int record_cuda_failure(cudaError_t e, const char* what) { return cuda_fail(e, what); }
+}  // namespace lqsgd
+namespace {
+
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -596,6 +603,8 @@ struct lqsgd_ctx {
   Tables tables{};                   // filled by prepare_step
   bool has_weights = false;
   int round_stage = 0;               // progress of a split round (lqsgd_round_*)
+  uint32_t test_wait_limit = 0;      // lqsgd_test_expire_wait: applies to the next step, then cleared
+  int test_skip_pass = 0, test_skip_stage = 0;
 };
 
 // The fp32 1-D tensors need no kernel of their own when the fused exchange of P runs anyway: their blocks (same
@@ -749,6 +758,20 @@ int lqsgd_set_phase_events(lqsgd_ctx* c, void* const* host_events) {
   return LQSGD_OK;
 }
 
+int lqsgd_test_expire_wait(lqsgd_ctx* c, int32_t pass, int32_t stage, uint32_t wait_limit) {
+  if (!c || pass < 1 || pass > 3 || stage < 0 || wait_limit < 16 || wait_limit > (1u << 18)) return LQSGD_ERR_INVALID_ARG;
+  c->test_wait_limit = wait_limit;
+  c->test_skip_pass = pass;
+  c->test_skip_stage = stage;
+  return LQSGD_OK;
+}
+
+int lqsgd_release_graph_tables(lqsgd_ctx* c) {
+  if (!c) return LQSGD_ERR_INVALID_ARG;
+  std::fill(c->ptr_pinned.begin(), c->ptr_pinned.end(), 0);
+  return LQSGD_OK;
+}
+
 int lqsgd_launches_per_step(const lqsgd_ctx* ctx, int32_t* out) {
   if (!ctx || !out) return LQSGD_ERR_INVALID_ARG;
   const Plan& p = ctx->plan;
@@ -818,11 +841,14 @@ static int prepare_step(lqsgd_ctx* c, const float* const* grads, float* const* g
     for (int k = 0; k < kPtrSets; ++k)
       if (!c->ptr_pinned[k] && (slot < 0 || c->ptr_used[k] < c->ptr_used[slot])) slot = k;
     if (slot < 0) return LQSGD_ERR_CAPTURE;                             // every table belongs to a captured graph
-    c->ptr_sets[slot] = ptrs;
+    // the host mirror names the slot's contents only once the copy has been accepted: after a failed copy the
+    // slot matches no pointer set, so no later call can take the stale device table for its own
+    c->ptr_sets[slot].clear();
     // stream-ordered after the kernels that may still read the slot; pageable source: the runtime stages it before
-    // returning, so the vector may change afterwards
-    CK(cudaMemcpyAsync(p.d_ptrs + (size_t)slot * c->ptr_count, c->ptr_sets[slot].data(), ptrs.size() * sizeof(void*),
+    // returning, so the vector may go afterwards
+    CK(cudaMemcpyAsync(p.d_ptrs + (size_t)slot * c->ptr_count, ptrs.data(), ptrs.size() * sizeof(void*),
                        cudaMemcpyHostToDevice, st));
+    c->ptr_sets[slot] = ptrs;
   }
   c->ptr_used[slot] = c->step_counter;
   if (cap != cudaStreamCaptureStatusNone) c->ptr_pinned[slot] = 1;
@@ -840,6 +866,11 @@ static int prepare_step(lqsgd_ctx* c, const float* const* grads, float* const* g
   t.W = W;
   t.col_scales = (c->cfg.flags & LQSGD_FLAG_COLUMN_SCALES) ? 1 : 0;
   t.clear_status = 0;
+  t.wait_limit = c->test_wait_limit;          // zero unless a test armed them for this step
+  t.test_skip_pass = c->test_skip_pass;
+  t.test_skip_stage = c->test_skip_stage;
+  c->test_wait_limit = 0;
+  c->test_skip_pass = c->test_skip_stage = 0;
   c->has_weights = weights != nullptr;
   return LQSGD_OK;
 }
@@ -1037,24 +1068,43 @@ int lqsgd_step_host(lqsgd_ctx* c, const float* const* host_grads, float* const* 
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   std::vector<const float*> dg((size_t)W * nl);
   std::vector<float*> dh(nl);
+  // Copies of tensors that follow one another both in the caller's memory and in the staging area are merged
+  // into one: a gradient set kept in one host buffer per worker goes up in a few large copies instead of one
+  // per tensor (most tensors of a network are a few hundred bytes of batch-norm parameters).
+  struct Run { char* dst; const char* src; size_t bytes; };
+  auto flush = [&](Run& r, cudaMemcpyKind kind) -> cudaError_t {
+    const cudaError_t e = r.bytes ? cudaMemcpyAsync(r.dst, r.src, r.bytes, kind, st) : cudaSuccess;
+    r.bytes = 0;
+    return e;
+  };
+  auto add = [&](Run& r, void* dst, const void* src, size_t bytes, cudaMemcpyKind kind) -> cudaError_t {
+    if (r.bytes && r.dst + r.bytes == dst && r.src + r.bytes == src) { r.bytes += bytes; return cudaSuccess; }
+    const cudaError_t e = flush(r, kind);
+    r = Run{static_cast<char*>(dst), static_cast<const char*>(src), bytes};
+    return e;
+  };
   for (int l = 0; l < nl; ++l) {
-    const size_t bytes = 4 * (size_t)c->shapes[l].rows * c->shapes[l].cols;
-    for (int w = 0; w < W; ++w) {
-      const float* src = host_grads[(size_t)w * nl + l];
-      if (!src) return LQSGD_ERR_INVALID_ARG;
-      float* dst = p.d_stage_g + (size_t)w * p.elems_total + p.elem_off[l];
-      CK(cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, st));
-      dg[(size_t)w * nl + l] = dst;
-    }
     if (!host_ghat[l]) return LQSGD_ERR_INVALID_ARG;
     dh[l] = p.d_stage_ghat + p.elem_off[l];
+    for (int w = 0; w < W; ++w)
+      if (!host_grads[(size_t)w * nl + l]) return LQSGD_ERR_INVALID_ARG;
   }
+  Run run{nullptr, nullptr, 0};
+  for (int w = 0; w < W; ++w)
+    for (int l = 0; l < nl; ++l) {
+      const size_t bytes = 4 * (size_t)c->shapes[l].rows * c->shapes[l].cols;
+      float* dst = p.d_stage_g + (size_t)w * p.elems_total + p.elem_off[l];
+      CK(add(run, dst, host_grads[(size_t)w * nl + l], bytes, cudaMemcpyHostToDevice));
+      dg[(size_t)w * nl + l] = dst;
+    }
+  CK(flush(run, cudaMemcpyHostToDevice));
   const int rc = lqsgd_step(c, dg.data(), dh.data(), cuda_stream);
   if (rc != LQSGD_OK) return rc;
   for (int l = 0; l < nl; ++l) {
     const size_t bytes = 4 * (size_t)c->shapes[l].rows * c->shapes[l].cols;
-    CK(cudaMemcpyAsync(host_ghat[l], dh[l], bytes, cudaMemcpyDeviceToHost, st));
+    CK(add(run, host_ghat[l], dh[l], bytes, cudaMemcpyDeviceToHost));
   }
+  CK(flush(run, cudaMemcpyDeviceToHost));
   if (host_payload) {
     CK(cudaMemcpy2DAsync(host_payload, p.payload_bytes, p.d_payload, p.payload_stride, p.payload_bytes, W,
                          cudaMemcpyDeviceToHost, st));

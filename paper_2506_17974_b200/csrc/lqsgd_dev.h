@@ -86,7 +86,17 @@ struct Tables {
   int32_t W;
   int32_t col_scales;         // 1: one quantiser scale per factor column (variant), 0: one per factor
   int32_t clear_status;       // > 0 only in the round's first pass-1 launch: that many status words are zeroed by CTA 0
+  // Test support (lqsgd_test_expire_wait; all zero in normal operation): the bounded waits of the staged and
+  // tensor-core passes give up after wait_limit timed polls instead of the built-in limit, and the loader of
+  // CTA 0 of pass test_skip_pass (1, 2 or 3) leaves out the copies of its stage number test_skip_stage, so
+  // that the waits on that stage run out.  Every address stays valid; only a wait expires.
+  uint32_t wait_limit;
+  int32_t test_skip_pass;
+  int32_t test_skip_stage;
 };
+__device__ __forceinline__ bool test_skips_stage(const Tables& t, int pass, uint32_t stage) {
+  return t.test_skip_pass == pass && blockIdx.x == 0 && stage == (uint32_t)t.test_skip_stage;
+}
 
 struct QuantTables {
   const float* thr;           // [L-1] ascending decision thresholds on |x|/s

@@ -27,6 +27,8 @@
 
 #include <mutex>
 
+namespace lqsgd { int record_cuda_failure(cudaError_t e, const char* what); }   // lqsgd_api.cu: text for lqsgd_last_cuda_error()
+
 namespace {
 
 constexpr int kR = 16;                        // internal column padding (rank <= 16)
@@ -176,11 +178,16 @@ extern "C" int lqsgd_orthonormalize_noalloc(const float* dev_p_in, float* dev_p_
   if ((reinterpret_cast<uintptr_t>(dev_p_in) & 3) || (reinterpret_cast<uintptr_t>(dev_p_out) & 3))
     return LQSGD_ERR_MISALIGNED;
   double* scratch = nullptr;
-  if (scratch_for_current_device(&scratch) != cudaSuccess) return LQSGD_ERR_CUDA;
+  cudaError_t e = scratch_for_current_device(&scratch);
+  if (e != cudaSuccess) return lqsgd::record_cuda_failure(e, "cudaGetSymbolAddress(scratch)");
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const int nblocks = (rows + kRowsPerBlock - 1) / kRowsPerBlock;
+  // every launch is checked by itself, so that the error reported is this call's own
   noalloc_gram_kernel<<<nblocks, 256, 0, st>>>(dev_p_in, rows, rank, scratch);
+  if ((e = cudaPeekAtLastError()) != cudaSuccess) return lqsgd::record_cuda_failure(e, "noalloc_gram_kernel launch");
   noalloc_cholesky_kernel<<<1, 256, 0, st>>>(nblocks, rank, scratch, dev_status_out);
+  if ((e = cudaPeekAtLastError()) != cudaSuccess) return lqsgd::record_cuda_failure(e, "noalloc_cholesky_kernel launch");
   noalloc_apply_kernel<<<nblocks, kRowsPerBlock, 0, st>>>(dev_p_in, dev_p_out, rows, rank, scratch);
-  return cudaGetLastError() == cudaSuccess ? LQSGD_OK : LQSGD_ERR_CUDA;
+  if ((e = cudaPeekAtLastError()) != cudaSuccess) return lqsgd::record_cuda_failure(e, "noalloc_apply_kernel launch");
+  return LQSGD_OK;
 }

@@ -182,9 +182,9 @@ stream_pass1_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
   float* sE = sG + NST * kSlab;
   float* red = sE + NST * kSlab;                              // [2][16 warps][NRED]
   uint64_t* bars = reinterpret_cast<uint64_t*>(red + 2 * kConsumerWarps * Shape<RP>::NRED);
-  volatile int* flags = reinterpret_cast<volatile int*>(bars + 3 * NST);   // abort, verdict[2]
+  volatile int* flags = reinterpret_cast<volatile int*>(bars + 3 * NST);   // abort, wait limit, verdict[2]
   const Ring ring{bars, bars + NST, bars + 2 * NST, flags};
-  ring_init(ring, NST, true);
+  ring_init(ring, NST, true, t.wait_limit);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   if (warp == kConsumerWarps) {                 // ---- loader
@@ -204,6 +204,7 @@ stream_pass1_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
         const int rows = min(c.geo.R, c.nrows - sr);
         if (k > 0) ok = warp_wait(ring.empty + s, (k - 1) & 1, ring.abort_flag, lane);
         if (!ok) break;
+        if (test_skips_stage(t, 1, it)) continue;     // test support: this stage's copies are left out, its waiters give up
         if (lane == 0) mbar_arrive_expect_tx(ring.full + s, 2u * rows * c.ncols * 4u);
         __syncwarp();
         load_slab(sG + s * kSlab, G, c, sr, rows, ring.full + s, lane, pol_first);
@@ -241,8 +242,8 @@ stream_pass1_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
     if (tiles[ti].pad) { pass1_plain_tile<RP>(t, tiles[ti]); continue; }
     const TileCtx c = tile_ctx<RP>(t, tiles[ti]);
     bool ok;
-    if (c.geo.qpt == 1) ok = pass1_consume<RP, NST, 1, Shape<RP>::RPT_NARROW>(t, c, ring, sG, sE, red, flags + 1, st);
-    else ok = pass1_consume<RP, NST, Shape<RP>::QPT_WIDE, Shape<RP>::RPT_WIDE>(t, c, ring, sG, sE, red, flags + 1, st);
+    if (c.geo.qpt == 1) ok = pass1_consume<RP, NST, 1, Shape<RP>::RPT_NARROW>(t, c, ring, sG, sE, red, flags + 2, st);
+    else ok = pass1_consume<RP, NST, Shape<RP>::QPT_WIDE, Shape<RP>::RPT_WIDE>(t, c, ring, sG, sE, red, flags + 2, st);
     if (!ok) return;
   }
 }
@@ -373,9 +374,9 @@ stream_pass3_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   float* sM = reinterpret_cast<float*>(smem_raw);
   uint64_t* bars = reinterpret_cast<uint64_t*>(sM + NST * kSlab);
-  volatile int* flags = reinterpret_cast<volatile int*>(bars + 3 * NST);
+  volatile int* flags = reinterpret_cast<volatile int*>(bars + 3 * NST);   // abort, wait limit
   const Ring ring{bars, bars + NST, bars + 2 * NST, flags};
-  ring_init(ring, NST, true);
+  ring_init(ring, NST, true, t.wait_limit);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int W = t.W;
 
@@ -397,6 +398,7 @@ stream_pass3_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
           const uint32_t k = it / NST;
           if (k > 0) ok = warp_wait(ring.empty + s, (k - 1) & 1, ring.abort_flag, lane);
           if (!ok) break;
+          if (test_skips_stage(t, 3, it)) continue;   // test support, as in pass 1
           if (lane == 0) mbar_arrive_expect_tx(ring.full + s, (uint32_t)rows * c.ncols * 4u);
           __syncwarp();
           load_slab(sM + s * kSlab, M0 + (size_t)w * plane, c, sr, rows, ring.full + s, lane, pol_first);

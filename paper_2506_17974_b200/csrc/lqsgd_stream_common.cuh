@@ -29,7 +29,14 @@ constexpr int kConsumers = kStreamConsumers;           // 512
 constexpr int kConsumerWarps = kConsumers / 32;        // 16
 constexpr int kThreads = kConsumers + 64;              // + loader warp + storer warp
 constexpr int kSlab = kStreamSlabFloats;               // floats per stage per array
-constexpr uint32_t kWaitLimit = 1u << 18;              // try_wait calls of <= ~1 us each
+constexpr uint32_t kWaitLimit = 1u << 18;              // try_wait calls of <= ~1 us each (the default limit)
+// The CTA's wait control lives in shared memory as consecutive ints: [0] the abort flag, [1] the limit of timed
+// polls per wait (kWaitLimit unless a test shortened it); the functions below take the address of [0].
+__device__ __forceinline__ void wait_ctl_init(volatile int* abort_flag, uint32_t limit_or_zero) {
+  abort_flag[0] = 0;
+  abort_flag[1] = (int)(limit_or_zero ? limit_or_zero : kWaitLimit);
+}
+__device__ __forceinline__ uint32_t wait_limit_of(volatile int* abort_flag) { return (uint32_t)abort_flag[1]; }
 constexpr uint32_t kStatusTimeout = 16u;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -56,7 +63,8 @@ __device__ __forceinline__ bool mbar_try(uint64_t* b, uint32_t parity) {
 // Bounded wait.  Returns false (and raises the abort flag) if the phase did not complete in
 // time, or as soon as another thread has raised the flag.
 __device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t i = 0; i < kWaitLimit; ++i) {
+  const uint32_t limit = wait_limit_of(abort_flag);
+  for (uint32_t i = 0; i < limit; ++i) {
     if (mbar_try(b, parity)) return true;
     if (*abort_flag) return false;
   }
@@ -125,14 +133,14 @@ struct Ring {
   volatile int* abort_flag;
 };
 
-__device__ __forceinline__ void ring_init(const Ring& r, int nst, bool stores) {
+__device__ __forceinline__ void ring_init(const Ring& r, int nst, bool stores, uint32_t wait_limit) {
   if (threadIdx.x == 0) {
     for (int s = 0; s < nst; ++s) {
       mbar_init(r.full + s, 1);                              // the loader's expect_tx arrival
       mbar_init(r.consumed + s, kConsumerWarps);
       mbar_init(r.empty + s, stores ? 1 : kConsumerWarps);   // storer, or the consumer warps directly
     }
-    *r.abort_flag = 0;
+    wait_ctl_init(r.abort_flag, wait_limit);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
   }
@@ -152,8 +160,9 @@ __device__ __forceinline__ void report_timeout(const Tables& t, int layer) { ato
 // flight; wait (bounded) for them so that no copy targets the CTA's memory after it exits.
 template <int NST>
 __device__ __forceinline__ void loader_drain(const Ring& r, uint32_t issued) {
+  const uint32_t limit = wait_limit_of(r.abort_flag);
   for (uint32_t it = issued > (uint32_t)NST ? issued - NST : 0; it < issued; ++it)
-    for (uint32_t i = 0; i < kWaitLimit && !mbar_try(r.full + (it % NST), (it / NST) & 1); ++i) {}
+    for (uint32_t i = 0; i < limit && !mbar_try(r.full + (it % NST), (it / NST) & 1); ++i) {}
 }
 
 // What every role needs to know about a tile, read once from the tables.

@@ -109,8 +109,9 @@ __device__ __forceinline__ bool thread_wait(uint64_t* b, uint32_t parity, volati
   return ok ? true : mbar_wait(b, parity, abort_flag);
 }
 // Bounded wait for a loader's copies that nobody will consume (abort path).
-__device__ __forceinline__ void drain(uint64_t* bar, uint32_t parity) {
-  for (uint32_t i = 0; i < kWaitLimit && !mbar_try(bar, parity); ++i) {}
+__device__ __forceinline__ void drain(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  const uint32_t limit = wait_limit_of(abort_flag);
+  for (uint32_t i = 0; i < limit && !mbar_try(bar, parity); ++i) {}
 }
 
 // Stages a tile takes: its rows in pieces of 32, rounded up to whole operand slots (a piece past
@@ -155,7 +156,7 @@ tc_pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, const uint
   uint64_t* d_empty = d_full + 2;                // [2] accumulator drained
   uint64_t* fin = d_empty + 2;                   // [1] every MMA of this CTA has completed
   volatile int* abort_flag = reinterpret_cast<volatile int*>(fin + 1);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(fin + 1) + 1;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(fin + 1) + 2;   // after the abort flag and the wait limit
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
@@ -163,7 +164,7 @@ tc_pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, const uint
     for (int s = 0; s < kTcAB; ++s) { mbar_init(ab_full + s, 4 * kTcPair + 1); mbar_init(ab_empty + s, 1); }
     for (int s = 0; s < 2; ++s) { mbar_init(d_full + s, 1); mbar_init(d_empty + s, 4); }
     mbar_init(fin, 1);
-    *abort_flag = 0;
+    wait_ctl_init(abort_flag, t.wait_limit);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
   }
@@ -187,6 +188,7 @@ tc_pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, const uint
       for (int k = 0; k < nk; ++k, ++kc) {
         const int s = kc % S::kMStages;
         if (!warp_wait(m_empty + s, ((kc / S::kMStages) & 1) ^ 1, abort_flag, lane)) { ok = false; break; }
+        if (test_skips_stage(t, 2, kc)) continue;     // test support: this piece is not fetched, its waiters give up
         if (lane == 0) {
           mbar_arrive_expect_tx(m_full + s, kTcMBytes);
           tma_load_3d(mring + (size_t)s * (kTcMBytes / 4), map, tl.col0, tl.row0 + k * kTcK, tl.worker, m_full + s);
@@ -195,7 +197,7 @@ tc_pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, const uint
     }
     if (!ok && lane == 0)
       for (uint32_t it = kc > (uint32_t)S::kMStages ? kc - S::kMStages : 0; it < kc; ++it)
-        drain(m_full + it % S::kMStages, (it / S::kMStages) & 1);
+        drain(m_full + it % S::kMStages, (it / S::kMStages) & 1, abort_flag);
   } else if (warp == 1) {
     // ---- B loader: rows [row0 + 32 k, +32) of the stacked P_bar terms
     uint32_t kc = 0;
@@ -216,7 +218,7 @@ tc_pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, const uint
       }
     }
     if (!ok && lane == 0)
-      for (uint32_t it = kc > (uint32_t)kTcAB ? kc - kTcAB : 0; it < kc; ++it) drain(ab_full + it % kTcAB, (it / kTcAB) & 1);
+      for (uint32_t it = kc > (uint32_t)kTcAB ? kc - kTcAB : 0; it < kc; ++it) drain(ab_full + it % kTcAB, (it / kTcAB) & 1, abort_flag);
   } else if (warp == 2) {
     // ---- MMA issue: one thread
     if (lane == 0) {
@@ -248,7 +250,7 @@ tc_pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, const uint
       }
       // every MMA issued so far must have completed before tensor memory is released
       tc_commit(fin);
-      drain(fin, 0);
+      drain(fin, 0, abort_flag);
     }
     __syncwarp();
   } else if (warp >= 4 && warp < 8) {
@@ -414,7 +416,7 @@ tc_pass1_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
   uint64_t* d_empty = d_full + 2;                // [2]
   uint64_t* fin = d_empty + 2;                   // [1]
   volatile int* abort_flag = reinterpret_cast<volatile int*>(fin + 1);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(fin + 1) + 1;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(fin + 1) + 2;   // after the abort flag and the wait limit
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int t_begin = cta_begin[blockIdx.x], t_end = cta_begin[blockIdx.x + 1];
@@ -423,7 +425,7 @@ tc_pass1_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
     for (int s = 0; s < kT1AB; ++s) { mbar_init(ab_full + s, 5); mbar_init(ab_empty + s, 1); }
     for (int s = 0; s < 2; ++s) { mbar_init(d_full + s, 1); mbar_init(d_empty + s, 4); }
     mbar_init(fin, 1);
-    *abort_flag = 0;
+    wait_ctl_init(abort_flag, t.wait_limit);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
   }
@@ -452,6 +454,7 @@ tc_pass1_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
       for (int k = 0; k < nk; ++k, ++kc) {
         const int s = kc % kT1Stages;
         if (!warp_wait(ge_empty + s, ((kc / kT1Stages) & 1) ^ 1, abort_flag, lane)) { ok = false; break; }
+        if (test_skips_stage(t, 1, kc)) continue;     // test support: this piece is not fetched, its waiters give up
         const int c0 = tl.col0 + k * kTcK;
         if (lane == 0) {
           mbar_arrive_expect_tx(ge_full + s, kT1PieceBytes);
@@ -475,7 +478,7 @@ tc_pass1_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
     }
     if (!ok && lane == 0)
       for (uint32_t it = kc > (uint32_t)kT1Stages ? kc - kT1Stages : 0; it < kc; ++it)
-        drain(ge_full + it % kT1Stages, (it / kT1Stages) & 1);
+        drain(ge_full + it % kT1Stages, (it / kT1Stages) & 1, abort_flag);
     asm volatile("cp.async.wait_all;" ::: "memory");
   } else if (warp == 1) {
     // ---- B loader: columns [c0, c0 + 32) of Q^T and of its remainders
@@ -495,7 +498,7 @@ tc_pass1_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
       }
     }
     if (!ok && lane == 0)
-      for (uint32_t it = kc > (uint32_t)kT1AB ? kc - kT1AB : 0; it < kc; ++it) drain(ab_full + it % kT1AB, (it / kT1AB) & 1);
+      for (uint32_t it = kc > (uint32_t)kT1AB ? kc - kT1AB : 0; it < kc; ++it) drain(ab_full + it % kT1AB, (it / kT1AB) & 1, abort_flag);
   } else if (warp == 2) {
     // ---- MMA issue: one thread
     if (lane == 0) {
@@ -524,7 +527,7 @@ tc_pass1_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
         }
       }
       tc_commit(fin);
-      drain(fin, 0);
+      drain(fin, 0, abort_flag);
     }
     __syncwarp();
   } else if (warp == 3) {
@@ -690,7 +693,7 @@ tc_pass3_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
   uint64_t* d_empty = d_full + 2;                // [2] all 16 consumer warps are past the tile
   uint64_t* fin = d_empty + 2;
   volatile int* abort_flag = reinterpret_cast<volatile int*>(fin + 1);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(fin + 1) + 1;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(fin + 1) + 2;   // after the abort flag and the wait limit
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int t_begin = cta_begin[blockIdx.x], t_end = cta_begin[blockIdx.x + 1];
@@ -700,7 +703,7 @@ tc_pass3_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
     mbar_init(op_full, 1); mbar_init(op_empty, 1);
     for (int s = 0; s < 2; ++s) { mbar_init(d_full + s, 1); mbar_init(d_empty + s, 4 * kT3Groups); }
     mbar_init(fin, 1);
-    *abort_flag = 0;
+    wait_ctl_init(abort_flag, t.wait_limit);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
   }
@@ -727,6 +730,7 @@ tc_pass3_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
         for (int pc = 0; pc < np; ++pc, ++kc) {
           const int s = kc % kT3Stages;
           if (!warp_wait(m_empty + s, ((kc / kT3Stages) & 1) ^ 1, abort_flag, lane)) { ok = false; break; }
+          if (test_skips_stage(t, 3, kc)) continue;   // test support, as in pass 1
           if (lane == 0) {
             mbar_arrive_expect_tx(m_full + s, kT1PieceBytes);
             tma_load_3d(piece(s), map, tl.col0 + pc * kTcK, tl.row0, w, m_full + s);
@@ -735,7 +739,7 @@ tc_pass3_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
     }
     if (!ok && lane == 0)
       for (uint32_t it = kc > (uint32_t)kT3Stages ? kc - kT3Stages : 0; it < kc; ++it)
-        drain(m_full + it % kT3Stages, (it / kT3Stages) & 1);
+        drain(m_full + it % kT3Stages, (it / kT3Stages) & 1, abort_flag);
   } else if (warp == 1) {
     // ---- operand loader: the tile's rows of the stacked P_bar terms and its columns' rows of the Q_bar terms
     uint32_t tseq = 0;
@@ -754,7 +758,7 @@ tc_pass3_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
         }
       }
     }
-    if (!ok && lane == 0 && tseq > 0) drain(op_full, (tseq - 1) & 1);
+    if (!ok && lane == 0 && tseq > 0) drain(op_full, (tseq - 1) & 1, abort_flag);
   } else if (warp == 2) {
     // ---- MMA issue: one thread, once per tile
     if (lane == 0) {
@@ -778,7 +782,7 @@ tc_pass3_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
         tc_commit(d_full + db);
       }
       tc_commit(fin);
-      drain(fin, 0);
+      drain(fin, 0, abort_flag);
     }
     __syncwarp();
   } else if (warp == 3) {

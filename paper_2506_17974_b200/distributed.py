@@ -1,7 +1,6 @@
 """One LQ-SGD round with the workers spread over several processes / GPUs.
 
-Algorithm 1 exchanges the quantised factors twice per iteration ("All-Reduce P_quant", "All-Reduce
-Q_quant").  Each rank simulates `workers` local workers with the CUDA library; this module only
+Algorithm 1 exchanges the quantised factors twice per iteration (its two All-Reduce steps, Section IV-A).  Each rank simulates `workers` local workers with the CUDA library; this module only
 sequences the library's round pieces and the collectives between them on torch.distributed
 (NCCL on GPUs): a MAX all-reduce of one scale per matrix and an all-gather of the packed b-bit
 streams, per factor.  The wire therefore carries r(n+m)b bits per worker (Section IV-C) plus the

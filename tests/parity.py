@@ -16,6 +16,29 @@ from paper_2506_17974_b200 import binding as B
 
 TOL = 1e-4          # relative Frobenius error allowed on P, Q, G_hat, E
 MAX_FLIP_FRACTION = 1e-5
+# Stage-isolated: both sides quantise the SAME fp32 factor with the SAME fp32 scale, so the only
+# legitimate difference is an element whose |x|/s lies within an fp32 ulp of a decision threshold;
+# the gate is that many ulps of |x|/s, converted to level units element by element.
+STAGE_ULPS = 4.0
+# Free-running: the oracle's factor differs from the device's by the fp32 rounding of everything
+# upstream, so codes next to a threshold may differ; the oracle adopts the device's code there.
+# Gates: distance from the threshold in level units, and the fraction of codes adopted (set to
+# about ten times the largest values observed over the whole suite, which the tests print).
+FREE_MARGIN = 2e-2
+FREE_FRACTION = 2e-3
+
+ALL_STATS = []      # one dict per test that ran run-level statistics (written out at session end)
+
+
+def level_ulp(x_dev, s, bits, alpha):
+    """One fp32 ulp of t = |x|/s expressed in level units: ulp(t) * d/dt[(L-1) log(1+alpha t)/log(1+alpha)]."""
+    L = orc.magnitude_levels(bits)
+    x32 = np.abs(np.asarray(x_dev, dtype=np.float32))
+    s32 = np.asarray(s, dtype=np.float32)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        t = np.where(np.broadcast_to(s32 == 0, x32.shape), np.float32(0), (x32 / s32).astype(np.float32))
+    slope = (L - 1) * alpha / ((1.0 + alpha * t.astype(np.float64)) * np.log1p(alpha))
+    return np.spacing(t).astype(np.float64) * slope
 
 
 def rel_fro(a, b):
@@ -69,7 +92,10 @@ def check_exchange(x_dev, codes_dev, scale_dev, bar_dev, bits, alpha, stats, ave
         bad = c != codes_dev[w]
         if bad.any():
             # a legitimate difference sits on a threshold (within fp32 resolution of |x|/s)
-            assert np.all(margin[bad] < 1e-4), ("codes differ away from a threshold", margin[bad].max())
+            ulp = level_ulp(x_dev[w], s, bits, alpha)
+            assert np.all(margin[bad] <= STAGE_ULPS * ulp[bad]), (
+                "codes differ away from a threshold", float((margin[bad] / ulp[bad]).max()))
+            stats["flip_margin_ulps"] = max(stats.get("flip_margin_ulps", 0.0), float((margin[bad] / ulp[bad]).max()))
             k_o = c[bad].astype(int) & ((1 << (bits - 1)) - 1)
             k_d = codes_dev[w][bad].astype(int) & ((1 << (bits - 1)) - 1)
             assert np.all(np.abs(k_o - k_d) <= 1)
@@ -185,14 +211,18 @@ def oracle_step_forced(oracle: orc.Oracle, grads_host, recs, stats):
         for w in range(oracle.W):
             diff = codes_differ(res["xp"]["codes"][w], rec.codes_p[w], oracle.bits_p)
             stats["forced"] = stats.get("forced", 0) + int(diff.sum())
-            assert np.all(res["xp"]["margin"][w][diff] < 2e-2), "P code differs far from a threshold"
+            if diff.any():
+                stats["forced_margin"] = max(stats.get("forced_margin", 0.0), float(res["xp"]["margin"][w][diff].max()))
+            assert np.all(res["xp"]["margin"][w][diff] < FREE_MARGIN), "P code differs far from a threshold"
             fp.append(np.where(diff, rec.codes_p[w].astype(np.int16), -1))
         res = orc.layer_round(*args, forced_p=fp, **kw)
         fq = []
         for w in range(oracle.W):
             diff = codes_differ(res["xq"]["codes"][w], rec.codes_q[w], oracle.bits_q)
             stats["forced"] = stats.get("forced", 0) + int(diff.sum())
-            assert np.all(res["xq"]["margin"][w][diff] < 2e-2), "Q code differs far from a threshold"
+            if diff.any():
+                stats["forced_margin"] = max(stats.get("forced_margin", 0.0), float(res["xq"]["margin"][w][diff].max()))
+            assert np.all(res["xq"]["margin"][w][diff] < FREE_MARGIN), "Q code differs far from a threshold"
             fq.append(np.where(diff, rec.codes_q[w].astype(np.int16), -1))
         forced[l] = (fp, fq)
         stats["free_codes"] = stats.get("free_codes", 0) + sum(c.size for c in rec.codes_p + rec.codes_q)

@@ -3,6 +3,7 @@ on the same seeded inputs.  Tolerances: relative Frobenius error <= 1e-4 on P, Q
 codes bit-exact except elements on a decision threshold, whose fraction (<= 1e-5) is counted;
 payload bytes exact."""
 import dataclasses
+import time
 
 import numpy as np
 import pytest
@@ -28,14 +29,16 @@ def new_oracle(comp: B.LQSGD):
                       quantize_vectors=comp.quantize_vectors, column_scales=comp.column_scales)
 
 
-def run_steps(w: wl.Workload, steps: int, free_run=True, comp=None):
+def run_steps(w: wl.Workload, steps: int, free_run=True, comp=None, allow_status=0):
+    """allow_status: status bits the data may legitimately raise (a dependent column or a zero scale with
+    very coarse codes); which columns are dropped is still compared with the oracle stage by stage."""
     comp = comp or make(w)
     stats = {}
     oracle = new_oracle(comp) if free_run else None
     for t in range(steps):
         grads = wl.draw_gradients(w, t, device=DEV)
         recs, grads_host, ghat = par.device_step_checked(comp, grads, stats)
-        assert all(f == 0 for f in comp.status()), comp.status()
+        assert all(f & ~allow_status == 0 for f in comp.status()), comp.status()
         if free_run:
             out = par.oracle_step_forced(oracle, grads_host, recs, stats)
             for l, rec in recs.items():
@@ -43,10 +46,16 @@ def run_steps(w: wl.Workload, steps: int, free_run=True, comp=None):
                 assert par.rel_fro(rec.E_new, out[l]["E_new"]) <= par.TOL, (t, l)
                 assert par.rel_fro(rec.Q_bar, out[l]["Q_bar"]) <= par.TOL, (t, l)
                 assert par.rel_fro(rec.P_bar, out[l]["P_bar"]) <= par.TOL, (t, l)
-    assert stats["flips"] <= max(1, par.MAX_FLIP_FRACTION * stats["codes"]), stats
+    # codes: bit-exact on identical inputs except elements on a decision threshold, fraction <= 1e-5
+    assert stats["flips"] <= par.MAX_FLIP_FRACTION * stats["codes"], stats
+    stats["flip_fraction"] = stats["flips"] / stats["codes"]
     if free_run:
-        assert stats.get("forced", 0) <= max(2, 2e-3 * stats["free_codes"]), stats
-    print({k: (f"{v:.2e}" if isinstance(v, float) else v) for k, v in stats.items()})
+        assert stats.get("forced", 0) <= par.FREE_FRACTION * stats["free_codes"], stats
+        stats["forced_fraction"] = stats.get("forced", 0) / stats["free_codes"]
+    shown = {k: (f"{v:.2e}" if isinstance(v, float) else v) for k, v in stats.items()}
+    print(w.name, shown)
+    par.ALL_STATS.append(dict(stats, workload=w.name, rank=comp.rank, bits_p=comp.bits_p, bits_q=comp.bits_q,
+                              workers=comp.W, steps=steps, free_run=free_run))
     return comp, stats
 
 
@@ -67,16 +76,28 @@ def test_config4_large_layers(rows, cols):
     run_steps(wl.config4(rows, cols), 2)
 
 
-@pytest.mark.parametrize("rank,bits", [(1, 2), (2, 3), (4, 4), (8, 8), (16, 8), (16, 2)])
-def test_config5_rank_bit_points(rank, bits):
-    w = dataclasses.replace(wl.config5(rank, bits), workers=4)      # full shapes, fewer workers
-    run_steps(w, 1, free_run=False)
+def test_config4_4096x16384_stage_isolated():
+    """The third size of the large-layer sweep: every stage of one round against the oracle."""
+    run_steps(wl.config4(4096, 16384), 1, free_run=False)
 
 
-@pytest.mark.parametrize("rank", [2, 16])
-def test_config5_sixteen_workers(rank):
-    """rank 16 puts the aligned layers on the tensor-core pass 2 with all 16 workers' tiles in one launch."""
-    run_steps(wl.config5(rank, 4), 1, free_run=False)
+# With one magnitude bit (b = 2) the averaged factors take few distinct values: from the second round on a
+# column of M Q can come out dependent, or a factor all zero.  That is the data, not a fault.
+COARSE_OK = B.STATUS_DEPENDENT_COLUMN | B.STATUS_ZERO_SCALE_P | B.STATUS_ZERO_SCALE_Q
+
+
+@pytest.mark.parametrize("bits", [2, 3, 4, 8])
+@pytest.mark.parametrize("rank", [1, 2, 4, 8, 16])
+def test_config5_rank_bit_grid_sixteen_workers(rank, bits):
+    """Every (r, b) point of the rank / bit sweep at its full size (16 workers, ResNet-18 with 100 classes),
+    one round, every stage against the oracle.  Rank 16 runs the products on the tensor cores."""
+    run_steps(wl.config5(rank, bits), 1, free_run=False)
+
+
+@pytest.mark.parametrize("rank,bits", [(1, 2), (1, 8), (16, 2), (16, 8)])
+def test_config5_corners_free_running(rank, bits):
+    """The four corners of the grid, two rounds with the oracle running free beside the device."""
+    run_steps(wl.config5(rank, bits), 2, allow_status=COARSE_OK if bits == 2 else 0)
 
 
 @pytest.mark.parametrize("name", ["mnist", "resnet", "large", "rank8_workers3"])
@@ -399,6 +420,46 @@ def test_non_finite_gradient_is_flagged_without_a_fault(rank):
     assert b.status() == [0, 0]
 
 
+@pytest.mark.parametrize("rank,pass_", [(2, 1), (2, 3), (8, 1), (8, 3), (16, 1), (16, 2), (16, 3)])
+def test_bounded_wait_runs_out_and_reports_timeout(rank, pass_):
+    """The path a bounded device-side wait takes when it runs out (ranks 2 and 8: the bulk-copy staged passes,
+    rank 16: the tcgen05 passes).  The test hook makes CTA 0's loader leave out one stage of copies and shortens
+    the limit of the waits; nothing faults or spins without a limit: the kernel returns, the layer's status word
+    carries LQSGD_STATUS_TIMEOUT, and once E and Q are restored the context computes, bit for bit, what a fresh
+    context computes - which is checked against the oracle."""
+    layers = ((256, 512), (24, 1))
+    w = wl.Workload("expire", layers, rank=rank, bits=4, workers=2, steps=3, dist="normal", scale="fan_in", seed=6)
+    comp, ref = make(w), make(w)
+    out = [torch.empty(s, device=DEV) for s in layers]
+    out_ref = [torch.empty(s, device=DEV) for s in layers]
+    comp.test_expire_wait(pass_, 0, 256)
+    t0 = time.time()
+    comp.step(wl.draw_gradients(w, 0, device=DEV), out)
+    torch.cuda.synchronize()
+    assert time.time() - t0 < 10.0                              # the waits gave up, nothing hung
+    st = comp.status()
+    assert st[0] & B.STATUS_TIMEOUT, st
+    # the hook armed that one step only; restore the state a time-out leaves undefined
+    for k in range(2):
+        comp.set_state(B.STATE_E, 0, k, torch.zeros(layers[0], device=DEV))
+    comp.set_state(B.STATE_Q, 0, 0, ref.get_state(B.STATE_Q, 0))
+    for t in (1, 2):
+        g = wl.draw_gradients(w, t, device=DEV)
+        comp.step(g, out)
+        ref.step(g, out_ref)
+        torch.cuda.synchronize()
+        assert comp.status() == [0, 0] and ref.status() == [0, 0]
+        for x, y in zip(out, out_ref):
+            assert torch.equal(x, y)
+        for k in range(2):
+            assert torch.equal(comp.payload(k), ref.payload(k))
+            assert torch.equal(comp.get_state(B.STATE_E, 0, k), ref.get_state(B.STATE_E, 0, k))
+    par.device_step_checked(comp, wl.draw_gradients(w, 3, device=DEV), {})      # and against the oracle
+    assert comp.status() == [0, 0]
+    with pytest.raises(B.LqsgdError):                          # limits outside 16 .. 2^18 are refused
+        comp.test_expire_wait(1, 0, 8)
+
+
 @pytest.mark.parametrize("rank", [4, 16])
 def test_bit_reproducible_and_checkpoint_resume(rank):
     w = dataclasses.replace(wl.config2(), workers=3, rank=rank)
@@ -488,6 +549,37 @@ def test_step_replays_from_a_cuda_graph():
     assert torch.equal(a.get_state(B.STATE_E, 2, 1), b.get_state(B.STATE_E, 2, 1))
 
 
+def test_captured_pointer_tables_can_be_released():
+    """Every capture pins its pointer table; after 16 of them a new pointer set is refused until the caller
+    declares its graphs destroyed."""
+    w = wl.Workload("pins", ((32, 64), (8, 1)), rank=2, bits=4, workers=1, steps=1, dist="normal", scale="fan_in")
+    comp = make(w)
+    out = [torch.empty(s, device=DEV) for s in w.layers]
+    keep = []
+
+    def capture_one():
+        g = wl.draw_gradients(w, len(keep), device=DEV)
+        keep.append(g)
+        arrs = comp.make_pointer_arrays(g, out)
+        comp.step_ptrs(*arrs)                                    # eager: uploads the table
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, capture_error_mode="thread_local"):
+            comp.step_ptrs(*arrs, torch.cuda.current_stream())
+        return graph
+
+    graphs = [capture_one() for _ in range(16)]
+    g = wl.draw_gradients(w, 99, device=DEV)
+    with pytest.raises(B.LqsgdError) as e:
+        comp.step(g, out)
+    assert e.value.code == B.ERR_CAPTURE
+    del graphs
+    comp.release_graph_tables()
+    comp.step(g, out)
+    torch.cuda.synchronize()
+    assert all(s == 0 for s in comp.status())
+
+
 def test_step_host_matches_device_step():
     w = dataclasses.replace(wl.config2(), workers=2)
     a, b = make(w), make(w, host_staging=True)
@@ -505,6 +597,20 @@ def test_step_host_matches_device_step():
     with pytest.raises(B.LqsgdError) as e:
         a.step_host(g_host, out_b, pay)
     assert e.value.code == B.ERR_NO_STAGING
+    # one flat pinned buffer per worker, tensors on 16-byte boundaries: the copies merge, the result is the same
+    offs, total = [], 0
+    for s in w.layers:
+        offs.append(total)
+        total += (s[0] * s[1] + 3) // 4 * 4
+    flat = [torch.empty(total).pin_memory() for _ in range(3)]
+    views = [[f[o:o + s[0] * s[1]].view(s) for o, s in zip(offs, w.layers)] for f in flat]
+    for k in range(2):
+        for v, x in zip(views[k], g[k]):
+            v.copy_(x)
+    c = make(w, host_staging=True)
+    c.step_host(views[:2], views[2], pay)
+    for x, y in zip(out_a, views[2]):
+        assert torch.equal(x.cpu(), y)
 
 
 def test_argument_errors_launch_nothing():

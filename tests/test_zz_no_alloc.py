@@ -10,6 +10,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import lqsgd_oracle as orc
 from paper_2506_17974_b200 import binding as B
 from paper_2506_17974_b200 import workloads as wl
 import parity as par
@@ -41,6 +42,7 @@ def test_no_alloc_orthonormalize_matches_workspace_path_twice():
         torch.cuda.synchronize()
         assert int(status.item()) == 0
         assert par.rel_fro(par.host(out), par.host(ref)) <= par.TOL
+        assert par.rel_fro(par.host(out), orc.orthonormalize(par.host(raw))[0]) <= par.TOL   # and the CPU oracle's
         gram = par.host(out).astype(np.float64)
         assert np.max(np.abs(gram.T @ gram - np.eye(raw.shape[1]))) < 1e-5
     # in place
@@ -63,6 +65,22 @@ def test_no_alloc_reports_dependent_column_and_clears_it_on_the_next_call():
     B.orthonormalize_noalloc(y, out, status)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
+
+
+@pytest.mark.parametrize("rows", [B.NOALLOC_MAX_ROWS, B.NOALLOC_MAX_ROWS - 127])
+def test_no_alloc_largest_accepted_sizes(rows):
+    """The last block's Gram matrix sits right before R^-1 in the fixed array: at the largest sizes the
+    result must still be orthonormal, equal to the oracle's, and report no condition."""
+    x = torch.randn(rows, 16, device=DEV, generator=torch.Generator(DEV).manual_seed(rows))
+    out = torch.empty_like(x)
+    status = torch.full((1,), 99, dtype=torch.int32, device=DEV)
+    for _ in range(2):
+        B.orthonormalize_noalloc(x, out, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    q = par.host(out).astype(np.float64)
+    assert np.max(np.abs(q.T @ q - np.eye(16))) < 1e-5
+    assert par.rel_fro(q, orc.orthonormalize(par.host(x))[0]) <= par.TOL
 
 
 def test_no_alloc_rejects_sizes_beyond_its_fixed_scratch():
