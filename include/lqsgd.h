@@ -95,6 +95,16 @@ typedef enum lqsgd_error {
                                         any column's scale is 0 (that column's codes and averages are 0).  Not available
                                         with workers on several GPUs (lqsgd_round_begin refuses). */
 
+#define LQSGD_FLAG_ONE_LAUNCH 32u /* run the round as ONE cooperative kernel that keeps M = G + E in the SMs' shared memory
+                                     from the first product to the error update (12 + 4/W instead of 24 + 4/W bytes of
+                                     memory traffic per worker-element), when the set qualifies: W * sum(n m) fp32 values
+                                     fit in the shared memory of all SMs together (about 27 MB on a B200), rank <= 8,
+                                     plain Algorithm 1 exchange or its variants except quantised 1-D tensors, one power
+                                     iteration, all workers on this GPU.  A set that does not qualify runs as the usual
+                                     sequence of kernels (lqsgd_launches_per_step tells which: 1 = one launch).  Same
+                                     results up to the order of the floating-point sums.  Off by default: the sequence of
+                                     kernels is the faster of the two on the sets measured so far. */
+
 typedef struct lqsgd_ctx lqsgd_ctx;
 
 typedef struct lqsgd_shape {
@@ -287,13 +297,24 @@ int lqsgd_set_phase_events(lqsgd_ctx* ctx, void* const* host_events);
  * after a fixed number of timed polls, the CTA's roles then leave their loops, copies in flight are waited for,
  * tensor memory is released, the layer's status word gets LQSGD_STATUS_TIMEOUT and the kernel returns.  This
  * call arms the NEXT step only: in pass `pass` (1, 2 or 3; pass 2 only where it runs on the tensor cores) the
- * loader of CTA 0 leaves out the copies of its stage number `stage` (counted from 0 over the CTA's tiles), and
+ * loader of CTA 0 issues no copies from its stage number `stage` on (counted from 0 over the CTA's tiles); with
+ * pass = 4 (a context that runs the round as one launch) CTA 0 stays away from grid barrier number `stage`; and
  * every bounded wait of that step gives up after `wait_limit` polls (16 .. 2^18, about a microsecond each)
  * instead of the built-in 2^18.  All addresses stay valid and nothing spins without a limit; the step's outputs
  * (E of the affected layer included) are undefined, as after any time-out: restore E and Q with
  * lqsgd_set_state, or use a fresh context, before relying on results again.  If the armed pass has no such
  * stage the step runs normally.  Host-only; never needed in production. */
 int lqsgd_test_expire_wait(lqsgd_ctx* ctx, int32_t pass, int32_t stage, uint32_t wait_limit);
+
+/* Profiling aid for contexts that run the round as ONE launch (see LQSGD_FLAG_ONE_LAUNCH), where no event can be
+ * recorded between the steps: the kernel itself notes the GPU's global timer (nanoseconds) as its first CTA starts,
+ * ends its pass 1, leaves each grid barrier, and ends.  Copies the stamps of the last completed round into
+ * host_ns[LQSGD_TIMELINE_MAX] and their number into *host_count (0 for a multi-kernel context); synchronises
+ * cuda_stream.  Stamps, in order: start | end of pass 1 on CTA 0 | Orthonormalize begins | (with tall layers:
+ * Cholesky and solve begin; else the same instant as the next) | P_bar and pass 2 begin | Q_w reduction begins |
+ * Q_bar and pass 3 begin | end. */
+#define LQSGD_TIMELINE_MAX 12
+int lqsgd_round_timeline(const lqsgd_ctx* ctx, uint64_t* host_ns, int32_t* host_count, void* cuda_stream);
 
 /* Kernel launches one lqsgd_step enqueues (for launch accounting). */
 int lqsgd_launches_per_step(const lqsgd_ctx* ctx, int32_t* host_out);

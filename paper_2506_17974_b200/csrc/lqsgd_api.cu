@@ -73,6 +73,15 @@ struct Plan {
   std::vector<Tile> tctiles3;                    // tensor-core pass 3 (all workers per tile), grouped by CTA
   std::vector<int> tcbegin3;
   int tc_grid = 0;
+  bool resident = false;                         // the one-launch round takes this set (lqsgd_resident.cu)
+  std::vector<ResTile> rtiles;                   // its tiles, grouped by CTA
+  std::vector<int> rbegin;                       // [res_grid + 1]
+  int res_grid = 0;
+  size_t res_smem = 0;                           // dynamic shared memory per CTA
+  ResTile* d_rtiles = nullptr;
+  int* d_rbegin = nullptr;
+  uint32_t* d_rsync = nullptr;                   // launch counter + two sets of grid-barrier counters
+  uint64_t* d_rstamps = nullptr;                 // timeline of the last one-launch round
   std::vector<uint8_t> tcmaps;                   // tensor maps of the tensor-core passes (filled at create)
   std::vector<FactorBlock> fbP, fbQ;             // 128-row blocks of P (layers orthonormalised in two launches) and of Q
   std::vector<FactorBlock> fbS;                  // (layer, worker) of the layers orthonormalised by one CTA
@@ -128,7 +137,7 @@ int check_config(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
     if (c->world_workers > c->workers && (c->bits_p == 32 || c->bits_q == 32)) return LQSGD_ERR_INVALID_ARG;
   }
   if (c->flags & ~(LQSGD_FLAG_HOST_STAGING | LQSGD_FLAG_REGISTER_PATH | LQSGD_FLAG_AVERAGE_VALUES |
-                   LQSGD_FLAG_QUANTIZE_VECTORS | LQSGD_FLAG_COLUMN_SCALES))
+                   LQSGD_FLAG_QUANTIZE_VECTORS | LQSGD_FLAG_COLUMN_SCALES | LQSGD_FLAG_ONE_LAUNCH))
     return LQSGD_ERR_INVALID_ARG;
   for (int i = 0; i < n_layers; ++i) {
     if (shapes[i].rows < 1 || shapes[i].cols < 1) return LQSGD_ERR_BAD_SHAPE;
@@ -190,9 +199,111 @@ double makespan_strided(const std::vector<double>& cost, size_t ctas) {
   return cost.empty() ? 0.0 : *std::max_element(load.begin(), load.end());
 }
 
+// Shared memory one CTA may ask for on this architecture (227 KB).
+constexpr size_t kMaxSmemPerCta = 227 * 1024;
+
+// Plan of the one-launch round (lqsgd_resident.cu): cuts every (layer, worker) into tiles that stay in shared
+// memory from pass 1 to pass 3 and deals them to one CTA per SM.  Returns false when the set does not qualify:
+// too large for the SMs' shared memory together, or a configuration the one-launch kernel does not take.
+// On success fills p.rtiles / p.rbegin / p.res_grid / p.res_smem and ncc[li], nrb[li] (chunks of the partial sums).
+bool plan_resident(const lqsgd_config& cfg, int sm_count, Plan& p, std::vector<int>& ncc, std::vector<int>& nrb) {
+  const int W = p.W, RP = p.RP;
+  if (!(cfg.flags & LQSGD_FLAG_ONE_LAUNCH) || (cfg.flags & LQSGD_FLAG_REGISTER_PATH)) return false;
+  if ((cfg.flags & LQSGD_FLAG_QUANTIZE_VECTORS) && cfg.bits_p != 32) return false;
+  if (RP > 8 || p.W_total != W || cfg.power_iters > 1 || p.mats.empty() || sm_count < 8) return false;
+  const size_t fixed = resident_scratch_bytes(RP);
+  if (fixed == 0 || fixed + 16384 > kMaxSmemPerCta) return false;
+  const size_t cap = (kMaxSmemPerCta - fixed) / 4 / 4 * 4;            // floats of tiles per CTA
+  size_t F = 0, rows_total = 0;
+  for (auto& mt : p.mats) {
+    if (mt.m % 4 != 0 && (size_t)mt.n * mt.m > (size_t)kStreamPlainElems) return false;
+    if (mt.m % 4 != 0 && mt.m > kResMaxTileCols) return false;
+    F += (size_t)W * mt.n * mt.m;
+    rows_total += (size_t)W * mt.n;
+  }
+  if ((double)F > 0.96 * (double)cap * sm_count) return false;
+  // the steps between the passes are spread over the CTAs in blocks of 128 rows or 256 elements: a set with very
+  // tall factors would make them, not the passes, the long part
+  if (rows_total * RP > (size_t)1 << 20) return false;
+  const double fill = (double)F / ((double)cap * sm_count);
+  // Tile size: one tile per CTA of the large layers when the set leaves some room (fewest partial sums, one long
+  // stream per CTA); a set that nearly fills the shared memory is cut finer so that the tiles pack.  A layer much
+  // smaller than a tile stays whole.  Tiles are as wide as a row copy should be (up to kResMaxTileCols columns).
+  const int per_cta = fill <= 0.88 ? 1 : 8;
+  double T = std::max(8192.0, (double)F / ((double)sm_count * per_cta));
+  std::vector<ResTile> tiles;
+  for (int attempt = 0; attempt < 60; ++attempt, T *= 1.03) {
+    tiles.clear();
+    size_t big_tiles = 0;
+    for (size_t li = 0; li < p.mats.size(); ++li) {
+      const MatHost& mt = p.mats[li];
+      const bool plain = mt.m % 4 != 0;
+      int cols = mt.m, nc = 1;
+      if (!plain && mt.m > kResMaxTileCols) {
+        nc = ceil_div(mt.m, kResMaxTileCols);
+        cols = (int)align_up((size_t)ceil_div(mt.m, nc), 4);
+        nc = ceil_div(mt.m, cols);
+      }
+      int rows = (int)std::min<double>(kResMaxTileRows, std::max(1.0, std::floor(T / cols)));
+      rows = std::min(rows, mt.n);
+      const int nr = ceil_div(mt.n, rows);
+      rows = ceil_div(mt.n, nr);
+      ncc[li] = nc;
+      nrb[li] = nr;
+      if ((double)rows * cols > 0.5 * T) big_tiles += (size_t)W * nr * nc;
+      for (int w = 0; w < W; ++w)
+        for (int rb = 0; rb < nr; ++rb)
+          for (int cc = 0; cc < nc; ++cc) {
+            ResTile tl{};
+            tl.layer = (int)li; tl.worker = w;
+            tl.row0 = rb * rows; tl.nrows = std::min(rows, mt.n - rb * rows);
+            tl.col0 = cc * cols; tl.ncols = std::min(cols, mt.m - cc * cols);
+            tl.part_c = cc; tl.part_r = rb;
+            tl.plain = plain ? 1 : 0;
+            tl.writes_ghat = (w == 0) ? 1 : 0;
+            tiles.push_back(tl);
+          }
+    }
+    // one tile per CTA: the large tiles must not need a second round of CTAs
+    if (per_cta > 1 || big_tiles <= (size_t)sm_count || T > (double)cap) break;
+  }
+  // longest tile first to the CTA with the least so far
+  std::vector<int> order(tiles.size());
+  for (size_t i = 0; i < order.size(); ++i) order[i] = (int)i;
+  auto fl = [&](const ResTile& tl) { return align_up((size_t)tl.nrows * tl.ncols, 4); };
+  std::stable_sort(order.begin(), order.end(), [&](int x, int y) { return fl(tiles[x]) > fl(tiles[y]); });
+  std::vector<std::vector<int>> per(sm_count);
+  std::vector<size_t> load(sm_count, 0);
+  for (int i : order) {
+    int best = -1;
+    for (int b = 0; b < sm_count; ++b)
+      if ((int)per[b].size() < kResMaxTiles && load[b] + fl(tiles[i]) <= cap && (best < 0 || load[b] < load[best])) best = b;
+    if (best < 0) return false;
+    per[best].push_back(i);
+    load[best] += fl(tiles[i]);
+  }
+  p.rtiles.clear();
+  p.rbegin.assign(sm_count + 1, 0);
+  size_t most = 0;
+  for (int b = 0; b < sm_count; ++b) {
+    size_t off = 0;
+    for (int i : per[b]) {
+      ResTile tl = tiles[i];
+      tl.smem_off = (int)off;
+      off += fl(tl);
+      p.rtiles.push_back(tl);
+    }
+    most = std::max(most, off);
+    p.rbegin[b + 1] = (int)p.rtiles.size();
+  }
+  p.res_grid = sm_count;
+  p.res_smem = fixed + most * 4;
+  return true;
+}
+
 // Lays out the workspace and builds every table.  base == nullptr: size only.
 void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg, void* base, int sm_count,
-               Plan& p) {
+               Plan& p, bool allow_resident = true) {
   const int W = cfg.workers, RP = padded_rank(cfg.rank);
   p.RP = RP;
   p.W = W;
@@ -239,6 +350,10 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
     p.region_off[1] = first.q_offset; p.region_bytes[1] = last.q_offset + last.q_bytes - first.q_offset;
   }
   p.payload_stride = align_up(off, 16);
+
+  // ---- a set small enough for the SMs' shared memory runs as one launch; its tiles decide the chunking below
+  std::vector<int> res_ncc(p.mats.size(), 1), res_nrb(p.mats.size(), 1);
+  p.resident = allow_resident && plan_resident(cfg, sm_count, p, res_ncc, res_nrb);
 
   // ---- tile sizes
   const size_t slots = (size_t)sm_count * 2, want = 3 * slots;
@@ -295,11 +410,11 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   // wider layers get chunks balanced in units of 128 columns.  Row chunks hold a target number
   // of elements and are multiples of the rows one stage takes.
   auto staged = [&](const MatHost& mt) {
-    return !(cfg.flags & LQSGD_FLAG_REGISTER_PATH) && RP <= kStreamMaxRP && mt.m % 4 == 0;
+    return !p.resident && !(cfg.flags & LQSGD_FLAG_REGISTER_PATH) && RP <= kStreamMaxRP && mt.m % 4 == 0;
   };
   // A small layer with unaligned rows rides in the staged kernels as plain tiles (no launch of its own).
   auto plain = [&](const MatHost& mt) {
-    return !(cfg.flags & LQSGD_FLAG_REGISTER_PATH) && RP <= kStreamMaxRP && mt.m % 4 != 0 &&
+    return !p.resident && !(cfg.flags & LQSGD_FLAG_REGISTER_PATH) && RP <= kStreamMaxRP && mt.m % 4 != 0 &&
            (size_t)mt.n * mt.m <= (size_t)kStreamPlainElems;
   };
   // Tensor-core passes: padded rank 16, rows 16-byte aligned.
@@ -393,8 +508,8 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
     const int tr2 = tc ? (int)align_up((size_t)balanced_rows(mt.n, kTcRowChunk), 64) : balanced_rows(mt.n, r2);
     // tensor-core pass 1: column chunks balanced in units of 32 columns, at most kTcPass1Cols wide
     const int tc_units = ceil_div(mt.m, 32), tc_ncc = ceil_div(tc_units * 32, kTcPass1Cols);
-    L.ncc = tc ? tc_ncc : (st ? (int)scols.size() : (pl ? 1 : ceil_div(mt.m, cw)));
-    L.nrb = ceil_div(mt.n, tr2);
+    L.ncc = p.resident ? res_ncc[li] : (tc ? tc_ncc : (st ? (int)scols.size() : (pl ? 1 : ceil_div(mt.m, cw))));
+    L.nrb = p.resident ? res_nrb[li] : ceil_div(mt.n, tr2);
     L.npb = ceil_div(mt.n, kFactorBlockRows);
     L.nqb = ceil_div(mt.m, kFactorBlockRows);
     const size_t nm = (size_t)mt.n * mt.m;
@@ -455,7 +570,7 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
       for (int cb = 0; cb < ceil_div(mt.m, 128); ++cb)
         p.tctiles3.push_back({li32, 0, rb * kTcRowsPerTile, std::min(kTcRowsPerTile, mt.n - rb * kTcRowsPerTile), cb * 128,
                               std::min(128, mt.m - cb * 128), 0, 0});
-    for (int rb = 0; !st && !tc && !pl && rb < ceil_div(mt.n, kPass1Rows); ++rb)
+    for (int rb = 0; !p.resident && !st && !tc && !pl && rb < ceil_div(mt.n, kPass1Rows); ++rb)
       for (int cc = 0; cc < L.ncc; ++cc)
         for (int w = 0; w < W; ++w) {
           const int row0 = rb * kPass1Rows, col0 = cc * cw;
@@ -466,7 +581,7 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
       for (int rb = 0; rb < L.nrb; ++rb)
         for (int cc = 0; cc < ceil_div(mt.m, cw2); ++cc) {
           const int row0 = rb * tr2, col0 = cc * cw2;
-          if (tc) continue;
+          if (tc || p.resident) continue;
           p.tiles2.push_back({li32, w, row0, std::min(tr2, mt.n - row0), col0, std::min(cw2, mt.m - col0), rb, 0});
         }
     for (int w = 0; tc && w < W; ++w)
@@ -476,7 +591,7 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
           p.tctiles2.push_back({li32, w, row0, std::min(tr2, mt.n - row0), col0, std::min(128, mt.m - col0), rb, 0});
         }
     const int tr3 = balanced_rows(mt.n, r3);
-    for (int rb = 0; !st && !tc && !pl && rb < ceil_div(mt.n, tr3); ++rb)
+    for (int rb = 0; !p.resident && !st && !tc && !pl && rb < ceil_div(mt.n, tr3); ++rb)
       for (int cc = 0; cc < ceil_div(mt.m, cw2); ++cc) {
         const int row0 = rb * tr3, col0 = cc * cw2;
         p.tiles3.push_back({li32, 0, row0, std::min(tr3, mt.n - row0), col0, std::min(cw2, mt.m - col0), 0, 0});
@@ -525,6 +640,8 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   p.d_xscales = a.take<float>(2 * p.mats.size());
   p.d_xsend[0] = a.take<uint8_t>((size_t)W * p.region_bytes[0]);
   p.d_xsend[1] = a.take<uint8_t>((size_t)W * p.region_bytes[1]);
+  p.d_rsync = a.take<uint32_t>(1 + 2 * kResBarriers);
+  p.d_rstamps = a.take<uint64_t>(kResStamps + 1);
   p.state_end = a.off;
 
   // value-domain average: the table of one worker's dequantised levels serves every worker
@@ -542,6 +659,8 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   p.d_tctiles3 = a.take<Tile>(p.tctiles3.size());
   p.d_tcbegin3 = a.take<int>(p.tcbegin3.size());
   p.d_tcmaps = a.take<uint8_t>(p.mats.size() * kTcMapsPerLayer * kTcMapBytes);
+  p.d_rtiles = a.take<ResTile>(p.rtiles.size());
+  p.d_rbegin = a.take<int>(p.rbegin.size());
   p.d_fbP = a.take<FactorBlock>(p.fbP.size());
   p.d_fbQ = a.take<FactorBlock>(p.fbQ.size());
   p.d_fbS = a.take<FactorBlock>(p.fbS.size());
@@ -643,9 +762,10 @@ int lqsgd_workspace_bytes(const lqsgd_shape* shapes, int32_t n_layers, const lqs
   Plan p;
   // The size must not depend on the device: plan for the largest SM count tile sizes consider.
   make_plan(shapes, n_layers, *cfg, nullptr, 148, p);
-  Plan p2;
+  Plan p2, p3;
   make_plan(shapes, n_layers, *cfg, nullptr, 1, p2);
-  *out = std::max(p.bytes, p2.bytes);
+  make_plan(shapes, n_layers, *cfg, nullptr, 148, p3, false);     // in case the one-launch round cannot run on the device
+  *out = std::max({p.bytes, p2.bytes, p3.bytes});
   return LQSGD_OK;
 }
 
@@ -678,6 +798,16 @@ int lqsgd_create(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
     sm_plan = 148;
     make_plan(shapes, n_layers, *cfg, dev_workspace, sm_plan, c->plan);
   }
+  if (c->plan.resident) {
+    // the one-launch round needs its CTA (shared memory, registers) to fit an SM; else the multi-kernel round
+    int grid = 0;
+    const cudaError_t e = resident_max_grid(c->plan.RP, c->plan.res_smem, c->sm_count, &grid);
+    if (e != cudaSuccess || grid == 0) {
+      (void)cudaGetLastError();
+      c->plan = Plan();
+      make_plan(shapes, n_layers, *cfg, dev_workspace, sm_plan, c->plan, false);
+    }
+  }
   Plan& p = c->plan;
   if (p.bytes > workspace_bytes) return LQSGD_ERR_WORKSPACE_TOO_SMALL;
 
@@ -702,6 +832,8 @@ int lqsgd_create(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
   rc = tc_encode_maps(p.layers.data(), (int)p.layers.size(), p.W, p.RP, p.tcmaps.data());
   if (rc != LQSGD_OK) { g_cuda_error = "cuTensorMapEncodeTiled failed or is not available"; return rc; }
   CK(up(p.d_tcmaps, p.tcmaps.data(), p.mats.size() * kTcMapsPerLayer * kTcMapBytes));
+  CK(up(p.d_rtiles, p.rtiles.data(), p.rtiles.size() * sizeof(ResTile)));
+  CK(up(p.d_rbegin, p.rbegin.data(), p.rbegin.size() * sizeof(int)));
   CK(up(p.d_fbP, p.fbP.data(), p.fbP.size() * sizeof(FactorBlock)));
   CK(up(p.d_fbQ, p.fbQ.data(), p.fbQ.size() * sizeof(FactorBlock)));
   CK(up(p.d_fbS, p.fbS.data(), p.fbS.size() * sizeof(FactorBlock)));
@@ -759,10 +891,24 @@ int lqsgd_set_phase_events(lqsgd_ctx* c, void* const* host_events) {
 }
 
 int lqsgd_test_expire_wait(lqsgd_ctx* c, int32_t pass, int32_t stage, uint32_t wait_limit) {
-  if (!c || pass < 1 || pass > 3 || stage < 0 || wait_limit < 16 || wait_limit > (1u << 18)) return LQSGD_ERR_INVALID_ARG;
+  if (!c || pass < 1 || pass > 4 || stage < 0 || wait_limit < 16 || wait_limit > (1u << 18)) return LQSGD_ERR_INVALID_ARG;
   c->test_wait_limit = wait_limit;
   c->test_skip_pass = pass;
   c->test_skip_stage = stage;
+  return LQSGD_OK;
+}
+
+int lqsgd_round_timeline(const lqsgd_ctx* c, uint64_t* host_ns, int32_t* host_count, void* cuda_stream) {
+  if (!c || !host_ns || !host_count) return LQSGD_ERR_INVALID_ARG;
+  *host_count = 0;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (!c->plan.resident) { CK(cudaStreamSynchronize(st)); return LQSGD_OK; }
+  uint64_t tmp[kResStamps + 1] = {};
+  CK(cudaMemcpyAsync(tmp, c->plan.d_rstamps, sizeof(tmp), cudaMemcpyDeviceToHost, st));
+  CK(cudaStreamSynchronize(st));
+  const int n = (int)std::min<uint64_t>(tmp[kResStamps], (uint64_t)LQSGD_TIMELINE_MAX);
+  for (int i = 0; i < n; ++i) host_ns[i] = tmp[i];
+  *host_count = n;
   return LQSGD_OK;
 }
 
@@ -775,6 +921,7 @@ int lqsgd_release_graph_tables(lqsgd_ctx* c) {
 int lqsgd_launches_per_step(const lqsgd_ctx* ctx, int32_t* out) {
   if (!ctx || !out) return LQSGD_ERR_INVALID_ARG;
   const Plan& p = ctx->plan;
+  if (p.resident) { *out = 1; return LQSGD_OK; }              // the whole round is one cooperative launch
   // Orthonormalize, exchange of P, Q_w reduction, exchange of Q; then one launch per non-empty tile list
   const int pass1 = (p.tiles1.empty() ? 0 : 1) + (p.stiles1.empty() ? 0 : 1) + (p.tctiles1.empty() ? 0 : 1);
   const int pass2 = (p.tiles2.empty() ? 0 : 1) + (p.tctiles2.empty() ? 0 : 1);
@@ -980,12 +1127,47 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
   return LQSGD_OK;
 }
 
+// The whole round as one cooperative launch (sets that fit the SMs' shared memory; see lqsgd_resident.cu).
+static int run_resident(lqsgd_ctx* c, cudaStream_t st) {
+  Plan& p = c->plan;
+  const int W = p.W;
+  const size_t nm = p.mats.size(), nv = p.vecs.size();
+  const size_t vbase = nm * (W + 2);
+  const int avg_values = (c->cfg.flags & LQSGD_FLAG_AVERAGE_VALUES) ? 1 : 0;
+  Tables t = c->tables;
+  t.clear_status = (int)nm;
+  ResidentArgs a{};
+  a.tiles = p.d_rtiles; a.cta_begin = p.d_rbegin;
+  a.fbS = p.d_fbS; a.nfbS = (int)p.fbS.size();
+  a.fbP = p.d_fbP; a.nfbP = (int)p.fbP.size();
+  a.fbQ = p.d_fbQ; a.nfbQ = (int)p.fbQ.size();
+  a.chP = p.d_chP; a.nchP = (int)p.chP.size();
+  a.chQ = p.d_chQ; a.nchQ = (int)p.chQ.size();
+  a.qp = QuantTables{p.d_thrP, p.d_deqP, c->cfg.bits_p, avg_values};
+  a.qq = QuantTables{p.d_thrQ, p.d_deqQ, c->cfg.bits_q, avg_values};
+  a.vj.vecs = p.d_vecs; a.vj.chunks = p.d_chV; a.vj.nchunks = (int)p.chV.size(); a.vj.W_total = p.W_total;
+  a.vj.vgrads = reinterpret_cast<const float* const*>(c->ptrs_cur + vbase);
+  a.vj.vghat = reinterpret_cast<float* const*>(c->ptrs_cur + vbase + nv * W);
+  a.vj.vweights = c->has_weights ? reinterpret_cast<float* const*>(c->ptrs_cur + vbase + nv * (W + 1)) : nullptr;
+  a.vj.lr = t.lr;
+  a.sync = p.d_rsync;
+  a.stamps = p.d_rstamps;
+  // phase events: one kernel, so the round's time shows as its first phase and the others as empty
+  if (c->have_events) CK(cudaEventRecord(c->phase_events[0], st));
+  CK(launch_resident(p.RP, t, a, p.res_grid, p.res_smem, st));
+  if (c->have_events)
+    for (int i = 1; i <= LQSGD_N_PHASES; ++i) CK(cudaEventRecord(c->phase_events[i], st));
+  c->have_events = false;
+  return LQSGD_OK;
+}
+
 static int step_impl(lqsgd_ctx* c, const float* const* grads, float* const* ghat, float* const* weights, float lr,
                      void* cuda_stream) {
   int rc = prepare_step(c, grads, ghat, weights, lr, cuda_stream);
   if (rc != LQSGD_OK) return rc;
   if (c->plan.W_total != c->plan.W) return LQSGD_ERR_INVALID_ARG;   // workers elsewhere: use the lqsgd_round_* calls
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (c->plan.resident) return run_resident(c, st);
   const int iters = std::max(1, c->cfg.power_iters);
   for (int it = 0; it < iters; ++it)
     for (int seg = 0; seg <= 4; ++seg) {
@@ -1071,16 +1253,30 @@ int lqsgd_step_host(lqsgd_ctx* c, const float* const* host_grads, float* const* 
   // Copies of tensors that follow one another both in the caller's memory and in the staging area are merged
   // into one: a gradient set kept in one host buffer per worker goes up in a few large copies instead of one
   // per tensor (most tensors of a network are a few hundred bytes of batch-norm parameters).
-  struct Run { char* dst; const char* src; size_t bytes; };
+  // (Neighbours in address space need not belong to one allocation: if the runtime refuses a merged copy, its
+  // pieces go one by one.)
+  struct Piece { char* dst; const char* src; size_t bytes; };
+  struct Run { std::vector<Piece> pieces; size_t bytes = 0; };
   auto flush = [&](Run& r, cudaMemcpyKind kind) -> cudaError_t {
-    const cudaError_t e = r.bytes ? cudaMemcpyAsync(r.dst, r.src, r.bytes, kind, st) : cudaSuccess;
+    cudaError_t e = cudaSuccess;
+    if (!r.pieces.empty()) {
+      e = cudaMemcpyAsync(r.pieces[0].dst, r.pieces[0].src, r.bytes, kind, st);
+      if (e != cudaSuccess && r.pieces.size() > 1) {
+        (void)cudaGetLastError();                                  // not sticky: clear it and copy piece by piece
+        e = cudaSuccess;
+        for (const Piece& pc : r.pieces)
+          if (e == cudaSuccess) e = cudaMemcpyAsync(pc.dst, pc.src, pc.bytes, kind, st);
+      }
+    }
+    r.pieces.clear();
     r.bytes = 0;
     return e;
   };
   auto add = [&](Run& r, void* dst, const void* src, size_t bytes, cudaMemcpyKind kind) -> cudaError_t {
-    if (r.bytes && r.dst + r.bytes == dst && r.src + r.bytes == src) { r.bytes += bytes; return cudaSuccess; }
-    const cudaError_t e = flush(r, kind);
-    r = Run{static_cast<char*>(dst), static_cast<const char*>(src), bytes};
+    cudaError_t e = cudaSuccess;
+    if (!r.pieces.empty() && !(r.pieces[0].dst + r.bytes == dst && r.pieces[0].src + r.bytes == src)) e = flush(r, kind);
+    r.pieces.push_back(Piece{static_cast<char*>(dst), static_cast<const char*>(src), bytes});
+    r.bytes += bytes;
     return e;
   };
   for (int l = 0; l < nl; ++l) {
@@ -1089,7 +1285,7 @@ int lqsgd_step_host(lqsgd_ctx* c, const float* const* host_grads, float* const* 
     for (int w = 0; w < W; ++w)
       if (!host_grads[(size_t)w * nl + l]) return LQSGD_ERR_INVALID_ARG;
   }
-  Run run{nullptr, nullptr, 0};
+  Run run;
   for (int w = 0; w < W; ++w)
     for (int l = 0; l < nl; ++l) {
       const size_t bytes = 4 * (size_t)c->shapes[l].rows * c->shapes[l].cols;

@@ -88,14 +88,16 @@ struct Tables {
   int32_t clear_status;       // > 0 only in the round's first pass-1 launch: that many status words are zeroed by CTA 0
   // Test support (lqsgd_test_expire_wait; all zero in normal operation): the bounded waits of the staged and
   // tensor-core passes give up after wait_limit timed polls instead of the built-in limit, and the loader of
-  // CTA 0 of pass test_skip_pass (1, 2 or 3) leaves out the copies of its stage number test_skip_stage, so
-  // that the waits on that stage run out.  Every address stays valid; only a wait expires.
+  // CTA 0 of pass test_skip_pass (1, 2 or 3) issues no copies from its stage number test_skip_stage on, so
+  // that the waits on those stages run out.  (From that stage ON, not that stage alone: a ring's barrier
+  // tells phases apart by parity only, so a waiter one ring turn further would take the missing phase for
+  // the one before it.)  Every address stays valid; only waits expire.
   uint32_t wait_limit;
   int32_t test_skip_pass;
   int32_t test_skip_stage;
 };
 __device__ __forceinline__ bool test_skips_stage(const Tables& t, int pass, uint32_t stage) {
-  return t.test_skip_pass == pass && blockIdx.x == 0 && stage == (uint32_t)t.test_skip_stage;
+  return t.test_skip_pass == pass && blockIdx.x == 0 && stage >= (uint32_t)t.test_skip_stage;
 }
 
 struct QuantTables {
@@ -123,6 +125,30 @@ __device__ __forceinline__ void clear_status_words(const Tables& t) {
   if (t.clear_status > 0 && blockIdx.x == 0)
     for (int i = threadIdx.x; i < t.clear_status; i += blockDim.x) t.status[i] = 0u;
 }
+// Sum of v[i] over the 32 lanes for every i, in log steps that halve the live values:
+// afterwards lane l holds the totals of indices [l*N/32, (l+1)*N/32) when N >= 32, and the
+// total of index l / (32/N) when N < 32 (in v[0 .. max(N/32,1))).  Fixed order: deterministic.
+template <int N, int O>
+__device__ __forceinline__ void warp_transpose_reduce(float* v, int lane) {
+  if constexpr (O >= 1) {
+    if constexpr (N > 1) {
+      constexpr int H = N / 2;
+      const bool up = (lane & O) != 0;
+#pragma unroll
+      for (int i = 0; i < H; ++i) {
+        const float a = v[i], b = v[i + H];
+        const float send = up ? a : b;
+        const float keep = up ? b : a;
+        v[i] = keep + __shfl_xor_sync(0xffffffffu, send, O);
+      }
+      warp_transpose_reduce<H, O / 2>(v, lane);
+    } else {
+      v[0] += __shfl_xor_sync(0xffffffffu, v[0], O);
+      warp_transpose_reduce<1, O / 2>(v, lane);
+    }
+  }
+}
+
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
                               Args... args) {
@@ -245,6 +271,39 @@ cudaError_t launch_tc_pass1(int RP, const Tables& t, const Tile* tiles, int ntil
                             Launch l);
 cudaError_t launch_tc_pass3(int RP, const Tables& t, const Tile* tiles, int ntiles, const int* cta_begin, const void* maps,
                             Launch l);
+// One-launch round (lqsgd_resident.cu) for sets whose M fits in the SMs' shared memory: one cooperative grid,
+// one CTA of kResThreads threads per SM, tiles of M resident from pass 1 to pass 3, grid barriers between the steps.
+constexpr int kResThreads = 512;
+constexpr int kResMaxTiles = 16;       // tiles one CTA may hold (one shared-memory barrier each)
+constexpr int kResMaxTileRows = 256;   // rows of a tile (its rows of P_bar wait in scratch)
+constexpr int kResMaxTileCols = 1024;  // columns of a tile (its rows of Q_bar wait in scratch)
+constexpr int kResBarriers = 6;        // grid barriers per launch at most (counters per set)
+constexpr int kResStamps = 12;         // timeline stamps per launch (then one word holding their number)
+struct ResTile {
+  int32_t layer, worker;
+  int32_t row0, nrows, col0, ncols;
+  int32_t part_c, part_r;     // column chunk (partial sums of P), row chunk (partial sums of Q)
+  int32_t smem_off;           // floats from the start of the CTA's resident area (multiple of 4)
+  int32_t plain;              // 1: the layer's rows are not 16-byte aligned: whole rows, ordinary loads and stores
+  int32_t writes_ghat;        // 1: this tile (worker 0's) also writes G_hat and applies the model update
+  int32_t pad;
+};
+struct ResidentArgs {
+  const ResTile* tiles;
+  const int* cta_begin;       // [grid + 1]: CTA b holds tiles [cta_begin[b], cta_begin[b + 1])
+  const FactorBlock* fbS; int32_t nfbS;
+  const FactorBlock* fbP; int32_t nfbP;
+  const FactorBlock* fbQ; int32_t nfbQ;
+  const ExchangeChunk* chP; int32_t nchP;
+  const ExchangeChunk* chQ; int32_t nchQ;
+  QuantTables qp, qq;
+  VectorJob vj;               // nchunks == 0: no 1-D tensors
+  uint32_t* sync;             // [1 + 2 * kResBarriers]: launch counter, two sets of barrier counters
+  uint64_t* stamps;           // [kResStamps + 1]: CTA 0's timeline of the launch in ns, then the number of stamps
+};
+size_t resident_scratch_bytes(int RP);   // shared memory per CTA that is not available to tiles
+cudaError_t launch_resident(int RP, const Tables& t, const ResidentArgs& a, int grid, size_t smem_bytes, cudaStream_t stream);
+cudaError_t resident_max_grid(int RP, size_t smem_bytes, int sm_count, int* grid_out);   // 0: the kernel does not fit
 cudaError_t launch_stream_pass1(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
 cudaError_t launch_stream_pass3(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
 // Resident CTAs per SM of each streaming pass for this RP (for persistent grid sizing).

@@ -15,7 +15,7 @@
 // Every kernel is a persistent or table-driven grid: CTAs walk a tile table the host planned
 // once, so a 64 x 27 layer costs a table entry, not a launch.  Nothing here spins or waits on
 // another CTA, and every reduction has a fixed order: results are bit-reproducible.
-#include "lqsgd_dev.h"
+#include "lqsgd_factor.cuh"
 
 #include <cuda_bf16.h>
 
@@ -28,36 +28,7 @@ namespace {
 // small helpers
 // ---------------------------------------------------------------------------------------
 template <int N>
-__device__ __forceinline__ void load_contig_ro(const float* __restrict__ p, float (&out)[N]) {
-  // N contiguous read-only floats, aligned to min(N,4)*4 bytes, through the read-only path
-  if constexpr (N % 4 == 0) {
-#pragma unroll
-    for (int i = 0; i < N / 4; ++i) {
-      float4 v = __ldg(reinterpret_cast<const float4*>(p) + i);
-      out[4 * i] = v.x; out[4 * i + 1] = v.y; out[4 * i + 2] = v.z; out[4 * i + 3] = v.w;
-    }
-  } else if constexpr (N == 2) {
-    float2 v = __ldg(reinterpret_cast<const float2*>(p));
-    out[0] = v.x; out[1] = v.y;
-  } else {
-#pragma unroll
-    for (int i = 0; i < N; ++i) out[i] = __ldg(p + i);
-  }
-}
-
-template <int N>
-__device__ __forceinline__ void store_contig(float* p, const float (&v)[N]) {
-  if constexpr (N % 4 == 0) {
-#pragma unroll
-    for (int i = 0; i < N / 4; ++i)
-      reinterpret_cast<float4*>(p)[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-  } else if constexpr (N == 2) {
-    *reinterpret_cast<float2*>(p) = make_float2(v[0], v[1]);
-  } else {
-#pragma unroll
-    for (int i = 0; i < N; ++i) p[i] = v[i];
-  }
-}
+__device__ __forceinline__ void load_contig_nc(const float* __restrict__ p, float (&out)[N]) { load_contig<N, false>(p, out); }
 
 // Packed fp32 arithmetic of sm_100: one instruction, two fused multiply-adds on a register pair,
 // d.lo = a.lo * b.lo + c.lo and d.hi likewise, each half rounded exactly like fmaf.  Pass 2 at
@@ -154,30 +125,6 @@ template <int VEC>
 __device__ __forceinline__ void st_stream(float* p, const Pack<VEC>& x) {
   if constexpr (VEC == 4) __stcs(reinterpret_cast<float4*>(p), make_float4(x.v[0], x.v[1], x.v[2], x.v[3]));
   else __stcs(p, x.v[0]);
-}
-
-// Sum of v[i] over the 32 lanes for every i, in log steps that halve the live values:
-// afterwards lane l holds the totals of indices [l*N/32, (l+1)*N/32) when N >= 32, and the
-// total of index l / (32/N) when N < 32 (in v[0 .. max(N/32,1))).  Fixed order: deterministic.
-template <int N, int O>
-__device__ __forceinline__ void warp_transpose_reduce(float* v, int lane) {
-  if constexpr (O >= 1) {
-    if constexpr (N > 1) {
-      constexpr int H = N / 2;
-      const bool up = (lane & O) != 0;
-#pragma unroll
-      for (int i = 0; i < H; ++i) {
-        const float a = v[i], b = v[i + H];
-        const float send = up ? a : b;
-        const float keep = up ? b : a;
-        v[i] = keep + __shfl_xor_sync(0xffffffffu, send, O);
-      }
-      warp_transpose_reduce<H, O / 2>(v, lane);
-    } else {
-      v[0] += __shfl_xor_sync(0xffffffffu, v[0], O);
-      warp_transpose_reduce<1, O / 2>(v, lane);
-    }
-  }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -318,7 +265,7 @@ __device__ __forceinline__ void pass2_tile(const Tables& t, const Tile& tl, floa
     constexpr int VW = RP < 4 ? RP : 4;
     for (int e = threadIdx.x; e < tl.nrows * (RP / VW); e += kPassThreads) {
       float v[VW];
-      load_contig_ro<VW>(Pbar + (size_t)tl.row0 * RP + (size_t)e * VW, v);
+      load_contig_nc<VW>(Pbar + (size_t)tl.row0 * RP + (size_t)e * VW, v);
       store_contig<VW>(pb + (size_t)e * VW, v);
     }
     __syncthreads();
@@ -374,7 +321,7 @@ __device__ __forceinline__ void pass2_tile(const Tables& t, const Tile& tl, floa
 #pragma unroll
       for (int u = 0; u < U; ++u) {
         float p[RP];
-        load_contig_ro<RP>(Pbar + (size_t)(i + u * cm.ng) * RP, p);
+        load_contig_nc<RP>(Pbar + (size_t)(i + u * cm.ng) * RP, p);
 #pragma unroll
         for (int k = 0; k < VEC; ++k)
 #pragma unroll
@@ -384,7 +331,7 @@ __device__ __forceinline__ void pass2_tile(const Tables& t, const Tile& tl, floa
     for (; i < rend; i += cm.ng) {
       const Pack<VEC> mv = ld_keep<VEC>(M + (size_t)i * m + col, pol);
       float p[RP];
-      load_contig_ro<RP>(Pbar + (size_t)i * RP, p);
+      load_contig_nc<RP>(Pbar + (size_t)i * RP, p);
 #pragma unroll
       for (int k = 0; k < VEC; ++k)
 #pragma unroll
@@ -470,7 +417,7 @@ __device__ __forceinline__ void pass3_tile(const Tables& t, const Tile& tl) {
       const int i = i0 + u * cm.ng;
       if (i < rend) {
         float p[RP];
-        load_contig_ro<RP>(Pbar + (size_t)i * RP, p);
+        load_contig_nc<RP>(Pbar + (size_t)i * RP, p);
 #pragma unroll
         for (int k = 0; k < VEC; ++k) {
           float s = 0.f;
@@ -520,658 +467,62 @@ pass3_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
 }
 
 // ---------------------------------------------------------------------------------------
-// Orthonormalize (Alg. 1) as CholeskyQR with the r x r part in fp64:
-//   p_reduce_gram: P_raw = sum of the column-chunk partials (fixed order); per-block Gram
-//   p_apply      : Gram = sum of block Grams; R^T R = Gram; R^-1 (redone by every CTA);
-//                  P = P_raw R^-1 (fp64 accumulate, stored fp32); block max |P|
-// The result is the thin-QR Q factor with positive-diagonal R, the same matrix Gram-Schmidt
-// produces.  A column whose pivot is <= 1e-10 of its squared norm (or zero, or not a number)
-// becomes a zero column and the layer's status word says so.
+// The small steps between the passes: one CTA per table entry, bodies in lqsgd_factor.cuh
+// (Orthonormalize as CholeskyQR, the factor exchange, the Q_w reduction, the 1-D tensors).
 // ---------------------------------------------------------------------------------------
-constexpr double kPivotEps = 1e-10;
-
 template <int RP>
 __global__ void __launch_bounds__(256)
 p_reduce_gram_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
   pdl_wait();
-  __shared__ double rows[kFactorBlockRows][RP];     // the block's rows, converted once
-  const FactorBlock fb = fbs[blockIdx.x];
-  const LayerDev& L = t.layers[fb.layer];
-  const int n = L.n;
-  const int tid = threadIdx.x;
-  if (tid < kFactorBlockRows) {
-    const int row = fb.blk * kFactorBlockRows + tid;
-    float p[RP];
-#pragma unroll
-    for (int j = 0; j < RP; ++j) p[j] = 0.f;
-    if (row < n) {
-      const float* src = L.Ppart + ((size_t)fb.worker * L.ncc * n + row) * RP;
-      // the partials' loads go out together (8 at a time); the additions keep the chunk order
-      int cc = 0;
-      if constexpr (RP <= 8) {
-        for (; cc + 8 <= L.ncc; cc += 8) {
-          float v[8][RP];
-#pragma unroll
-          for (int u = 0; u < 8; ++u) load_contig_ro<RP>(src + (size_t)(cc + u) * n * RP, v[u]);
-#pragma unroll
-          for (int u = 0; u < 8; ++u)
-#pragma unroll
-            for (int j = 0; j < RP; ++j) p[j] += v[u][j];
-        }
-      }
-      for (; cc < L.ncc; ++cc) {
-        float v[RP];
-        load_contig_ro<RP>(src + (size_t)cc * n * RP, v);
-#pragma unroll
-        for (int j = 0; j < RP; ++j) p[j] += v[j];
-      }
-      if (L.ncc > 1) store_contig<RP>(L.Praw + ((size_t)fb.worker * n + row) * RP, p);
-    }
-#pragma unroll
-    for (int j = 0; j < RP; ++j) rows[tid][j] = (double)p[j];
-  }
-  __syncthreads();
-  for (int e = tid; e < RP * RP; e += 256) {
-    const int i = e / RP, j = e % RP;
-    if (j < i) continue;                                 // the Gram matrix is symmetric: upper triangle, mirrored
-    double s = 0.0;
-    for (int k = 0; k < kFactorBlockRows; ++k) s = fma(rows[k][i], rows[k][j], s);
-    double* gp = L.gram_part + ((size_t)fb.worker * L.npb + fb.blk) * (RP * RP);
-    gp[i * RP + j] = s;
-    gp[j * RP + i] = s;
-  }
-}
-
-// Gram = sum of the block Grams (block order), Cholesky  Gram = L L^T  (R = L^T), by a whole CTA;
-// every CTA that orthonormalises a block of rows redoes this small factorisation itself, which
-// costs less than a kernel boundary.  Lf (shared, RP*RP doubles, row-major) receives L, invd the
-// reciprocals of its diagonal, dead[j] = 1 for a column dropped as dependent (its row and column
-// of L are then those of the identity).  Returns true if any column was dropped.
-template <int RP>
-__device__ __forceinline__ bool cholesky_factor(double (*A)[RP + 1], int r, double* Lf, double* invd, int* dead);
-
-template <int RP>
-__device__ __forceinline__ bool cholesky_lower(const LayerDev& L, int worker, double* Lf, double* invd, int* dead) {
-  __shared__ double A[RP][RP + 1];     // Gram, overwritten by L (lower triangle)
-  const int tid = threadIdx.x, nt = blockDim.x;
-  // Gram = sum of the block Grams.  With more threads than entries the blocks are dealt to SEG
-  // segments (segment g takes blocks g, g + SEG, ...), eight loads in flight each; the segments'
-  // sums are then added in segment order: a fixed order, and a chain SEG times shorter.
-  constexpr int SEG = (RP * RP <= 64) ? 128 / (RP * RP) : 1;      // the factor kernels run 128 threads
-  if constexpr (SEG > 1) {
-    __shared__ double segsum[SEG][RP * RP];
-    if (tid < SEG * RP * RP) {
-      const int e = tid % (RP * RP), g = tid / (RP * RP);
-      const double* gp = L.gram_part + (size_t)worker * L.npb * (RP * RP) + e;
-      double s = 0.0;
-      int b = g;
-      for (; b + 7 * SEG < L.npb; b += 8 * SEG) {
-        double x[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) x[u] = gp[(size_t)(b + u * SEG) * (RP * RP)];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) s += x[u];
-      }
-      for (; b < L.npb; b += SEG) s += gp[(size_t)b * (RP * RP)];
-      segsum[g][e] = s;
-    }
-    __syncthreads();
-    if (tid < RP * RP) {
-      double s = segsum[0][tid];
-#pragma unroll
-      for (int g = 1; g < SEG; ++g) s += segsum[g][tid];
-      A[tid / RP][tid % RP] = s;
-    }
-  } else {
-    for (int e = tid; e < RP * RP; e += nt) {
-      const double* gp = L.gram_part + (size_t)worker * L.npb * (RP * RP) + e;
-      double s = 0.0;
-      int b = 0;
-      for (; b + 8 <= L.npb; b += 8) {        // eight loads in flight, additions in block order
-        double x[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) x[u] = gp[(size_t)(b + u) * (RP * RP)];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) s += x[u];
-      }
-      for (; b < L.npb; ++b) s += gp[(size_t)b * (RP * RP)];
-      A[e / RP][e % RP] = s;
-    }
-  }
-  __syncthreads();
-  return cholesky_factor<RP>(A, L.r, Lf, invd, dead);
-}
-
-// Cholesky of the Gram matrix in A (shared, complete and visible to the CTA on entry).
-template <int RP>
-__device__ __forceinline__ bool cholesky_factor(double (*A)[RP + 1], int r, double* Lf, double* invd, int* dead) {
-  __shared__ double diag0[RP];
-  const int tid = threadIdx.x, nt = blockDim.x;
-  if (tid < RP) { diag0[tid] = A[tid][tid]; dead[tid] = 0; invd[tid] = 1.0; }
-  __syncthreads();
-  // right-looking Cholesky by ONE warp (warp-level barriers only; the other warps wait once, below):
-  // pivot, column j, then the rank-1 update of the trailing lower triangle with its entries dealt to
-  // the lanes (every entry sees the updates in the order of j, so the result does not depend on how
-  // the entries are dealt)
-  if (tid < 32) {
-    for (int j = 0; j < r; ++j) {
-      const double d = A[j][j];
-      const bool ok = (d > kPivotEps * diag0[j]) && (d < INFINITY);   // false for nan too
-      // 1 / sqrt(d) by the hardware seed plus refinement (the library sqrt and division are long
-      // software sequences, and this loop is a chain of r of them); l_jj = d / sqrt(d)
-      const double inv = ok ? rsqrt(d) : 1.0;
-      const double ljj = ok ? d * inv : 1.0;
-      __syncwarp();                      // every lane has read the pivot
-      for (int i = j + tid; i < r; i += 32) {
-        if (i == j) { A[j][j] = ljj; invd[j] = inv; if (!ok) dead[j] = 1; }
-        else A[i][j] = ok ? A[i][j] * inv : 0.0;
-      }
-      __syncwarp();
-      if (ok) {
-        const int w = r - j - 1;         // trailing block: rows and columns j+1 .. r-1
-        for (int e = tid; e < w * w; e += 32) {
-          const int i = j + 1 + e / w, k = j + 1 + e % w;
-          if (k <= i) A[i][k] -= A[i][j] * A[k][j];
-        }
-      }
-      __syncwarp();
-    }
-  }
-  __syncthreads();
-  for (int e = tid; e < RP * RP; e += nt) {
-    const int i = e / RP, k = e % RP;
-    Lf[e] = (k <= i && i < r) ? A[i][k] : 0.0;
-  }
-  int any = 0;
-  for (int j = 0; j < r; ++j) any |= dead[j];
-  __syncthreads();
-  return any != 0;
-}
-
-__device__ __forceinline__ float block_max_128(float v, float* sm) {
-  // max over a 128-thread block; NaN compares false and is dropped (reported separately)
-#pragma unroll
-  for (int o = 16; o >= 1; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-  if ((threadIdx.x & 31) == 0) sm[threadIdx.x >> 5] = v;
-  __syncthreads();
-  return fmaxf(fmaxf(sm[0], sm[1]), fmaxf(sm[2], sm[3]));
+  __shared__ __align__(16) unsigned char smem[sizeof(ReduceGramSmem<RP>)];
+  p_reduce_gram_body<RP, 256, false>(t, fbs[blockIdx.x], threadIdx.x, smem);
 }
 
 template <int RP>
 __global__ void __launch_bounds__(kFactorBlockRows)
 p_apply_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
   pdl_wait();
-  __shared__ double Lf[RP * RP];
-  __shared__ double invd[RP];
-  __shared__ int dead[RP];
-  __shared__ float smax[4];
-  __shared__ float scol[4][RP];
-  const FactorBlock fb = fbs[blockIdx.x];
-  const LayerDev& L = t.layers[fb.layer];
-  const int n = L.n, tid = threadIdx.x;
-  const bool dropped = cholesky_lower<RP>(L, fb.worker, Lf, invd, dead);
-  if (dropped && fb.blk == 0 && tid == 0) atomicOr(&t.status[fb.layer], 1u);
-  const int row = fb.blk * kFactorBlockRows + tid;
-  float amax = 0.f;
-  float o[RP];
-#pragma unroll
-  for (int j = 0; j < RP; ++j) o[j] = 0.f;
-  if (row < n) {
-    // the row of P solves  o R = p  with R = L^T upper triangular: forward substitution in fp64,
-    //   o[j] = (p[j] - sum_{k<j} o[k] L[j][k]) / L[j][j];   a dropped column gives 0
-    float p[RP];
-    load_contig_ro<RP>(L.Praw + ((size_t)fb.worker * n + row) * RP, p);
-    double od[RP];
-    bool bad = false;
-#pragma unroll
-    for (int j = 0; j < RP; ++j) {
-      double s = (double)p[j];
-#pragma unroll
-      for (int k = 0; k < j; ++k) s = fma(-od[k], Lf[j * RP + k], s);
-      od[j] = (j < L.r && !dead[j]) ? s * invd[j] : 0.0;
-      o[j] = (float)od[j];
-      amax = fmaxf(amax, fabsf(o[j]));
-      bad |= !(fabsf(o[j]) < INFINITY);
-    }
-    store_contig<RP>(L.P + ((size_t)fb.worker * n + row) * RP, o);
-    if (bad) atomicOr(&t.status[fb.layer], 8u);
-  }
-  if (t.col_scales) {            // variant: one maximum per column
-#pragma unroll
-    for (int j = 0; j < RP; ++j) {
-      float v = fabsf(o[j]);
-#pragma unroll
-      for (int off = 16; off >= 1; off >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, off));
-      if ((tid & 31) == 0) scol[tid >> 5][j] = v;
-    }
-    __syncthreads();
-    if (tid < RP)
-      L.maxp[((size_t)fb.worker * L.npb + fb.blk) * RP + tid] =
-          fmaxf(fmaxf(scol[0][tid], scol[1][tid]), fmaxf(scol[2][tid], scol[3][tid]));
-    return;
-  }
-  amax = block_max_128(amax, smax);
-  if (tid == 0) L.maxp[(size_t)fb.worker * L.npb + fb.blk] = amax;
+  __shared__ __align__(16) unsigned char smem[sizeof(ApplySmem<RP, kFactorBlockRows>)];
+  p_apply_body<RP, kFactorBlockRows, false>(t, fbs[blockIdx.x], threadIdx.x, smem);
 }
 
-// Orthonormalize for a layer of at most 512 rows (every layer of the ResNet-18 set), one CTA per
-// (layer, worker), one thread per row: the sum of pass 1's column-chunk partials, the Gram matrix in
-// fp64 (every entry summed over eight 64-row segments, the segments then added in order), its
-// Cholesky factor, the rows of P by substitution and the block maxima: what p_reduce_gram and
-// p_apply do in two launches for taller layers.
-constexpr int kOrthSmallRows = 512;
 template <int RP>
 __global__ void __launch_bounds__(kOrthSmallRows, 3)   // three CTAs per SM: 444 at once, one wave for 21 layers x 16 workers
 p_orth_small_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
   pdl_wait();
-  constexpr int NE = RP * RP, NSEG = 8, SEGROWS = kOrthSmallRows / NSEG;
-  __shared__ double rows[kOrthSmallRows][RP];
-  __shared__ double seg[NSEG][NE];
-  __shared__ double A[RP][RP + 1];
-  __shared__ double Lf[NE];
-  __shared__ double invd[RP];
-  __shared__ int dead[RP];
-  __shared__ float wmax[kOrthSmallRows / 32][RP];
-  const FactorBlock fb = fbs[blockIdx.x];
-  const LayerDev& L = t.layers[fb.layer];
-  const int n = L.n, tid = threadIdx.x, row = tid;
-  float p[RP];
-#pragma unroll
-  for (int j = 0; j < RP; ++j) p[j] = 0.f;
-  if (row < n) {
-    const float* src = L.Ppart + ((size_t)fb.worker * L.ncc * n + row) * RP;
-    for (int cc = 0; cc < L.ncc; ++cc) {
-      float v[RP];
-      load_contig_ro<RP>(src + (size_t)cc * n * RP, v);
-#pragma unroll
-      for (int j = 0; j < RP; ++j) p[j] += v[j];
-    }
-    if (L.ncc > 1) store_contig<RP>(L.Praw + ((size_t)fb.worker * n + row) * RP, p);
-  }
-#pragma unroll
-  for (int j = 0; j < RP; ++j) rows[tid][j] = (double)p[j];
-  __syncthreads();
-  for (int idx = tid; idx < NSEG * NE; idx += kOrthSmallRows) {
-    const int e = idx % NE, g = idx / NE, i = e / RP, j = e % RP;
-    if (j < i) continue;                                   // upper triangle; mirrored below
-    double s = 0.0;
-    for (int k = g * SEGROWS; k < (g + 1) * SEGROWS; ++k) s = fma(rows[k][i], rows[k][j], s);
-    seg[g][e] = s;
-  }
-  __syncthreads();
-  if (tid < NE) {
-    const int i = tid / RP, j = tid % RP;
-    if (j >= i) {
-      double s = seg[0][tid];
-#pragma unroll
-      for (int g = 1; g < NSEG; ++g) s += seg[g][tid];
-      A[i][j] = s;
-      A[j][i] = s;
-    }
-  }
-  __syncthreads();
-  const bool dropped = cholesky_factor<RP>(A, L.r, Lf, invd, dead);
-  if (dropped && tid == 0) atomicOr(&t.status[fb.layer], 1u);
-  float o[RP];
-#pragma unroll
-  for (int j = 0; j < RP; ++j) o[j] = 0.f;
-  if (row < n) {
-    double od[RP];
-    bool bad = false;
-#pragma unroll
-    for (int j = 0; j < RP; ++j) {
-      double s = (double)p[j];
-#pragma unroll
-      for (int k = 0; k < j; ++k) s = fma(-od[k], Lf[j * RP + k], s);
-      od[j] = (j < L.r && !dead[j]) ? s * invd[j] : 0.0;
-      o[j] = (float)od[j];
-      bad |= !(fabsf(o[j]) < INFINITY);
-    }
-    store_contig<RP>(L.P + ((size_t)fb.worker * n + row) * RP, o);
-    if (bad) atomicOr(&t.status[fb.layer], 8u);
-  }
-  // maxima per block of 128 rows (4 warps), as the exchange reads them; one per column in the column-scale variant
-#pragma unroll
-  for (int j = 0; j < RP; ++j) {
-    float v = fabsf(o[j]);
-#pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, off));
-    if ((tid & 31) == 0) wmax[tid >> 5][j] = v;
-  }
-  __syncthreads();
-  const int ncs = t.col_scales ? RP : 1;
-  if (tid < L.npb * ncs) {
-    const int blk = tid / ncs, j0 = tid % ncs;
-    float a = 0.f;
-    for (int w4 = 4 * blk; w4 < 4 * blk + 4; ++w4)
-      for (int j = (t.col_scales ? j0 : 0); j < (t.col_scales ? j0 + 1 : RP); ++j) a = fmaxf(a, wmax[w4][j]);
-    L.maxp[((size_t)fb.worker * L.npb + blk) * ncs + j0] = a;
-  }
+  __shared__ __align__(16) unsigned char smem[sizeof(OrthSmallSmem<RP>)];
+  p_orth_small_body<RP, false>(t, fbs[blockIdx.x], threadIdx.x, smem);
 }
 
-// Q_w = sum of the row-chunk partials of pass 2, in chunk order; block max |Q_w|.  A thread owns
-// V = min(RP, 4) consecutive columns of a row (one 128-bit load per partial when RP >= 4) and the
-// loads of several partials are in flight together: the chain of nrb dependent additions, not a
-// chain of nrb memory latencies, is what a row costs.
 template <int RP> struct QReduceThreads { static constexpr int value = RP >= 8 ? 256 : 128; };   // one item per thread up to rank 8
 template <int RP>
 __global__ void __launch_bounds__(QReduceThreads<RP>::value)
 q_reduce_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
   pdl_wait();
-  constexpr int kQReduceThreads = QReduceThreads<RP>::value;
-  constexpr int V = RP < 4 ? RP : 4;        // floats per thread item
-  constexpr int TPR = RP / V;               // items per row: 1, 2, 4 or 8 (divides the block size and 32)
-  __shared__ float smax[kQReduceThreads / 32][TPR * V];
-  const FactorBlock fb = fbs[blockIdx.x];
-  const LayerDev& L = t.layers[fb.layer];
-  const int m = L.m, tid = threadIdx.x, nrb = L.nrb;
-  const size_t plane = (size_t)m * RP;      // floats of one partial
-  float cmax[V];
-#pragma unroll
-  for (int v = 0; v < V; ++v) cmax[v] = 0.f;
-  bool bad = false;
-  for (int item = tid; item < kFactorBlockRows * TPR; item += kQReduceThreads) {
-    const int row = fb.blk * kFactorBlockRows + item / TPR;
-    if (row >= m) break;
-    const size_t off = (size_t)row * RP + (size_t)(item % TPR) * V;
-    const float* src = L.Qpart + (size_t)fb.worker * nrb * plane + off;
-    float q[V];
-#pragma unroll
-    for (int v = 0; v < V; ++v) q[v] = 0.f;
-    int rb = 0;
-    for (; rb + 8 <= nrb; rb += 8) {
-      float x[8][V];
-#pragma unroll
-      for (int u = 0; u < 8; ++u) load_contig_ro<V>(src + (size_t)(rb + u) * plane, x[u]);
-#pragma unroll
-      for (int u = 0; u < 8; ++u)
-#pragma unroll
-        for (int v = 0; v < V; ++v) q[v] += x[u][v];
-    }
-    for (; rb < nrb; ++rb) {
-      float x[V];
-      load_contig_ro<V>(src + (size_t)rb * plane, x);
-#pragma unroll
-      for (int v = 0; v < V; ++v) q[v] += x[v];
-    }
-    if (nrb > 1) store_contig<V>(L.Qw + (size_t)fb.worker * plane + off, q);
-#pragma unroll
-    for (int v = 0; v < V; ++v) {
-      cmax[v] = fmaxf(cmax[v], fabsf(q[v]));
-      bad |= !(fabsf(q[v]) < INFINITY);
-    }
-  }
-  if (bad) atomicOr(&t.status[fb.layer], 8u);
-  // maxima: the columns a thread owns are fixed (256 and 32 are multiples of TPR): columns (tid % TPR) V + v
-  const int warp = tid >> 5, lane = tid & 31;
-  if (t.col_scales) {
-#pragma unroll
-    for (int v = 0; v < V; ++v) {
-#pragma unroll
-      for (int o = 16; o >= TPR; o >>= 1) cmax[v] = fmaxf(cmax[v], __shfl_xor_sync(0xffffffffu, cmax[v], o));
-      if (lane < TPR) smax[warp][lane * V + v] = cmax[v];
-    }
-    __syncthreads();
-    if (tid < RP) {
-      float a = smax[0][tid];
-#pragma unroll
-      for (int w = 1; w < kQReduceThreads / 32; ++w) a = fmaxf(a, smax[w][tid]);
-      L.maxq[((size_t)fb.worker * L.nqb + fb.blk) * RP + tid] = a;
-    }
-    return;
-  }
-  float amax = cmax[0];
-#pragma unroll
-  for (int v = 1; v < V; ++v) amax = fmaxf(amax, cmax[v]);
-#pragma unroll
-  for (int o = 16; o >= 1; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-  if (lane == 0) smax[warp][0] = amax;
-  __syncthreads();
-  if (tid == 0) {
-#pragma unroll
-    for (int w = 1; w < kQReduceThreads / 32; ++w) amax = fmaxf(amax, smax[w][0]);
-    L.maxq[(size_t)fb.worker * L.nqb + fb.blk] = amax;
-  }
+  constexpr int NT = QReduceThreads<RP>::value;
+  __shared__ __align__(16) unsigned char smem[sizeof(QReduceSmem<RP, NT>)];
+  q_reduce_body<RP, NT, false>(t, fbs[blockIdx.x], threadIdx.x, smem);
 }
 
-// One element of an averaged factor (P_bar or Q_bar) goes to its row-major home and to the
-// copies the passes read: the transposed Q of passes 1 and 3 and, for layers on the tensor-core
-// passes, the operands in the narrow terms those passes multiply (see lqsgd_tc.cu).
-__device__ __forceinline__ float tf32_remainder(float x) {
-  return x - __uint_as_float(__float_as_uint(x) & 0xffffe000u);
-}
-template <int RP>
-__device__ __forceinline__ void store_factor(const LayerDev& L, int which, int row, int col, float v) {
-  if (which) {
-    L.Q[(size_t)row * RP + col] = v;
-    L.Qt[(size_t)col * L.mt + row] = v;
-    if (L.tc) {
-      const float lo = tf32_remainder(v);
-      L.Qt[(size_t)(RP + col) * L.mt + row] = lo;
-      float* qc = L.Qcat + (size_t)row * L.kcat + col;
-      qc[0] = v; qc[RP] = lo; qc[2 * RP] = v;
-    }
-  } else {
-    L.Pbar[(size_t)row * RP + col] = v;
-    if (L.tc) {
-      float* pc = L.Pcat + (size_t)row * L.kcat + col;
-      pc[0] = v; pc[RP] = v; pc[2 * RP] = tf32_remainder(v);
-      // three bf16 terms v = b1 + b2 + b3 (24 bits), each stored twice in one word: the two K slots
-      // that face the bf16 pair of an element of M in the tensor-core pass 2
-      float rest = v;
-#pragma unroll
-      for (int term = 0; term < 3; ++term) {
-        const __nv_bfloat16 b = __float2bfloat16_rn(rest);
-        rest -= __bfloat162float(b);
-        const uint32_t h = __bfloat16_as_ushort(b);
-        reinterpret_cast<uint32_t*>(L.Pbt)[(size_t)(term * RP + col) * L.nt + row] = h | (h << 16);
-      }
-    }
-  }
-}
-
-// ---------------------------------------------------------------------------------------
-// 1-D tensors: mean over the workers (Eq. 1) in worker order, and the raw fp32 values into
-// each worker's payload.  One block = 256 entries of one tensor.  Runs as a kernel of its own or
-// as extra blocks of the exchange of P (same block shape), which saves a launch per round.
-// ---------------------------------------------------------------------------------------
-__device__ __forceinline__ void vectors_block(const VectorJob& vj, int blk, uint8_t* payload, uint64_t payload_stride,
-                                              int W) {
-  const ExchangeChunk ch = vj.chunks[blk];
-  const VectorDev v = vj.vecs[ch.layer];
-  const int i = ch.chunk * 256 + threadIdx.x;
-  if (i >= v.len) return;
-  float s = 0.f;
-  for (int w = 0; w < W; ++w) {
-    const float x = vj.vgrads[(size_t)ch.layer * W + w][i];
-    reinterpret_cast<float*>(payload + (size_t)w * payload_stride + v.pay_off)[i] = x;
-    s += x;
-  }
-  const float mean = s / (float)vj.W_total;     // with workers on other GPUs too: this rank's share of the mean
-  if (vj.vghat[ch.layer]) vj.vghat[ch.layer][i] = mean;
-  if (vj.vweights && vj.vweights[ch.layer]) vj.vweights[ch.layer][i] = fmaf(-vj.lr, mean, vj.vweights[ch.layer][i]);
-}
 __global__ void __launch_bounds__(256)
 vectors_kernel(VectorJob vj, uint8_t* payload, uint64_t payload_stride, int W) {
   pdl_wait();
-  vectors_block(vj, blockIdx.x, payload, payload_stride, W);
+  vectors_block(vj, blockIdx.x, threadIdx.x, payload, payload_stride, W);
 }
 
-// ---------------------------------------------------------------------------------------
-// Factor exchange (Alg. 1: LogQuantize, All-Reduce, LogDequantize) for one chunk of 256
-// factor elements of one layer, all W workers:
-//   s      = max |x| over the layer's block maxima (shared scale)
-//   code_w = sign bit | k,  k = number of thresholds <= |x_w| / s        (Eq. 4, nearest level)
-//   stream = little-endian b-bit packing of code_w into worker w's payload
-//   S      = sum_w (+-k_w)   exact integer;   x_bar = s * deq[S]          (Eq. 1, Eq. 5)
-// The threshold table holds, for every level boundary, the smallest fp32 not below the exact
-// boundary, so "t >= thr" decides exactly like the real-number comparison.
-// ---------------------------------------------------------------------------------------
-// B = bits per code (2..8), or 32: quantiser bypassed.  One block = 256 factor elements.
+// Factor exchange, one block per chunk of 256 factor elements; blocks past the factor chunks take the
+// round's 1-D tensors (same block shape), which saves a launch per round.
 template <int RP, int B>
 __global__ void __launch_bounds__(256)
 exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __restrict__ chunks, int nchunks,
                 SplitExchange sx, VectorJob vj) {
   pdl_wait();
-  if ((int)blockIdx.x >= nchunks) {      // blocks past the factor chunks: the round's 1-D tensors
-    vectors_block(vj, (int)blockIdx.x - nchunks, t.payload, t.payload_stride, t.W);
+  if ((int)blockIdx.x >= nchunks) {
+    vectors_block(vj, (int)blockIdx.x - nchunks, threadIdx.x, t.payload, t.payload_stride, t.W);
     return;
   }
-  constexpr int CH = kExchangeChunk;   // 256 factor elements per block, one per thread
-  constexpr int WB = 8;                // workers handled per round
-  constexpr int NLEV = (B == 32) ? 2 : 1 << (B - 1);
-  __shared__ float thr[128];
-  __shared__ __align__(4) uint8_t codes[WB][CH + 4];
-  __shared__ float sred[8];
-  __shared__ float scol8[8][RP];
-  __shared__ float scol[RP];
-  const ExchangeChunk ch = chunks[blockIdx.x];
-  const LayerDev& L = t.layers[ch.layer];
-  const int W = t.W, tid = threadIdx.x;
-  const int rows = which ? L.m : L.n, r = L.r;
-  const int count = rows * r;
-  const int nblk = which ? L.nqb : L.npb;
-  const float* __restrict__ maxes = which ? L.maxq : L.maxp;
-  const float* __restrict__ src = which ? L.Qw : L.P;   // [W][rows][RP]
-  const uint64_t pay_off = which ? L.pay_q_off : L.pay_p_off;
-
-  for (int i = tid; i < NLEV - 1; i += 256) thr[i] = qt.thr[i];
-  if (tid < WB) *reinterpret_cast<uint32_t*>(&codes[tid][CH]) = 0u;     // what a word task reads past the chunk
-  float s = 0.f;
-  const bool cs = t.col_scales != 0;
-  if (cs) {
-    // variant: one scale per column.  Block maxima are [W][nblk][RP]; thread tid only meets column tid % RP.
-    for (int i = tid; i < W * nblk * RP; i += 256) s = fmaxf(s, __ldg(maxes + i));
-#pragma unroll
-    for (int o = 16; o >= RP; o >>= 1) s = fmaxf(s, __shfl_xor_sync(0xffffffffu, s, o));
-    if ((tid & 31) < RP) scol8[tid >> 5][tid & 31] = s;
-    __syncthreads();
-    if (tid < RP) {
-      float a = scol8[0][tid];
-#pragma unroll
-      for (int i = 1; i < 8; ++i) a = fmaxf(a, scol8[i][tid]);
-      scol[tid] = a;
-    }
-    __syncthreads();
-  } else {
-    for (int i = tid; i < W * nblk; i += 256) s = fmaxf(s, __ldg(maxes + i));
-#pragma unroll
-    for (int o = 16; o >= 1; o >>= 1) s = fmaxf(s, __shfl_xor_sync(0xffffffffu, s, o));
-    if ((tid & 31) == 0) sred[tid >> 5] = s;
-    __syncthreads();
-    s = sred[0];
-#pragma unroll
-    for (int i = 1; i < 8; ++i) s = fmaxf(s, sred[i]);
-    if (sx.pack_only) s = sx.scales[which * sx.n_mat + ch.layer];   // scale agreed between the ranks
-  }
-  // scales, status: once per layer
-  if (ch.chunk == 0 && (cs ? tid < r : tid == 0)) {
-    const float sj = cs ? scol[tid] : s;
-    L.scales[cs ? which * RP + tid : which] = sj;
-    for (int w = 0; w < W; ++w) {
-      float* ps = reinterpret_cast<float*>(t.payload + (size_t)w * t.payload_stride + L.pay_scale_off);
-      ps[cs ? which * r + tid : which] = sj;
-    }
-    if (B != 32 && !(sj > 0.f)) atomicOr(&t.status[ch.layer], which ? 4u : 2u);
-    if (!(sj < INFINITY)) atomicOr(&t.status[ch.layer], 8u);
-  }
-
-  if constexpr (B == 32) {
-    // Quantiser bypassed (plain PowerSGD exchange): the factor travels as fp32 and the workers'
-    // factors are averaged directly (Eq. 1), in worker order.
-    const int e = ch.chunk * CH + tid;
-    if (e < count) {
-      const int row = e / r, col = e - row * r;
-      float sum = 0.f;
-      for (int w = 0; w < W; ++w) {
-        const float x = __ldg(src + ((size_t)w * rows + row) * RP + col);
-        sum += x;
-        uint8_t* pay = t.payload + (size_t)w * t.payload_stride + pay_off + (size_t)e * 4;
-        const unsigned bits32 = __float_as_uint(x);               // the stream may start on any byte
-        pay[0] = bits32 & 0xff; pay[1] = (bits32 >> 8) & 0xff; pay[2] = (bits32 >> 16) & 0xff; pay[3] = bits32 >> 24;
-      }
-      store_factor<RP>(L, which, row, col, sum / (float)W);
-    }
-    return;
-  } else {
-    constexpr int NW = CH * B / 32;      // 32-bit words of one worker's stream in this chunk
-    const int e0 = ch.chunk * CH;
-    const int cnt = min(CH, count - e0);
-    const bool valid = tid < cnt;
-    const int e = e0 + tid;
-    const int row = valid ? e / r : 0, col = valid ? e % r : 0;
-    if (cs) s = scol[col];
-    const bool s_ok = (s > 0.f) && (s < INFINITY);
-    const size_t nbytes_total = ((size_t)count * B + 7) / 8;
-    const size_t byte0 = (size_t)ch.chunk * (CH / 8) * B;
-    const int nbytes = (int)min((size_t)(CH / 8) * B, nbytes_total - byte0);
-    int S = 0;
-    float Sv = 0.f;          // value-domain variant: sum of the workers' dequantised levels, in worker order
-
-    for (int w0 = 0; w0 < W; w0 += WB) {
-      const int wn = min(WB, W - w0);
-      float x[WB];
-#pragma unroll
-      for (int u = 0; u < WB; ++u)
-        x[u] = (valid && u < wn) ? __ldg(src + ((size_t)(w0 + u) * rows + row) * RP + col) : 0.f;
-#pragma unroll
-      for (int u = 0; u < WB; ++u) {
-        if (u < wn) {
-          int k = 0;
-          if (s_ok && valid) {
-            const float tt = __fdiv_rn(fabsf(x[u]), s);
-            // k = #{i : tt >= thr[i]}, thr ascending, NLEV - 1 = 2^(B-1) - 1 entries: B - 1 halving steps
-#pragma unroll
-            for (int step = NLEV / 2; step >= 1; step >>= 1)
-              if (tt >= thr[k + step - 1]) k += step;
-          }
-          const int neg = (valid && x[u] < 0.f) ? 1 : 0;
-          codes[u][tid] = (uint8_t)((neg << (B - 1)) | k);   // 0 beyond the factor's end: pads the last byte
-          const int sk = neg ? -k : k;
-          S += sk;
-          if (qt.avg_values) Sv += __ldg(qt.deq + sk + (NLEV - 1));
-        }
-      }
-      __syncthreads();
-      // little-endian bit stream: word j of the chunk holds bits [32 j, 32 j + 32) = the codes of
-      // elements 32 j / B .. (32 j + 31) / B
-      for (int task = tid; task < wn * NW; task += 256) {
-        const int u = task / NW, j = task - u * NW;
-        const int bit0 = 32 * j;
-        const int q0 = bit0 / B;
-        uint32_t word = 0;
-#pragma unroll
-        for (int i = 0; i < 32 / B + 2; ++i) {
-          const int q = q0 + i;
-          const int sh = q * B - bit0;
-          if (sh < 32) {
-            const uint32_t c = codes[u][min(q, CH + 3)];
-            word |= (sh >= 0) ? (c << sh) : (c >> (-sh));
-          }
-        }
-        const int nb = min(4, nbytes - 4 * j);       // bytes of this word inside the stream
-        uint8_t* pay = t.payload + (size_t)(w0 + u) * t.payload_stride + pay_off + byte0 + 4 * j;
-        uint8_t* snd = sx.pack_only
-            ? sx.send[which] + (size_t)(w0 + u) * sx.region_bytes[which] + (pay_off - sx.region_off[which]) + byte0 + 4 * j
-            : nullptr;
-        if (nb == 4 && (reinterpret_cast<uintptr_t>(pay) & 3) == 0) *reinterpret_cast<uint32_t*>(pay) = word;
-        else
-          for (int i = 0; i < nb; ++i) pay[i] = (uint8_t)(word >> (8 * i));
-        if (snd) {           // the same stream, contiguous over the local workers, for the all-gather
-          if (nb == 4 && (reinterpret_cast<uintptr_t>(snd) & 3) == 0) *reinterpret_cast<uint32_t*>(snd) = word;
-          else
-            for (int i = 0; i < nb; ++i) snd[i] = (uint8_t)(word >> (8 * i));
-        }
-      }
-      __syncthreads();
-    }
-
-    if (valid && !sx.pack_only) {
-      float v = 0.f;
-      if (s_ok) v = qt.avg_values ? s * (Sv / (float)W) : s * __ldg(qt.deq + S + W * (NLEV - 1));
-      store_factor<RP>(L, which, row, col, v);
-    }
-  }
+  __shared__ __align__(16) unsigned char smem[sizeof(ExchangeSmem<RP, 256>)];
+  exchange_body<RP, B, 256, false>(t, qt, which, chunks[blockIdx.x], sx, threadIdx.x, smem);
 }
 
 // One worker's unpacked codes (one per byte) from its packed stream: what lqsgd_get_state returns

@@ -105,27 +105,6 @@ __device__ __forceinline__ void bulk_wait_all0() { asm volatile("cp.async.bulk.w
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory"); }
 
-// Sums v[i] over the 32 lanes in log steps that halve the live values; afterwards lane l holds
-// indices [l*N/32, (l+1)*N/32) (N >= 32) or index l / (32/N) (N < 32).  Fixed order.
-template <int N, int O>
-__device__ __forceinline__ void warp_transpose_reduce(float* v, int lane) {
-  if constexpr (O >= 1) {
-    if constexpr (N > 1) {
-      constexpr int H = N / 2;
-      const bool up = (lane & O) != 0;
-#pragma unroll
-      for (int i = 0; i < H; ++i) {
-        const float a = v[i], b = v[i + H];
-        v[i] = (up ? b : a) + __shfl_xor_sync(0xffffffffu, up ? a : b, O);
-      }
-      warp_transpose_reduce<H, O / 2>(v, lane);
-    } else {
-      v[0] += __shfl_xor_sync(0xffffffffu, v[0], O);
-      warp_transpose_reduce<1, O / 2>(v, lane);
-    }
-  }
-}
-
 struct Ring {
   uint64_t* full;      // [NST] loads landed (tx bytes)
   uint64_t* consumed;  // [NST] consumers done (one arrival per consumer warp)

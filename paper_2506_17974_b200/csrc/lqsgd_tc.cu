@@ -838,7 +838,7 @@ tc_pass3_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
           const int s = kc % kT3Stages;
           uint32_t gh[32];
           tc_ld32(taddr + pc * 32, gh);
-          if (!warp_wait(m_full + s, (kc / kT3Stages) & 1, abort_flag, lane)) { ok = false; break; }
+          if (!warp_wait(m_full + s, (kc / kT3Stages) & 1, abort_flag, lane)) { tc_wait_ld(); ok = false; break; }
           tc_wait_ld();
           uint8_t* mp = piece(s) + row_in_tile * 128;
 #pragma unroll

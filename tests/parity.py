@@ -22,10 +22,14 @@ MAX_FLIP_FRACTION = 1e-5
 STAGE_ULPS = 4.0
 # Free-running: the oracle's factor differs from the device's by the fp32 rounding of everything
 # upstream, so codes next to a threshold may differ; the oracle adopts the device's code there.
-# Gates: distance from the threshold in level units, and the fraction of codes adopted (set to
-# about ten times the largest values observed over the whole suite, which the tests print).
-FREE_MARGIN = 2e-2
-FREE_FRACTION = 2e-3
+# Gates: distance from the threshold in level units, and the fraction of codes adopted, about ten
+# times (tensor-core ranks: five times) the largest values observed over the whole suite, which the
+# tests print and PARITY_STATS_DIR collects: ranks <= 8 (fp32 FMA products) 4.1e-5 and 6.9e-6 over
+# 2.4e7 codes; ranks 9..32 (products from split tf32 / bf16 terms, relative rounding up to 2^-17 of M)
+# 4.1e-3 and 1.6e-4 over 2.1e7 codes.  Stage-isolated: 0 differing codes in 1.2e8.
+def free_gates(rank):
+    return (4e-4, 7e-5) if rank <= 8 else (2e-2, 1.6e-3)
+
 
 ALL_STATS = []      # one dict per test that ran run-level statistics (written out at session end)
 
@@ -198,6 +202,7 @@ def codes_differ(a, b, bits):
 
 
 def oracle_step_forced(oracle: orc.Oracle, grads_host, recs, stats):
+    FREE_MARGIN = free_gates(oracle.rank)[0]
     """Free-running oracle step that adopts the device's code where its own differs (counted).
     Returns the oracle's per-layer results."""
     forced = {}

@@ -50,7 +50,8 @@ def run_steps(w: wl.Workload, steps: int, free_run=True, comp=None, allow_status
     assert stats["flips"] <= par.MAX_FLIP_FRACTION * stats["codes"], stats
     stats["flip_fraction"] = stats["flips"] / stats["codes"]
     if free_run:
-        assert stats.get("forced", 0) <= par.FREE_FRACTION * stats["free_codes"], stats
+        # a lone adopted code is let through on sets of a few thousand codes, where the fraction says nothing
+        assert stats.get("forced", 0) <= max(1, par.free_gates(comp.rank)[1] * stats["free_codes"]), stats
         stats["forced_fraction"] = stats.get("forced", 0) / stats["free_codes"]
     shown = {k: (f"{v:.2e}" if isinstance(v, float) else v) for k, v in stats.items()}
     print(w.name, shown)
@@ -59,21 +60,33 @@ def run_steps(w: wl.Workload, steps: int, free_run=True, comp=None, allow_status
     return comp, stats
 
 
-def test_config1_single_matrix_ten_steps():
-    run_steps(wl.config1(), 10)
+# one_launch=True: the round as ONE cooperative kernel with M resident in shared memory (for sets that fit), next
+# to the default sequence of kernels that streams M through memory: both implementations meet the oracle on the
+# same cases.
+@pytest.mark.parametrize("one_launch", [False, True])
+def test_config1_single_matrix_ten_steps(one_launch):
+    comp = make(wl.config1(), one_launch=one_launch)
+    assert (comp.launches_per_step == 1) == one_launch
+    run_steps(wl.config1(), 10, comp=comp)
 
 
-def test_config2_mnist_cnn_four_workers():
-    run_steps(wl.config2(), 6)
+@pytest.mark.parametrize("one_launch", [False, True])
+def test_config2_mnist_cnn_four_workers(one_launch):
+    comp = make(wl.config2(), one_launch=one_launch)
+    assert (comp.launches_per_step == 1) == one_launch
+    run_steps(wl.config2(), 6, comp=comp)
 
 
 def test_config3_resnet18_eight_workers():
     run_steps(wl.config3(), 2)
 
 
-@pytest.mark.parametrize("rows,cols", [(1024, 4096), (4096, 4096)])
-def test_config4_large_layers(rows, cols):
-    run_steps(wl.config4(rows, cols), 2)
+@pytest.mark.parametrize("rows,cols,one_launch", [(1024, 4096, False), (1024, 4096, True), (4096, 4096, False), (4096, 4096, True)])
+def test_config4_large_layers(rows, cols, one_launch):
+    w = wl.config4(rows, cols)
+    comp = make(w, one_launch=one_launch)
+    assert (comp.launches_per_step == 1) == (rows == 1024 and one_launch)     # 16.8 MB fit on chip, 67 MB do not
+    run_steps(w, 2, comp=comp)
 
 
 def test_config4_4096x16384_stage_isolated():
@@ -130,10 +143,13 @@ def test_staged_and_register_paths_agree():
 
 @pytest.mark.parametrize("shape", [(2, 2), (3, 5), (5, 3), (17, 33), (33, 17), (40, 129), (130, 36), (64, 27), (10, 512)])
 @pytest.mark.parametrize("rank,bits,W", [(1, 2, 1), (3, 3, 2), (7, 5, 3), (16, 8, 2)])
-def test_small_and_ragged_shapes(shape, rank, bits, W):
+@pytest.mark.parametrize("one_launch", [False, True])
+def test_small_and_ragged_shapes(shape, rank, bits, W, one_launch):
+    if one_launch and rank == 16:
+        pytest.skip("rank 16 always runs as a sequence of kernels")
     w = wl.Workload("tiny", (shape, (7, 1), (1, 5)), rank=rank, bits=bits, workers=W, steps=3,
                     dist="normal", scale="fan_in", seed=shape[0] * 1000 + shape[1])
-    comp = make(w)
+    comp = make(w, one_launch=one_launch)
     stats = {}
     oracle = new_oracle(comp)
     for t in range(3):
@@ -313,6 +329,24 @@ def test_unaligned_layers_as_plain_tiles_and_on_the_register_path(rank):
     only_small = make(dataclasses.replace(w, layers=small))
     assert only_small.launches_per_step == 7
     run_steps(dataclasses.replace(w, layers=small), 1, comp=only_small)
+    # the one-launch round takes the small set (unaligned layers as plain tiles), not the one with the large unaligned layer
+    assert make(w, one_launch=True).launches_per_step == 9
+    on_chip = make(dataclasses.replace(w, layers=small), one_launch=True)
+    assert on_chip.launches_per_step == 1
+    run_steps(dataclasses.replace(w, layers=small), 2, comp=on_chip)
+
+
+@pytest.mark.parametrize("kw", [dict(average="values"), dict(column_scales=True), dict(bits_p=3, bits_q=7), dict()])
+def test_one_launch_round_variants(kw):
+    """The exchange's variants inside the one-launch round: value-domain average, column scales, different bit
+    counts for the two factors; a tall layer (two-step Orthonormalize), an unaligned one, 1-D tensors, 5 workers."""
+    w = wl.Workload("one", ((96, 200), (130, 36), (64, 27), (20, 1), (700, 512), (1, 33)), rank=5, bits=5, workers=5,
+                    steps=3, dist="student_t3", scale="fan_in", seed=61)
+    comp = make(w, one_launch=True, **kw)
+    assert comp.launches_per_step == 1
+    run_steps(w, 3, comp=comp)
+    tl = comp.round_timeline()
+    assert len(tl) >= 6 and all(b >= a for a, b in zip(tl, tl[1:]))       # the kernel's own timeline of the round
 
 
 def test_different_bits_for_p_and_q():
@@ -360,10 +394,10 @@ def test_full_size_largest_layer_properties():
     assert resid <= 4e-7 * g[0][0].abs().max().item()
 
 
-@pytest.mark.parametrize("rank", [3, 16])
-def test_zero_gradient_sets_status_and_zero_outputs(rank):
+@pytest.mark.parametrize("rank,one_launch", [(3, False), (16, False), (3, True)])
+def test_zero_gradient_sets_status_and_zero_outputs(rank, one_launch):
     layers = ((40, 64), (16, 1))
-    comp = B.LQSGD(layers, rank, 4, workers=2)
+    comp = B.LQSGD(layers, rank, 4, workers=2, one_launch=one_launch)
     grads = [[torch.zeros(s, device=DEV) for s in layers] for _ in range(2)]
     ghat = [torch.full(s, 7.0, device=DEV) for s in layers]
     comp.step(grads, ghat)
@@ -379,12 +413,12 @@ def test_zero_gradient_sets_status_and_zero_outputs(rank):
     assert res["dependent"].all() and np.all(res["G_hat"] == 0)
 
 
-@pytest.mark.parametrize("rank", [3, 12, 24])
-def test_dependent_column_matches_oracle(rank):
+@pytest.mark.parametrize("rank,one_launch", [(3, False), (12, False), (24, False), (3, True)])
+def test_dependent_column_matches_oracle(rank, one_launch):
     """Q with two identical columns: the second column of M Q is dependent and becomes zero
     (ranks 12 and 24 run the products on the tensor cores)."""
     layers = ((48, 80),)
-    comp = B.LQSGD(layers, rank, 4, workers=1)
+    comp = B.LQSGD(layers, rank, 4, workers=1, one_launch=one_launch)
     Q = torch.randn(80, rank, generator=torch.Generator().manual_seed(3))
     Q[:, 1] = Q[:, 0]
     comp.set_state(B.STATE_Q, 0, 0, Q)
@@ -420,19 +454,21 @@ def test_non_finite_gradient_is_flagged_without_a_fault(rank):
     assert b.status() == [0, 0]
 
 
-@pytest.mark.parametrize("rank,pass_", [(2, 1), (2, 3), (8, 1), (8, 3), (16, 1), (16, 2), (16, 3)])
-def test_bounded_wait_runs_out_and_reports_timeout(rank, pass_):
+@pytest.mark.parametrize("rank,pass_,stage", [(2, 1, 0), (2, 3, 0), (8, 1, 0), (8, 3, 0), (16, 1, 0), (16, 2, 0), (16, 3, 0),
+                                              (16, 1, 3), (2, 4, 0), (8, 4, 3), (4, 4, 2)])
+def test_bounded_wait_runs_out_and_reports_timeout(rank, pass_, stage):
     """The path a bounded device-side wait takes when it runs out (ranks 2 and 8: the bulk-copy staged passes,
-    rank 16: the tcgen05 passes).  The test hook makes CTA 0's loader leave out one stage of copies and shortens
-    the limit of the waits; nothing faults or spins without a limit: the kernel returns, the layer's status word
+    rank 16: the tcgen05 passes, pass 4: a grid barrier of the one-launch round).  The test hook makes CTA 0's
+    loader stop issuing copies (or CTA 0 stay away from a grid barrier) and shortens the limit of the waits; nothing faults or spins without a limit: the kernel returns, the layer's status word
     carries LQSGD_STATUS_TIMEOUT, and once E and Q are restored the context computes, bit for bit, what a fresh
     context computes - which is checked against the oracle."""
     layers = ((256, 512), (24, 1))
     w = wl.Workload("expire", layers, rank=rank, bits=4, workers=2, steps=3, dist="normal", scale="fan_in", seed=6)
-    comp, ref = make(w), make(w)
+    comp, ref = make(w, one_launch=pass_ == 4), make(w, one_launch=pass_ == 4)
+    assert (comp.launches_per_step == 1) == (pass_ == 4)
     out = [torch.empty(s, device=DEV) for s in layers]
     out_ref = [torch.empty(s, device=DEV) for s in layers]
-    comp.test_expire_wait(pass_, 0, 256)
+    comp.test_expire_wait(pass_, stage, 256)
     t0 = time.time()
     comp.step(wl.draw_gradients(w, 0, device=DEV), out)
     torch.cuda.synchronize()
@@ -460,10 +496,10 @@ def test_bounded_wait_runs_out_and_reports_timeout(rank, pass_):
         comp.test_expire_wait(1, 0, 8)
 
 
-@pytest.mark.parametrize("rank", [4, 16])
-def test_bit_reproducible_and_checkpoint_resume(rank):
+@pytest.mark.parametrize("rank,one_launch", [(4, False), (16, False), (4, True)])
+def test_bit_reproducible_and_checkpoint_resume(rank, one_launch):
     w = dataclasses.replace(wl.config2(), workers=3, rank=rank)
-    a, b = make(w), make(w)
+    a, b = make(w, one_launch=one_launch), make(w, one_launch=one_launch)
     gh = lambda: [torch.empty(s, device=DEV) for s in w.layers]
     oa, ob = gh(), gh()
     for t in range(4):
@@ -476,7 +512,7 @@ def test_bit_reproducible_and_checkpoint_resume(rank):
     for wk in range(3):
         assert torch.equal(a.payload(wk), b.payload(wk))
     # resume: copy E and Q of `a` after 4 steps into a fresh context, then both take step 4
-    c = make(w)
+    c = make(w, one_launch=one_launch)
     for l in range(len(w.layers)):
         if c.is_matrix(l):
             c.set_state(B.STATE_Q, l, 0, a.get_state(B.STATE_Q, l))
@@ -493,11 +529,12 @@ def test_bit_reproducible_and_checkpoint_resume(rank):
     assert torch.equal(a.get_state(B.STATE_E, 2, 2), c.get_state(B.STATE_E, 2, 2))
 
 
-def test_step_replays_from_a_cuda_graph():
-    """A step captured into a CUDA graph (kernels only, dependent launches included) replays to
-    the same bits as eager steps; a capture with unseen tensor pointers is refused."""
+@pytest.mark.parametrize("one_launch", [False, True])
+def test_step_replays_from_a_cuda_graph(one_launch):
+    """A step captured into a CUDA graph (kernels only, dependent launches included; or the one cooperative
+    launch) replays to the same bits as eager steps; a capture with unseen tensor pointers is refused."""
     w = dataclasses.replace(wl.config2(), workers=2)
-    a, b = make(w), make(w)
+    a, b = make(w, one_launch=one_launch), make(w, one_launch=one_launch)
     g0 = wl.draw_gradients(w, 0, device=DEV)
     bufs = [[torch.empty_like(x) for x in per] for per in g0]
     other = [[torch.empty_like(x) for x in per] for per in g0]
@@ -633,11 +670,13 @@ def test_argument_errors_launch_nothing():
     torch.cuda.synchronize()
 
 
-def test_quantiser_bypass_is_plain_powersgd():
+@pytest.mark.parametrize("one_launch", [False, True])
+def test_quantiser_bypass_is_plain_powersgd(one_launch):
     """bits = 32: factors travel as fp32 and are averaged directly (Section III-B, Eq. 1)."""
     w = wl.Workload("bypass", ((96, 200), (130, 36), (20, 1)), rank=4, bits=32, workers=3, steps=3,
                     dist="student_t3", scale="fan_in", seed=9)
-    comp = make(w)
+    comp = make(w, one_launch=one_launch)
+    assert (comp.launches_per_step == 1) == one_launch
     oracle = new_oracle(comp)
     assert comp.payload_nbytes == orc.payload_bytes(w.layers, 4, 32, 32) == 4 * 4 * (96 + 200 + 130 + 36) + 16 + 80
     for t in range(3):
@@ -683,13 +722,13 @@ def test_planted_rank_r_gradient_is_recovered_on_the_device():
     assert float(comp.get_state(B.STATE_E, 0, 0).abs().max()) <= 1e-4 * float(G.abs().max())
 
 
-@pytest.mark.parametrize("rank", [4, 16])
-def test_fused_model_update_matches_separate_update(rank):
+@pytest.mark.parametrize("rank,one_launch", [(4, False), (16, False), (4, True)])
+def test_fused_model_update_matches_separate_update(rank, one_launch):
     """Algorithm 1's last line, w <- w - lr * G_hat, fused into pass 3: same weights as updating
     from the G_hat a plain step returns (and as the oracle's G_hat), with and without G_hat output.
     Rank 16 runs it in the tensor-core pass 3."""
     w = dataclasses.replace(wl.config2(), workers=2, rank=rank)   # includes a 32 x 25 layer and 1-D tensors
-    a, b, c = make(w), make(w), make(w)
+    a, b, c = make(w, one_launch=one_launch), make(w, one_launch=one_launch), make(w, one_launch=one_launch)
     lr = 0.125
     gen = torch.Generator(DEV).manual_seed(1)
     w0 = [torch.randn(s, device=DEV, generator=gen) for s in w.layers]
