@@ -115,7 +115,7 @@ typedef struct lqsgd_shape {
 /* Inputs of Algorithm 1 (rank r, bits b_p and b_q, curvature alpha) plus the worker count. */
 typedef struct lqsgd_config {
   uint32_t struct_size; /* sizeof(lqsgd_config), for versioning */
-  int32_t rank;         /* r, 1..32 (any integer); from 9 up the products of aligned layers run on the tensor cores */
+  int32_t rank;         /* r, 1..64 (any integer); from 9 up the products of aligned layers run on the tensor cores */
   int32_t bits_p;       /* b_p, total bits per P scalar including the sign, 2..8; 32 = no quantiser: the
                            factor is sent as fp32 and averaged directly (the PowerSGD exchange of Section III-B) */
   int32_t bits_q;       /* b_q, likewise for Q */

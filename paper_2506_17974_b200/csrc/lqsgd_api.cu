@@ -120,7 +120,7 @@ struct Plan {
   size_t bytes = 0;
 };
 
-int padded_rank(int r) { return r <= 1 ? 1 : r <= 2 ? 2 : r <= 4 ? 4 : r <= 8 ? 8 : r <= 16 ? 16 : 32; }
+int padded_rank(int r) { return r <= 1 ? 1 : r <= 2 ? 2 : r <= 4 ? 4 : r <= 8 ? 8 : r <= 16 ? 16 : r <= 32 ? 32 : 64; }
 
 int check_config(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config* c) {
   if (!shapes || !c || n_layers < 1) return LQSGD_ERR_INVALID_ARG;

@@ -6,14 +6,14 @@
 
 namespace lqsgd {
 
-constexpr int kMaxRank = 32;           // padded rank 32: the tensor-core passes' shared memory ends there
+constexpr int kMaxRank = 64;           // padded rank 64: the tensor-core passes' shared memory and tensor memory end there
 constexpr int kPassThreads = 256;      // threads per CTA of the three streaming passes
 constexpr int kPass1Rows = 32;         // rows per pass-1 tile: 8 warps x 4 rows
 constexpr int kFactorBlockRows = 128;  // rows of P (or Q) per block of the small factor kernels
 constexpr int kExchangeChunk = 256;    // factor elements per block of the exchange kernel
 
 // One matrix layer (n x m), as the kernels see it.  Factors are stored with a row stride of
-// RP floats (rank padded to 1, 2, 4, 8, 16 or 32); columns >= r are kept zero.
+// RP floats (rank padded to 1, 2, 4, 8, 16, 32 or 64); columns >= r are kept zero.
 struct LayerDev {
   int32_t n, m, r;            // r = r_eff
   int32_t vec;                // 1: m % 4 == 0, rows are 16-byte aligned -> float4 path

@@ -69,7 +69,7 @@ __device__ __forceinline__ void store_contig(float* p, const float (&v)[N]) {
 // ---------------------------------------------------------------------------------------
 constexpr double kPivotEps = 1e-10;
 
-template <int RP> struct ReduceGramSmem { double rows[kFactorBlockRows][RP]; };   // the block's rows, converted once
+template <int RP> struct ReduceGramSmem { float rows[kFactorBlockRows][RP]; };   // the block's rows (fp32: they are fp32 data)
 
 template <int RP, int NT, bool COH>
 __device__ __forceinline__ void p_reduce_gram_body(const Tables& t, const FactorBlock fb, int tid, void* smem) {
@@ -105,14 +105,14 @@ __device__ __forceinline__ void p_reduce_gram_body(const Tables& t, const Factor
       if (L.ncc > 1) store_contig<RP>(L.Praw + ((size_t)fb.worker * n + row) * RP, p);
     }
 #pragma unroll
-    for (int j = 0; j < RP; ++j) S.rows[tid][j] = (double)p[j];
+    for (int j = 0; j < RP; ++j) S.rows[tid][j] = p[j];
   }
   __syncthreads();
   for (int e = tid; e < RP * RP; e += NT) {
     const int i = e / RP, j = e % RP;
     if (j < i) continue;                                 // the Gram matrix is symmetric: upper triangle, mirrored
     double s = 0.0;
-    for (int k = 0; k < kFactorBlockRows; ++k) s = fma(S.rows[k][i], S.rows[k][j], s);
+    for (int k = 0; k < kFactorBlockRows; ++k) s = fma((double)S.rows[k][i], (double)S.rows[k][j], s);
     double* gp = L.gram_part + ((size_t)fb.worker * L.npb + fb.blk) * (RP * RP);
     gp[i * RP + j] = s;
     gp[j * RP + i] = s;
@@ -120,12 +120,11 @@ __device__ __forceinline__ void p_reduce_gram_body(const Tables& t, const Factor
 }
 
 // Cholesky of the Gram matrix in A (shared, complete and visible to the CTA on entry):  Gram = L L^T  (R = L^T).
-// Lf (shared, RP*RP doubles, row-major) receives L, invd the reciprocals of its diagonal, dead[j] = 1 for a
-// column dropped as dependent (its row and column of L are then those of the identity).  Returns true if
-// any column was dropped.
+// On return the lower triangle of A holds L, invd the reciprocals of its diagonal, dead[j] = 1 for a column
+// dropped as dependent (its row and column of L are then those of the identity).  Returns true if any column
+// was dropped.
 template <int RP, int NT>
-__device__ __forceinline__ bool cholesky_factor(double (*A)[RP + 1], double* diag0, int r, double* Lf, double* invd, int* dead,
-                                                int tid) {
+__device__ __forceinline__ bool cholesky_factor(double (*A)[RP + 1], double* diag0, int r, double* invd, int* dead, int tid) {
   if (tid < RP) { diag0[tid] = A[tid][tid]; dead[tid] = 0; invd[tid] = 1.0; }
   __syncthreads();
   // right-looking Cholesky by ONE warp (warp-level barriers only; the other warps wait once, below):
@@ -157,13 +156,8 @@ __device__ __forceinline__ bool cholesky_factor(double (*A)[RP + 1], double* dia
     }
   }
   __syncthreads();
-  for (int e = tid; e < RP * RP; e += NT) {
-    const int i = e / RP, k = e % RP;
-    Lf[e] = (k <= i && i < r) ? A[i][k] : 0.0;
-  }
   int any = 0;
   for (int j = 0; j < r; ++j) any |= dead[j];
-  __syncthreads();
   return any != 0;
 }
 
@@ -173,13 +167,12 @@ __device__ __forceinline__ bool cholesky_factor(double (*A)[RP + 1], double* dia
 template <int RP> struct CholSmem {
   static constexpr int SEG = (RP * RP <= 64) ? 128 / (RP * RP) : 1;   // at least 128 threads take part
   double A[RP][RP + 1];                // Gram, overwritten by L (lower triangle)
-  double segsum[SEG][RP * RP];
+  double segsum[SEG > 1 ? SEG : 1][SEG > 1 ? RP * RP : 1];
   double diag0[RP];
 };
 
 template <int RP, int NT, bool COH>
-__device__ __forceinline__ bool cholesky_lower(const LayerDev& L, int worker, CholSmem<RP>& C, double* Lf, double* invd,
-                                               int* dead, int tid) {
+__device__ __forceinline__ bool cholesky_lower(const LayerDev& L, int worker, CholSmem<RP>& C, double* invd, int* dead, int tid) {
   // Gram = sum of the block Grams.  With more threads than entries the blocks are dealt to SEG
   // segments (segment g takes blocks g, g + SEG, ...), eight loads in flight each; the segments'
   // sums are then added in segment order: a fixed order, and a chain SEG times shorter.
@@ -224,12 +217,11 @@ __device__ __forceinline__ bool cholesky_lower(const LayerDev& L, int worker, Ch
     }
   }
   __syncthreads();
-  return cholesky_factor<RP, NT>(C.A, C.diag0, L.r, Lf, invd, dead, tid);
+  return cholesky_factor<RP, NT>(C.A, C.diag0, L.r, invd, dead, tid);
 }
 
 template <int RP, int NT> struct ApplySmem {
   CholSmem<RP> chol;
-  double Lf[RP * RP];
   double invd[RP];
   int dead[RP];
   float smax[NT / 32];
@@ -243,7 +235,7 @@ __device__ __forceinline__ void p_apply_body(const Tables& t, const FactorBlock 
   auto& S = *static_cast<ApplySmem<RP, NT>*>(smem);
   const LayerDev& L = t.layers[fb.layer];
   const int n = L.n;
-  const bool dropped = cholesky_lower<RP, NT, COH>(L, fb.worker, S.chol, S.Lf, S.invd, S.dead, tid);
+  const bool dropped = cholesky_lower<RP, NT, COH>(L, fb.worker, S.chol, S.invd, S.dead, tid);
   if (dropped && fb.blk == 0 && tid == 0) atomicOr(&t.status[fb.layer], 1u);
   const int row = fb.blk * kFactorBlockRows + tid;
   float o[RP];
@@ -261,7 +253,7 @@ __device__ __forceinline__ void p_apply_body(const Tables& t, const FactorBlock 
     for (int j = 0; j < RP; ++j) {
       double s = (double)p[j];
 #pragma unroll
-      for (int k = 0; k < j; ++k) s = fma(-od[k], S.Lf[j * RP + k], s);
+      for (int k = 0; k < j; ++k) s = fma(-od[k], S.chol.A[j][k], s);
       od[j] = (j < L.r && !S.dead[j]) ? s * S.invd[j] : 0.0;
       o[j] = (float)od[j];
       amax = fmaxf(amax, fabsf(o[j]));
@@ -311,7 +303,6 @@ template <int RP> struct OrthSmallSmem {
   double seg[NSEG][NE];
   double A[RP][RP + 1];
   double diag0[RP];
-  double Lf[NE];
   double invd[RP];
   int dead[RP];
   float wmax[kOrthSmallRows / 32][RP];
@@ -359,7 +350,7 @@ __device__ __forceinline__ void p_orth_small_body(const Tables& t, const FactorB
     }
   }
   __syncthreads();
-  const bool dropped = cholesky_factor<RP, kOrthSmallRows>(S.A, S.diag0, L.r, S.Lf, S.invd, S.dead, tid);
+  const bool dropped = cholesky_factor<RP, kOrthSmallRows>(S.A, S.diag0, L.r, S.invd, S.dead, tid);
   if (dropped && tid == 0) atomicOr(&t.status[fb.layer], 1u);
   float o[RP];
 #pragma unroll
@@ -371,7 +362,7 @@ __device__ __forceinline__ void p_orth_small_body(const Tables& t, const FactorB
     for (int j = 0; j < RP; ++j) {
       double s = (double)p[j];
 #pragma unroll
-      for (int k = 0; k < j; ++k) s = fma(-od[k], S.Lf[j * RP + k], s);
+      for (int k = 0; k < j; ++k) s = fma(-od[k], S.A[j][k], s);
       od[j] = (j < L.r && !S.dead[j]) ? s * S.invd[j] : 0.0;
       o[j] = (float)od[j];
       bad |= !(fabsf(o[j]) < INFINITY);
@@ -569,7 +560,6 @@ template <int RP, int NT> struct ExchangeSmem {
   float thr[128];
   alignas(4) uint8_t codes[8][kExchangeChunk + 4];
   float sred[NT / 32];
-  float scol8[NT / 32][RP];
   float scol[RP];
 };
 
@@ -608,17 +598,11 @@ __device__ __forceinline__ void exchange_body(const Tables& t, const QuantTables
   const bool cs = t.col_scales != 0;
   if (cs) {
     // variant: one scale per column.  Block maxima are [W][nblk][RP]; thread tid only meets column tid % RP.
-    for (int i = tid; i < W * nblk * RP; i += NT) s = fmaxf(s, ld_in<COH>(maxes + i));
-#pragma unroll
-    for (int o = 16; o >= RP; o >>= 1) s = fmaxf(s, __shfl_xor_sync(0xffffffffu, s, o));
-    if ((tid & 31) < RP) S.scol8[tid >> 5][tid & 31] = s;
+    // (a maximum of non-negative floats is the maximum of their bit patterns as integers: exact, in any order)
+    if (tid < RP) S.scol[tid] = 0.f;
     __syncthreads();
-    if (tid < RP) {
-      float a = S.scol8[0][tid];
-#pragma unroll
-      for (int i = 1; i < NT / 32; ++i) a = fmaxf(a, S.scol8[i][tid]);
-      S.scol[tid] = a;
-    }
+    for (int i = tid; i < W * nblk * RP; i += NT) s = fmaxf(s, ld_in<COH>(maxes + i));
+    atomicMax(reinterpret_cast<int*>(S.scol) + tid % RP, __float_as_int(s));
     __syncthreads();
   } else {
     for (int i = tid; i < W * nblk; i += NT) s = fmaxf(s, ld_in<COH>(maxes + i));
@@ -749,7 +733,6 @@ __device__ __forceinline__ void exchange_body(const Tables& t, const QuantTables
 template <int RP, int NT> struct ExchangeLocalSmem {
   float thr[128];
   float sred[NT / 32];
-  float scol8[NT / 32][RP];
   float scol[RP];
 };
 
@@ -771,16 +754,10 @@ __device__ __noinline__ void exchange_rows_local(const Tables& t, const QuantTab
   const bool cs = t.col_scales != 0;
   if (bits != 32) {
     if (cs) {
-      for (int i = tid; i < W * nblk * RP; i += NT) s = fmaxf(s, ld_in<COH>(maxes + i));
-#pragma unroll
-      for (int o = 16; o >= RP; o >>= 1) s = fmaxf(s, __shfl_xor_sync(0xffffffffu, s, o));
-      if ((tid & 31) < RP) S.scol8[tid >> 5][tid & 31] = s;
+      if (tid < RP) S.scol[tid] = 0.f;
       __syncthreads();
-      if (tid < RP) {
-        float a = S.scol8[0][tid];
-        for (int i = 1; i < NT / 32; ++i) a = fmaxf(a, S.scol8[i][tid]);
-        S.scol[tid] = a;
-      }
+      for (int i = tid; i < W * nblk * RP; i += NT) s = fmaxf(s, ld_in<COH>(maxes + i));
+      atomicMax(reinterpret_cast<int*>(S.scol) + tid % RP, __float_as_int(s));      // non-negative floats order like their bits
       __syncthreads();
     } else {
       for (int i = tid; i < W * nblk; i += NT) s = fmaxf(s, ld_in<COH>(maxes + i));

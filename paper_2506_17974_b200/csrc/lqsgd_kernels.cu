@@ -725,7 +725,7 @@ vectors_quant_kernel(const VectorDev* __restrict__ vecs, const float* const* __r
 }  // namespace
 
 // ---------------------------------------------------------------------------------------
-// host launchers: dispatch on the padded rank RP in {1, 2, 4, 8, 16, 32}
+// host launchers: dispatch on the padded rank RP in {1, 2, 4, 8, 16, 32, 64}
 // ---------------------------------------------------------------------------------------
 #define LQSGD_DISPATCH_RP(RPV, ...)                 \
   switch (RPV) {                                    \
@@ -735,6 +735,7 @@ vectors_quant_kernel(const VectorDev* __restrict__ vecs, const float* const* __r
     case 8: { constexpr int RP = 8; __VA_ARGS__; } break;   \
     case 16: { constexpr int RP = 16; __VA_ARGS__; } break; \
     case 32: { constexpr int RP = 32; __VA_ARGS__; } break; \
+    case 64: { constexpr int RP = 64; __VA_ARGS__; } break; \
     default: return cudaErrorInvalidValue;          \
   }
 

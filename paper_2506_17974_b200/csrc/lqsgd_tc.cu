@@ -123,18 +123,20 @@ __device__ __forceinline__ int tile_stages(int nrows) {
 template <int RP>
 struct Pass2Cfg {
   static constexpr int kN = 3 * RP;                                      // stacked bf16 terms of P_bar
+  static constexpr int kAB = RP <= 32 ? kTcAB : 2;                       // operand slots: at padded rank 64 a B stage is 24 KB
   static constexpr int kDStride = kN <= 64 ? 64 : (kN <= 128 ? 128 : 256);   // TMEM columns per accumulator
-  static constexpr int kDBufs = (2 * kDStride + kTcAB * kTcSlotK <= 512) ? 2 : 1;
+  static constexpr int kDBufs = (2 * kDStride + kAB * kTcSlotK <= 512) ? 2 : 1;
   static constexpr int kACol0 = kDBufs * kDStride;
-  static constexpr int kTmemCols = (kACol0 + kTcAB * kTcSlotK) <= 256 ? 256 : 512;
+  static constexpr int kTmemCols = (kACol0 + kAB * kTcSlotK) <= 256 ? 256 : 512;
   static constexpr uint32_t kBBytes = kN * 128;                          // one B stage: 3 RP rows of 64 bf16
   static constexpr uint32_t kBStride = (kBBytes + 1023) / 1024 * 1024;   // stages stay 1024-byte aligned
   static constexpr int kMStages = RP <= 16 ? 8 : 6;                      // ring of M pieces (16 KB each): what fits beside B
   static constexpr uint32_t kBOff = kMStages * kTcMBytes;
-  static constexpr uint32_t kBarOff = kBOff + kTcAB * kTcPair * kBStride;
-  static constexpr int kBars = 2 * kMStages + 2 * kTcAB + 2 + 2 + 1;
+  static constexpr uint32_t kBarOff = kBOff + kAB * kTcPair * kBStride;
+  static constexpr int kBars = 2 * kMStages + 2 * kAB + 2 + 2 + 1;
   static constexpr uint32_t kTotal = kBarOff + kBars * 8 + 16 + 1024;    // + abort flag, TMEM slot, alignment slack
-  static_assert(kACol0 + kTcAB * kTcSlotK <= 512, "tensor memory");
+  static_assert(kACol0 + kAB * kTcSlotK <= 512, "tensor memory");
+  static_assert(kTotal <= 227 * 1024, "shared memory");
   static_assert(kN % 16 == 0 && kN <= 256, "N of one MMA");
 };
 
@@ -150,9 +152,9 @@ tc_pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, const uint
   uint64_t* bars = reinterpret_cast<uint64_t*>(base + S::kBarOff);
   uint64_t* m_full = bars;                       // [S::kMStages] TMA landed
   uint64_t* m_empty = m_full + S::kMStages;       // [S::kMStages] consumer warps have the piece in registers
-  uint64_t* ab_full = m_empty + S::kMStages;      // [kTcAB] slot ready: A written to TMEM (4 warps per stage) and B landed
-  uint64_t* ab_empty = ab_full + kTcAB;          // [kTcAB] the MMAs that read buffer i have completed
-  uint64_t* d_full = ab_empty + kTcAB;           // [2] accumulator complete
+  uint64_t* ab_full = m_empty + S::kMStages;      // [S::kAB] slot ready: A written to TMEM (4 warps per stage) and B landed
+  uint64_t* ab_empty = ab_full + S::kAB;          // [S::kAB] the MMAs that read buffer i have completed
+  uint64_t* d_full = ab_empty + S::kAB;           // [2] accumulator complete
   uint64_t* d_empty = d_full + 2;                // [2] accumulator drained
   uint64_t* fin = d_empty + 2;                   // [1] every MMA of this CTA has completed
   volatile int* abort_flag = reinterpret_cast<volatile int*>(fin + 1);
@@ -161,7 +163,7 @@ tc_pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, const uint
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
     for (int s = 0; s < S::kMStages; ++s) { mbar_init(m_full + s, 1); mbar_init(m_empty + s, 4); }
-    for (int s = 0; s < kTcAB; ++s) { mbar_init(ab_full + s, 4 * kTcPair + 1); mbar_init(ab_empty + s, 1); }
+    for (int s = 0; s < S::kAB; ++s) { mbar_init(ab_full + s, 4 * kTcPair + 1); mbar_init(ab_empty + s, 1); }
     for (int s = 0; s < 2; ++s) { mbar_init(d_full + s, 1); mbar_init(d_empty + s, 4); }
     mbar_init(fin, 1);
     wait_ctl_init(abort_flag, t.wait_limit);
@@ -207,8 +209,8 @@ tc_pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, const uint
       const uint8_t* map = maps + ((size_t)tl.layer * kTcMapsPerLayer + 1) * kTcMapBytes;
       const int nslots = tile_stages(tl.nrows) / kTcPair;
       for (int k = 0; k < nslots; ++k, ++kc) {            // kc counts slots here
-        const int s = kc % kTcAB;
-        if (!warp_wait(ab_empty + s, ((kc / kTcAB) & 1) ^ 1, abort_flag, lane)) { ok = false; break; }
+        const int s = kc % S::kAB;
+        if (!warp_wait(ab_empty + s, ((kc / S::kAB) & 1) ^ 1, abort_flag, lane)) { ok = false; break; }
         if (lane == 0) {
           mbar_arrive_expect_tx(ab_full + s, kTcPair * S::kBBytes);
 #pragma unroll
@@ -218,7 +220,7 @@ tc_pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, const uint
       }
     }
     if (!ok && lane == 0)
-      for (uint32_t it = kc > (uint32_t)kTcAB ? kc - kTcAB : 0; it < kc; ++it) drain(ab_full + it % kTcAB, (it / kTcAB) & 1, abort_flag);
+      for (uint32_t it = kc > (uint32_t)S::kAB ? kc - S::kAB : 0; it < kc; ++it) drain(ab_full + it % S::kAB, (it / S::kAB) & 1, abort_flag);
   } else if (warp == 2) {
     // ---- MMA issue: one thread
     if (lane == 0) {
@@ -233,8 +235,8 @@ tc_pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, const uint
         const uint32_t dpar = S::kDBufs == 2 ? ((tseq >> 1) & 1) : (tseq & 1);
         if (!thread_wait(d_empty + db, dpar ^ 1, abort_flag)) { ok = false; break; }
         for (int k = 0; k < nslots; ++k, ++kc) {            // kc counts slots here
-          const int s = kc % kTcAB;
-          if (!thread_wait(ab_full + s, (kc / kTcAB) & 1, abort_flag)) { ok = false; break; }
+          const int s = kc % S::kAB;
+          if (!thread_wait(ab_full + s, (kc / S::kAB) & 1, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint64_t bd0 = bdesc0 + (uint64_t)((s * kTcPair * S::kBStride) >> 4);
           const uint32_t acol = tmem + S::kACol0 + s * kTcSlotK;
@@ -301,7 +303,7 @@ tc_pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, const uint
       for (int k = 0; k < nk; ++k, ++kc) {
         if ((int)(kc % kTcGroups) != g) continue;
         const int s = kc % S::kMStages;
-        const uint32_t slot = kc / kTcPair, ab = slot % kTcAB;
+        const uint32_t slot = kc / kTcPair, ab = slot % S::kAB;
         if (!warp_wait(m_full + s, (kc / S::kMStages) & 1, abort_flag, lane)) { ok = false; break; }
         const float* src = mring + (size_t)s * (kTcMBytes / 4) + 32 * q + lane;
         uint32_t v[32];
@@ -316,7 +318,7 @@ tc_pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, const uint
           const __nv_bfloat16 a2 = __float2bfloat16_rn(r);
           v[kk] = a1 | (uint32_t)__bfloat16_as_ushort(a2);                      // a1 in the high half, a2 in the low half
         }
-        if (!warp_wait(ab_empty + ab, ((slot / kTcAB) & 1) ^ 1, abort_flag, lane)) { ok = false; break; }
+        if (!warp_wait(ab_empty + ab, ((slot / S::kAB) & 1) ^ 1, abort_flag, lane)) { ok = false; break; }
         tc_fence_after();
         tc_st32(lane_base + ab * kTcSlotK + (kc % kTcPair) * kTcK, v);
         tc_wait_st();
@@ -395,6 +397,7 @@ struct Pass1Cfg {
   static constexpr uint32_t kTotal = kBarOff + kBars * 8 + 16 + 1024;
   static_assert(kACol0 + kT1AB * 64 <= 512, "tensor memory");
   static_assert(kBBytes % 1024 == 0, "B stages stay 1024-byte aligned");
+  static_assert(kTotal <= 227 * 1024, "shared memory");
 };
 
 template <int RP>
@@ -665,13 +668,16 @@ __device__ __forceinline__ void tc_mma_tf32_ss(uint32_t tmem_d, uint64_t adesc, 
 template <int RP>
 struct Pass3Cfg {
   static constexpr int kCat = (3 * RP + 31) / 32 * 32;                   // K extent of the factor product
-  static constexpr int kSub = kCat / 32;                                 // 128-byte sub-tiles per operand
-  static constexpr uint32_t kOpBytes = kSub * kT1PieceBytes;             // one operand: kSub pieces of 128 rows x 32
+  static constexpr int kHalves = RP <= 32 ? 1 : 2;                       // the operands come in this many K slices, one after
+                                                                         // the other through the same buffer (rank 64: 2 x 96)
+  static constexpr int kSub = kCat / 32 / kHalves;                       // 128-byte sub-tiles per operand slice
+  static constexpr uint32_t kOpBytes = kSub * kT1PieceBytes;             // one operand slice: kSub pieces of 128 rows x 32
   static constexpr uint32_t kOpOff = kT3Stages * kT1PieceBytes;
   static constexpr uint32_t kBarOff = kOpOff + 2 * kOpBytes;
   static constexpr int kBars = 3 * kT3Stages + 2 + 2 + 2 + 2 + 1;      // m_full, e_ready, m_empty; op_full, op_empty, d_full, d_empty (2 each); fin
   static constexpr uint32_t kTotal = kBarOff + kBars * 8 + 16 + 1024;
   static constexpr int kTmemCols = 256;                                  // two accumulators of 128 columns
+  static_assert((kCat / 32) % kHalves == 0 && kTotal <= 227 * 1024, "operand slices, shared memory");
 };
 
 template <int RP>
@@ -742,44 +748,48 @@ tc_pass3_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
         drain(m_full + it % kT3Stages, (it / kT3Stages) & 1, abort_flag);
   } else if (warp == 1) {
     // ---- operand loader: the tile's rows of the stacked P_bar terms and its columns' rows of the Q_bar terms
-    uint32_t tseq = 0;
+    uint32_t oseq = 0;                      // operand slices loaded so far (kHalves per tile)
     bool ok = true;
-    for (int ti = t_begin; ti < t_end && ok; ++ti, ++tseq) {
+    for (int ti = t_begin; ti < t_end && ok; ++ti) {
       const Tile tl = tiles[ti];
       const uint8_t* mapp = maps + ((size_t)tl.layer * kTcMapsPerLayer + 4) * kTcMapBytes;
       const uint8_t* mapq = maps + ((size_t)tl.layer * kTcMapsPerLayer + 5) * kTcMapBytes;
-      if (!warp_wait(op_empty, (tseq & 1) ^ 1, abort_flag, lane)) { ok = false; break; }
-      if (lane == 0) {
-        mbar_arrive_expect_tx(op_full, 2 * S::kOpBytes);
+      for (int h = 0; h < S::kHalves; ++h, ++oseq) {
+        if (!warp_wait(op_empty, (oseq & 1) ^ 1, abort_flag, lane)) { ok = false; break; }
+        if (lane == 0) {
+          mbar_arrive_expect_tx(op_full, 2 * S::kOpBytes);
 #pragma unroll
-        for (int kt = 0; kt < S::kSub; ++kt) {
-          tma_load_2d(opa + (size_t)kt * kT1PieceBytes, mapp, kt * 32, tl.row0, op_full);
-          tma_load_2d(opb + (size_t)kt * kT1PieceBytes, mapq, kt * 32, tl.col0, op_full);
+          for (int kt = 0; kt < S::kSub; ++kt) {
+            tma_load_2d(opa + (size_t)kt * kT1PieceBytes, mapp, (h * S::kSub + kt) * 32, tl.row0, op_full);
+            tma_load_2d(opb + (size_t)kt * kT1PieceBytes, mapq, (h * S::kSub + kt) * 32, tl.col0, op_full);
+          }
         }
       }
     }
-    if (!ok && lane == 0 && tseq > 0) drain(op_full, (tseq - 1) & 1, abort_flag);
+    if (!ok && lane == 0 && oseq > 0) drain(op_full, (oseq - 1) & 1, abort_flag);
   } else if (warp == 2) {
     // ---- MMA issue: one thread, once per tile
     if (lane == 0) {
-      uint32_t tseq = 0;
+      uint32_t tseq = 0, oseq = 0;
       bool ok = true;
       const uint32_t idesc = tc_idesc_tf32(128);
       const uint64_t adesc0 = tc_desc_sw128(smem_u32(opa)), bdesc0 = tc_desc_sw128(smem_u32(opb));
       for (int ti = t_begin; ti < t_end && ok; ++ti, ++tseq) {
         const uint32_t db = tseq & 1;
         if (!thread_wait(d_empty + db, ((tseq >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
-        if (!thread_wait(op_full, tseq & 1, abort_flag)) { ok = false; break; }
-        tc_fence_after();
+        for (int h = 0; h < S::kHalves && ok; ++h, ++oseq) {
+          if (!thread_wait(op_full, oseq & 1, abort_flag)) { ok = false; break; }
+          tc_fence_after();
 #pragma unroll
-        for (int kt = 0; kt < S::kSub; ++kt)
+          for (int kt = 0; kt < S::kSub; ++kt)
 #pragma unroll
-          for (int ks = 0; ks < 4; ++ks) {
-            const uint64_t off = (uint64_t)((kt * kT1PieceBytes + ks * 32) >> 4);
-            tc_mma_tf32_ss(tmem + db * 128, adesc0 + off, bdesc0 + off, idesc, (kt > 0 || ks > 0) ? 1u : 0u);
-          }
-        tc_commit(op_empty);
-        tc_commit(d_full + db);
+            for (int ks = 0; ks < 4; ++ks) {
+              const uint64_t off = (uint64_t)((kt * kT1PieceBytes + ks * 32) >> 4);
+              tc_mma_tf32_ss(tmem + db * 128, adesc0 + off, bdesc0 + off, idesc, (h > 0 || kt > 0 || ks > 0) ? 1u : 0u);
+            }
+          tc_commit(op_empty);            // the slice's buffer may be refilled once these MMAs have read it
+        }
+        if (ok) tc_commit(d_full + db);
       }
       tc_commit(fin);
       drain(fin, 0, abort_flag);
@@ -972,6 +982,7 @@ cudaError_t launch_tc_pass3(int RP, const Tables& t, const Tile* tiles, int ntil
   };
   if (RP == 16) return go(tc_pass3_kernel<16>, Pass3Cfg<16>::kTotal);
   if (RP == 32) return go(tc_pass3_kernel<32>, Pass3Cfg<32>::kTotal);
+  if (RP == 64) return go(tc_pass3_kernel<64>, Pass3Cfg<64>::kTotal);
   return cudaErrorInvalidValue;
 }
 
@@ -985,6 +996,7 @@ cudaError_t launch_tc_pass1(int RP, const Tables& t, const Tile* tiles, int ntil
   };
   if (RP == 16) return go(tc_pass1_kernel<16>, Pass1Cfg<16>::kTotal);
   if (RP == 32) return go(tc_pass1_kernel<32>, Pass1Cfg<32>::kTotal);
+  if (RP == 64) return go(tc_pass1_kernel<64>, Pass1Cfg<64>::kTotal);
   return cudaErrorInvalidValue;
 }
 
@@ -997,6 +1009,7 @@ cudaError_t launch_tc_pass2(int RP, const Tables& t, const Tile* tiles, int ntil
   };
   if (RP == 16) return go(tc_pass2_kernel<16>, Pass2Cfg<16>::kTotal);
   if (RP == 32) return go(tc_pass2_kernel<32>, Pass2Cfg<32>::kTotal);
+  if (RP == 64) return go(tc_pass2_kernel<64>, Pass2Cfg<64>::kTotal);
   return cudaErrorInvalidValue;
 }
 

@@ -45,7 +45,7 @@ def test_workspace_bytes_covers_the_persistent_state(lib):
 
 
 @pytest.mark.parametrize("kw,code", [
-    (dict(rank=0), B.ERR_INVALID_ARG), (dict(rank=33), B.ERR_INVALID_ARG),
+    (dict(rank=0), B.ERR_INVALID_ARG), (dict(rank=65), B.ERR_INVALID_ARG),
     (dict(bits_p=1), B.ERR_INVALID_ARG), (dict(bits_q=9), B.ERR_INVALID_ARG),
     (dict(alpha=0.0), B.ERR_INVALID_ARG), (dict(alpha=float("nan")), B.ERR_INVALID_ARG),
     (dict(workers=0), B.ERR_INVALID_ARG), (dict(workers=257), B.ERR_INVALID_ARG),

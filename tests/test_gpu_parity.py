@@ -182,9 +182,9 @@ def test_value_domain_average_variant(W, bits):
     assert not torch.equal(b.get_state(B.STATE_P_BAR, 0), c.get_state(B.STATE_P_BAR, 0))
 
 
-@pytest.mark.parametrize("rank,W", [(30, 3), (32, 2), (20, 1)])
+@pytest.mark.parametrize("rank,W", [(30, 3), (32, 2), (20, 1), (50, 2), (64, 1), (40, 3)])
 def test_ranks_above_sixteen(rank, W):
-    """Ranks 17..32 (the paper's figures go to 30 and beyond): padded rank 32, products of the
+    """Ranks 17..64 (the paper's figures use ranks 30 and 50): padded rank 32 or 64, products of the
     aligned layers on the tensor cores, the 64 x 27 and 33 x 17 layers on the scalar register
     kernels; stage by stage and free-running against the oracle."""
     w = wl.Workload("r32", ((128, 576), (512, 1152), (64, 27), (100, 512), (33, 17), (40, 129), (130, 36), (24, 1)),
@@ -192,8 +192,9 @@ def test_ranks_above_sixteen(rank, W):
     run_steps(w, 2)
 
 
-def test_rank_thirty_on_the_resnet_set():
-    w = dataclasses.replace(wl.config5(30, 8), workers=2)
+@pytest.mark.parametrize("rank", [30, 50])
+def test_ranks_of_the_papers_figures_on_the_resnet_set(rank):
+    w = dataclasses.replace(wl.config5(rank, 8), workers=2)
     run_steps(w, 1, free_run=False)
 
 
@@ -220,7 +221,7 @@ def test_quantised_vectors_variant(bits, W, average):
 
 
 @pytest.mark.parametrize("rank,bits,W,average", [(3, 4, 3, "codes"), (8, 3, 2, "values"), (1, 2, 1, "codes"),
-                                                  (16, 6, 2, "codes"), (30, 8, 9, "codes")])
+                                                  (16, 6, 2, "codes"), (30, 8, 9, "codes"), (50, 5, 2, "codes")])
 def test_column_scales_variant(rank, bits, W, average):
     """LQSGD_FLAG_COLUMN_SCALES: one scale per factor column.  Scales, codes, averages, payload (2 r_eff
     scales per matrix) and the free-running trajectory against the oracle in the same mode; the columns'
