@@ -576,19 +576,37 @@ def run_exchange(args):
     dist.barrier()
     peak, peak_kind = load_peaks()
     wl_obj, desc = get_workload(args.workload)
-    comp = B.LQSGD(wl_obj.layers, wl_obj.rank, wl_obj.bits, alpha=wl_obj.alpha, workers=wl_obj.workers,
-                   seed=wl_obj.seed, device=dev, world_workers=wl_obj.workers * world)
+    def make(layers):
+        return B.LQSGD(layers, wl_obj.rank, wl_obj.bits, alpha=wl_obj.alpha, workers=wl_obj.workers,
+                       seed=wl_obj.seed, device=dev, world_workers=wl_obj.workers * world)
+    comp = make(wl_obj.layers)
     seeded = dataclasses.replace(wl_obj, seed=wl_obj.seed + 1000 * rank)
     sets = [wl.draw_gradients(seeded, t, device=dev) for t in range(3)]
     ghat = [torch.empty_like(g) for g in sets[0][0]]
+    one_round = lambda t: D.distributed_round(comp, sets[t % 3], ghat)
+    if args.overlap:
+        # the layer table cut in two, one context per half on its own stream: one half's collectives run under the
+        # other half's streaming passes
+        idx = D.split_layers(wl_obj.layers)
+        halves = [make([wl_obj.layers[i] for i in part]) for part in idx]
+        streams = [torch.cuda.Stream(device=dev) for _ in range(2)]
+        main = torch.cuda.current_stream()
+
+        def one_round(t):
+            for s in streams:
+                s.wait_stream(main)
+            D.distributed_round_overlapped([(halves[h], [[per[i] for i in idx[h]] for per in sets[t % 3]], [ghat[i] for i in idx[h]])
+                                            for h in range(2)], streams=streams)
+            for s in streams:
+                main.wait_stream(s)
     for t in range(args.warmup):
-        D.distributed_round(comp, sets[t % 3], ghat)
+        one_round(t)
     dist.barrier()
     torch.cuda.synchronize()
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     start.record()
     for t in range(args.steps):
-        D.distributed_round(comp, sets[(args.warmup + t) % 3], ghat)
+        one_round(args.warmup + t)
     stop.record()
     dist.barrier()
     torch.cuda.synchronize()
@@ -604,8 +622,9 @@ def run_exchange(args):
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": desc, "l2": "inputs larger than L2; 3 gradient sets rotate",
                        "parallelism": f"{wl_obj.workers} workers per GPU x {world} GPUs in one average: 2 MAX "
-                                      "all-reduces of scales + 2 all-gathers of packed codes per step (NCCL)"},
-            "gpu_launches": args.steps * (comp.launches_per_step + 4),
+                                      "all-reduces of scales + 2 all-gathers of packed codes + 1 SUM all-reduce of the 1-D "
+                                      "tensors per step (NCCL)" + (", layer table in two halves on two streams" if args.overlap else "")},
+            "gpu_launches": args.steps * (comp.launches_per_step + 5),
             "roofline": {"bound": "hbm", "kernel": "whole round per GPU", "achieved": rb / (ms * 1e-3) / 1e9, "peak": peak,
                          "unit": "GB/s", "frac": rb / (ms * 1e-3) / 1e9 / peak, "peak_kind": f"of {peak_kind}", "traffic": None},
             "exchange_bytes_per_rank_per_step": int(comp.exchange_view(B.XCHG_STREAMS_P).numel()
@@ -633,6 +652,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle")
     ap.add_argument("--min-ms", type=float, default=500.0,
                     help="repeat the block of --steps steps until this much device time has been timed (0: one block)")
+    ap.add_argument("--overlap", action="store_true",
+                    help="with --exchange: the layer table cut in two halves on two streams, collectives under compute")
     ap.add_argument("--exchange", action="store_true",
                     help="workers of all GPUs in one average, with the real NCCL exchange (default: independent replicas)")
     args = ap.parse_args()

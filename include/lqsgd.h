@@ -92,8 +92,7 @@ typedef enum lqsgd_error {
                                         rescaled by s_j after Eq. 5.  A matrix then sends 2 r_eff scales: in the payload
                                         s_P[0..r_eff) is followed by s_Q[0..r_eff) (8 r_eff bytes at scale_offset), and
                                         LQSGD_STATE_SCALES is fp32 [2][r_eff].  The zero-scale status bits are set when
-                                        any column's scale is 0 (that column's codes and averages are 0).  Not available
-                                        with workers on several GPUs (lqsgd_round_begin refuses). */
+                                        any column's scale is 0 (that column's codes and averages are 0). */
 
 #define LQSGD_FLAG_ONE_LAUNCH 32u /* run the round as ONE cooperative kernel that keeps M = G + E in the SMs' shared memory
                                      from the first product to the error update (12 + 4/W instead of 24 + 4/W bytes of
@@ -218,28 +217,34 @@ int lqsgd_step_update(lqsgd_ctx* ctx, const float* const* host_grads, float* con
  * other processes hold more workers (config.world_workers = total over all ranks, each rank
  * simulating `workers` of them), a rank runs the round as
  *
- *   lqsgd_round_begin(grads, ghat, weights, lr)   pass 1, Orthonormalize, local scales of P
- *   all-reduce MAX over ranks of  view(LQSGD_XCHG_SCALES_P)     (one fp32 per matrix)
+ *   lqsgd_round_begin(grads, ghat, weights, lr)   pass 1, Orthonormalize, local scales of P, and this rank's
+ *                                                  share of every 1-D tensor's mean into one flat buffer
+ *   all-reduce MAX over ranks of  view(LQSGD_XCHG_SCALES_P)     (one fp32 per matrix; r_eff per matrix padded to the
+ *                                                                padded rank with LQSGD_FLAG_COLUMN_SCALES)
  *   lqsgd_round_pack(0)                            quantise + pack this rank's P with those scales
  *   all-gather of                 view(LQSGD_XCHG_STREAMS_P)    (workers x P-stream bytes, contiguous)
  *   lqsgd_round_reduce(0, gathered, n_ranks)       exact integer sum over ALL workers' codes,
  *                                                  Eq. 5, pass 2, local scales of Q
  *   all-reduce MAX of view(LQSGD_XCHG_SCALES_Q);  lqsgd_round_pack(1);  all-gather of
  *   view(LQSGD_XCHG_STREAMS_Q);  lqsgd_round_reduce(1, gathered, n_ranks)
- *   lqsgd_round_end()                              pass 3 (G_hat, E, optional model update)
+ *   all-reduce SUM of view(LQSGD_XCHG_VECTORS)     (the 1-D tensors, fp32, all in one buffer; any time after begin)
+ *   lqsgd_round_end()                              pass 3 (G_hat, E, optional model update); the 1-D tensors'
+ *                                                  means go to their G_hat tensors and into the weights
  *
  * The collectives run on the same stream between the calls (NCCL, or any other transport: the
  * library only reads and writes the buffers).  `gathered` is n_ranks x the bytes of the STREAMS
  * view, rank after rank, in caller memory.  The wire carries exactly the b-bit streams
- * (r(n+m)b bits per worker, Section IV-C) plus one scale per factor and layer.  Results are
- * identical, bit for bit, to one process simulating all world_workers workers.  G_hat of a
- * 1-D tensor comes out as this rank's share of the mean (local sum / world_workers): sum it
- * over the ranks.  Calls out of order return LQSGD_ERR_INVALID_ARG; the bits = 32 bypass is not
- * available across ranks.  ghat / weights as in lqsgd_step_update (weights may be NULL). */
+ * (r(n+m)b bits per worker, Section IV-C) plus one scale per factor and layer - five collectives per round,
+ * whatever the number of layers.  With bits = 32 the streams are the fp32 factors and the scales are not used
+ * (the PowerSGD exchange of Section III-B).  Results are identical, bit for bit, to one process simulating all
+ * world_workers workers (the 1-D means up to the order of their sum).  Calls out of order return
+ * LQSGD_ERR_INVALID_ARG; quantised 1-D tensors and several power iterations are not available across ranks.
+ * ghat / weights as in lqsgd_step_update (weights may be NULL). */
 #define LQSGD_XCHG_SCALES_P 0
 #define LQSGD_XCHG_SCALES_Q 1
 #define LQSGD_XCHG_STREAMS_P 2
 #define LQSGD_XCHG_STREAMS_Q 3
+#define LQSGD_XCHG_VECTORS 4
 int lqsgd_round_begin(lqsgd_ctx* ctx, const float* const* host_grads, float* const* host_ghat,
                       float* const* host_weights, float lr, void* cuda_stream);
 int lqsgd_round_pack(lqsgd_ctx* ctx, int32_t which, void* cuda_stream);

@@ -27,7 +27,7 @@ FLAG_COLUMN_SCALES = 16
 FLAG_ONE_LAUNCH = 32
 STATUS_TIMEOUT = 16
 N_PHASES = 5
-XCHG_SCALES_P, XCHG_SCALES_Q, XCHG_STREAMS_P, XCHG_STREAMS_Q = range(4)
+XCHG_SCALES_P, XCHG_SCALES_Q, XCHG_STREAMS_P, XCHG_STREAMS_Q, XCHG_VECTORS = range(5)
 PHASE_NAMES = ("pass1", "finish_p", "pass2", "finish_q", "pass3")
 
 ERR_INVALID_ARG, ERR_BAD_SHAPE, ERR_WORKSPACE_TOO_SMALL, ERR_MISALIGNED = -1, -2, -3, -4
@@ -310,7 +310,7 @@ class LQSGD:
         _check(self.lib.lqsgd_exchange_view(self.ctx, which, C.byref(ptr), C.byref(nb)))
         off = ptr.value - self.workspace.data_ptr()
         raw = self.workspace[off:off + nb.value]
-        return raw.view(torch.float32) if which in (XCHG_SCALES_P, XCHG_SCALES_Q) else raw
+        return raw.view(torch.float32) if which in (XCHG_SCALES_P, XCHG_SCALES_Q, XCHG_VECTORS) else raw
 
     def step_host(self, grads, ghat, payload: Optional[torch.Tensor] = None,
                   stream: Optional[torch.cuda.Stream] = None) -> None:

@@ -108,7 +108,11 @@ struct Plan {
   void** d_ptrs = nullptr;                    // kPtrSets pointer tables, see prepare_step for the layout of one
   uint32_t* d_status = nullptr;
   uint8_t* d_payload = nullptr;
-  float* d_xscales = nullptr;                 // [2][n_mat] scales the ranks agree on (split exchange)
+  float* d_xscales = nullptr;                 // [2][n_mat][ns] scales the ranks agree on (split exchange); ns = 1, or RP per column
+  int xscale_ns = 1;
+  float* d_xvec = nullptr;                    // the 1-D tensors' means, all in one buffer (split round: one all-reduce)
+  size_t vec_elems = 0;
+  uint64_t vec_pay_base = 0;                  // payload offset of the first 1-D tensor's values
   uint8_t* d_xsend[2] = {nullptr, nullptr};   // [W][region_bytes]: local P / Q streams, contiguous, for the all-gather
   uint64_t region_off[2] = {0, 0}, region_bytes[2] = {0, 0};
   size_t zero_elems = 0;
@@ -132,9 +136,8 @@ int check_config(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
   if (c->workers < 1 || c->workers > 256) return LQSGD_ERR_INVALID_ARG;
   if (c->power_iters < 0 || c->power_iters > 8) return LQSGD_ERR_INVALID_ARG;
   if (c->power_iters > 1 && c->world_workers > c->workers) return LQSGD_ERR_INVALID_ARG;
-  if (c->world_workers != 0) {     // workers of all ranks: a multiple of the local ones; no bypass mode across ranks
+  if (c->world_workers != 0) {     // workers of all ranks: a multiple of the local ones
     if (c->world_workers < c->workers || c->world_workers > 4096 || c->world_workers % c->workers) return LQSGD_ERR_INVALID_ARG;
-    if (c->world_workers > c->workers && (c->bits_p == 32 || c->bits_q == 32)) return LQSGD_ERR_INVALID_ARG;
   }
   if (c->flags & ~(LQSGD_FLAG_HOST_STAGING | LQSGD_FLAG_REGISTER_PATH | LQSGD_FLAG_AVERAGE_VALUES |
                    LQSGD_FLAG_QUANTIZE_VECTORS | LQSGD_FLAG_COLUMN_SCALES | LQSGD_FLAG_ONE_LAUNCH))
@@ -637,7 +640,12 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   deal(p.tctiles3, p.tcbegin3);     // same cost model: pieces of 32 columns (times W for every tile alike)
   p.d_status = a.take<uint32_t>(p.mats.size());
   p.d_payload = a.take<uint8_t>((size_t)W * p.payload_stride);
-  p.d_xscales = a.take<float>(2 * p.mats.size());
+  p.xscale_ns = colscales ? RP : 1;
+  p.d_xscales = a.take<float>(2 * p.mats.size() * p.xscale_ns);
+  p.vec_elems = 0;
+  for (auto& v : p.vecs) p.vec_elems += (size_t)v.len;
+  p.vec_pay_base = p.vecs.empty() ? 0 : p.vecs.front().pay_off;
+  p.d_xvec = a.take<float>(p.vec_elems);
   p.d_xsend[0] = a.take<uint8_t>((size_t)W * p.region_bytes[0]);
   p.d_xsend[1] = a.take<uint8_t>((size_t)W * p.region_bytes[1]);
   p.d_rsync = a.take<uint32_t>(1 + 2 * kResBarriers);
@@ -1043,6 +1051,7 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
   sx.pack_only = split ? 1 : 0;
   sx.n_mat = (int)nm;
   sx.scales = p.d_xscales;
+  sx.ns = p.xscale_ns;
   sx.send[0] = p.d_xsend[0]; sx.send[1] = p.d_xsend[1];
   sx.region_bytes[0] = p.region_bytes[0]; sx.region_bytes[1] = p.region_bytes[1];
   sx.region_off[0] = p.region_off[0]; sx.region_off[1] = p.region_off[1];
@@ -1052,6 +1061,8 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
   vj.vghat = reinterpret_cast<float* const*>(c->ptrs_cur + vbase + nv * W);
   vj.vweights = c->has_weights ? reinterpret_cast<float* const*>(c->ptrs_cur + vbase + nv * (W + 1)) : nullptr;
   vj.lr = t.lr;
+  vj.xvec = split ? p.d_xvec : nullptr;
+  vj.xvec_base = p.vec_pay_base;
   const bool ride = vectors_ride(c);     // the 1-D tensors travel as extra blocks of the exchange of P
   const bool ev = c->have_events && !split;
 #define PHASE_MARK(i) do { if (ev) CK(cudaEventRecord(c->phase_events[i], st)); } while (0)
@@ -1086,7 +1097,7 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
         CK(launch_p_orth_small(RP, t, p.d_fbS, (int)p.fbS.size(), {st, 0}));
         CK(launch_p_reduce_gram(RP, t, p.d_fbP, (int)p.fbP.size(), {st, 0}));
         CK(launch_p_apply(RP, t, p.d_fbP, (int)p.fbP.size(), {st, 0}));
-        if (split) CK(launch_scale_reduce(t, 0, p.d_xscales, (int)nm, {st, 0}));
+        if (split) CK(launch_scale_reduce(RP, t, 0, p.d_xscales, (int)nm, {st, 0}));
       }
       break;
     case 1:
@@ -1103,7 +1114,7 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
       PHASE_MARK(3);
       if (nm) {
         CK(launch_q_reduce(RP, t, p.d_fbQ, (int)p.fbQ.size(), {st, 0}));
-        if (split) CK(launch_scale_reduce(t, 1, p.d_xscales, (int)nm, {st, 0}));
+        if (split) CK(launch_scale_reduce(RP, t, 1, p.d_xscales, (int)nm, {st, 0}));
       }
       break;
     case 3:
@@ -1119,6 +1130,7 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
         CK(launch_stream_pass3(RP, t, p.d_stiles3, (int)p.stiles3.size(), {st, (int)std::min<size_t>(p.stiles3.size(), c->sm_count)}));
         CK(launch_tc_pass3(RP, t, p.d_tctiles3, (int)p.tctiles3.size(), p.d_tcbegin3, p.d_tcmaps, {st, p.tc_grid}));
       }
+      if (split && nv) CK(launch_vectors_finish(vj, {st, 0}));     // the shares were summed over the ranks meanwhile
       PHASE_MARK(5);
       break;
     default: return LQSGD_ERR_INVALID_ARG;
@@ -1196,8 +1208,8 @@ int lqsgd_round_begin(lqsgd_ctx* c, const float* const* grads, float* const* gha
                       void* cuda_stream) {
   const int rc = prepare_step(c, grads, ghat, weights, lr, cuda_stream);
   if (rc != LQSGD_OK) return rc;
-  if (c->cfg.bits_p == 32 || c->cfg.bits_q == 32 || c->cfg.power_iters > 1) return LQSGD_ERR_INVALID_ARG;
-  if (c->cfg.flags & LQSGD_FLAG_COLUMN_SCALES) return LQSGD_ERR_INVALID_ARG;   // the ranks agree on one scale per factor
+  if (c->cfg.power_iters > 1) return LQSGD_ERR_INVALID_ARG;
+  if ((c->cfg.flags & LQSGD_FLAG_QUANTIZE_VECTORS) && c->cfg.bits_p != 32 && !c->plan.vecs.empty()) return LQSGD_ERR_INVALID_ARG;
   c->round_stage = 0;
   const int rs = run_segment(c, 0, true, nullptr, 0, static_cast<cudaStream_t>(cuda_stream));
   if (rs == LQSGD_OK) c->round_stage = 1;
@@ -1232,8 +1244,9 @@ int lqsgd_exchange_view(const lqsgd_ctx* c, int32_t which, void** dev_ptr, size_
   if (!c || !dev_ptr || !bytes) return LQSGD_ERR_INVALID_ARG;
   const Plan& p = c->plan;
   switch (which) {
-    case LQSGD_XCHG_SCALES_P: *dev_ptr = p.d_xscales; *bytes = 4 * p.mats.size(); break;
-    case LQSGD_XCHG_SCALES_Q: *dev_ptr = p.d_xscales + p.mats.size(); *bytes = 4 * p.mats.size(); break;
+    case LQSGD_XCHG_SCALES_P: *dev_ptr = p.d_xscales; *bytes = 4 * p.mats.size() * p.xscale_ns; break;
+    case LQSGD_XCHG_SCALES_Q: *dev_ptr = p.d_xscales + p.mats.size() * p.xscale_ns; *bytes = 4 * p.mats.size() * p.xscale_ns; break;
+    case LQSGD_XCHG_VECTORS: *dev_ptr = p.d_xvec; *bytes = 4 * p.vec_elems; break;
     case LQSGD_XCHG_STREAMS_P: *dev_ptr = p.d_xsend[0]; *bytes = (size_t)p.W * p.region_bytes[0]; break;
     case LQSGD_XCHG_STREAMS_Q: *dev_ptr = p.d_xsend[1]; *bytes = (size_t)p.W * p.region_bytes[1]; break;
     default: return LQSGD_ERR_OUT_OF_RANGE;

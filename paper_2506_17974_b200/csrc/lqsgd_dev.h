@@ -182,7 +182,8 @@ cudaError_t launch_p_orth_small(int RP, const Tables& t, const FactorBlock* fb, 
 struct SplitExchange {
   int32_t pack_only;
   int32_t n_mat;
-  const float* scales;
+  int32_t ns;                 // scales per factor and layer: 1, or RP with one scale per column
+  const float* scales;        // [2][n_mat][ns]
   uint8_t* send[2];
   uint64_t region_bytes[2];   // bytes of all layers' P (or Q) streams of one worker
   uint64_t region_off[2];     // offset of that region inside a payload
@@ -197,12 +198,15 @@ struct VectorJob {
   float* const* vghat;           // [n_vec], entries may be null
   float* const* vweights;        // [n_vec] or null
   float lr;
+  float* xvec;                   // workers on several GPUs: this rank's shares of the means go here (all tensors, in
+                                 // payload order, contiguous) for ONE all-reduce, instead of into vghat / vweights
+  uint64_t xvec_base;            // payload offset of the first 1-D tensor's values
 };
 // ride: the 1-D tensors' blocks appended to this launch (or null)
 cudaError_t launch_exchange(int RP, int which /*0 = P, 1 = Q*/, const Tables& t, const QuantTables& q,
                             const ExchangeChunk* ch, int nch, const SplitExchange& sx, const VectorJob* ride, Launch l);
 cudaError_t launch_unpack_codes(const uint8_t* stream, int count, int bits, uint8_t* out, cudaStream_t st);
-cudaError_t launch_scale_reduce(const Tables& t, int which, float* scales, int n_mat, Launch l);
+cudaError_t launch_scale_reduce(int RP, const Tables& t, int which, float* scales, int n_mat, Launch l);
 cudaError_t launch_sum_dequant(int RP, int which, const Tables& t, const QuantTables& q, const ExchangeChunk* ch,
                                int nch, const SplitExchange& sx, const uint8_t* gathered, int n_streams, Launch l);
 cudaError_t launch_q_transpose(const float* Q, float* Qt, float* Qcat, int m, int RP, int mt, int kcat, int tc,
@@ -215,6 +219,8 @@ cudaError_t launch_vectors_quant(const VectorDev* vecs, int nvecs, const float* 
                                  float* const* vweights, float lr, uint8_t* payload, uint64_t payload_stride, int W,
                                  const QuantTables& q, Launch l);
 cudaError_t launch_vectors(const VectorJob& vj, uint8_t* payload, uint64_t payload_stride, int W, Launch l);
+// after the all-reduce of xvec: the means go to vghat, and into the weights (model update)
+cudaError_t launch_vectors_finish(const VectorJob& vj, Launch l);
 // Bulk-copy staged passes (lqsgd_stream.cu): layers with m % 4 == 0 and RP <= 8.  One CTA per SM,
 // 512 consumer threads.  The copy engine limits the number of bulk copies in flight, not their
 // bytes, so tiles are wide (few, large row segments per stage) and a tile that spans whole rows

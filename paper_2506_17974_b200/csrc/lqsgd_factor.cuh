@@ -527,6 +527,7 @@ __device__ __forceinline__ void vectors_block(const VectorJob& vj, int job, int 
     s += x;
   }
   const float mean = s / (float)vj.W_total;     // with workers on other GPUs too: this rank's share of the mean
+  if (vj.xvec) { vj.xvec[(v.pay_off - vj.xvec_base) / 4 + i] = mean; return; }   // summed over the ranks before it is used
   if (vj.vghat[ch.layer]) vj.vghat[ch.layer][i] = mean;
   if (vj.vweights && vj.vweights[ch.layer]) vj.vweights[ch.layer][i] = fmaf(-vj.lr, mean, vj.vweights[ch.layer][i]);
 }
@@ -604,6 +605,10 @@ __device__ __forceinline__ void exchange_body(const Tables& t, const QuantTables
     for (int i = tid; i < W * nblk * RP; i += NT) s = fmaxf(s, ld_in<COH>(maxes + i));
     atomicMax(reinterpret_cast<int*>(S.scol) + tid % RP, __float_as_int(s));
     __syncthreads();
+    if (sx.pack_only) {                                   // scales agreed between the ranks
+      if (tid < RP) S.scol[tid] = sx.scales[(size_t)(which * sx.n_mat + ch.layer) * sx.ns + tid];
+      __syncthreads();
+    }
   } else {
     for (int i = tid; i < W * nblk; i += NT) s = fmaxf(s, ld_in<COH>(maxes + i));
 #pragma unroll
@@ -613,7 +618,7 @@ __device__ __forceinline__ void exchange_body(const Tables& t, const QuantTables
     s = S.sred[0];
 #pragma unroll
     for (int i = 1; i < NT / 32; ++i) s = fmaxf(s, S.sred[i]);
-    if (sx.pack_only) s = sx.scales[which * sx.n_mat + ch.layer];   // scale agreed between the ranks
+    if (sx.pack_only) s = sx.scales[(size_t)(which * sx.n_mat + ch.layer) * sx.ns];   // scale agreed between the ranks
   }
   // scales, status: once per layer
   if (ch.chunk == 0 && (cs ? tid < r : tid == 0)) {
@@ -640,8 +645,12 @@ __device__ __forceinline__ void exchange_body(const Tables& t, const QuantTables
         uint8_t* pay = t.payload + (size_t)w * t.payload_stride + pay_off + (size_t)e * 4;
         const unsigned bits32 = __float_as_uint(x);               // the stream may start on any byte
         pay[0] = bits32 & 0xff; pay[1] = (bits32 >> 8) & 0xff; pay[2] = (bits32 >> 16) & 0xff; pay[3] = bits32 >> 24;
+        if (sx.pack_only) {                                       // the same bytes, contiguous, for the all-gather
+          uint8_t* snd = sx.send[which] + (size_t)w * sx.region_bytes[which] + (pay_off - sx.region_off[which]) + (size_t)e * 4;
+          snd[0] = pay[0]; snd[1] = pay[1]; snd[2] = pay[2]; snd[3] = pay[3];
+        }
       }
-      store_factor<RP>(L, which, row, col, sum / (float)W);
+      if (!sx.pack_only) store_factor<RP>(L, which, row, col, sum / (float)W);
     }
     return;
   } else {

@@ -565,15 +565,26 @@ q_transpose_kernel(const float* __restrict__ Q, float* __restrict__ Qt, float* _
 // scale (exchange_kernel in pack-only mode), the packed streams are all-gathered, and
 // sum_dequant_kernel adds the signed levels of ALL workers (exact integers) and applies Eq. 5.
 // ---------------------------------------------------------------------------------------
+template <int RP>
 __global__ void __launch_bounds__(256)
 scale_reduce_kernel(Tables t, int which, float* scales, int n_mat) {
   pdl_wait();
   __shared__ float sred[8];
+  __shared__ float scol[RP];
   const int layer = blockIdx.x, tid = threadIdx.x;
   const LayerDev& L = t.layers[layer];
   const int nblk = which ? L.nqb : L.npb;
   const float* __restrict__ maxes = which ? L.maxq : L.maxp;
   float s = 0.f;
+  if (t.col_scales) {              // one scale per column: maxes are [W][nblk][RP]; 256 is a multiple of RP
+    if (tid < RP) scol[tid] = 0.f;
+    __syncthreads();
+    for (int i = tid; i < t.W * nblk * RP; i += 256) s = fmaxf(s, maxes[i]);
+    atomicMax(reinterpret_cast<int*>(scol) + tid % RP, __float_as_int(s));     // non-negative floats order like their bits
+    __syncthreads();
+    if (tid < RP) scales[(size_t)(which * n_mat + layer) * RP + tid] = scol[tid];
+    return;
+  }
   for (int i = tid; i < t.W * nblk; i += 256) s = fmaxf(s, maxes[i]);
 #pragma unroll
   for (int o = 16; o >= 1; o >>= 1) s = fmaxf(s, __shfl_xor_sync(0xffffffffu, s, o));
@@ -585,6 +596,8 @@ scale_reduce_kernel(Tables t, int which, float* scales, int n_mat) {
   }
 }
 
+// The sum over ALL workers' streams (n_streams of them, rank after rank) and Eq. 5, for one chunk of 256 factor
+// elements.  bits = 32: the streams are the fp32 factors themselves, averaged in stream order (Eq. 1).
 template <int RP>
 __global__ void __launch_bounds__(256)
 sum_dequant_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __restrict__ chunks, SplitExchange sx,
@@ -593,43 +606,68 @@ sum_dequant_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __r
   const ExchangeChunk ch = chunks[blockIdx.x];
   const LayerDev& L = t.layers[ch.layer];
   const int tid = threadIdx.x, b = qt.bits;
-  const int nlev = 1 << (b - 1);
+  const int nlev = b == 32 ? 2 : 1 << (b - 1);
   const int rows = which ? L.m : L.n, r = L.r;
   const int count = rows * r;
   const int e = ch.chunk * kExchangeChunk + tid;
-  const float s = sx.scales[which * sx.n_mat + ch.layer];
-  const bool s_ok = (s > 0.f) && (s < INFINITY);
+  const float* sc = sx.scales + (size_t)(which * sx.n_mat + ch.layer) * sx.ns;
   if (e < count) {
-    const uint64_t off = (which ? L.pay_q_off : L.pay_p_off) - sx.region_off[which];   // this layer's stream
-    const size_t nbytes = ((size_t)count * b + 7) / 8;
-    const size_t bit = (size_t)e * b, byte = bit >> 3;
-    const int sh = (int)(bit & 7);
-    int S = 0;
-    float Sv = 0.f;
-    for (int w = 0; w < n_streams; ++w) {
-      const uint8_t* st = gathered + (size_t)w * sx.region_bytes[which] + off;
-      unsigned v = st[byte];
-      if (sh + b > 8 && byte + 1 < nbytes) v |= (unsigned)st[byte + 1] << 8;
-      const unsigned code = (v >> sh) & ((1u << b) - 1u);
-      const int k = (int)(code & (unsigned)(nlev - 1));
-      const int sk = (code >> (b - 1)) ? -k : k;
-      S += sk;
-      if (qt.avg_values) Sv += __ldg(qt.deq + sk + (nlev - 1));
-    }
-    float v = 0.f;
-    if (s_ok) v = qt.avg_values ? s * (Sv / (float)n_streams) : s * __ldg(qt.deq + S + n_streams * (nlev - 1));
     const int row = e / r, col = e - row * r;
+    const uint64_t off = (which ? L.pay_q_off : L.pay_p_off) - sx.region_off[which];   // this layer's stream
+    float v = 0.f;
+    if (b == 32) {
+      float sum = 0.f;
+      for (int w = 0; w < n_streams; ++w) {
+        const uint8_t* st = gathered + (size_t)w * sx.region_bytes[which] + off + (size_t)e * 4;
+        sum += __uint_as_float((unsigned)st[0] | ((unsigned)st[1] << 8) | ((unsigned)st[2] << 16) | ((unsigned)st[3] << 24));
+      }
+      v = sum / (float)n_streams;
+    } else {
+      const float s = sc[sx.ns > 1 ? col : 0];
+      const bool s_ok = (s > 0.f) && (s < INFINITY);
+      const size_t nbytes = ((size_t)count * b + 7) / 8;
+      const size_t bit = (size_t)e * b, byte = bit >> 3;
+      const int sh = (int)(bit & 7);
+      int S = 0;
+      float Sv = 0.f;
+      for (int w = 0; w < n_streams; ++w) {
+        const uint8_t* st = gathered + (size_t)w * sx.region_bytes[which] + off;
+        unsigned u = st[byte];
+        if (sh + b > 8 && byte + 1 < nbytes) u |= (unsigned)st[byte + 1] << 8;
+        const unsigned code = (u >> sh) & ((1u << b) - 1u);
+        const int k = (int)(code & (unsigned)(nlev - 1));
+        const int sk = (code >> (b - 1)) ? -k : k;
+        S += sk;
+        if (qt.avg_values) Sv += __ldg(qt.deq + sk + (nlev - 1));
+      }
+      if (s_ok) v = qt.avg_values ? s * (Sv / (float)n_streams) : s * __ldg(qt.deq + S + n_streams * (nlev - 1));
+    }
     store_factor<RP>(L, which, row, col, v);
   }
-  if (ch.chunk == 0 && tid == 0) {
-    L.scales[which] = s;
+  if (ch.chunk == 0 && tid < (sx.ns > 1 ? r : 1)) {
+    const float s = sc[tid];
+    L.scales[sx.ns > 1 ? which * RP + tid : which] = s;
     for (int w = 0; w < t.W; ++w) {
       float* ps = reinterpret_cast<float*>(t.payload + (size_t)w * t.payload_stride + L.pay_scale_off);
-      ps[which] = s;
+      ps[sx.ns > 1 ? which * r + tid : which] = s;
     }
-    if (!(s > 0.f)) atomicOr(&t.status[ch.layer], which ? 4u : 2u);
+    if (b != 32 && !(s > 0.f)) atomicOr(&t.status[ch.layer], which ? 4u : 2u);
     if (!(s < INFINITY)) atomicOr(&t.status[ch.layer], 8u);
   }
+}
+
+// Workers on several GPUs: after the ranks' shares of the 1-D tensors' means have been summed (one all-reduce
+// of the flat buffer), the means go to their tensors and into the weights.  One block = 256 entries of one tensor.
+__global__ void __launch_bounds__(256)
+vectors_finish_kernel(VectorJob vj) {
+  pdl_wait();
+  const ExchangeChunk ch = vj.chunks[blockIdx.x];
+  const VectorDev v = vj.vecs[ch.layer];
+  const int i = ch.chunk * 256 + threadIdx.x;
+  if (i >= v.len) return;
+  const float mean = vj.xvec[(v.pay_off - vj.xvec_base) / 4 + i];
+  if (vj.vghat[ch.layer]) vj.vghat[ch.layer][i] = mean;
+  if (vj.vweights && vj.vweights[ch.layer]) vj.vweights[ch.layer][i] = fmaf(-vj.lr, mean, vj.vweights[ch.layer][i]);
 }
 
 // Variant (LQSGD_FLAG_QUANTIZE_VECTORS): a 1-D tensor goes through the factor exchange, one CTA per
@@ -816,9 +854,9 @@ cudaError_t launch_unpack_codes(const uint8_t* stream, int count, int bits, uint
   return cudaGetLastError();
 }
 
-cudaError_t launch_scale_reduce(const Tables& t, int which, float* scales, int n_mat, Launch l) {
+cudaError_t launch_scale_reduce(int rp, const Tables& t, int which, float* scales, int n_mat, Launch l) {
   if (n_mat == 0) return cudaSuccess;
-  launch_pdl(scale_reduce_kernel, n_mat, 256, 0, l.stream, t, which, scales, n_mat);
+  LQSGD_DISPATCH_RP(rp, (launch_pdl(scale_reduce_kernel<RP>, n_mat, 256, 0, l.stream, t, which, scales, n_mat)));
   return cudaGetLastError();
 }
 
@@ -827,6 +865,12 @@ cudaError_t launch_sum_dequant(int rp, int which, const Tables& t, const QuantTa
   if (nch == 0) return cudaSuccess;
   LQSGD_DISPATCH_RP(rp, (launch_pdl(sum_dequant_kernel<RP>, nch, 256, 0, l.stream, t, q, which, ch, sx, gathered,
                                     n_streams)));
+  return cudaGetLastError();
+}
+
+cudaError_t launch_vectors_finish(const VectorJob& vj, Launch l) {
+  if (vj.nchunks == 0) return cudaSuccess;
+  launch_pdl(vectors_finish_kernel, vj.nchunks, 256, 0, l.stream, vj);
   return cudaGetLastError();
 }
 
