@@ -104,6 +104,11 @@ typedef enum lqsgd_error {
                                      results up to the order of the floating-point sums.  Off by default: the sequence of
                                      kernels is the faster of the two on the sets measured so far. */
 
+#define LQSGD_FLAG_GUARD_WORDS 64u /* debugging aid: every piece the library carves out of the workspace (error buffers,
+                                      factors, partial sums, payloads, tables ...) is followed by 256 bytes of a fixed
+                                      pattern that no kernel may write; lqsgd_check_guards tells whether any changed,
+                                      i.e. whether a kernel wrote past the end of its piece.  Costs a little workspace. */
+
 typedef struct lqsgd_ctx lqsgd_ctx;
 
 typedef struct lqsgd_shape {
@@ -320,6 +325,13 @@ int lqsgd_test_expire_wait(lqsgd_ctx* ctx, int32_t pass, int32_t stage, uint32_t
  * Q_bar and pass 3 begin | end. */
 #define LQSGD_TIMELINE_MAX 12
 int lqsgd_round_timeline(const lqsgd_ctx* ctx, uint64_t* host_ns, int32_t* host_count, void* cuda_stream);
+
+/* Contexts created with LQSGD_FLAG_GUARD_WORDS: checks the guard blocks between the pieces of the workspace after
+ * everything enqueued on cuda_stream so far, and synchronises it.  *host_changed_words receives the number of
+ * 32-bit guard words that no longer hold their pattern (0 = no kernel wrote outside its piece),
+ * *host_first_offset (may be NULL) the byte offset in the workspace of the first of them, or -1.
+ * LQSGD_ERR_INVALID_ARG for a context without guards. */
+int lqsgd_check_guards(const lqsgd_ctx* ctx, int64_t* host_changed_words, int64_t* host_first_offset, void* cuda_stream);
 
 /* Kernel launches one lqsgd_step enqueues (for launch accounting). */
 int lqsgd_launches_per_step(const lqsgd_ctx* ctx, int32_t* host_out);

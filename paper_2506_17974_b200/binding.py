@@ -25,6 +25,7 @@ FLAG_AVERAGE_VALUES = 4
 FLAG_QUANTIZE_VECTORS = 8
 FLAG_COLUMN_SCALES = 16
 FLAG_ONE_LAUNCH = 32
+FLAG_GUARD_WORDS = 64
 STATUS_TIMEOUT = 16
 N_PHASES = 5
 XCHG_SCALES_P, XCHG_SCALES_Q, XCHG_STREAMS_P, XCHG_STREAMS_Q, XCHG_VECTORS = range(5)
@@ -41,7 +42,7 @@ EXPORTED = [
     "lqsgd_payload", "lqsgd_payload_layout", "lqsgd_get_state", "lqsgd_set_state", "lqsgd_status",
     "lqsgd_orthonormalize_noalloc",
     "lqsgd_round_begin", "lqsgd_round_pack", "lqsgd_round_reduce", "lqsgd_round_end", "lqsgd_exchange_view",
-    "lqsgd_launches_per_step", "lqsgd_set_phase_events", "lqsgd_release_graph_tables", "lqsgd_test_expire_wait", "lqsgd_round_timeline", "lqsgd_destroy", "lqsgd_strerror", "lqsgd_last_cuda_error", "lqsgd_version",
+    "lqsgd_launches_per_step", "lqsgd_set_phase_events", "lqsgd_release_graph_tables", "lqsgd_test_expire_wait", "lqsgd_round_timeline", "lqsgd_check_guards", "lqsgd_destroy", "lqsgd_strerror", "lqsgd_last_cuda_error", "lqsgd_version",
 ]
 
 
@@ -101,6 +102,7 @@ def load_library() -> C.CDLL:
     lib.lqsgd_release_graph_tables.argtypes = [vp]
     lib.lqsgd_test_expire_wait.argtypes = [vp, i32, i32, C.c_uint32]
     lib.lqsgd_round_timeline.argtypes = [vp, C.POINTER(C.c_uint64), C.POINTER(i32), vp]
+    lib.lqsgd_check_guards.argtypes = [vp, C.POINTER(C.c_int64), C.POINTER(C.c_int64), vp]
     lib.lqsgd_destroy.argtypes = [vp]
     lib.lqsgd_destroy.restype = None
     lib.lqsgd_strerror.argtypes = [C.c_int]
@@ -160,7 +162,7 @@ class LQSGD:
                  alpha: float = 127.0, workers: int = 1, seed: int = 0, host_staging: bool = False,
                  device: str = "cuda:0", register_path: bool = False, world_workers: int = 0,
                  average: str = "codes", quantize_vectors: bool = False, power_iters: int = 1,
-                 column_scales: bool = False, one_launch: bool = False):
+                 column_scales: bool = False, one_launch: bool = False, guard_words: bool = False):
         self.lib = load_library()
         self.layers = [(int(n), int(m)) for n, m in layers]
         self.rank, self.bits_p = rank, bits_p
@@ -179,7 +181,8 @@ class LQSGD:
                                | (FLAG_AVERAGE_VALUES if average == "values" else 0)
                                | (FLAG_QUANTIZE_VECTORS if quantize_vectors else 0)
                                | (FLAG_COLUMN_SCALES if column_scales else 0)
-                               | (FLAG_ONE_LAUNCH if one_launch else 0), world_workers, power_iters)
+                               | (FLAG_ONE_LAUNCH if one_launch else 0)
+                               | (FLAG_GUARD_WORDS if guard_words else 0), world_workers, power_iters)
         nbytes = workspace_bytes(self.layers, self.cfg)
         with torch.cuda.device(self.device):
             self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
@@ -241,6 +244,12 @@ class LQSGD:
         n = C.c_int32(0)
         _check(self.lib.lqsgd_round_timeline(self.ctx, buf, C.byref(n), self._stream_ptr()))
         return [int(buf[i]) for i in range(n.value)]
+
+    def check_guards(self) -> Tuple[int, int]:
+        """(guard words changed, byte offset of the first or -1) for a context created with guard_words=True."""
+        bad, first = C.c_int64(0), C.c_int64(0)
+        _check(self.lib.lqsgd_check_guards(self.ctx, C.byref(bad), C.byref(first), self._stream_ptr()))
+        return bad.value, first.value
 
     def release_graph_tables(self) -> None:
         """Every graph captured from this context's steps is gone: its pointer tables may be reused."""

@@ -13,7 +13,7 @@ HEADERS = [os.path.join(_HERE, "csrc", "lqsgd_dev.h"), os.path.join(_HERE, "csrc
 TARGET = os.path.join(_HERE, "liblqsgd.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-Xcompiler", "-fPIC", "-shared", "-cudart", "shared"]
+              "-Xcompiler", "-fPIC", "-shared", "-cudart", "shared", "-ldl"]
 
 
 def _nvcc() -> str:

@@ -3,6 +3,8 @@
 #include "../../include/lqsgd.h"
 #include "lqsgd_dev.h"
 
+#include <nvtx3/nvToolsExt.h>
+
 #include <algorithm>
 #include <cmath>
 #include <cstring>
@@ -34,19 +36,36 @@ int record_cuda_failure(cudaError_t e, const char* what) { return cuda_fail(e, w
 }  // namespace lqsgd
 namespace {
 
+// NVTX range around the launches of one phase of the round: shows in a timeline tool next to the kernels, costs
+// nothing when no tool is attached (the NVTX header only forwards to an injected library).
+struct NvtxRange {
+  explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+  ~NvtxRange() { nvtxRangePop(); }
+};
+
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // Hands out 256-byte aligned pieces of the workspace; with base == nullptr it only counts.
+// With `guards` set (LQSGD_FLAG_GUARD_WORDS) every piece is followed by kGuardBytes of a fixed pattern that no
+// kernel may touch; their offsets are collected for lqsgd_check_guards.
+constexpr size_t kGuardBytes = 256;
+constexpr uint32_t kGuardPattern = 0xA5C3F00Du;
 struct Arena {
   char* base;
   size_t off = 0;
+  std::vector<uint64_t>* guards = nullptr;
   explicit Arena(void* b) : base(static_cast<char*>(b)) {}
   template <typename T>
   T* take(size_t count) {
     off = align_up(off, 256);
     T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
     off += count * sizeof(T);
+    if (guards) {
+      off = align_up(off, 256);
+      guards->push_back(off);
+      off += kGuardBytes;
+    }
     return p;
   }
 };
@@ -73,6 +92,9 @@ struct Plan {
   std::vector<Tile> tctiles3;                    // tensor-core pass 3 (all workers per tile), grouped by CTA
   std::vector<int> tcbegin3;
   int tc_grid = 0;
+  std::vector<uint64_t> guards;                  // byte offsets of the guard blocks (LQSGD_FLAG_GUARD_WORDS)
+  uint64_t* d_guards = nullptr;
+  unsigned long long* d_guard_result = nullptr;  // [2]: words found changed, offset of the first of them
   bool resident = false;                         // the one-launch round takes this set (lqsgd_resident.cu)
   std::vector<ResTile> rtiles;                   // its tiles, grouped by CTA
   std::vector<int> rbegin;                       // [res_grid + 1]
@@ -140,7 +162,7 @@ int check_config(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
     if (c->world_workers < c->workers || c->world_workers > 4096 || c->world_workers % c->workers) return LQSGD_ERR_INVALID_ARG;
   }
   if (c->flags & ~(LQSGD_FLAG_HOST_STAGING | LQSGD_FLAG_REGISTER_PATH | LQSGD_FLAG_AVERAGE_VALUES |
-                   LQSGD_FLAG_QUANTIZE_VECTORS | LQSGD_FLAG_COLUMN_SCALES | LQSGD_FLAG_ONE_LAUNCH))
+                   LQSGD_FLAG_QUANTIZE_VECTORS | LQSGD_FLAG_COLUMN_SCALES | LQSGD_FLAG_ONE_LAUNCH | LQSGD_FLAG_GUARD_WORDS))
     return LQSGD_ERR_INVALID_ARG;
   for (int i = 0; i < n_layers; ++i) {
     if (shapes[i].rows < 1 || shapes[i].cols < 1) return LQSGD_ERR_BAD_SHAPE;
@@ -495,6 +517,8 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
 
   // ---- carve
   Arena a(base);
+  p.guards.clear();
+  if (cfg.flags & LQSGD_FLAG_GUARD_WORDS) a.guards = &p.guards;
   p.d_layers = a.take<LayerDev>(p.mats.size());
   p.d_vecs = a.take<VectorDev>(p.vecs.size());
   p.state_begin = align_up(a.off, 256);
@@ -691,6 +715,11 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
     p.d_stage_g = a.take<float>((size_t)W * p.elems_total);
     p.d_stage_ghat = a.take<float>(p.elems_total);
   }
+  if (a.guards) {                                   // the table of guard offsets itself, and the check's result
+    a.guards = nullptr;
+    p.d_guards = a.take<uint64_t>(p.guards.size());
+    p.d_guard_result = a.take<unsigned long long>(2);
+  }
   p.bytes = align_up(a.off, 256);
 }
 
@@ -840,6 +869,10 @@ int lqsgd_create(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
   rc = tc_encode_maps(p.layers.data(), (int)p.layers.size(), p.W, p.RP, p.tcmaps.data());
   if (rc != LQSGD_OK) { g_cuda_error = "cuTensorMapEncodeTiled failed or is not available"; return rc; }
   CK(up(p.d_tcmaps, p.tcmaps.data(), p.mats.size() * kTcMapsPerLayer * kTcMapBytes));
+  if (!p.guards.empty()) {
+    CK(up(p.d_guards, p.guards.data(), p.guards.size() * sizeof(uint64_t)));
+    CK(launch_guards(base, p.d_guards, (int)p.guards.size(), kGuardPattern, nullptr, nullptr));
+  }
   CK(up(p.d_rtiles, p.rtiles.data(), p.rtiles.size() * sizeof(ResTile)));
   CK(up(p.d_rbegin, p.rbegin.data(), p.rbegin.size() * sizeof(int)));
   CK(up(p.d_fbP, p.fbP.data(), p.fbP.size() * sizeof(FactorBlock)));
@@ -903,6 +936,22 @@ int lqsgd_test_expire_wait(lqsgd_ctx* c, int32_t pass, int32_t stage, uint32_t w
   c->test_wait_limit = wait_limit;
   c->test_skip_pass = pass;
   c->test_skip_stage = stage;
+  return LQSGD_OK;
+}
+
+int lqsgd_check_guards(const lqsgd_ctx* c, int64_t* host_changed_words, int64_t* host_first_offset, void* cuda_stream) {
+  if (!c || !host_changed_words) return LQSGD_ERR_INVALID_ARG;
+  const Plan& p = c->plan;
+  if (p.guards.empty()) return LQSGD_ERR_INVALID_ARG;            // created without LQSGD_FLAG_GUARD_WORDS
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  CK(cudaMemsetAsync(p.d_guard_result, 0xff, 2 * sizeof(unsigned long long), st));
+  CK(cudaMemsetAsync(p.d_guard_result, 0, sizeof(unsigned long long), st));
+  CK(launch_guards(static_cast<char*>(c->workspace), p.d_guards, (int)p.guards.size(), kGuardPattern, p.d_guard_result, st));
+  unsigned long long res[2] = {0, 0};
+  CK(cudaMemcpyAsync(res, p.d_guard_result, sizeof(res), cudaMemcpyDeviceToHost, st));
+  CK(cudaStreamSynchronize(st));
+  *host_changed_words = (int64_t)res[0];
+  if (host_first_offset) *host_first_offset = res[0] ? (int64_t)res[1] : -1;
   return LQSGD_OK;
 }
 
@@ -1066,6 +1115,9 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
   const bool ride = vectors_ride(c);     // the 1-D tensors travel as extra blocks of the exchange of P
   const bool ev = c->have_events && !split;
 #define PHASE_MARK(i) do { if (ev) CK(cudaEventRecord(c->phase_events[i], st)); } while (0)
+  static const char* const kSegName[6] = {"lqsgd: pass 1 + Orthonormalize", "lqsgd: exchange of P", "lqsgd: pass 2 + Q_w",
+                                          "lqsgd: exchange of Q", "lqsgd: sum of Q over ranks", "lqsgd: pass 3"};
+  NvtxRange nvtx(kSegName[seg >= 0 && seg <= 5 ? seg : 0]);
   switch (seg) {
     case 0:
       if (nv && !repeat) {
@@ -1165,6 +1217,7 @@ static int run_resident(lqsgd_ctx* c, cudaStream_t st) {
   a.sync = p.d_rsync;
   a.stamps = p.d_rstamps;
   // phase events: one kernel, so the round's time shows as its first phase and the others as empty
+  NvtxRange nvtx("lqsgd: round in one launch");
   if (c->have_events) CK(cudaEventRecord(c->phase_events[0], st));
   CK(launch_resident(p.RP, t, a, p.res_grid, p.res_smem, st));
   if (c->have_events)

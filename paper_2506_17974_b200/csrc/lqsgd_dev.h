@@ -205,6 +205,9 @@ struct VectorJob {
 // ride: the 1-D tensors' blocks appended to this launch (or null)
 cudaError_t launch_exchange(int RP, int which /*0 = P, 1 = Q*/, const Tables& t, const QuantTables& q,
                             const ExchangeChunk* ch, int nch, const SplitExchange& sx, const VectorJob* ride, Launch l);
+// Guard blocks of the workspace (256 bytes each at base + offs[i]): result == null fills them with the pattern, else
+// counts the words that no longer hold it into result[0] and keeps the smallest byte offset of one in result[1].
+cudaError_t launch_guards(char* base, const uint64_t* offs, int n, uint32_t pattern, unsigned long long* result, cudaStream_t st);
 cudaError_t launch_unpack_codes(const uint8_t* stream, int count, int bits, uint8_t* out, cudaStream_t st);
 cudaError_t launch_scale_reduce(int RP, const Tables& t, int which, float* scales, int n_mat, Launch l);
 cudaError_t launch_sum_dequant(int RP, int which, const Tables& t, const QuantTables& q, const ExchangeChunk* ch,

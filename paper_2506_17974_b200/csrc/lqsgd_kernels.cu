@@ -539,6 +539,18 @@ unpack_codes_kernel(const uint8_t* __restrict__ stream, int count, int b, uint8_
   out[e] = (uint8_t)((v >> sh) & ((1u << b) - 1u));
 }
 
+// Guard blocks between the pieces of the workspace: one block of 64 threads per guard, one word per thread.
+__global__ void __launch_bounds__(64)
+guards_kernel(char* base, const uint64_t* __restrict__ offs, uint32_t pattern, unsigned long long* result) {
+  const uint64_t off = offs[blockIdx.x] + 4ull * threadIdx.x;
+  uint32_t* w = reinterpret_cast<uint32_t*>(base + off);
+  if (!result) { *w = pattern; return; }
+  if (*w != pattern) {
+    atomicAdd(result, 1ull);
+    atomicMin(result + 1, (unsigned long long)off);
+  }
+}
+
 // Qt[j][i] = Q[i][j]: refreshes the transposed copy after Q was set from outside.
 __global__ void __launch_bounds__(256)
 q_transpose_kernel(const float* __restrict__ Q, float* __restrict__ Qt, float* __restrict__ Qcat, int m, int RP, int mt,
@@ -845,6 +857,12 @@ cudaError_t launch_exchange(int rp, int which, const Tables& t, const QuantTable
     }
   });
 #undef LQSGD_EXCHANGE_BITS
+  return cudaGetLastError();
+}
+
+cudaError_t launch_guards(char* base, const uint64_t* offs, int n, uint32_t pattern, unsigned long long* result, cudaStream_t st) {
+  if (n == 0) return cudaSuccess;
+  guards_kernel<<<n, 64, 0, st>>>(base, offs, pattern, result);
   return cudaGetLastError();
 }
 

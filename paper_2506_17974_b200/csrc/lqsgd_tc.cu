@@ -137,6 +137,11 @@ struct Pass2Cfg {
   static constexpr uint32_t kTotal = kBarOff + kBars * 8 + 16 + 1024;    // + abort flag, TMEM slot, alignment slack
   static_assert(kACol0 + kAB * kTcSlotK <= 512, "tensor memory");
   static_assert(kTotal <= 227 * 1024, "shared memory");
+  // A ring's barrier tells its phases apart by parity alone: a waiter two phases ahead of the barrier would take
+  // the phase before the one in progress for its own.  A consumer group can run at most the M ring (kMStages
+  // pieces) ahead of the slowest group, and the MMA thread waits for all groups: that must stay below two turns of
+  // the operand ring (2 kAB slots of kTcPair pieces).
+  static_assert(kMStages < 2 * kAB * kTcPair, "a consumer must not get two turns of the operand ring ahead");
   static_assert(kN % 16 == 0 && kN <= 256, "N of one MMA");
 };
 
@@ -398,6 +403,7 @@ struct Pass1Cfg {
   static_assert(kACol0 + kT1AB * 64 <= 512, "tensor memory");
   static_assert(kBBytes % 1024 == 0, "B stages stay 1024-byte aligned");
   static_assert(kTotal <= 227 * 1024, "shared memory");
+  static_assert(kT1Stages < 2 * kT1AB, "a consumer must not get two turns of the operand ring ahead (see Pass2Cfg)");
 };
 
 template <int RP>

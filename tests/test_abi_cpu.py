@@ -49,7 +49,7 @@ def test_workspace_bytes_covers_the_persistent_state(lib):
     (dict(bits_p=1), B.ERR_INVALID_ARG), (dict(bits_q=9), B.ERR_INVALID_ARG),
     (dict(alpha=0.0), B.ERR_INVALID_ARG), (dict(alpha=float("nan")), B.ERR_INVALID_ARG),
     (dict(workers=0), B.ERR_INVALID_ARG), (dict(workers=257), B.ERR_INVALID_ARG),
-    (dict(flags=64), B.ERR_INVALID_ARG), (dict(flags=128), B.ERR_INVALID_ARG), (dict(power_iters=9), B.ERR_INVALID_ARG), (dict(power_iters=-1), B.ERR_INVALID_ARG),
+    (dict(flags=256), B.ERR_INVALID_ARG), (dict(flags=128), B.ERR_INVALID_ARG), (dict(power_iters=9), B.ERR_INVALID_ARG), (dict(power_iters=-1), B.ERR_INVALID_ARG),
     (dict(power_iters=2, world_workers=2), B.ERR_INVALID_ARG),
 ])
 def test_bad_config_is_rejected_on_the_host(lib, kw, code):

@@ -2,6 +2,7 @@
 on the same seeded inputs.  Tolerances: relative Frobenius error <= 1e-4 on P, Q, G_hat and E;
 codes bit-exact except elements on a decision threshold, whose fraction (<= 1e-5) is counted;
 payload bytes exact."""
+import ctypes as C
 import dataclasses
 import time
 
@@ -344,6 +345,47 @@ def test_one_launch_round_variants(kw):
     run_steps(w, 3, comp=comp)
     tl = comp.round_timeline()
     assert len(tl) >= 6 and all(b >= a for a, b in zip(tl, tl[1:]))       # the kernel's own timeline of the round
+
+
+GUARDED_CASES = {
+    "staged_ragged": dict(layers=((250, 250), (64, 27), (128, 64), (9, 1), (300, 251), (33, 17), (1030, 516)), rank=3, W=3),
+    "rank8_plain": dict(layers=((96, 200), (130, 36), (17, 33), (5, 3), (2, 2), (700, 512)), rank=8, W=2),
+    "tensor_core_16": dict(layers=((128, 576), (520, 1156), (64, 27), (100, 512), (40, 129)), rank=16, W=3),
+    "tensor_core_50": dict(layers=((128, 576), (300, 260), (64, 27), (33, 17)), rank=50, W=2),
+    "one_launch": dict(layers=((96, 200), (130, 36), (64, 27), (20, 1), (700, 512)), rank=5, W=3, one_launch=True),
+    "register_path": dict(layers=((96, 200), (64, 27), (300, 251)), rank=4, W=2, register_path=True),
+    "column_scales": dict(layers=((96, 200), (64, 27), (300, 252)), rank=6, W=2, column_scales=True),
+}
+
+
+@pytest.mark.parametrize("name", sorted(GUARDED_CASES))
+def test_no_kernel_writes_outside_its_workspace_piece(name):
+    """The stand-in for a memory checker: with LQSGD_FLAG_GUARD_WORDS every piece of the workspace is followed by a
+    block of pattern words.  After rounds over ragged shapes on every kernel family none of them may have changed;
+    and a write planted by the test right behind the payloads is found, at its offset."""
+    case = dict(GUARDED_CASES[name])
+    layers, rank, W = case.pop("layers"), case.pop("rank"), case.pop("W")
+    w = wl.Workload("guards", layers, rank=rank, bits=5, workers=W, steps=3, dist="student_t3", scale="fan_in", seed=23)
+    comp = make(w, guard_words=True, **case)
+    assert comp.check_guards() == (0, -1)
+    for t in range(3):
+        g = wl.draw_gradients(w, t, device=DEV)
+        comp.step(g, [torch.empty(s, device=DEV) for s in layers])
+    for l in range(len(layers)):                                   # state reads and writes go through kernels too
+        if comp.is_matrix(l):
+            comp.get_state(B.STATE_CODES_Q, l, W - 1)
+            comp.set_state(B.STATE_Q, l, 0, comp.get_state(B.STATE_Q, l))
+    assert comp.check_guards() == (0, -1)
+    assert all(s & B.STATUS_TIMEOUT == 0 for s in comp.status())
+    # a planted write: the first byte behind the last worker's payload slot is the start of a guard block
+    ptr, nb = C.c_void_p(), C.c_size_t(0)
+    B._check(comp.lib.lqsgd_payload(comp.ctx, 0, C.byref(ptr), C.byref(nb)))
+    stride = (comp.payload_nbytes + 15) // 16 * 16
+    end = ptr.value - comp._ws_ptr + W * stride
+    guard = (end + 255) // 256 * 256
+    comp.workspace[comp._ws_ptr - comp.workspace.data_ptr() + guard + 5] = 1
+    bad, first = comp.check_guards()
+    assert bad == 1 and first == guard + 4, (bad, first, guard)
 
 
 def test_different_bits_for_p_and_q():
