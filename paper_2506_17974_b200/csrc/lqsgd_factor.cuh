@@ -564,9 +564,17 @@ template <int RP, int NT> struct ExchangeSmem {
   float scol[RP];
 };
 
-template <int RP, int B, int NT, bool COH>
-__device__ __forceinline__ void exchange_body(const Tables& t, const QuantTables& qt, int which, const ExchangeChunk ch,
-                                              const SplitExchange& sx, int tid, void* smem) {
+// PLAIN: Algorithm 1's exchange as it stands - one scale per factor, average of the level indices, all workers on
+// this GPU - with the variants compiled out: the kernel is then half the size, and for a step this short the
+// size of its code is a large part of its cost.
+template <int RP, int B, int NT, bool COH, bool PLAIN = false>
+__device__ __forceinline__ void exchange_body(const Tables& t, const QuantTables& qt_in, int which, const ExchangeChunk ch,
+                                              const SplitExchange& sx_in, int tid, void* smem) {
+  struct QtView { const float* thr; const float* deq; int32_t bits; int32_t avg_values; };
+  struct SxView { int32_t pack_only, n_mat, ns; const float* scales; uint8_t* send[2]; uint64_t region_bytes[2], region_off[2]; };
+  const QtView qt{qt_in.thr, qt_in.deq, qt_in.bits, PLAIN ? 0 : qt_in.avg_values};
+  const SxView sx{PLAIN ? 0 : sx_in.pack_only, sx_in.n_mat, sx_in.ns, sx_in.scales, {sx_in.send[0], sx_in.send[1]},
+                  {sx_in.region_bytes[0], sx_in.region_bytes[1]}, {sx_in.region_off[0], sx_in.region_off[1]}};
   constexpr int CH = kExchangeChunk;   // 256 factor elements per job, one per thread
   constexpr int WB = 8;                // workers handled per round
   const int bits = B ? B : qt.bits;    // a compile-time constant unless B == 0
@@ -596,7 +604,7 @@ __device__ __forceinline__ void exchange_body(const Tables& t, const QuantTables
   for (int i = tid; i < NLEV - 1; i += NT) S.thr[i] = qt.thr[i];
   if (tid < WB) *reinterpret_cast<uint32_t*>(&S.codes[tid][CH]) = 0u;     // what a word task reads past the chunk
   float s = 0.f;
-  const bool cs = t.col_scales != 0;
+  const bool cs = PLAIN ? false : t.col_scales != 0;
   if (cs) {
     // variant: one scale per column.  Block maxima are [W][nblk][RP]; thread tid only meets column tid % RP.
     // (a maximum of non-negative floats is the maximum of their bit patterns as integers: exact, in any order)
@@ -672,9 +680,11 @@ __device__ __forceinline__ void exchange_body(const Tables& t, const QuantTables
       const int wn = min(WB, W - w0);
       float x[WB];
 #pragma unroll
-      for (int u = 0; u < WB; ++u) {
-        if (w0 == 0) x[u] = xfirst[u];
-        else x[u] = (valid && u < wn) ? ld_in<COH>(src + ((size_t)(w0 + u) * rows + row) * RP + col) : 0.f;
+      for (int u = 0; u < WB; ++u) x[u] = xfirst[u];
+      if (w0 + WB < W) {           // the next round's values set out before this round is quantised and packed
+#pragma unroll
+        for (int u = 0; u < WB; ++u)
+          xfirst[u] = (valid && w0 + WB + u < W) ? ld_in<COH>(src + ((size_t)(w0 + WB + u) * rows + row) * RP + col) : 0.f;
       }
       if (tid < CH) {
 #pragma unroll

@@ -512,7 +512,7 @@ vectors_kernel(VectorJob vj, uint8_t* payload, uint64_t payload_stride, int W) {
 
 // Factor exchange, one block per chunk of 256 factor elements; blocks past the factor chunks take the
 // round's 1-D tensors (same block shape), which saves a launch per round.
-template <int RP, int B>
+template <int RP, int B, bool PLAIN>
 __global__ void __launch_bounds__(256)
 exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __restrict__ chunks, int nchunks,
                 SplitExchange sx, VectorJob vj) {
@@ -522,7 +522,7 @@ exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __rest
     return;
   }
   __shared__ __align__(16) unsigned char smem[sizeof(ExchangeSmem<RP, 256>)];
-  exchange_body<RP, B, 256, false>(t, qt, which, chunks[blockIdx.x], sx, threadIdx.x, smem);
+  exchange_body<RP, B, 256, false, PLAIN>(t, qt, which, chunks[blockIdx.x], sx, threadIdx.x, smem);
 }
 
 // One worker's unpacked codes (one per byte) from its packed stream: what lqsgd_get_state returns
@@ -848,7 +848,11 @@ cudaError_t launch_exchange(int rp, int which, const Tables& t, const QuantTable
   if (nch == 0) return cudaSuccess;
   const VectorJob vj = ride ? *ride : VectorJob{};
   const int grid = nch + vj.nchunks;
-#define LQSGD_EXCHANGE_BITS(BV) case BV: launch_pdl(exchange_kernel<RP, BV>, grid, 256, 0, l.stream, t, q, which, ch, nch, sx, vj); break;
+  const bool plain = !t.col_scales && !q.avg_values && !sx.pack_only;
+#define LQSGD_EXCHANGE_BITS(BV) case BV: \
+    if (plain) launch_pdl(exchange_kernel<RP, BV, true>, grid, 256, 0, l.stream, t, q, which, ch, nch, sx, vj); \
+    else launch_pdl(exchange_kernel<RP, BV, false>, grid, 256, 0, l.stream, t, q, which, ch, nch, sx, vj); \
+    break;
   LQSGD_DISPATCH_RP(rp, {
     switch (q.bits) {
       LQSGD_EXCHANGE_BITS(2) LQSGD_EXCHANGE_BITS(3) LQSGD_EXCHANGE_BITS(4) LQSGD_EXCHANGE_BITS(5)
