@@ -70,6 +70,8 @@ def recorded_traffic(workload: str, phase: str):
 def kernel_name(phase: str, rank: int) -> str:
     """The kernel that carries a pass for layers with 16-byte aligned rows at this rank (unaligned layers,
     a few KB in the ResNet set, run on the register kernels of the same phase)."""
+    if phase == "round":
+        return "resident_round_kernel"
     n = phase[-1]
     if rank > 8:
         return f"tc_pass{n}_kernel"
@@ -267,9 +269,10 @@ def run_ours(args):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         return [float(v) for v in t.tolist()]
 
-    def bench_workload(wl_obj, steps, warmup, nsets, want_e2e, sample_clocks, want_graph=False, min_ms=0.0):
+    def bench_workload(wl_obj, steps, warmup, nsets, want_e2e, sample_clocks, want_graph=False, min_ms=0.0,
+                       one_launch=False):
         comp = B.LQSGD(wl_obj.layers, wl_obj.rank, wl_obj.bits, alpha=wl_obj.alpha, workers=wl_obj.workers,
-                       seed=wl_obj.seed + rank, device=dev)
+                       seed=wl_obj.seed + rank, device=dev, one_launch=one_launch)
         seeded = dataclasses.replace(wl_obj, seed=wl_obj.seed + 1000 * rank)
         sets = [wl.draw_gradients(seeded, t, device=dev) for t in range(nsets)]
         ghat = [torch.empty_like(g) for g in sets[0][0]]
@@ -448,8 +451,9 @@ def run_ours(args):
         wl_obj = dataclasses.replace(wl_obj, workers=args.workers)
         desc += f" [workers overridden: W={args.workers}]"
     gbytes = gradient_bytes(wl_obj)
-    res = bench_workload(wl_obj, args.steps, args.warmup, nsets=3, want_e2e=not args.no_e2e, sample_clocks=True,
-                         want_graph=not args.no_graph, min_ms=args.min_ms)
+    nsets_main = max(3, min(16, -(-int(2.5e8) // gbytes)))          # a rotation streams more than twice the L2
+    res = bench_workload(wl_obj, args.steps, args.warmup, nsets=nsets_main, want_e2e=not args.no_e2e, sample_clocks=True,
+                         want_graph=not args.no_graph, min_ms=args.min_ms, one_launch=args.one_launch)
 
     ms = res["ms"]
     e2e_ms = allmax(res.get("e2e_ms", float("nan")))
@@ -457,9 +461,21 @@ def run_ours(args):
     pb = phase_bytes(wl_obj)
     dom = max(("pass1", "pass2", "pass3"), key=lambda k: res["phases_ms"][k])
     achieved = pb[dom] / (res["phases_ms"][dom] * 1e-3) / 1e9
-    round_bytes = sum(pb.values())
+    round_bytes = sum(v for k, v in pb.items() if k != "round")
     traffic = recorded_traffic(args.workload, dom)
+    one_launch = res["launches"] == 1 and args.one_launch
+    if one_launch:
+        # the whole round is one kernel that reads G and E and writes E and G_hat: 12 + 4/W bytes per worker-element
+        from paper_2506_17974_b200 import workloads as _wl
+        nm = _wl.matrix_elements(wl_obj.layers)
+        dom = "round"
+        pb = dict(pb, round=12 * wl_obj.workers * nm + 4 * nm)
+        res["phases_ms"] = dict(res["phases_ms"], round=ms)
+        achieved = pb["round"] / (ms * 1e-3) / 1e9
+        traffic = recorded_traffic(args.workload, "round")
     cfg = config_dict(wl_obj, desc)
+    if args.one_launch:
+        cfg["one_launch"] = bool(one_launch)
     cfg["parallelism"] = f"{world} independent replica(s), one per GPU, no collective"
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -517,6 +533,14 @@ def run_ours(args):
             ro = bench_workload(wo, steps=20, warmup=3, nsets=nso, want_e2e=False, sample_clocks=False, min_ms=30.0)
             others[name] = dict(compact(wo, ro), gradient_sets_rotated=nso,
                                 compression_ratio=4 * sum(n * m for n, m in wo.layers) / ro["payload"])
+            if name in ("single", "mnist"):
+                # the same set as ONE cooperative launch with M resident in shared memory (LQSGD_FLAG_ONE_LAUNCH)
+                r1 = bench_workload(wo, steps=20, warmup=3, nsets=nso, want_e2e=False, sample_clocks=False, min_ms=30.0,
+                                    one_launch=True)
+                others[name]["one_launch"] = {"ms_per_step": r1["ms"], "launches_per_step": r1["launches"]}
+        w4 = wl.config4(1024, 4096)
+        r1 = bench_workload(w4, steps=30, warmup=3, nsets=15, want_e2e=False, sample_clocks=False, min_ms=50.0, one_launch=True)
+        line["large_layer_sweep"]["1024x4096"]["one_launch"] = {"ms_per_step": r1["ms"], "launches_per_step": r1["launches"]}
         line["other_configs"] = others
     if rank == 0 and world == 1 and args.config5_sweep:
         # rank x bits grid on the 16-worker ResNet-18 (100 classes) set: throughput, compression ratio and
@@ -652,6 +676,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle")
     ap.add_argument("--min-ms", type=float, default=500.0,
                     help="repeat the block of --steps steps until this much device time has been timed (0: one block)")
+    ap.add_argument("--one-launch", action="store_true",
+                    help="run the round as one cooperative kernel with M resident in shared memory, if the set qualifies")
     ap.add_argument("--overlap", action="store_true",
                     help="with --exchange: the layer table cut in two halves on two streams, collectives under compute")
     ap.add_argument("--exchange", action="store_true",

@@ -107,6 +107,8 @@ struct Plan {
   std::vector<uint8_t> tcmaps;                   // tensor maps of the tensor-core passes (filled at create)
   std::vector<FactorBlock> fbP, fbQ;             // 128-row blocks of P (layers orthonormalised in two launches) and of Q
   std::vector<FactorBlock> fbS;                  // (layer, worker) of the layers orthonormalised by one CTA
+  std::vector<FactorBlock> fbC;                  // padded rank >= 32: (layer, worker) whose Cholesky factor a CTA of its own computes
+  FactorBlock* d_fbC = nullptr;
   std::vector<ExchangeChunk> chP, chQ, chV;
   std::vector<float> thrP, thrQ, deqP, deqQ;
   std::vector<lqsgd_layer_layout> layout;     // by user layer index
@@ -557,6 +559,7 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
     L.Qpart = a.take<float>((size_t)W * L.nrb * mt.m * RP);
     L.Qw = (L.nrb == 1) ? L.Qpart : a.take<float>((size_t)W * mt.m * RP);
     L.gram_part = a.take<double>((size_t)W * L.npb * RP * RP);
+    L.chol = RP >= kCholSplitRP ? a.take<double>((size_t)W * (RP * RP + 2 * RP)) : nullptr;
     L.maxp = a.take<float>((size_t)W * L.npb * (colscales ? RP : 1));
     L.maxq = a.take<float>((size_t)W * L.nqb * (colscales ? RP : 1));
     L.scales = a.take<float>(2 * (size_t)RP);
@@ -626,6 +629,7 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
     const bool one_cta = RP <= 8 && mt.n <= kOrthSmallMaxRows;
     for (int w = 0; w < W; ++w) {
       if (one_cta) p.fbS.push_back({li32, w, 0, 0});
+      if (!one_cta && RP >= kCholSplitRP) p.fbC.push_back({li32, w, 0, 0});
       for (int b = 0; !one_cta && b < L.npb; ++b) p.fbP.push_back({li32, w, b, 0});
       for (int b = 0; b < L.nqb; ++b) p.fbQ.push_back({li32, w, b, 0});
     }
@@ -696,6 +700,7 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   p.d_fbP = a.take<FactorBlock>(p.fbP.size());
   p.d_fbQ = a.take<FactorBlock>(p.fbQ.size());
   p.d_fbS = a.take<FactorBlock>(p.fbS.size());
+  p.d_fbC = a.take<FactorBlock>(p.fbC.size());
   p.d_chP = a.take<ExchangeChunk>(p.chP.size());
   p.d_chQ = a.take<ExchangeChunk>(p.chQ.size());
   p.d_chV = a.take<ExchangeChunk>(p.chV.size());
@@ -878,6 +883,7 @@ int lqsgd_create(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
   CK(up(p.d_fbP, p.fbP.data(), p.fbP.size() * sizeof(FactorBlock)));
   CK(up(p.d_fbQ, p.fbQ.data(), p.fbQ.size() * sizeof(FactorBlock)));
   CK(up(p.d_fbS, p.fbS.data(), p.fbS.size() * sizeof(FactorBlock)));
+  CK(up(p.d_fbC, p.fbC.data(), p.fbC.size() * sizeof(FactorBlock)));
   CK(up(p.d_chP, p.chP.data(), p.chP.size() * sizeof(ExchangeChunk)));
   CK(up(p.d_chQ, p.chQ.data(), p.chQ.size() * sizeof(ExchangeChunk)));
   CK(up(p.d_chV, p.chV.data(), p.chV.size() * sizeof(ExchangeChunk)));
@@ -984,7 +990,7 @@ int lqsgd_launches_per_step(const lqsgd_ctx* ctx, int32_t* out) {
   const int pass2 = (p.tiles2.empty() ? 0 : 1) + (p.tctiles2.empty() ? 0 : 1);
   const int pass3 = (p.tiles3.empty() ? 0 : 1) + (p.stiles3.empty() ? 0 : 1) + (p.tctiles3.empty() ? 0 : 1);
   const int iters = std::max(1, ctx->cfg.power_iters);
-  const int orth = (p.fbS.empty() ? 0 : 1) + (p.fbP.empty() ? 0 : 2);     // one CTA per small layer / Gram + apply
+  const int orth = (p.fbS.empty() ? 0 : 1) + (p.fbP.empty() ? 0 : 2) + (p.fbC.empty() ? 0 : 1);   // one CTA per small layer / Gram (+ Cholesky) + apply
   *out = iters * ((p.mats.empty() ? 0 : orth + 3) + pass1 + pass2) + pass3 + ((p.chV.empty() || vectors_ride(ctx)) ? 0 : 1);
   return LQSGD_OK;
 }
@@ -1148,6 +1154,7 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
       if (nm) {
         CK(launch_p_orth_small(RP, t, p.d_fbS, (int)p.fbS.size(), {st, 0}));
         CK(launch_p_reduce_gram(RP, t, p.d_fbP, (int)p.fbP.size(), {st, 0}));
+        if (RP >= kCholSplitRP) CK(launch_p_chol(RP, t, p.d_fbC, (int)p.fbC.size(), {st, 0}));
         CK(launch_p_apply(RP, t, p.d_fbP, (int)p.fbP.size(), {st, 0}));
         if (split) CK(launch_scale_reduce(RP, t, 0, p.d_xscales, (int)nm, {st, 0}));
       }

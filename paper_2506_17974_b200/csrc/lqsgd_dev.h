@@ -39,6 +39,7 @@ struct LayerDev {
   float* Qpart;               // [W][nrb][m][RP]
   float* Qw;                  // [W][m][RP]  (== Qpart when nrb == 1)
   double* gram_part;          // [W][npb][RP*RP]
+  double* chol;               // padded rank >= 32: [W][RP*RP + 2 RP]  Cholesky factor L (row-major), 1 / diag, dropped flags
   float* maxp;                // [W][npb] block maxima of |P|; with column scales [W][npb][RP], one per column
   float* maxq;                // [W][nqb] (or [W][nqb][RP])
   float* scales;              // [2 RP]: s_P at [0], s_Q at [1]; with column scales s_P[j] at [j], s_Q[j] at [RP + j]
@@ -173,6 +174,10 @@ struct Launch {
 cudaError_t launch_pass1(int RP, const Tables& t, const Tile* tiles, int ntiles, Launch l);
 cudaError_t launch_p_reduce_gram(int RP, const Tables& t, const FactorBlock* fb, int nfb, Launch l);
 cudaError_t launch_p_apply(int RP, const Tables& t, const FactorBlock* fb, int nfb, Launch l);
+// padded rank >= kCholSplitRP: the Cholesky factor of each (layer, worker) once, by a CTA of its own, instead of again in
+// every CTA of p_apply (at rank 64 the factorisation is the long part); fb lists one entry per (layer, worker)
+constexpr int kCholSplitRP = 32;
+cudaError_t launch_p_chol(int RP, const Tables& t, const FactorBlock* fb, int nfb, Launch l);
 // Orthonormalize in one launch for layers of at most kOrthSmallMaxRows rows at RP <= 8: one CTA per (layer, worker)
 constexpr int kOrthSmallMaxRows = 512;
 cudaError_t launch_p_orth_small(int RP, const Tables& t, const FactorBlock* fb, int nfb, Launch l);

@@ -69,7 +69,7 @@ __device__ __forceinline__ void store_contig(float* p, const float (&v)[N]) {
 // ---------------------------------------------------------------------------------------
 constexpr double kPivotEps = 1e-10;
 
-template <int RP> struct ReduceGramSmem { float rows[kFactorBlockRows][RP]; };   // the block's rows (fp32: they are fp32 data)
+template <int RP> struct ReduceGramSmem { alignas(16) float rows[kFactorBlockRows][RP]; };   // the block's rows (fp32: they are fp32 data)
 
 template <int RP, int NT, bool COH>
 __device__ __forceinline__ void p_reduce_gram_body(const Tables& t, const FactorBlock fb, int tid, void* smem) {
@@ -108,14 +108,46 @@ __device__ __forceinline__ void p_reduce_gram_body(const Tables& t, const Factor
     for (int j = 0; j < RP; ++j) S.rows[tid][j] = p[j];
   }
   __syncthreads();
-  for (int e = tid; e < RP * RP; e += NT) {
-    const int i = e / RP, j = e % RP;
-    if (j < i) continue;                                 // the Gram matrix is symmetric: upper triangle, mirrored
-    double s = 0.0;
-    for (int k = 0; k < kFactorBlockRows; ++k) s = fma((double)S.rows[k][i], (double)S.rows[k][j], s);
-    double* gp = L.gram_part + ((size_t)fb.worker * L.npb + fb.blk) * (RP * RP);
-    gp[i * RP + j] = s;
-    gp[j * RP + i] = s;
+  double* gp = L.gram_part + ((size_t)fb.worker * L.npb + fb.blk) * (RP * RP);
+  if constexpr (RP >= 32) {
+    // 4 x 4 entries per thread: two 128-bit reads of a row feed 16 multiply-adds (one entry per thread would read
+    // two values per multiply-add, and the shared-memory reads, not the fp64 units, would set the pace)
+    constexpr int TD = RP / 4;
+    for (int tile = tid; tile < TD * TD; tile += NT) {
+      const int ti = tile / TD, tj = tile % TD;
+      if (tj < ti) continue;                               // symmetric: upper triangle of tiles, mirrored
+      double acc[4][4];
+#pragma unroll
+      for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) acc[a][b] = 0.0;
+      for (int k = 0; k < kFactorBlockRows; ++k) {
+        const float4 x = *reinterpret_cast<const float4*>(&S.rows[k][4 * ti]);
+        const float4 y = *reinterpret_cast<const float4*>(&S.rows[k][4 * tj]);
+        const double xa[4] = {(double)x.x, (double)x.y, (double)x.z, (double)x.w};
+        const double yb[4] = {(double)y.x, (double)y.y, (double)y.z, (double)y.w};
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+          for (int b = 0; b < 4; ++b) acc[a][b] = fma(xa[a], yb[b], acc[a][b]);
+      }
+#pragma unroll
+      for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+          gp[(4 * ti + a) * RP + 4 * tj + b] = acc[a][b];
+          gp[(4 * tj + b) * RP + 4 * ti + a] = acc[a][b];
+        }
+    }
+  } else {
+    for (int e = tid; e < RP * RP; e += NT) {
+      const int i = e / RP, j = e % RP;
+      if (j < i) continue;                                 // the Gram matrix is symmetric: upper triangle, mirrored
+      double s = 0.0;
+      for (int k = 0; k < kFactorBlockRows; ++k) s = fma((double)S.rows[k][i], (double)S.rows[k][j], s);
+      gp[i * RP + j] = s;
+      gp[j * RP + i] = s;
+    }
   }
 }
 
@@ -220,6 +252,68 @@ __device__ __forceinline__ bool cholesky_lower(const LayerDev& L, int worker, Ch
   return cholesky_factor<RP, NT>(C.A, C.diag0, L.r, invd, dead, tid);
 }
 
+// Padded rank >= kCholSplitRP: Gram = sum of the block Grams and its Cholesky factor, ONCE per (layer, worker), by a CTA
+// of its own whose threads all take part in the trailing updates (CTA barriers between the steps); the factor,
+// the reciprocals of its diagonal and the dropped-column flags go to L.chol for p_apply_body to fetch.
+template <int RP, int NT> struct CholOnceSmem {
+  double A[RP][RP + 1];
+  double diag0[RP];
+  double invd[RP];
+  int dead[RP];
+};
+
+template <int RP, int NT, bool COH>
+__device__ __forceinline__ void p_chol_body(const Tables& t, const FactorBlock fb, int tid, void* smem) {
+  auto& S = *static_cast<CholOnceSmem<RP, NT>*>(smem);
+  const LayerDev& L = t.layers[fb.layer];
+  const int r = L.r;
+  for (int e = tid; e < RP * RP; e += NT) {
+    const double* gp = L.gram_part + (size_t)fb.worker * L.npb * (RP * RP) + e;
+    double s = 0.0;
+    int b = 0;
+    for (; b + 8 <= L.npb; b += 8) {        // eight loads in flight, additions in block order
+      double x[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) x[u] = ld_in<COH>(gp + (size_t)(b + u) * (RP * RP));
+#pragma unroll
+      for (int u = 0; u < 8; ++u) s += x[u];
+    }
+    for (; b < L.npb; ++b) s += ld_in<COH>(gp + (size_t)b * (RP * RP));
+    S.A[e / RP][e % RP] = s;
+  }
+  __syncthreads();
+  if (tid < RP) { S.diag0[tid] = S.A[tid][tid]; S.dead[tid] = 0; S.invd[tid] = 1.0; }
+  __syncthreads();
+  for (int j = 0; j < r; ++j) {
+    const double d = S.A[j][j];
+    const bool ok = (d > kPivotEps * S.diag0[j]) && (d < INFINITY);   // false for nan too
+    const double inv = ok ? rsqrt(d) : 1.0;
+    const double ljj = ok ? d * inv : 1.0;
+    __syncthreads();                       // everybody has read the pivot
+    for (int i = j + tid; i < r; i += NT) {
+      if (i == j) { S.A[j][j] = ljj; S.invd[j] = inv; if (!ok) S.dead[j] = 1; }
+      else S.A[i][j] = ok ? S.A[i][j] * inv : 0.0;
+    }
+    __syncthreads();
+    if (ok) {
+      const int w = r - j - 1;             // trailing block: rows and columns j+1 .. r-1, lower triangle
+      for (int e = tid; e < w * w; e += NT) {
+        const int i = j + 1 + e / w, k = j + 1 + e % w;
+        if (k <= i) S.A[i][k] -= S.A[i][j] * S.A[k][j];
+      }
+    }
+    __syncthreads();                       // the next pivot is read only after its last update
+  }
+  double* dst = L.chol + (size_t)fb.worker * (RP * RP + 2 * RP);
+  for (int e = tid; e < RP * RP; e += NT) dst[e] = S.A[e / RP][e % RP];
+  if (tid < RP) { dst[RP * RP + tid] = S.invd[tid]; dst[RP * RP + RP + tid] = S.dead[tid] ? 1.0 : 0.0; }
+  if (tid == 0) {
+    int any = 0;
+    for (int j = 0; j < r; ++j) any |= S.dead[j];
+    if (any) atomicOr(&t.status[fb.layer], 1u);
+  }
+}
+
 template <int RP, int NT> struct ApplySmem {
   CholSmem<RP> chol;
   double invd[RP];
@@ -235,8 +329,16 @@ __device__ __forceinline__ void p_apply_body(const Tables& t, const FactorBlock 
   auto& S = *static_cast<ApplySmem<RP, NT>*>(smem);
   const LayerDev& L = t.layers[fb.layer];
   const int n = L.n;
-  const bool dropped = cholesky_lower<RP, NT, COH>(L, fb.worker, S.chol, S.invd, S.dead, tid);
-  if (dropped && fb.blk == 0 && tid == 0) atomicOr(&t.status[fb.layer], 1u);
+  if constexpr (RP >= kCholSplitRP) {
+    // the factor was computed once for this (layer, worker) by p_chol_body: fetch it
+    const double* src = L.chol + (size_t)fb.worker * (RP * RP + 2 * RP);
+    for (int e = tid; e < RP * RP; e += NT) S.chol.A[e / RP][e % RP] = ld_in<COH>(src + e);
+    if (tid < RP) { S.invd[tid] = ld_in<COH>(src + RP * RP + tid); S.dead[tid] = ld_in<COH>(src + RP * RP + RP + tid) != 0.0; }
+    __syncthreads();
+  } else {
+    const bool dropped = cholesky_lower<RP, NT, COH>(L, fb.worker, S.chol, S.invd, S.dead, tid);
+    if (dropped && fb.blk == 0 && tid == 0) atomicOr(&t.status[fb.layer], 1u);
+  }
   const int row = fb.blk * kFactorBlockRows + tid;
   float o[RP];
 #pragma unroll

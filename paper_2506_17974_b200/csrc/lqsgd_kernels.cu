@@ -487,6 +487,14 @@ p_apply_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
 }
 
 template <int RP>
+__global__ void __launch_bounds__(256)
+p_chol_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
+  pdl_wait();
+  __shared__ __align__(16) unsigned char smem[sizeof(CholOnceSmem<RP, 256>)];
+  p_chol_body<RP, 256, false>(t, fbs[blockIdx.x], threadIdx.x, smem);
+}
+
+template <int RP>
 __global__ void __launch_bounds__(kOrthSmallRows, 3)   // three CTAs per SM: 444 at once, one wave for 21 layers x 16 workers
 p_orth_small_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
   pdl_wait();
@@ -822,6 +830,16 @@ cudaError_t launch_p_reduce_gram(int rp, const Tables& t, const FactorBlock* fb,
 cudaError_t launch_p_apply(int rp, const Tables& t, const FactorBlock* fb, int nfb, Launch l) {
   if (nfb == 0) return cudaSuccess;
   LQSGD_DISPATCH_RP(rp, (launch_pdl(p_apply_kernel<RP>, nfb, kFactorBlockRows, 0, l.stream, t, fb)));
+  return cudaGetLastError();
+}
+
+cudaError_t launch_p_chol(int rp, const Tables& t, const FactorBlock* fb, int nfb, Launch l) {
+  if (nfb == 0) return cudaSuccess;
+  switch (rp) {
+    case 32: launch_pdl(p_chol_kernel<32>, nfb, 256, 0, l.stream, t, fb); break;
+    case 64: launch_pdl(p_chol_kernel<64>, nfb, 256, 0, l.stream, t, fb); break;
+    default: return cudaErrorInvalidValue;
+  }
   return cudaGetLastError();
 }
 
