@@ -109,6 +109,8 @@ struct Plan {
   std::vector<FactorBlock> fbS;                  // (layer, worker) of the layers orthonormalised by one CTA
   std::vector<FactorBlock> fbC;                  // padded rank >= 32: (layer, worker) whose Cholesky factor a CTA of its own computes
   FactorBlock* d_fbC = nullptr;
+  std::vector<FoldJob> foldP, foldG, foldQ;      // layers with many partial sums: groups summed first (after pass 1, the block Grams, after pass 2)
+  FoldJob *d_foldP = nullptr, *d_foldG = nullptr, *d_foldQ = nullptr;
   std::vector<ExchangeChunk> chP, chQ, chV;
   std::vector<float> thrP, thrQ, deqP, deqQ;
   std::vector<lqsgd_layer_layout> layout;     // by user layer index
@@ -560,6 +562,26 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
     L.Qw = (L.nrb == 1) ? L.Qpart : a.take<float>((size_t)W * mt.m * RP);
     L.gram_part = a.take<double>((size_t)W * L.npb * RP * RP);
     L.chol = RP >= kCholSplitRP ? a.take<double>((size_t)W * (RP * RP + 2 * RP)) : nullptr;
+    // many partial sums: folded in groups first (fold_kernel), the steps then add the groups' sums
+    auto fold = [&](std::vector<FoldJob>& jobs, const void* src, int nparts, size_t plane, bool dbl, int& nsum) -> const void* {
+      nsum = nparts;
+      if (p.resident || nparts <= kFoldAbove) return src;
+      const int ng = ceil_div(nparts, kFoldGroup);
+      const size_t esz = dbl ? sizeof(double) : sizeof(float);
+      unsigned char* dst = dbl ? reinterpret_cast<unsigned char*>(a.take<double>((size_t)W * ng * plane))
+                               : reinterpret_cast<unsigned char*>(a.take<float>((size_t)W * ng * plane));
+      for (int w = 0; w < W; ++w)
+        for (int g = 0; g < ng; ++g)
+          for (size_t e0 = 0; e0 < plane; e0 += kFoldElems)
+            jobs.push_back({static_cast<const unsigned char*>(src) + ((size_t)w * nparts + (size_t)g * kFoldGroup) * plane * esz,
+                            dst + ((size_t)w * ng + g) * plane * esz, (uint32_t)plane, (uint32_t)e0,
+                            (uint16_t)std::min(kFoldGroup, nparts - g * kFoldGroup), (uint16_t)(dbl ? 1 : 0), 0u});
+      nsum = ng;
+      return dst;
+    };
+    L.Psum = static_cast<const float*>(fold(p.foldP, L.Ppart, L.ncc, (size_t)mt.n * RP, false, L.nps));
+    L.Qsum = static_cast<const float*>(fold(p.foldQ, L.Qpart, L.nrb, (size_t)mt.m * RP, false, L.nqs));
+    L.gram_sum = static_cast<const double*>(fold(p.foldG, L.gram_part, L.npb, (size_t)RP * RP, true, L.ngs));
     L.maxp = a.take<float>((size_t)W * L.npb * (colscales ? RP : 1));
     L.maxq = a.take<float>((size_t)W * L.nqb * (colscales ? RP : 1));
     L.scales = a.take<float>(2 * (size_t)RP);
@@ -701,6 +723,9 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   p.d_fbQ = a.take<FactorBlock>(p.fbQ.size());
   p.d_fbS = a.take<FactorBlock>(p.fbS.size());
   p.d_fbC = a.take<FactorBlock>(p.fbC.size());
+  p.d_foldP = a.take<FoldJob>(p.foldP.size());
+  p.d_foldG = a.take<FoldJob>(p.foldG.size());
+  p.d_foldQ = a.take<FoldJob>(p.foldQ.size());
   p.d_chP = a.take<ExchangeChunk>(p.chP.size());
   p.d_chQ = a.take<ExchangeChunk>(p.chQ.size());
   p.d_chV = a.take<ExchangeChunk>(p.chV.size());
@@ -884,6 +909,9 @@ int lqsgd_create(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
   CK(up(p.d_fbQ, p.fbQ.data(), p.fbQ.size() * sizeof(FactorBlock)));
   CK(up(p.d_fbS, p.fbS.data(), p.fbS.size() * sizeof(FactorBlock)));
   CK(up(p.d_fbC, p.fbC.data(), p.fbC.size() * sizeof(FactorBlock)));
+  CK(up(p.d_foldP, p.foldP.data(), p.foldP.size() * sizeof(FoldJob)));
+  CK(up(p.d_foldG, p.foldG.data(), p.foldG.size() * sizeof(FoldJob)));
+  CK(up(p.d_foldQ, p.foldQ.data(), p.foldQ.size() * sizeof(FoldJob)));
   CK(up(p.d_chP, p.chP.data(), p.chP.size() * sizeof(ExchangeChunk)));
   CK(up(p.d_chQ, p.chQ.data(), p.chQ.size() * sizeof(ExchangeChunk)));
   CK(up(p.d_chV, p.chV.data(), p.chV.size() * sizeof(ExchangeChunk)));
@@ -991,7 +1019,8 @@ int lqsgd_launches_per_step(const lqsgd_ctx* ctx, int32_t* out) {
   const int pass3 = (p.tiles3.empty() ? 0 : 1) + (p.stiles3.empty() ? 0 : 1) + (p.tctiles3.empty() ? 0 : 1);
   const int iters = std::max(1, ctx->cfg.power_iters);
   const int orth = (p.fbS.empty() ? 0 : 1) + (p.fbP.empty() ? 0 : 2) + (p.fbC.empty() ? 0 : 1);   // one CTA per small layer / Gram (+ Cholesky) + apply
-  *out = iters * ((p.mats.empty() ? 0 : orth + 3) + pass1 + pass2) + pass3 + ((p.chV.empty() || vectors_ride(ctx)) ? 0 : 1);
+  const int folds = (p.foldP.empty() ? 0 : 1) + (p.foldG.empty() ? 0 : 1) + (p.foldQ.empty() ? 0 : 1);
+  *out = iters * ((p.mats.empty() ? 0 : orth + 3 + folds) + pass1 + pass2) + pass3 + ((p.chV.empty() || vectors_ride(ctx)) ? 0 : 1);
   return LQSGD_OK;
 }
 
@@ -1152,8 +1181,10 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
       }
       PHASE_MARK(1);
       if (nm) {
+        CK(launch_fold(p.d_foldP, (int)p.foldP.size(), {st, 0}));
         CK(launch_p_orth_small(RP, t, p.d_fbS, (int)p.fbS.size(), {st, 0}));
         CK(launch_p_reduce_gram(RP, t, p.d_fbP, (int)p.fbP.size(), {st, 0}));
+        CK(launch_fold(p.d_foldG, (int)p.foldG.size(), {st, 0}));
         if (RP >= kCholSplitRP) CK(launch_p_chol(RP, t, p.d_fbC, (int)p.fbC.size(), {st, 0}));
         CK(launch_p_apply(RP, t, p.d_fbP, (int)p.fbP.size(), {st, 0}));
         if (split) CK(launch_scale_reduce(RP, t, 0, p.d_xscales, (int)nm, {st, 0}));
@@ -1172,6 +1203,7 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
       }
       PHASE_MARK(3);
       if (nm) {
+        CK(launch_fold(p.d_foldQ, (int)p.foldQ.size(), {st, 0}));
         CK(launch_q_reduce(RP, t, p.d_fbQ, (int)p.fbQ.size(), {st, 0}));
         if (split) CK(launch_scale_reduce(RP, t, 1, p.d_xscales, (int)nm, {st, 0}));
       }

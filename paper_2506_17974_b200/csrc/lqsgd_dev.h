@@ -44,6 +44,28 @@ struct LayerDev {
   float* maxq;                // [W][nqb] (or [W][nqb][RP])
   float* scales;              // [2 RP]: s_P at [0], s_Q at [1]; with column scales s_P[j] at [j], s_Q[j] at [RP + j]
   uint64_t pay_scale_off, pay_p_off, pay_q_off;   // byte offsets inside one worker's payload
+  // What the steps after a pass add up.  A layer with many partial sums (more than kFoldAbove) has them summed in
+  // groups of kFoldGroup first, by many CTAs (fold_kernel); the step then adds the groups' sums, in order.
+  const float* Psum;          // [W][nps][n][RP]: Ppart (nps = ncc) or the folded partials
+  const float* Qsum;          // [W][nqs][m][RP]: Qpart (nqs = nrb) or the folded partials
+  const double* gram_sum;     // [W][ngs][RP*RP]: gram_part (ngs = npb) or the folded block Grams
+  int32_t nps, nqs, ngs;
+  int32_t pad_;
+};
+
+constexpr int kFoldAbove = 64;     // partial sums per layer and worker above which they are folded first
+constexpr int kFoldGroup = 32;     // partial sums per fold group
+constexpr int kFoldElems = 256;    // elements of a plane per CTA of the fold kernel
+
+// One CTA of the fold kernel: dst[e] = src[e] + src[plane + e] + ... (count planes, in order), e0 <= e < e0 + kFoldElems.
+struct FoldJob {
+  const void* src;            // the group's first plane
+  void* dst;
+  uint32_t plane;             // elements per plane
+  uint32_t e0;
+  uint16_t count;             // planes in this group (1..kFoldGroup)
+  uint16_t is_double;         // 0: float planes, 1: double planes
+  uint32_t pad_;
 };
 
 // One 1-D tensor.
@@ -178,6 +200,7 @@ cudaError_t launch_p_apply(int RP, const Tables& t, const FactorBlock* fb, int n
 // every CTA of p_apply (at rank 64 the factorisation is the long part); fb lists one entry per (layer, worker)
 constexpr int kCholSplitRP = 32;
 cudaError_t launch_p_chol(int RP, const Tables& t, const FactorBlock* fb, int nfb, Launch l);
+cudaError_t launch_fold(const FoldJob* jobs, int njobs, Launch l);
 // Orthonormalize in one launch for layers of at most kOrthSmallMaxRows rows at RP <= 8: one CTA per (layer, worker)
 constexpr int kOrthSmallMaxRows = 512;
 cudaError_t launch_p_orth_small(int RP, const Tables& t, const FactorBlock* fb, int nfb, Launch l);

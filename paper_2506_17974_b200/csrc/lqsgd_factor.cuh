@@ -82,11 +82,11 @@ __device__ __forceinline__ void p_reduce_gram_body(const Tables& t, const Factor
 #pragma unroll
     for (int j = 0; j < RP; ++j) p[j] = 0.f;
     if (row < n) {
-      const float* src = L.Ppart + ((size_t)fb.worker * L.ncc * n + row) * RP;
+      const float* src = L.Psum + ((size_t)fb.worker * L.nps * n + row) * RP;
       // the partials' loads go out together (8 at a time); the additions keep the chunk order
       int cc = 0;
       if constexpr (RP <= 8) {
-        for (; cc + 8 <= L.ncc; cc += 8) {
+        for (; cc + 8 <= L.nps; cc += 8) {
           float v[8][RP];
 #pragma unroll
           for (int u = 0; u < 8; ++u) load_contig<RP, COH>(src + (size_t)(cc + u) * n * RP, v[u]);
@@ -96,7 +96,7 @@ __device__ __forceinline__ void p_reduce_gram_body(const Tables& t, const Factor
             for (int j = 0; j < RP; ++j) p[j] += v[u][j];
         }
       }
-      for (; cc < L.ncc; ++cc) {
+      for (; cc < L.nps; ++cc) {
         float v[RP];
         load_contig<RP, COH>(src + (size_t)cc * n * RP, v);
 #pragma unroll
@@ -212,17 +212,17 @@ __device__ __forceinline__ bool cholesky_lower(const LayerDev& L, int worker, Ch
   if constexpr (SEG > 1) {
     if (tid < SEG * RP * RP) {
       const int e = tid % (RP * RP), g = tid / (RP * RP);
-      const double* gp = L.gram_part + (size_t)worker * L.npb * (RP * RP) + e;
+      const double* gp = L.gram_sum + (size_t)worker * L.ngs * (RP * RP) + e;
       double s = 0.0;
       int b = g;
-      for (; b + 7 * SEG < L.npb; b += 8 * SEG) {
+      for (; b + 7 * SEG < L.ngs; b += 8 * SEG) {
         double x[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) x[u] = ld_in<COH>(gp + (size_t)(b + u * SEG) * (RP * RP));
 #pragma unroll
         for (int u = 0; u < 8; ++u) s += x[u];
       }
-      for (; b < L.npb; b += SEG) s += ld_in<COH>(gp + (size_t)b * (RP * RP));
+      for (; b < L.ngs; b += SEG) s += ld_in<COH>(gp + (size_t)b * (RP * RP));
       C.segsum[g][e] = s;
     }
     __syncthreads();
@@ -234,17 +234,17 @@ __device__ __forceinline__ bool cholesky_lower(const LayerDev& L, int worker, Ch
     }
   } else {
     for (int e = tid; e < RP * RP; e += NT) {
-      const double* gp = L.gram_part + (size_t)worker * L.npb * (RP * RP) + e;
+      const double* gp = L.gram_sum + (size_t)worker * L.ngs * (RP * RP) + e;
       double s = 0.0;
       int b = 0;
-      for (; b + 8 <= L.npb; b += 8) {        // eight loads in flight, additions in block order
+      for (; b + 8 <= L.ngs; b += 8) {        // eight loads in flight, additions in block order
         double x[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) x[u] = ld_in<COH>(gp + (size_t)(b + u) * (RP * RP));
 #pragma unroll
         for (int u = 0; u < 8; ++u) s += x[u];
       }
-      for (; b < L.npb; ++b) s += ld_in<COH>(gp + (size_t)b * (RP * RP));
+      for (; b < L.ngs; ++b) s += ld_in<COH>(gp + (size_t)b * (RP * RP));
       C.A[e / RP][e % RP] = s;
     }
   }
@@ -268,17 +268,17 @@ __device__ __forceinline__ void p_chol_body(const Tables& t, const FactorBlock f
   const LayerDev& L = t.layers[fb.layer];
   const int r = L.r;
   for (int e = tid; e < RP * RP; e += NT) {
-    const double* gp = L.gram_part + (size_t)fb.worker * L.npb * (RP * RP) + e;
+    const double* gp = L.gram_sum + (size_t)fb.worker * L.ngs * (RP * RP) + e;
     double s = 0.0;
     int b = 0;
-    for (; b + 8 <= L.npb; b += 8) {        // eight loads in flight, additions in block order
+    for (; b + 8 <= L.ngs; b += 8) {        // eight loads in flight, additions in block order
       double x[8];
 #pragma unroll
       for (int u = 0; u < 8; ++u) x[u] = ld_in<COH>(gp + (size_t)(b + u) * (RP * RP));
 #pragma unroll
       for (int u = 0; u < 8; ++u) s += x[u];
     }
-    for (; b < L.npb; ++b) s += ld_in<COH>(gp + (size_t)b * (RP * RP));
+    for (; b < L.ngs; ++b) s += ld_in<COH>(gp + (size_t)b * (RP * RP));
     S.A[e / RP][e % RP] = s;
   }
   __syncthreads();
@@ -421,8 +421,8 @@ __device__ __forceinline__ void p_orth_small_body(const Tables& t, const FactorB
 #pragma unroll
   for (int j = 0; j < RP; ++j) p[j] = 0.f;
   if (row < n) {
-    const float* src = L.Ppart + ((size_t)fb.worker * L.ncc * n + row) * RP;
-    for (int cc = 0; cc < L.ncc; ++cc) {
+    const float* src = L.Psum + ((size_t)fb.worker * L.nps * n + row) * RP;
+    for (int cc = 0; cc < L.nps; ++cc) {
       float v[RP];
       load_contig<RP, COH>(src + (size_t)cc * n * RP, v);
 #pragma unroll
@@ -506,7 +506,7 @@ __device__ __forceinline__ void q_reduce_body(const Tables& t, const FactorBlock
   constexpr int TPR = RP / V;               // items per row: 1, 2, 4 or 8 (divides the block size and 32)
   auto& S = *static_cast<QReduceSmem<RP, NT>*>(smem);
   const LayerDev& L = t.layers[fb.layer];
-  const int m = L.m, nrb = L.nrb;
+  const int m = L.m, nrb = L.nqs;
   const size_t plane = (size_t)m * RP;      // floats of one partial
   float cmax[V];
 #pragma unroll
@@ -516,7 +516,7 @@ __device__ __forceinline__ void q_reduce_body(const Tables& t, const FactorBlock
     const int row = fb.blk * kFactorBlockRows + item / TPR;
     if (row >= m) break;
     const size_t off = (size_t)row * RP + (size_t)(item % TPR) * V;
-    const float* src = L.Qpart + (size_t)fb.worker * nrb * plane + off;
+    const float* src = L.Qsum + (size_t)fb.worker * nrb * plane + off;
     float q[V];
 #pragma unroll
     for (int v = 0; v < V; ++v) q[v] = 0.f;
@@ -536,7 +536,7 @@ __device__ __forceinline__ void q_reduce_body(const Tables& t, const FactorBlock
 #pragma unroll
       for (int v = 0; v < V; ++v) q[v] += x[v];
     }
-    if (nrb > 1) store_contig<V>(L.Qw + (size_t)fb.worker * plane + off, q);
+    if (L.nrb > 1) store_contig<V>(L.Qw + (size_t)fb.worker * plane + off, q);
 #pragma unroll
     for (int v = 0; v < V; ++v) {
       cmax[v] = fmaxf(cmax[v], fabsf(q[v]));

@@ -494,6 +494,36 @@ p_chol_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
   p_chol_body<RP, 256, false>(t, fbs[blockIdx.x], threadIdx.x, smem);
 }
 
+// Many partial sums per layer (a very tall or very wide layer): the sums of groups of kFoldGroup consecutive
+// planes, one CTA per group and kFoldElems elements.  Plane order inside a group, eight loads in flight.
+template <typename T>
+__device__ __forceinline__ void fold_planes(const FoldJob& j, int tid) {
+  const T* __restrict__ src = static_cast<const T*>(j.src);
+  T* __restrict__ dst = static_cast<T*>(j.dst);
+  const size_t plane = j.plane;
+  for (uint32_t e = j.e0 + tid; e < j.e0 + kFoldElems && e < j.plane; e += 256) {
+    T s = T(0);
+    int u0 = 0;
+    for (; u0 + 8 <= j.count; u0 += 8) {
+      T x[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) x[u] = __ldg(src + (size_t)(u0 + u) * plane + e);
+#pragma unroll
+      for (int u = 0; u < 8; ++u) s += x[u];
+    }
+    for (; u0 < j.count; ++u0) s += __ldg(src + (size_t)u0 * plane + e);
+    dst[e] = s;
+  }
+}
+
+__global__ void __launch_bounds__(256)
+fold_kernel(const FoldJob* __restrict__ jobs) {
+  pdl_wait();
+  const FoldJob j = jobs[blockIdx.x];
+  if (j.is_double) fold_planes<double>(j, threadIdx.x);
+  else fold_planes<float>(j, threadIdx.x);
+}
+
 template <int RP>
 __global__ void __launch_bounds__(kOrthSmallRows, 3)   // three CTAs per SM: 444 at once, one wave for 21 layers x 16 workers
 p_orth_small_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
@@ -840,6 +870,12 @@ cudaError_t launch_p_chol(int rp, const Tables& t, const FactorBlock* fb, int nf
     case 64: launch_pdl(p_chol_kernel<64>, nfb, 256, 0, l.stream, t, fb); break;
     default: return cudaErrorInvalidValue;
   }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_fold(const FoldJob* jobs, int njobs, Launch l) {
+  if (njobs == 0) return cudaSuccess;
+  launch_pdl(fold_kernel, njobs, 256, 0, l.stream, jobs);
   return cudaGetLastError();
 }
 

@@ -248,42 +248,14 @@ stream_pass1_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
   }
 }
 
-// Rows g, g + ng, ... (RPT of them) of P_bar for this thread's group, fetched from global memory
-// (warp-uniform addresses) BEFORE the wait on the stage, so that the latency hides behind it.
-template <int RP, int RPT>
-__device__ __forceinline__ void load_pbar_rows(const float* __restrict__ Pbar, int first_row, int ng, int rows_left,
-                                               int g, float (&p)[RPT * RP]) {
-#pragma unroll
-  for (int u = 0; u < RPT; ++u) {
-    const int lr = g + u * ng;
-    if (lr < rows_left) {
-      const float* src = Pbar + (size_t)(first_row + lr) * RP;
-      if constexpr (RP % 4 == 0) {
-#pragma unroll
-        for (int j = 0; j < RP / 4; ++j) {
-          const float4 v = __ldg(reinterpret_cast<const float4*>(src) + j);
-          p[u * RP + 4 * j] = v.x; p[u * RP + 4 * j + 1] = v.y; p[u * RP + 4 * j + 2] = v.z; p[u * RP + 4 * j + 3] = v.w;
-        }
-      } else if constexpr (RP == 2) {
-        const float2 v = __ldg(reinterpret_cast<const float2*>(src));
-        p[u * RP] = v.x; p[u * RP + 1] = v.y;
-      } else {
-        p[u * RP] = __ldg(src);
-      }
-    } else {
-#pragma unroll
-      for (int j = 0; j < RP; ++j) p[u * RP + j] = 0.f;
-    }
-  }
-}
-
 // ---------------------------------------------------------------------------------------
 // pass 3: G_hat = P_bar Q_bar^T (Eq. 6), E_w = M_w - G_hat (Eq. 7).  For every block of R rows
 // the workers' M slabs follow one another through the ring; G_hat of the block is formed once
 // (before waiting for the first worker's slab) and kept in registers.
 // ---------------------------------------------------------------------------------------
 template <int RP, int NST, int QPT, int RPT>
-__device__ __forceinline__ bool pass3_consume(const Tables& t, const TileCtx& c, const Ring& ring, float* sM, uint32_t& it) {
+__device__ __forceinline__ bool pass3_consume(const Tables& t, const TileCtx& c, const Ring& ring, float* sM, float* pb_warp,
+                                              uint32_t& it) {
   const int tid = threadIdx.x, lane = tid & 31;
   const LayerDev& L = t.layers[c.layer];
   const StreamGeo geo = c.geo;
@@ -297,12 +269,36 @@ __device__ __forceinline__ bool pass3_consume(const Tables& t, const TileCtx& c,
   float* Gh = Gh0 ? Gh0 + (size_t)c.row0 * m + c.col0 : nullptr;
   float* Wt = Wt0 ? Wt0 + (size_t)c.row0 * m + c.col0 : nullptr;
   const float step = t.lr;
+  // The block's rows of P_bar (RPT rows of RP floats, the same for the whole warp: at most 32 floats) are fetched
+  // one float per lane, as soon as the previous block's last slab has been handed on, and passed round through the
+  // warp's 128 bytes of shared memory: one load per warp and block instead of eight per thread.  (Fetching a whole
+  // block ahead, under the previous block's slabs, is faster still on narrow layers and up to 9 % slower on
+  // matrices of a gigabyte, where the pass runs at the memory's speed and the consumers' pace matters: not kept.)
+  auto fetch_pbar = [&](int sr) -> float {
+    const int u = lane / RP, lr = o.g + u * geo.ng;
+    const bool want = lane < RPT * RP && o.in_group && lr < min(geo.R, c.nrows - sr);
+    return want ? __ldg(Pbar + (size_t)(c.row0 + sr + lr) * RP + (lane % RP)) : 0.f;
+  };
+  float pnext = fetch_pbar(0);
   for (int sr = 0; sr < c.nrows; sr += geo.R) {
     const int rows = min(geo.R, c.nrows - sr);
     float4 gh[RPT * QPT];
     {
       float p[RPT * RP];
-      load_pbar_rows<RP, RPT>(Pbar, c.row0 + sr, geo.ng, o.in_group ? rows : 0, o.g, p);
+      pb_warp[lane] = pnext;
+      __syncwarp();
+#pragma unroll
+      for (int i = 0; i < RPT * RP; i += (RP % 4 == 0 ? 4 : RP)) {
+        if constexpr (RP % 4 == 0) {
+          const float4 v = *reinterpret_cast<const float4*>(pb_warp + i);
+          p[i] = v.x; p[i + 1] = v.y; p[i + 2] = v.z; p[i + 3] = v.w;
+        } else if constexpr (RP == 2) {
+          const float2 v = *reinterpret_cast<const float2*>(pb_warp + i);
+          p[i] = v.x; p[i + 1] = v.y;
+        } else {
+          p[i] = pb_warp[i];
+        }
+      }
 #pragma unroll
       for (int u = 0; u < RPT; ++u) {
         const int lr = o.g + u * geo.ng;
@@ -359,6 +355,7 @@ __device__ __forceinline__ bool pass3_consume(const Tables& t, const TileCtx& c,
       __syncwarp();
       if (lane == 0) mbar_arrive(ring.consumed + s);
     }
+    if (sr + geo.R < c.nrows) pnext = fetch_pbar(sr + geo.R);
   }
   if (*ring.abort_flag) {                      // no common barrier in this pass: each consumer leaves on its own
     if (tid == 0) report_timeout(t, c.layer);
@@ -376,6 +373,7 @@ stream_pass3_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
   uint64_t* bars = reinterpret_cast<uint64_t*>(sM + NST * kSlab);
   volatile int* flags = reinterpret_cast<volatile int*>(bars + 3 * NST);   // abort, wait limit
   const Ring ring{bars, bars + NST, bars + 2 * NST, flags};
+  __shared__ __align__(16) float pb_rows[kConsumerWarps][32];     // a block's rows of P_bar, per consumer warp
   ring_init(ring, NST, true, t.wait_limit);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int W = t.W;
@@ -439,8 +437,8 @@ stream_pass3_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
     if (tiles[ti].pad) { pass3_plain_tile<RP>(t, tiles[ti]); continue; }
     const TileCtx c = tile_ctx<RP>(t, tiles[ti]);
     bool ok;
-    if (c.geo.qpt == 1) ok = pass3_consume<RP, NST, 1, Shape<RP>::RPT_NARROW>(t, c, ring, sM, it);
-    else ok = pass3_consume<RP, NST, Shape<RP>::QPT_WIDE, Shape<RP>::RPT_WIDE>(t, c, ring, sM, it);
+    if (c.geo.qpt == 1) ok = pass3_consume<RP, NST, 1, Shape<RP>::RPT_NARROW>(t, c, ring, sM, pb_rows[warp], it);
+    else ok = pass3_consume<RP, NST, Shape<RP>::QPT_WIDE, Shape<RP>::RPT_WIDE>(t, c, ring, sM, pb_rows[warp], it);
     if (!ok) return;
   }
 }

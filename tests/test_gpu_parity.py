@@ -95,6 +95,31 @@ def test_config4_4096x16384_stage_isolated():
     run_steps(wl.config4(4096, 16384), 1, free_run=False)
 
 
+# Shapes outside the benchmark's families.  The tile sizes come from models of the schedule whose constants were
+# fitted on the ResNet-18 set and the four large layers; these are what a language model brings: an embedding
+# or output table (very tall or very wide), MLP matrices with widths that are no power of two.  Very tall and
+# very wide layers have more than 64 partial sums per layer, which are then added in two levels.
+OTHER_SHAPES = {
+    "embedding_50304x768":      dict(layers=((50304, 768),), rank=8, workers=1),
+    "tall_16500x36_w3":         dict(layers=((16500, 36),), rank=4, workers=3),       # 129 Gram blocks, 100+ row chunks
+    "tall_unaligned_16500x35":  dict(layers=((16500, 35),), rank=2, workers=2),       # register passes (m % 4 != 0)
+    "wide_40x150000_w2":        dict(layers=((40, 150000),), rank=4, workers=2),      # 74 column chunks
+    "wide_600x140000":          dict(layers=((600, 140000),), rank=8, workers=1),     # the same with the two-step Orthonormalize
+    "mlp_4096x11008":           dict(layers=((4096, 11008),), rank=8, workers=1),
+    "mlp_11008x4096":           dict(layers=((11008, 4096),), rank=8, workers=1),
+    "tall_rank16_20000x64_w2":  dict(layers=((20000, 64),), rank=16, workers=2),      # tensor-core passes
+    "mixed_tall_wide_small":    dict(layers=((9000, 128), (128, 9000), (64, 1), (300, 300)), rank=8, workers=2),
+}
+
+
+@pytest.mark.parametrize("name", sorted(OTHER_SHAPES))
+def test_other_shape_families(name):
+    spec = OTHER_SHAPES[name]
+    w = dataclasses.replace(wl.config4(8, 8), name=name, layers=tuple(spec["layers"]), rank=spec["rank"],
+                            workers=spec["workers"], bits=4)
+    run_steps(w, 1, free_run=False)
+
+
 # With one magnitude bit (b = 2) the averaged factors take few distinct values: from the second round on a
 # column of M Q can come out dependent, or a factor all zero.  That is the data, not a fault.
 COARSE_OK = B.STATUS_DEPENDENT_COLUMN | B.STATUS_ZERO_SCALE_P | B.STATUS_ZERO_SCALE_Q
