@@ -87,10 +87,8 @@ struct Plan {
   std::vector<Tile> tiles1, tiles2, tiles3;      // register-path passes
   std::vector<Tile> stiles1, stiles3;            // bulk-copy staged passes 1 and 3
   std::vector<Tile> tctiles2;                    // tensor-core pass 2
-  std::vector<Tile> tctiles1;                    // tensor-core pass 1, grouped by CTA
-  std::vector<int> tcbegin1;                     // [tc_grid + 1]
-  std::vector<Tile> tctiles3;                    // tensor-core pass 3 (all workers per tile), grouped by CTA
-  std::vector<int> tcbegin3;
+  std::vector<Tile> tctiles1;                    // tensor-core pass 1, handed out at run time in this order
+  std::vector<Tile> tctiles3;                    // tensor-core pass 3 (a range of workers per entry), handed out at run time
   int tc_grid = 0;
   std::vector<uint64_t> guards;                  // byte offsets of the guard blocks (LQSGD_FLAG_GUARD_WORDS)
   uint64_t* d_guards = nullptr;
@@ -103,6 +101,7 @@ struct Plan {
   ResTile* d_rtiles = nullptr;
   int* d_rbegin = nullptr;
   uint32_t* d_rsync = nullptr;                   // launch counter + two sets of grid-barrier counters
+  int* d_tcsched = nullptr;                      // tensor-core passes that hand out their tiles at run time
   uint64_t* d_rstamps = nullptr;                 // timeline of the last one-launch round
   std::vector<uint8_t> tcmaps;                   // tensor maps of the tensor-core passes (filled at create)
   std::vector<FactorBlock> fbP, fbQ;             // 128-row blocks of P (layers orthonormalised in two launches) and of Q
@@ -124,9 +123,7 @@ struct Plan {
   Tile *d_stiles1 = nullptr, *d_stiles3 = nullptr;
   Tile* d_tctiles2 = nullptr;
   Tile* d_tctiles1 = nullptr;
-  int* d_tcbegin1 = nullptr;
   Tile* d_tctiles3 = nullptr;
-  int* d_tcbegin3 = nullptr;
   uint8_t* d_tcmaps = nullptr;
   FactorBlock *d_fbP = nullptr, *d_fbQ = nullptr, *d_fbS = nullptr;
   ExchangeChunk *d_chP = nullptr, *d_chQ = nullptr, *d_chV = nullptr;
@@ -144,6 +141,9 @@ struct Plan {
   size_t zero_elems = 0;
   float* d_zero = nullptr;                    // power_iters > 1: zeros, as large as the largest matrix
   void** d_zero_ptrs = nullptr;               // [n_mat * W] pointers to d_zero: the "gradient" of a repeated power step
+  uint8_t* d_gmaps = nullptr;                 // tensor-core passes: [kPtrSets][n_mat * W] tensor maps of the gradients, beside the pointer tables
+  uint8_t* d_zero_gmaps = nullptr;            // [n_mat * W] the same over d_zero
+  bool any_tc = false;
   float* d_stage_g = nullptr;                 // [W][elems_total]
   float* d_stage_ghat = nullptr;              // [elems_total]
   size_t state_begin = 0, state_end = 0;      // byte range to zero at create (E, factors, codes ...)
@@ -548,6 +548,7 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
     L.Q = a.take<float>((size_t)mt.m * RP);
     L.mt = (int)align_up((size_t)mt.m, 4);
     L.tc = tc ? 1 : 0;
+    if (tc) p.any_tc = true;
     L.nt = (int)align_up((size_t)mt.n, 4);
     L.Qt = a.take<float>((size_t)(tc ? 2 : 1) * RP * L.mt);
     L.Pbt = tc ? a.take<float>((size_t)3 * RP * L.nt) : nullptr;
@@ -663,31 +664,31 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   // Pass 2 walks the data in the reverse of pass 1's order and pass 3 again in pass 1's order:
   // each pass starts on what the previous one touched last, which is still in L2.
   std::reverse(p.tiles2.begin(), p.tiles2.end());
-  // The tensor-core kernels deal their tiles round-robin to one CTA per SM: largest first, so the
-  // CTAs finish together.
+  // Tensor-core pass 2 deals its tiles round-robin to one CTA per SM: tallest first, so the CTAs finish together.
   std::stable_sort(p.tctiles2.begin(), p.tctiles2.end(), [](const Tile& x, const Tile& y) { return x.nrows > y.nrows; });
-  // Pass 1: longest tile first to the CTA with the least work so far (a tile costs its column count:
-  // every stage is 128 rows deep whatever the tile's row count), then grouped by CTA.
+  // Pass 1 hands its tiles out at run time: widest first (a tile costs its column count: every stage is 128 rows
+  // deep whatever the tile's row count), so that the short ones fill the end.
   p.tc_grid = sm_count;
-  auto deal = [&](std::vector<Tile>& tiles, std::vector<int>& begin) {
-    std::vector<Tile> sorted = tiles;
-    std::stable_sort(sorted.begin(), sorted.end(), [](const Tile& x, const Tile& y) { return x.ncols > y.ncols; });
-    std::vector<std::vector<Tile>> per(p.tc_grid);
-    std::vector<long> load(p.tc_grid, 0);
-    for (const Tile& tl : sorted) {
-      const int b = (int)(std::min_element(load.begin(), load.end()) - load.begin());
-      per[b].push_back(tl);
-      load[b] += ceil_div(tl.ncols, 32);
-    }
-    tiles.clear();
-    begin.assign(p.tc_grid + 1, 0);
-    for (int b = 0; b < p.tc_grid; ++b) {
-      tiles.insert(tiles.end(), per[b].begin(), per[b].end());
-      begin[b + 1] = (int)tiles.size();
-    }
-  };
-  deal(p.tctiles1, p.tcbegin1);
-  deal(p.tctiles3, p.tcbegin3);     // same cost model: pieces of 32 columns (times W for every tile alike)
+  std::stable_sort(p.tctiles1.begin(), p.tctiles1.end(), [](const Tile& x, const Tile& y) { return x.ncols > y.ncols; });
+  // Pass 3 hands its tiles out at run time, in table order (CTAs that walk neighbouring tiles at the same time are
+  // what the memory likes: contiguous shares of the list per CTA ran 11 % slower).  A tile with all its workers is
+  // a megabyte and more, too coarse a unit for an even finish: its workers are cut into ranges [worker, part) so
+  // that there are about a dozen units per SM; every unit forms the tile's G_hat itself (the factors are small),
+  // the one that has worker 0 writes it.
+  {
+    const std::vector<Tile> in = p.tctiles3;
+    const size_t want_units = (size_t)12 * p.tc_grid;
+    const int per = (int)std::max<size_t>(1, std::min<size_t>((size_t)W, in.size() * (size_t)W / std::max<size_t>(1, want_units)));
+    const int nr = ceil_div(W, per);             // ranges per tile, of nearly equal size
+    p.tctiles3.clear();
+    for (const Tile& tl : in)
+      for (int r = 0; r < nr; ++r) {
+        Tile e = tl;
+        e.worker = (int)((long)W * r / nr);
+        e.part = (int)((long)W * (r + 1) / nr);
+        p.tctiles3.push_back(e);
+      }
+  }
   p.d_status = a.take<uint32_t>(p.mats.size());
   p.d_payload = a.take<uint8_t>((size_t)W * p.payload_stride);
   p.xscale_ns = colscales ? RP : 1;
@@ -699,6 +700,7 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   p.d_xsend[0] = a.take<uint8_t>((size_t)W * p.region_bytes[0]);
   p.d_xsend[1] = a.take<uint8_t>((size_t)W * p.region_bytes[1]);
   p.d_rsync = a.take<uint32_t>(1 + 2 * kResBarriers);
+  p.d_tcsched = a.take<int>(2 * 3);              // per tensor-core pass: draw counter, CTAs that have left (zero between launches)
   p.d_rstamps = a.take<uint64_t>(kResStamps + 1);
   p.state_end = a.off;
 
@@ -713,9 +715,7 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   p.d_stiles3 = a.take<Tile>(p.stiles3.size());
   p.d_tctiles2 = a.take<Tile>(p.tctiles2.size());
   p.d_tctiles1 = a.take<Tile>(p.tctiles1.size());
-  p.d_tcbegin1 = a.take<int>(p.tcbegin1.size());
   p.d_tctiles3 = a.take<Tile>(p.tctiles3.size());
-  p.d_tcbegin3 = a.take<int>(p.tcbegin3.size());
   p.d_tcmaps = a.take<uint8_t>(p.mats.size() * kTcMapsPerLayer * kTcMapBytes);
   p.d_rtiles = a.take<ResTile>(p.rtiles.size());
   p.d_rbegin = a.take<int>(p.rbegin.size());
@@ -734,11 +734,13 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
   p.d_deqP = a.take<float>(p.deqP.size());
   p.d_deqQ = a.take<float>(p.deqQ.size());
   p.d_ptrs = a.take<void*>(kPtrSets * (p.mats.size() + p.vecs.size()) * (size_t)(W + 2));
+  if (p.any_tc) p.d_gmaps = a.take<uint8_t>(kPtrSets * p.mats.size() * (size_t)W * kTcMapBytes);
   if (cfg.power_iters > 1) {
     size_t big = 0;
     for (auto& mt : p.mats) big = std::max(big, (size_t)mt.n * mt.m);
     p.zero_elems = big;
     p.d_zero_ptrs = a.take<void*>(p.mats.size() * (size_t)W);
+    if (p.any_tc) p.d_zero_gmaps = a.take<uint8_t>(p.mats.size() * (size_t)W * kTcMapBytes);
     p.d_zero = a.take<float>(big);
   }
   if (cfg.flags & LQSGD_FLAG_HOST_STAGING) {
@@ -892,9 +894,7 @@ int lqsgd_create(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
   CK(up(p.d_stiles3, p.stiles3.data(), p.stiles3.size() * sizeof(Tile)));
   CK(up(p.d_tctiles2, p.tctiles2.data(), p.tctiles2.size() * sizeof(Tile)));
   CK(up(p.d_tctiles1, p.tctiles1.data(), p.tctiles1.size() * sizeof(Tile)));
-  CK(up(p.d_tcbegin1, p.tcbegin1.data(), p.tcbegin1.size() * sizeof(int)));
   CK(up(p.d_tctiles3, p.tctiles3.data(), p.tctiles3.size() * sizeof(Tile)));
-  CK(up(p.d_tcbegin3, p.tcbegin3.data(), p.tcbegin3.size() * sizeof(int)));
   p.tcmaps.resize(p.mats.size() * kTcMapsPerLayer * kTcMapBytes + 1);
   rc = tc_encode_maps(p.layers.data(), (int)p.layers.size(), p.W, p.RP, p.tcmaps.data());
   if (rc != LQSGD_OK) { g_cuda_error = "cuTensorMapEncodeTiled failed or is not available"; return rc; }
@@ -923,6 +923,12 @@ int lqsgd_create(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config
     CK(cudaMemset(p.d_zero, 0, p.zero_elems * sizeof(float)));
     std::vector<void*> zp(p.mats.size() * (size_t)p.W, p.d_zero);
     CK(up(p.d_zero_ptrs, zp.data(), zp.size() * sizeof(void*)));
+    if (p.d_zero_gmaps) {
+      std::vector<uint8_t> gm(zp.size() * kTcMapBytes);
+      rc = tc_encode_grad_maps(p.layers.data(), (int)p.layers.size(), p.W, zp.data(), gm.data());
+      if (rc != LQSGD_OK) { g_cuda_error = "cuTensorMapEncodeTiled failed or is not available"; return rc; }
+      CK(up(p.d_zero_gmaps, gm.data(), gm.size()));
+    }
   }
   // Q_0
   std::vector<float> q0;
@@ -1087,6 +1093,15 @@ static int prepare_step(lqsgd_ctx* c, const float* const* grads, float* const* g
     // returning, so the vector may go afterwards
     CK(cudaMemcpyAsync(p.d_ptrs + (size_t)slot * c->ptr_count, ptrs.data(), ptrs.size() * sizeof(void*),
                        cudaMemcpyHostToDevice, st));
+    if (p.d_gmaps) {
+      // the tensor-core pass 1 reads the gradients through tensor maps: encoded once per pointer set, kept with the table
+      std::vector<uint8_t> gm(nm * (size_t)W * kTcMapBytes);
+      if (tc_encode_grad_maps(p.layers.data(), (int)nm, W, ptrs.data(), gm.data()) != LQSGD_OK) {
+        g_cuda_error = "cuTensorMapEncodeTiled failed on a gradient tensor";
+        return LQSGD_ERR_CUDA;
+      }
+      CK(cudaMemcpyAsync(p.d_gmaps + (size_t)slot * gm.size(), gm.data(), gm.size(), cudaMemcpyHostToDevice, st));
+    }
     c->ptr_sets[slot] = ptrs;
   }
   c->ptr_used[slot] = c->step_counter;
@@ -1102,6 +1117,7 @@ static int prepare_step(lqsgd_ctx* c, const float* const* grads, float* const* g
   t.payload = p.d_payload;
   t.payload_stride = p.payload_stride;
   t.status = p.d_status;
+  t.gmaps = p.d_gmaps ? p.d_gmaps + (size_t)slot * nm * (size_t)W * kTcMapBytes : nullptr;
   t.W = W;
   t.col_scales = (c->cfg.flags & LQSGD_FLAG_COLUMN_SCALES) ? 1 : 0;
   t.clear_status = 0;
@@ -1125,7 +1141,7 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
   Plan& p = c->plan;
   // a repeated power step (power_iters > 1) runs pass 1 on M itself: its "gradient" is the zero buffer
   Tables t = c->tables;
-  if (repeat) t.grads = reinterpret_cast<const float* const*>(p.d_zero_ptrs);
+  if (repeat) { t.grads = reinterpret_cast<const float* const*>(p.d_zero_ptrs); t.gmaps = p.d_zero_gmaps; }
   const int W = p.W, RP = p.RP;
   const size_t nm = p.mats.size(), nv = p.vecs.size();
   const size_t vbase = nm * (W + 2);
@@ -1176,7 +1192,7 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
         CK(launch_pass1(RP, reg1 ? first : rest, p.d_tiles1, (int)p.tiles1.size(), {st, c->grid1}));
         CK(launch_stream_pass1(RP, (!reg1 && st1) ? first : rest, p.d_stiles1, (int)p.stiles1.size(),
                                {st, (int)std::min<size_t>(p.stiles1.size(), c->sm_count)}));
-        CK(launch_tc_pass1(RP, (!reg1 && !st1) ? first : rest, p.d_tctiles1, (int)p.tctiles1.size(), p.d_tcbegin1, p.d_tcmaps,
+        CK(launch_tc_pass1(RP, (!reg1 && !st1) ? first : rest, p.d_tctiles1, (int)p.tctiles1.size(), p.d_tcsched, p.d_tcmaps,
                            {st, p.tc_grid}));
       }
       PHASE_MARK(1);
@@ -1219,7 +1235,7 @@ static int run_segment(lqsgd_ctx* c, int seg, bool split, const void* gathered, 
       if (nm) {
         CK(launch_pass3(RP, t, p.d_tiles3, (int)p.tiles3.size(), {st, c->grid3}));
         CK(launch_stream_pass3(RP, t, p.d_stiles3, (int)p.stiles3.size(), {st, (int)std::min<size_t>(p.stiles3.size(), c->sm_count)}));
-        CK(launch_tc_pass3(RP, t, p.d_tctiles3, (int)p.tctiles3.size(), p.d_tcbegin3, p.d_tcmaps, {st, p.tc_grid}));
+        CK(launch_tc_pass3(RP, t, p.d_tctiles3, (int)p.tctiles3.size(), p.d_tcsched + 4, p.d_tcmaps, {st, p.tc_grid}));
       }
       if (split && nv) CK(launch_vectors_finish(vj, {st, 0}));     // the shares were summed over the ranks meanwhile
       PHASE_MARK(5);

@@ -106,6 +106,7 @@ struct Tables {
   uint8_t* payload;           // [W][payload_stride]
   uint64_t payload_stride;
   uint32_t* status;           // [n_mat]
+  const uint8_t* gmaps;       // [n_mat][W] tensor maps of the gradients (layers on the tensor-core passes), or null
   int32_t W;
   int32_t col_scales;         // 1: one quantiser scale per factor column (variant), 0: one per factor
   int32_t clear_status;       // > 0 only in the round's first pass-1 launch: that many status words are zeroed by CTA 0
@@ -302,11 +303,14 @@ constexpr int kTcPass1Cols = 1152;   // most columns of a pass-1 tile (multiple 
 constexpr int kTcMapBytes = 128;
 constexpr int kTcRowChunk = 4096;    // most rows of a layer one pass-2 tile sums over (multiple of 64)
 int tc_encode_maps(const LayerDev* host_layers, int n_layers, int W, int RP, void* host_maps_out);   // 0 or LQSGD_ERR_CUDA
+// one map per (layer, worker) over the caller's gradients (grads: [n_layers][W] device pointers); out: [n_layers][W] maps
+int tc_encode_grad_maps(const LayerDev* host_layers, int n_layers, int W, const void* const* grads, void* host_maps_out);
 cudaError_t launch_tc_pass2(int RP, const Tables& t, const Tile* tiles, int ntiles, const void* maps, Launch l);
-// tiles are grouped by CTA: CTA b takes tiles [cta_begin[b], cta_begin[b + 1]); l.grid CTAs
-cudaError_t launch_tc_pass1(int RP, const Tables& t, const Tile* tiles, int ntiles, const int* cta_begin, const void* maps,
+// passes 1 and 3 hand their tiles out at run time, in list order: sched = {draw counter, CTAs that have left}, zero before
+// the first launch (the kernels leave it zero); l.grid CTAs
+cudaError_t launch_tc_pass1(int RP, const Tables& t, const Tile* tiles, int ntiles, int* sched, const void* maps,
                             Launch l);
-cudaError_t launch_tc_pass3(int RP, const Tables& t, const Tile* tiles, int ntiles, const int* cta_begin, const void* maps,
+cudaError_t launch_tc_pass3(int RP, const Tables& t, const Tile* tiles, int ntiles, int* sched, const void* maps,
                             Launch l);
 // One-launch round (lqsgd_resident.cu) for sets whose M fits in the SMs' shared memory: one cooperative grid,
 // one CTA of kResThreads threads per SM, tiles of M resident from pass 1 to pass 3, grid barriers between the steps.

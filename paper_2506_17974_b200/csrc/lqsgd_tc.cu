@@ -114,6 +114,59 @@ __device__ __forceinline__ void drain(uint64_t* bar, uint32_t parity, volatile i
   for (uint32_t i = 0; i < limit && !mbar_try(bar, parity); ++i) {}
 }
 
+// ---------------------------------------------------------------------------------------
+// Tiles handed out at run time (passes 1 and 3).  The SMs do not stream equally fast (two dies, memory partitions
+// nearer or farther: 15 % between the quickest and the slowest in these passes), so equal shares dealt in
+// advance leave the quick ones idle at the end.  CTA b starts on tile b; after that the loader thread draws the
+// next index from a counter in global memory (asked for one tile ahead, so that the answer is there when it is
+// needed) and announces it to the CTA's other roles through a small queue in shared memory.  Which CTA takes a
+// tile does not change a result: every tile writes its own places.  The last CTA to leave puts the counter back
+// to zero, so the next launch (or replay of a captured graph) finds it ready.
+// ---------------------------------------------------------------------------------------
+constexpr int kTqDepth = 4;
+constexpr int kTqEnd = -1, kTqAbort = -2;
+struct TileQueue {
+  uint64_t* full;        // [kTqDepth] entry announced
+  uint64_t* empty;       // [kTqDepth] every reader has taken the entry
+  volatile int* idx;     // [kTqDepth] tile index, or kTqEnd
+};
+// the loader thread announces entry number seq
+__device__ __forceinline__ bool tq_put(const TileQueue& q, uint32_t seq, int tile, volatile int* abort_flag) {
+  const int s = seq % kTqDepth;
+  if (!mbar_wait(q.empty + s, ((seq / kTqDepth) & 1) ^ 1, abort_flag)) return false;
+  q.idx[s] = tile;
+  mbar_arrive(q.full + s);
+  return true;
+}
+// a reader thread takes entry number seq: the tile index, kTqEnd, or kTqAbort when a wait gave up
+__device__ __forceinline__ int tq_take(const TileQueue& q, uint32_t seq, volatile int* abort_flag) {
+  const int s = seq % kTqDepth;
+  if (!mbar_wait(q.full + s, (seq / kTqDepth) & 1, abort_flag)) return kTqAbort;
+  const int v = q.idx[s];
+  mbar_arrive(q.empty + s);
+  return v;
+}
+// a reader warp: lane 0 takes the entry, the warp learns it
+__device__ __forceinline__ int tq_take_warp(const TileQueue& q, uint32_t seq, volatile int* abort_flag, int lane) {
+  int v = 0;
+  if (lane == 0) v = tq_take(q, seq, abort_flag);
+  return __shfl_sync(0xffffffffu, v, 0);
+}
+// the loader thread's draw: tiles gridDim.x, gridDim.x + 1, ... in the order asked for
+__device__ __forceinline__ int tq_draw(int* sched, int ntiles) {
+  const int v = (int)gridDim.x + atomicAdd(sched, 1);
+  return v < ntiles ? v : kTqEnd;
+}
+// at the very end of the kernel, one thread per CTA: the last CTA to leave readies the counter for the next launch
+__device__ __forceinline__ void tq_leave(int* sched) {
+  __threadfence();
+  if (atomicAdd(sched + 1, 1) == (int)gridDim.x - 1) {
+    sched[0] = 0;
+    sched[1] = 0;
+    __threadfence();
+  }
+}
+
 // Stages a tile takes: its rows in pieces of 32, rounded up to whole operand slots (a piece past
 // the layer's last row reads as zeros and costs no memory traffic).
 __device__ __forceinline__ int tile_stages(int nrows) {
@@ -309,6 +362,11 @@ tc_pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, const uint
         if ((int)(kc % kTcGroups) != g) continue;
         const int s = kc % S::kMStages;
         const uint32_t slot = kc / kTcPair, ab = slot % S::kAB;
+        // The slot's previous piece may have been another group's.  A barrier tells its phases apart by parity
+        // alone, so this group first makes sure that piece has been taken (then its copy had landed and the
+        // barrier below is in this piece's phase); asked before that, the barrier would answer for the phase
+        // before, and pieces do not always land in the order they were asked for.
+        if (!warp_wait(m_empty + s, ((kc / S::kMStages) & 1) ^ 1, abort_flag, lane)) { ok = false; break; }
         if (!warp_wait(m_full + s, (kc / S::kMStages) & 1, abort_flag, lane)) { ok = false; break; }
         const float* src = mring + (size_t)s * (kTcMBytes / 4) + 32 * q + lane;
         uint32_t v[32];
@@ -353,9 +411,10 @@ tc_pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, const uint
 // two halves of D.
 //
 // Stage of the ring: the 128 x 32 piece of E by TMA (128-byte swizzle: a thread reading its own
-// row touches every bank once per quarter warp) and the same piece of G by cp.async from the
-// caller's tensor (16-byte granules placed at the swizzled positions; rows and columns past the
-// layer are zero-filled).  A consumer thread adds its row of the two pieces, puts m back into the
+// row touches every bank once per quarter warp) and the same piece of G, also by TMA, through a
+// tensor map of the caller's tensor that the host encodes when it first meets a set of gradient
+// pointers (kept beside the pointer table; rows and columns past the layer are zero-filled).  A warp
+// that fetched G with cp.async instead spent two thirds of the pass issuing those copies.  A consumer thread adds its row of the two pieces, puts m back into the
 // E piece (a storer thread sends it to global memory with a TMA tensor store) and writes hi and
 // lo to TMEM.
 // ---------------------------------------------------------------------------------------
@@ -396,27 +455,29 @@ struct Pass1Cfg {
   static constexpr int kACol0 = 2 * kDStride;
   static constexpr int kTmemCols = 512;
   static constexpr uint32_t kBBytes = 2 * RP * 128;                      // Q_hi rows, then Q_lo rows, 32 columns
-  static constexpr uint32_t kBOff = kT1Stages * 2 * kT1PieceBytes;
+  static constexpr int kStages = kT1Stages;                               // ring of (G, E) pieces
+  static constexpr uint32_t kBOff = kStages * 2 * kT1PieceBytes;
   static constexpr uint32_t kBarOff = kBOff + kT1AB * kBBytes;
-  static constexpr int kBars = 3 * kT1Stages + 2 * kT1AB + 2 + 2 + 1;
-  static constexpr uint32_t kTotal = kBarOff + kBars * 8 + 16 + 1024;
+  static constexpr int kBars = 3 * kStages + 2 * kT1AB + 2 + 2 + 1 + 2 * kTqDepth;   // ..., fin, tile queue
+  static constexpr uint32_t kTotal = kBarOff + kBars * 8 + 16 + 4 * kTqDepth + 1024;
   static_assert(kACol0 + kT1AB * 64 <= 512, "tensor memory");
   static_assert(kBBytes % 1024 == 0, "B stages stay 1024-byte aligned");
   static_assert(kTotal <= 227 * 1024, "shared memory");
-  static_assert(kT1Stages < 2 * kT1AB, "a consumer must not get two turns of the operand ring ahead (see Pass2Cfg)");
+  static_assert(kStages < 2 * kT1AB, "a consumer must not get two turns of the operand ring ahead (see Pass2Cfg)");
 };
 
 template <int RP>
 __global__ void __launch_bounds__(kTcThreads, 1)
-tc_pass1_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict__ cta_begin, const uint8_t* __restrict__ maps) {
+tc_pass1_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, int* __restrict__ sched, const uint8_t* __restrict__ maps) {
   pdl_wait();
   clear_status_words(t);
   using S = Pass1Cfg<RP>;
+  constexpr int kT1Stages = S::kStages;          // this rank's ring depth
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* bring = base + S::kBOff;
   uint64_t* bars = reinterpret_cast<uint64_t*>(base + S::kBarOff);
-  uint64_t* ge_full = bars;                      // [kT1Stages] G (32 cp.async arrivals) and E (TMA) landed
+  uint64_t* ge_full = bars;                      // [kT1Stages] G and E landed
   uint64_t* m_ready = ge_full + kT1Stages;       // [kT1Stages] consumers have put m into the E piece
   uint64_t* ge_empty = m_ready + kT1Stages;      // [kT1Stages] the store of m has read the piece: refill
   uint64_t* ab_full = ge_empty + kT1Stages;      // [kT1AB] A written to TMEM (4 warps) and B landed
@@ -424,16 +485,20 @@ tc_pass1_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
   uint64_t* d_full = ab_empty + kT1AB;           // [2]
   uint64_t* d_empty = d_full + 2;                // [2]
   uint64_t* fin = d_empty + 2;                   // [1]
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(fin + 1);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(fin + 1) + 2;   // after the abort flag and the wait limit
+  uint64_t* q_full = fin + 1;                    // [kTqDepth] tile queue
+  uint64_t* q_empty = q_full + kTqDepth;         // [kTqDepth]
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(q_empty + kTqDepth);
+  uint32_t* tmem_slot = const_cast<uint32_t*>(reinterpret_cast<volatile uint32_t*>(abort_flag)) + 2;   // after the abort flag and the wait limit
+  const TileQueue tq{q_full, q_empty, reinterpret_cast<volatile int*>(tmem_slot + 2)};
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int t_begin = cta_begin[blockIdx.x], t_end = cta_begin[blockIdx.x + 1];
   if (tid == 0) {
-    for (int s = 0; s < kT1Stages; ++s) { mbar_init(ge_full + s, 33); mbar_init(m_ready + s, 4); mbar_init(ge_empty + s, 1); }
+    for (int s = 0; s < kT1Stages; ++s) { mbar_init(ge_full + s, 1); mbar_init(m_ready + s, 4); mbar_init(ge_empty + s, 1); }
     for (int s = 0; s < kT1AB; ++s) { mbar_init(ab_full + s, 5); mbar_init(ab_empty + s, 1); }
     for (int s = 0; s < 2; ++s) { mbar_init(d_full + s, 1); mbar_init(d_empty + s, 4); }
     mbar_init(fin, 1);
+    // readers of the tile queue: B loader, MMA thread, storer, 4 epilogue warps, 12 consumer warps
+    for (int s = 0; s < kTqDepth; ++s) { mbar_init(q_full + s, 1); mbar_init(q_empty + s, 3 + 4 + 4 * kTcGroups); }
     wait_ctl_init(abort_flag, t.wait_limit);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
@@ -450,15 +515,22 @@ tc_pass1_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
   auto e_piece = [&](int s) { return base + (size_t)s * 2 * kT1PieceBytes + kT1PieceBytes; };
 
   if (warp == 0) {
-    // ---- loader: E by TMA (lane 0), G by cp.async (all lanes)
-    uint32_t kc = 0;
+    // ---- loader: the piece of E and the same piece of this worker's G, two tensor copies
+    uint32_t kc = 0, qs = 0;
     bool ok = true;
-    for (int ti = t_begin; ti < t_end && ok; ++ti) {
+    int ti = (int)blockIdx.x < ntiles ? (int)blockIdx.x : kTqEnd;
+    for (;; ++qs) {
+      int put = 1, drawn = kTqEnd;
+      if (lane == 0) {
+        put = tq_put(tq, qs, ti, abort_flag) ? 1 : 0;
+        if (put && ti != kTqEnd) drawn = tq_draw(sched, ntiles);        // the tile after this one: the answer comes meanwhile
+      }
+      if (!__shfl_sync(0xffffffffu, put, 0)) { ok = false; break; }
+      if (ti == kTqEnd) break;
       const Tile tl = tiles[ti];
       const LayerDev& L = t.layers[tl.layer];
       const uint8_t* map = maps + ((size_t)tl.layer * kTcMapsPerLayer + 2) * kTcMapBytes;
-      const float* G = t.grads[(size_t)tl.layer * t.W + tl.worker];
-      const int n = L.n, m = L.m;
+      const uint8_t* gmap = t.gmaps + ((size_t)tl.layer * t.W + tl.worker) * kTcMapBytes;   // this worker's gradient
       const int nk = (tl.ncols + kTcK - 1) / kTcK;
       for (int k = 0; k < nk; ++k, ++kc) {
         const int s = kc % kT1Stages;
@@ -466,34 +538,24 @@ tc_pass1_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
         if (test_skips_stage(t, 1, kc)) continue;     // test support: this piece is not fetched, its waiters give up
         const int c0 = tl.col0 + k * kTcK;
         if (lane == 0) {
-          mbar_arrive_expect_tx(ge_full + s, kT1PieceBytes);
+          mbar_arrive_expect_tx(ge_full + s, 2 * kT1PieceBytes);
           tma_load_3d(e_piece(s), map, c0, tl.row0, tl.worker, ge_full + s);
+          tma_load_2d(g_piece(s), gmap, c0, tl.row0, ge_full + s);
         }
-        // lane = (row within a group of 4, 16-byte granule): per iteration 4 rows further down
-        const int r0 = lane >> 3, c16 = lane & 7, gc = c0 + c16 * 4;
-        const int rows_in = (gc < m) ? n - (tl.row0 + r0) : 0;          // row 4 it + r0 is inside iff 4 it < rows_in
-        const float* src = G + (size_t)(tl.row0 + r0) * m + gc;
-        const uint32_t dst = smem_u32(g_piece(s)) + r0 * 128;
-        const uint32_t sw_even = (uint32_t)(c16 ^ r0) << 4, sw_odd = (uint32_t)(c16 ^ (r0 + 4)) << 4;
-#pragma unroll
-        for (int it = 0; it < 32; ++it) {
-          const bool in = 4 * it < rows_in;
-          asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;"
-                       ::"r"(dst + it * 512 + ((it & 1) ? sw_odd : sw_even)), "l"(in ? src : G), "r"(in ? 16u : 0u) : "memory");
-          src += 4 * (size_t)m;
-        }
-        cp_async_arrive(ge_full + s);
       }
+      if (!ok) break;
+      ti = __shfl_sync(0xffffffffu, drawn, 0);
     }
     if (!ok && lane == 0)
       for (uint32_t it = kc > (uint32_t)kT1Stages ? kc - kT1Stages : 0; it < kc; ++it)
         drain(ge_full + it % kT1Stages, (it / kT1Stages) & 1, abort_flag);
-    asm volatile("cp.async.wait_all;" ::: "memory");
   } else if (warp == 1) {
     // ---- B loader: columns [c0, c0 + 32) of Q^T and of its remainders
     uint32_t kc = 0;
     bool ok = true;
-    for (int ti = t_begin; ti < t_end && ok; ++ti) {
+    for (uint32_t qs = 0; ok; ++qs) {
+      const int ti = tq_take_warp(tq, qs, abort_flag, lane);
+      if (ti < 0) { ok = ti == kTqEnd; break; }
       const Tile tl = tiles[ti];
       const uint8_t* map = maps + ((size_t)tl.layer * kTcMapsPerLayer + 3) * kTcMapBytes;
       const int nk = (tl.ncols + kTcK - 1) / kTcK;
@@ -515,7 +577,9 @@ tc_pass1_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
       bool ok = true;
       const uint32_t idesc2 = tc_idesc_tf32(2 * RP), idesc1 = tc_idesc_tf32(RP);
       const uint64_t bdesc0 = tc_desc_sw128(smem_u32(bring));
-      for (int ti = t_begin; ti < t_end && ok; ++ti, ++tseq) {
+      for (; ok; ++tseq) {
+        const int ti = tq_take(tq, tseq, abort_flag);
+        if (ti < 0) { ok = ti == kTqEnd; break; }
         const int nk = (tiles[ti].ncols + kTcK - 1) / kTcK;
         const uint32_t db = tseq & 1;
         const uint32_t dcol = tmem + db * S::kDStride;
@@ -543,7 +607,9 @@ tc_pass1_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
     // ---- storer: m pieces back to global memory (over E)
     uint32_t kc = 0;
     bool ok = true;
-    for (int ti = t_begin; ti < t_end && ok; ++ti) {
+    for (uint32_t qs = 0; ok; ++qs) {
+      const int ti = tq_take_warp(tq, qs, abort_flag, lane);
+      if (ti < 0) { ok = ti == kTqEnd; break; }
       const Tile tl = tiles[ti];
       const uint8_t* map = maps + ((size_t)tl.layer * kTcMapsPerLayer + 2) * kTcMapBytes;
       const int nk = (tl.ncols + kTcK - 1) / kTcK;
@@ -571,7 +637,9 @@ tc_pass1_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
     // ---- epilogue: P_part[row][j] = D[row][j] + D[row][RP + j]
     uint32_t tseq = 0;
     const int q = warp & 3;
-    for (int ti = t_begin; ti < t_end; ++ti, ++tseq) {
+    for (;; ++tseq) {
+      const int ti = tq_take_warp(tq, tseq, abort_flag, lane);
+      if (ti < 0) break;
       const Tile tl = tiles[ti];
       const LayerDev& L = t.layers[tl.layer];
       const uint32_t db = tseq & 1;
@@ -605,11 +673,15 @@ tc_pass1_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
     bool ok = true;
     const uint32_t lane_base = tmem + ((uint32_t)(32 * q) << 16) + S::kACol0;
     const int row = 32 * q + lane;
-    for (int ti = t_begin; ti < t_end && ok; ++ti) {
+    for (uint32_t qs = 0; ok; ++qs) {
+      const int ti = tq_take_warp(tq, qs, abort_flag, lane);
+      if (ti < 0) { ok = ti == kTqEnd; break; }
       const int nk = (tiles[ti].ncols + kTcK - 1) / kTcK;
       for (int k = 0; k < nk; ++k, ++kc) {
         if ((int)(kc % kTcGroups) != g) continue;
         const int s = kc % kT1Stages, ab = kc % kT1AB;
+        // first the slot's previous piece must have been taken, by whichever group had it (see pass 2)
+        if (!warp_wait(m_ready + s, ((kc / kT1Stages) & 1) ^ 1, abort_flag, lane)) { ok = false; break; }
         if (!warp_wait(ge_full + s, (kc / kT1Stages) & 1, abort_flag, lane)) { ok = false; break; }
         const uint8_t* gp = g_piece(s) + row * 128;
         uint8_t* ep = e_piece(s) + row * 128;
@@ -645,14 +717,15 @@ tc_pass1_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
   }
   tc_fence_before();
   __syncthreads();
-  if (tid == 0 && *abort_flag && t_end > t_begin) report_timeout(t, tiles[t_begin].layer);
+  if (tid == 0 && *abort_flag && ntiles > 0) report_timeout(t, tiles[min((int)blockIdx.x, ntiles - 1)].layer);
+  if (tid == 0) tq_leave(sched);
   if (warp == 2)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)S::kTmemCols) : "memory");
 }
 
 // ---------------------------------------------------------------------------------------
 // Pass 3 on the tensor core (G_hat = P_bar Q_bar^T, E_w = M_w - G_hat, Alg. 1; optional model
-// update).  A tile is 128 rows x 128 columns of one layer, for all workers.  Once per tile the
+// update).  A tile is 128 rows x 128 columns of one layer, for a range of workers [worker, part).  Once per tile the
 // accumulator D = G_hat tile is formed from the factors: both operands come from shared memory,
 // K-major, as rows of kCat = 3 RP (padded to a multiple of 32) tf32 values
 //   P side: [P_bar | P_bar | P_bar_lo | 0]      Q side: [Q_bar | Q_bar_lo | Q_bar | 0]
@@ -678,19 +751,21 @@ struct Pass3Cfg {
                                                                          // the other through the same buffer (rank 64: 2 x 96)
   static constexpr int kSub = kCat / 32 / kHalves;                       // 128-byte sub-tiles per operand slice
   static constexpr uint32_t kOpBytes = kSub * kT1PieceBytes;             // one operand slice: kSub pieces of 128 rows x 32
-  static constexpr uint32_t kOpOff = kT3Stages * kT1PieceBytes;
+  static constexpr int kStages = kT3Stages;                               // ring of M pieces
+  static constexpr uint32_t kOpOff = kStages * kT1PieceBytes;
   static constexpr uint32_t kBarOff = kOpOff + 2 * kOpBytes;
-  static constexpr int kBars = 3 * kT3Stages + 2 + 2 + 2 + 2 + 1;      // m_full, e_ready, m_empty; op_full, op_empty, d_full, d_empty (2 each); fin
-  static constexpr uint32_t kTotal = kBarOff + kBars * 8 + 16 + 1024;
+  static constexpr int kBars = 3 * kStages + 2 + 2 + 2 + 2 + 1 + 2 * kTqDepth;   // m_full, e_ready, m_empty; op_full, op_empty, d_full, d_empty (2 each); fin; tile queue
+  static constexpr uint32_t kTotal = kBarOff + kBars * 8 + 16 + 4 * kTqDepth + 1024;
   static constexpr int kTmemCols = 256;                                  // two accumulators of 128 columns
   static_assert((kCat / 32) % kHalves == 0 && kTotal <= 227 * 1024, "operand slices, shared memory");
 };
 
 template <int RP>
 __global__ void __launch_bounds__(kTcThreads, 1)
-tc_pass3_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict__ cta_begin, const uint8_t* __restrict__ maps) {
+tc_pass3_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, int* __restrict__ sched, const uint8_t* __restrict__ maps) {
   pdl_wait();
   using S = Pass3Cfg<RP>;
+  constexpr int kT3Stages = S::kStages;          // this rank's ring depth
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* opa = base + S::kOpOff;               // P side
@@ -704,17 +779,20 @@ tc_pass3_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
   uint64_t* d_full = op_empty + 2;               // [2]
   uint64_t* d_empty = d_full + 2;                // [2] all 16 consumer warps are past the tile
   uint64_t* fin = d_empty + 2;
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(fin + 1);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(fin + 1) + 2;   // after the abort flag and the wait limit
+  uint64_t* q_full = fin + 1;                    // [kTqDepth] tile queue
+  uint64_t* q_empty = q_full + kTqDepth;         // [kTqDepth]
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(q_empty + kTqDepth);
+  uint32_t* tmem_slot = const_cast<uint32_t*>(reinterpret_cast<volatile uint32_t*>(abort_flag)) + 2;   // after the abort flag and the wait limit
+  const TileQueue tq{q_full, q_empty, reinterpret_cast<volatile int*>(tmem_slot + 2)};
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int t_begin = cta_begin[blockIdx.x], t_end = cta_begin[blockIdx.x + 1];
-  const int W = t.W;
   if (tid == 0) {
     for (int s = 0; s < kT3Stages; ++s) { mbar_init(m_full + s, 1); mbar_init(e_ready + s, 4); mbar_init(m_empty + s, 1); }
     mbar_init(op_full, 1); mbar_init(op_empty, 1);
     for (int s = 0; s < 2; ++s) { mbar_init(d_full + s, 1); mbar_init(d_empty + s, 4 * kT3Groups); }
     mbar_init(fin, 1);
+    // readers of the tile queue: operand loader, MMA thread, storer, 16 consumer warps
+    for (int s = 0; s < kTqDepth; ++s) { mbar_init(q_full + s, 1); mbar_init(q_empty + s, 3 + 4 * kT3Groups); }
     wait_ctl_init(abort_flag, t.wait_limit);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
@@ -732,13 +810,21 @@ tc_pass3_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
 
   if (warp == 0) {
     // ---- M loader
-    uint32_t kc = 0;
+    uint32_t kc = 0, qs = 0;
     bool ok = true;
-    for (int ti = t_begin; ti < t_end && ok; ++ti) {
+    int ti = (int)blockIdx.x < ntiles ? (int)blockIdx.x : kTqEnd;
+    for (;; ++qs) {
+      int put = 1, drawn = kTqEnd;
+      if (lane == 0) {
+        put = tq_put(tq, qs, ti, abort_flag) ? 1 : 0;
+        if (put && ti != kTqEnd) drawn = tq_draw(sched, ntiles);        // the tile after this one: the answer comes meanwhile
+      }
+      if (!__shfl_sync(0xffffffffu, put, 0)) { ok = false; break; }
+      if (ti == kTqEnd) break;
       const Tile tl = tiles[ti];
       const uint8_t* map = maps + ((size_t)tl.layer * kTcMapsPerLayer + 2) * kTcMapBytes;
       const int np = pieces_of(tl);
-      for (int w = 0; w < W && ok; ++w)
+      for (int w = tl.worker; w < tl.part && ok; ++w)
         for (int pc = 0; pc < np; ++pc, ++kc) {
           const int s = kc % kT3Stages;
           if (!warp_wait(m_empty + s, ((kc / kT3Stages) & 1) ^ 1, abort_flag, lane)) { ok = false; break; }
@@ -748,6 +834,8 @@ tc_pass3_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
             tma_load_3d(piece(s), map, tl.col0 + pc * kTcK, tl.row0, w, m_full + s);
           }
         }
+      if (!ok) break;
+      ti = __shfl_sync(0xffffffffu, drawn, 0);
     }
     if (!ok && lane == 0)
       for (uint32_t it = kc > (uint32_t)kT3Stages ? kc - kT3Stages : 0; it < kc; ++it)
@@ -756,7 +844,9 @@ tc_pass3_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
     // ---- operand loader: the tile's rows of the stacked P_bar terms and its columns' rows of the Q_bar terms
     uint32_t oseq = 0;                      // operand slices loaded so far (kHalves per tile)
     bool ok = true;
-    for (int ti = t_begin; ti < t_end && ok; ++ti) {
+    for (uint32_t qs = 0; ok; ++qs) {
+      const int ti = tq_take_warp(tq, qs, abort_flag, lane);
+      if (ti < 0) { ok = ti == kTqEnd; break; }
       const Tile tl = tiles[ti];
       const uint8_t* mapp = maps + ((size_t)tl.layer * kTcMapsPerLayer + 4) * kTcMapBytes;
       const uint8_t* mapq = maps + ((size_t)tl.layer * kTcMapsPerLayer + 5) * kTcMapBytes;
@@ -780,7 +870,9 @@ tc_pass3_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
       bool ok = true;
       const uint32_t idesc = tc_idesc_tf32(128);
       const uint64_t adesc0 = tc_desc_sw128(smem_u32(opa)), bdesc0 = tc_desc_sw128(smem_u32(opb));
-      for (int ti = t_begin; ti < t_end && ok; ++ti, ++tseq) {
+      for (; ok; ++tseq) {
+        const int ti = tq_take(tq, tseq, abort_flag);
+        if (ti < 0) { ok = ti == kTqEnd; break; }
         const uint32_t db = tseq & 1;
         if (!thread_wait(d_empty + db, ((tseq >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
         for (int h = 0; h < S::kHalves && ok; ++h, ++oseq) {
@@ -805,11 +897,13 @@ tc_pass3_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
     // ---- storer: E pieces back to global memory
     uint32_t kc = 0;
     bool ok = true;
-    for (int ti = t_begin; ti < t_end && ok; ++ti) {
+    for (uint32_t qs = 0; ok; ++qs) {
+      const int ti = tq_take_warp(tq, qs, abort_flag, lane);
+      if (ti < 0) { ok = ti == kTqEnd; break; }
       const Tile tl = tiles[ti];
       const uint8_t* map = maps + ((size_t)tl.layer * kTcMapsPerLayer + 2) * kTcMapBytes;
       const int np = pieces_of(tl);
-      for (int w = 0; w < W && ok; ++w)
+      for (int w = tl.worker; w < tl.part && ok; ++w)
         for (int pc = 0; pc < np; ++pc, ++kc) {
           const int s = kc % kT3Stages;
           if (!warp_wait(e_ready + s, (kc / kT3Stages) & 1, abort_flag, lane)) { ok = false; break; }
@@ -835,7 +929,9 @@ tc_pass3_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
     uint32_t kc = 0, tseq = 0;
     bool ok = true;
     const int row_in_tile = 32 * q + lane;
-    for (int ti = t_begin; ti < t_end && ok; ++ti, ++tseq) {
+    for (; ok; ++tseq) {
+      const int ti = tq_take_warp(tq, tseq, abort_flag, lane);
+      if (ti < 0) { ok = ti == kTqEnd; break; }
       const Tile tl = tiles[ti];
       const LayerDev& L = t.layers[tl.layer];
       const int np = pieces_of(tl);
@@ -848,10 +944,12 @@ tc_pass3_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
       // arrival on d_empty below must not run ahead of the tile
       if (!warp_wait(d_full + db, (tseq >> 1) & 1, abort_flag, lane)) { ok = false; break; }
       tc_fence_after();
-      for (int w = 0; w < W && ok; ++w)
+      for (int w = tl.worker; w < tl.part && ok; ++w)
         for (int pc = 0; pc < np; ++pc, ++kc) {
           if ((int)(kc % kT3Groups) != g) continue;
           const int s = kc % kT3Stages;
+          // first the slot's previous piece must have been taken, by whichever group had it (see pass 2)
+          if (!warp_wait(e_ready + s, ((kc / kT3Stages) & 1) ^ 1, abort_flag, lane)) { ok = false; break; }
           uint32_t gh[32];
           tc_ld32(taddr + pc * 32, gh);
           if (!warp_wait(m_full + s, (kc / kT3Stages) & 1, abort_flag, lane)) { tc_wait_ld(); ok = false; break; }
@@ -897,7 +995,8 @@ tc_pass3_kernel(Tables t, const Tile* __restrict__ tiles, const int* __restrict_
   }
   tc_fence_before();
   __syncthreads();
-  if (tid == 0 && *abort_flag && t_end > t_begin) report_timeout(t, tiles[t_begin].layer);
+  if (tid == 0 && *abort_flag && ntiles > 0) report_timeout(t, tiles[min((int)blockIdx.x, ntiles - 1)].layer);
+  if (tid == 0) tq_leave(sched);
   if (warp == 2)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)S::kTmemCols) : "memory");
 }
@@ -978,13 +1077,42 @@ int tc_encode_maps(const LayerDev* layers, int n_layers, int W, int RP, void* ou
   return LQSGD_OK;
 }
 
-cudaError_t launch_tc_pass3(int RP, const Tables& t, const Tile* tiles, int ntiles, const int* cta_begin, const void* maps,
+// One tensor map per (layer, worker) over the caller's gradient, [n][m] fp32: pieces of 128 rows x 32 columns, 128-byte
+// swizzle (pass 1).  grads: [n_layers][W] device pointers, 16-byte aligned for the layers concerned; out: [n_layers][W] maps.
+int tc_encode_grad_maps(const LayerDev* layers, int n_layers, int W, const void* const* grads, void* out) {
+  std::memset(out, 0, (size_t)n_layers * W * kTcMapBytes);
+  static EncodeTiledFn encode = nullptr;
+  if (!encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+        qres != cudaDriverEntryPointSuccess)
+      return LQSGD_ERR_CUDA;
+    encode = reinterpret_cast<EncodeTiledFn>(fn);
+  }
+  CUtensorMap* maps = static_cast<CUtensorMap*>(out);
+  for (int i = 0; i < n_layers; ++i) {
+    const LayerDev& L = layers[i];
+    if (!L.tc) continue;
+    const cuuint64_t dim[2] = {(cuuint64_t)L.m, (cuuint64_t)L.n};
+    const cuuint64_t stride[1] = {(cuuint64_t)L.m * 4};
+    const cuuint32_t box[2] = {kTcK, 128}, es[2] = {1, 1};
+    for (int w = 0; w < W; ++w)
+      if (encode(&maps[(size_t)i * W + w], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(grads[(size_t)i * W + w]), dim, stride,
+                 box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return LQSGD_ERR_CUDA;
+  }
+  return LQSGD_OK;
+}
+
+cudaError_t launch_tc_pass3(int RP, const Tables& t, const Tile* tiles, int ntiles, int* sched, const void* maps,
                             Launch l) {
   if (ntiles == 0) return cudaSuccess;
   auto go = [&](auto kernel, size_t smem) -> cudaError_t {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    return launch_pdl(kernel, dim3(l.grid), dim3(kTcThreads), smem, l.stream, t, tiles, cta_begin, static_cast<const uint8_t*>(maps));
+    return launch_pdl(kernel, dim3(l.grid), dim3(kTcThreads), smem, l.stream, t, tiles, ntiles, sched, static_cast<const uint8_t*>(maps));
   };
   if (RP == 16) return go(tc_pass3_kernel<16>, Pass3Cfg<16>::kTotal);
   if (RP == 32) return go(tc_pass3_kernel<32>, Pass3Cfg<32>::kTotal);
@@ -992,13 +1120,13 @@ cudaError_t launch_tc_pass3(int RP, const Tables& t, const Tile* tiles, int ntil
   return cudaErrorInvalidValue;
 }
 
-cudaError_t launch_tc_pass1(int RP, const Tables& t, const Tile* tiles, int ntiles, const int* cta_begin, const void* maps,
+cudaError_t launch_tc_pass1(int RP, const Tables& t, const Tile* tiles, int ntiles, int* sched, const void* maps,
                             Launch l) {
   if (ntiles == 0) return cudaSuccess;
   auto go = [&](auto kernel, size_t smem) -> cudaError_t {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    return launch_pdl(kernel, dim3(l.grid), dim3(kTcThreads), smem, l.stream, t, tiles, cta_begin, static_cast<const uint8_t*>(maps));
+    return launch_pdl(kernel, dim3(l.grid), dim3(kTcThreads), smem, l.stream, t, tiles, ntiles, sched, static_cast<const uint8_t*>(maps));
   };
   if (RP == 16) return go(tc_pass1_kernel<16>, Pass1Cfg<16>::kTotal);
   if (RP == 32) return go(tc_pass1_kernel<32>, Pass1Cfg<32>::kTotal);
