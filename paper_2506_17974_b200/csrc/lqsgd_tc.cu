@@ -152,9 +152,9 @@ __device__ __forceinline__ int tq_take_warp(const TileQueue& q, uint32_t seq, vo
   if (lane == 0) v = tq_take(q, seq, abort_flag);
   return __shfl_sync(0xffffffffu, v, 0);
 }
-// the loader thread's draw: tiles gridDim.x, gridDim.x + 1, ... in the order asked for
-__device__ __forceinline__ int tq_draw(int* sched, int ntiles) {
-  const int v = (int)gridDim.x + atomicAdd(sched, 1);
+// the loader thread's draw: the tiles after the fixed ones (fixed_per_cta per CTA), in the order asked for
+__device__ __forceinline__ int tq_draw(int* sched, int ntiles, int fixed_per_cta = 1) {
+  const int v = fixed_per_cta * (int)gridDim.x + atomicAdd(sched, 1);
   return v < ntiles ? v : kTqEnd;
 }
 // at the very end of the kernel, one thread per CTA: the last CTA to leave readies the counter for the next launch
@@ -810,17 +810,26 @@ tc_pass3_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, int* __res
 
   if (warp == 0) {
     // ---- M loader
+    // The queue runs one entry ahead of the loads: while this warp fetches the pieces of one entry, the operand
+    // loader and the MMA thread already form G_hat of the next (two accumulators), so that the consumers find it
+    // ready.  The first two entries are fixed (tiles b and b + gridDim.x), the counter hands out the rest.
     uint32_t kc = 0, qs = 0;
     bool ok = true;
     int ti = (int)blockIdx.x < ntiles ? (int)blockIdx.x : kTqEnd;
-    for (;; ++qs) {
+    int nxt = ti != kTqEnd && (int)(blockIdx.x + gridDim.x) < ntiles ? (int)(blockIdx.x + gridDim.x) : kTqEnd;
+    {
+      int put = 1;
+      if (lane == 0) put = tq_put(tq, qs, ti, abort_flag) ? 1 : 0;
+      ++qs;
+      if (!__shfl_sync(0xffffffffu, put, 0)) { ok = false; ti = kTqEnd; }
+    }
+    for (; ti != kTqEnd; ++qs) {
       int put = 1, drawn = kTqEnd;
       if (lane == 0) {
-        put = tq_put(tq, qs, ti, abort_flag) ? 1 : 0;
-        if (put && ti != kTqEnd) drawn = tq_draw(sched, ntiles);        // the tile after this one: the answer comes meanwhile
+        put = tq_put(tq, qs, nxt, abort_flag) ? 1 : 0;
+        if (put && nxt != kTqEnd) drawn = tq_draw(sched, ntiles, 2);    // the entry after the next: the answer comes meanwhile
       }
       if (!__shfl_sync(0xffffffffu, put, 0)) { ok = false; break; }
-      if (ti == kTqEnd) break;
       const Tile tl = tiles[ti];
       const uint8_t* map = maps + ((size_t)tl.layer * kTcMapsPerLayer + 2) * kTcMapBytes;
       const int np = pieces_of(tl);
@@ -835,7 +844,8 @@ tc_pass3_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, int* __res
           }
         }
       if (!ok) break;
-      ti = __shfl_sync(0xffffffffu, drawn, 0);
+      ti = nxt;
+      nxt = __shfl_sync(0xffffffffu, drawn, 0);
     }
     if (!ok && lane == 0)
       for (uint32_t it = kc > (uint32_t)kT3Stages ? kc - kT3Stages : 0; it < kc; ++it)
