@@ -593,11 +593,13 @@ def test_bit_reproducible_and_checkpoint_resume(rank, one_launch):
     assert torch.equal(a.get_state(B.STATE_E, 2, 2), c.get_state(B.STATE_E, 2, 2))
 
 
-@pytest.mark.parametrize("one_launch", [False, True])
-def test_step_replays_from_a_cuda_graph(one_launch):
+@pytest.mark.parametrize("one_launch,rank", [(False, 4), (True, 4), (False, 16)])
+def test_step_replays_from_a_cuda_graph(one_launch, rank):
     """A step captured into a CUDA graph (kernels only, dependent launches included; or the one cooperative
-    launch) replays to the same bits as eager steps; a capture with unseen tensor pointers is refused."""
-    w = dataclasses.replace(wl.config2(), workers=2)
+    launch) replays to the same bits as eager steps; a capture with unseen tensor pointers is refused.
+    Rank 16: the tensor-core passes, whose tile counters must be back at zero after every replay and whose
+    gradient tensor maps belong to the captured pointer table."""
+    w = dataclasses.replace(wl.config2(), workers=2, rank=rank)
     a, b = make(w, one_launch=one_launch), make(w, one_launch=one_launch)
     g0 = wl.draw_gradients(w, 0, device=DEV)
     bufs = [[torch.empty_like(x) for x in per] for per in g0]
