@@ -684,8 +684,10 @@ def main():
                     help="workers of all GPUs in one average, with the real NCCL exchange (default: independent replicas)")
     args = ap.parse_args()
     if args.source_digest:
-        for group in (["lqsgd_stream.cu", "lqsgd_stream_common.cuh", "lqsgd_dev.h"], ["lqsgd_kernels.cu", "lqsgd_dev.h"],
-                      ["lqsgd_tc.cu", "lqsgd_stream_common.cuh", "lqsgd_dev.h"]):
+        for group in (["lqsgd_stream.cu", "lqsgd_stream_common.cuh", "lqsgd_dev.h"],
+                      ["lqsgd_kernels.cu", "lqsgd_factor.cuh", "lqsgd_dev.h"],
+                      ["lqsgd_tc.cu", "lqsgd_stream_common.cuh", "lqsgd_dev.h"],
+                      ["lqsgd_resident.cu", "lqsgd_factor.cuh", "lqsgd_stream_common.cuh", "lqsgd_dev.h"]):
             print(" ".join(group), csrc_digest(group))
         return
     if args.impl == "ours" and args.gpus > 1 and "WORLD_SIZE" not in os.environ:
