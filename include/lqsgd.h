@@ -64,7 +64,8 @@ typedef enum lqsgd_error {
   LQSGD_ERR_NO_STAGING = -6,          /* lqsgd_step_host() on a context created without LQSGD_FLAG_HOST_STAGING */
   LQSGD_ERR_OUT_OF_RANGE = -7,        /* layer / worker / state index out of range, or state not defined for that layer */
   LQSGD_ERR_TOO_LARGE = -8,           /* size beyond the fixed built-in scratch of lqsgd_orthonormalize_noalloc */
-  LQSGD_ERR_CAPTURE = -9              /* stream is capturing and the tensor pointers differ from the previous call's */
+  LQSGD_ERR_CAPTURE = -9,             /* stream is capturing and the tensor pointers differ from the previous call's */
+  LQSGD_ERR_PLAN = -10                /* lqsgd_plan_check: the work tables of this configuration fail an invariant (a defect of the library) */
 } lqsgd_error;
 
 /* Bits of the per-layer status word. */
@@ -332,6 +333,24 @@ int lqsgd_round_timeline(const lqsgd_ctx* ctx, uint64_t* host_ns, int32_t* host_
  * *host_first_offset (may be NULL) the byte offset in the workspace of the first of them, or -1.
  * LQSGD_ERR_INVALID_ARG for a context without guards. */
 int lqsgd_check_guards(const lqsgd_ctx* ctx, int64_t* host_changed_words, int64_t* host_first_offset, void* cuda_stream);
+
+/* Host-only self-check of the work tables the library would build for this configuration on a device with sm_count
+ * SMs (148 on a B200; the tile sizes depend on it): no device is touched, nothing is allocated on one.  Verifies
+ * that every pass's tiles cover every (layer, worker, row, column) exactly once, that the partial sums each tile
+ * writes (Section IV-A's two products, summed over column or row chunks) are exactly the ones the following step
+ * adds up, that the factor blocks and exchange chunks cover every factor element once, and that the second-level
+ * sums of layers with many partial sums take every partial once.  Returns LQSGD_OK, the configuration's own error
+ * (as lqsgd_workspace_bytes), or LQSGD_ERR_PLAN with a description of the first failed invariant in msg (may be
+ * NULL; at most msg_len bytes including the terminator).  Meant for tests: a planner defect shows here, on the
+ * CPU, for any shape, before a kernel runs on wrong tables. */
+int lqsgd_plan_check(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config* cfg, int32_t sm_count, char* msg,
+                     size_t msg_len);
+
+/* Test support for lqsgd_plan_check: the calling thread's NEXT lqsgd_plan_check first damages its (private) copy of
+ * the tables and must then report LQSGD_ERR_PLAN: kind 1 drops a tile of pass 1, 2 gives two tiles of pass 2 the same
+ * partial-sum slot, 3 drops the last tile of pass 3 (for a tile with ranges of workers: its last range), 4 drops a
+ * second-level sum (configurations with none stay undamaged), 5 drops an exchange chunk of Q.  0 disarms.  Nothing a context uses is touched. */
+int lqsgd_test_plan_defect(int32_t kind);
 
 /* Kernel launches one lqsgd_step enqueues (for launch accounting). */
 int lqsgd_launches_per_step(const lqsgd_ctx* ctx, int32_t* host_out);

@@ -35,6 +35,7 @@ ERR_INVALID_ARG, ERR_BAD_SHAPE, ERR_WORKSPACE_TOO_SMALL, ERR_MISALIGNED = -1, -2
 ERR_CUDA, ERR_NO_STAGING, ERR_OUT_OF_RANGE = -5, -6, -7
 ERR_TOO_LARGE = -8
 ERR_CAPTURE = -9
+ERR_PLAN = -10
 NOALLOC_MAX_ROWS = 65536
 
 EXPORTED = [
@@ -42,7 +43,7 @@ EXPORTED = [
     "lqsgd_payload", "lqsgd_payload_layout", "lqsgd_get_state", "lqsgd_set_state", "lqsgd_status",
     "lqsgd_orthonormalize_noalloc",
     "lqsgd_round_begin", "lqsgd_round_pack", "lqsgd_round_reduce", "lqsgd_round_end", "lqsgd_exchange_view",
-    "lqsgd_launches_per_step", "lqsgd_set_phase_events", "lqsgd_release_graph_tables", "lqsgd_test_expire_wait", "lqsgd_round_timeline", "lqsgd_check_guards", "lqsgd_destroy", "lqsgd_strerror", "lqsgd_last_cuda_error", "lqsgd_version",
+    "lqsgd_launches_per_step", "lqsgd_set_phase_events", "lqsgd_release_graph_tables", "lqsgd_test_expire_wait", "lqsgd_round_timeline", "lqsgd_check_guards", "lqsgd_plan_check", "lqsgd_test_plan_defect", "lqsgd_destroy", "lqsgd_strerror", "lqsgd_last_cuda_error", "lqsgd_version",
 ]
 
 
@@ -103,6 +104,8 @@ def load_library() -> C.CDLL:
     lib.lqsgd_test_expire_wait.argtypes = [vp, i32, i32, C.c_uint32]
     lib.lqsgd_round_timeline.argtypes = [vp, C.POINTER(C.c_uint64), C.POINTER(i32), vp]
     lib.lqsgd_check_guards.argtypes = [vp, C.POINTER(C.c_int64), C.POINTER(C.c_int64), vp]
+    lib.lqsgd_plan_check.argtypes = [vp, i32, vp, i32, C.c_char_p, C.c_size_t]
+    lib.lqsgd_test_plan_defect.argtypes = [i32]
     lib.lqsgd_destroy.argtypes = [vp]
     lib.lqsgd_destroy.restype = None
     lib.lqsgd_strerror.argtypes = [C.c_int]
@@ -153,6 +156,22 @@ def workspace_bytes(layers, cfg: Config) -> int:
     out = C.c_size_t(0)
     _check(load_library().lqsgd_workspace_bytes(_shapes(layers), len(layers), C.byref(cfg), C.byref(out)))
     return out.value
+
+
+def test_plan_defect(kind: int) -> None:
+    """Test support: the next plan_check of this thread damages its private tables first (see the header)."""
+    _check(load_library().lqsgd_test_plan_defect(kind))
+
+
+def plan_check(layers, cfg: Config, sm_count: int = 148) -> str:
+    """Host-only self-check of the work tables for this configuration (lqsgd_plan_check): "" when every invariant
+    holds, else the description of the first one that fails; raises for an invalid configuration."""
+    msg = C.create_string_buffer(512)
+    rc = load_library().lqsgd_plan_check(_shapes(layers), len(layers), C.byref(cfg), sm_count, msg, len(msg))
+    if rc == ERR_PLAN:
+        return msg.value.decode() or "plan check failed"
+    _check(rc)
+    return ""
 
 
 class LQSGD:

@@ -6,11 +6,14 @@
 #include <nvtx3/nvToolsExt.h>
 
 #include <algorithm>
+#include <array>
 #include <cmath>
 #include <cstring>
+#include <map>
 #include <new>
 #include <queue>
 #include <string>
+#include <tuple>
 #include <vector>
 
 using namespace lqsgd;
@@ -820,6 +823,7 @@ const char* lqsgd_strerror(int code) {
     case LQSGD_ERR_OUT_OF_RANGE: return "index out of range";
     case LQSGD_ERR_TOO_LARGE: return "size exceeds the built-in scratch of the no-allocation entry point";
     case LQSGD_ERR_CAPTURE: return "stream is capturing and the tensor pointers changed since the previous call";
+    case LQSGD_ERR_PLAN: return "the work tables of this configuration fail an invariant (lqsgd_plan_check)";
     default: return "unknown error";
   }
 }
@@ -835,6 +839,242 @@ int lqsgd_workspace_bytes(const lqsgd_shape* shapes, int32_t n_layers, const lqs
   make_plan(shapes, n_layers, *cfg, nullptr, 1, p2);
   make_plan(shapes, n_layers, *cfg, nullptr, 148, p3, false);     // in case the one-launch round cannot run on the device
   *out = std::max({p.bytes, p2.bytes, p3.bytes});
+  return LQSGD_OK;
+}
+
+namespace {
+// lqsgd_plan_check: the invariants of a plan.  Every tiling here is a grid (row bands cut into column chunks), so
+// "covers once" is checked band by band.
+struct Rect { int row0, nrows, col0, ncols, part; };
+std::string check_grid(std::vector<Rect> v, int n, int m, int nparts, bool parts_along_cols, const char* what) {
+  // rows: bands in order, contiguous from 0 to n; inside a band the chunks contiguous from 0 to m
+  std::sort(v.begin(), v.end(), [](const Rect& a, const Rect& b) { return a.row0 != b.row0 ? a.row0 < b.row0 : a.col0 < b.col0; });
+  std::map<int, std::vector<int>> parts_of;       // chunk position along the OTHER axis -> parts seen
+  size_t i = 0;
+  int row = 0;
+  while (i < v.size()) {
+    if (v[i].row0 != row) return std::string(what) + ": row band does not start where the last ended";
+    const int nr = v[i].nrows;
+    if (nr < 1) return std::string(what) + ": empty tile";
+    int col = 0;
+    for (; i < v.size() && v[i].row0 == row; ++i) {
+      if (v[i].nrows != nr) return std::string(what) + ": tiles of one band differ in height";
+      if (v[i].col0 != col || v[i].ncols < 1) return std::string(what) + ": column chunk does not start where the last ended";
+      col += v[i].ncols;
+      if (nparts > 0) {
+        if (v[i].part < 0 || v[i].part >= nparts) return std::string(what) + ": partial-sum index out of range";
+        parts_of[parts_along_cols ? row : v[i].col0].push_back(v[i].part);
+      }
+    }
+    if (col != m) return std::string(what) + ": a band's chunks do not end at the last column";
+    row += nr;
+  }
+  if (row != n) return std::string(what) + ": bands do not end at the last row";
+  for (auto& kv : parts_of) {                      // every partial sum written exactly once
+    std::vector<int>& ps = kv.second;
+    std::sort(ps.begin(), ps.end());
+    if ((int)ps.size() != nparts) return std::string(what) + ": partial sums written != partial sums added up";
+    for (int k = 0; k < nparts; ++k)
+      if (ps[k] != k) return std::string(what) + ": a partial sum is written twice or never";
+  }
+  return "";
+}
+
+std::string check_plan(const Plan& p) {
+  const int W = p.W;
+  const size_t nm = p.mats.size();
+  auto layer_name = [&](size_t li) { return " (layer " + std::to_string(p.mats[li].user_index) + ", " + std::to_string(p.mats[li].n) + " x " + std::to_string(p.mats[li].m) + ")"; };
+  // ---- passes 1 and 2: per (layer, worker) one grid; pass 3: per layer one grid over all workers
+  std::vector<std::vector<Rect>> g1(nm * W), g2(nm * W), g3(nm);
+  std::map<std::array<int, 3>, std::vector<std::pair<int, int>>> tc3;     // (layer, row0, col0) -> worker ranges
+  auto bad_tile = [&](const Tile& tl) { return tl.layer < 0 || tl.layer >= (int)nm || tl.worker < 0 || tl.worker >= W; };
+  for (auto* list : {&p.tiles1, &p.stiles1, &p.tctiles1})
+    for (const Tile& tl : *list) {
+      if (bad_tile(tl)) return "pass 1: tile with a layer or worker out of range";
+      g1[(size_t)tl.layer * W + tl.worker].push_back({tl.row0, tl.nrows, tl.col0, tl.ncols, tl.part});
+    }
+  for (auto* list : {&p.tiles2, &p.tctiles2})
+    for (const Tile& tl : *list) {
+      if (bad_tile(tl)) return "pass 2: tile with a layer or worker out of range";
+      g2[(size_t)tl.layer * W + tl.worker].push_back({tl.row0, tl.nrows, tl.col0, tl.ncols, tl.part});
+    }
+  for (auto* list : {&p.tiles3, &p.stiles3})
+    for (const Tile& tl : *list) {
+      if (tl.layer < 0 || tl.layer >= (int)nm) return "pass 3: tile with a layer out of range";
+      g3[tl.layer].push_back({tl.row0, tl.nrows, tl.col0, tl.ncols, 0});
+    }
+  for (const Tile& tl : p.tctiles3) {
+    if (tl.layer < 0 || tl.layer >= (int)nm) return "pass 3: tile with a layer out of range";
+    auto& ranges = tc3[{tl.layer, tl.row0, tl.col0}];
+    if (ranges.empty()) g3[tl.layer].push_back({tl.row0, tl.nrows, tl.col0, tl.ncols, 0});
+    ranges.push_back({tl.worker, tl.part});
+  }
+  for (auto& kv : tc3) {                           // a tile's ranges of workers: 0 .. W without gap or overlap
+    auto r = kv.second;
+    std::sort(r.begin(), r.end());
+    int w = 0;
+    for (auto& ab : r) {
+      if (ab.first != w || ab.second <= ab.first) return "pass 3: a tile's ranges of workers leave a gap or overlap" + layer_name(kv.first[0]);
+      w = ab.second;
+    }
+    if (w != W) return "pass 3: a tile's ranges of workers do not end at the last worker" + layer_name(kv.first[0]);
+  }
+  if (p.resident) {
+    for (const ResTile& tl : p.rtiles) {
+      if (tl.layer < 0 || tl.layer >= (int)nm || tl.worker < 0 || tl.worker >= W) return "one-launch round: tile out of range";
+      g1[(size_t)tl.layer * W + tl.worker].push_back({tl.row0, tl.nrows, tl.col0, tl.ncols, tl.part_c});
+      g2[(size_t)tl.layer * W + tl.worker].push_back({tl.row0, tl.nrows, tl.col0, tl.ncols, tl.part_r});
+      if (tl.worker == 0) g3[tl.layer].push_back({tl.row0, tl.nrows, tl.col0, tl.ncols, 0});
+      if ((tl.worker == 0) != (tl.writes_ghat != 0)) return "one-launch round: G_hat is written by worker 0's tiles, and only those";
+    }
+  }
+  for (size_t li = 0; li < nm; ++li) {
+    const LayerDev& L = p.layers[li];
+    for (int w = 0; w < W; ++w) {
+      std::string e = check_grid(g1[li * W + w], L.n, L.m, L.ncc, true, "pass 1");
+      if (e.empty()) e = check_grid(g2[li * W + w], L.n, L.m, L.nrb, false, "pass 2");
+      if (!e.empty()) return e + layer_name(li) + ", worker " + std::to_string(w);
+    }
+    std::string e = check_grid(g3[li], L.n, L.m, 0, true, "pass 3");
+    if (!e.empty()) return e + layer_name(li);
+    if (L.npb != ceil_div(L.n, kFactorBlockRows) || L.nqb != ceil_div(L.m, kFactorBlockRows)) return "factor block counts" + layer_name(li);
+  }
+  // ---- factor blocks and exchange chunks
+  {
+    std::vector<int> seenP(nm * W, 0), seenQ(nm * W, 0), seenS(nm * W, 0);
+    std::map<std::pair<size_t, int>, int> blkP, blkQ;
+    for (const FactorBlock& f : p.fbS) { if (f.layer < 0 || f.layer >= (int)nm || f.worker < 0 || f.worker >= W) return "Orthonormalize: block out of range"; ++seenS[(size_t)f.layer * W + f.worker]; }
+    for (const FactorBlock& f : p.fbP) { if (f.layer < 0 || f.layer >= (int)nm || f.worker < 0 || f.worker >= W) return "Orthonormalize: block out of range"; ++blkP[{(size_t)f.layer * W + f.worker, f.blk}]; }
+    for (const FactorBlock& f : p.fbQ) { if (f.layer < 0 || f.layer >= (int)nm || f.worker < 0 || f.worker >= W) return "Q_w reduction: block out of range"; ++blkQ[{(size_t)f.layer * W + f.worker, f.blk}]; }
+    for (size_t li = 0; li < nm; ++li)
+      for (int w = 0; w < W; ++w) {
+        const size_t k = li * W + w;
+        const LayerDev& L = p.layers[li];
+        int np = 0;
+        for (int b = 0; b < L.npb; ++b) { auto it = blkP.find({k, b}); if (it != blkP.end()) { if (it->second != 1) return "Orthonormalize: a block of rows twice" + layer_name(li); ++np; } }
+        if (!((seenS[k] == 1 && np == 0) || (seenS[k] == 0 && np == L.npb))) return "Orthonormalize: every row of P once, by one CTA or by blocks of 128" + layer_name(li);
+        for (int b = 0; b < L.nqb; ++b) { auto it = blkQ.find({k, b}); if (it == blkQ.end() || it->second != 1) return "Q_w reduction: every block of 128 rows of Q once" + layer_name(li); }
+      }
+    if (blkP.size() + 0 != [&] { size_t t = 0; for (size_t li = 0; li < nm; ++li) for (int w = 0; w < W; ++w) if (!seenS[li * W + w]) t += p.layers[li].npb; return t; }()) return "Orthonormalize: blocks beyond the layers' rows";
+    std::vector<std::vector<int>> cP(nm), cQ(nm);
+    for (const ExchangeChunk& c : p.chP) { if (c.layer < 0 || c.layer >= (int)nm) return "exchange of P: chunk out of range"; cP[c.layer].push_back(c.chunk); }
+    for (const ExchangeChunk& c : p.chQ) { if (c.layer < 0 || c.layer >= (int)nm) return "exchange of Q: chunk out of range"; cQ[c.layer].push_back(c.chunk); }
+    for (size_t li = 0; li < nm; ++li) {
+      const LayerDev& L = p.layers[li];
+      auto full = [&](std::vector<int>& c, int elems) {
+        std::sort(c.begin(), c.end());
+        if ((int)c.size() != ceil_div(elems, kExchangeChunk)) return false;
+        for (int k = 0; k < (int)c.size(); ++k) if (c[k] != k) return false;
+        return true;
+      };
+      if (!full(cP[li], L.n * L.r) || !full(cQ[li], L.m * L.r)) return "exchange: every 256 factor elements once" + layer_name(li);
+    }
+  }
+  // ---- second-level sums: every partial of a folded layer in exactly one group, every element of the plane once
+  auto check_fold = [&](const std::vector<FoldJob>& jobs, const char* what, auto src_of, auto dst_of, auto nparts_of, auto nsum_of,
+                        auto plane_of, size_t esz) -> std::string {
+    std::map<std::tuple<size_t, int, int>, std::vector<std::pair<uint32_t, int>>> seen;   // (layer, worker, group) -> (e0, count)
+    for (const FoldJob& j : jobs) {
+      bool placed = false;
+      for (size_t li = 0; li < nm && !placed; ++li) {
+        const int nparts = nparts_of(li), ng = nsum_of(li);
+        if (ng == nparts) continue;                                      // not folded
+        const size_t plane = plane_of(li);
+        const unsigned char* s0 = static_cast<const unsigned char*>(src_of(li));
+        const unsigned char* d0 = static_cast<const unsigned char*>(dst_of(li));
+        const unsigned char* js = static_cast<const unsigned char*>(j.src);
+        if (js < s0 || js >= s0 + (size_t)W * nparts * plane * esz) continue;
+        const size_t part_index = (size_t)(js - s0) / (plane * esz);
+        if ((size_t)(js - s0) % (plane * esz)) return std::string(what) + ": a group does not start on a partial sum";
+        const int w = (int)(part_index / nparts), first = (int)(part_index % nparts);
+        if (first % kFoldGroup) return std::string(what) + ": a group does not start on a multiple of the group size";
+        const int g = first / kFoldGroup;
+        if (j.count != std::min(kFoldGroup, nparts - first) || j.plane != plane || (j.is_double != 0) != (esz == 8))
+          return std::string(what) + ": a group's extent is wrong";
+        if (static_cast<unsigned char*>(j.dst) != d0 + ((size_t)w * ng + g) * plane * esz) return std::string(what) + ": a group's sum goes to the wrong place";
+        seen[{li, w, g}].push_back({j.e0, 0});
+        placed = true;
+      }
+      if (!placed) return std::string(what) + ": a job outside every folded layer";
+    }
+    for (size_t li = 0; li < nm; ++li) {
+      const int nparts = nparts_of(li), ng = nsum_of(li);
+      if (ng == nparts) { if (nparts > kFoldAbove && !p.resident) return std::string(what) + ": a layer with many partial sums is not folded"; continue; }
+      if (ng != ceil_div(nparts, kFoldGroup)) return std::string(what) + ": group count";
+      for (int w = 0; w < W; ++w)
+        for (int g = 0; g < ng; ++g) {
+          auto it = seen.find({li, w, g});
+          if (it == seen.end()) return std::string(what) + ": a group is never summed" + layer_name(li);
+          auto& v = it->second;
+          std::sort(v.begin(), v.end());
+          uint32_t e = 0;
+          for (auto& x : v) { if (x.first != e) return std::string(what) + ": a plane's elements twice or never" + layer_name(li); e += kFoldElems; }
+          if (e < plane_of(li)) return std::string(what) + ": a plane's last elements are never summed" + layer_name(li);
+        }
+    }
+    return "";
+  };
+  {
+    std::string e = check_fold(p.foldP, "fold of P partials", [&](size_t li) { return (const void*)p.layers[li].Ppart; },
+                               [&](size_t li) { return (const void*)p.layers[li].Psum; }, [&](size_t li) { return p.layers[li].ncc; },
+                               [&](size_t li) { return p.layers[li].nps; }, [&](size_t li) { return (size_t)p.layers[li].n * p.RP; }, 4);
+    if (e.empty())
+      e = check_fold(p.foldQ, "fold of Q partials", [&](size_t li) { return (const void*)p.layers[li].Qpart; },
+                     [&](size_t li) { return (const void*)p.layers[li].Qsum; }, [&](size_t li) { return p.layers[li].nrb; },
+                     [&](size_t li) { return p.layers[li].nqs; }, [&](size_t li) { return (size_t)p.layers[li].m * p.RP; }, 4);
+    if (e.empty())
+      e = check_fold(p.foldG, "fold of block Grams", [&](size_t li) { return (const void*)p.layers[li].gram_part; },
+                     [&](size_t li) { return (const void*)p.layers[li].gram_sum; }, [&](size_t li) { return p.layers[li].npb; },
+                     [&](size_t li) { return p.layers[li].ngs; }, [&](size_t li) { return (size_t)p.RP * p.RP; }, 8);
+    if (!e.empty()) return e;
+  }
+  return "";
+}
+}  // namespace
+
+static thread_local int g_plan_defect = 0;
+int lqsgd_test_plan_defect(int32_t kind) {
+  if (kind < 0 || kind > 5) return LQSGD_ERR_INVALID_ARG;
+  g_plan_defect = kind;
+  return LQSGD_OK;
+}
+
+int lqsgd_plan_check(const lqsgd_shape* shapes, int32_t n_layers, const lqsgd_config* cfg, int32_t sm_count, char* msg,
+                     size_t msg_len) {
+  if (msg && msg_len) msg[0] = 0;
+  const int rc = check_config(shapes, n_layers, cfg);
+  if (rc != LQSGD_OK) return rc;
+  if (sm_count < 1 || sm_count > 1024) return LQSGD_ERR_INVALID_ARG;
+  // a base address that keeps every piece's address distinct and non-null (nothing is dereferenced)
+  std::vector<std::string> found;
+  for (int allow_resident = 1; allow_resident >= 0; --allow_resident) {
+    Plan p;
+    make_plan(shapes, n_layers, *cfg, reinterpret_cast<void*>((uintptr_t)1 << 40), sm_count, p, allow_resident != 0);
+    if (g_plan_defect) {                       // test support: see lqsgd_test_plan_defect
+      const int kind = g_plan_defect;
+      auto drop_last = [](auto& v) { if (!v.empty()) v.pop_back(); };
+      if (kind == 1) { if (!p.tctiles1.empty()) drop_last(p.tctiles1); else if (!p.stiles1.empty()) drop_last(p.stiles1); else if (!p.tiles1.empty()) drop_last(p.tiles1); else drop_last(p.rtiles); }
+      if (kind == 2) {
+        auto& v = !p.tctiles2.empty() ? p.tctiles2 : p.tiles2;
+        if (v.size() >= 2) {                   // two tiles of one (layer, worker, column chunk), if there are such
+          for (size_t i = 1; i < v.size(); ++i)
+            if (v[i].layer == v[0].layer && v[i].worker == v[0].worker && v[i].col0 == v[0].col0) { v[i].part = v[0].part; break; }
+          if (p.layers[v[0].layer].nrb == 1) v[0].part = 1;
+        }
+      }
+      if (kind == 3) { if (!p.tctiles3.empty()) drop_last(p.tctiles3); else if (!p.stiles3.empty()) drop_last(p.stiles3); else drop_last(p.tiles3); }
+      if (kind == 4) { if (!p.foldQ.empty()) drop_last(p.foldQ); else if (!p.foldG.empty()) drop_last(p.foldG); else drop_last(p.foldP); }
+      if (kind == 5) drop_last(p.chQ);
+    }
+    const std::string e = check_plan(p);
+    if (!e.empty()) {
+      if (msg && msg_len) { std::strncpy(msg, e.c_str(), msg_len - 1); msg[msg_len - 1] = 0; }
+      g_plan_defect = 0;
+      return LQSGD_ERR_PLAN;
+    }
+    if (!p.resident) break;                     // the same plan again
+  }
+  g_plan_defect = 0;
   return LQSGD_OK;
 }
 

@@ -20,8 +20,12 @@ DEV = "cuda:0"
 
 
 def make(w: wl.Workload, **kw):
-    return B.LQSGD(w.layers, w.rank, kw.pop("bits_p", w.bits), kw.pop("bits_q", None), alpha=w.alpha,
+    comp = B.LQSGD(w.layers, w.rank, kw.pop("bits_p", w.bits), kw.pop("bits_q", None), alpha=w.alpha,
                    workers=w.workers, seed=w.seed, **kw)
+    # every context these tests run on: its work tables pass the library's own host-side check for this device
+    sms = torch.cuda.get_device_properties(comp.device).multi_processor_count
+    assert B.plan_check(comp.layers, comp.cfg, sms) == ""
+    return comp
 
 
 def new_oracle(comp: B.LQSGD):
