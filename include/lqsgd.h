@@ -174,7 +174,10 @@ int lqsgd_workspace_bytes(const lqsgd_shape* host_shapes, int32_t n_layers,
  * contents until lqsgd_destroy().  Initialises E_0 = 0 and Q_0 ~ N(0,1) from config->seed
  * (Alg. 1 initialisation; the same Q_0 for every worker) and uploads the planning tables:
  * it issues copies and a memset on the legacy default stream and synchronises it.
- * The context itself is host memory owned by the library. */
+ * The context itself is host memory owned by the library.  Device memory is never allocated; a context whose layer set
+ * has both large layers and small ones with rows that are not 16-byte aligned also owns one non-blocking CUDA stream
+ * and two events (released by lqsgd_destroy): in every pass the small layers' kernel runs on that stream beside the
+ * large layers' kernel, forked from and joined to the caller's stream inside the call, also under stream capture. */
 int lqsgd_create(const lqsgd_shape* host_shapes, int32_t n_layers, const lqsgd_config* host_config,
                  void* dev_workspace, size_t workspace_bytes, lqsgd_ctx** ctx_out);
 
