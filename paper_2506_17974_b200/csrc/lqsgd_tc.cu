@@ -4,9 +4,9 @@
 // CUDA cores can issue at HBM speed.  These kernels run them on tcgen05, with fp32 accumulators
 // in tensor memory (TMEM) and every fp32 operand fed as a sum of narrow terms.
 //
-// Pass 2 (Q_w = M_w^T P_bar, Alg. 1).  One tcgen05.mma with M = 128 costs about 90 cycles
-// whatever N <= 128 is (the feed of the A operand bounds it), so the streamed matrix must pass
-// through the tensor core once, with as few instructions per byte as possible:
+// Pass 2 (Q_w = M_w^T P_bar, Alg. 1).  What a tcgen05.mma with M = 128 costs hardly depends on N <= 128
+// (timing the first versions of this kernel: the feed of the A operand bounds it), so the streamed matrix must
+// pass through the tensor core once, with as few instructions per byte as possible:
 //   * M (the A operand, 128 columns of one worker's M per tile, lane = column) is split into two
 //     bf16 terms, a = a1 + a2 (a1 the truncation of a to 8 mantissa bits, a2 = rn(a - a1): 16
 //     significant bits, |a - a1 - a2| <= 2^-17 |a|), stored as a bf16 pair in ONE 32-bit TMEM
