@@ -283,27 +283,35 @@ __device__ __forceinline__ void p_chol_body(const Tables& t, const FactorBlock f
   }
   __syncthreads();
   if (tid < RP) { S.diag0[tid] = S.A[tid][tid]; S.dead[tid] = 0; S.invd[tid] = 1.0; }
-  __syncthreads();
+  // Right-looking, ONE barrier per step: column j stays unscaled while the steps run (the update of entry (i, k)
+  // takes a_ij a_kj (1 / sqrt d_j)^2 instead of (a_ij / sqrt d_j)(a_kj / sqrt d_j)); the columns are scaled at the end.  The
+  // threads form a 16 x 16 grid over the trailing block's rows and columns (no index arithmetic with divisions).
+  static_assert(NT == 256, "16 x 16 threads");
+  const int ta = tid >> 4, tb = tid & 15;
   for (int j = 0; j < r; ++j) {
+    __syncthreads();                       // the updates of step j - 1 (and the initial values) are in place
     const double d = S.A[j][j];
     const bool ok = (d > kPivotEps * S.diag0[j]) && (d < INFINITY);   // false for nan too
-    const double inv = ok ? rsqrt(d) : 1.0;
-    const double ljj = ok ? d * inv : 1.0;
-    __syncthreads();                       // everybody has read the pivot
-    for (int i = j + tid; i < r; i += NT) {
-      if (i == j) { S.A[j][j] = ljj; S.invd[j] = inv; if (!ok) S.dead[j] = 1; }
-      else S.A[i][j] = ok ? S.A[i][j] * inv : 0.0;
-    }
-    __syncthreads();
+    const double inv = ok ? rsqrt(d) : 1.0;       // (hardware seed plus refinement: a division is a much longer sequence)
+    if (tid == 0) { S.invd[j] = inv; if (!ok) S.dead[j] = 1; }
     if (ok) {
-      const int w = r - j - 1;             // trailing block: rows and columns j+1 .. r-1, lower triangle
-      for (int e = tid; e < w * w; e += NT) {
-        const int i = j + 1 + e / w, k = j + 1 + e % w;
-        if (k <= i) S.A[i][k] -= S.A[i][j] * S.A[k][j];
+      const double inv2 = inv * inv;
+      for (int i = j + 1 + ta; i < r; i += 16) {
+        const double aij = S.A[i][j] * inv2;
+        for (int k = j + 1 + tb; k <= i; k += 16) S.A[i][k] -= aij * S.A[k][j];
       }
     }
-    __syncthreads();                       // the next pivot is read only after its last update
   }
+  __syncthreads();
+  // L: column j of the lower triangle times 1 / sqrt d_j; a dropped column is that of the identity
+  for (int e = tid; e < r * RP; e += NT) {
+    const int i = e / RP, j = e - i * RP;
+    if (j < r && j <= i) {
+      const bool deadj = S.dead[j] != 0;
+      S.A[i][j] = (i == j) ? (deadj ? 1.0 : S.A[j][j] * S.invd[j]) : (deadj ? 0.0 : S.A[i][j] * S.invd[j]);
+    }
+  }
+  __syncthreads();
   double* dst = L.chol + (size_t)fb.worker * (RP * RP + 2 * RP);
   for (int e = tid; e < RP * RP; e += NT) dst[e] = S.A[e / RP][e % RP];
   if (tid < RP) { dst[RP * RP + tid] = S.invd[tid]; dst[RP * RP + RP + tid] = S.dead[tid] ? 1.0 : 0.0; }
