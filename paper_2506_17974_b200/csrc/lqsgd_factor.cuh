@@ -357,17 +357,21 @@ __device__ __forceinline__ void p_apply_body(const Tables& t, const FactorBlock 
     //   o[j] = (p[j] - sum_{k<j} o[k] L[j][k]) / L[j][j];   a dropped column gives 0
     float p[RP];
     load_contig<RP, COH>(L.Praw + ((size_t)fb.worker * n + row) * RP, p);
-    double od[RP];
+    // Column by column: once o[k] is known it is taken out of every later entry.  Each entry still sees its terms in
+    // the order k = 0, 1, ... (the same sums, the same bits as entry by entry), but the updates of one k are
+    // independent of one another, where the sum of one entry is a chain of dependent fp64 operations.
+    double sd[RP];
+#pragma unroll
+    for (int j = 0; j < RP; ++j) sd[j] = (double)p[j];
     bool bad = false;
 #pragma unroll
-    for (int j = 0; j < RP; ++j) {
-      double s = (double)p[j];
+    for (int k = 0; k < RP; ++k) {
+      const double ok_ = (k < L.r && !S.dead[k]) ? sd[k] * S.invd[k] : 0.0;
+      o[k] = (float)ok_;
+      amax = fmaxf(amax, fabsf(o[k]));
+      bad |= !(fabsf(o[k]) < INFINITY);
 #pragma unroll
-      for (int k = 0; k < j; ++k) s = fma(-od[k], S.chol.A[j][k], s);
-      od[j] = (j < L.r && !S.dead[j]) ? s * S.invd[j] : 0.0;
-      o[j] = (float)od[j];
-      amax = fmaxf(amax, fabsf(o[j]));
-      bad |= !(fabsf(o[j]) < INFINITY);
+      for (int j = k + 1; j < RP; ++j) sd[j] = fma(-ok_, S.chol.A[j][k], sd[j]);
     }
     store_contig<RP>(L.P + ((size_t)fb.worker * n + row) * RP, o);
     if (bad) atomicOr(&t.status[fb.layer], 8u);
