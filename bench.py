@@ -685,7 +685,7 @@ def main():
     args = ap.parse_args()
     if args.source_digest:
         for group in (["lqsgd_stream.cu", "lqsgd_stream_common.cuh", "lqsgd_dev.h"],
-                      ["lqsgd_kernels.cu", "lqsgd_factor.cuh", "lqsgd_dev.h"],
+                      ["lqsgd_kernels.cu", "lqsgd_dev.h"],
                       ["lqsgd_tc.cu", "lqsgd_stream_common.cuh", "lqsgd_dev.h"],
                       ["lqsgd_resident.cu", "lqsgd_factor.cuh", "lqsgd_stream_common.cuh", "lqsgd_dev.h"]):
             print(" ".join(group), csrc_digest(group))
