@@ -716,6 +716,16 @@ __device__ __forceinline__ void exchange_body(const Tables& t, const QuantTables
       xfirst[u] = (v1 && u < W) ? ld_in<COH>(src + ((size_t)u * rows + row1) * RP + col1) : 0.f;
   }
   for (int i = tid; i < NLEV - 1; i += NT) S.thr[i] = qt.thr[i];
+  // With at most 7 thresholds (b <= 4) a kernel of its own keeps them in registers and counts the thresholds not
+  // above |x| / s directly (the same number the halving search finds in the ascending table): at ranks 16 and up
+  // this kernel is bound by its instruction count, and the search with its call was half of it.
+  constexpr bool kRegThr = !COH && B >= 2 && B <= 4;
+  constexpr int kNThr = kRegThr ? (1 << (B - 1)) - 1 : 1;
+  float thr_r[kNThr];
+  if constexpr (kRegThr) {
+#pragma unroll
+    for (int i = 0; i < kNThr; ++i) thr_r[i] = __ldg(qt.thr + i);
+  }
   if (tid < WB) *reinterpret_cast<uint32_t*>(&S.codes[tid][CH]) = 0u;     // what a word task reads past the chunk
   float s = 0.f;
   const bool cs = PLAIN ? false : t.col_scales != 0;
@@ -805,7 +815,15 @@ __device__ __forceinline__ void exchange_body(const Tables& t, const QuantTables
         for (int u = 0; u < WB; ++u) {
           if (u < wn) {
             int k = 0;      // k = #{i : |x| / s >= thr[i]}, thr ascending, NLEV - 1 = 2^(B-1) - 1 entries
-            if (s_ok && valid) k = level_of_call(x[u], s, S.thr, NLEV);
+            if (s_ok && valid) {
+              if constexpr (kRegThr) {
+                const float tt = __fdiv_rn(fabsf(x[u]), s);
+#pragma unroll
+                for (int i = 0; i < kNThr; ++i) k += (tt >= thr_r[i]) ? 1 : 0;
+              } else {
+                k = level_of_call(x[u], s, S.thr, NLEV);
+              }
+            }
             const int neg = (valid && x[u] < 0.f) ? 1 : 0;
             S.codes[u][tid] = (uint8_t)((neg << (bits - 1)) | k);   // 0 beyond the factor's end: pads the last byte
             const int sk = neg ? -k : k;
