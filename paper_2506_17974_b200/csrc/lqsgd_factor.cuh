@@ -840,6 +840,14 @@ __device__ __forceinline__ void exchange_body(const Tables& t, const QuantTables
         const int bit0 = 32 * j;
         const int q0 = bit0 / bits;
         uint32_t word = 0;
+        if constexpr (B == 4) {
+          // eight codes per word, one per byte in shared memory (each below 16): byte pairs to nibble pairs, twice
+          const uint32_t* cw = reinterpret_cast<const uint32_t*>(&S.codes[u][8 * j]);
+          auto nib = [](uint32_t x) { x = (x | (x >> 4)) & 0x00FF00FFu; return (x | (x >> 8)) & 0xFFFFu; };
+          word = nib(cw[0]) | (nib(cw[1]) << 16);
+        } else if constexpr (B == 8) {
+          word = *reinterpret_cast<const uint32_t*>(&S.codes[u][4 * j]);
+        } else {
 #pragma unroll
         for (int i = 0; i < 32 / bits + 2; ++i) {
           const int q = q0 + i;
@@ -848,6 +856,7 @@ __device__ __forceinline__ void exchange_body(const Tables& t, const QuantTables
             const uint32_t c = S.codes[u][min(q, CH + 3)];
             word |= (sh >= 0) ? (c << sh) : (c >> (-sh));
           }
+        }
         }
         const int nb = min(4, nbytes - 4 * j);       // bytes of this word inside the stream
         uint8_t* pay = t.payload + (size_t)(w0 + u) * t.payload_stride + pay_off + byte0 + 4 * j;
