@@ -546,6 +546,7 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
     L.nrb = p.resident ? res_nrb[li] : ceil_div(mt.n, tr2);
     L.npb = ceil_div(mt.n, kFactorBlockRows);
     L.nqb = ceil_div(mt.m, kFactorBlockRows);
+    L.qfused = (tc && L.nrb == 1 && !colscales && !p.resident) ? 1 : 0;
     const size_t nm = (size_t)mt.n * mt.m;
     L.E = a.take<float>((size_t)W * nm);
     L.Q = a.take<float>((size_t)mt.m * RP);
@@ -657,7 +658,7 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
       if (one_cta) p.fbS.push_back({li32, w, 0, 0});
       if (!one_cta && RP >= kCholSplitRP) p.fbC.push_back({li32, w, 0, 0});
       for (int b = 0; !one_cta && b < L.npb; ++b) p.fbP.push_back({li32, w, b, 0});
-      for (int b = 0; b < L.nqb; ++b) p.fbQ.push_back({li32, w, b, 0});
+      for (int b = 0; !L.qfused && b < L.nqb; ++b) p.fbQ.push_back({li32, w, b, 0});
     }
     for (int c = 0; c < ceil_div(mt.n * mt.r, kExchangeChunk); ++c) p.chP.push_back({li32, c});
     for (int c = 0; c < ceil_div(mt.m * mt.r, kExchangeChunk); ++c) p.chQ.push_back({li32, c});
@@ -963,7 +964,11 @@ std::string check_plan(const Plan& p) {
         int np = 0;
         for (int b = 0; b < L.npb; ++b) { auto it = blkP.find({k, b}); if (it != blkP.end()) { if (it->second != 1) return "Orthonormalize: a block of rows twice" + layer_name(li); ++np; } }
         if (!((seenS[k] == 1 && np == 0) || (seenS[k] == 0 && np == L.npb))) return "Orthonormalize: every row of P once, by one CTA or by blocks of 128" + layer_name(li);
-        for (int b = 0; b < L.nqb; ++b) { auto it = blkQ.find({k, b}); if (it == blkQ.end() || it->second != 1) return "Q_w reduction: every block of 128 rows of Q once" + layer_name(li); }
+        for (int b = 0; b < L.nqb; ++b) {
+          auto it = blkQ.find({k, b});
+          if (L.qfused ? it != blkQ.end() : (it == blkQ.end() || it->second != 1)) return "Q_w reduction: every block of 128 rows of Q once, or none where pass 2 takes the maxima" + layer_name(li);
+        }
+        if (L.qfused && (!L.tc || L.nrb != 1)) return "Q_w maxima in pass 2 need the whole sum in one tile" + layer_name(li);
       }
     if (blkP.size() + 0 != [&] { size_t t = 0; for (size_t li = 0; li < nm; ++li) for (int w = 0; w < W; ++w) if (!seenS[li * W + w]) t += p.layers[li].npb; return t; }()) return "Orthonormalize: blocks beyond the layers' rows";
     std::vector<std::vector<int>> cP(nm), cQ(nm);
@@ -1281,7 +1286,7 @@ int lqsgd_launches_per_step(const lqsgd_ctx* ctx, int32_t* out) {
   const int iters = std::max(1, ctx->cfg.power_iters);
   const int orth = (p.fbS.empty() ? 0 : 1) + (p.fbP.empty() ? 0 : 2) + (p.fbC.empty() ? 0 : 1);   // one CTA per small layer / Gram (+ Cholesky) + apply
   const int folds = (p.foldP.empty() ? 0 : 1) + (p.foldG.empty() ? 0 : 1) + (p.foldQ.empty() ? 0 : 1);
-  *out = iters * ((p.mats.empty() ? 0 : orth + 3 + folds) + pass1 + pass2) + pass3 + ((p.chV.empty() || vectors_ride(ctx)) ? 0 : 1);
+  *out = iters * ((p.mats.empty() ? 0 : orth + 2 + (p.fbQ.empty() ? 0 : 1) + folds) + pass1 + pass2) + pass3 + ((p.chV.empty() || vectors_ride(ctx)) ? 0 : 1);
   return LQSGD_OK;
 }
 

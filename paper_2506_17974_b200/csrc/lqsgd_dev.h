@@ -50,7 +50,8 @@ struct LayerDev {
   const float* Qsum;          // [W][nqs][m][RP]: Qpart (nqs = nrb) or the folded partials
   const double* gram_sum;     // [W][ngs][RP*RP]: gram_part (ngs = npb) or the folded block Grams
   int32_t nps, nqs, ngs;
-  int32_t pad_;
+  int32_t qfused;             // 1: the tensor-core pass 2 holds the whole sum Q_w (one row chunk) and takes the block maxima of
+                              // |Q_w| itself (its epilogue; p_apply zeroes them first): no q_reduce blocks for this layer
 };
 
 constexpr int kFoldAbove = 64;     // partial sums per layer and worker above which they are folded first

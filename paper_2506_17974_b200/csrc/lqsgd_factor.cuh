@@ -347,6 +347,8 @@ __device__ __forceinline__ void p_apply_body(const Tables& t, const FactorBlock 
     const bool dropped = cholesky_lower<RP, NT, COH>(L, fb.worker, S.chol, S.invd, S.dead, tid);
     if (dropped && fb.blk == 0 && tid == 0) atomicOr(&t.status[fb.layer], 1u);
   }
+  if (L.qfused && fb.blk == 0)                 // the block maxima of |Q_w| that pass 2 will raise start from zero
+    for (int i = tid; i < L.nqb; i += NT) L.maxq[(size_t)fb.worker * L.nqb + i] = 0.f;
   const int row = fb.blk * kFactorBlockRows + tid;
   float o[RP];
 #pragma unroll

@@ -327,6 +327,8 @@ tc_pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, const uint
       const uint32_t taddr = tmem + ((uint32_t)(32 * q) << 16) + db * S::kDStride;
       const int col = tl.col0 + 32 * q + lane;
       float* dst = L.Qpart + (((size_t)tl.worker * L.nrb + tl.part) * L.m + (size_t)min(col, L.m - 1)) * RP;
+      float vmax = 0.f;           // max |Q_w| over this thread's row of Q; a NaN is dropped here and reported below
+      float zsum = 0.f;           // sum of 0 * value: not zero (a NaN) once a value is not finite
 #pragma unroll
       for (int j0 = 0; j0 < RP; j0 += 16) {
         uint32_t a[16], b[16], c[16];
@@ -334,6 +336,11 @@ tc_pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, const uint
         tc_ld16(taddr + RP + j0, b);
         tc_ld16(taddr + 2 * RP + j0, c);
         tc_wait_ld();
+        if (j0 + 16 >= RP) {      // the accumulator is in registers: the MMA thread may have it back
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(d_empty + db);
+        }
         if (col < L.m) {
 #pragma unroll
           for (int j = 0; j < 16; j += 4) {
@@ -343,12 +350,20 @@ tc_pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles, const uint
             o.z = (__uint_as_float(c[j + 2]) + __uint_as_float(b[j + 2])) + __uint_as_float(a[j + 2]);
             o.w = (__uint_as_float(c[j + 3]) + __uint_as_float(b[j + 3])) + __uint_as_float(a[j + 3]);
             *reinterpret_cast<float4*>(dst + j0 + j) = o;
+            vmax = fmaxf(fmaxf(vmax, fmaxf(fabsf(o.x), fabsf(o.y))), fmaxf(fabsf(o.z), fabsf(o.w)));
+            zsum = fmaf(0.f, o.x, fmaf(0.f, o.y, fmaf(0.f, o.z, fmaf(0.f, o.w, zsum))));
           }
         }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(d_empty + db);
+      const bool bad = !(zsum == 0.f);
+      if (L.qfused) {
+        // the tile's 128 columns of M are one block of 128 rows of Q and this is the whole sum (one row chunk): the
+        // block's maximum, which q_reduce would find, is taken here (non-negative floats order like their bits)
+#pragma unroll
+        for (int o = 16; o >= 1; o >>= 1) vmax = fmaxf(vmax, __shfl_xor_sync(0xffffffffu, vmax, o));
+        if (lane == 0) atomicMax(reinterpret_cast<int*>(L.maxq) + (size_t)tl.worker * L.nqb + tl.col0 / kFactorBlockRows, __float_as_int(vmax));
+        if (bad) atomicOr(&t.status[tl.layer], 8u);
+      }
     }
   } else if (warp >= 8) {
     // ---- consumers: M piece -> registers (lane = column) -> bf16 pair -> tensor memory
