@@ -347,7 +347,16 @@ def run_ours(args):
         # a dependent column or a zero scale is a property of the data (it happens with 2-bit codes);
         # a non-finite value or an expired wait would make the timing meaningless
         assert all(s & (B.STATUS_NONFINITE | B.STATUS_TIMEOUT) == 0 for s in status), f"device status flags: {status}"
-        out = {"ms": ms, "repeats": len(blocks), "block_ms_min_max": [blocks[0], blocks[-1]],
+        # the library's own figures of the last round (outside the timed region): codes that sit within one fp32 step
+        # of a decision threshold, the only ones a correct implementation may code differently
+        lst = [comp.step_stats(l) for l in range(len(comp.layers)) if comp.is_matrix(l)]
+        n_codes = sum(x["codes_p"] + x["codes_q"] for x in lst)
+        n_near = sum(x["near_p"] + x["near_q"] for x in lst)
+        quantiser = {"codes": n_codes, "within_one_ulp_of_a_threshold": n_near,
+                     "fraction": n_near / n_codes if n_codes else 0.0,
+                     "min_pivot_ratio": min((x["pivot_ratio"] for x in lst), default=0.0),
+                     "what": "last timed round, all workers, from lqsgd_step_stats"}
+        out = {"ms": ms, "repeats": len(blocks), "block_ms_min_max": [blocks[0], blocks[-1]], "quantiser": quantiser,
                "phases_ms": dict(zip(B.PHASE_NAMES, phases)), "launches": comp.launches_per_step,
                "payload": comp.payload_nbytes, "clocks": sampler.summary() if sampler else None, "graph_ms": graph_ms,
                "flagged_layers": sum(1 for x in status if x),
@@ -507,6 +516,7 @@ def run_ours(args):
                        "(larger than L2); the timed `value` above uses plain launches"} if res.get("graph_ms") else None,
         "compression_ratio": 4 * sum(n * m for n, m in wl_obj.layers) / res["payload"],
         "payload_bytes_per_worker": res["payload"],
+        "quantiser": res["quantiser"],
     }
 
     def compact(w, r):

@@ -297,6 +297,29 @@ int lqsgd_set_state(lqsgd_ctx* ctx, int32_t which, int32_t layer, int32_t worker
  * synchronises cuda_stream. */
 int lqsgd_status(const lqsgd_ctx* ctx, uint32_t* host_flags, void* cuda_stream);
 
+/* Figures of the last round for one layer (a logging aid; nothing on the round's path computes them). */
+typedef struct lqsgd_layer_stats {
+  uint32_t status;         /* the layer's status word (LQSGD_STATUS_*) */
+  int32_t rank_eff;        /* r_eff; 0 for a 1-D tensor, whose other fields are then 0 except payload_bytes */
+  float scale_p, scale_q;  /* s_P, s_Q of Eq. 4's normalisation (LQSGD_FLAG_COLUMN_SCALES: the largest column scale) */
+  float pivot_ratio;       /* conditioning of the factor given to Orthonormalize (Algorithm 1): with M Q = P R, R upper
+                              triangular, min_j R_jj / max_j R_jj, the smallest over this GPU's workers; 0 when a column
+                              was dropped (LQSGD_STATUS_DEPENDENT_COLUMN) */
+  uint32_t pad_;
+  uint64_t codes_p, codes_q; /* factor entries quantised by Eq. 4 over this GPU's workers: W n r_eff and W m r_eff
+                                (0 with bits 32) */
+  uint64_t near_p, near_q;   /* of them, entries whose |x| / s lies within one fp32 step of a decision threshold: the
+                                two fp32 neighbours of |x| / s fall into different levels.  Only for these may an
+                                implementation that rounds |x| / s differently in the last place produce another code */
+  uint64_t payload_bytes;    /* this layer's bytes in one worker's payload (scales + P stream + Q stream, or the 1-D
+                                tensor's values) */
+} lqsgd_layer_stats;
+
+/* Fills host_out for one layer from what the last step left in the workspace (one small kernel over the layer's
+ * factors on cuda_stream, then a copy of three words); synchronises cuda_stream.  Call it after a step on the same
+ * stream, or after synchronising the step's stream.  Matrix layers whose round has not run yet report zeros. */
+int lqsgd_step_stats(const lqsgd_ctx* ctx, int32_t layer, lqsgd_layer_stats* host_out, void* cuda_stream);
+
 /* Profiling aid.  host_events: LQSGD_N_PHASES + 1 cudaEvent_t handles owned by the caller (or
  * NULL to cancel).  The NEXT lqsgd_step records them on its stream at the phase boundaries and
  * then forgets them: event i before phase i, the last one after phase LQSGD_N_PHASES - 1.

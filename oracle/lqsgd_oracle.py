@@ -118,6 +118,27 @@ def log_quantize(x, s, bits, alpha, return_margin=False):
     return codes
 
 
+def near_threshold_count(x, s, bits, alpha):
+    """How many entries of x have |x|/s (an fp32 number) within one fp32 step of a decision
+    threshold of Eq. 4's nearest-level rule: the two fp32 neighbours of |x|/s get different
+    level indices.  These are the codes a last-place difference in |x|/s can change."""
+    L = magnitude_levels(bits)
+    x32 = np.asarray(x, dtype=np.float32)
+    s32 = np.asarray(s, dtype=np.float32)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        t = (np.abs(x32) / s32).astype(np.float32)
+    ok = np.broadcast_to((s32 > 0) & np.isfinite(s32), x32.shape) & np.isfinite(t)
+    t = np.where(ok, t, np.float32(0))
+    below = np.where(t > 0, np.nextafter(t, np.float32(-np.inf)), np.float32(0)).astype(np.float32)
+    above = np.nextafter(t, np.float32(np.inf)).astype(np.float32)
+
+    def level(u):
+        u = np.minimum(u.astype(np.float64), np.finfo(np.float32).max)
+        return np.clip(np.floor((L - 1) * compand(u, alpha) + 0.5), 0, L - 1)
+
+    return int(np.count_nonzero(ok & (level(below) != level(above))))
+
+
 def signed_levels(codes, bits):
     """Signed level index (-1)^sign * k of each code, as int64."""
     codes = np.asarray(codes).astype(np.int64)
@@ -196,6 +217,26 @@ def orthonormalize(P):
         else:
             A[:, j] /= np.sqrt(norm1)
     return A, dependent
+
+
+def pivot_ratio(P):
+    """Conditioning of the factor given to Orthonormalize: with P = P_orth R (R upper triangular,
+    positive diagonal; R_jj is the norm left of column j after the earlier columns are taken
+    out), min_j R_jj / max_j R_jj; 0 when a column is dropped as dependent."""
+    A = np.array(P, dtype=np.float64, copy=True)
+    r = A.shape[1]
+    diag = np.zeros(r)
+    for j in range(r):
+        norm0 = float(A[:, j] @ A[:, j])
+        for i in range(j):
+            A[:, j] -= (A[:, i] @ A[:, j]) * A[:, i]
+        norm1 = float(A[:, j] @ A[:, j])
+        if norm0 == 0.0 or norm1 <= RANK_EPS * norm0:
+            A[:, j] = 0.0
+        else:
+            diag[j] = np.sqrt(norm1)
+            A[:, j] /= diag[j]
+    return float(diag.min() / diag.max()) if diag.max() > 0 else 0.0
 
 
 # ----------------------------------------------------------------------------

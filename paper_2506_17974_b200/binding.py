@@ -40,7 +40,7 @@ NOALLOC_MAX_ROWS = 65536
 
 EXPORTED = [
     "lqsgd_workspace_bytes", "lqsgd_create", "lqsgd_step", "lqsgd_step_update", "lqsgd_step_host", "lqsgd_payload_bytes",
-    "lqsgd_payload", "lqsgd_payload_layout", "lqsgd_get_state", "lqsgd_set_state", "lqsgd_status",
+    "lqsgd_payload", "lqsgd_payload_layout", "lqsgd_get_state", "lqsgd_set_state", "lqsgd_status", "lqsgd_step_stats",
     "lqsgd_orthonormalize_noalloc",
     "lqsgd_round_begin", "lqsgd_round_pack", "lqsgd_round_reduce", "lqsgd_round_end", "lqsgd_exchange_view",
     "lqsgd_launches_per_step", "lqsgd_set_phase_events", "lqsgd_release_graph_tables", "lqsgd_test_expire_wait", "lqsgd_round_timeline", "lqsgd_check_guards", "lqsgd_plan_check", "lqsgd_test_plan_defect", "lqsgd_destroy", "lqsgd_strerror", "lqsgd_last_cuda_error", "lqsgd_version",
@@ -61,6 +61,12 @@ class LayerLayout(C.Structure):
     _fields_ = [("is_matrix", C.c_int32), ("rank_eff", C.c_int32), ("scale_offset", C.c_uint64),
                 ("p_offset", C.c_uint64), ("p_bytes", C.c_uint64), ("q_offset", C.c_uint64),
                 ("q_bytes", C.c_uint64), ("vec_offset", C.c_uint64), ("vec_bytes", C.c_uint64)]
+
+
+class LayerStats(C.Structure):
+    _fields_ = [("status", C.c_uint32), ("rank_eff", C.c_int32), ("scale_p", C.c_float), ("scale_q", C.c_float),
+                ("pivot_ratio", C.c_float), ("pad_", C.c_uint32), ("codes_p", C.c_uint64), ("codes_q", C.c_uint64),
+                ("near_p", C.c_uint64), ("near_q", C.c_uint64), ("payload_bytes", C.c_uint64)]
 
 
 class LqsgdError(RuntimeError):
@@ -97,6 +103,7 @@ def load_library() -> C.CDLL:
     lib.lqsgd_get_state.argtypes = [vp, i32, i32, i32, vp, vp]
     lib.lqsgd_set_state.argtypes = [vp, i32, i32, i32, vp, vp]
     lib.lqsgd_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
+    lib.lqsgd_step_stats.argtypes = [vp, i32, C.POINTER(LayerStats), vp]
     lib.lqsgd_launches_per_step.argtypes = [vp, C.POINTER(i32)]
     lib.lqsgd_orthonormalize_noalloc.argtypes = [vp, vp, i32, i32, vp, vp]
     lib.lqsgd_set_phase_events.argtypes = [vp, C.POINTER(vp)]
@@ -387,6 +394,12 @@ class LQSGD:
         assert tuple(v.shape) == tuple(shape), (v.shape, shape)
         _check(self.lib.lqsgd_set_state(self.ctx, which, layer, worker, C.c_void_p(v.data_ptr()), self._stream_ptr()))
         torch.cuda.current_stream(self.device).synchronize()      # v may be a temporary
+
+    def step_stats(self, layer: int) -> dict:
+        """Figures of the last round for one layer (lqsgd_layer_stats as a dict)."""
+        st = LayerStats()
+        _check(self.lib.lqsgd_step_stats(self.ctx, layer, C.byref(st), self._stream_ptr()))
+        return {name: getattr(st, name) for name, _ in LayerStats._fields_ if name != "pad_"}
 
     def status(self) -> List[int]:
         flags = (C.c_uint32 * len(self.layers))()

@@ -6,9 +6,9 @@ import shutil
 import subprocess
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-SOURCES = [os.path.join(_HERE, "csrc", f) for f in ("lqsgd_kernels.cu", "lqsgd_api.cu", "lqsgd_noalloc.cu", "lqsgd_stream.cu", "lqsgd_tc.cu", "lqsgd_resident.cu")]
+SOURCES = [os.path.join(_HERE, "csrc", f) for f in ("lqsgd_kernels.cu", "lqsgd_api.cu", "lqsgd_noalloc.cu", "lqsgd_stream.cu", "lqsgd_tc.cu", "lqsgd_resident.cu", "lqsgd_stats.cu")]
 HEADERS = [os.path.join(_HERE, "csrc", "lqsgd_dev.h"), os.path.join(_HERE, "csrc", "lqsgd_stream_common.cuh"),
-           os.path.join(_HERE, "csrc", "lqsgd_factor.cuh"),
+           os.path.join(_HERE, "csrc", "lqsgd_factor.cuh"), os.path.join(_HERE, "csrc", "lqsgd_stats.h"),
            os.path.join(os.path.dirname(_HERE), "include", "lqsgd.h")]
 TARGET = os.path.join(_HERE, "liblqsgd.so")
 

@@ -2,6 +2,7 @@
 // table upload and the per-step launch sequence behind the C ABI of include/lqsgd.h.
 #include "../../include/lqsgd.h"
 #include "lqsgd_dev.h"
+#include "lqsgd_stats.h"
 
 #include <nvtx3/nvToolsExt.h>
 
@@ -133,6 +134,7 @@ struct Plan {
   float *d_thrP = nullptr, *d_thrQ = nullptr, *d_deqP = nullptr, *d_deqQ = nullptr;
   void** d_ptrs = nullptr;                    // kPtrSets pointer tables, see prepare_step for the layout of one
   uint32_t* d_status = nullptr;
+  unsigned long long* d_stats = nullptr;      // [4]: result words of lqsgd_step_stats (one layer at a time)
   uint8_t* d_payload = nullptr;
   float* d_xscales = nullptr;                 // [2][n_mat][ns] scales the ranks agree on (split exchange); ns = 1, or RP per column
   int xscale_ns = 1;
@@ -694,6 +696,7 @@ void make_plan(const lqsgd_shape* shapes, int n_layers, const lqsgd_config& cfg,
       }
   }
   p.d_status = a.take<uint32_t>(p.mats.size());
+  p.d_stats = a.take<unsigned long long>(4);
   p.d_payload = a.take<uint8_t>((size_t)W * p.payload_stride);
   p.xscale_ns = colscales ? RP : 1;
   p.d_xscales = a.take<float>(2 * p.mats.size() * p.xscale_ns);
@@ -1813,6 +1816,67 @@ int lqsgd_status(const lqsgd_ctx* c, uint32_t* host_flags, void* cuda_stream) {
   }
   CK(cudaStreamSynchronize(st));
   for (size_t i = 0; i < p.mats.size(); ++i) host_flags[p.mats[i].user_index] = tmp[i];
+  return LQSGD_OK;
+}
+
+int lqsgd_step_stats(const lqsgd_ctx* c, int32_t layer, lqsgd_layer_stats* out, void* cuda_stream) {
+  if (!c || !out) return LQSGD_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= (int)c->shapes.size()) return LQSGD_ERR_OUT_OF_RANGE;
+  const Plan& p = c->plan;
+  std::memset(out, 0, sizeof(*out));
+  const lqsgd_layer_layout& lay = p.layout[layer];
+  const bool cs = (c->cfg.flags & LQSGD_FLAG_COLUMN_SCALES) != 0;
+  if (!lay.is_matrix) {
+    const bool quantised = (c->cfg.flags & LQSGD_FLAG_QUANTIZE_VECTORS) && c->cfg.bits_p != 32;
+    out->payload_bytes = lay.vec_bytes + (quantised ? 4 : 0);        // its scale travels too
+    return LQSGD_OK;
+  }
+  out->payload_bytes = (cs ? 8 * (uint64_t)lay.rank_eff : 8) + lay.p_bytes + lay.q_bytes;
+  int li = -1;
+  for (size_t i = 0; i < p.mats.size(); ++i)
+    if (p.mats[i].user_index == layer) li = (int)i;
+  if (li < 0) return LQSGD_ERR_OUT_OF_RANGE;
+  const MatHost& mh = p.mats[li];
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const unsigned long long init[4] = {0ull, 0ull, ~0ull, 0ull};
+  CK(cudaMemcpyAsync(p.d_stats, init, sizeof(init), cudaMemcpyHostToDevice, st));
+  StatsArgs a{};
+  a.layers = p.d_layers + li;
+  a.thr_p = p.d_thrP;
+  a.thr_q = p.d_thrQ;
+  a.nthr_p = c->cfg.bits_p == 32 ? 0 : (1 << (c->cfg.bits_p - 1)) - 1;
+  a.nthr_q = c->cfg.bits_q == 32 ? 0 : (1 << (c->cfg.bits_q - 1)) - 1;
+  a.RP = p.RP;
+  a.W = p.W;
+  a.column_scales = cs ? 1 : 0;
+  a.out = p.d_stats;
+  CK(launch_stats(a, 1, st));
+  unsigned long long res[4];
+  float sc[2 * kMaxRank];
+  uint32_t status = 0;
+  const int ns = cs ? 2 * p.RP : 2;
+  CK(cudaMemcpyAsync(res, p.d_stats, sizeof(res), cudaMemcpyDeviceToHost, st));
+  CK(cudaMemcpyAsync(sc, p.layers[li].scales, ns * sizeof(float), cudaMemcpyDeviceToHost, st));
+  CK(cudaMemcpyAsync(&status, p.d_status + li, sizeof(status), cudaMemcpyDeviceToHost, st));
+  CK(cudaStreamSynchronize(st));
+  out->status = status;
+  out->rank_eff = mh.r;
+  if (cs) {
+    for (int j = 0; j < mh.r; ++j) {
+      out->scale_p = std::max(out->scale_p, sc[j]);
+      out->scale_q = std::max(out->scale_q, sc[p.RP + j]);
+    }
+  } else {
+    out->scale_p = sc[0];
+    out->scale_q = sc[1];
+  }
+  const uint32_t ratio_bits = (uint32_t)(res[2] & 0xffffffffull);
+  std::memcpy(&out->pivot_ratio, &ratio_bits, 4);
+  if (ratio_bits == 0xffffffffu) out->pivot_ratio = 0.f;
+  out->codes_p = c->cfg.bits_p == 32 ? 0 : (uint64_t)p.W * mh.n * mh.r;
+  out->codes_q = c->cfg.bits_q == 32 ? 0 : (uint64_t)p.W * mh.m * mh.r;
+  out->near_p = res[0];
+  out->near_q = res[1];
   return LQSGD_OK;
 }
 

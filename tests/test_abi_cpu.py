@@ -31,6 +31,7 @@ def test_library_exports_every_declared_symbol(lib):
 
 def test_config_struct_matches_header_layout():
     assert C.sizeof(B.Config) == 48 and C.sizeof(B.Shape) == 8 and C.sizeof(B.LayerLayout) == 64
+    assert C.sizeof(B.LayerStats) == 64 and B.LayerStats.codes_p.offset == 24 and B.LayerStats.payload_bytes.offset == 56
 
 
 def test_workspace_bytes_covers_the_persistent_state(lib):

@@ -226,3 +226,42 @@ def test_pack_layout_and_size(bits):
     if bits == 3:
         # 5,1,7 -> bits 101 | 001<<3 | 111<<6 = 0b1_1100_1101 -> bytes CD 01
         assert orc.pack_codes(np.array([5, 1, 7], np.uint8), 3).tolist() == [0xCD, 0x01]
+
+
+def test_near_threshold_count_on_a_hand_worked_threshold():
+    """b = 2, alpha = 3: the single decision point sits at compand = 1/2, i.e. |x|/s = (sqrt(4) - 1)/3 = 1/3
+    exactly.  fp32(1/3) lies just above 1/3, so of nine consecutive fp32 numbers centred on it exactly two
+    have neighbours on both sides of the threshold: fp32(1/3) itself and the number below it."""
+    c = np.float32(1.0) / np.float32(3.0)
+    assert float(c) > 1.0 / 3.0
+    xs = [c]
+    for _ in range(4):
+        xs.insert(0, np.nextafter(xs[0], np.float32(0)))
+        xs.append(np.nextafter(xs[-1], np.float32(1)))
+    flags = [orc.near_threshold_count(np.array([x], dtype=np.float32), np.float32(1), 2, 3.0) for x in xs]
+    assert flags == [0, 0, 0, 1, 1, 0, 0, 0, 0]
+    # the sign and the scale do not matter (|x|/s is the same fp32 number for a power-of-two scale)
+    assert orc.near_threshold_count(-np.array(xs, dtype=np.float32) * np.float32(8), np.float32(8), 2, 3.0) == 2
+    # zero, a zero scale, and values far from every threshold count nothing
+    assert orc.near_threshold_count(np.zeros(5, dtype=np.float32), np.float32(1), 4, 127.0) == 0
+    assert orc.near_threshold_count(np.ones(5, dtype=np.float32), np.float32(0), 4, 127.0) == 0
+    assert orc.near_threshold_count(np.array([1.0, 0.5], dtype=np.float32), np.float32(1), 2, 3.0) == 0
+
+
+def test_near_threshold_count_agrees_with_brute_force_over_the_thresholds():
+    """Against the definition written with exact thresholds: an entry counts when some decision point b_k
+    satisfies below(t) < b_k <= above(t).  Values are planted on and next to every threshold of several
+    quantisers, among random ones."""
+    rng = np.random.default_rng(5)
+    for bits, alpha in [(2, 3.0), (3, 15.0), (4, 127.0), (8, 127.0)]:
+        L = orc.magnitude_levels(bits)
+        b = np.expm1((np.arange(L - 1) + 0.5) / (L - 1) * np.log1p(alpha)) / alpha          # exact decision points
+        near = np.float32(b)
+        planted = np.concatenate([near, np.nextafter(near, np.float32(0)), np.nextafter(near, np.float32(2)),
+                                  np.nextafter(np.nextafter(near, np.float32(2)), np.float32(2))])
+        x = np.concatenate([planted, rng.random(2000).astype(np.float32)]).astype(np.float32)
+        lo = np.where(x > 0, np.nextafter(x, np.float32(-1)), np.float32(0)).astype(np.float64)
+        hi = np.nextafter(x, np.float32(2)).astype(np.float64)
+        want = int(np.count_nonzero(((lo[:, None] < b[None, :]) & (b[None, :] <= hi[:, None])).any(axis=1)))
+        assert want >= 2 * (L - 1)
+        assert orc.near_threshold_count(x, np.float32(1), bits, alpha) == want, (bits, alpha)

@@ -327,3 +327,19 @@ def test_several_power_iterations_option():
     # one iteration is Algorithm 1 as it stands
     one = orc.layer_round(G, E, Q0, 4, 4, 127.0)
     assert np.array_equal(one["G_hat"], orc.layer_round(G, E, Q0, 4, 4, 127.0, power_iters=1)["G_hat"])
+
+
+def test_pivot_ratio_is_the_diagonal_of_the_qr_factor():
+    """pivot_ratio against LAPACK: min |R_jj| / max |R_jj| of numpy's QR; a hand case; a dependent column."""
+    A = np.zeros((4, 2))
+    A[0, 0], A[1, 1], A[0, 1] = 3.0, 1.0, 5.0          # R = [[3, 5], [0, 1]]
+    assert orc.pivot_ratio(A) == pytest.approx(1.0 / 3.0, rel=1e-14)
+    rng = np.random.default_rng(11)
+    for n, r in [(50, 1), (40, 5), (300, 16)]:
+        X = rng.standard_normal((n, r)) * np.logspace(0, -3, r)
+        d = np.abs(np.diag(np.linalg.qr(X)[1]))
+        assert orc.pivot_ratio(X) == pytest.approx(d.min() / d.max(), rel=1e-10)
+    X = rng.standard_normal((30, 3))
+    X[:, 2] = X[:, 0] - 2 * X[:, 1]
+    assert orc.pivot_ratio(X) == 0.0
+    assert orc.pivot_ratio(np.zeros((6, 2))) == 0.0
