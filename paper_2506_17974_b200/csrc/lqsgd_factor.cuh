@@ -72,9 +72,10 @@ constexpr double kPivotEps = 1e-10;
 template <int RP> struct ReduceGramSmem { alignas(16) float rows[kFactorBlockRows][RP]; };   // the block's rows (fp32: they are fp32 data)
 
 template <int RP, int NT, bool COH>
-__device__ __forceinline__ void p_reduce_gram_body(const Tables& t, const FactorBlock fb, int tid, void* smem) {
+__device__ __forceinline__ void p_reduce_gram_body(const Tables& t, const FactorBlock fb, int tid, void* smem,
+                                                   const LayerDev* staged = nullptr) {
   auto& S = *static_cast<ReduceGramSmem<RP>*>(smem);
-  const LayerDev& L = t.layers[fb.layer];
+  const LayerDev& L = staged ? *staged : t.layers[fb.layer];   // staged: the wrapper's copy of the entry
   const int n = L.n;
   if (tid < kFactorBlockRows) {
     const int row = fb.blk * kFactorBlockRows + tid;
@@ -263,9 +264,10 @@ template <int RP, int NT> struct CholOnceSmem {
 };
 
 template <int RP, int NT, bool COH>
-__device__ __forceinline__ void p_chol_body(const Tables& t, const FactorBlock fb, int tid, void* smem) {
+__device__ __forceinline__ void p_chol_body(const Tables& t, const FactorBlock fb, int tid, void* smem,
+                                            const LayerDev* staged = nullptr) {
   auto& S = *static_cast<CholOnceSmem<RP, NT>*>(smem);
-  const LayerDev& L = t.layers[fb.layer];
+  const LayerDev& L = staged ? *staged : t.layers[fb.layer];   // staged: the wrapper's copy of the entry
   const int r = L.r;
   for (int e = tid; e < RP * RP; e += NT) {
     const double* gp = L.gram_sum + (size_t)fb.worker * L.ngs * (RP * RP) + e;
@@ -332,10 +334,11 @@ template <int RP, int NT> struct ApplySmem {
 
 // One block of kFactorBlockRows rows of one worker's P: thread tid < kFactorBlockRows owns a row.
 template <int RP, int NT, bool COH>
-__device__ __forceinline__ void p_apply_body(const Tables& t, const FactorBlock fb, int tid, void* smem) {
+__device__ __forceinline__ void p_apply_body(const Tables& t, const FactorBlock fb, int tid, void* smem,
+                                             const LayerDev* staged = nullptr) {
   static_assert(NT >= kFactorBlockRows, "one thread per row of the block");
   auto& S = *static_cast<ApplySmem<RP, NT>*>(smem);
-  const LayerDev& L = t.layers[fb.layer];
+  const LayerDev& L = staged ? *staged : t.layers[fb.layer];   // staged: the wrapper's copy of the entry
   const int n = L.n;
   if constexpr (RP >= kCholSplitRP) {
     // the factor was computed once for this (layer, worker) by p_chol_body: fetch it
@@ -425,11 +428,12 @@ template <int RP> struct OrthSmallSmem {
 };
 
 template <int RP, bool COH>
-__device__ __forceinline__ void p_orth_small_body(const Tables& t, const FactorBlock fb, int tid, void* smem) {
+__device__ __forceinline__ void p_orth_small_body(const Tables& t, const FactorBlock fb, int tid, void* smem,
+                                                  const LayerDev* staged = nullptr) {
   using SM = OrthSmallSmem<RP>;
   constexpr int NE = SM::NE, NSEG = SM::NSEG, SEGROWS = kOrthSmallRows / NSEG;
   auto& S = *static_cast<SM*>(smem);
-  const LayerDev& L = t.layers[fb.layer];
+  const LayerDev& L = staged ? *staged : t.layers[fb.layer];   // staged: the wrapper's copy of the entry
   const int n = L.n, row = tid;
   float p[RP];
 #pragma unroll
@@ -515,11 +519,12 @@ template <int RP, int NT> struct QReduceSmem {
 };
 
 template <int RP, int NT, bool COH>
-__device__ __forceinline__ void q_reduce_body(const Tables& t, const FactorBlock fb, int tid, void* smem) {
+__device__ __forceinline__ void q_reduce_body(const Tables& t, const FactorBlock fb, int tid, void* smem,
+                                              const LayerDev* staged = nullptr) {
   constexpr int V = RP < 4 ? RP : 4;        // floats per thread item
   constexpr int TPR = RP / V;               // items per row: 1, 2, 4 or 8 (divides the block size and 32)
   auto& S = *static_cast<QReduceSmem<RP, NT>*>(smem);
-  const LayerDev& L = t.layers[fb.layer];
+  const LayerDev& L = staged ? *staged : t.layers[fb.layer];   // staged: the wrapper's copy of the entry
   const int m = L.m, nrb = L.nqs;
   const size_t plane = (size_t)m * RP;      // floats of one partial
   float cmax[V];
@@ -685,7 +690,8 @@ template <int RP, int NT> struct ExchangeSmem {
 // size of its code is a large part of its cost.
 template <int RP, int B, int NT, bool COH, bool PLAIN = false>
 __device__ __forceinline__ void exchange_body(const Tables& t, const QuantTables& qt_in, int which, const ExchangeChunk ch,
-                                              const SplitExchange& sx_in, int tid, void* smem) {
+                                              const SplitExchange& sx_in, int tid, void* smem,
+                                              const LayerDev* staged = nullptr) {
   struct QtView { const float* thr; const float* deq; int32_t bits; int32_t avg_values; };
   struct SxView { int32_t pack_only, n_mat, ns; const float* scales; uint8_t* send[2]; uint64_t region_bytes[2], region_off[2]; };
   const QtView qt{qt_in.thr, qt_in.deq, qt_in.bits, PLAIN ? 0 : qt_in.avg_values};
@@ -697,7 +703,7 @@ __device__ __forceinline__ void exchange_body(const Tables& t, const QuantTables
   const int NLEV = (bits == 32) ? 2 : 1 << (bits - 1);
   static_assert(NT >= CH && NT % 32 == 0 && (NT % RP == 0), "block shape");
   auto& S = *static_cast<ExchangeSmem<RP, NT>*>(smem);
-  const LayerDev& L = t.layers[ch.layer];
+  const LayerDev& L = staged ? *staged : t.layers[ch.layer];
   const int W = t.W;
   const int rows = which ? L.m : L.n, r = L.r;
   const int count = rows * r;

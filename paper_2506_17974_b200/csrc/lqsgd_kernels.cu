@@ -470,28 +470,49 @@ pass3_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
 // The small steps between the passes: one CTA per table entry, bodies in lqsgd_factor.cuh
 // (Orthonormalize as CholeskyQR, the factor exchange, the Q_w reduction, the 1-D tensors).
 // ---------------------------------------------------------------------------------------
+// The work tables (factor blocks, exchange chunks, the layer entries) are written at create and never change: a small
+// kernel fetches its entry and its layer's entry into shared memory BEFORE it waits for the kernel in front of it, so
+// that these two dependent memory latencies pass under that kernel's tail instead of heading the step's own chain.
+__device__ __forceinline__ const LayerDev* stage_layer(const Tables& t, int layer, LayerDev* sL) {
+  static_assert(sizeof(LayerDev) % 4 == 0, "copied word by word");
+  const uint32_t* src = reinterpret_cast<const uint32_t*>(t.layers + layer);
+  uint32_t* dst = reinterpret_cast<uint32_t*>(sL);
+  for (int i = threadIdx.x; i < (int)(sizeof(LayerDev) / 4); i += blockDim.x) dst[i] = __ldg(src + i);
+  __syncthreads();
+  return sL;
+}
+
 template <int RP>
 __global__ void __launch_bounds__(256)
 p_reduce_gram_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
+  __shared__ LayerDev sL;
+  const FactorBlock fb = fbs[blockIdx.x];
+  const LayerDev* L = stage_layer(t, fb.layer, &sL);
   pdl_wait();
   __shared__ __align__(16) unsigned char smem[sizeof(ReduceGramSmem<RP>)];
-  p_reduce_gram_body<RP, 256, false>(t, fbs[blockIdx.x], threadIdx.x, smem);
+  p_reduce_gram_body<RP, 256, false>(t, fb, threadIdx.x, smem, L);
 }
 
 template <int RP>
 __global__ void __launch_bounds__(kFactorBlockRows)
 p_apply_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
+  __shared__ LayerDev sL;
+  const FactorBlock fb = fbs[blockIdx.x];
+  const LayerDev* L = stage_layer(t, fb.layer, &sL);
   pdl_wait();
   __shared__ __align__(16) unsigned char smem[sizeof(ApplySmem<RP, kFactorBlockRows>)];
-  p_apply_body<RP, kFactorBlockRows, false>(t, fbs[blockIdx.x], threadIdx.x, smem);
+  p_apply_body<RP, kFactorBlockRows, false>(t, fb, threadIdx.x, smem, L);
 }
 
 template <int RP>
 __global__ void __launch_bounds__(256)
 p_chol_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
+  __shared__ LayerDev sL;
+  const FactorBlock fb = fbs[blockIdx.x];
+  const LayerDev* L = stage_layer(t, fb.layer, &sL);
   pdl_wait();
   __shared__ __align__(16) unsigned char smem[sizeof(CholOnceSmem<RP, 256>)];
-  p_chol_body<RP, 256, false>(t, fbs[blockIdx.x], threadIdx.x, smem);
+  p_chol_body<RP, 256, false>(t, fb, threadIdx.x, smem, L);
 }
 
 // Many partial sums per layer (a very tall or very wide layer): the sums of groups of kFoldGroup consecutive
@@ -527,19 +548,25 @@ fold_kernel(const FoldJob* __restrict__ jobs) {
 template <int RP>
 __global__ void __launch_bounds__(kOrthSmallRows, 3)   // three CTAs per SM: 444 at once, one wave for 21 layers x 16 workers
 p_orth_small_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
+  __shared__ LayerDev sL;
+  const FactorBlock fb = fbs[blockIdx.x];
+  const LayerDev* L = stage_layer(t, fb.layer, &sL);
   pdl_wait();
   __shared__ __align__(16) unsigned char smem[sizeof(OrthSmallSmem<RP>)];
-  p_orth_small_body<RP, false>(t, fbs[blockIdx.x], threadIdx.x, smem);
+  p_orth_small_body<RP, false>(t, fb, threadIdx.x, smem, L);
 }
 
 template <int RP> struct QReduceThreads { static constexpr int value = RP >= 8 ? 256 : 128; };   // one item per thread up to rank 8
 template <int RP>
 __global__ void __launch_bounds__(QReduceThreads<RP>::value)
 q_reduce_kernel(Tables t, const FactorBlock* __restrict__ fbs) {
+  __shared__ LayerDev sL;
+  const FactorBlock fb = fbs[blockIdx.x];
+  const LayerDev* L = stage_layer(t, fb.layer, &sL);
   pdl_wait();
   constexpr int NT = QReduceThreads<RP>::value;
   __shared__ __align__(16) unsigned char smem[sizeof(QReduceSmem<RP, NT>)];
-  q_reduce_body<RP, NT, false>(t, fbs[blockIdx.x], threadIdx.x, smem);
+  q_reduce_body<RP, NT, false>(t, fb, threadIdx.x, smem, L);
 }
 
 __global__ void __launch_bounds__(256)
@@ -554,13 +581,17 @@ template <int RP, int B, bool PLAIN>
 __global__ void __launch_bounds__(256)
 exchange_kernel(Tables t, QuantTables qt, int which, const ExchangeChunk* __restrict__ chunks, int nchunks,
                 SplitExchange sx, VectorJob vj) {
-  pdl_wait();
   if ((int)blockIdx.x >= nchunks) {
+    pdl_wait();
     vectors_block(vj, (int)blockIdx.x - nchunks, threadIdx.x, t.payload, t.payload_stride, t.W);
     return;
   }
+  __shared__ LayerDev sL;
+  const ExchangeChunk ch = chunks[blockIdx.x];
+  const LayerDev* L = stage_layer(t, ch.layer, &sL);
+  pdl_wait();
   __shared__ __align__(16) unsigned char smem[sizeof(ExchangeSmem<RP, 256>)];
-  exchange_body<RP, B, 256, false, PLAIN>(t, qt, which, chunks[blockIdx.x], sx, threadIdx.x, smem);
+  exchange_body<RP, B, 256, false, PLAIN>(t, qt, which, ch, sx, threadIdx.x, smem, L);
 }
 
 // One worker's unpacked codes (one per byte) from its packed stream: what lqsgd_get_state returns
