@@ -141,6 +141,19 @@ __device__ __forceinline__ void pdl_wait() {
   asm volatile("griddepcontrol.wait;" ::: "memory");
 #endif
 }
+// Called before pdl_wait() by the pass kernels: the CTA's first tile and that tile's layer entry (tables written at
+// create, never changed) are asked for while the kernel in front is still finishing, the entry into L2 only, so that
+// the loads after the wait find them close by.
+__device__ __forceinline__ void prefetch_first_tile(const Tables& t, const Tile* tiles, int ntiles) {
+#if defined(__CUDA_ARCH__)
+  if (threadIdx.x == 0 && (int)blockIdx.x < ntiles) {
+    const int layer = __ldg(&tiles[blockIdx.x].layer);
+    const char* e = reinterpret_cast<const char*>(t.layers + layer);
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(e));
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(e + sizeof(LayerDev) - 1));
+  }
+#endif
+}
 // The status words of a round start at zero.  The first pass-1 kernel of the round clears them itself (CTA 0, right
 // after its wait on the previous kernel), which saves a memset node between two rounds and lets this kernel's launch
 // overlap the previous round's tail.  Nothing can set a bit before the clear: the only bits a pass-1 kernel sets are

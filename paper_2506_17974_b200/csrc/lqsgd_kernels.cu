@@ -362,6 +362,7 @@ __device__ __forceinline__ void pass2_tile(const Tables& t, const Tile& tl, floa
 template <int RP>
 __global__ void __launch_bounds__(kPassThreads, (RP <= 2 ? 4 : (RP <= 8 ? 3 : 1)))
 pass2_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
+  prefetch_first_tile(t, tiles, ntiles);
   pdl_wait();
   __shared__ float red[128 * (RP > 16 ? 1 : 4) * RP];
   __shared__ __align__(16) float pb[(RP >= 2 && RP <= 8) ? (RP <= 4 ? 128 : 32 * RP) * RP : 4];   // a tile's rows of P_bar: up to max(128, 32 RP)

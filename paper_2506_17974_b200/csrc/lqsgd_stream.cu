@@ -175,6 +175,7 @@ __device__ __forceinline__ bool pass1_consume(const Tables& t, const TileCtx& c,
 template <int RP, int NST>
 __global__ void __launch_bounds__(kThreads, 1)
 stream_pass1_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
+  prefetch_first_tile(t, tiles, ntiles);
   pdl_wait();
   clear_status_words(t);
   extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -367,6 +368,7 @@ __device__ __forceinline__ bool pass3_consume(const Tables& t, const TileCtx& c,
 template <int RP, int NST>
 __global__ void __launch_bounds__(kThreads, 1)
 stream_pass3_kernel(Tables t, const Tile* __restrict__ tiles, int ntiles) {
+  prefetch_first_tile(t, tiles, ntiles);
   pdl_wait();
   extern __shared__ __align__(128) unsigned char smem_raw[];
   float* sM = reinterpret_cast<float*>(smem_raw);
