@@ -451,9 +451,38 @@ def run_ours(args):
                     c = comp.get_state(which, l, w).cpu().numpy()
                     differ += int((c != out[l][key]["codes"][w]).sum())
                     total += c.size
+        # The same round stage by stage: every stage of the device against the oracle's stage ON THE DEVICE'S OWN INPUT
+        # to that stage (how the tolerances are stated: <= 1e-4 relative Frobenius error per stage, codes equal), so
+        # that one code next to a threshold does not carry over into everything computed after it.
+        def rel(a, b):
+            nb = float(np.linalg.norm(b))
+            return float(np.linalg.norm(np.asarray(a, dtype=np.float64) - b)) / nb if nb > 0 else 0.0
+        hostf = lambda which, l, w=0: comp.get_state(which, l, w).cpu().numpy()
+        stage = {"P_raw": 0.0, "P": 0.0, "Q_w": 0.0, "G_hat": 0.0, "E": 0.0}
+        sdiffer = 0
+        for l in mats:
+            n, m = wl_obj.layers[l]
+            sc = hostf(B.STATE_SCALES, l)
+            P_bar, Q_bar = hostf(B.STATE_P_BAR, l), hostf(B.STATE_Q, l)
+            G_hat = orc.reconstruct(P_bar, Q_bar)
+            stage["G_hat"] = max(stage["G_hat"], rel(ghat[l].cpu().numpy(), G_hat))
+            for w in range(wl_obj.workers):
+                M = orc.error_feedback(g[w][l].cpu().numpy().reshape(n, m), np.zeros((n, m)))     # E_0 = 0
+                P_raw, P, Qw = hostf(B.STATE_P_RAW, l, w), hostf(B.STATE_P, l, w), hostf(B.STATE_Q_W, l, w)
+                stage["P_raw"] = max(stage["P_raw"], rel(P_raw, orc.power_step_p(M, Q0[l])))
+                stage["P"] = max(stage["P"], rel(P, orc.orthonormalize(P_raw)[0]))
+                stage["Q_w"] = max(stage["Q_w"], rel(Qw, orc.power_step_q(M, P_bar)))
+                stage["E"] = max(stage["E"], rel(hostf(B.STATE_E, l, w), orc.error_update(M, G_hat)))
+                sdiffer += int((hostf(B.STATE_CODES_P, l, w) != orc.log_quantize(P, np.float32(sc[0]), wl_obj.bits, wl_obj.alpha)).sum())
+                sdiffer += int((hostf(B.STATE_CODES_Q, l, w) != orc.log_quantize(Qw, np.float32(sc[1]), wl_obj.bits, wl_obj.alpha)).sum())
+        near = sum(comp.step_stats(l)["near_p"] + comp.step_stats(l)["near_q"] for l in mats)
         del comp
         return {"ghat_vs_oracle_rel": (num / den) ** 0.5 if den > 0 else 0.0, "codes_differing": differ,
-                "codes": total, "oracle_s": secs}
+                "codes": total, "oracle_s": secs,
+                "stage_by_stage": dict(stage, codes_differing=sdiffer, codes_within_one_ulp_of_a_threshold=near,
+                                       what="max over layers and workers of the relative Frobenius error of each stage "
+                                            "against the oracle's stage on the device's own input; codes from the "
+                                            "device's own factors")}
 
     wl_obj, desc = get_workload(args.workload)
     if args.workers:
