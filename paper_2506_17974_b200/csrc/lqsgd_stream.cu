@@ -470,7 +470,7 @@ cudaError_t launch_staged(K kernel, size_t smem, const Tables& t, const Tile* ti
     default: return cudaErrorInvalidValue;                  \
   }
 
-constexpr int kNst1 = 3, kNst3 = 5;
+constexpr int kNst1 = 3, kNst3 = 4;   // pass 3: a ring of 4 slabs; with 5 the loads ran further ahead than the memory likes on matrices of a gigabyte
 
 cudaError_t launch_stream_pass1(int rp, const Tables& t, const Tile* tiles, int ntiles, Launch l) {
   if (ntiles == 0) return cudaSuccess;
