@@ -69,7 +69,11 @@ __device__ __forceinline__ void store_contig(float* p, const float (&v)[N]) {
 // ---------------------------------------------------------------------------------------
 constexpr double kPivotEps = 1e-10;
 
-template <int RP> struct ReduceGramSmem { alignas(16) float rows[kFactorBlockRows][RP]; };   // the block's rows (fp32: they are fp32 data)
+template <int RP> struct ReduceGramSmem {
+  static constexpr int NSEG = RP <= 4 ? 8 : (RP == 8 ? 4 : 1);   // up to rank 8 an entry is summed in NSEG segments of the block's rows
+  alignas(16) float rows[kFactorBlockRows][RP];                  // the block's rows (fp32: they are fp32 data)
+  double seg[RP <= 8 ? NSEG : 1][RP <= 8 ? RP * RP : 1];
+};
 
 template <int RP, int NT, bool COH>
 __device__ __forceinline__ void p_reduce_gram_body(const Tables& t, const FactorBlock fb, int tid, void* smem,
@@ -139,6 +143,31 @@ __device__ __forceinline__ void p_reduce_gram_body(const Tables& t, const Factor
           gp[(4 * ti + a) * RP + 4 * tj + b] = acc[a][b];
           gp[(4 * tj + b) * RP + 4 * ti + a] = acc[a][b];
         }
+    }
+  } else if constexpr (RP <= 8) {
+    // few entries (at most 36 of the upper triangle): one thread per entry would leave the CTA idle behind a chain of
+    // 128 dependent fp64 multiply-adds.  Every entry is summed over NSEG segments of the rows by NSEG threads, and the
+    // segments' sums are added in segment order (the same split whatever the block size: the same bits on every path).
+    constexpr int NE = RP * RP, NSEG = ReduceGramSmem<RP>::NSEG, SEG = kFactorBlockRows / NSEG;
+    static_assert(NT >= NSEG * NE && kFactorBlockRows % NSEG == 0, "one thread per entry and segment");
+    if (tid < NSEG * NE) {
+      const int e = tid % NE, g = tid / NE, i = e / RP, j = e % RP;
+      if (j >= i) {                                        // the Gram matrix is symmetric: upper triangle, mirrored
+        double s = 0.0;
+        for (int k = g * SEG; k < (g + 1) * SEG; ++k) s = fma((double)S.rows[k][i], (double)S.rows[k][j], s);
+        S.seg[g][e] = s;
+      }
+    }
+    __syncthreads();
+    if (tid < NE) {
+      const int i = tid / RP, j = tid % RP;
+      if (j >= i) {
+        double s = S.seg[0][tid];
+#pragma unroll
+        for (int g = 1; g < NSEG; ++g) s += S.seg[g][tid];
+        gp[i * RP + j] = s;
+        gp[j * RP + i] = s;
+      }
     }
   } else {
     for (int e = tid; e < RP * RP; e += NT) {
