@@ -70,7 +70,7 @@ def level_values(bits, alpha):
 
 
 # ----------------------------------------------------------------------------
-# LogQuantize / LogDequantize (Alg. 1, quantise and dequantise lines; Section IV-A)
+# LogQuantize / LogDequantize (the quantise and dequantise steps of Alg. 1; Section IV-A)
 # ----------------------------------------------------------------------------
 def factor_scale(factors, per_column=False):
     """s = max over workers and entries of |x| (fp32 values, exact).  per_column (a variant):
@@ -199,7 +199,7 @@ def unpack_codes(stream, count, bits):
 
 
 # ----------------------------------------------------------------------------
-# Orthonormalize (Alg. 1, orthonormalisation line)
+# Orthonormalize (the orthonormalisation step of Alg. 1)
 # ----------------------------------------------------------------------------
 def orthonormalize(P):
     """Modified Gram-Schmidt, columns left to right.  Returns (P_orth, dependent_mask)."""
@@ -243,7 +243,7 @@ def pivot_ratio(P):
 # One factor exchange: scale, quantise, All-Reduce, dequantise
 # ----------------------------------------------------------------------------
 def exchange_factor(factors, bits, alpha, forced_codes=None, average="codes", column_scales=False):
-    """Quantise every worker's factor, average, dequantise (Alg. 1, the three lines
+    """Quantise every worker's factor, average, dequantise (Alg. 1, the three steps
     after each product).  bits == 32 bypasses the quantiser (plain PowerSGD mean).
 
     forced_codes: optional list (per worker) of int16 arrays; entries >= 0 replace

@@ -1,6 +1,6 @@
 // Per-layer figures of the last round, computed on request (lqsgd_step_stats): how many factor
 // entries sat within one fp32 step of a decision threshold of the quantiser (Eq. 4), and how well
-// conditioned the factor handed to Orthonormalize was (Alg. 1, the Orthonormalize line).  Off the
+// conditioned the factor handed to Orthonormalize was (the Orthonormalize step of Algorithm 1).  Off the
 // round's path: the kernel reads what the round left in the workspace (the orthonormal P, M Q
 // before Orthonormalize, M^T P_bar, the scales) and writes three words per layer.
 //
