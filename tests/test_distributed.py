@@ -94,6 +94,8 @@ def test_one_rank_nccl_round_equals_the_fused_step(overlapped):
     if not dist.is_initialized():
         dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{29400 + os.getpid() % 500}", rank=0, world_size=1,
                                 device_id=torch.device(DEV))
+        import atexit
+        atexit.register(lambda: dist.is_initialized() and dist.destroy_process_group())   # shared by both cases of this test
     w = wl.Workload("nccl1", ((96, 200), (64, 27), (130, 36), (20, 1), (256, 1152), (1, 77)), rank=4, bits=4, workers=3,
                     steps=3, dist="student_t3", scale="fan_in", seed=8)
     ref = B.LQSGD(w.layers, w.rank, w.bits, workers=3, seed=8)
